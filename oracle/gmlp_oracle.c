@@ -1,0 +1,202 @@
+/*
+ * CPU oracle for the Gated MLP   Y = (SiLU(X * W_gate) (.) (X * W_up)) * W_down
+ * with an optional RMSNorm prologue on X.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the plain, slow, fp64 statement of what the
+ * operator computes.  It is used by the tests, by the smoke check and by the benchmark's
+ * CPU-baseline leg; the product (the CUDA library) never links, imports or calls it, and
+ * it shares no code, header, table or helper with the CUDA path.
+ *
+ * What it follows (paper of the Axon superoptimizer):
+ *   - the Gated-MLP dataflow graph, figure "mlp-example" (a): matmul(X,W1) -> silu ->
+ *     multiply <- matmul(X,W2); matmul(multiply, W3) -> Z.  W1 = gate, W2 = up, W3 = down.
+ *   - the granular-operation table of Section 5: matmul(x,y) = sum_k mul(x[i,k], y[k,j]);
+ *     silu(x) = mul(x, sigmoid(x)).
+ *   - RMSNorm, Eq. (1) of Section 2: X (.) 1/sqrt(mean_i(X_i^2) + eps) along the last
+ *     dimension, computed in the graph order square -> mean -> add eps -> rsqrt -> multiply.
+ *
+ * Readings taken where the paper is silent (the paper is FP32 and proves equivalence over
+ * the reals; it fixes no reduced-precision behaviour):
+ *   - storage is bf16; every input is widened exactly to fp64 and all arithmetic is fp64;
+ *   - the gated product H = silu(G) * U is rounded ONCE to bf16 (round-to-nearest-even),
+ *     because that is the one place the GPU data path stores an intermediate (rounding R1);
+ *   - with RMSNorm, Xn = x * r * gamma is rounded ONCE to bf16 (rounding R0); gamma is an
+ *     optional per-column gain (an extension; gamma == NULL means ones = the paper's form);
+ *   - Y is left in fp64 (the reference value the tolerance is taken around);
+ *   - every sum runs over its index in ascending order.
+ *
+ * Pins (tests/test_oracle_*.py): rounding helper against an integer-arithmetic
+ * restatement and a library conversion; SiLU identities; RMSNorm unit-RMS / scale
+ * invariance; zero-gate, zero-up, zero-down; one-hot closed forms; integer-exact inputs;
+ * naive triple-loop matmul from a separate translation unit; torch fp64 cross-check.
+ * Not pinned ("parity unpinned"): behaviour on NaN/Inf inputs.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* bf16 bits -> double, exact: a bf16 is the upper half of an IEEE binary32. */
+double gmlp_oracle_bf16_to_double(uint16_t b)
+{
+    uint32_t w = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &w, sizeof f);
+    return (double)f;
+}
+
+/*
+ * double -> bf16 bits, round-to-nearest-even, in ONE rounding (not via binary32).
+ * bf16 has 8 significant bits and binary32's exponent range; the spacing of bf16 values
+ * around |v| = m * 2^e (m in [0.5,1)) is 2^(e-8), and never finer than 2^-133 (subnormals).
+ */
+uint16_t gmlp_oracle_bf16_rn(double v)
+{
+    uint32_t sign = signbit(v) ? 0x8000u : 0u;
+    if (isnan(v)) return (uint16_t)(sign | 0x7FC0u);
+    if (isinf(v)) return (uint16_t)(sign | 0x7F80u);
+    double a = fabs(v);
+    if (a == 0.0) return (uint16_t)sign;
+    int e;
+    (void)frexp(a, &e);
+    int q = e - 8;
+    if (q < -133) q = -133;
+    double r = ldexp(rint(ldexp(a, -q)), q);      /* rint: ties-to-even in the default mode */
+    if (r >= ldexp(1.0, 128)) return (uint16_t)(sign | 0x7F80u);
+    float f = (float)r;                            /* exact: r is a bf16 value */
+    uint32_t w;
+    memcpy(&w, &f, sizeof w);
+    return (uint16_t)(sign | (w >> 16));
+}
+
+/* silu(g) = g * sigmoid(g), written g / (1 + exp(-g)) so that g -> -inf gives -0, not NaN. */
+double gmlp_oracle_silu(double g)
+{
+    return g / (1.0 + exp(-g));
+}
+
+/*
+ * RMSNorm of one row (Eq. 1; graph order square, mean, add eps, rsqrt, multiply):
+ *   ms = (1/d) sum_k x[k]^2 ;  r = 1/sqrt(ms + eps) ;  xn[k] = bf16_rn(x[k] * r * gamma[k]).
+ * Also returns r through *r_out when non-NULL.
+ */
+void gmlp_oracle_rmsnorm_row(const uint16_t* x, const uint16_t* gamma, float eps,
+                             int64_t d_model, uint16_t* xn_out, double* r_out)
+{
+    double ss = 0.0;
+    for (int64_t k = 0; k < d_model; ++k) {
+        double v = gmlp_oracle_bf16_to_double(x[k]);
+        ss += v * v;
+    }
+    double ms = ss / (double)d_model;
+    double r = 1.0 / sqrt(ms + (double)eps);
+    for (int64_t k = 0; k < d_model; ++k) {
+        double v = gmlp_oracle_bf16_to_double(x[k]) * r;
+        if (gamma) v *= gmlp_oracle_bf16_to_double(gamma[k]);
+        xn_out[k] = gmlp_oracle_bf16_rn(v);
+    }
+    if (r_out) *r_out = r;
+}
+
+/*
+ * The operator on a list of rows.  All matrices are dense row-major bf16 bit patterns:
+ *   X [M, d_model], Wg/Wu [d_model, d_ff], Wd [d_ff, d_model], gamma [d_model] or NULL.
+ * rows[0..n_rows) selects the rows of X to compute (rows are independent of each other).
+ * Outputs: Y_ref [n_rows, d_model] fp64 (not rounded); H_bits [n_rows, d_ff] bf16 bits
+ * (may be NULL); Xn_bits [n_rows, d_model] (may be NULL; the row as fed to the matmuls).
+ * Returns 0, or -1 on a bad argument / allocation failure.
+ */
+int gmlp_oracle_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu, const uint16_t* Wd,
+                     const uint16_t* gamma, float eps, int rmsnorm,
+                     int64_t M, int64_t d_model, int64_t d_ff,
+                     const int64_t* rows, int64_t n_rows,
+                     double* Y_ref, uint16_t* H_bits, uint16_t* Xn_bits, int num_threads)
+{
+    if (!X || !Wg || !Wu || !Wd || !rows || !Y_ref || M < 0 || d_model <= 0 || d_ff <= 0 || n_rows < 0)
+        return -1;
+    for (int64_t i = 0; i < n_rows; ++i)
+        if (rows[i] < 0 || rows[i] >= M) return -1;
+    int failed = 0;
+#ifdef _OPENMP
+    if (num_threads > 0) omp_set_num_threads(num_threads);
+#else
+    (void)num_threads;
+#endif
+#pragma omp parallel
+    {
+        double* xn = (double*)malloc(sizeof(double) * (size_t)d_model);
+        uint16_t* xnb = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)d_model);
+        double* g = (double*)malloc(sizeof(double) * (size_t)d_ff);
+        double* u = (double*)malloc(sizeof(double) * (size_t)d_ff);
+        double* h = (double*)malloc(sizeof(double) * (size_t)d_ff);
+        if (!xn || !xnb || !g || !u || !h) {
+#pragma omp atomic write
+            failed = 1;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int64_t i = 0; i < n_rows; ++i) {
+                const uint16_t* x = X + rows[i] * d_model;
+                /* a0: optional RMSNorm prologue, rounding R0 */
+                if (rmsnorm) {
+                    gmlp_oracle_rmsnorm_row(x, gamma, eps, d_model, xnb, NULL);
+                } else {
+                    memcpy(xnb, x, sizeof(uint16_t) * (size_t)d_model);
+                }
+                for (int64_t k = 0; k < d_model; ++k) xn[k] = gmlp_oracle_bf16_to_double(xnb[k]);
+                if (Xn_bits) memcpy(Xn_bits + i * d_model, xnb, sizeof(uint16_t) * (size_t)d_model);
+                /* a1, a2: G = xn * Wg, U = xn * Wu; each g[n], u[n] sums k = 0, 1, 2, ... */
+                for (int64_t n = 0; n < d_ff; ++n) { g[n] = 0.0; u[n] = 0.0; }
+                for (int64_t k = 0; k < d_model; ++k) {
+                    const double xk = xn[k];
+                    const uint16_t* wg = Wg + k * d_ff;
+                    const uint16_t* wu = Wu + k * d_ff;
+                    for (int64_t n = 0; n < d_ff; ++n) {
+                        g[n] += xk * gmlp_oracle_bf16_to_double(wg[n]);
+                        u[n] += xk * gmlp_oracle_bf16_to_double(wu[n]);
+                    }
+                }
+                /* a3, a4: H = bf16_rn(silu(G) * U), rounding R1 */
+                for (int64_t n = 0; n < d_ff; ++n) {
+                    uint16_t hb = gmlp_oracle_bf16_rn(gmlp_oracle_silu(g[n]) * u[n]);
+                    if (H_bits) H_bits[i * d_ff + n] = hb;
+                    h[n] = gmlp_oracle_bf16_to_double(hb);
+                }
+                /* a5: Y = H * Wd; each y[c] sums n = 0, 1, 2, ... ; not rounded */
+                double* y = Y_ref + i * d_model;
+                for (int64_t c = 0; c < d_model; ++c) y[c] = 0.0;
+                for (int64_t n = 0; n < d_ff; ++n) {
+                    const double hn = h[n];
+                    const uint16_t* wd = Wd + n * d_model;
+                    for (int64_t c = 0; c < d_model; ++c)
+                        y[c] += hn * gmlp_oracle_bf16_to_double(wd[c]);
+                }
+            }
+        }
+        free(xn); free(xnb); free(g); free(u); free(h);
+    }
+    return failed ? -1 : 0;
+}
+
+/* Array forms of the two scalar helpers (plain loops), for the tests. */
+void gmlp_oracle_bf16_rn_array(const double* v, uint16_t* out, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = gmlp_oracle_bf16_rn(v[i]);
+}
+
+void gmlp_oracle_silu_array(const double* v, double* out, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = gmlp_oracle_silu(v[i]);
+}
+
+/* Threads the parallel region above will use (for the benchmark's "cores" field). */
+int gmlp_oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

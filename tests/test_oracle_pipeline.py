@@ -1,0 +1,263 @@
+"""Pins for the oracle's whole pipeline  Y = (silu(X Wg) * (X Wu)) Wd  (figure
+"mlp-example" (a); granular-operation table, Section 5).
+
+Each test fixes the result by something other than the oracle: a closed form, an
+invariant of the mathematics, a textbook triple loop from another translation unit
+composed in numpy, or torch's fp64 routines.  Together they are chosen so that a dropped
+term, a swapped gate/up branch, a transposed operand or a missing rounding fails at
+least one of them.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2606_26344_b200 import inputs as I
+
+
+def _bits(t):
+    return t.to(torch.bfloat16).contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def _rand(M, dm, dff, seed, rmsnorm=False, eps=1e-5):
+    return I.custom_inputs(M, dm, dff, seed, rmsnorm=rmsnorm, eps=eps)
+
+
+def _py_silu(v):
+    return v / (1.0 + math.exp(-v))
+
+
+# ---------------------------------------------------------------- zero operands
+@pytest.mark.parametrize("rmsnorm", [False, True])
+def test_zero_gate_up_or_down_gives_zero(rmsnorm):
+    inp = _rand(5, 64, 96, 11, rmsnorm=rmsnorm)
+    z_ff = np.zeros((64, 96), dtype=np.uint16)
+    z_dm = np.zeros((96, 64), dtype=np.uint16)
+    gam = inp.bits("gamma") if rmsnorm else None
+    kw = dict(gamma=gam, eps=1e-5, rmsnorm=rmsnorm)
+    X, Wg, Wu, Wd = (inp.bits(n) for n in ("X", "Wg", "Wu", "Wd"))
+    assert np.all(oracle.gmlp_rows(X, z_ff, Wu, Wd, **kw) == 0.0)      # silu(0) = 0
+    assert np.all(oracle.gmlp_rows(X, Wg, z_ff, Wd, **kw) == 0.0)
+    assert np.all(oracle.gmlp_rows(X, Wg, Wu, z_dm, **kw) == 0.0)
+    assert np.any(oracle.gmlp_rows(X, Wg, Wu, Wd, **kw) != 0.0)
+
+
+# ---------------------------------------------------------------- one-hot closed forms
+def test_one_hot_rows_give_elementwise_closed_form():
+    # Wg has a single row of ones (k1), Wu a single row of ones (k0), Wd[n, c] = [n == c mod d_ff]
+    # => g[m,n] = x[m,k1], u[m,n] = x[m,k0], Y[m,c] = bf16_rn(silu(x[m,k1]) * x[m,k0]).
+    M, dm, dff, k1, k0 = 6, 40, 24, 3, 17
+    inp = _rand(M, dm, dff, 12)
+    X = inp.bits("X")
+    one = _bits(torch.ones(1))[0]
+    Wg = np.zeros((dm, dff), np.uint16); Wg[k1, :] = one
+    Wu = np.zeros((dm, dff), np.uint16); Wu[k0, :] = one
+    Wd = np.zeros((dff, dm), np.uint16)
+    for c in range(dm):
+        Wd[c % dff, c] = one
+    Y = oracle.gmlp_rows(X, Wg, Wu, Wd)
+    xd = oracle.bf16_to_double(X)
+    for m in range(M):
+        v = _py_silu(xd[m, k1]) * xd[m, k0]
+        want = oracle.bf16_to_double(np.array([_round_bf16_py(v)], dtype=np.uint16))[0]
+        assert np.all(Y[m] == want)
+    # swapping the roles of gate and up must change the answer (the gate is the SiLU'd branch)
+    Y_swapped = oracle.gmlp_rows(X, Wu, Wg, Wd)
+    assert not np.array_equal(Y, Y_swapped)
+
+
+def _round_bf16_py(v):
+    """Nearest-even bf16 of a Python float by exact rational arithmetic (independent of oracle/)."""
+    if v == 0.0:
+        return 0x8000 if math.copysign(1.0, v) < 0 else 0
+    sign = 0x8000 if v < 0 else 0
+    a = abs(v)
+    e = math.floor(math.log2(a))
+    while 2.0 ** e > a:
+        e -= 1
+    while 2.0 ** (e + 1) <= a:
+        e += 1
+    q = max(e - 7, -133)
+    num, den = a.as_integer_ratio()
+    n2, d2 = (num << max(-q, 0)), (den << max(q, 0))
+    j, rem = divmod(n2, d2)
+    if 2 * rem > d2 or (2 * rem == d2 and (j & 1)):
+        j += 1
+    val = np.float32(j * 2.0 ** q)
+    return sign | int(np.array([val]).view(np.uint32)[0] >> 16)
+
+
+def test_per_column_one_hots_cover_every_column():
+    # Wg[n mod dm, n] = 1, Wu[(n+1) mod dm, n] = 1  =>  h[m,n] = bf16_rn(silu(x[m, n mod dm]) * x[m,(n+1) mod dm])
+    M, dm, dff = 3, 16, 50
+    inp = _rand(M, dm, dff, 13)
+    X = inp.bits("X")
+    one = _bits(torch.ones(1))[0]
+    Wg = np.zeros((dm, dff), np.uint16); Wu = np.zeros((dm, dff), np.uint16)
+    for n in range(dff):
+        Wg[n % dm, n] = one
+        Wu[(n + 1) % dm, n] = one
+    Y, H = oracle.gmlp_rows(X, Wg, Wu, inp.bits("Wd"), want_h=True)
+    xd = oracle.bf16_to_double(X)
+    for m in range(M):
+        for n in range(dff):
+            assert H[m, n] == _round_bf16_py(_py_silu(xd[m, n % dm]) * xd[m, (n + 1) % dm])
+    # and Y is H times Wd by the textbook loop
+    want = oracle.naive_matmul(oracle.bf16_to_double(H), oracle.bf16_to_double(inp.bits("Wd")))
+    assert np.array_equal(Y, want)
+
+
+# ---------------------------------------------------------------- textbook loops / library
+@pytest.mark.parametrize("shape", [(1, 8, 8), (4, 24, 40), (16, 64, 96)])
+@pytest.mark.parametrize("rmsnorm", [False, True])
+def test_matches_naive_triple_loops_bit_for_bit(shape, rmsnorm):
+    M, dm, dff = shape
+    inp = _rand(M, dm, dff, 20 + M, rmsnorm=rmsnorm, eps=1e-6)
+    X, Wg, Wu, Wd = (inp.bits(n) for n in ("X", "Wg", "Wu", "Wd"))
+    xd = oracle.bf16_to_double(X)
+    if rmsnorm:
+        gd = oracle.bf16_to_double(inp.bits("gamma"))
+        eps = float(np.float32(1e-6))
+        rows = []
+        for m in range(M):
+            ss = 0.0
+            for k in range(dm):
+                ss += xd[m, k] * xd[m, k]
+            r = 1.0 / math.sqrt(ss / dm + eps)
+            rows.append([_round_bf16_py(xd[m, k] * r * gd[k]) for k in range(dm)])
+        xd = oracle.bf16_to_double(np.array(rows, dtype=np.uint16))
+    G = oracle.naive_matmul(xd, oracle.bf16_to_double(Wg))
+    U = oracle.naive_matmul(xd, oracle.bf16_to_double(Wu))
+    Hb = np.array([[_round_bf16_py(_py_silu(G[m, n]) * U[m, n]) for n in range(dff)] for m in range(M)],
+                  dtype=np.uint16)
+    want = oracle.naive_matmul(oracle.bf16_to_double(Hb), oracle.bf16_to_double(Wd))
+    Y, H = oracle.gmlp_rows(X, Wg, Wu, Wd, gamma=inp.bits("gamma") if rmsnorm else None,
+                            eps=1e-6, rmsnorm=rmsnorm, want_h=True)
+    assert np.array_equal(H, Hb)
+    assert np.array_equal(Y, want)
+
+
+@pytest.mark.parametrize("rmsnorm", [False, True])
+def test_against_torch_fp64(rmsnorm):
+    M, dm, dff = 33, 320, 520
+    inp = _rand(M, dm, dff, 31, rmsnorm=rmsnorm, eps=1e-5)
+    Xd, Wg, Wu, Wd = inp.X.double(), inp.Wg.double(), inp.Wu.double(), inp.Wd.double()
+    if rmsnorm:
+        eps = float(np.float32(1e-5))
+        v = Xd * torch.rsqrt((Xd * Xd).mean(dim=1, keepdim=True) + eps) * inp.gamma.double()
+        Xd = torch.tensor(oracle.bf16_to_double(oracle.bf16_rn(v.numpy())))
+    Hv = torch.nn.functional.silu(Xd @ Wg) * (Xd @ Wu)
+    Hd = torch.tensor(oracle.bf16_to_double(oracle.bf16_rn(Hv.numpy())))
+    want = (Hd @ Wd).numpy()
+    Y, H = oracle.gmlp_rows(inp.bits("X"), inp.bits("Wg"), inp.bits("Wu"), inp.bits("Wd"),
+                            gamma=inp.bits("gamma") if rmsnorm else None, eps=1e-5, rmsnorm=rmsnorm, want_h=True)
+    # torch's BLAS sums in another order: H may differ in the last place on a few near-ties
+    hd = oracle.bf16_to_double(H)
+    flips = np.count_nonzero(hd != Hd.numpy())
+    assert flips <= 3
+    if flips == 0:
+        assert np.allclose(Y, want, rtol=1e-12, atol=1e-12)
+    else:
+        assert np.allclose(Y, want, rtol=0, atol=2e-2)
+
+
+def test_integer_valued_inputs_are_exact():
+    # small integers: every product and partial sum is an exact integer in fp64, so the
+    # pre-activation G, U can be checked through H in closed form.
+    rng = np.random.default_rng(5)
+    M, dm, dff = 4, 32, 48
+    X = torch.tensor(rng.integers(-4, 5, (M, dm)), dtype=torch.float32)
+    Wg = torch.tensor(rng.integers(-2, 3, (dm, dff)), dtype=torch.float32)
+    Wu = torch.tensor(rng.integers(-2, 3, (dm, dff)), dtype=torch.float32)
+    Wd = torch.tensor(rng.integers(-2, 3, (dff, dm)), dtype=torch.float32)
+    G = (X.long() @ Wg.long()).numpy(); U = (X.long() @ Wu.long()).numpy()
+    Hb = np.array([[_round_bf16_py(_py_silu(float(G[m, n])) * float(U[m, n])) for n in range(dff)]
+                   for m in range(M)], dtype=np.uint16)
+    Y, H = oracle.gmlp_rows(_bits(X), _bits(Wg), _bits(Wu), _bits(Wd), want_h=True)
+    assert np.array_equal(H, Hb)
+    want = oracle.bf16_to_double(Hb) @ Wd.double().numpy()
+    assert np.allclose(Y, want, rtol=1e-14, atol=1e-12)
+
+
+# ---------------------------------------------------------------- invariants
+def test_linearity_in_wd_row_permutation_and_row_independence():
+    inp = _rand(9, 48, 80, 41)
+    X, Wg, Wu, Wd = (inp.bits(n) for n in ("X", "Wg", "Wu", "Wd"))
+    Y = oracle.gmlp_rows(X, Wg, Wu, Wd)
+    Y4 = oracle.gmlp_rows(X, Wg, Wu, _bits(inp.Wd * 4.0))
+    assert np.array_equal(Y4, 4.0 * Y)                         # exact power-of-two scaling
+    perm = np.array([3, 0, 8, 1, 7, 2, 6, 4, 5])
+    assert np.array_equal(oracle.gmlp_rows(X[perm], Wg, Wu, Wd), Y[perm])
+    for m in (0, 4, 8):                                        # a row alone == the row in the batch
+        assert np.array_equal(oracle.gmlp_rows(X[m:m + 1], Wg, Wu, Wd)[0], Y[m])
+    assert np.array_equal(oracle.gmlp_rows(X, Wg, Wu, Wd, rows=np.array([8, 2])), Y[[8, 2]])
+    assert np.array_equal(oracle.gmlp_rows(X, Wg, Wu, Wd, num_threads=1), Y)   # thread count is immaterial
+
+
+def test_gate_is_applied_before_the_product_illegal_swap():
+    # Section 5's rejected rewrite: silu(X) * G != silu(X * G).  With one-hot weights the
+    # oracle must produce the left-hand side.
+    dm, dff = 8, 8
+    x = torch.tensor([[1.5, -2.0, 0.75, 3.0, -0.5, 2.5, -1.25, 0.25]])
+    one = _bits(torch.ones(1))[0]
+    Wg = np.zeros((dm, dff), np.uint16); Wu = np.zeros((dm, dff), np.uint16); Wd = np.zeros((dff, dm), np.uint16)
+    for n in range(dff):
+        Wg[n, n] = one; Wu[(n + 3) % dm, n] = one; Wd[n, n] = one
+    Y = oracle.gmlp_rows(_bits(x), Wg, Wu, Wd)[0]
+    xs = x[0].double().numpy()
+    gaps = []
+    for n in range(dff):
+        a, b = xs[n], xs[(n + 3) % dm]
+        lhs = oracle.bf16_to_double(np.array([_round_bf16_py(_py_silu(a) * b)], dtype=np.uint16))[0]
+        assert Y[n] == lhs
+        gaps.append(abs(Y[n] - _py_silu(a * b)))
+    assert max(gaps) > 0.5 and sum(g > 1e-2 for g in gaps) >= 6
+
+
+def test_row_scale_commutes_with_matmul_legal_swap():
+    # Section 5's accepted rewrite: (X (.) r) W == (X W) (.) r for a per-row scalar r.
+    # In the oracle: with eps = 0 and no rounding loss (power-of-two r), scaling X's rows
+    # leaves the normalised pipeline unchanged, and without the norm a power-of-two row
+    # scale passes through both matmuls only via silu's non-linearity -> checked on G, U.
+    inp = _rand(4, 64, 32, 51, rmsnorm=True, eps=0.0)
+    X, Wg, Wu, Wd, gam = (inp.bits(n) for n in ("X", "Wg", "Wu", "Wd", "gamma"))
+    base = oracle.gmlp_rows(X, Wg, Wu, Wd, gamma=gam, eps=0.0, rmsnorm=True)
+    Xs = inp.X.clone()
+    Xs[0] *= 8.0; Xs[1] *= 0.25; Xs[3] *= 1024.0
+    scaled = oracle.gmlp_rows(_bits(Xs), Wg, Wu, Wd, gamma=gam, eps=0.0, rmsnorm=True)
+    assert np.array_equal(base, scaled)
+    # r past the matmul in fp64 (no rounding point involved)
+    xd = inp.X.double().numpy(); wd_ = inp.Wg.double().numpy()
+    r = 1.0 / np.sqrt(np.mean(xd * xd, axis=1, keepdims=True))
+    lhs = oracle.naive_matmul(xd * r, wd_)
+    rhs = oracle.naive_matmul(xd, wd_) * r
+    assert np.allclose(lhs, rhs, rtol=1e-12, atol=1e-14)
+
+
+def test_h_is_rounded_to_bf16_once():
+    # Y computed from an unrounded H differs; Y computed from H rounded via fp32 first can differ
+    # only on double-rounding ties.  Check the oracle equals "round the fp64 product once".
+    inp = _rand(8, 96, 128, 61)
+    Xd, Wg, Wu, Wd = inp.X.double().numpy(), inp.Wg.double().numpy(), inp.Wu.double().numpy(), inp.Wd.double().numpy()
+    G = oracle.naive_matmul(Xd, Wg); U = oracle.naive_matmul(Xd, Wu)
+    prod = np.vectorize(_py_silu)(G) * U
+    Hb = np.array([[_round_bf16_py(float(v)) for v in row] for row in prod], dtype=np.uint16)
+    Y, H = oracle.gmlp_rows(inp.bits("X"), inp.bits("Wg"), inp.bits("Wu"), inp.bits("Wd"), want_h=True)
+    assert np.array_equal(H, Hb)
+    unrounded = oracle.naive_matmul(prod, Wd)
+    assert not np.array_equal(Y, unrounded)
+    assert np.max(np.abs(Y - unrounded)) < 2e-2
+
+
+def test_bad_arguments_are_rejected():
+    inp = _rand(2, 16, 16, 1)
+    X, Wg, Wu, Wd = (inp.bits(n) for n in ("X", "Wg", "Wu", "Wd"))
+    with pytest.raises(RuntimeError):
+        oracle.gmlp_rows(X, Wg, Wu, Wd, rows=np.array([2]))
+    with pytest.raises(ValueError):
+        oracle.gmlp_rows(X, Wg, Wu, Wd[:8])
+    with pytest.raises(TypeError):
+        oracle.gmlp_rows(X.astype(np.float32), Wg, Wu, Wd)
+    assert oracle.gmlp_rows(X, Wg, Wu, Wd, rows=np.zeros(0, dtype=np.int64)).shape == (0, 16)
