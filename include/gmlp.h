@@ -1,0 +1,158 @@
+/*
+ * libgmlp — the fused Gated MLP for NVIDIA B200 (sm_100a), C ABI.
+ *
+ *     Y = ( SiLU(Xn * W_gate)  (.)  (Xn * W_up) ) * W_down,      Xn = X  or  RMSNorm(X)
+ *
+ * The operator is the five-node dataflow graph of the paper's Gated-MLP example (figure
+ * "mlp-example" (a): matmul, matmul, silu, multiply, matmul; W1 = gate, W2 = up,
+ * W3 = down) with the element-level meanings of its granular-operation table (Section 5:
+ * matmul(x,y) = sum_k x[i,k]*y[k,j]; silu(x) = x*sigmoid(x)).  The optional prologue is
+ * RMSNorm as in Eq. (1) of Section 2, Xn = X (.) 1/sqrt(mean_k(X^2) + eps), followed by an
+ * optional per-column gain (an extension; no gain = the paper's form).
+ *
+ * Data: bf16 in, bf16 out, fp32 accumulation.  The gated product H = silu(G)*U is rounded
+ * once to bf16 (round-to-nearest-even); so is Xn when the prologue is on; so is Y.
+ *
+ * Layout (operand convention of the paper's matmul, a[..., i0, i1] * b[..., i1, i2]):
+ *   X  [M, d_model]      row-major bf16
+ *   Wg [d_model, d_ff]   row-major bf16   ("[in, out]")
+ *   Wu [d_model, d_ff]   row-major bf16
+ *   Wd [d_ff, d_model]   row-major bf16
+ *   Y  [M, d_model]      row-major bf16
+ * All pointers are DEVICE pointers unless a parameter says "host".  Every pointer must be
+ * 16-byte aligned; d_model and d_ff must be positive multiples of 8; M >= 0 (M == 0 is a
+ * successful no-op).  Y must not overlap any input.  Inputs are only read.
+ *
+ * Ownership: the caller owns every buffer.  The library allocates nothing per call when a
+ * workspace is passed; with workspace == NULL it uses a library-owned buffer that grows on
+ * demand (cudaMalloc on the calling thread's current device) and is freed by
+ * gmlp_shutdown().
+ *
+ * Errors: every entry point returns a gmlp_status code; nothing throws, aborts or prints.
+ * Calls are asynchronous on the given stream: device-side problems (a bounded wait that
+ * ran out) surface after the stream is synchronised, through gmlp_device_status(), or at
+ * once with GMLP_FLAG_CHECKED.  On a device that is not sm_100 the calls return
+ * GMLP_ERR_ARCH: there is no fallback of any kind.
+ */
+#ifndef GMLP_H_
+#define GMLP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gmlp_status {
+    GMLP_OK = 0,
+    GMLP_ERR_NULL = -1,       /* a required pointer is NULL */
+    GMLP_ERR_SHAPE = -2,      /* M < 0, or d_model / d_ff not a positive multiple of 8, or too large */
+    GMLP_ERR_ALIGN = -3,      /* a pointer is not 16-byte aligned */
+    GMLP_ERR_FLAGS = -4,      /* unknown flag bit, unknown variant, or bad struct_bytes */
+    GMLP_ERR_WORKSPACE = -5,  /* workspace too small (or could not be grown) */
+    GMLP_ERR_ARCH = -6,       /* no CUDA device, or the current device is not sm_100 */
+    GMLP_ERR_LAUNCH = -7,     /* a CUDA runtime call failed (cudaGetLastError is left readable) */
+    GMLP_ERR_TIMEOUT = -8,    /* a bounded device-side wait ran out (see gmlp_device_status) */
+    GMLP_ERR_UNSUPPORTED = -9 /* the forced variant cannot run this shape */
+} gmlp_status;
+
+enum {
+    GMLP_FLAG_RMSNORM = 1u << 0, /* apply the RMSNorm prologue to X */
+    GMLP_FLAG_CHECKED = 1u << 2  /* synchronise the stream and report the device status before returning */
+};
+
+/* Kernel schedule.  AUTO picks by shape; the others force one schedule (tests, benchmarks). */
+enum {
+    GMLP_VARIANT_AUTO = 0,
+    GMLP_VARIANT_SIMT = 1,   /* CUDA-core tiled GEMMs: any shape, slow; bring-up and cross-check */
+    GMLP_VARIANT_STREAM = 2, /* small M: weight-streaming split-K kernels (HBM-bound regime) */
+    GMLP_VARIANT_UMMA = 3    /* large M: tcgen05 tensor-core GEMMs fed by TMA, accumulators in TMEM */
+};
+
+typedef struct gmlp_args {
+    uint32_t struct_bytes;    /* sizeof(gmlp_args); guards against ABI drift */
+    uint32_t flags;           /* GMLP_FLAG_* */
+    const void* X;            /* device, [M, d_model] bf16 */
+    const void* Wg;           /* device, [d_model, d_ff] bf16 */
+    const void* Wu;           /* device, [d_model, d_ff] bf16 */
+    const void* Wd;           /* device, [d_ff, d_model] bf16 */
+    void* Y;                  /* device, [M, d_model] bf16, written */
+    int64_t M, d_model, d_ff;
+    const void* rms_gain;     /* device, [d_model] bf16, or NULL for no gain; read only with GMLP_FLAG_RMSNORM */
+    float rms_eps;            /* eps of Eq. (1); used only with GMLP_FLAG_RMSNORM */
+    int32_t variant;          /* GMLP_VARIANT_* */
+    void* stream;             /* cudaStream_t; NULL = the legacy default stream */
+    void* workspace;          /* device scratch of >= gmlp_workspace_bytes(...) bytes, 256-byte aligned, or NULL */
+    uint64_t workspace_bytes;
+} gmlp_args;
+
+/*
+ * The operator as the paper states it: Y = (silu(X Wg) (.) (X Wu)) Wd.
+ * Runs on the stream set by gmlp_set_stream (default: legacy default stream) with the
+ * library-owned workspace.  With GMLP_FLAG_RMSNORM the prologue has no gain and uses the eps
+ * set by gmlp_set_default_eps (default 1e-5).  Asynchronous; returns a gmlp_status.
+ */
+int gmlp_forward(const void* X, const void* Wg, const void* Wu, const void* Wd, void* Y,
+                 int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);
+
+/* Same operator with every option explicit (gain, eps, stream, workspace, variant). */
+int gmlp_forward_ex(const gmlp_args* args);
+
+/*
+ * The same call for a caller whose activations live in HOST memory: copies X_host
+ * (M*d_model bf16, ideally pinned) to args->X, runs gmlp_forward_ex, and copies args->Y
+ * to Y_host, all asynchronously on args->stream.  args->X and args->Y are device staging
+ * buffers owned by the caller; weights, gain and workspace are device-resident as usual.
+ * Y_host is valid once the stream has been synchronised.
+ */
+int gmlp_forward_host(const gmlp_args* args, const void* X_host, void* Y_host);
+
+/*
+ * Bytes of scratch gmlp_forward_ex needs for this shape, for the schedule `variant` would
+ * run (AUTO = the one the library would pick): the bf16 intermediate H [M, d_ff], Xn
+ * [M, d_model] when the prologue is on, and split-K partial sums and arrival counters for
+ * the small-M schedule.  Returns 0 for invalid shapes.
+ */
+uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant);
+
+/* The schedule AUTO resolves to for this shape (one of GMLP_VARIANT_SIMT/STREAM/UMMA). */
+int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);
+
+/*
+ * Reads and clears the device status word of the current device (synchronises the device).
+ * 0 = no device-side problem since the last read; otherwise a code naming the wait that ran
+ * out (high 16 bits: kernel id, low 16 bits: site).  Returns GMLP_ERR_* (< 0) on failure.
+ */
+int gmlp_device_status(void);
+
+/* Number of kernels the library launched on this host thread since the last reset. */
+uint64_t gmlp_launch_count(void);
+void gmlp_reset_launch_count(void);
+
+/*
+ * Per-kernel timing for benchmarks (per host thread, off by default).  While enabled, every
+ * gmlp_forward_ex call records a CUDA event on its stream before its first kernel and after
+ * each kernel.  gmlp_profile_read synchronises on the last event of the most recent call and
+ * writes the duration of each of its kernels, in launch order, in milliseconds; *count gets
+ * their number (at most max_count are written).  gmlp_profile_kernel_name(i) names the i-th
+ * kernel of that call ("rmsnorm", "gate_up", "down").  Events add launch overhead: do not
+ * leave this on in a timed region.
+ */
+int gmlp_profile_enable(int on);
+int gmlp_profile_read(float* ms, int max_count, int* count);
+const char* gmlp_profile_kernel_name(int index);
+
+const char* gmlp_status_string(int status);
+int gmlp_version(void);
+
+/* Per-host-thread defaults for the 9-argument call. */
+int gmlp_set_stream(void* cuda_stream);
+int gmlp_set_default_eps(float eps);
+
+/* Frees the library-owned workspace of every device.  Safe to call more than once. */
+void gmlp_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GMLP_H_ */

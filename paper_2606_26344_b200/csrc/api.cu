@@ -1,0 +1,524 @@
+// libgmlp: C-ABI entry points, argument checks, schedule selection, workspace layout and
+// kernel launches.  See include/gmlp.h for the contract of each call.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <mutex>
+#include <new>
+
+#include "../../include/gmlp.h"
+#include "common.cuh"
+#include "rmsnorm.cuh"
+#include "simt_gemm.cuh"
+#include "stream_small_m.cuh"
+#include "umma_gemm.cuh"
+
+namespace {
+
+using gmlp::bf16;
+
+constexpr int kVersion = 100;
+constexpr int kMaxDevices = 64;
+constexpr int64_t kMaxDim = (int64_t)1 << 30;      // per-dimension limit (TMA coordinates are int32)
+constexpr uint32_t kKnownFlags = GMLP_FLAG_RMSNORM | GMLP_FLAG_CHECKED;
+
+thread_local cudaStream_t t_stream = nullptr;
+thread_local float t_default_eps = 1e-5f;
+thread_local uint64_t t_launches = 0;
+
+// Optional per-kernel event timing of the most recent call (benchmarks only).
+constexpr int kMaxProfKernels = 4;
+struct Profile {
+    bool on = false;
+    cudaEvent_t ev[kMaxProfKernels + 1] = {};
+    bool created = false;
+    int n = 0;                                  // kernels recorded by the last call
+    const char* names[kMaxProfKernels] = {};
+};
+thread_local Profile t_prof;
+
+void prof_begin(cudaStream_t st) {
+    if (!t_prof.on) return;
+    if (!t_prof.created) {
+        for (auto& e : t_prof.ev) if (cudaEventCreate(&e) != cudaSuccess) { t_prof.on = false; return; }
+        t_prof.created = true;
+    }
+    t_prof.n = 0;
+    (void)cudaEventRecord(t_prof.ev[0], st);
+}
+void prof_mark(const char* name, cudaStream_t st) {
+    if (!t_prof.on || t_prof.n >= kMaxProfKernels) return;
+    t_prof.names[t_prof.n] = name;
+    ++t_prof.n;
+    (void)cudaEventRecord(t_prof.ev[t_prof.n], st);
+}
+
+struct DeviceState {
+    bool probed = false;
+    bool is_sm100 = false;
+    int sm_count = 0;
+    void* workspace = nullptr;
+    uint64_t workspace_bytes = 0;
+    bool umma_attr_set = false;
+};
+std::mutex g_mutex;
+DeviceState g_dev[kMaxDevices];
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode_tiled = nullptr;
+
+inline uint64_t align256(uint64_t v) { return (v + 255u) & ~(uint64_t)255u; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Returns the state of the current device, probing it on first use; nullptr if there is none.
+DeviceState* current_device(int* status) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        *status = GMLP_ERR_ARCH;
+        return nullptr;
+    }
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState& d = g_dev[dev];
+    if (!d.probed) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            *status = GMLP_ERR_ARCH;
+            return nullptr;
+        }
+        d.is_sm100 = (major == 10);
+        d.sm_count = sms;
+        d.probed = true;
+    }
+    if (!d.is_sm100) {
+        *status = GMLP_ERR_ARCH;
+        return nullptr;
+    }
+    if (g_encode_tiled == nullptr) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess || fn == nullptr) {
+            (void)cudaGetLastError();
+            *status = GMLP_ERR_ARCH;
+            return nullptr;
+        }
+        g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    *status = GMLP_OK;
+    return &d;
+}
+
+// ------------------------------------------------------------------ small-M plan
+struct StreamPlan {
+    int MT, row_tiles, slabs, KS, kchunk;
+};
+
+StreamPlan make_stream_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_count) {
+    StreamPlan p;
+    p.MT = M <= 1 ? 1 : (M <= 2 ? 2 : (M <= 4 ? 4 : 8));
+    p.row_tiles = (int)((M + p.MT - 1) / p.MT);
+    if (p.row_tiles < 1) p.row_tiles = 1;
+    p.slabs = (int)((N + gmlp::kStreamSlab - 1) / gmlp::kStreamSlab);
+    const int64_t resident = (int64_t)(sm_count > 0 ? sm_count : 148) * 4;      // 4 CTAs of 128 threads per SM
+    int64_t ks = resident / ((int64_t)p.slabs * nmat * p.row_tiles);
+    const int64_t ks_min = (K + gmlp::kStreamMaxChunk - 1) / gmlp::kStreamMaxChunk;
+    const int64_t ks_max = (K + 31) / 32;
+    if (ks < ks_min) ks = ks_min;
+    if (ks > ks_max) ks = ks_max;
+    if (ks < 1) ks = 1;
+    int64_t chunk = (K + ks - 1) / ks;
+    chunk = (chunk + gmlp::kStreamWarps - 1) / gmlp::kStreamWarps * gmlp::kStreamWarps;
+    if (chunk > gmlp::kStreamMaxChunk) chunk = gmlp::kStreamMaxChunk;
+    p.kchunk = (int)chunk;
+    p.KS = (int)((K + chunk - 1) / chunk);
+    return p;
+}
+
+// ------------------------------------------------------------------ workspace layout
+struct Layout {
+    uint64_t xn_off, h_off, partial_off, counters_off, total;
+    uint64_t counters_bytes;
+    StreamPlan p1, p2;
+};
+
+int resolve_variant(int64_t M, int32_t variant) {
+    if (variant != GMLP_VARIANT_AUTO) return variant;
+    return M <= 16 ? GMLP_VARIANT_STREAM : GMLP_VARIANT_UMMA;
+}
+
+Layout make_layout(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int variant, int sm_count) {
+    Layout L{};
+    uint64_t off = 0;
+    L.xn_off = off;
+    if (flags & GMLP_FLAG_RMSNORM) off += align256((uint64_t)M * d_model * 2);
+    L.h_off = off;
+    off += align256((uint64_t)M * d_ff * 2);
+    L.partial_off = off;
+    L.counters_off = off;
+    if (variant == GMLP_VARIANT_STREAM) {
+        L.p1 = make_stream_plan(M, d_model, d_ff, 2, sm_count);
+        L.p2 = make_stream_plan(M, d_ff, d_model, 1, sm_count);
+        const uint64_t b1 = (uint64_t)2 * L.p1.KS * M * d_ff * 4;
+        const uint64_t b2 = (uint64_t)L.p2.KS * M * d_model * 4;
+        off += align256(b1 > b2 ? b1 : b2);      // the two phases run one after the other and share it
+        L.counters_off = off;
+        L.counters_bytes = align256((uint64_t)(L.p1.row_tiles * L.p1.slabs + L.p2.row_tiles * L.p2.slabs) * 4);
+        off += L.counters_bytes;
+    }
+    L.total = off;
+    return L;
+}
+
+int check_shape(int64_t M, int64_t d_model, int64_t d_ff) {
+    if (M < 0 || d_model <= 0 || d_ff <= 0 || (d_model & 7) || (d_ff & 7)) return GMLP_ERR_SHAPE;
+    if (M > kMaxDim || d_model > kMaxDim || d_ff > kMaxDim) return GMLP_ERR_SHAPE;
+    return GMLP_OK;
+}
+
+// ------------------------------------------------------------------ TMA descriptors
+// 2-D bf16 tensor, row-major [outer, inner]; box = box_outer rows x box_inner elements, 128-byte swizzle,
+// out-of-bounds elements read as zero.
+bool encode_2d(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_inner, uint32_t box_outer) {
+    const cuuint64_t gdim[2] = {inner, outer};
+    const cuuint64_t gstride[1] = {inner * 2};
+    const cuuint32_t box[2] = {box_inner, box_outer};
+    const cuuint32_t estride[2] = {1, 1};
+    return g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estride,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// ------------------------------------------------------------------ launches
+#define GMLP_CHECK_LAUNCH()                                   \
+    do {                                                      \
+        if (cudaPeekAtLastError() != cudaSuccess) return GMLP_ERR_LAUNCH; \
+        ++t_launches;                                         \
+    } while (0)
+
+int launch_rmsnorm(const bf16* X, const bf16* gain, bf16* Xn, int64_t M, int64_t d_model, float eps, cudaStream_t st) {
+    gmlp::rmsnorm_kernel<<<(unsigned)M, gmlp::kRmsThreads, 0, st>>>(X, gain, Xn, M, (int)d_model, eps);
+    GMLP_CHECK_LAUNCH();
+    return GMLP_OK;
+}
+
+int run_simt(const bf16* A, const bf16* Wg, const bf16* Wu, const bf16* Wd, bf16* H, bf16* Y,
+             int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st) {
+    const int T = gmlp::kSimtTile;
+    dim3 g1((unsigned)((d_ff + T - 1) / T), (unsigned)((M + T - 1) / T));
+    gmlp::simt_gemm_kernel<true><<<g1, 256, 0, st>>>(A, Wg, Wu, H, M, (int)d_model, (int)d_ff);
+    GMLP_CHECK_LAUNCH();
+    prof_mark("gate_up", st);
+    dim3 g2((unsigned)((d_model + T - 1) / T), (unsigned)((M + T - 1) / T));
+    gmlp::simt_gemm_kernel<false><<<g2, 256, 0, st>>>(H, Wd, nullptr, Y, M, (int)d_ff, (int)d_model);
+    GMLP_CHECK_LAUNCH();
+    prof_mark("down", st);
+    return GMLP_OK;
+}
+
+template <bool GATEUP>
+int launch_stream(const StreamPlan& p, const bf16* A, const bf16* W0, const bf16* W1, float* partial,
+                  unsigned int* counters, bf16* out, int64_t M, int64_t K, int64_t N, cudaStream_t st) {
+    dim3 grid((unsigned)p.slabs, (unsigned)(p.KS * (GATEUP ? 2 : 1)), (unsigned)p.row_tiles);
+    const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
+    switch (p.MT) {
+        case 1: gmlp::stream_gemm_kernel<1, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS); break;
+        case 2: gmlp::stream_gemm_kernel<2, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS); break;
+        case 4: gmlp::stream_gemm_kernel<4, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS); break;
+        default: gmlp::stream_gemm_kernel<8, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS); break;
+    }
+    GMLP_CHECK_LAUNCH();
+    return GMLP_OK;
+}
+
+int run_stream(const Layout& L, uint8_t* ws, const bf16* A, const bf16* Wg, const bf16* Wu, const bf16* Wd, bf16* H,
+               bf16* Y, int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st) {
+    float* partial = reinterpret_cast<float*>(ws + L.partial_off);
+    unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
+    unsigned int* c2 = c1 + L.p1.row_tiles * L.p1.slabs;
+    if (cudaMemsetAsync(c1, 0, L.counters_bytes, st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    int rc = launch_stream<true>(L.p1, A, Wg, Wu, partial, c1, H, M, d_model, d_ff, st);
+    if (rc != GMLP_OK) return rc;
+    prof_mark("gate_up", st);
+    rc = launch_stream<false>(L.p2, H, Wd, nullptr, partial, c2, Y, M, d_ff, d_model, st);
+    if (rc == GMLP_OK) prof_mark("down", st);
+    return rc;
+}
+
+template <bool GATEUP>
+int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
+                int64_t M, int64_t K, int64_t N, cudaStream_t st) {
+    CUtensorMap tmA, tmB0, tmB1;
+    if (!encode_2d(&tmA, A, (uint64_t)K, (uint64_t)M, gmlp::kUmmaBK, gmlp::kUmmaBM)) return GMLP_ERR_LAUNCH;
+    if (!encode_2d(&tmB0, W0, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
+    if (GATEUP) {
+        if (!encode_2d(&tmB1, W1, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
+    } else {
+        tmB1 = tmB0;
+    }
+    if (!dev->umma_attr_set) {
+        if (cudaFuncSetAttribute(gmlp::umma_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)gmlp::kUmmaSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::umma_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)gmlp::kUmmaSmemBytes) != cudaSuccess)
+            return GMLP_ERR_LAUNCH;
+        dev->umma_attr_set = true;
+    }
+    const int bn = GATEUP ? 128 : 256;
+    const int num_m = (int)((M + gmlp::kUmmaBM - 1) / gmlp::kUmmaBM);
+    const int num_n = (int)((N + bn - 1) / bn);
+    gmlp::umma_gemm_kernel<GATEUP><<<(unsigned)(num_m * num_n), gmlp::kUmmaThreads, gmlp::kUmmaSmemBytes, st>>>(
+        tmA, tmB0, tmB1, C, (int)M, (int)K, (int)N, num_m);
+    GMLP_CHECK_LAUNCH();
+    return GMLP_OK;
+}
+
+int read_device_status() {
+    if (cudaDeviceSynchronize() != cudaSuccess) return GMLP_ERR_LAUNCH;
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, gmlp::g_device_status, sizeof(int)) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    if (v != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(gmlp::g_device_status, &zero, sizeof(int)) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    }
+    return v;
+}
+
+int forward_impl(const gmlp_args* a) {
+    if (a == nullptr) return GMLP_ERR_NULL;
+    if (a->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
+    if (a->flags & ~kKnownFlags) return GMLP_ERR_FLAGS;
+    if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_UMMA) return GMLP_ERR_FLAGS;
+    int rc = check_shape(a->M, a->d_model, a->d_ff);
+    if (rc != GMLP_OK) return rc;
+    if (!a->X || !a->Wg || !a->Wu || !a->Wd || !a->Y) return GMLP_ERR_NULL;
+    if (!aligned16(a->X) || !aligned16(a->Wg) || !aligned16(a->Wu) || !aligned16(a->Wd) || !aligned16(a->Y) ||
+        !aligned16(a->rms_gain))
+        return GMLP_ERR_ALIGN;
+    if (a->workspace != nullptr && (reinterpret_cast<uintptr_t>(a->workspace) & 255u)) return GMLP_ERR_ALIGN;
+    const bool norm = (a->flags & GMLP_FLAG_RMSNORM) != 0;
+
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    if (a->M == 0) return GMLP_OK;
+
+    const int variant = resolve_variant(a->M, a->variant);
+    const Layout L = make_layout(a->M, a->d_model, a->d_ff, a->flags, variant, dev->sm_count);
+
+    uint8_t* ws = static_cast<uint8_t*>(a->workspace);
+    if (ws == nullptr) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (dev->workspace_bytes < L.total) {
+            // grow the library-owned buffer; work queued on the old one must finish first
+            if (dev->workspace != nullptr) {
+                if (cudaDeviceSynchronize() != cudaSuccess || cudaFree(dev->workspace) != cudaSuccess) return GMLP_ERR_LAUNCH;
+                dev->workspace = nullptr;
+                dev->workspace_bytes = 0;
+            }
+            void* p = nullptr;
+            if (cudaMalloc(&p, L.total) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return GMLP_ERR_WORKSPACE;
+            }
+            dev->workspace = p;
+            dev->workspace_bytes = L.total;
+        }
+        ws = static_cast<uint8_t*>(dev->workspace);
+    } else if (a->workspace_bytes < L.total) {
+        return GMLP_ERR_WORKSPACE;
+    }
+
+    cudaStream_t st = static_cast<cudaStream_t>(a->stream);
+    const bf16* X = static_cast<const bf16*>(a->X);
+    const bf16* Wg = static_cast<const bf16*>(a->Wg);
+    const bf16* Wu = static_cast<const bf16*>(a->Wu);
+    const bf16* Wd = static_cast<const bf16*>(a->Wd);
+    bf16* Y = static_cast<bf16*>(a->Y);
+    bf16* H = reinterpret_cast<bf16*>(ws + L.h_off);
+
+    prof_begin(st);
+    const bf16* A = X;
+    if (norm) {
+        bf16* Xn = reinterpret_cast<bf16*>(ws + L.xn_off);
+        rc = launch_rmsnorm(X, static_cast<const bf16*>(a->rms_gain), Xn, a->M, a->d_model, a->rms_eps, st);
+        if (rc != GMLP_OK) return rc;
+        prof_mark("rmsnorm", st);
+        A = Xn;
+    }
+
+    switch (variant) {
+        case GMLP_VARIANT_SIMT:
+            rc = run_simt(A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
+            break;
+        case GMLP_VARIANT_STREAM:
+            rc = run_stream(L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
+            break;
+        default:
+            rc = launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st);
+            if (rc == GMLP_OK) {
+                prof_mark("gate_up", st);
+                rc = launch_umma<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st);
+                if (rc == GMLP_OK) prof_mark("down", st);
+            }
+            break;
+    }
+    if (rc != GMLP_OK) return rc;
+
+    if (a->flags & GMLP_FLAG_CHECKED) {
+        if (cudaStreamSynchronize(st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+        const int s = read_device_status();
+        if (s < 0) return s;
+        if (s != 0) return GMLP_ERR_TIMEOUT;
+    }
+    return GMLP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gmlp_forward_ex(const gmlp_args* args) {
+    try {
+        return forward_impl(args);
+    } catch (...) {
+        return GMLP_ERR_LAUNCH;
+    }
+}
+
+int gmlp_forward(const void* X, const void* Wg, const void* Wu, const void* Wd, void* Y,
+                 int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags) {
+    gmlp_args a{};
+    a.struct_bytes = sizeof(gmlp_args);
+    a.flags = flags;
+    a.X = X; a.Wg = Wg; a.Wu = Wu; a.Wd = Wd; a.Y = Y;
+    a.M = M; a.d_model = d_model; a.d_ff = d_ff;
+    a.rms_gain = nullptr;
+    a.rms_eps = t_default_eps;
+    a.variant = GMLP_VARIANT_AUTO;
+    a.stream = t_stream;
+    a.workspace = nullptr;
+    a.workspace_bytes = 0;
+    return gmlp_forward_ex(&a);
+}
+
+int gmlp_forward_host(const gmlp_args* args, const void* X_host, void* Y_host) {
+    if (args == nullptr || X_host == nullptr || Y_host == nullptr) return GMLP_ERR_NULL;
+    if (args->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
+    int rc = check_shape(args->M, args->d_model, args->d_ff);
+    if (rc != GMLP_OK) return rc;
+    if (!args->X || !args->Y) return GMLP_ERR_NULL;
+    if (args->M == 0) return gmlp_forward_ex(args);
+    const size_t bytes = (size_t)args->M * (size_t)args->d_model * 2;
+    cudaStream_t st = static_cast<cudaStream_t>(args->stream);
+    if (cudaMemcpyAsync(const_cast<void*>(args->X), X_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return GMLP_ERR_LAUNCH;
+    rc = gmlp_forward_ex(args);
+    if (rc != GMLP_OK) return rc;
+    if (cudaMemcpyAsync(Y_host, args->Y, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    return GMLP_OK;
+}
+
+uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant) {
+    if (check_shape(M, d_model, d_ff) != GMLP_OK) return 0;
+    if (variant < GMLP_VARIANT_AUTO || variant > GMLP_VARIANT_UMMA) return 0;
+    int sm_count = 148;
+    int dev = -1;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) sm_count = sms;
+    }
+    (void)cudaGetLastError();
+    const Layout L = make_layout(M, d_model, d_ff, flags, resolve_variant(M, variant), sm_count);
+    return L.total > 256 ? L.total : 256;
+}
+
+int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags) {
+    (void)flags;
+    if (check_shape(M, d_model, d_ff) != GMLP_OK) return GMLP_ERR_SHAPE;
+    return resolve_variant(M, GMLP_VARIANT_AUTO);
+}
+
+int gmlp_device_status(void) {
+    int rc = GMLP_OK;
+    if (current_device(&rc) == nullptr) return rc;
+    return read_device_status();
+}
+
+int gmlp_profile_enable(int on) {
+    t_prof.on = (on != 0);
+    t_prof.n = 0;
+    return GMLP_OK;
+}
+
+int gmlp_profile_read(float* ms, int max_count, int* count) {
+    if (ms == nullptr || count == nullptr) return GMLP_ERR_NULL;
+    *count = 0;
+    if (!t_prof.created || t_prof.n == 0) return GMLP_OK;
+    if (cudaEventSynchronize(t_prof.ev[t_prof.n]) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    for (int i = 0; i < t_prof.n && i < max_count; ++i) {
+        if (cudaEventElapsedTime(&ms[i], t_prof.ev[i], t_prof.ev[i + 1]) != cudaSuccess) return GMLP_ERR_LAUNCH;
+        *count = i + 1;
+    }
+    return GMLP_OK;
+}
+
+const char* gmlp_profile_kernel_name(int index) {
+    if (index < 0 || index >= t_prof.n) return "";
+    return t_prof.names[index];
+}
+
+uint64_t gmlp_launch_count(void) { return t_launches; }
+void gmlp_reset_launch_count(void) { t_launches = 0; }
+
+const char* gmlp_status_string(int status) {
+    switch (status) {
+        case GMLP_OK: return "ok";
+        case GMLP_ERR_NULL: return "a required pointer is NULL";
+        case GMLP_ERR_SHAPE: return "bad shape: M < 0, or d_model/d_ff not a positive multiple of 8, or too large";
+        case GMLP_ERR_ALIGN: return "a pointer is not sufficiently aligned (16 bytes; workspace 256)";
+        case GMLP_ERR_FLAGS: return "unknown flag bit, unknown variant or wrong struct_bytes";
+        case GMLP_ERR_WORKSPACE: return "workspace too small or could not be allocated";
+        case GMLP_ERR_ARCH: return "no CUDA device, or the current device is not sm_100";
+        case GMLP_ERR_LAUNCH: return "a CUDA runtime call failed";
+        case GMLP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case GMLP_ERR_UNSUPPORTED: return "the forced variant cannot run this shape";
+        default: return "unknown status";
+    }
+}
+
+int gmlp_version(void) { return kVersion; }
+
+int gmlp_set_stream(void* cuda_stream) {
+    t_stream = static_cast<cudaStream_t>(cuda_stream);
+    return GMLP_OK;
+}
+
+int gmlp_set_default_eps(float eps) {
+    if (!(eps >= 0.0f)) return GMLP_ERR_FLAGS;
+    t_default_eps = eps;
+    return GMLP_OK;
+}
+
+void gmlp_shutdown(void) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) { (void)cudaGetLastError(); return; }
+    for (int d = 0; d < kMaxDevices; ++d) {
+        if (g_dev[d].workspace != nullptr) {
+            if (cudaSetDevice(d) == cudaSuccess) {
+                (void)cudaDeviceSynchronize();
+                (void)cudaFree(g_dev[d].workspace);
+            }
+            g_dev[d].workspace = nullptr;
+            g_dev[d].workspace_bytes = 0;
+        }
+    }
+    (void)cudaSetDevice(prev);
+    (void)cudaGetLastError();
+}
+
+}  // extern "C"

@@ -1,0 +1,40 @@
+// Shared device helpers of libgmlp (sm_100a only).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gmlp {
+
+typedef __nv_bfloat16 bf16;
+
+// Device status word: 0, or (kernel id << 16 | site) of the first bounded wait that ran out.
+__device__ int g_device_status = 0;
+
+__device__ __forceinline__ void report_timeout(int kernel_id, int site) {
+    atomicCAS(&g_device_status, 0, (kernel_id << 16) | (site & 0xFFFF));
+}
+
+// silu(g) = g * sigmoid(g), written g / (1 + e^-g): for g -> -inf this tends to -0 and never
+// forms 0 * inf.  ex2.approx / fast division are ~2^-21 relative, far below a bf16 ulp.
+__device__ __forceinline__ float silu_f32(float g) {
+    return __fdividef(g, 1.0f + __expf(-g));
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // .x = lo (low half), .y = hi
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// 16-byte read-only load that does not allocate in L1 (weights are streamed once).
+__device__ __forceinline__ uint4 ld_stream_16B(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+}  // namespace gmlp

@@ -1,0 +1,67 @@
+// RMSNorm prologue (Eq. 1, Section 2; graph order square -> mean -> add eps -> rsqrt ->
+// multiply), with an optional per-column gain:  Xn[m,k] = bf16_rn(X[m,k] * r_m * gamma[k]),
+// r_m = rsqrt(mean_k X[m,k]^2 + eps).  One CTA per row; fp32 arithmetic; one rounding.
+#pragma once
+#include "common.cuh"
+
+namespace gmlp {
+
+constexpr int kRmsThreads = 256;
+
+__global__ void __launch_bounds__(kRmsThreads)
+rmsnorm_kernel(const bf16* __restrict__ X, const bf16* __restrict__ gamma, bf16* __restrict__ Xn,
+               int64_t M, int d_model, float eps)
+{
+    const int64_t row = blockIdx.x;
+    if (row >= M) return;
+    const uint4* x = reinterpret_cast<const uint4*>(X + row * d_model);
+    const uint4* g = reinterpret_cast<const uint4*>(gamma);
+    uint4* out = reinterpret_cast<uint4*>(Xn + row * d_model);
+    const int nvec = d_model >> 3;
+
+    float ss = 0.0f;
+    for (int i = threadIdx.x; i < nvec; i += kRmsThreads) {
+        const uint4 v = x[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float a = bf16_lo(w[j]), b = bf16_hi(w[j]);
+            ss = fmaf(a, a, ss);
+            ss = fmaf(b, b, ss);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+    __shared__ float warp_sums[kRmsThreads / 32];
+    __shared__ float r_shared;
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kRmsThreads / 32; ++w) t += warp_sums[w];
+        r_shared = rsqrtf(t / (float)d_model + eps);
+    }
+    __syncthreads();
+    const float r = r_shared;
+
+    for (int i = threadIdx.x; i < nvec; i += kRmsThreads) {
+        const uint4 v = x[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t gw[4] = {0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u};   // bf16 ones
+        if (gamma != nullptr) {
+            const uint4 gv = g[i];
+            gw[0] = gv.x; gw[1] = gv.y; gw[2] = gv.z; gw[3] = gv.w;
+        }
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float a = bf16_lo(w[j]) * r * bf16_lo(gw[j]);
+            const float b = bf16_hi(w[j]) * r * bf16_hi(gw[j]);
+            o[j] = pack_bf16x2(a, b);
+        }
+        out[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+}  // namespace gmlp

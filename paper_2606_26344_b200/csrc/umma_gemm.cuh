@@ -1,0 +1,210 @@
+// Large-M schedule: tcgen05 tensor-core GEMMs with the Gated-MLP epilogues.
+//
+//   GATEUP = true :  H[m, n] = bf16_rn( silu(sum_k A[m,k] Wg[k,n]) * (sum_k A[m,k] Wu[k,n]) )
+//                    one CTA tile = 128 rows x 128 H-columns; a single N = 256 MMA holds the
+//                    gate columns in TMEM columns [0,128) and the up columns in [128,256),
+//                    so an epilogue thread owns g and u of the same element: SiLU and the
+//                    product happen in registers and H is written once
+//   GATEUP = false:  Y[m, c] = bf16_rn( sum_n H[m,n] Wd[n,c] ),  tile = 128 rows x 256 columns
+//
+// Operands: A is row-major [M, K] = K-major for the MMA; the weights are row-major [K, N]
+// ("[in, out]"), i.e. MN-major B operands, which tcgen05 consumes directly (no transpose is
+// ever materialised).  TMA (128-byte swizzle) fills a ring of shared-memory stages; one
+// thread issues tcgen05.mma; fp32 accumulators live in TMEM; four epilogue warps read them
+// back with tcgen05.ld.  Ragged M / N / K come from TMA's zero fill and predicated stores.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
+// warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31).
+// Every mbarrier wait is bounded; a wait that runs out records a status word, raises a
+// CTA-wide abort flag and the CTA leaves through the normal teardown (TMEM freed).
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace gmlp {
+
+constexpr int kUmmaBM = 128;
+constexpr int kUmmaBK = 64;
+constexpr int kUmmaN = 256;                 // MMA N: 128 gate + 128 up, or 256 plain columns
+constexpr int kUmmaStages = 4;
+constexpr int kUmmaThreads = 192;
+constexpr uint32_t kUmmaABytes = kUmmaBM * kUmmaBK * 2;          // 16 KB: 128 rows x 128 B
+constexpr uint32_t kUmmaBoxBBytes = 64 * kUmmaBK * 2;            // 8 KB: 64 k-rows x 128 B (64 columns)
+constexpr uint32_t kUmmaBBytes = 4 * kUmmaBoxBBytes;             // 32 KB
+constexpr uint32_t kUmmaStageBytes = kUmmaABytes + kUmmaBBytes;  // 48 KB
+constexpr uint32_t kUmmaSmemBytes = kUmmaStages * kUmmaStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr long long kWaitLimitCycles = 2000000000LL;             // about a second
+
+// kind::f16 instruction descriptor: D = fp32, A = B = bf16, A K-major, B MN-major, M = 128, N = 256.
+constexpr uint32_t kUmmaIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                                ((uint32_t)(kUmmaN >> 3) << 17) | ((uint32_t)(kUmmaBM >> 4) << 24);
+
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                             int kernel_id, int site) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long start = clock64();
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - start > kWaitLimitCycles) {
+            *abort_flag = 1;
+            report_timeout(kernel_id, site);
+            return false;
+        }
+    }
+    return true;
+}
+
+template <bool GATEUP>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+                 const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
+                 int M, int K, int N, int num_m_tiles)
+{
+    constexpr int KERNEL_ID = GATEUP ? 1 : 2;
+    constexpr int BN_OUT = GATEUP ? 128 : 256;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;            // swizzle atoms need 1024-byte alignment
+    uint8_t* base_ptr = smem_raw + (base - raw_addr);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + kUmmaStages * kUmmaStageBytes);
+    const uint32_t full0 = ptx::smem_addr(bars);
+    const uint32_t empty0 = ptx::smem_addr(bars + kUmmaStages);
+    const uint32_t tmem_full = ptx::smem_addr(bars + 2 * kUmmaStages);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kUmmaStages + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m_tile = blockIdx.x % num_m_tiles;                  // row tiles fastest: CTAs of a wave share weight panels
+    const int n_tile = blockIdx.x / num_m_tiles;
+    const int m0 = m_tile * kUmmaBM;
+    const int n0 = n_tile * BN_OUT;
+    const int num_kb = (K + kUmmaBK - 1) / kUmmaBK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kUmmaStages; ++s) {
+            ptx::mbar_init(full0 + 8 * s, 1);
+            ptx::mbar_init(empty0 + 8 * s, 1);
+        }
+        ptx::mbar_init(tmem_full, 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::fence_proxy_async_smem();
+        ptx::prefetch_tensormap(&tmA);
+        ptx::prefetch_tensormap(&tmB0);
+        if (GATEUP) ptx::prefetch_tensormap(&tmB1);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_addr(tmem_slot), kUmmaN);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % kUmmaStages;
+                const uint32_t ph = (uint32_t)(kb / kUmmaStages) & 1u;
+                if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
+                const uint32_t full = full0 + 8 * s;
+                const uint32_t a_dst = base + s * kUmmaStageBytes;
+                const uint32_t b_dst = a_dst + kUmmaABytes;
+                ptx::mbar_arrive_expect_tx(full, kUmmaStageBytes);
+                ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const CUtensorMap* map = (GATEUP && i >= 2) ? &tmB1 : &tmB0;
+                    const int x = GATEUP ? n0 + (i & 1) * 64 : n0 + i * 64;
+                    ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            bool ok = true;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % kUmmaStages;
+                const uint32_t ph = (uint32_t)(kb / kUmmaStages) & 1u;
+                if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
+                ptx::tc_fence_after_sync();
+                const uint32_t a_base = base + s * kUmmaStageBytes;
+                const uint32_t b_base = a_base + kUmmaABytes;
+#pragma unroll
+                for (int k = 0; k < kUmmaBK / 16; ++k) {
+                    // A: K-major, rows of 128 B, 8-row groups 1024 B apart; +32 B per K = 16 step.
+                    // B: MN-major, 64-column chunks 8 KB apart (LBO), 8-row k-groups 1024 B apart (SBO);
+                    //    K = 16 is two k-groups: +2048 B per step.
+                    const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
+                    const uint64_t b_desc = ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
+                    ptx::umma_bf16(tmem_base, a_desc, b_desc, kUmmaIdesc, (kb | k) != 0 ? 1u : 0u);
+                }
+                ptx::umma_commit(empty0 + 8 * s);      // stage is free once these MMAs have read it
+            }
+            if (ok) ptx::umma_commit(tmem_full);       // accumulator complete
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue ----------------
+        const int q = warp & 3;
+        const int row = m0 + q * 32 + lane;
+        const bool ok = wait_bounded(tmem_full, 0u, abort_flag, KERNEL_ID, 3);
+        ptx::tc_fence_after_sync();
+        if (ok) {
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+            bf16* crow = C + (size_t)row * N + n0;
+#pragma unroll 1
+            for (int c = 0; c < BN_OUT; c += 32) {
+                uint32_t g[32];
+                uint32_t packed[16];
+                if (GATEUP) {
+                    uint32_t u[32];
+                    ptx::tmem_ld_32x32(taddr + c, g);
+                    ptx::tmem_ld_32x32(taddr + 128 + c, u);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float h0 = silu_f32(__uint_as_float(g[2 * j])) * __uint_as_float(u[2 * j]);
+                        const float h1 = silu_f32(__uint_as_float(g[2 * j + 1])) * __uint_as_float(u[2 * j + 1]);
+                        packed[j] = pack_bf16x2(h0, h1);
+                    }
+                } else {
+                    ptx::tmem_ld_32x32(taddr + c, g);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        packed[j] = pack_bf16x2(__uint_as_float(g[2 * j]), __uint_as_float(g[2 * j + 1]));
+                }
+                if (row < M) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        if (n0 + c + v * 8 < N)
+                            *reinterpret_cast<uint4*>(crow + c + v * 8) =
+                                make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                    }
+                }
+            }
+        }
+    }
+
+    if (*abort_flag) {
+        // A wait ran out: give copies that may still be in flight time to land before the
+        // shared memory is handed back, then leave through the same teardown.
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kUmmaN);
+    }
+}
+
+}  // namespace gmlp

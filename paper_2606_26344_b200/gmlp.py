@@ -1,0 +1,194 @@
+"""Thin ctypes binding over ``libgmlp.so`` (argument marshalling only).
+
+Every step of the operator runs in the library's CUDA kernels; torch is used here for
+device memory and streams.  The names mirror ``include/gmlp.h``.  If the library has not
+been built this module raises on first use: there is no CPU or eager fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+OK = 0
+ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_FLAGS, ERR_WORKSPACE, ERR_ARCH, ERR_LAUNCH, ERR_TIMEOUT, ERR_UNSUPPORTED = \
+    -1, -2, -3, -4, -5, -6, -7, -8, -9
+FLAG_RMSNORM = 1 << 0
+FLAG_CHECKED = 1 << 2
+VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA = 0, 1, 2, 3
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgmlp.so")
+_lib = None
+
+
+class GmlpArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_bytes", ctypes.c_uint32), ("flags", ctypes.c_uint32),
+        ("X", ctypes.c_void_p), ("Wg", ctypes.c_void_p), ("Wu", ctypes.c_void_p), ("Wd", ctypes.c_void_p),
+        ("Y", ctypes.c_void_p),
+        ("M", ctypes.c_int64), ("d_model", ctypes.c_int64), ("d_ff", ctypes.c_int64),
+        ("rms_gain", ctypes.c_void_p), ("rms_eps", ctypes.c_float), ("variant", ctypes.c_int32),
+        ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_uint64),
+    ]
+
+
+class GmlpError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__(f"libgmlp error {status}: {status_string(status)}")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libgmlp.so (once).  Raises if it is missing: build it with ``__graft_entry__.build()``."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} not found: the CUDA library must be built first "
+                               "(python -m paper_2606_26344_b200.build); there is no fallback path")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i64, u32, u64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int32
+        L.gmlp_forward.restype = ctypes.c_int
+        L.gmlp_forward.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, u32]
+        L.gmlp_forward_ex.restype = ctypes.c_int
+        L.gmlp_forward_ex.argtypes = [ctypes.POINTER(GmlpArgs)]
+        L.gmlp_forward_host.restype = ctypes.c_int
+        L.gmlp_forward_host.argtypes = [ctypes.POINTER(GmlpArgs), vp, vp]
+        L.gmlp_workspace_bytes.restype = u64
+        L.gmlp_workspace_bytes.argtypes = [i64, i64, i64, u32, i32]
+        L.gmlp_pick_variant.restype = ctypes.c_int
+        L.gmlp_pick_variant.argtypes = [i64, i64, i64, u32]
+        L.gmlp_device_status.restype = ctypes.c_int
+        L.gmlp_device_status.argtypes = []
+        L.gmlp_launch_count.restype = u64
+        L.gmlp_launch_count.argtypes = []
+        L.gmlp_reset_launch_count.restype = None
+        L.gmlp_reset_launch_count.argtypes = []
+        L.gmlp_profile_enable.restype = ctypes.c_int
+        L.gmlp_profile_enable.argtypes = [ctypes.c_int]
+        L.gmlp_profile_read.restype = ctypes.c_int
+        L.gmlp_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+        L.gmlp_profile_kernel_name.restype = ctypes.c_char_p
+        L.gmlp_profile_kernel_name.argtypes = [ctypes.c_int]
+        L.gmlp_status_string.restype = ctypes.c_char_p
+        L.gmlp_status_string.argtypes = [ctypes.c_int]
+        L.gmlp_version.restype = ctypes.c_int
+        L.gmlp_version.argtypes = []
+        L.gmlp_set_stream.restype = ctypes.c_int
+        L.gmlp_set_stream.argtypes = [vp]
+        L.gmlp_set_default_eps.restype = ctypes.c_int
+        L.gmlp_set_default_eps.argtypes = [ctypes.c_float]
+        L.gmlp_shutdown.restype = None
+        L.gmlp_shutdown.argtypes = []
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().gmlp_status_string(int(status)).decode()
+
+
+def workspace_bytes(M: int, d_model: int, d_ff: int, flags: int = 0, variant: int = VARIANT_AUTO) -> int:
+    return int(lib().gmlp_workspace_bytes(M, d_model, d_ff, flags, variant))
+
+
+def pick_variant(M: int, d_model: int, d_ff: int, flags: int = 0) -> int:
+    return int(lib().gmlp_pick_variant(M, d_model, d_ff, flags))
+
+
+def device_status() -> int:
+    return int(lib().gmlp_device_status())
+
+
+def launch_count() -> int:
+    return int(lib().gmlp_launch_count())
+
+
+def reset_launch_count() -> None:
+    lib().gmlp_reset_launch_count()
+
+
+def profile_enable(on: bool) -> None:
+    lib().gmlp_profile_enable(1 if on else 0)
+
+
+def profile_read() -> dict:
+    """Durations (ms) of the kernels of the most recent forward_ex call, keyed by kernel name."""
+    ms = (ctypes.c_float * 8)()
+    n = ctypes.c_int(0)
+    rc = lib().gmlp_profile_read(ms, 8, ctypes.byref(n))
+    if rc != OK:
+        raise GmlpError(rc)
+    return {lib().gmlp_profile_kernel_name(i).decode(): float(ms[i]) for i in range(n.value)}
+
+
+def _check_bf16_cuda(t: torch.Tensor, name: str) -> None:
+    if not (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA bfloat16 tensor")
+
+
+def make_args(X, Wg, Wu, Wd, Y, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, variant: int = VARIANT_AUTO,
+              workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
+              checked: bool = False) -> GmlpArgs:
+    for t, n in ((X, "X"), (Wg, "Wg"), (Wu, "Wu"), (Wd, "Wd"), (Y, "Y")):
+        _check_bf16_cuda(t, n)
+    M, d_model = X.shape
+    d_ff = Wg.shape[1]
+    if Wg.shape != (d_model, d_ff) or Wu.shape != (d_model, d_ff) or Wd.shape != (d_ff, d_model) or Y.shape != X.shape:
+        raise ValueError("shape mismatch")
+    flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0)
+    if gamma is not None:
+        _check_bf16_cuda(gamma, "gamma")
+    st = stream if stream is not None else torch.cuda.current_stream(X.device)
+    a = GmlpArgs()
+    a.struct_bytes = ctypes.sizeof(GmlpArgs)
+    a.flags = flags
+    a.X, a.Wg, a.Wu, a.Wd, a.Y = X.data_ptr(), Wg.data_ptr(), Wu.data_ptr(), Wd.data_ptr(), Y.data_ptr()
+    a.M, a.d_model, a.d_ff = M, d_model, d_ff
+    a.rms_gain = gamma.data_ptr() if gamma is not None else None
+    a.rms_eps = eps
+    a.variant = variant
+    a.stream = st.cuda_stream
+    a.workspace = workspace.data_ptr() if workspace is not None else None
+    a.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    return a
+
+
+def alloc_workspace(M: int, d_model: int, d_ff: int, rmsnorm: bool = False, variant: int = VARIANT_AUTO,
+                    device="cuda") -> torch.Tensor:
+    n = workspace_bytes(M, d_model, d_ff, FLAG_RMSNORM if rmsnorm else 0, variant)
+    return torch.empty(n + 256, dtype=torch.uint8, device=device)[:n] if n else torch.empty(256, dtype=torch.uint8, device=device)
+
+
+def forward_ex(args: GmlpArgs) -> None:
+    rc = lib().gmlp_forward_ex(ctypes.byref(args))
+    if rc != OK:
+        raise GmlpError(rc)
+
+
+def forward(X, Wg, Wu, Wd, Y=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False,
+            variant: int = VARIANT_AUTO, workspace=None, stream=None, checked: bool = False) -> torch.Tensor:
+    """Y = (silu(Xn Wg) * (Xn Wu)) Wd on the GPU; asynchronous on ``stream`` (default: torch's current stream)."""
+    if Y is None:
+        Y = torch.empty_like(X)
+    with torch.cuda.device(X.device):
+        forward_ex(make_args(X, Wg, Wu, Wd, Y, gamma, eps, rmsnorm, variant, workspace, stream, checked))
+    return Y
+
+
+def forward_host(args: GmlpArgs, X_host: torch.Tensor, Y_host: torch.Tensor) -> None:
+    """gmlp_forward_host: X_host / Y_host are host (ideally pinned) bf16 tensors; args.X / args.Y device staging."""
+    rc = lib().gmlp_forward_host(ctypes.byref(args), X_host.data_ptr(), Y_host.data_ptr())
+    if rc != OK:
+        raise GmlpError(rc)
+
+
+def forward_simple(X, Wg, Wu, Wd, Y, flags: int = 0) -> None:
+    """The nine-argument call exactly as the operator is stated."""
+    M, d_model = X.shape
+    with torch.cuda.device(X.device):
+        rc = lib().gmlp_forward(X.data_ptr(), Wg.data_ptr(), Wu.data_ptr(), Wd.data_ptr(), Y.data_ptr(),
+                                M, d_model, Wg.shape[1], flags)
+    if rc != OK:
+        raise GmlpError(rc)

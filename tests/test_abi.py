@@ -1,0 +1,107 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol
+the header declares, and rejects bad arguments with the documented codes before any device
+work."""
+import ctypes
+import os
+import re
+
+import pytest
+import torch
+
+from paper_2606_26344_b200 import build as B
+from paper_2606_26344_b200 import gmlp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "gmlp.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    B.build_libgmlp()
+    return gmlp.lib()
+
+
+def declared_symbols():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gmlp_[a-z_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(lib):
+    names = declared_symbols()
+    assert "gmlp_forward" in names and "gmlp_forward_ex" in names and "gmlp_workspace_bytes" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in gmlp.h but not exported"
+
+
+def test_struct_layout_matches_header(lib):
+    # 2 x u32, 5 pointers, 3 x i64, pointer, float, i32, 2 pointers, u64 on LP64
+    assert ctypes.sizeof(gmlp.GmlpArgs) == 8 + 5 * 8 + 3 * 8 + 8 + 4 + 4 + 8 + 8 + 8
+
+
+def test_version_and_status_strings(lib):
+    assert lib.gmlp_version() >= 100
+    for code in range(-9, 1):
+        assert gmlp.status_string(code) and gmlp.status_string(code) != "unknown status"
+    assert gmlp.status_string(-99) == "unknown status"
+
+
+def _args(**kw):
+    a = gmlp.GmlpArgs()
+    a.struct_bytes = ctypes.sizeof(gmlp.GmlpArgs)
+    a.X = a.Wg = a.Wu = a.Wd = a.Y = 0x1000
+    a.M, a.d_model, a.d_ff = 4, 64, 128
+    for k, v in kw.items():
+        setattr(a, k, v)
+    return a
+
+
+def test_argument_validation_happens_before_device_work(lib):
+    f = lambda a: lib.gmlp_forward_ex(ctypes.byref(a))
+    assert lib.gmlp_forward_ex(None) == gmlp.ERR_NULL
+    assert f(_args(struct_bytes=8)) == gmlp.ERR_FLAGS
+    assert f(_args(flags=1 << 7)) == gmlp.ERR_FLAGS
+    assert f(_args(variant=17)) == gmlp.ERR_FLAGS
+    assert f(_args(M=-1)) == gmlp.ERR_SHAPE
+    assert f(_args(d_model=60)) == gmlp.ERR_SHAPE
+    assert f(_args(d_ff=0)) == gmlp.ERR_SHAPE
+    assert f(_args(d_ff=12)) == gmlp.ERR_SHAPE
+    assert f(_args(X=None)) == gmlp.ERR_NULL
+    assert f(_args(Y=None)) == gmlp.ERR_NULL
+    assert f(_args(Wd=0x1008)) == gmlp.ERR_ALIGN
+    assert f(_args(workspace=0x1010, workspace_bytes=1 << 20)) == gmlp.ERR_ALIGN
+    assert lib.gmlp_forward(None, 0x1000, 0x1000, 0x1000, 0x1000, 4, 64, 128, 0) == gmlp.ERR_NULL
+    assert lib.gmlp_forward_host(None, 0x1000, 0x1000) == gmlp.ERR_NULL
+    assert lib.gmlp_forward_host(ctypes.byref(_args()), None, 0x1000) == gmlp.ERR_NULL
+    assert lib.gmlp_set_default_eps(-1.0) == gmlp.ERR_FLAGS
+    assert lib.gmlp_set_default_eps(1e-5) == gmlp.OK
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-device behaviour")
+def test_no_device_means_arch_error_not_fallback(lib):
+    assert lib.gmlp_forward_ex(ctypes.byref(_args())) == gmlp.ERR_ARCH
+    assert lib.gmlp_device_status() == gmlp.ERR_ARCH
+
+
+def test_workspace_sizes_and_variant_choice(lib):
+    wb = gmlp.workspace_bytes
+    assert wb(0, 64, 128) >= 256 and wb(-1, 64, 128) == 0 and wb(4, 60, 128) == 0
+    M, dm, dff = 2048, 4096, 14336
+    h = M * dff * 2
+    assert wb(M, dm, dff, 0, gmlp.VARIANT_UMMA) >= h
+    assert wb(M, dm, dff, gmlp.FLAG_RMSNORM, gmlp.VARIANT_UMMA) >= h + M * dm * 2
+    assert wb(M, dm, dff, 0, gmlp.VARIANT_UMMA) < h + 4096
+    assert wb(8, dm, dff, 0, gmlp.VARIANT_STREAM) > wb(8, dm, dff, 0, gmlp.VARIANT_SIMT)     # split-K partials
+    assert wb(8, dm, dff, 0, gmlp.VARIANT_STREAM) < 64 << 20
+    assert gmlp.pick_variant(8, dm, dff) == gmlp.VARIANT_STREAM
+    assert gmlp.pick_variant(1, 2048, 5632) == gmlp.VARIANT_STREAM
+    assert gmlp.pick_variant(2048, dm, dff) == gmlp.VARIANT_UMMA
+    assert gmlp.pick_variant(4096, 8192, 28672) == gmlp.VARIANT_UMMA
+    assert gmlp.pick_variant(4, 60, 128) == gmlp.ERR_SHAPE
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(gmlp, "_lib", None)
+    monkeypatch.setattr(gmlp, "_LIB_PATH", str(tmp_path / "libgmlp.so"))
+    with pytest.raises(RuntimeError, match="no fallback"):
+        gmlp.lib()
