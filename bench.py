@@ -1,0 +1,393 @@
+#!/usr/bin/env python
+"""Benchmark of the fused Gated MLP (libgmlp) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--no-extra]
+    python bench.py --impl reference ...          # times the CPU oracle on the host cores
+
+One "step" is one pass of the whole hot path (optional RMSNorm, gate/up GEMM with the SiLU
+product epilogue, down GEMM) over one batch of synthetic, seeded input.  Rank 0 prints ONE
+JSON line.  ``value`` is whole-job tokens/s with the inputs resident in HBM; ``e2e`` is the
+same metric through the host-buffer entry point (host->device copy of X and device->host
+copy of Y inside the timed region).  The line also carries the roofline of the dominant
+kernel (measured with CUDA events around that kernel), the CPU oracle timed on the host
+cores, the SM clocks sampled during the timed region, and, unless --no-extra, the same
+measurements for the other stated workloads under "workloads".
+
+With N > 1 (torchrun) every rank runs the same workload on its own rows (data parallel:
+rows are independent, weights replicated, no collective on the data path): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+PRIMARY = "llama3-8b-decode-M8"
+EXTRA = ["llama3-8b-prefill-M2048-rmsnorm", "llama3-70b-prefill-M4096-outliers", "ragged-M8192-plain",
+         "ragged-M1000-plain", "ragged-M129-plain", "ragged-M7-plain", "ragged-M1-plain"]
+L2_BYTES = 126 * 1024 * 1024
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons in the background during a timed region."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def cpu_oracle_rate(inp, rows, min_seconds: float):
+    """Times the oracle as it stands on `rows`, repeating whole passes until min_seconds have elapsed."""
+    import oracle
+    w = inp.workload
+    args = (inp.bits("X"), inp.bits("Wg"), inp.bits("Wu"), inp.bits("Wd"))
+    kw = dict(rows=rows, gamma=inp.bits("gamma") if w.rmsnorm else None, eps=w.eps, rmsnorm=w.rmsnorm)
+    oracle.build()
+    done, t0 = 0, time.perf_counter()
+    while True:
+        oracle.gmlp_rows(*args, **kw)
+        done += len(rows)
+        dt = time.perf_counter() - t0
+        if dt >= min_seconds:
+            break
+    return done / dt, done, dt, oracle.max_threads()
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, as it stands, on the host cores; one step = one bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    from paper_2606_26344_b200 import inputs as I
+    w = I.WORKLOADS[args.workload]
+    inp = I.make_inputs(w)
+    rows = I.sample_rows(w, inp.outlier_rows)
+    n_rows = min(len(rows), 8)
+    rows = rows[:n_rows]
+    X, Wg, Wu, Wd = (inp.bits(n) for n in ("X", "Wg", "Wu", "Wd"))
+    kw = dict(rows=rows, gamma=inp.bits("gamma") if w.rmsnorm else None, eps=w.eps, rmsnorm=w.rmsnorm)
+    oracle.build()
+    for _ in range(args.warmup):
+        oracle.gmlp_rows(X, Wg, Wu, Wd, **kw)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.gmlp_rows(X, Wg, Wu, Wd, **kw)
+    dt = time.perf_counter() - t0
+    value = n_rows * args.steps / dt
+    cores = oracle.max_threads()
+    sample = f"{n_rows} rows of the workload per step (rows are independent), fp64, OpenMP over rows"
+    print(json.dumps({
+        "impl": "reference", "metric": "gated_mlp_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "M": w.M, "d_model": w.d_model, "d_ff": w.d_ff, "rmsnorm": w.rmsnorm},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sample_clocks=True):
+    """Times one workload on this rank's GPU.  Returns a dict of measurements."""
+    import torch
+    from paper_2606_26344_b200 import gmlp, inputs as I
+
+    inp = I.make_inputs(w)
+    X, Wg, Wu, Wd = (t.to(dev) for t in (inp.X, inp.Wg, inp.Wu, inp.Wd))
+    gamma = inp.gamma.to(dev) if inp.gamma is not None else None
+    Y = torch.empty_like(X)
+    variant = gmlp.pick_variant(w.M, w.d_model, w.d_ff)
+    ws = gmlp.alloc_workspace(w.M, w.d_model, w.d_ff, w.rmsnorm)
+    stream = torch.cuda.current_stream(dev)
+    a = gmlp.make_args(X, Wg, Wu, Wd, Y, gamma, w.eps, w.rmsnorm, gmlp.VARIANT_AUTO, ws, stream)
+    weight_bytes = 3 * w.d_model * w.d_ff * 2
+    fits_l2 = weight_bytes < L2_BYTES
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if fits_l2 else None
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(warmup):
+        gmlp.forward_ex(a)
+    torch.cuda.synchronize(dev)
+    st = gmlp.device_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st:#x} after warm-up")
+
+    # The timed region of a small workload lasts a few milliseconds, shorter than nvidia-smi's sampling
+    # period.  The clocks are therefore sampled over an untimed pre-roll of the same steps, the timed
+    # region and an untimed post-roll: one continuous stretch of identical load.
+    sampler = ClockSampler(dev.index or 0) if sample_clocks else None
+
+    def roll(seconds):
+        t_end = time.perf_counter() + seconds
+        while time.perf_counter() < t_end:
+            for _ in range(20):
+                gmlp.forward_ex(a)
+            torch.cuda.synchronize(dev)
+
+    if sampler:
+        sampler.start()
+        roll(0.6)
+    gmlp.reset_launch_count()
+    if not fits_l2:
+        # inputs are larger than L2: back-to-back steps, one pair of events around the region
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            gmlp.forward_ex(a)
+        e1.record(stream)
+        barrier()
+        total_ms = e0.elapsed_time(e1)
+        per_step = [total_ms / steps]
+    else:
+        # weights would stay in L2: overwrite L2 between steps and time each step on its own
+        barrier()
+        evs = []
+        for _ in range(steps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            gmlp.forward_ex(a)
+            e1.record(stream)
+            evs.append((e0, e1))
+        barrier()
+        per_step = [x.elapsed_time(y) for x, y in evs]
+        total_ms = sum(per_step)
+    launches = gmlp.launch_count()
+    if sampler:
+        roll(0.6)
+    clocks = sampler.stop() if sampler else None
+    if clocks is not None:
+        clocks["window"] = "pre-roll 0.6 s + timed region + post-roll 0.6 s of the same steps"
+    ms = total_ms / steps
+
+    # per-kernel durations, in a loop of their own (events between kernels perturb the launch stream)
+    gmlp.profile_enable(True)
+    kern = {}
+    n_prof = max(3, min(steps, 20))
+    for _ in range(n_prof):
+        if flush is not None:
+            flush.fill_(1)
+        gmlp.forward_ex(a)
+        for k, v in gmlp.profile_read().items():
+            kern.setdefault(k, []).append(v)
+    gmlp.profile_enable(False)
+    kern_ms = {k: sum(v) / len(v) for k, v in kern.items()}
+
+    res = {"name": w.name, "M": w.M, "d_model": w.d_model, "d_ff": w.d_ff, "rmsnorm": w.rmsnorm,
+           "variant": {1: "simt", 2: "stream", 3: "umma", 4: "skinny"}[variant], "ms_per_step": ms,
+           "ms_min": min(per_step), "tokens_per_s": w.M / (ms * 1e-3), "tflops": w.flops / (ms * 1e-3) / 1e12,
+           "gbps_min_bytes": w.min_bytes / (ms * 1e-3) / 1e9, "launches": launches, "clocks": clocks,
+           "kernel_ms": kern_ms,
+           "l2": "L2 overwritten between steps (weights fit L2); each step timed alone" if fits_l2
+                 else "inputs larger than L2; steps back to back"}
+
+    # roofline of the path and of its dominant kernel
+    t_tensor = w.flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = w.min_bytes / (peaks["hbm_gbs"] * 1e9)
+    res["roofline_path"] = {"bound": "tensor" if t_tensor >= t_hbm else "hbm",
+                            "frac": max(t_tensor, t_hbm) / (ms * 1e-3)}
+    if "gate_up" in kern_ms:
+        kms = kern_ms["gate_up"] * 1e-3
+        if t_tensor >= t_hbm:
+            flops = 4 * w.M * w.d_model * w.d_ff
+            ach = flops / kms / 1e12
+            res["roofline"] = {"kernel": "gate_up", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
+                               "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"], "traffic": None,
+                               "peak_source": peaks["source"] + " (burst bf16)"}
+        else:
+            nbytes = 2 * (2 * w.d_model * w.d_ff + w.M * w.d_model + w.M * w.d_ff)
+            ach = nbytes / kms / 1e9
+            res["roofline"] = {"kernel": "gate_up", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                               "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                               "peak_source": peaks["source"] + " (copy)"}
+
+    if want_e2e:
+        Xh, Yh = inp.X.pin_memory(), torch.empty_like(inp.X).pin_memory()
+        for _ in range(3):
+            gmlp.forward_host(a, Xh, Yh)
+        barrier()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        n_e2e = max(3, min(steps, 50))
+        t0.record(stream)
+        for _ in range(n_e2e):
+            gmlp.forward_host(a, Xh, Yh)
+        t1.record(stream)
+        barrier()
+        e2e_ms = t0.elapsed_time(t1) / n_e2e
+        nb = w.M * w.d_model * 2
+        res["e2e"] = {"value": w.M / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+                      "h2d_bytes_per_step": nb, "d2h_bytes_per_step": nb, "steps": n_e2e}
+    res["_inputs"] = inp
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="gmlp", choices=["gmlp", "reference"])
+    ap.add_argument("--workload", default=PRIMARY)
+    ap.add_argument("--no-extra", action="store_true", help="time only the primary workload")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time spent on the oracle baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2606_26344_b200 import build as B
+    from paper_2606_26344_b200 import gmlp, inputs as I
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if rank == 0:
+        B.build_libgmlp()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist = dist_mod
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    if dist is not None:
+        dist.barrier()
+    gmlp.lib()
+    peaks = load_peaks()
+    warmup = max(args.warmup, 3)
+
+    w = I.WORKLOADS[args.workload]
+    res = measure_workload(w, args.steps, warmup, dev, peaks, dist=dist)
+    ms = res["ms_per_step"]
+    if dist is not None:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        e = torch.tensor([res["e2e"]["ms_per_step"]], device=dev, dtype=torch.float64)
+        dist.all_reduce(e, op=dist.ReduceOp.MAX)
+        res["e2e"]["ms_per_step"] = float(e.item())
+        res["e2e"]["value"] = world * w.M / (res["e2e"]["ms_per_step"] * 1e-3)
+    value = world * w.M / (ms * 1e-3)
+
+    extras = []
+    if not args.no_extra and world == 1:
+        for name in EXTRA:
+            try:
+                r = measure_workload(I.WORKLOADS[name], max(5, min(args.steps, 30)), 3, dev, peaks,
+                                     want_e2e=False, sample_clocks=False)
+                r.pop("_inputs", None)
+                extras.append(r)
+            except Exception as exc:  # a failed extra must not hide the primary number
+                extras.append({"name": name, "error": repr(exc)})
+            torch.cuda.empty_cache()
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    inp = res.pop("_inputs")
+    rows = I.sample_rows(w, inp.outlier_rows)
+    if world == 1:
+        cpu_rate, cpu_rows, cpu_dt, cores = cpu_oracle_rate(inp, rows[: min(len(rows), 32)], args.cpu_seconds)
+        cpu = {"value": cpu_rate, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+               "sample": f"{cpu_rows} row evaluations of this workload ({min(len(rows), 32)} rows per pass, "
+                         f"repeated for {cpu_dt:.1f} s); fp64, OpenMP over rows"}
+    else:
+        cpu = None
+
+    line = {
+        "metric": "gated_mlp_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "M": w.M, "d_model": w.d_model, "d_ff": w.d_ff, "rmsnorm": w.rmsnorm,
+                   "schedule": res["variant"], "l2": res["l2"], "parallelism": f"dp{world} (rows sharded, no collective)"},
+        "tflops": world * w.flops / (ms * 1e-3) / 1e12,
+        "gbps_min_bytes": world * w.min_bytes / (ms * 1e-3) / 1e9,
+        "roofline_path": res["roofline_path"],
+        "roofline": res.get("roofline"),
+        "kernel_ms": res["kernel_ms"],
+        "cpu_baseline": cpu,
+        "e2e": {k: res["e2e"][k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step")},
+        "gpu_launches": res["launches"],
+        "clocks": res["clocks"],
+        "peaks": peaks,
+        "workloads": extras,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

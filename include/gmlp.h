@@ -21,7 +21,7 @@
  *   Y  [M, d_model]      row-major bf16
  * All pointers are DEVICE pointers unless a parameter says "host".  Every pointer must be
  * 16-byte aligned; d_model and d_ff must be positive multiples of 8; M >= 0 (M == 0 is a
- * successful no-op).  Y must not overlap any input.  Inputs are only read.
+ * successful no-op that looks at no pointer).  Y must not overlap any input.  Inputs are only read.
  *
  * Ownership: the caller owns every buffer.  The library allocates nothing per call when a
  * workspace is passed; with workspace == NULL it uses a library-owned buffer that grows on
@@ -53,7 +53,7 @@ typedef enum gmlp_status {
     GMLP_ERR_ARCH = -6,       /* no CUDA device, or the current device is not sm_100 */
     GMLP_ERR_LAUNCH = -7,     /* a CUDA runtime call failed (cudaGetLastError is left readable) */
     GMLP_ERR_TIMEOUT = -8,    /* a bounded device-side wait ran out (see gmlp_device_status) */
-    GMLP_ERR_UNSUPPORTED = -9 /* the forced variant cannot run this shape */
+    GMLP_ERR_UNSUPPORTED = -9 /* the forced variant cannot run this shape (SKINNY needs M <= 128) */
 } gmlp_status;
 
 enum {
@@ -65,8 +65,9 @@ enum {
 enum {
     GMLP_VARIANT_AUTO = 0,
     GMLP_VARIANT_SIMT = 1,   /* CUDA-core tiled GEMMs: any shape, slow; bring-up and cross-check */
-    GMLP_VARIANT_STREAM = 2, /* small M: weight-streaming split-K kernels (HBM-bound regime) */
-    GMLP_VARIANT_UMMA = 3    /* large M: tcgen05 tensor-core GEMMs fed by TMA, accumulators in TMEM */
+    GMLP_VARIANT_STREAM = 2, /* small M: weight-streaming split-K kernels on CUDA cores (HBM-bound regime) */
+    GMLP_VARIANT_UMMA = 3,   /* large M: tcgen05 tensor-core GEMMs fed by TMA, accumulators in TMEM */
+    GMLP_VARIANT_SKINNY = 4  /* M <= 128: operand-swapped tcgen05 GEMMs, stream-K over all SMs (HBM-bound regime) */
 };
 
 typedef struct gmlp_args {
@@ -115,7 +116,7 @@ int gmlp_forward_host(const gmlp_args* args, const void* X_host, void* Y_host);
  */
 uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant);
 
-/* The schedule AUTO resolves to for this shape (one of GMLP_VARIANT_SIMT/STREAM/UMMA). */
+/* The schedule AUTO resolves to for this shape (one of GMLP_VARIANT_SIMT/STREAM/UMMA/SKINNY). */
 int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);
 
 /*

@@ -12,6 +12,7 @@
 #include "simt_gemm.cuh"
 #include "stream_small_m.cuh"
 #include "umma_gemm.cuh"
+#include "umma_skinny.cuh"
 
 namespace {
 
@@ -60,6 +61,7 @@ struct DeviceState {
     void* workspace = nullptr;
     uint64_t workspace_bytes = 0;
     bool umma_attr_set = false;
+    bool skinny_attr_set = false;
 };
 std::mutex g_mutex;
 DeviceState g_dev[kMaxDevices];
@@ -139,16 +141,46 @@ StreamPlan make_stream_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
     return p;
 }
 
+// ------------------------------------------------------------------ skinny (swap-AB tcgen05) plan
+struct SkinnyPlan {
+    int Mpad, NH, num_tiles, KB, stages, grid;
+    uint32_t tmem_cols;
+    uint64_t scratch_bytes;
+};
+
+SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_count) {
+    SkinnyPlan p;
+    p.Mpad = (int)((M + 15) / 16 * 16);
+    if (p.Mpad < 16) p.Mpad = 16;
+    p.NH = (N >= 256 && 2 * nmat * 2 * p.Mpad <= 512) ? 2 : 1;
+    const int tile_n = 128 * p.NH;
+    p.num_tiles = (int)((N + tile_n - 1) / tile_n);
+    p.KB = (int)((K + 63) / 64);
+    const uint32_t stage_bytes = (uint32_t)nmat * p.NH * 2 * gmlp::kSkinnyBoxBytes + (uint32_t)p.Mpad * 128u;
+    int st = (int)((gmlp::kSkinnySmemBudget - 1024 - 256) / stage_bytes);
+    p.stages = st > gmlp::kSkinnyMaxStages ? gmlp::kSkinnyMaxStages : st;
+    uint32_t cols = (uint32_t)(2 * nmat * p.NH * p.Mpad);
+    uint32_t pow2 = 32;
+    while (pow2 < cols) pow2 <<= 1;
+    p.tmem_cols = pow2;
+    const int64_t total = (int64_t)p.num_tiles * p.KB;
+    const int sms = sm_count > 0 ? sm_count : 148;
+    p.grid = (int)(total < sms ? total : sms);
+    p.scratch_bytes = (uint64_t)p.grid * 2 * nmat * p.NH * p.Mpad * 128 * 4;
+    return p;
+}
+
 // ------------------------------------------------------------------ workspace layout
 struct Layout {
     uint64_t xn_off, h_off, partial_off, counters_off, total;
     uint64_t counters_bytes;
     StreamPlan p1, p2;
+    SkinnyPlan s1, s2;
 };
 
 int resolve_variant(int64_t M, int32_t variant) {
     if (variant != GMLP_VARIANT_AUTO) return variant;
-    return M <= 16 ? GMLP_VARIANT_STREAM : GMLP_VARIANT_UMMA;
+    return M <= 128 ? GMLP_VARIANT_SKINNY : GMLP_VARIANT_UMMA;
 }
 
 Layout make_layout(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int variant, int sm_count) {
@@ -168,6 +200,13 @@ Layout make_layout(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int
         off += align256(b1 > b2 ? b1 : b2);      // the two phases run one after the other and share it
         L.counters_off = off;
         L.counters_bytes = align256((uint64_t)(L.p1.row_tiles * L.p1.slabs + L.p2.row_tiles * L.p2.slabs) * 4);
+        off += L.counters_bytes;
+    } else if (variant == GMLP_VARIANT_SKINNY) {
+        L.s1 = make_skinny_plan(M, d_model, d_ff, 2, sm_count);
+        L.s2 = make_skinny_plan(M, d_ff, d_model, 1, sm_count);
+        off += align256(L.s1.scratch_bytes > L.s2.scratch_bytes ? L.s1.scratch_bytes : L.s2.scratch_bytes);
+        L.counters_off = off;
+        L.counters_bytes = align256((uint64_t)(L.s1.num_tiles + L.s2.num_tiles) * 4);
         off += L.counters_bytes;
     }
     L.total = off;
@@ -277,6 +316,52 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     return GMLP_OK;
 }
 
+template <bool GATEUP>
+int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf16* W0, const bf16* W1, float* scratch,
+                  unsigned int* counters, bf16* out, int64_t M, int64_t K, int64_t N, cudaStream_t st) {
+    if (p.stages < 2 || p.tmem_cols > 512) return GMLP_ERR_UNSUPPORTED;
+    CUtensorMap tmX, tmW0, tmW1;
+    if (!encode_2d(&tmX, X, (uint64_t)K, (uint64_t)M, 64, (uint32_t)p.Mpad)) return GMLP_ERR_LAUNCH;
+    if (!encode_2d(&tmW0, W0, (uint64_t)N, (uint64_t)K, 64, 64)) return GMLP_ERR_LAUNCH;
+    if (GATEUP) {
+        if (!encode_2d(&tmW1, W1, (uint64_t)N, (uint64_t)K, 64, 64)) return GMLP_ERR_LAUNCH;
+    } else {
+        tmW1 = tmW0;
+    }
+    if (!dev->skinny_attr_set) {
+        const int b = (int)gmlp::kSkinnySmemBudget;
+        if (cudaFuncSetAttribute(gmlp::skinny_gemm_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::skinny_gemm_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::skinny_gemm_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::skinny_gemm_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess)
+            return GMLP_ERR_LAUNCH;
+        dev->skinny_attr_set = true;
+    }
+    const unsigned grid = (unsigned)p.grid;
+    if (p.NH == 2)
+        gmlp::skinny_gemm_kernel<GATEUP, 2><<<grid, gmlp::kSkinnyThreads, gmlp::kSkinnySmemBudget, st>>>(
+            tmX, tmW0, tmW1, scratch, counters, out, (int)M, p.Mpad, (int)N, p.num_tiles, p.KB, p.stages, p.tmem_cols);
+    else
+        gmlp::skinny_gemm_kernel<GATEUP, 1><<<grid, gmlp::kSkinnyThreads, gmlp::kSkinnySmemBudget, st>>>(
+            tmX, tmW0, tmW1, scratch, counters, out, (int)M, p.Mpad, (int)N, p.num_tiles, p.KB, p.stages, p.tmem_cols);
+    GMLP_CHECK_LAUNCH();
+    return GMLP_OK;
+}
+
+int run_skinny(DeviceState* dev, const Layout& L, uint8_t* ws, const bf16* A, const bf16* Wg, const bf16* Wu,
+               const bf16* Wd, bf16* H, bf16* Y, int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st) {
+    float* scratch = reinterpret_cast<float*>(ws + L.partial_off);
+    unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
+    unsigned int* c2 = c1 + L.s1.num_tiles;
+    if (cudaMemsetAsync(c1, 0, L.counters_bytes, st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    int rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, H, M, d_model, d_ff, st);
+    if (rc != GMLP_OK) return rc;
+    prof_mark("gate_up", st);
+    rc = launch_skinny<false>(dev, L.s2, H, Wd, nullptr, scratch, c2, Y, M, d_ff, d_model, st);
+    if (rc == GMLP_OK) prof_mark("down", st);
+    return rc;
+}
+
 int read_device_status() {
     if (cudaDeviceSynchronize() != cudaSuccess) return GMLP_ERR_LAUNCH;
     int v = 0;
@@ -292,9 +377,10 @@ int forward_impl(const gmlp_args* a) {
     if (a == nullptr) return GMLP_ERR_NULL;
     if (a->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
     if (a->flags & ~kKnownFlags) return GMLP_ERR_FLAGS;
-    if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_UMMA) return GMLP_ERR_FLAGS;
+    if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_SKINNY) return GMLP_ERR_FLAGS;
     int rc = check_shape(a->M, a->d_model, a->d_ff);
     if (rc != GMLP_OK) return rc;
+    if (a->M == 0) return GMLP_OK;              // nothing to compute; pointers may be NULL
     if (!a->X || !a->Wg || !a->Wu || !a->Wd || !a->Y) return GMLP_ERR_NULL;
     if (!aligned16(a->X) || !aligned16(a->Wg) || !aligned16(a->Wu) || !aligned16(a->Wd) || !aligned16(a->Y) ||
         !aligned16(a->rms_gain))
@@ -304,9 +390,9 @@ int forward_impl(const gmlp_args* a) {
 
     DeviceState* dev = current_device(&rc);
     if (dev == nullptr) return rc;
-    if (a->M == 0) return GMLP_OK;
 
     const int variant = resolve_variant(a->M, a->variant);
+    if (variant == GMLP_VARIANT_SKINNY && a->M > 128) return GMLP_ERR_UNSUPPORTED;
     const Layout L = make_layout(a->M, a->d_model, a->d_ff, a->flags, variant, dev->sm_count);
 
     uint8_t* ws = static_cast<uint8_t*>(a->workspace);
@@ -356,6 +442,9 @@ int forward_impl(const gmlp_args* a) {
             break;
         case GMLP_VARIANT_STREAM:
             rc = run_stream(L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
+            break;
+        case GMLP_VARIANT_SKINNY:
+            rc = run_skinny(dev, L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
             break;
         default:
             rc = launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st);
@@ -410,8 +499,8 @@ int gmlp_forward_host(const gmlp_args* args, const void* X_host, void* Y_host) {
     if (args->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
     int rc = check_shape(args->M, args->d_model, args->d_ff);
     if (rc != GMLP_OK) return rc;
-    if (!args->X || !args->Y) return GMLP_ERR_NULL;
     if (args->M == 0) return gmlp_forward_ex(args);
+    if (!args->X || !args->Y) return GMLP_ERR_NULL;
     const size_t bytes = (size_t)args->M * (size_t)args->d_model * 2;
     cudaStream_t st = static_cast<cudaStream_t>(args->stream);
     if (cudaMemcpyAsync(const_cast<void*>(args->X), X_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
@@ -424,7 +513,7 @@ int gmlp_forward_host(const gmlp_args* args, const void* X_host, void* Y_host) {
 
 uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant) {
     if (check_shape(M, d_model, d_ff) != GMLP_OK) return 0;
-    if (variant < GMLP_VARIANT_AUTO || variant > GMLP_VARIANT_UMMA) return 0;
+    if (variant < GMLP_VARIANT_AUTO || variant > GMLP_VARIANT_SKINNY) return 0;
     int sm_count = 148;
     int dev = -1;
     if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) {

@@ -1,0 +1,291 @@
+// Small-M schedule on the tensor cores: operand-swapped ("swap-AB") tcgen05 GEMMs that
+// stream each weight matrix once from HBM.
+//
+// For M <= 128 tokens the Gated MLP is bound by reading the weights, and CUDA cores cannot
+// keep up with HBM beyond a few tokens.  Here the WEIGHT tile is the MMA's 128-row operand
+// and the tokens are its N dimension (16..128): D[n, m] = sum_k W[k, n] * X[m, k].  With
+// row-major [K, N] weights the weight tile is an MN-major A operand, which tcgen05 reads
+// directly from the TMA-swizzled tile, and X (row-major [M, K]) is a K-major B operand: no
+// transpose exists anywhere.  This is the B200 image of the paper's instruction fusion
+// transpose(nc_matmul(X^T, W)) -> nc_matmul(W, X^T) (Section 4.5).
+//
+// Work split ("stream-K"): the (column tile, 64-deep k-block) pairs form one flat sequence
+// that is cut into gridDim.x equal contiguous ranges, one per persistent CTA (one CTA per
+// SM), so every SM streams the same number of bytes.  A CTA that covers only part of a
+// column tile's K range writes its fp32 partial accumulators to scratch; the last CTA to
+// arrive on that tile (atomic ticket, nobody waits) adds the partials in fixed CTA order and
+// applies the epilogue.  SiLU is not linear, so it must come after this K reduction.
+//   GATEUP: two weight matrices share the X tile; epilogue H = bf16_rn(silu(g) * u)
+//   else  : one matrix; epilogue Y = bf16_rn(sum)
+// NH = number of 128-column halves per tile (2 -> 512-byte contiguous weight rows per stage).
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+#include "umma_gemm.cuh"
+
+namespace gmlp {
+
+constexpr int kSkinnyThreads = 192;
+constexpr int kSkinnyMaxStages = 8;
+constexpr uint32_t kSkinnyBoxBytes = 64 * 64 * 2;            // 64 k-rows x 128 B
+constexpr uint32_t kSkinnySmemBudget = 230400;               // dynamic shared memory requested
+
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Flat work sequence of `total` units cut into `parts` ranges: range c = [c*total/parts, (c+1)*total/parts).
+__device__ __forceinline__ long long range_start(long long c, long long total, long long parts) {
+    return (c * total) / parts;
+}
+__device__ __forceinline__ int range_owner(long long unit, long long total, long long parts) {
+    return (int)(((unit + 1) * parts - 1) / total);
+}
+
+template <bool GATEUP, int NH>
+__global__ void __launch_bounds__(kSkinnyThreads, 1)
+skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW0,
+                   const __grid_constant__ CUtensorMap tmW1, float* __restrict__ scratch,
+                   unsigned int* __restrict__ counters, bf16* __restrict__ out,
+                   int M, int Mpad, int N, int num_tiles, int KB, int stages, uint32_t tmem_cols)
+{
+    constexpr int KERNEL_ID = GATEUP ? 3 : 4;
+    constexpr int NMAT = GATEUP ? 2 : 1;
+    constexpr int TILE_N = 128 * NH;
+    constexpr uint32_t W_BYTES = NMAT * NH * 2 * kSkinnyBoxBytes;     // weight bytes per stage
+    const uint32_t x_bytes = (uint32_t)Mpad * 128u;
+    const uint32_t stage_bytes = W_BYTES + x_bytes;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - raw_addr);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + (size_t)stages * stage_bytes);
+    const uint32_t full0 = ptx::smem_addr(bars);
+    const uint32_t empty0 = ptx::smem_addr(bars + kSkinnyMaxStages);
+    const uint32_t tfull0 = ptx::smem_addr(bars + 2 * kSkinnyMaxStages);
+    const uint32_t tempty0 = ptx::smem_addr(bars + 2 * kSkinnyMaxStages + 2);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kSkinnyMaxStages + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long total = (long long)num_tiles * KB;
+    const long long parts = gridDim.x;
+    const long long u_begin = range_start(blockIdx.x, total, parts);
+    const long long u_end = range_start(blockIdx.x + 1, total, parts);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            ptx::mbar_init(full0 + 8 * s, 1);
+            ptx::mbar_init(empty0 + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(tfull0 + 8 * b, 1);
+            ptx::mbar_init(tempty0 + 8 * b, 4);          // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        *last_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::fence_proxy_async_smem();
+        ptx::prefetch_tensormap(&tmX);
+        ptx::prefetch_tensormap(&tmW0);
+        if (GATEUP) ptx::prefetch_tensormap(&tmW1);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_addr(tmem_slot), tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    // TMEM column of accumulator (buffer b, matrix j, half h): Mpad fp32 columns each
+    auto acc_col = [&](int b, int j, int h) -> uint32_t { return (uint32_t)(((b * NMAT + j) * NH + h) * Mpad); };
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            int it = 0;
+            for (long long u = u_begin; u < u_end; ++u, ++it) {
+                const int s = it % stages;
+                const uint32_t ph = (uint32_t)(it / stages) & 1u;
+                const int tile = (int)(u / KB), kb = (int)(u % KB);
+                if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
+                const uint32_t full = full0 + 8 * s;
+                const uint32_t st = base + s * stage_bytes;
+                ptx::mbar_arrive_expect_tx(full, stage_bytes);
+                ptx::tma_load_2d(st + W_BYTES, &tmX, kb * 64, 0, full);
+#pragma unroll
+                for (int j = 0; j < NMAT; ++j)
+#pragma unroll
+                    for (int hb = 0; hb < NH * 2; ++hb)
+                        ptx::tma_load_2d(st + (j * NH * 2 + hb) * kSkinnyBoxBytes, j ? &tmW1 : &tmW0,
+                                         tile * TILE_N + hb * 64, kb * 64, full);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            // D = fp32, A = B = bf16, A (weights) MN-major, B (tokens) K-major, M = 128, N = Mpad
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (0u << 16) |
+                                   ((uint32_t)(Mpad >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+            int it = 0, seg = 0;
+            bool fresh = true;
+            for (long long u = u_begin; u < u_end; ++u, ++it) {
+                const int s = it % stages;
+                const uint32_t ph = (uint32_t)(it / stages) & 1u;
+                const int kb = (int)(u % KB);
+                const int buf = seg & 1;
+                if (fresh) {
+                    // the accumulator buffer must have been drained by the epilogue two segments ago
+                    if (!wait_bounded(tempty0 + 8 * buf, (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4)) break;
+                    ptx::tc_fence_after_sync();
+                }
+                if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t st = base + s * stage_bytes;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint64_t b_desc = ptx::make_smem_desc_sw128(st + W_BYTES + k * 32, 16, 1024);
+#pragma unroll
+                    for (int j = 0; j < NMAT; ++j)
+#pragma unroll
+                        for (int h = 0; h < NH; ++h) {
+                            const uint64_t a_desc = ptx::make_smem_desc_sw128(
+                                st + (j * NH + h) * 2 * kSkinnyBoxBytes + k * 2048, kSkinnyBoxBytes, 1024);
+                            ptx::umma_bf16(tmem_base + acc_col(buf, j, h), a_desc, b_desc, idesc,
+                                           (fresh && k == 0) ? 0u : 1u);
+                        }
+                }
+                fresh = false;
+                ptx::umma_commit(empty0 + 8 * s);
+                if (kb == KB - 1 || u == u_end - 1) {
+                    ptx::umma_commit(tfull0 + 8 * buf);
+                    ++seg;
+                    fresh = true;
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue (128 threads: one weight column each) ----------------
+        const int q = warp & 3;
+        const int nl = q * 32 + lane;                       // column within a 128-column half = TMEM lane
+        const int et = threadIdx.x - 64;
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        const size_t slot_floats = (size_t)NMAT * NH * Mpad * 128;
+        int seg = 0;
+        bool ok = true;
+        for (long long u = u_begin; u < u_end && ok; ++seg) {
+            const int tile = (int)(u / KB);
+            const long long tile_first = (long long)tile * KB;
+            const long long seg_end = (tile_first + KB < u_end) ? tile_first + KB : u_end;
+            const int buf = seg & 1;
+            ok = wait_bounded(tfull0 + 8 * buf, ((uint32_t)seg >> 1) & 1u, abort_flag, KERNEL_ID, 3);
+            ptx::tc_fence_after_sync();
+            if (!ok) break;
+            const int first_c = range_owner(tile_first, total, parts);
+            const int last_c = range_owner(tile_first + KB - 1, total, parts);
+            const int n_base = tile * TILE_N;
+
+            if (first_c == last_c) {
+                // this CTA owns the whole K range of the tile: epilogue straight from TMEM
+#pragma unroll
+                for (int h = 0; h < NH; ++h) {
+                    const int n = n_base + h * 128 + nl;
+                    for (int c0 = 0; c0 < Mpad; c0 += 16) {
+                        uint32_t g[16], uu[16];
+                        tmem_ld_32x16(tmem_base + lane_base + acc_col(buf, 0, h) + c0, g);
+                        if (GATEUP) tmem_ld_32x16(tmem_base + lane_base + acc_col(buf, 1, h) + c0, uu);
+                        ptx::tmem_ld_wait();
+                        if (n < N) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const int m = c0 + i;
+                                if (m < M) {
+                                    const float v = GATEUP ? silu_f32(__uint_as_float(g[i])) * __uint_as_float(uu[i])
+                                                           : __uint_as_float(g[i]);
+                                    out[(size_t)m * N + n] = __float2bfloat16_rn(v);
+                                }
+                            }
+                        }
+                    }
+                }
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(tempty0 + 8 * buf);
+            } else {
+                // partial K range: park the fp32 accumulators in this CTA's scratch slot
+                const int slot = (tile == (int)(u_begin / KB)) ? 0 : 1;
+                float* mine = scratch + ((size_t)blockIdx.x * 2 + slot) * slot_floats;
+#pragma unroll
+                for (int j = 0; j < NMAT; ++j)
+#pragma unroll
+                    for (int h = 0; h < NH; ++h)
+                        for (int c0 = 0; c0 < Mpad; c0 += 16) {
+                            uint32_t v[16];
+                            tmem_ld_32x16(tmem_base + lane_base + acc_col(buf, j, h) + c0, v);
+                            ptx::tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i)
+                                __stcg(mine + ((size_t)(j * NH + h) * Mpad + c0 + i) * 128 + nl, __uint_as_float(v[i]));
+                        }
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(tempty0 + 8 * buf);
+                __threadfence();
+                epi_bar_sync();
+                if (et == 0) {
+                    const unsigned int ticket = atomicAdd(counters + tile, 1u);
+                    *last_flag = (ticket == (unsigned int)(last_c - first_c)) ? 1 : 0;
+                }
+                epi_bar_sync();
+                const bool is_last = (*last_flag != 0);
+                if (is_last) {
+                    __threadfence();
+#pragma unroll
+                    for (int h = 0; h < NH; ++h) {
+                        const int n = n_base + h * 128 + nl;
+                        if (n >= N) continue;
+                        for (int m = 0; m < M; ++m) {
+                            float g = 0.0f, uu = 0.0f;
+                            for (int c = first_c; c <= last_c; ++c) {
+                                const int cslot = ((int)(range_start(c, total, parts) / KB) == tile) ? 0 : 1;
+                                const float* p = scratch + ((size_t)c * 2 + cslot) * slot_floats;
+                                g += __ldcg(p + ((size_t)(0 * NH + h) * Mpad + m) * 128 + nl);
+                                if (GATEUP) uu += __ldcg(p + ((size_t)(1 * NH + h) * Mpad + m) * 128 + nl);
+                            }
+                            const float v = GATEUP ? silu_f32(g) * uu : g;
+                            out[(size_t)m * N + n] = __float2bfloat16_rn(v);
+                        }
+                    }
+                    if (et == 0) counters[tile] = 0u;        // clean for the next call
+                }
+            }
+            u = seg_end;
+        }
+    }
+
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+}  // namespace gmlp

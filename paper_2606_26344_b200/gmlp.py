@@ -17,7 +17,7 @@ ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_FLAGS, ERR_WORKSPACE, ERR_ARCH, ERR_LAUNCH, 
     -1, -2, -3, -4, -5, -6, -7, -8, -9
 FLAG_RMSNORM = 1 << 0
 FLAG_CHECKED = 1 << 2
-VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA = 0, 1, 2, 3
+VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA, VARIANT_SKINNY = 0, 1, 2, 3, 4
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgmlp.so")
 _lib = None

@@ -62,6 +62,7 @@ def test_argument_validation_happens_before_device_work(lib):
     assert f(_args(struct_bytes=8)) == gmlp.ERR_FLAGS
     assert f(_args(flags=1 << 7)) == gmlp.ERR_FLAGS
     assert f(_args(variant=17)) == gmlp.ERR_FLAGS
+    assert f(_args(variant=-1)) == gmlp.ERR_FLAGS
     assert f(_args(M=-1)) == gmlp.ERR_SHAPE
     assert f(_args(d_model=60)) == gmlp.ERR_SHAPE
     assert f(_args(d_ff=0)) == gmlp.ERR_SHAPE
@@ -93,8 +94,10 @@ def test_workspace_sizes_and_variant_choice(lib):
     assert wb(M, dm, dff, 0, gmlp.VARIANT_UMMA) < h + 4096
     assert wb(8, dm, dff, 0, gmlp.VARIANT_STREAM) > wb(8, dm, dff, 0, gmlp.VARIANT_SIMT)     # split-K partials
     assert wb(8, dm, dff, 0, gmlp.VARIANT_STREAM) < 64 << 20
-    assert gmlp.pick_variant(8, dm, dff) == gmlp.VARIANT_STREAM
-    assert gmlp.pick_variant(1, 2048, 5632) == gmlp.VARIANT_STREAM
+    assert gmlp.pick_variant(8, dm, dff) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(1, 2048, 5632) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(128, 2048, 5632) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(129, 2048, 5632) == gmlp.VARIANT_UMMA
     assert gmlp.pick_variant(2048, dm, dff) == gmlp.VARIANT_UMMA
     assert gmlp.pick_variant(4096, 8192, 28672) == gmlp.VARIANT_UMMA
     assert gmlp.pick_variant(4, 60, 128) == gmlp.ERR_SHAPE
