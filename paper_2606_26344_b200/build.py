@@ -42,4 +42,5 @@ def build_libgmlp(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build_libgmlp(force=True, verbose=True))
+    import sys
+    print(build_libgmlp(force=True, verbose="-v" in sys.argv))

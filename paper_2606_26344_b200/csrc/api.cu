@@ -62,6 +62,9 @@ struct DeviceState {
     uint64_t workspace_bytes = 0;
     bool umma_attr_set = false;
     bool skinny_attr_set = false;
+    // arrival counters last zeroed by the library (the kernels leave them zero after every call)
+    const void* clean_counters = nullptr;
+    uint64_t clean_counters_bytes = 0;
 };
 std::mutex g_mutex;
 DeviceState g_dev[kMaxDevices];
@@ -232,6 +235,23 @@ bool encode_2d(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The split-K kernels leave their arrival counters at zero when they finish, so the counters only
+// need clearing the first time a given counter region is used (or after a failed call).
+int ensure_counters_zero(DeviceState* dev, void* ptr, uint64_t bytes, cudaStream_t st) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (dev->clean_counters == ptr && dev->clean_counters_bytes == bytes) return GMLP_OK;
+    if (cudaMemsetAsync(ptr, 0, bytes, st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    dev->clean_counters = ptr;
+    dev->clean_counters_bytes = bytes;
+    return GMLP_OK;
+}
+
+void forget_counters(DeviceState* dev) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    dev->clean_counters = nullptr;
+    dev->clean_counters_bytes = 0;
+}
+
 // ------------------------------------------------------------------ launches
 #define GMLP_CHECK_LAUNCH()                                   \
     do {                                                      \
@@ -274,13 +294,14 @@ int launch_stream(const StreamPlan& p, const bf16* A, const bf16* W0, const bf16
     return GMLP_OK;
 }
 
-int run_stream(const Layout& L, uint8_t* ws, const bf16* A, const bf16* Wg, const bf16* Wu, const bf16* Wd, bf16* H,
+int run_stream(DeviceState* dev, const Layout& L, uint8_t* ws, const bf16* A, const bf16* Wg, const bf16* Wu, const bf16* Wd, bf16* H,
                bf16* Y, int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st) {
     float* partial = reinterpret_cast<float*>(ws + L.partial_off);
     unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
     unsigned int* c2 = c1 + L.p1.row_tiles * L.p1.slabs;
-    if (cudaMemsetAsync(c1, 0, L.counters_bytes, st) != cudaSuccess) return GMLP_ERR_LAUNCH;
-    int rc = launch_stream<true>(L.p1, A, Wg, Wu, partial, c1, H, M, d_model, d_ff, st);
+    int rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
+    if (rc != GMLP_OK) return rc;
+    rc = launch_stream<true>(L.p1, A, Wg, Wu, partial, c1, H, M, d_model, d_ff, st);
     if (rc != GMLP_OK) return rc;
     prof_mark("gate_up", st);
     rc = launch_stream<false>(L.p2, H, Wd, nullptr, partial, c2, Y, M, d_ff, d_model, st);
@@ -337,13 +358,27 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
             return GMLP_ERR_LAUNCH;
         dev->skinny_attr_set = true;
     }
-    const unsigned grid = (unsigned)p.grid;
+    // programmatic stream serialization: this kernel may become resident while the previous kernel on
+    // the stream drains; it orders itself with griddepcontrol.wait
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.grid);
+    cfg.blockDim = dim3(gmlp::kSkinnyThreads);
+    cfg.dynamicSmemBytes = gmlp::kSkinnySmemBudget;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int Mi = (int)M, Ni = (int)N;
+    cudaError_t err;
     if (p.NH == 2)
-        gmlp::skinny_gemm_kernel<GATEUP, 2><<<grid, gmlp::kSkinnyThreads, gmlp::kSkinnySmemBudget, st>>>(
-            tmX, tmW0, tmW1, scratch, counters, out, (int)M, p.Mpad, (int)N, p.num_tiles, p.KB, p.stages, p.tmem_cols);
+        err = cudaLaunchKernelEx(&cfg, gmlp::skinny_gemm_kernel<GATEUP, 2>, tmX, tmW0, tmW1, scratch, counters, out,
+                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols);
     else
-        gmlp::skinny_gemm_kernel<GATEUP, 1><<<grid, gmlp::kSkinnyThreads, gmlp::kSkinnySmemBudget, st>>>(
-            tmX, tmW0, tmW1, scratch, counters, out, (int)M, p.Mpad, (int)N, p.num_tiles, p.KB, p.stages, p.tmem_cols);
+        err = cudaLaunchKernelEx(&cfg, gmlp::skinny_gemm_kernel<GATEUP, 1>, tmX, tmW0, tmW1, scratch, counters, out,
+                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols);
+    if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
 }
@@ -353,8 +388,9 @@ int run_skinny(DeviceState* dev, const Layout& L, uint8_t* ws, const bf16* A, co
     float* scratch = reinterpret_cast<float*>(ws + L.partial_off);
     unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
     unsigned int* c2 = c1 + L.s1.num_tiles;
-    if (cudaMemsetAsync(c1, 0, L.counters_bytes, st) != cudaSuccess) return GMLP_ERR_LAUNCH;
-    int rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, H, M, d_model, d_ff, st);
+    int rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
+    if (rc != GMLP_OK) return rc;
+    rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, H, M, d_model, d_ff, st);
     if (rc != GMLP_OK) return rc;
     prof_mark("gate_up", st);
     rc = launch_skinny<false>(dev, L.s2, H, Wd, nullptr, scratch, c2, Y, M, d_ff, d_model, st);
@@ -404,6 +440,8 @@ int forward_impl(const gmlp_args* a) {
                 if (cudaDeviceSynchronize() != cudaSuccess || cudaFree(dev->workspace) != cudaSuccess) return GMLP_ERR_LAUNCH;
                 dev->workspace = nullptr;
                 dev->workspace_bytes = 0;
+                dev->clean_counters = nullptr;
+                dev->clean_counters_bytes = 0;
             }
             void* p = nullptr;
             if (cudaMalloc(&p, L.total) != cudaSuccess) {
@@ -441,7 +479,7 @@ int forward_impl(const gmlp_args* a) {
             rc = run_simt(A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
             break;
         case GMLP_VARIANT_STREAM:
-            rc = run_stream(L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
+            rc = run_stream(dev, L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
             break;
         case GMLP_VARIANT_SKINNY:
             rc = run_skinny(dev, L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
@@ -455,11 +493,15 @@ int forward_impl(const gmlp_args* a) {
             }
             break;
     }
-    if (rc != GMLP_OK) return rc;
+    if (rc != GMLP_OK) {
+        forget_counters(dev);
+        return rc;
+    }
 
     if (a->flags & GMLP_FLAG_CHECKED) {
-        if (cudaStreamSynchronize(st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+        if (cudaStreamSynchronize(st) != cudaSuccess) { forget_counters(dev); return GMLP_ERR_LAUNCH; }
         const int s = read_device_status();
+        if (s != 0) forget_counters(dev);
         if (s < 0) return s;
         if (s != 0) return GMLP_ERR_TIMEOUT;
     }
@@ -533,8 +575,11 @@ int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags) 
 
 int gmlp_device_status(void) {
     int rc = GMLP_OK;
-    if (current_device(&rc) == nullptr) return rc;
-    return read_device_status();
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    const int s = read_device_status();
+    if (s != 0) forget_counters(dev);
+    return s;
 }
 
 int gmlp_profile_enable(int on) {

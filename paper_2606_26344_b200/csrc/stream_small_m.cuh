@@ -111,21 +111,32 @@ stream_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W0, cons
     if (!is_last) return;
     __threadfence();
     if (nc < N) {
-        for (int m = 0; m < rows; ++m) {
-            float g0 = 0.0f, g1 = 0.0f, u0 = 0.0f, u1 = 0.0f;
-            for (int s = 0; s < KS; ++s) {
-                const float2 pg = __ldcg(reinterpret_cast<const float2*>(
-                    partial + ((size_t)s * M + (m0 + m)) * N + nc));
-                g0 += pg.x; g1 += pg.y;
-                if (GATEUP) {
-                    const float2 pu = __ldcg(reinterpret_cast<const float2*>(
-                        partial + ((size_t)(KS + s) * M + (m0 + m)) * N + nc));
-                    u0 += pu.x; u1 += pu.y;
+        // K-chunks are added in ascending order; the MT rows are independent, so each chunk's loads overlap
+        float2 g[MT], u[MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) { g[m] = make_float2(0.0f, 0.0f); u[m] = make_float2(0.0f, 0.0f); }
+        for (int s = 0; s < KS; ++s) {
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                if (m < rows) {
+                    const float2 pg = __ldcg(reinterpret_cast<const float2*>(
+                        partial + ((size_t)s * M + (m0 + m)) * N + nc));
+                    g[m].x += pg.x; g[m].y += pg.y;
+                    if (GATEUP) {
+                        const float2 pu = __ldcg(reinterpret_cast<const float2*>(
+                            partial + ((size_t)(KS + s) * M + (m0 + m)) * N + nc));
+                        u[m].x += pu.x; u[m].y += pu.y;
+                    }
                 }
             }
-            const float o0 = GATEUP ? silu_f32(g0) * u0 : g0;
-            const float o1 = GATEUP ? silu_f32(g1) * u1 : g1;
-            *reinterpret_cast<uint32_t*>(out + (size_t)(m0 + m) * N + nc) = pack_bf16x2(o0, o1);
+        }
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            if (m < rows) {
+                const float o0 = GATEUP ? silu_f32(g[m].x) * u[m].x : g[m].x;
+                const float o1 = GATEUP ? silu_f32(g[m].y) * u[m].y : g[m].y;
+                *reinterpret_cast<uint32_t*>(out + (size_t)(m0 + m) * N + nc) = pack_bf16x2(o0, o1);
+            }
         }
     }
     if (tid == 0) *counter = 0u;     // leave the counter clean for the next call

@@ -18,6 +18,12 @@
 //   GATEUP: two weight matrices share the X tile; epilogue H = bf16_rn(silu(g) * u)
 //   else  : one matrix; epilogue Y = bf16_rn(sum)
 // NH = number of 128-column halves per tile (2 -> 512-byte contiguous weight rows per stage).
+//
+// Overlap between the two phases (and between calls): the kernels are launched with
+// programmatic stream serialization.  Weight tiles do not depend on the previous kernel, so the
+// producer fills its whole shared-memory ring with weights BEFORE griddepcontrol.wait and only
+// then loads the token tile (X, or the H written by the previous kernel); every other access
+// to global memory comes after the wait.
 #pragma once
 #include <cuda.h>
 
@@ -30,7 +36,8 @@ namespace gmlp {
 constexpr int kSkinnyThreads = 192;
 constexpr int kSkinnyMaxStages = 8;
 constexpr uint32_t kSkinnyBoxBytes = 64 * 64 * 2;            // 64 k-rows x 128 B
-constexpr uint32_t kSkinnySmemBudget = 230400;               // dynamic shared memory requested
+constexpr uint32_t kSkinnySmemBudget = 229376;               // dynamic shared memory requested (224 KB)
+constexpr int kSkinnyMaxContrib = 256;                       // CTAs that can share one column tile (>= grid size)
 
 __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile(
@@ -66,6 +73,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     const uint32_t stage_bytes = W_BYTES + x_bytes;
 
     extern __shared__ uint8_t smem_raw[];
+    __shared__ unsigned long long slot_off[kSkinnyMaxContrib];     // scratch offsets of a tile's contributors
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - raw_addr);
@@ -84,6 +92,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     const long long u_begin = range_start(blockIdx.x, total, parts);
     const long long u_end = range_start(blockIdx.x + 1, total, parts);
 
+    ptx::launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             ptx::mbar_init(full0 + 8 * s, 1);
@@ -115,22 +124,34 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            int it = 0;
-            for (long long u = u_begin; u < u_end; ++u, ++it) {
-                const int s = it % stages;
-                const uint32_t ph = (uint32_t)(it / stages) & 1u;
+            auto load_weights = [&](long long u, int s) {
                 const int tile = (int)(u / KB), kb = (int)(u % KB);
-                if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
                 const uint32_t full = full0 + 8 * s;
                 const uint32_t st = base + s * stage_bytes;
                 ptx::mbar_arrive_expect_tx(full, stage_bytes);
-                ptx::tma_load_2d(st + W_BYTES, &tmX, kb * 64, 0, full);
 #pragma unroll
                 for (int j = 0; j < NMAT; ++j)
 #pragma unroll
                     for (int hb = 0; hb < NH * 2; ++hb)
                         ptx::tma_load_2d(st + (j * NH * 2 + hb) * kSkinnyBoxBytes, j ? &tmW1 : &tmW0,
                                          tile * TILE_N + hb * 64, kb * 64, full);
+            };
+            auto load_tokens = [&](long long u, int s) {
+                ptx::tma_load_2d(base + s * stage_bytes + W_BYTES, &tmX, (int)(u % KB) * 64, 0, full0 + 8 * s);
+            };
+            // weights of the first ring-full of units do not depend on the previous kernel
+            const long long n_units = u_end - u_begin;
+            const int head = (int)(n_units < stages ? n_units : stages);
+            for (int i = 0; i < head; ++i) load_weights(u_begin + i, i);
+            ptx::grid_dependency_wait();
+            for (int i = 0; i < head; ++i) load_tokens(u_begin + i, i);
+            int it = head;
+            for (long long u = u_begin + head; u < u_end; ++u, ++it) {
+                const int s = it % stages;
+                const uint32_t ph = (uint32_t)(it / stages) & 1u;
+                if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
+                load_weights(u, s);
+                load_tokens(u, s);
             }
         }
         __syncwarp();
@@ -187,6 +208,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         const size_t slot_floats = (size_t)NMAT * NH * Mpad * 128;
         int seg = 0;
         bool ok = true;
+        ptx::grid_dependency_wait();          // scratch, counters and `out` may still be in use by the previous kernel
         for (long long u = u_begin; u < u_end && ok; ++seg) {
             const int tile = (int)(u / KB);
             const long long tile_first = (long long)tile * KB;
@@ -254,20 +276,51 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 const bool is_last = (*last_flag != 0);
                 if (is_last) {
                     __threadfence();
+                    // Sum the contributors' partials in CTA order.  Thread mapping: 32 column groups of 4
+                    // columns x 4 row groups; float4 loads, contributors fetched four at a time so that
+                    // many loads are in flight while the additions keep their fixed order.
+                    const int ncontrib = last_c - first_c + 1;
+                    for (int i = et; i < ncontrib; i += 128) {
+                        const int c = first_c + i;
+                        const int cslot = ((int)(range_start(c, total, parts) / KB) == tile) ? 0 : 1;
+                        slot_off[i] = ((unsigned long long)c * 2 + cslot) * slot_floats;
+                    }
+                    epi_bar_sync();
+                    const int cg = et & 31, rg = et >> 5;
+                    auto add4 = [](float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; };
 #pragma unroll
                     for (int h = 0; h < NH; ++h) {
-                        const int n = n_base + h * 128 + nl;
+                        const int n = n_base + h * 128 + cg * 4;
                         if (n >= N) continue;
-                        for (int m = 0; m < M; ++m) {
-                            float g = 0.0f, uu = 0.0f;
-                            for (int c = first_c; c <= last_c; ++c) {
-                                const int cslot = ((int)(range_start(c, total, parts) / KB) == tile) ? 0 : 1;
-                                const float* p = scratch + ((size_t)c * 2 + cslot) * slot_floats;
-                                g += __ldcg(p + ((size_t)(0 * NH + h) * Mpad + m) * 128 + nl);
-                                if (GATEUP) uu += __ldcg(p + ((size_t)(1 * NH + h) * Mpad + m) * 128 + nl);
+                        for (int m = rg; m < M; m += 4) {
+                            const size_t og = ((size_t)h * Mpad + m) * 128 + cg * 4;
+                            const size_t ou = og + (size_t)NH * Mpad * 128;
+                            float4 g = make_float4(0.f, 0.f, 0.f, 0.f), uu = g;
+                            int i = 0;
+                            for (; i + 4 <= ncontrib; i += 4) {
+                                float4 a[4], b[4];
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) {
+                                    const float* p = scratch + slot_off[i + t];
+                                    a[t] = __ldcg(reinterpret_cast<const float4*>(p + og));
+                                    if (GATEUP) b[t] = __ldcg(reinterpret_cast<const float4*>(p + ou));
+                                }
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) { add4(g, a[t]); if (GATEUP) add4(uu, b[t]); }
                             }
-                            const float v = GATEUP ? silu_f32(g) * uu : g;
-                            out[(size_t)m * N + n] = __float2bfloat16_rn(v);
+                            for (; i < ncontrib; ++i) {
+                                const float* p = scratch + slot_off[i];
+                                add4(g, __ldcg(reinterpret_cast<const float4*>(p + og)));
+                                if (GATEUP) add4(uu, __ldcg(reinterpret_cast<const float4*>(p + ou)));
+                            }
+                            float v[4] = {g.x, g.y, g.z, g.w};
+                            if (GATEUP) {
+                                v[0] = silu_f32(g.x) * uu.x; v[1] = silu_f32(g.y) * uu.y;
+                                v[2] = silu_f32(g.z) * uu.z; v[3] = silu_f32(g.w) * uu.w;
+                            }
+                            // N is a multiple of 8 and n of 4: the four columns are all inside or all outside
+                            *reinterpret_cast<uint2*>(out + (size_t)m * N + n) =
+                                make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
                         }
                     }
                     if (et == 0) counters[tile] = 0u;        // clean for the next call
