@@ -147,7 +147,7 @@ def run_reference(args):
     }))
 
 
-def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sample_clocks=True):
+def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sample_clocks=True, clock_roll=0.6):
     """Times one workload on this rank's GPU.  Returns a dict of measurements."""
     import torch
     from paper_2606_26344_b200 import gmlp, inputs as I
@@ -179,7 +179,7 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
     # The timed region of a small workload lasts a few milliseconds, shorter than nvidia-smi's sampling
     # period.  The clocks are therefore sampled over an untimed pre-roll of the same steps, the timed
     # region and an untimed post-roll: one continuous stretch of identical load.
-    sampler = ClockSampler(dev.index or 0) if sample_clocks else None
+    sampler = ClockSampler(dev.index or 0) if (sample_clocks and clock_roll > 0) else None
 
     def roll(seconds):
         t_end = time.perf_counter() + seconds
@@ -190,7 +190,7 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
 
     if sampler:
         sampler.start()
-        roll(0.6)
+        roll(clock_roll)
     gmlp.reset_launch_count()
     if not fits_l2:
         # inputs are larger than L2: back-to-back steps, one pair of events around the region
@@ -219,24 +219,30 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
         total_ms = sum(per_step)
     launches = gmlp.launch_count()
     if sampler:
-        roll(0.6)
+        roll(clock_roll)
     clocks = sampler.stop() if sampler else None
     if clocks is not None:
-        clocks["window"] = "pre-roll 0.6 s + timed region + post-roll 0.6 s of the same steps"
+        clocks["window"] = f"pre-roll {clock_roll} s + timed region + post-roll {clock_roll} s of the same steps"
     ms = total_ms / steps
 
-    # per-kernel durations, in a loop of their own (events between kernels perturb the launch stream)
+    # per-kernel durations, in a loop of their own (an event between two kernels stops the second from
+    # overlapping the first's tail, so these are stand-alone kernel times, like a profiler's)
     gmlp.profile_enable(True)
-    kern = {}
-    n_prof = max(3, min(steps, 20))
-    for _ in range(n_prof):
-        if flush is not None:
+    n_prof = max(3, min(steps, 50))
+    if flush is None:
+        for _ in range(n_prof):
+            gmlp.forward_ex(a)
+        kern_ms = gmlp.profile_read()
+    else:
+        acc = {}
+        for _ in range(n_prof):
+            gmlp.profile_enable(True)
             flush.fill_(1)
-        gmlp.forward_ex(a)
-        for k, v in gmlp.profile_read().items():
-            kern.setdefault(k, []).append(v)
+            gmlp.forward_ex(a)
+            for k, v in gmlp.profile_read().items():
+                acc.setdefault(k, []).append(v)
+        kern_ms = {k: sum(v) / len(v) for k, v in acc.items()}
     gmlp.profile_enable(False)
-    kern_ms = {k: sum(v) / len(v) for k, v in kern.items()}
 
     res = {"name": w.name, "M": w.M, "d_model": w.d_model, "d_ff": w.d_ff, "rmsnorm": w.rmsnorm,
            "variant": {1: "simt", 2: "stream", 3: "umma", 4: "skinny"}[variant], "ms_per_step": ms,
@@ -294,7 +300,10 @@ def main():
     ap.add_argument("--impl", default="gmlp", choices=["gmlp", "reference"])
     ap.add_argument("--workload", default=PRIMARY)
     ap.add_argument("--no-extra", action="store_true", help="time only the primary workload")
-    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time spent on the oracle baseline")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time spent on the oracle baseline (0 = skip)")
+    ap.add_argument("--clock-roll", type=float, default=0.6,
+                    help="seconds of untimed identical steps before and after the timed region while clocks are "
+                         "sampled (0 = no clock sampling; for runs under a profiler)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -325,7 +334,7 @@ def main():
     warmup = max(args.warmup, 3)
 
     w = I.WORKLOADS[args.workload]
-    res = measure_workload(w, args.steps, warmup, dev, peaks, dist=dist)
+    res = measure_workload(w, args.steps, warmup, dev, peaks, dist=dist, clock_roll=args.clock_roll)
     ms = res["ms_per_step"]
     if dist is not None:
         t = torch.tensor([ms], device=dev, dtype=torch.float64)
@@ -357,7 +366,7 @@ def main():
 
     inp = res.pop("_inputs")
     rows = I.sample_rows(w, inp.outlier_rows)
-    if world == 1:
+    if world == 1 and args.cpu_seconds > 0:
         cpu_rate, cpu_rows, cpu_dt, cores = cpu_oracle_rate(inp, rows[: min(len(rows), 32)], args.cpu_seconds)
         cpu = {"value": cpu_rate, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                "sample": f"{cpu_rows} row evaluations of this workload ({min(len(rows), 32)} rows per pass, "

@@ -133,11 +133,13 @@ void gmlp_reset_launch_count(void);
 /*
  * Per-kernel timing for benchmarks (per host thread, off by default).  While enabled, every
  * gmlp_forward_ex call records a CUDA event on its stream before its first kernel and after
- * each kernel.  gmlp_profile_read synchronises on the last event of the most recent call and
- * writes the duration of each of its kernels, in launch order, in milliseconds; *count gets
- * their number (at most max_count are written).  gmlp_profile_kernel_name(i) names the i-th
- * kernel of that call ("rmsnorm", "gate_up", "down").  Events add launch overhead: do not
- * leave this on in a timed region.
+ * each kernel; the library keeps the events of the 64 most recent calls, so calls can be
+ * enqueued back to back.  gmlp_profile_read synchronises on those events and writes the
+ * AVERAGE duration of each kernel over the recorded calls, in launch order, in milliseconds;
+ * *count gets the number of kernels (at most max_count are written).
+ * gmlp_profile_kernel_name(i) names the i-th kernel ("rmsnorm", "gate_up", "down").  An event
+ * between two kernels keeps the second from overlapping the first's tail, so these are
+ * stand-alone kernel durations; do not leave profiling on in a timed region.
  */
 int gmlp_profile_enable(int on);
 int gmlp_profile_read(float* ms, int max_count, int* count);

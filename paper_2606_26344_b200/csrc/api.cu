@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstdlib>
 #include <mutex>
 #include <new>
 
@@ -27,31 +28,43 @@ thread_local cudaStream_t t_stream = nullptr;
 thread_local float t_default_eps = 1e-5f;
 thread_local uint64_t t_launches = 0;
 
-// Optional per-kernel event timing of the most recent call (benchmarks only).
+// Optional per-kernel event timing (benchmarks only): a ring of the most recent calls, so that a
+// benchmark can enqueue many calls back to back and read the averages afterwards.
 constexpr int kMaxProfKernels = 4;
+constexpr int kProfRing = 64;
+struct ProfCall {
+    cudaEvent_t ev[kMaxProfKernels + 1] = {};
+    int n = 0;
+    const char* names[kMaxProfKernels] = {};
+};
 struct Profile {
     bool on = false;
-    cudaEvent_t ev[kMaxProfKernels + 1] = {};
     bool created = false;
-    int n = 0;                                  // kernels recorded by the last call
-    const char* names[kMaxProfKernels] = {};
+    ProfCall calls[kProfRing];
+    int recorded = 0;                           // calls recorded since profiling was enabled
+    ProfCall* cur = nullptr;
 };
 thread_local Profile t_prof;
 
 void prof_begin(cudaStream_t st) {
     if (!t_prof.on) return;
     if (!t_prof.created) {
-        for (auto& e : t_prof.ev) if (cudaEventCreate(&e) != cudaSuccess) { t_prof.on = false; return; }
+        for (auto& c : t_prof.calls)
+            for (auto& e : c.ev)
+                if (cudaEventCreate(&e) != cudaSuccess) { t_prof.on = false; return; }
         t_prof.created = true;
     }
-    t_prof.n = 0;
-    (void)cudaEventRecord(t_prof.ev[0], st);
+    t_prof.cur = &t_prof.calls[t_prof.recorded % kProfRing];
+    ++t_prof.recorded;
+    t_prof.cur->n = 0;
+    (void)cudaEventRecord(t_prof.cur->ev[0], st);
 }
 void prof_mark(const char* name, cudaStream_t st) {
-    if (!t_prof.on || t_prof.n >= kMaxProfKernels) return;
-    t_prof.names[t_prof.n] = name;
-    ++t_prof.n;
-    (void)cudaEventRecord(t_prof.ev[t_prof.n], st);
+    if (!t_prof.on || t_prof.cur == nullptr || t_prof.cur->n >= kMaxProfKernels) return;
+    ProfCall* c = t_prof.cur;
+    c->names[c->n] = name;
+    ++c->n;
+    (void)cudaEventRecord(c->ev[c->n], st);
 }
 
 struct DeviceState {
@@ -156,6 +169,9 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
     p.Mpad = (int)((M + 15) / 16 * 16);
     if (p.Mpad < 16) p.Mpad = 16;
     p.NH = (N >= 256 && 2 * nmat * 2 * p.Mpad <= 512) ? 2 : 1;
+    if (const char* e = getenv(nmat == 2 ? "GMLP_SKINNY_NH1" : "GMLP_SKINNY_NH2")) {      // tuning override
+        if (e[0] == '1') p.NH = 1;
+    }
     const int tile_n = 128 * p.NH;
     p.num_tiles = (int)((N + tile_n - 1) / tile_n);
     p.KB = (int)((K + 63) / 64);
@@ -584,25 +600,43 @@ int gmlp_device_status(void) {
 
 int gmlp_profile_enable(int on) {
     t_prof.on = (on != 0);
-    t_prof.n = 0;
+    t_prof.recorded = 0;
+    t_prof.cur = nullptr;
     return GMLP_OK;
 }
 
 int gmlp_profile_read(float* ms, int max_count, int* count) {
     if (ms == nullptr || count == nullptr) return GMLP_ERR_NULL;
     *count = 0;
-    if (!t_prof.created || t_prof.n == 0) return GMLP_OK;
-    if (cudaEventSynchronize(t_prof.ev[t_prof.n]) != cudaSuccess) return GMLP_ERR_LAUNCH;
-    for (int i = 0; i < t_prof.n && i < max_count; ++i) {
-        if (cudaEventElapsedTime(&ms[i], t_prof.ev[i], t_prof.ev[i + 1]) != cudaSuccess) return GMLP_ERR_LAUNCH;
-        *count = i + 1;
+    if (!t_prof.created || t_prof.recorded == 0) return GMLP_OK;
+    const int ncalls = t_prof.recorded < kProfRing ? t_prof.recorded : kProfRing;
+    const ProfCall& last = t_prof.calls[(t_prof.recorded - 1) % kProfRing];
+    const int nk = last.n;
+    double sum[kMaxProfKernels] = {};
+    int used = 0;
+    for (int i = 0; i < ncalls; ++i) {
+        const ProfCall& c = t_prof.calls[i];
+        if (c.n != nk) continue;                 // a call of another shape/schedule: not averaged in
+        if (cudaEventSynchronize(c.ev[c.n]) != cudaSuccess) return GMLP_ERR_LAUNCH;
+        for (int k = 0; k < nk; ++k) {
+            float t = 0.0f;
+            if (cudaEventElapsedTime(&t, c.ev[k], c.ev[k + 1]) != cudaSuccess) return GMLP_ERR_LAUNCH;
+            sum[k] += t;
+        }
+        ++used;
+    }
+    for (int k = 0; k < nk && k < max_count && used > 0; ++k) {
+        ms[k] = (float)(sum[k] / used);
+        *count = k + 1;
     }
     return GMLP_OK;
 }
 
 const char* gmlp_profile_kernel_name(int index) {
-    if (index < 0 || index >= t_prof.n) return "";
-    return t_prof.names[index];
+    if (t_prof.recorded == 0) return "";
+    const ProfCall& last = t_prof.calls[(t_prof.recorded - 1) % kProfRing];
+    if (index < 0 || index >= last.n) return "";
+    return last.names[index];
 }
 
 uint64_t gmlp_launch_count(void) { return t_launches; }

@@ -261,7 +261,8 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                             ptx::tmem_ld_wait();
 #pragma unroll
                             for (int i = 0; i < 16; ++i)
-                                __stcg(mine + ((size_t)(j * NH + h) * Mpad + c0 + i) * 128 + nl, __uint_as_float(v[i]));
+                                if (c0 + i < M)      // rows past M are padding: never read back
+                                    __stcg(mine + ((size_t)(j * NH + h) * Mpad + c0 + i) * 128 + nl, __uint_as_float(v[i]));
                         }
                 ptx::tc_fence_before_sync();
                 __syncwarp();
@@ -292,35 +293,55 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     for (int h = 0; h < NH; ++h) {
                         const int n = n_base + h * 128 + cg * 4;
                         if (n >= N) continue;
-                        for (int m = rg; m < M; m += 4) {
-                            const size_t og = ((size_t)h * Mpad + m) * 128 + cg * 4;
-                            const size_t ou = og + (size_t)NH * Mpad * 128;
-                            float4 g = make_float4(0.f, 0.f, 0.f, 0.f), uu = g;
+                        for (int m = rg; m < M; m += 8) {
+                            // two token rows (m and m + 4) and CB contributors per round: 2 * CB * NMAT
+                            // independent 16-byte loads in flight per thread
+                            constexpr int CB = GATEUP ? 4 : 8;
+                            const bool two = (m + 4) < M;
+                            const size_t og0 = ((size_t)h * Mpad + m) * 128 + cg * 4;
+                            const size_t og1 = two ? og0 + 4 * 128 : og0;
+                            const size_t du = (size_t)NH * Mpad * 128;      // gate -> up offset inside a slot
+                            float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0, u0 = g0, u1 = g0;
                             int i = 0;
-                            for (; i + 4 <= ncontrib; i += 4) {
-                                float4 a[4], b[4];
+                            for (; i + CB <= ncontrib; i += CB) {
+                                float4 a0[CB], a1[CB], b0[CB], b1[CB];
 #pragma unroll
-                                for (int t = 0; t < 4; ++t) {
+                                for (int t = 0; t < CB; ++t) {
                                     const float* p = scratch + slot_off[i + t];
-                                    a[t] = __ldcg(reinterpret_cast<const float4*>(p + og));
-                                    if (GATEUP) b[t] = __ldcg(reinterpret_cast<const float4*>(p + ou));
+                                    a0[t] = __ldcg(reinterpret_cast<const float4*>(p + og0));
+                                    a1[t] = __ldcg(reinterpret_cast<const float4*>(p + og1));
+                                    if (GATEUP) {
+                                        b0[t] = __ldcg(reinterpret_cast<const float4*>(p + og0 + du));
+                                        b1[t] = __ldcg(reinterpret_cast<const float4*>(p + og1 + du));
+                                    }
                                 }
 #pragma unroll
-                                for (int t = 0; t < 4; ++t) { add4(g, a[t]); if (GATEUP) add4(uu, b[t]); }
+                                for (int t = 0; t < CB; ++t) {
+                                    add4(g0, a0[t]); add4(g1, a1[t]);
+                                    if (GATEUP) { add4(u0, b0[t]); add4(u1, b1[t]); }
+                                }
                             }
                             for (; i < ncontrib; ++i) {
                                 const float* p = scratch + slot_off[i];
-                                add4(g, __ldcg(reinterpret_cast<const float4*>(p + og)));
-                                if (GATEUP) add4(uu, __ldcg(reinterpret_cast<const float4*>(p + ou)));
+                                add4(g0, __ldcg(reinterpret_cast<const float4*>(p + og0)));
+                                add4(g1, __ldcg(reinterpret_cast<const float4*>(p + og1)));
+                                if (GATEUP) {
+                                    add4(u0, __ldcg(reinterpret_cast<const float4*>(p + og0 + du)));
+                                    add4(u1, __ldcg(reinterpret_cast<const float4*>(p + og1 + du)));
+                                }
                             }
-                            float v[4] = {g.x, g.y, g.z, g.w};
-                            if (GATEUP) {
-                                v[0] = silu_f32(g.x) * uu.x; v[1] = silu_f32(g.y) * uu.y;
-                                v[2] = silu_f32(g.z) * uu.z; v[3] = silu_f32(g.w) * uu.w;
-                            }
-                            // N is a multiple of 8 and n of 4: the four columns are all inside or all outside
-                            *reinterpret_cast<uint2*>(out + (size_t)m * N + n) =
-                                make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+                            auto finish = [&](const float4& g, const float4& uu, int mm) {
+                                float v[4] = {g.x, g.y, g.z, g.w};
+                                if (GATEUP) {
+                                    v[0] = silu_f32(g.x) * uu.x; v[1] = silu_f32(g.y) * uu.y;
+                                    v[2] = silu_f32(g.z) * uu.z; v[3] = silu_f32(g.w) * uu.w;
+                                }
+                                // N is a multiple of 8 and n of 4: the four columns are all inside or all outside
+                                *reinterpret_cast<uint2*>(out + (size_t)mm * N + n) =
+                                    make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+                            };
+                            finish(g0, u0, m);
+                            if (two) finish(g1, u1, m + 4);
                         }
                     }
                     if (et == 0) counters[tile] = 0u;        // clean for the next call

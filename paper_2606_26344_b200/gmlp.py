@@ -114,7 +114,7 @@ def profile_enable(on: bool) -> None:
 
 
 def profile_read() -> dict:
-    """Durations (ms) of the kernels of the most recent forward_ex call, keyed by kernel name."""
+    """Average durations (ms) of the kernels of the calls recorded since profile_enable(True), by kernel name."""
     ms = (ctypes.c_float * 8)()
     n = ctypes.c_int(0)
     rc = lib().gmlp_profile_read(ms, 8, ctypes.byref(n))
