@@ -53,7 +53,8 @@ typedef enum gmlp_status {
     GMLP_ERR_ARCH = -6,       /* no CUDA device, or the current device is not sm_100 */
     GMLP_ERR_LAUNCH = -7,     /* a CUDA runtime call failed (cudaGetLastError is left readable) */
     GMLP_ERR_TIMEOUT = -8,    /* a bounded device-side wait ran out (see gmlp_device_status) */
-    GMLP_ERR_UNSUPPORTED = -9 /* the forced variant cannot run this shape (SKINNY needs M <= 128) */
+    GMLP_ERR_UNSUPPORTED = -9,/* the forced variant cannot run this shape (SKINNY needs M <= 128) */
+    GMLP_ERR_STATIC_LIMIT = -10 /* gmlp_forward_static: the shape needs more than its fixed built-in scratch */
 } gmlp_status;
 
 enum {
@@ -107,6 +108,38 @@ int gmlp_forward_ex(const gmlp_args* args);
  * Y_host is valid once the stream has been synchronised.
  */
 int gmlp_forward_host(const gmlp_args* args, const void* X_host, void* Y_host);
+
+/*
+ * The same operator for callers that must not allocate device memory.  (The paper has no
+ * counterpart of this call; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs after an application has frozen its memory plan, e.g. a
+ * serving loop that handed the whole device to its own pool at start-up, a process under a
+ * memory manager that forbids further cudaMalloc, or a real-time path where an allocation's
+ * implicit synchronisation is not acceptable.  gmlp_forward may grow a library-owned buffer
+ * with cudaMalloc and gmlp_forward_ex wants a caller-made workspace; this call wants
+ * neither.  Its scratch (the bf16 intermediate H, the split-K partial sums and the arrival
+ * counters of the small-M schedule) lives in a fixed array of GMLP_STATIC_SCRATCH_BYTES that
+ * is part of the library image: every GPU that loads the library holds that much memory
+ * until the process exits, whether or not this call is ever used.
+ *
+ * Limits: M <= GMLP_STATIC_MAX_M tokens, no RMSNorm prologue, and a shape whose scratch fits
+ * the array (any Llama-sized layer does at M <= 16).  Anything larger is refused with
+ * GMLP_ERR_STATIC_LIMIT before any device work.  X, Wg, Wu, Wd, Y: device pointers as for
+ * gmlp_forward; stream: cudaStream_t (NULL = legacy default stream).  Asynchronous.
+ *
+ * It calls no cudaMalloc, cudaFree or allocating library routine.  The FIRST call on each
+ * device looks up the device address of the built-in array (cudaGetSymbolAddress, with that
+ * device current) and sets kernel attributes; make that first call outside any stream
+ * capture.  All calls on a device share the one array, and it keeps whatever the previous
+ * call left: each call clears the counters it needs itself, so back-to-back calls on one
+ * stream are fine, but two calls that can overlap on the GPU (different streams, no
+ * ordering) race on the scratch and give wrong results.
+ */
+#define GMLP_STATIC_SCRATCH_BYTES (12u << 20)
+#define GMLP_STATIC_MAX_M 16
+int gmlp_forward_static(const void* X, const void* Wg, const void* Wu, const void* Wd, void* Y,
+                        int64_t M, int64_t d_model, int64_t d_ff, void* stream);
 
 /*
  * Bytes of scratch gmlp_forward_ex needs for this shape, for the schedule `variant` would

@@ -524,9 +524,76 @@ int forward_impl(const gmlp_args* a) {
     return GMLP_OK;
 }
 
+// ------------------------------------------------------------------ allocation-free entry point
+// Scratch of gmlp_forward_static: part of the library image, one copy per GPU that loads it.  In host
+// code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[GMLP_STATIC_SCRATCH_BYTES];
+
+struct StaticScratch {
+    bool ready = false;
+    uint8_t* ptr = nullptr;          // device address of g_static_scratch on this device
+};
+StaticScratch g_static[kMaxDevices];
+
+int forward_static_impl(const void* Xp, const void* Wgp, const void* Wup, const void* Wdp, void* Yp,
+                        int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st) {
+    int rc = check_shape(M, d_model, d_ff);
+    if (rc != GMLP_OK) return rc;
+    if (M > GMLP_STATIC_MAX_M) return GMLP_ERR_STATIC_LIMIT;
+    if (M == 0) return GMLP_OK;
+    if (!Xp || !Wgp || !Wup || !Wdp || !Yp) return GMLP_ERR_NULL;
+    if (!aligned16(Xp) || !aligned16(Wgp) || !aligned16(Wup) || !aligned16(Wdp) || !aligned16(Yp)) return GMLP_ERR_ALIGN;
+
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    const Layout L = make_layout(M, d_model, d_ff, 0, GMLP_VARIANT_SKINNY, dev->sm_count);
+    if (L.total > (uint64_t)GMLP_STATIC_SCRATCH_BYTES) return GMLP_ERR_STATIC_LIMIT;
+
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess) return GMLP_ERR_ARCH;
+    uint8_t* ws = nullptr;
+    {
+        // once per device, with that device current: the array's device address
+        std::lock_guard<std::mutex> lock(g_mutex);
+        StaticScratch& s = g_static[device];
+        if (!s.ready) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+                (void)cudaGetLastError();
+                return GMLP_ERR_LAUNCH;
+            }
+            s.ptr = static_cast<uint8_t*>(p);
+            s.ready = true;
+        }
+        ws = s.ptr;
+    }
+
+    const bf16* X = static_cast<const bf16*>(Xp);
+    bf16* H = reinterpret_cast<bf16*>(ws + L.h_off);
+    float* scratch = reinterpret_cast<float*>(ws + L.partial_off);
+    unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
+    unsigned int* c2 = c1 + L.s1.num_tiles;
+    // the array keeps the previous call's contents: the arrival counters must start at zero
+    if (cudaMemsetAsync(c1, 0, L.counters_bytes, st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    rc = launch_skinny<true>(dev, L.s1, X, static_cast<const bf16*>(Wgp), static_cast<const bf16*>(Wup), scratch, c1, H,
+                             M, d_model, d_ff, st);
+    if (rc != GMLP_OK) return rc;
+    return launch_skinny<false>(dev, L.s2, H, static_cast<const bf16*>(Wdp), nullptr, scratch, c2,
+                                static_cast<bf16*>(Yp), M, d_ff, d_model, st);
+}
+
 }  // namespace
 
 extern "C" {
+
+int gmlp_forward_static(const void* X, const void* Wg, const void* Wu, const void* Wd, void* Y,
+                        int64_t M, int64_t d_model, int64_t d_ff, void* stream) {
+    try {
+        return forward_static_impl(X, Wg, Wu, Wd, Y, M, d_model, d_ff, static_cast<cudaStream_t>(stream));
+    } catch (...) {
+        return GMLP_ERR_LAUNCH;
+    }
+}
 
 int gmlp_forward_ex(const gmlp_args* args) {
     try {
@@ -654,6 +721,8 @@ const char* gmlp_status_string(int status) {
         case GMLP_ERR_LAUNCH: return "a CUDA runtime call failed";
         case GMLP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
         case GMLP_ERR_UNSUPPORTED: return "the forced variant cannot run this shape";
+        case GMLP_ERR_STATIC_LIMIT:
+            return "gmlp_forward_static: shape exceeds its fixed scratch (M <= 16, no RMSNorm, scratch <= 12 MiB)";
         default: return "unknown status";
     }
 }

@@ -15,6 +15,9 @@ import torch
 OK = 0
 ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_FLAGS, ERR_WORKSPACE, ERR_ARCH, ERR_LAUNCH, ERR_TIMEOUT, ERR_UNSUPPORTED = \
     -1, -2, -3, -4, -5, -6, -7, -8, -9
+ERR_STATIC_LIMIT = -10
+STATIC_MAX_M = 16
+STATIC_SCRATCH_BYTES = 12 << 20
 FLAG_RMSNORM = 1 << 0
 FLAG_CHECKED = 1 << 2
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA, VARIANT_SKINNY = 0, 1, 2, 3, 4
@@ -55,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.gmlp_forward_ex.argtypes = [ctypes.POINTER(GmlpArgs)]
         L.gmlp_forward_host.restype = ctypes.c_int
         L.gmlp_forward_host.argtypes = [ctypes.POINTER(GmlpArgs), vp, vp]
+        L.gmlp_forward_static.restype = ctypes.c_int
+        L.gmlp_forward_static.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.gmlp_workspace_bytes.restype = u64
         L.gmlp_workspace_bytes.argtypes = [i64, i64, i64, u32, i32]
         L.gmlp_pick_variant.restype = ctypes.c_int
@@ -190,5 +195,22 @@ def forward_simple(X, Wg, Wu, Wd, Y, flags: int = 0) -> None:
     with torch.cuda.device(X.device):
         rc = lib().gmlp_forward(X.data_ptr(), Wg.data_ptr(), Wu.data_ptr(), Wd.data_ptr(), Y.data_ptr(),
                                 M, d_model, Wg.shape[1], flags)
+    if rc != OK:
+        raise GmlpError(rc)
+
+
+def forward_static(X, Wg, Wu, Wd, Y, stream=None) -> None:
+    """gmlp_forward_static: the operator for callers that may not allocate device memory.
+
+    Scratch comes from a fixed array inside the library (M <= STATIC_MAX_M, no RMSNorm); nothing is
+    allocated.  Calls that can overlap on the GPU race on that array: keep them on one stream.
+    """
+    for t, n in ((X, "X"), (Wg, "Wg"), (Wu, "Wu"), (Wd, "Wd"), (Y, "Y")):
+        _check_bf16_cuda(t, n)
+    M, d_model = X.shape
+    st = stream if stream is not None else torch.cuda.current_stream(X.device)
+    with torch.cuda.device(X.device):
+        rc = lib().gmlp_forward_static(X.data_ptr(), Wg.data_ptr(), Wu.data_ptr(), Wd.data_ptr(), Y.data_ptr(),
+                                       M, d_model, Wg.shape[1], st.cuda_stream)
     if rc != OK:
         raise GmlpError(rc)
