@@ -335,16 +335,11 @@ def main():
 
     w = I.WORKLOADS[args.workload]
     res = measure_workload(w, args.steps, warmup, dev, peaks, dist=dist, clock_roll=args.clock_roll)
-    ms = res["ms_per_step"]
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        e = torch.tensor([res["e2e"]["ms_per_step"]], device=dev, dtype=torch.float64)
-        dist.all_reduce(e, op=dist.ReduceOp.MAX)
-        res["e2e"]["ms_per_step"] = float(e.item())
-        res["e2e"]["value"] = world * w.M / (res["e2e"]["ms_per_step"] * 1e-3)
-    value = world * w.M / (ms * 1e-3)
+    from paper_2606_26344_b200 import sharding
+    ms = sharding.max_over_ranks(res["ms_per_step"], dist, dev)          # the slowest rank bounds the step
+    res["e2e"]["ms_per_step"] = sharding.max_over_ranks(res["e2e"]["ms_per_step"], dist, dev)
+    res["e2e"]["value"] = sharding.job_throughput(w.M, world, res["e2e"]["ms_per_step"])
+    value = sharding.job_throughput(w.M, world, ms)
 
     extras = []
     if not args.no_extra and world == 1:
