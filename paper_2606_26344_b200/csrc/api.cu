@@ -347,8 +347,21 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     const int bn = GATEUP ? 128 : 256;
     const int num_m = (int)((M + gmlp::kUmmaBM - 1) / gmlp::kUmmaBM);
     const int num_n = (int)((N + bn - 1) / bn);
-    gmlp::umma_gemm_kernel<GATEUP><<<(unsigned)(num_m * num_n), gmlp::kUmmaThreads, gmlp::kUmmaSmemBytes, st>>>(
-        tmA, tmB0, tmB1, C, (int)M, (int)K, (int)N, num_m);
+    const int num_tiles = num_m * num_n;
+    const int sms = dev->sm_count > 0 ? dev->sm_count : 148;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(num_tiles < sms ? num_tiles : sms));     // persistent: one CTA per SM
+    cfg.blockDim = dim3(gmlp::kUmmaThreads);
+    cfg.dynamicSmemBytes = gmlp::kUmmaSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<GATEUP>, tmA, tmB0, tmB1, C, (int)M, (int)K, (int)N, num_m,
+                           num_tiles) != cudaSuccess)
+        return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
 }

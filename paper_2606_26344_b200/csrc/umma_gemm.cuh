@@ -15,6 +15,8 @@
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
 // warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31).
+// CTAs are persistent (one per SM, tiles taken round-robin) and TMEM holds two accumulator
+// buffers, so the epilogue of one tile runs while the MMAs of the next tile are issued.
 // Every mbarrier wait is bounded; a wait that runs out records a status word, raises a
 // CTA-wide abort flag and the CTA leaves through the normal teardown (TMEM freed).
 #pragma once
@@ -29,6 +31,7 @@ constexpr int kUmmaBM = 128;
 constexpr int kUmmaBK = 64;
 constexpr int kUmmaN = 256;                 // MMA N: 128 gate + 128 up, or 256 plain columns
 constexpr int kUmmaStages = 4;
+constexpr uint32_t kUmmaTmemCols = 512;      // two accumulator buffers of 256 columns
 constexpr int kUmmaThreads = 192;
 constexpr uint32_t kUmmaABytes = kUmmaBM * kUmmaBK * 2;          // 16 KB: 128 rows x 128 B
 constexpr uint32_t kUmmaBoxBBytes = 64 * kUmmaBK * 2;            // 8 KB: 64 k-rows x 128 B (64 columns)
@@ -60,7 +63,7 @@ template <bool GATEUP>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
-                 int M, int K, int N, int num_m_tiles)
+                 int M, int K, int N, int num_m_tiles, int num_tiles)
 {
     constexpr int KERNEL_ID = GATEUP ? 1 : 2;
     constexpr int BN_OUT = GATEUP ? 128 : 256;
@@ -72,23 +75,24 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + kUmmaStages * kUmmaStageBytes);
     const uint32_t full0 = ptx::smem_addr(bars);
     const uint32_t empty0 = ptx::smem_addr(bars + kUmmaStages);
-    const uint32_t tmem_full = ptx::smem_addr(bars + 2 * kUmmaStages);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kUmmaStages + 1);
+    const uint32_t tfull0 = ptx::smem_addr(bars + 2 * kUmmaStages);          // accumulator buffer b is complete
+    const uint32_t tempty0 = ptx::smem_addr(bars + 2 * kUmmaStages + 2);     // accumulator buffer b has been read out
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kUmmaStages + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m_tile = blockIdx.x % num_m_tiles;                  // row tiles fastest: CTAs of a wave share weight panels
-    const int n_tile = blockIdx.x / num_m_tiles;
-    const int m0 = m_tile * kUmmaBM;
-    const int n0 = n_tile * BN_OUT;
     const int num_kb = (K + kUmmaBK - 1) / kUmmaBK;
 
+    ptx::launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < kUmmaStages; ++s) {
             ptx::mbar_init(full0 + 8 * s, 1);
             ptx::mbar_init(empty0 + 8 * s, 1);
         }
-        ptx::mbar_init(tmem_full, 1);
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(tfull0 + 8 * b, 1);
+            ptx::mbar_init(tempty0 + 8 * b, 4);                   // one arrival per epilogue warp
+        }
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
@@ -97,7 +101,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (GATEUP) ptx::prefetch_tensormap(&tmB1);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_addr(tmem_slot), kUmmaN);
+        ptx::tmem_alloc(ptx::smem_addr(tmem_slot), kUmmaTmemCols);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before_sync();
@@ -105,23 +109,32 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
+    // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...; row tiles vary fastest, so the CTAs of
+    // one round work on the same few weight panels (L2 reuse).
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % kUmmaStages;
-                const uint32_t ph = (uint32_t)(kb / kUmmaStages) & 1u;
-                if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
-                const uint32_t full = full0 + 8 * s;
-                const uint32_t a_dst = base + s * kUmmaStageBytes;
-                const uint32_t b_dst = a_dst + kUmmaABytes;
-                ptx::mbar_arrive_expect_tx(full, kUmmaStageBytes);
-                ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
+            ptx::grid_dependency_wait();                          // A (X, Xn or H) may come from the previous kernel
+            int it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % num_m_tiles) * kUmmaBM;
+                const int n0 = (tile / num_m_tiles) * BN_OUT;
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % kUmmaStages;
+                    const uint32_t ph = (uint32_t)(it / kUmmaStages) & 1u;
+                    if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) { ok = false; break; }
+                    const uint32_t full = full0 + 8 * s;
+                    const uint32_t a_dst = base + s * kUmmaStageBytes;
+                    const uint32_t b_dst = a_dst + kUmmaABytes;
+                    ptx::mbar_arrive_expect_tx(full, kUmmaStageBytes);
+                    ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const CUtensorMap* map = (GATEUP && i >= 2) ? &tmB1 : &tmB0;
-                    const int x = GATEUP ? n0 + (i & 1) * 64 : n0 + i * 64;
-                    ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
+                    for (int i = 0; i < 4; ++i) {
+                        const CUtensorMap* map = (GATEUP && i >= 2) ? &tmB1 : &tmB0;
+                        const int x = GATEUP ? n0 + (i & 1) * 64 : n0 + i * 64;
+                        ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
+                    }
                 }
             }
         }
@@ -129,36 +142,49 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
+            int it = 0, t = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % kUmmaStages;
-                const uint32_t ph = (uint32_t)(kb / kUmmaStages) & 1u;
-                if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
+                const int buf = t & 1;
+                // the epilogue must have drained this accumulator buffer (two tiles ago)
+                if (!wait_bounded(tempty0 + 8 * buf, (((uint32_t)t >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4)) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t a_base = base + s * kUmmaStageBytes;
-                const uint32_t b_base = a_base + kUmmaABytes;
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kUmmaN);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % kUmmaStages;
+                    const uint32_t ph = (uint32_t)(it / kUmmaStages) & 1u;
+                    if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_base = base + s * kUmmaStageBytes;
+                    const uint32_t b_base = a_base + kUmmaABytes;
 #pragma unroll
-                for (int k = 0; k < kUmmaBK / 16; ++k) {
-                    // A: K-major, rows of 128 B, 8-row groups 1024 B apart; +32 B per K = 16 step.
-                    // B: MN-major, 64-column chunks 8 KB apart (LBO), 8-row k-groups 1024 B apart (SBO);
-                    //    K = 16 is two k-groups: +2048 B per step.
-                    const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
-                    const uint64_t b_desc = ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
-                    ptx::umma_bf16(tmem_base, a_desc, b_desc, kUmmaIdesc, (kb | k) != 0 ? 1u : 0u);
+                    for (int k = 0; k < kUmmaBK / 16; ++k) {
+                        // A: K-major, rows of 128 B, 8-row groups 1024 B apart; +32 B per K = 16 step.
+                        // B: MN-major, 64-column chunks 8 KB apart (LBO), 8-row k-groups 1024 B apart (SBO);
+                        //    K = 16 is two k-groups: +2048 B per step.
+                        const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
+                        const uint64_t b_desc = ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
+                        ptx::umma_bf16(d_tmem, a_desc, b_desc, kUmmaIdesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    ptx::umma_commit(empty0 + 8 * s);      // stage is free once these MMAs have read it
                 }
-                ptx::umma_commit(empty0 + 8 * s);      // stage is free once these MMAs have read it
+                if (ok) ptx::umma_commit(tfull0 + 8 * buf);   // accumulator complete
             }
-            if (ok) ptx::umma_commit(tmem_full);       // accumulator complete
         }
         __syncwarp();
     } else {
         // ---------------- epilogue ----------------
         const int q = warp & 3;
-        const int row = m0 + q * 32 + lane;
-        const bool ok = wait_bounded(tmem_full, 0u, abort_flag, KERNEL_ID, 3);
-        ptx::tc_fence_after_sync();
-        if (ok) {
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+        ptx::grid_dependency_wait();                              // C may still be read by the previous kernel
+        int t = 0;
+        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++t) {
+            const int buf = t & 1;
+            const int m0 = (tile % num_m_tiles) * kUmmaBM;
+            const int n0 = (tile / num_m_tiles) * BN_OUT;
+            const int row = m0 + q * 32 + lane;
+            if (!wait_bounded(tfull0 + 8 * buf, ((uint32_t)t >> 1) & 1u, abort_flag, KERNEL_ID, 3)) break;
+            ptx::tc_fence_after_sync();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * kUmmaN);
             bf16* crow = C + (size_t)row * N + n0;
 #pragma unroll 1
             for (int c = 0; c < BN_OUT; c += 32) {
@@ -191,6 +217,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                 }
             }
+            // all of this warp's TMEM reads of the buffer are done: hand it back to the MMA issuer
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(tempty0 + 8 * buf);
         }
     }
 
@@ -203,7 +233,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, kUmmaN);
+        ptx::tmem_dealloc(tmem_base, kUmmaTmemCols);
     }
 }
 
