@@ -35,6 +35,12 @@ PRIMARY = "llama3-8b-decode-M8"
 EXTRA = ["llama3-8b-prefill-M2048-rmsnorm", "llama3-70b-prefill-M4096-outliers", "ragged-M8192-plain",
          "ragged-M1000-plain", "ragged-M129-plain", "ragged-M7-plain", "ragged-M1-plain"]
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
+# summarised under profiles/ (skinny_gemm_decode_M8.md, umma_gemm_prefill8b_M2048.md)
+NCU_TRAFFIC_BYTES = {
+    ("llama3-8b-decode-M8", "gate_up"): 235.5e6 + 4.0e6,
+    ("llama3-8b-prefill-M2048-rmsnorm", "gate_up"): 251.9e6 + 49.1e6,
+}
 
 
 def load_peaks():
@@ -263,13 +269,15 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
             flops = 4 * w.M * w.d_model * w.d_ff
             ach = flops / kms / 1e12
             res["roofline"] = {"kernel": "gate_up", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
-                               "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"], "traffic": None,
+                               "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
+                               "traffic": NCU_TRAFFIC_BYTES.get((w.name, "gate_up")), "algorithmic_flops": flops,
                                "peak_source": peaks["source"] + " (burst bf16)"}
         else:
             nbytes = 2 * (2 * w.d_model * w.d_ff + w.M * w.d_model + w.M * w.d_ff)
             ach = nbytes / kms / 1e9
             res["roofline"] = {"kernel": "gate_up", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
-                               "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                               "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                               "traffic": NCU_TRAFFIC_BYTES.get((w.name, "gate_up")), "algorithmic_bytes": nbytes,
                                "peak_source": peaks["source"] + " (copy)"}
 
     if want_e2e:

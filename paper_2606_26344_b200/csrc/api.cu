@@ -178,6 +178,7 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
     const uint32_t stage_bytes = (uint32_t)nmat * p.NH * 2 * gmlp::kSkinnyBoxBytes + (uint32_t)p.Mpad * 128u;
     int st = (int)((gmlp::kSkinnySmemBudget - 1024 - 256) / stage_bytes);
     p.stages = st > gmlp::kSkinnyMaxStages ? gmlp::kSkinnyMaxStages : st;
+    if (const char* e = getenv("GMLP_SKINNY_STAGES")) { int v = atoi(e); if (v >= 2 && v < p.stages) p.stages = v; }   // tuning override
     uint32_t cols = (uint32_t)(2 * nmat * p.NH * p.Mpad);
     uint32_t pow2 = 32;
     while (pow2 < cols) pow2 <<= 1;
@@ -400,13 +401,15 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const int Mi = (int)M, Ni = (int)N;
+    int evict_first = 1;                                // weights are read once: let L2 drop them first
+    if (const char* e = getenv("GMLP_SKINNY_EVICT_FIRST")) evict_first = atoi(e);      // tuning override
     cudaError_t err;
     if (p.NH == 2)
         err = cudaLaunchKernelEx(&cfg, gmlp::skinny_gemm_kernel<GATEUP, 2>, tmX, tmW0, tmW1, scratch, counters, out,
-                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols);
+                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first);
     else
         err = cudaLaunchKernelEx(&cfg, gmlp::skinny_gemm_kernel<GATEUP, 1>, tmX, tmW0, tmW1, scratch, counters, out,
-                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols);
+                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;

@@ -34,7 +34,7 @@
 namespace gmlp {
 
 constexpr int kSkinnyThreads = 192;
-constexpr int kSkinnyMaxStages = 8;
+constexpr int kSkinnyMaxStages = 12;
 constexpr uint32_t kSkinnyBoxBytes = 64 * 64 * 2;            // 64 k-rows x 128 B
 constexpr uint32_t kSkinnySmemBudget = 229376;               // dynamic shared memory requested (224 KB)
 constexpr int kSkinnyMaxContrib = 256;                       // CTAs that can share one column tile (>= grid size)
@@ -58,12 +58,160 @@ __device__ __forceinline__ int range_owner(long long unit, long long total, long
     return (int)(((unit + 1) * parts - 1) / total);
 }
 
+// One segment (this CTA's share of one column tile's K range) as seen by the 128 epilogue threads:
+// either the CTA owns the tile's whole K range and applies the epilogue straight from TMEM, or it parks its
+// fp32 partial in scratch, draws an arrival ticket, and - if it is the last contributor - adds all partials
+// in CTA order and applies the epilogue.  Returns true when this CTA wrote the tile's final output.
+//   acc0        TMEM address (lane quarter and first column) of the accumulator buffer; accumulator (j, h)
+//               starts at column (j * NH + h) * Mpad
+//   total/parts/KB  the flat work sequence (see range_start / range_owner) this phase was cut from
+template <bool GATEUP, int NH>
+__device__ __forceinline__ bool skinny_epilogue_segment(
+    uint32_t acc0, uint32_t tempty_bar, int tile, bool first_segment_of_cta, int cta, long long total, long long parts,
+    int KB, int M, int Mpad, int N, float* __restrict__ scratch, unsigned int* __restrict__ counters,
+    bf16* __restrict__ out, unsigned long long* slot_off, volatile int* last_flag, int et, int nl, int lane)
+{
+    constexpr int NMAT = GATEUP ? 2 : 1;
+    constexpr int TILE_N = 128 * NH;
+    const size_t slot_floats = (size_t)NMAT * NH * Mpad * 128;
+    const long long tile_first = (long long)tile * KB;
+    const int first_c = range_owner(tile_first, total, parts);
+    const int last_c = range_owner(tile_first + KB - 1, total, parts);
+    const int n_base = tile * TILE_N;
+
+    if (first_c == last_c) {
+        // this CTA owns the whole K range of the tile: epilogue straight from TMEM
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+            const int n = n_base + h * 128 + nl;
+            for (int c0 = 0; c0 < Mpad; c0 += 16) {
+                uint32_t g[16], uu[16];
+                tmem_ld_32x16(acc0 + (uint32_t)((0 * NH + h) * Mpad + c0), g);
+                if (GATEUP) tmem_ld_32x16(acc0 + (uint32_t)((1 * NH + h) * Mpad + c0), uu);
+                ptx::tmem_ld_wait();
+                if (n < N) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int m = c0 + i;
+                        if (m < M) {
+                            const float v = GATEUP ? silu_f32(__uint_as_float(g[i])) * __uint_as_float(uu[i])
+                                                   : __uint_as_float(g[i]);
+                            out[(size_t)m * N + n] = __float2bfloat16_rn(v);
+                        }
+                    }
+                }
+            }
+        }
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(tempty_bar);
+        return true;
+    }
+
+    // partial K range: park the fp32 accumulators in this CTA's scratch slot
+    const int slot = first_segment_of_cta ? 0 : 1;
+    float* mine = scratch + ((size_t)cta * 2 + slot) * slot_floats;
+#pragma unroll
+    for (int j = 0; j < NMAT; ++j)
+#pragma unroll
+        for (int h = 0; h < NH; ++h)
+            for (int c0 = 0; c0 < Mpad; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld_32x16(acc0 + (uint32_t)((j * NH + h) * Mpad + c0), v);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if (c0 + i < M)      // rows past M are padding: never read back
+                        __stcg(mine + ((size_t)(j * NH + h) * Mpad + c0 + i) * 128 + nl, __uint_as_float(v[i]));
+            }
+    ptx::tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(tempty_bar);
+    __threadfence();
+    epi_bar_sync();
+    if (et == 0) {
+        const unsigned int ticket = atomicAdd(counters + tile, 1u);
+        *last_flag = (ticket == (unsigned int)(last_c - first_c)) ? 1 : 0;
+    }
+    epi_bar_sync();
+    if (*last_flag == 0) return false;
+
+    __threadfence();
+    // Sum the contributors' partials in CTA order.  Thread mapping: 32 column groups of 4 columns x 4 row
+    // groups; float4 loads, several contributors and two token rows per round, so that many loads are in
+    // flight while the additions keep their fixed order.
+    const int ncontrib = last_c - first_c + 1;
+    for (int i = et; i < ncontrib; i += 128) {
+        const int c = first_c + i;
+        const int cslot = ((int)(range_start(c, total, parts) / KB) == tile) ? 0 : 1;
+        slot_off[i] = ((unsigned long long)c * 2 + cslot) * slot_floats;
+    }
+    epi_bar_sync();
+    const int cg = et & 31, rg = et >> 5;
+    auto add4 = [](float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; };
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+        const int n = n_base + h * 128 + cg * 4;
+        if (n >= N) continue;
+        for (int m = rg; m < M; m += 8) {
+            constexpr int CB = GATEUP ? 4 : 8;
+            const bool two = (m + 4) < M;
+            const size_t og0 = ((size_t)h * Mpad + m) * 128 + cg * 4;
+            const size_t og1 = two ? og0 + 4 * 128 : og0;
+            const size_t du = (size_t)NH * Mpad * 128;      // gate -> up offset inside a slot
+            float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0, u0 = g0, u1 = g0;
+            int i = 0;
+            for (; i + CB <= ncontrib; i += CB) {
+                float4 a0[CB], a1[CB], b0[CB], b1[CB];
+#pragma unroll
+                for (int t = 0; t < CB; ++t) {
+                    const float* p = scratch + slot_off[i + t];
+                    a0[t] = __ldcg(reinterpret_cast<const float4*>(p + og0));
+                    a1[t] = __ldcg(reinterpret_cast<const float4*>(p + og1));
+                    if (GATEUP) {
+                        b0[t] = __ldcg(reinterpret_cast<const float4*>(p + og0 + du));
+                        b1[t] = __ldcg(reinterpret_cast<const float4*>(p + og1 + du));
+                    }
+                }
+#pragma unroll
+                for (int t = 0; t < CB; ++t) {
+                    add4(g0, a0[t]); add4(g1, a1[t]);
+                    if (GATEUP) { add4(u0, b0[t]); add4(u1, b1[t]); }
+                }
+            }
+            for (; i < ncontrib; ++i) {
+                const float* p = scratch + slot_off[i];
+                add4(g0, __ldcg(reinterpret_cast<const float4*>(p + og0)));
+                add4(g1, __ldcg(reinterpret_cast<const float4*>(p + og1)));
+                if (GATEUP) {
+                    add4(u0, __ldcg(reinterpret_cast<const float4*>(p + og0 + du)));
+                    add4(u1, __ldcg(reinterpret_cast<const float4*>(p + og1 + du)));
+                }
+            }
+            auto finish = [&](const float4& g, const float4& uu, int mm) {
+                float v[4] = {g.x, g.y, g.z, g.w};
+                if (GATEUP) {
+                    v[0] = silu_f32(g.x) * uu.x; v[1] = silu_f32(g.y) * uu.y;
+                    v[2] = silu_f32(g.z) * uu.z; v[3] = silu_f32(g.w) * uu.w;
+                }
+                // N is a multiple of 8 and n of 4: the four columns are all inside or all outside
+                *reinterpret_cast<uint2*>(out + (size_t)mm * N + n) =
+                    make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+            };
+            finish(g0, u0, m);
+            if (two) finish(g1, u1, m + 4);
+        }
+    }
+    if (et == 0) counters[tile] = 0u;        // clean for the next call
+    return true;
+}
+
 template <bool GATEUP, int NH>
 __global__ void __launch_bounds__(kSkinnyThreads, 1)
 skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW0,
                    const __grid_constant__ CUtensorMap tmW1, float* __restrict__ scratch,
                    unsigned int* __restrict__ counters, bf16* __restrict__ out,
-                   int M, int Mpad, int N, int num_tiles, int KB, int stages, uint32_t tmem_cols)
+                   int M, int Mpad, int N, int num_tiles, int KB, int stages, uint32_t tmem_cols, int evict_first)
 {
     constexpr int KERNEL_ID = GATEUP ? 3 : 4;
     constexpr int NMAT = GATEUP ? 2 : 1;
@@ -124,6 +272,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
+            const uint64_t policy = ptx::l2_policy_evict_first();
             auto load_weights = [&](long long u, int s) {
                 const int tile = (int)(u / KB), kb = (int)(u % KB);
                 const uint32_t full = full0 + 8 * s;
@@ -133,8 +282,12 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 for (int j = 0; j < NMAT; ++j)
 #pragma unroll
                     for (int hb = 0; hb < NH * 2; ++hb)
-                        ptx::tma_load_2d(st + (j * NH * 2 + hb) * kSkinnyBoxBytes, j ? &tmW1 : &tmW0,
-                                         tile * TILE_N + hb * 64, kb * 64, full);
+                        if (evict_first)
+                            ptx::tma_load_2d_hint(st + (j * NH * 2 + hb) * kSkinnyBoxBytes, j ? &tmW1 : &tmW0,
+                                                  tile * TILE_N + hb * 64, kb * 64, full, policy);
+                        else
+                            ptx::tma_load_2d(st + (j * NH * 2 + hb) * kSkinnyBoxBytes, j ? &tmW1 : &tmW0,
+                                             tile * TILE_N + hb * 64, kb * 64, full);
             };
             auto load_tokens = [&](long long u, int s) {
                 ptx::tma_load_2d(base + s * stage_bytes + W_BYTES, &tmX, (int)(u % KB) * 64, 0, full0 + 8 * s);
@@ -205,148 +358,19 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         const int nl = q * 32 + lane;                       // column within a 128-column half = TMEM lane
         const int et = threadIdx.x - 64;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-        const size_t slot_floats = (size_t)NMAT * NH * Mpad * 128;
         int seg = 0;
-        bool ok = true;
         ptx::grid_dependency_wait();          // scratch, counters and `out` may still be in use by the previous kernel
-        for (long long u = u_begin; u < u_end && ok; ++seg) {
+        for (long long u = u_begin; u < u_end; ++seg) {
             const int tile = (int)(u / KB);
             const long long tile_first = (long long)tile * KB;
             const long long seg_end = (tile_first + KB < u_end) ? tile_first + KB : u_end;
             const int buf = seg & 1;
-            ok = wait_bounded(tfull0 + 8 * buf, ((uint32_t)seg >> 1) & 1u, abort_flag, KERNEL_ID, 3);
+            const bool ok = wait_bounded(tfull0 + 8 * buf, ((uint32_t)seg >> 1) & 1u, abort_flag, KERNEL_ID, 3);
             ptx::tc_fence_after_sync();
             if (!ok) break;
-            const int first_c = range_owner(tile_first, total, parts);
-            const int last_c = range_owner(tile_first + KB - 1, total, parts);
-            const int n_base = tile * TILE_N;
-
-            if (first_c == last_c) {
-                // this CTA owns the whole K range of the tile: epilogue straight from TMEM
-#pragma unroll
-                for (int h = 0; h < NH; ++h) {
-                    const int n = n_base + h * 128 + nl;
-                    for (int c0 = 0; c0 < Mpad; c0 += 16) {
-                        uint32_t g[16], uu[16];
-                        tmem_ld_32x16(tmem_base + lane_base + acc_col(buf, 0, h) + c0, g);
-                        if (GATEUP) tmem_ld_32x16(tmem_base + lane_base + acc_col(buf, 1, h) + c0, uu);
-                        ptx::tmem_ld_wait();
-                        if (n < N) {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const int m = c0 + i;
-                                if (m < M) {
-                                    const float v = GATEUP ? silu_f32(__uint_as_float(g[i])) * __uint_as_float(uu[i])
-                                                           : __uint_as_float(g[i]);
-                                    out[(size_t)m * N + n] = __float2bfloat16_rn(v);
-                                }
-                            }
-                        }
-                    }
-                }
-                ptx::tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(tempty0 + 8 * buf);
-            } else {
-                // partial K range: park the fp32 accumulators in this CTA's scratch slot
-                const int slot = (tile == (int)(u_begin / KB)) ? 0 : 1;
-                float* mine = scratch + ((size_t)blockIdx.x * 2 + slot) * slot_floats;
-#pragma unroll
-                for (int j = 0; j < NMAT; ++j)
-#pragma unroll
-                    for (int h = 0; h < NH; ++h)
-                        for (int c0 = 0; c0 < Mpad; c0 += 16) {
-                            uint32_t v[16];
-                            tmem_ld_32x16(tmem_base + lane_base + acc_col(buf, j, h) + c0, v);
-                            ptx::tmem_ld_wait();
-#pragma unroll
-                            for (int i = 0; i < 16; ++i)
-                                if (c0 + i < M)      // rows past M are padding: never read back
-                                    __stcg(mine + ((size_t)(j * NH + h) * Mpad + c0 + i) * 128 + nl, __uint_as_float(v[i]));
-                        }
-                ptx::tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(tempty0 + 8 * buf);
-                __threadfence();
-                epi_bar_sync();
-                if (et == 0) {
-                    const unsigned int ticket = atomicAdd(counters + tile, 1u);
-                    *last_flag = (ticket == (unsigned int)(last_c - first_c)) ? 1 : 0;
-                }
-                epi_bar_sync();
-                const bool is_last = (*last_flag != 0);
-                if (is_last) {
-                    __threadfence();
-                    // Sum the contributors' partials in CTA order.  Thread mapping: 32 column groups of 4
-                    // columns x 4 row groups; float4 loads, contributors fetched four at a time so that
-                    // many loads are in flight while the additions keep their fixed order.
-                    const int ncontrib = last_c - first_c + 1;
-                    for (int i = et; i < ncontrib; i += 128) {
-                        const int c = first_c + i;
-                        const int cslot = ((int)(range_start(c, total, parts) / KB) == tile) ? 0 : 1;
-                        slot_off[i] = ((unsigned long long)c * 2 + cslot) * slot_floats;
-                    }
-                    epi_bar_sync();
-                    const int cg = et & 31, rg = et >> 5;
-                    auto add4 = [](float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; };
-#pragma unroll
-                    for (int h = 0; h < NH; ++h) {
-                        const int n = n_base + h * 128 + cg * 4;
-                        if (n >= N) continue;
-                        for (int m = rg; m < M; m += 8) {
-                            // two token rows (m and m + 4) and CB contributors per round: 2 * CB * NMAT
-                            // independent 16-byte loads in flight per thread
-                            constexpr int CB = GATEUP ? 4 : 8;
-                            const bool two = (m + 4) < M;
-                            const size_t og0 = ((size_t)h * Mpad + m) * 128 + cg * 4;
-                            const size_t og1 = two ? og0 + 4 * 128 : og0;
-                            const size_t du = (size_t)NH * Mpad * 128;      // gate -> up offset inside a slot
-                            float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0, u0 = g0, u1 = g0;
-                            int i = 0;
-                            for (; i + CB <= ncontrib; i += CB) {
-                                float4 a0[CB], a1[CB], b0[CB], b1[CB];
-#pragma unroll
-                                for (int t = 0; t < CB; ++t) {
-                                    const float* p = scratch + slot_off[i + t];
-                                    a0[t] = __ldcg(reinterpret_cast<const float4*>(p + og0));
-                                    a1[t] = __ldcg(reinterpret_cast<const float4*>(p + og1));
-                                    if (GATEUP) {
-                                        b0[t] = __ldcg(reinterpret_cast<const float4*>(p + og0 + du));
-                                        b1[t] = __ldcg(reinterpret_cast<const float4*>(p + og1 + du));
-                                    }
-                                }
-#pragma unroll
-                                for (int t = 0; t < CB; ++t) {
-                                    add4(g0, a0[t]); add4(g1, a1[t]);
-                                    if (GATEUP) { add4(u0, b0[t]); add4(u1, b1[t]); }
-                                }
-                            }
-                            for (; i < ncontrib; ++i) {
-                                const float* p = scratch + slot_off[i];
-                                add4(g0, __ldcg(reinterpret_cast<const float4*>(p + og0)));
-                                add4(g1, __ldcg(reinterpret_cast<const float4*>(p + og1)));
-                                if (GATEUP) {
-                                    add4(u0, __ldcg(reinterpret_cast<const float4*>(p + og0 + du)));
-                                    add4(u1, __ldcg(reinterpret_cast<const float4*>(p + og1 + du)));
-                                }
-                            }
-                            auto finish = [&](const float4& g, const float4& uu, int mm) {
-                                float v[4] = {g.x, g.y, g.z, g.w};
-                                if (GATEUP) {
-                                    v[0] = silu_f32(g.x) * uu.x; v[1] = silu_f32(g.y) * uu.y;
-                                    v[2] = silu_f32(g.z) * uu.z; v[3] = silu_f32(g.w) * uu.w;
-                                }
-                                // N is a multiple of 8 and n of 4: the four columns are all inside or all outside
-                                *reinterpret_cast<uint2*>(out + (size_t)mm * N + n) =
-                                    make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
-                            };
-                            finish(g0, u0, m);
-                            if (two) finish(g1, u1, m + 4);
-                        }
-                    }
-                    if (et == 0) counters[tile] = 0u;        // clean for the next call
-                }
-            }
+            skinny_epilogue_segment<GATEUP, NH>(tmem_base + lane_base + acc_col(buf, 0, 0), tempty0 + 8 * buf, tile,
+                                                tile == (int)(u_begin / KB), blockIdx.x, total, parts, KB, M, Mpad, N,
+                                                scratch, counters, out, slot_off, last_flag, et, nl, lane);
             u = seg_end;
         }
     }
