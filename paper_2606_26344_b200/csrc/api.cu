@@ -326,6 +326,16 @@ int run_stream(DeviceState* dev, const Layout& L, uint8_t* ws, const bf16* A, co
     return rc;
 }
 
+// Tile width for the plain (down) GEMM: 256 columns unless the grid would be so small, or the last round so
+// empty, that 128-column tiles (about 0.75 of the cost each, measured) finish sooner.
+int pick_umma_boxes(int64_t num_m, int64_t N, int sms) {
+    const int64_t t256 = num_m * ((N + 255) / 256), t128 = num_m * ((N + 127) / 128);
+    const double c256 = (double)((t256 + sms - 1) / sms), c128 = 0.75 * (double)((t128 + sms - 1) / sms);
+    int nb = c128 < c256 ? 2 : 4;
+    if (const char* e = getenv("GMLP_UMMA_NB")) { if (e[0] == '2') nb = 2; if (e[0] == '4') nb = 4; }   // tuning override
+    return nb;
+}
+
 template <bool GATEUP>
 int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
                 int64_t M, int64_t K, int64_t N, cudaStream_t st) {
@@ -338,18 +348,19 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
         tmB1 = tmB0;
     }
     if (!dev->umma_attr_set) {
-        if (cudaFuncSetAttribute(gmlp::umma_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)gmlp::kUmmaSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(gmlp::umma_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)gmlp::kUmmaSmemBytes) != cudaSuccess)
+        const int b = (int)gmlp::kUmmaSmemBytes;
+        if (cudaFuncSetAttribute(gmlp::umma_gemm_kernel<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::umma_gemm_kernel<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::umma_gemm_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess)
             return GMLP_ERR_LAUNCH;
         dev->umma_attr_set = true;
     }
-    const int bn = GATEUP ? 128 : 256;
+    const int sms = dev->sm_count > 0 ? dev->sm_count : 148;
     const int num_m = (int)((M + gmlp::kUmmaBM - 1) / gmlp::kUmmaBM);
+    const int nb = GATEUP ? 4 : pick_umma_boxes(num_m, N, sms);
+    const int bn = GATEUP ? 128 : 64 * nb;
     const int num_n = (int)((N + bn - 1) / bn);
     const int num_tiles = num_m * num_n;
-    const int sms = dev->sm_count > 0 ? dev->sm_count : 148;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(num_tiles < sms ? num_tiles : sms));     // persistent: one CTA per SM
     cfg.blockDim = dim3(gmlp::kUmmaThreads);
@@ -360,9 +371,15 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<GATEUP>, tmA, tmB0, tmB1, C, (int)M, (int)K, (int)N, num_m,
-                           num_tiles) != cudaSuccess)
-        return GMLP_ERR_LAUNCH;
+    const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
+    cudaError_t err;
+    if (GATEUP)
+        err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles);
+    else if (nb == 4)
+        err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles);
+    else
+        err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles);
+    if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
 }

@@ -38,11 +38,11 @@ constexpr uint32_t kUmmaBoxBBytes = 64 * kUmmaBK * 2;            // 8 KB: 64 k-r
 constexpr uint32_t kUmmaBBytes = 4 * kUmmaBoxBBytes;             // 32 KB
 constexpr uint32_t kUmmaStageBytes = kUmmaABytes + kUmmaBBytes;  // 48 KB
 constexpr uint32_t kUmmaSmemBytes = kUmmaStages * kUmmaStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+// stages for a kernel with NB weight boxes per stage: the ring fills the same shared-memory budget
+__host__ __device__ constexpr int umma_stages(int nb) {
+    return (int)((kUmmaStages * kUmmaStageBytes) / (kUmmaABytes + nb * kUmmaBoxBBytes));
+}
 constexpr long long kWaitLimitCycles = 2000000000LL;             // about a second
-
-// kind::f16 instruction descriptor: D = fp32, A = B = bf16, A K-major, B MN-major, M = 128, N = 256.
-constexpr uint32_t kUmmaIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
-                                ((uint32_t)(kUmmaN >> 3) << 17) | ((uint32_t)(kUmmaBM >> 4) << 24);
 
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                              int kernel_id, int site) {
@@ -59,25 +59,33 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
     return true;
 }
 
-template <bool GATEUP>
+// NB = 64-column weight boxes per stage: 4 -> MMA N = 256 (the default), 2 -> MMA N = 128 (smaller tiles for
+// shapes that would otherwise leave most SMs without a tile; more stages, lower arithmetic intensity).
+template <bool GATEUP, int NB>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
                  int M, int K, int N, int num_m_tiles, int num_tiles)
 {
     constexpr int KERNEL_ID = GATEUP ? 1 : 2;
-    constexpr int BN_OUT = GATEUP ? 128 : 256;
+    constexpr int N_MMA = 64 * NB;
+    constexpr int BN_OUT = GATEUP ? N_MMA / 2 : N_MMA;
+    constexpr int kStages = umma_stages(NB);
+    constexpr uint32_t kStageBytes = kUmmaABytes + NB * kUmmaBoxBBytes;
+    // kind::f16 instruction descriptor: D = fp32, A = B = bf16, A K-major, B MN-major, M = 128, N = N_MMA
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                                ((uint32_t)(N_MMA >> 3) << 17) | ((uint32_t)(kUmmaBM >> 4) << 24);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;            // swizzle atoms need 1024-byte alignment
     uint8_t* base_ptr = smem_raw + (base - raw_addr);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + kUmmaStages * kUmmaStageBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + kStages * kStageBytes);
     const uint32_t full0 = ptx::smem_addr(bars);
-    const uint32_t empty0 = ptx::smem_addr(bars + kUmmaStages);
-    const uint32_t tfull0 = ptx::smem_addr(bars + 2 * kUmmaStages);          // accumulator buffer b is complete
-    const uint32_t tempty0 = ptx::smem_addr(bars + 2 * kUmmaStages + 2);     // accumulator buffer b has been read out
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kUmmaStages + 4);
+    const uint32_t empty0 = ptx::smem_addr(bars + kStages);
+    const uint32_t tfull0 = ptx::smem_addr(bars + 2 * kStages);          // accumulator buffer b is complete
+    const uint32_t tempty0 = ptx::smem_addr(bars + 2 * kStages + 2);     // accumulator buffer b has been read out
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -85,7 +93,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     ptx::launch_dependents();
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kUmmaStages; ++s) {
+        for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(full0 + 8 * s, 1);
             ptx::mbar_init(empty0 + 8 * s, 1);
         }
@@ -121,18 +129,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int m0 = (tile % num_m_tiles) * kUmmaBM;
                 const int n0 = (tile / num_m_tiles) * BN_OUT;
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % kUmmaStages;
-                    const uint32_t ph = (uint32_t)(it / kUmmaStages) & 1u;
+                    const int s = it % kStages;
+                    const uint32_t ph = (uint32_t)(it / kStages) & 1u;
                     if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) { ok = false; break; }
                     const uint32_t full = full0 + 8 * s;
-                    const uint32_t a_dst = base + s * kUmmaStageBytes;
+                    const uint32_t a_dst = base + s * kStageBytes;
                     const uint32_t b_dst = a_dst + kUmmaABytes;
-                    ptx::mbar_arrive_expect_tx(full, kUmmaStageBytes);
+                    ptx::mbar_arrive_expect_tx(full, kStageBytes);
                     ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const CUtensorMap* map = (GATEUP && i >= 2) ? &tmB1 : &tmB0;
-                        const int x = GATEUP ? n0 + (i & 1) * 64 : n0 + i * 64;
+                    for (int i = 0; i < NB; ++i) {
+                        // gate/up: the first NB/2 boxes are gate columns, the rest the same columns of up
+                        const CUtensorMap* map = (GATEUP && i >= NB / 2) ? &tmB1 : &tmB0;
+                        const int x = GATEUP ? n0 + (i % (NB / 2)) * 64 : n0 + i * 64;
                         ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
                     }
                 }
@@ -151,11 +160,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kUmmaN);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % kUmmaStages;
-                    const uint32_t ph = (uint32_t)(it / kUmmaStages) & 1u;
+                    const int s = it % kStages;
+                    const uint32_t ph = (uint32_t)(it / kStages) & 1u;
                     if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
-                    const uint32_t a_base = base + s * kUmmaStageBytes;
+                    const uint32_t a_base = base + s * kStageBytes;
                     const uint32_t b_base = a_base + kUmmaABytes;
 #pragma unroll
                     for (int k = 0; k < kUmmaBK / 16; ++k) {
@@ -164,7 +173,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         //    K = 16 is two k-groups: +2048 B per step.
                         const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
                         const uint64_t b_desc = ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
-                        ptx::umma_bf16(d_tmem, a_desc, b_desc, kUmmaIdesc, (kb | k) != 0 ? 1u : 0u);
+                        ptx::umma_bf16(d_tmem, a_desc, b_desc, kIdesc, (kb | k) != 0 ? 1u : 0u);
                     }
                     ptx::umma_commit(empty0 + 8 * s);      // stage is free once these MMAs have read it
                 }
@@ -193,7 +202,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (GATEUP) {
                     uint32_t u[32];
                     ptx::tmem_ld_32x32(taddr + c, g);
-                    ptx::tmem_ld_32x32(taddr + 128 + c, u);
+                    ptx::tmem_ld_32x32(taddr + N_MMA / 2 + c, u);
                     ptx::tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
