@@ -13,6 +13,7 @@
 #include "simt_gemm.cuh"
 #include "stream_small_m.cuh"
 #include "umma_gemm.cuh"
+#include "umma_gemm_2cta.cuh"
 #include "umma_skinny.cuh"
 
 namespace {
@@ -74,6 +75,7 @@ struct DeviceState {
     void* workspace = nullptr;
     uint64_t workspace_bytes = 0;
     bool umma_attr_set = false;
+    bool pair_attr_set = false;
     bool skinny_attr_set = false;
     // arrival counters last zeroed by the library (the kernels leave them zero after every call)
     const void* clean_counters = nullptr;
@@ -336,9 +338,62 @@ int pick_umma_boxes(int64_t num_m, int64_t N, int sms) {
     return nb;
 }
 
+// CTA-pair (cta_group::2) schedule: pair tiles of 256 rows.
+bool use_pair_schedule(int64_t M) {
+    bool on = M >= 1024;
+    if (const char* e = getenv("GMLP_UMMA_PAIR")) on = (e[0] == '1');      // tuning override
+    return on;
+}
+
+template <bool GATEUP>
+int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
+                     int64_t M, int64_t K, int64_t N, cudaStream_t st) {
+    CUtensorMap tmA, tmB0, tmB1;
+    if (!encode_2d(&tmA, A, (uint64_t)K, (uint64_t)M, gmlp::kUmmaBK, 128)) return GMLP_ERR_LAUNCH;
+    if (!encode_2d(&tmB0, W0, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
+    if (GATEUP) {
+        if (!encode_2d(&tmB1, W1, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
+    } else {
+        tmB1 = tmB0;
+    }
+    if (!dev->pair_attr_set) {
+        const int b = (int)gmlp::kPairSmemBytes;
+        if (cudaFuncSetAttribute(gmlp::umma_pair_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::umma_pair_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess)
+            return GMLP_ERR_LAUNCH;
+        dev->pair_attr_set = true;
+    }
+    const int sms = dev->sm_count > 0 ? dev->sm_count : 148;
+    const int num_m = (int)((M + 255) / 256);
+    const int bn = GATEUP ? 128 : 256;
+    const int num_tiles = num_m * (int)((N + bn - 1) / bn);
+    const int pairs = num_tiles < sms / 2 ? num_tiles : sms / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    cfg.blockDim = dim3(gmlp::kUmmaThreads);
+    cfg.dynamicSmemBytes = gmlp::kPairSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
+    if (cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles) !=
+        cudaSuccess)
+        return GMLP_ERR_LAUNCH;
+    GMLP_CHECK_LAUNCH();
+    return GMLP_OK;
+}
+
 template <bool GATEUP>
 int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
                 int64_t M, int64_t K, int64_t N, cudaStream_t st) {
+    if (use_pair_schedule(M)) return launch_umma_pair<GATEUP>(dev, A, W0, W1, C, M, K, N, st);
     CUtensorMap tmA, tmB0, tmB1;
     if (!encode_2d(&tmA, A, (uint64_t)K, (uint64_t)M, gmlp::kUmmaBK, gmlp::kUmmaBM)) return GMLP_ERR_LAUNCH;
     if (!encode_2d(&tmB0, W0, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;

@@ -1,0 +1,263 @@
+// Large-M schedule on CTA pairs: the same two GEMMs as umma_gemm.cuh, issued as
+// tcgen05.mma.cta_group::2 by thread-block clusters of two CTAs (the two SMs of a TPC).
+//
+// One pair tile = 256 rows x 256 MMA columns (gate/up: 128 gate + 128 up columns of H; down: 256
+// columns of Y).  CTA r of the pair holds rows [128 r, 128 r + 128) of A and HALF of the B columns
+// (gate/up: CTA 0 the gate columns, CTA 1 the up columns; down: columns [128 r, 128 r + 128)), so a
+// stage is 16 KB of A + 16 KB of B per CTA instead of 16 + 32: the ring is six stages deep and the
+// shared-memory fill per MMA cycle drops from 96 to 64 bytes.  No TMA multicast is involved: each
+// CTA loads its own halves; the tensor cores of the pair read B from both CTAs' shared memory.
+//
+// Only the leader (cluster rank 0) issues MMAs.  Barriers:
+//   full[s]   (leader's)  two arrivals: each CTA's producer arms its own 32 KB; both CTAs' TMA loads
+//                         complete on it (the peer's through .cta_group::2 addressing)
+//   empty[s]  (per CTA)   tcgen05.commit multicast to both CTAs when the stage's MMAs are done
+//   tfull[b]  (per CTA)   tcgen05.commit multicast: accumulator buffer b is complete
+//   tempty[b] (leader's)  eight arrivals: the four epilogue warps of both CTAs have drained buffer b
+// Each CTA's TMEM holds its 128 rows x 256 columns, two buffers; the epilogue is the one of
+// umma_gemm.cuh.  Every wait is bounded; the pair leaves through a cluster barrier so that neither
+// CTA's shared memory or TMEM disappears under the other.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+#include "umma_gemm.cuh"
+
+namespace gmlp {
+
+constexpr int kPairStages = 6;
+constexpr uint32_t kPairABytes = 128 * kUmmaBK * 2;               // 16 KB: this CTA's 128 rows
+constexpr uint32_t kPairBBytes = 2 * kUmmaBoxBBytes;              // 16 KB: this CTA's 128 columns
+constexpr uint32_t kPairStageBytes = kPairABytes + kPairBBytes;   // 32 KB per CTA
+constexpr uint32_t kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + 256;
+
+namespace ptx {
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr_local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr_local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t bar_cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(bar_cluster_addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// TMA load whose completion is counted on a barrier that may live in the pair's other CTA (no multicast)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const void* tmap, int x, int y, uint32_t bar_cluster_addr) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst_smem), "l"(tmap), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// one arrival on the barrier at this shared-memory offset in BOTH CTAs once the MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+}  // namespace ptx
+
+template <bool GATEUP>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+                      const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
+                      int M, int K, int N, int num_m_tiles, int num_tiles)
+{
+    constexpr int KERNEL_ID = GATEUP ? 6 : 7;
+    constexpr int BN_OUT = GATEUP ? 128 : 256;
+    // D = fp32, A = B = bf16, A K-major, B MN-major, M = 256 (128 per CTA), N = 256
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                                ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;            // identical in both CTAs of the pair
+    uint8_t* base_ptr = smem_raw + (base - raw_addr);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + kPairStages * kPairStageBytes);
+    const uint32_t full0 = ptx::smem_addr(bars);
+    const uint32_t empty0 = ptx::smem_addr(bars + kPairStages);
+    const uint32_t tfull0 = ptx::smem_addr(bars + 2 * kPairStages);
+    const uint32_t tempty0 = ptx::smem_addr(bars + 2 * kPairStages + 2);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kPairStages + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();                 // 0 = leader
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_kb = (K + kUmmaBK - 1) / kUmmaBK;
+
+    ptx::launch_dependents();
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairStages; ++s) {
+            ptx::mbar_init(full0 + 8 * s, 2);                     // one arming arrival per CTA (used in the leader)
+            ptx::mbar_init(empty0 + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(tfull0 + 8 * b, 1);
+            ptx::mbar_init(tempty0 + 8 * b, 8);                   // four epilogue warps of each CTA (used in the leader)
+        }
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::fence_proxy_async_smem();
+        ptx::prefetch_tensormap(&tmA);
+        ptx::prefetch_tensormap(&tmB0);
+        if (GATEUP) ptx::prefetch_tensormap(&tmB1);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(ptx::smem_addr(tmem_slot), kUmmaTmemCols);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();                                          // the peer's barriers exist before anyone signals them
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer (both CTAs) ----------------
+        if (lane == 0) {
+            ptx::grid_dependency_wait();
+            const uint32_t leader_full0 = ptx::map_to_cta(full0, 0);
+            int it = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+                const int m0 = (tile % num_m_tiles) * 256 + (int)rank * 128;
+                const int n0 = (tile / num_m_tiles) * BN_OUT;
+                // this CTA's half of the B columns: gate/up -> gate (rank 0) or up (rank 1) columns n0..n0+127
+                const CUtensorMap* bmap = (GATEUP && rank == 1) ? &tmB1 : &tmB0;
+                const int bx = GATEUP ? n0 : n0 + (int)rank * 128;
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % kPairStages;
+                    const uint32_t ph = (uint32_t)(it / kPairStages) & 1u;
+                    if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) { ok = false; break; }
+                    const uint32_t full = leader_full0 + 8 * s;
+                    const uint32_t a_dst = base + s * kPairStageBytes;
+                    const uint32_t b_dst = a_dst + kPairABytes;
+                    ptx::mbar_arrive_expect_tx_cluster(full, kPairStageBytes);
+                    ptx::tma_load_2d_pair(a_dst, &tmA, kb * kUmmaBK, m0, full);
+                    ptx::tma_load_2d_pair(b_dst, bmap, bx, kb * kUmmaBK, full);
+                    ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, bx + 64, kb * kUmmaBK, full);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (leader only) ----------------
+        if (lane == 0 && rank == 0) {
+            int it = 0, t = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++t) {
+                const int buf = t & 1;
+                if (!wait_bounded(tempty0 + 8 * buf, (((uint32_t)t >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4)) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % kPairStages;
+                    const uint32_t ph = (uint32_t)(it / kPairStages) & 1u;
+                    if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_base = base + s * kPairStageBytes;
+                    const uint32_t b_base = a_base + kPairABytes;
+#pragma unroll
+                    for (int k = 0; k < kUmmaBK / 16; ++k) {
+                        const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
+                        const uint64_t b_desc = ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
+                        ptx::umma_bf16_pair(d_tmem, a_desc, b_desc, kIdesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    ptx::umma_commit_pair(empty0 + 8 * s);
+                }
+                if (ok) ptx::umma_commit_pair(tfull0 + 8 * buf);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue (both CTAs, own 128 rows) ----------------
+        const int q = warp & 3;
+        ptx::grid_dependency_wait();
+        const uint32_t leader_tempty0 = ptx::map_to_cta(tempty0, 0);
+        int t = 0;
+        for (int tile = pair; tile < num_tiles; tile += num_pairs, ++t) {
+            const int buf = t & 1;
+            const int m0 = (tile % num_m_tiles) * 256 + (int)rank * 128;
+            const int n0 = (tile / num_m_tiles) * BN_OUT;
+            const int row = m0 + q * 32 + lane;
+            if (!wait_bounded(tfull0 + 8 * buf, ((uint32_t)t >> 1) & 1u, abort_flag, KERNEL_ID, 3)) break;
+            ptx::tc_fence_after_sync();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256);
+            bf16* crow = C + (size_t)row * N + n0;
+#pragma unroll 1
+            for (int c = 0; c < BN_OUT; c += 32) {
+                uint32_t g[32];
+                uint32_t packed[16];
+                if (GATEUP) {
+                    uint32_t u[32];
+                    ptx::tmem_ld_32x32(taddr + c, g);
+                    ptx::tmem_ld_32x32(taddr + 128 + c, u);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float h0 = silu_f32(__uint_as_float(g[2 * j])) * __uint_as_float(u[2 * j]);
+                        const float h1 = silu_f32(__uint_as_float(g[2 * j + 1])) * __uint_as_float(u[2 * j + 1]);
+                        packed[j] = pack_bf16x2(h0, h1);
+                    }
+                } else {
+                    ptx::tmem_ld_32x32(taddr + c, g);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        packed[j] = pack_bf16x2(__uint_as_float(g[2 * j]), __uint_as_float(g[2 * j + 1]));
+                }
+                if (row < M) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        if (n0 + c + v * 8 < N)
+                            *reinterpret_cast<uint4*>(crow + c + v * 8) =
+                                make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                    }
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty0 + 8 * buf);
+        }
+    }
+
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();                       // the peer may still be reading this CTA's shared memory through the MMA
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc_pair(tmem_base, kUmmaTmemCols);
+    }
+}
+
+}  // namespace gmlp
