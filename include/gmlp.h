@@ -67,8 +67,9 @@ enum {
     GMLP_VARIANT_AUTO = 0,
     GMLP_VARIANT_SIMT = 1,   /* CUDA-core tiled GEMMs: any shape, slow; bring-up and cross-check */
     GMLP_VARIANT_STREAM = 2, /* small M: weight-streaming split-K kernels on CUDA cores (HBM-bound regime) */
-    GMLP_VARIANT_UMMA = 3,   /* large M: tcgen05 tensor-core GEMMs fed by TMA, accumulators in TMEM */
-    GMLP_VARIANT_SKINNY = 4  /* M <= 128: operand-swapped tcgen05 GEMMs, stream-K over all SMs (HBM-bound regime) */
+    GMLP_VARIANT_UMMA = 3,   /* medium M: tcgen05 tensor-core GEMMs fed by TMA, accumulators in TMEM, one CTA per tile */
+    GMLP_VARIANT_SKINNY = 4, /* M <= 128: operand-swapped tcgen05 GEMMs, stream-K over all SMs (HBM-bound regime) */
+    GMLP_VARIANT_PAIR = 5    /* large M: the same GEMMs on CTA pairs (tcgen05 cta_group::2, 256-row tiles) */
 };
 
 typedef struct gmlp_args {
@@ -149,7 +150,7 @@ int gmlp_forward_static(const void* X, const void* Wg, const void* Wu, const voi
  */
 uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant);
 
-/* The schedule AUTO resolves to for this shape (one of GMLP_VARIANT_SIMT/STREAM/UMMA/SKINNY). */
+/* The schedule AUTO resolves to for this shape (GMLP_VARIANT_SKINNY, _UMMA or _PAIR). */
 int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);
 
 /*

@@ -202,7 +202,8 @@ struct Layout {
 
 int resolve_variant(int64_t M, int32_t variant) {
     if (variant != GMLP_VARIANT_AUTO) return variant;
-    return M <= 128 ? GMLP_VARIANT_SKINNY : GMLP_VARIANT_UMMA;
+    if (M <= 128) return GMLP_VARIANT_SKINNY;
+    return M < 1024 ? GMLP_VARIANT_UMMA : GMLP_VARIANT_PAIR;
 }
 
 Layout make_layout(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int variant, int sm_count) {
@@ -338,13 +339,6 @@ int pick_umma_boxes(int64_t num_m, int64_t N, int sms) {
     return nb;
 }
 
-// CTA-pair (cta_group::2) schedule: pair tiles of 256 rows.
-bool use_pair_schedule(int64_t M) {
-    bool on = M >= 1024;
-    if (const char* e = getenv("GMLP_UMMA_PAIR")) on = (e[0] == '1');      // tuning override
-    return on;
-}
-
 template <bool GATEUP>
 int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
                      int64_t M, int64_t K, int64_t N, cudaStream_t st) {
@@ -393,7 +387,6 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
 template <bool GATEUP>
 int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
                 int64_t M, int64_t K, int64_t N, cudaStream_t st) {
-    if (use_pair_schedule(M)) return launch_umma_pair<GATEUP>(dev, A, W0, W1, C, M, K, N, st);
     CUtensorMap tmA, tmB0, tmB1;
     if (!encode_2d(&tmA, A, (uint64_t)K, (uint64_t)M, gmlp::kUmmaBK, gmlp::kUmmaBM)) return GMLP_ERR_LAUNCH;
     if (!encode_2d(&tmB0, W0, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
@@ -517,7 +510,7 @@ int forward_impl(const gmlp_args* a) {
     if (a == nullptr) return GMLP_ERR_NULL;
     if (a->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
     if (a->flags & ~kKnownFlags) return GMLP_ERR_FLAGS;
-    if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_SKINNY) return GMLP_ERR_FLAGS;
+    if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_PAIR) return GMLP_ERR_FLAGS;
     int rc = check_shape(a->M, a->d_model, a->d_ff);
     if (rc != GMLP_OK) return rc;
     if (a->M == 0) return GMLP_OK;              // nothing to compute; pointers may be NULL
@@ -587,6 +580,14 @@ int forward_impl(const gmlp_args* a) {
             break;
         case GMLP_VARIANT_SKINNY:
             rc = run_skinny(dev, L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
+            break;
+        case GMLP_VARIANT_PAIR:
+            rc = launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st);
+            if (rc == GMLP_OK) {
+                prof_mark("gate_up", st);
+                rc = launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st);
+                if (rc == GMLP_OK) prof_mark("down", st);
+            }
             break;
         default:
             rc = launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st);
@@ -726,7 +727,7 @@ int gmlp_forward_host(const gmlp_args* args, const void* X_host, void* Y_host) {
 
 uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant) {
     if (check_shape(M, d_model, d_ff) != GMLP_OK) return 0;
-    if (variant < GMLP_VARIANT_AUTO || variant > GMLP_VARIANT_SKINNY) return 0;
+    if (variant < GMLP_VARIANT_AUTO || variant > GMLP_VARIANT_PAIR) return 0;
     int sm_count = 148;
     int dev = -1;
     if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) {

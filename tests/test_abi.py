@@ -98,8 +98,9 @@ def test_workspace_sizes_and_variant_choice(lib):
     assert gmlp.pick_variant(1, 2048, 5632) == gmlp.VARIANT_SKINNY
     assert gmlp.pick_variant(128, 2048, 5632) == gmlp.VARIANT_SKINNY
     assert gmlp.pick_variant(129, 2048, 5632) == gmlp.VARIANT_UMMA
-    assert gmlp.pick_variant(2048, dm, dff) == gmlp.VARIANT_UMMA
-    assert gmlp.pick_variant(4096, 8192, 28672) == gmlp.VARIANT_UMMA
+    assert gmlp.pick_variant(1000, 2048, 5632) == gmlp.VARIANT_UMMA
+    assert gmlp.pick_variant(2048, dm, dff) == gmlp.VARIANT_PAIR
+    assert gmlp.pick_variant(4096, 8192, 28672) == gmlp.VARIANT_PAIR
     assert gmlp.pick_variant(4, 60, 128) == gmlp.ERR_SHAPE
 
 

@@ -13,11 +13,12 @@ from _parity import check_case, err_over_tol, gpu_forward, oracle_rows, to_devic
 
 pytestmark = pytest.mark.gpu
 
-SIMT, STREAM, UMMA, SKINNY = gmlp.VARIANT_SIMT, gmlp.VARIANT_STREAM, gmlp.VARIANT_UMMA, gmlp.VARIANT_SKINNY
+SIMT, STREAM, UMMA, SKINNY, PAIR = (gmlp.VARIANT_SIMT, gmlp.VARIANT_STREAM, gmlp.VARIANT_UMMA, gmlp.VARIANT_SKINNY,
+                                     gmlp.VARIANT_PAIR)
 
 
 # ---------------------------------------------------------------- small cases, every schedule
-@pytest.mark.parametrize("variant", [SIMT, STREAM, UMMA, SKINNY])
+@pytest.mark.parametrize("variant", [SIMT, STREAM, UMMA, SKINNY, PAIR])
 def test_tiny_config_all_rows(variant):
     inp = I.make_inputs(I.WORKLOADS["tiny"])
     check_case(inp, variant, f"tiny/v{variant}")
@@ -91,8 +92,18 @@ def test_skinny_rejects_more_than_128_rows():
     assert ei.value.status == gmlp.ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("rmsnorm", [False, True])
+@pytest.mark.parametrize("shape", [(256, 64, 256), (1, 64, 128), (129, 320, 392), (257, 1096, 648), (300, 512, 1024),
+                                   (640, 256, 2048), (1300, 264, 520)])
+def test_pair_schedule_tiles_and_ragged_tails(shape, rmsnorm):
+    # CTA-pair kernel: row counts around the 128-row CTA half and the 256-row pair tile, column counts
+    # that do not fill a CTA's 128-column half, K tails, more pair tiles than CTA pairs (1300 rows)
+    M, dm, dff = shape
+    check_case(I.custom_inputs(M, dm, dff, 500 + M, rmsnorm=rmsnorm, eps=1e-5), PAIR, f"pair{shape}")
+
+
 # ---------------------------------------------------------------- structured inputs that expose layout mistakes
-@pytest.mark.parametrize("variant", [SIMT, STREAM, UMMA, SKINNY])
+@pytest.mark.parametrize("variant", [SIMT, STREAM, UMMA, SKINNY, PAIR])
 def test_one_hot_weights_closed_form(variant):
     # Wg[n mod dm, n] = 1, Wu[(n+1) mod dm, n] = 1, Wd[n, c] = [n == c]:
     #   Y[m, c] = bf16(silu(x[m, c mod dm]) * x[m, (c+1) mod dm])  for c < min(d_ff, d_model)
@@ -114,7 +125,7 @@ def test_one_hot_weights_closed_form(variant):
     assert ((Y.double() - want).abs() <= want.abs() * 2.0 ** -7 + 1e-30).all()
 
 
-@pytest.mark.parametrize("variant", [SIMT, STREAM, UMMA, SKINNY])
+@pytest.mark.parametrize("variant", [SIMT, STREAM, UMMA, SKINNY, PAIR])
 def test_integer_inputs_with_exact_preactivations(variant):
     # Small integers make G and U exact in fp32 and fp64 alike, so what is left to differ is the SiLU
     # approximation and the roundings.  Each weight column has four entries of +-1 and X lies in
@@ -166,7 +177,7 @@ def test_workspace_too_small_is_rejected_and_results_are_deterministic():
     with pytest.raises(gmlp.GmlpError) as ei:
         gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], Y, workspace=small)
     assert ei.value.status == gmlp.ERR_WORKSPACE
-    for variant, M in ((STREAM, 8), (SKINNY, 40), (UMMA, 40), (SIMT, 40)):
+    for variant, M in ((STREAM, 8), (SKINNY, 40), (UMMA, 40), (PAIR, 40), (SIMT, 40)):
         a = gmlp.forward(t["X"][:M].contiguous(), t["Wg"], t["Wu"], t["Wd"], variant=variant).clone()
         b = gmlp.forward(t["X"][:M].contiguous(), t["Wg"], t["Wu"], t["Wd"], variant=variant).clone()
         torch.cuda.synchronize()
@@ -191,9 +202,10 @@ def test_schedules_agree_on_the_whole_output():
     # the slow CUDA-core schedule and the tensor-core schedule on every element of a mid-size case
     inp = I.custom_inputs(520, 1024, 2816, 8, rmsnorm=True)
     a = gpu_forward(inp, SIMT).float()
-    b = gpu_forward(inp, UMMA).float()
     tol = 2e-2 * torch.clamp(a.abs(), min=1.0)
-    assert ((a - b).abs() <= tol).all()
+    for variant in (UMMA, PAIR):
+        b = gpu_forward(inp, variant).float()
+        assert ((a - b).abs() <= tol).all()
 
 
 def test_silu_on_device_over_a_dense_sweep():
@@ -207,7 +219,7 @@ def test_silu_on_device_over_a_dense_sweep():
     Wu = torch.zeros(dm, dff); Wu[1, :] = 1.0
     Wd = torch.eye(dff, dm)
     inp.X, inp.Wg, inp.Wu, inp.Wd = X.bfloat16(), Wg.bfloat16(), Wu.bfloat16(), Wd.bfloat16()
-    for variant in (SIMT, UMMA):
+    for variant in (SIMT, UMMA, PAIR):
         Y = gpu_forward(inp, variant).float().cpu()
         assert torch.isfinite(Y).all()
         want = oracle.silu(gs.double().numpy())
