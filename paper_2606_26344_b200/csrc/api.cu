@@ -162,6 +162,7 @@ StreamPlan make_stream_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
 // ------------------------------------------------------------------ skinny (swap-AB tcgen05) plan
 struct SkinnyPlan {
     int Mpad, NH, num_tiles, KB, stages, grid;
+    uint32_t smem_bytes;
     uint32_t tmem_cols;
     uint64_t scratch_bytes;
 };
@@ -170,16 +171,24 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
     SkinnyPlan p;
     p.Mpad = (int)((M + 15) / 16 * 16);
     if (p.Mpad < 16) p.Mpad = 16;
-    p.NH = (N >= 256 && 2 * nmat * 2 * p.Mpad <= 512) ? 2 : 1;
+    // Few tokens: half-size shared-memory rings (112 KB), so that the next kernel on the stream - launched with
+    // programmatic stream serialization - is co-resident on every SM and has its weight ring full by the time
+    // this one drains.  The gate/up kernel then uses 128-column tiles (34 KB stages), the down kernel 256.
+    const bool small = p.Mpad <= 32;
+    p.NH = (N >= 256 && 2 * nmat * 2 * p.Mpad <= 512 && !(small && nmat == 2)) ? 2 : 1;
     if (const char* e = getenv(nmat == 2 ? "GMLP_SKINNY_NH1" : "GMLP_SKINNY_NH2")) {      // tuning override
         if (e[0] == '1') p.NH = 1;
+        if (e[0] == '2' && N >= 256 && 2 * nmat * 2 * p.Mpad <= 512) p.NH = 2;
     }
     const int tile_n = 128 * p.NH;
     p.num_tiles = (int)((N + tile_n - 1) / tile_n);
     p.KB = (int)((K + 63) / 64);
     const uint32_t stage_bytes = (uint32_t)nmat * p.NH * 2 * gmlp::kSkinnyBoxBytes + (uint32_t)p.Mpad * 128u;
-    int st = (int)((gmlp::kSkinnySmemBudget - 1024 - 256) / stage_bytes);
+    uint32_t budget = small ? gmlp::kSkinnySmemBudget / 2 : gmlp::kSkinnySmemBudget;
+    if (const char* e = getenv("GMLP_SKINNY_SMEM_KB")) { int v = atoi(e); if (v >= 48 && v <= 224) budget = (uint32_t)v * 1024u; }  // tuning override
+    int st = (int)((budget - 1024 - 256) / stage_bytes);
     p.stages = st > gmlp::kSkinnyMaxStages ? gmlp::kSkinnyMaxStages : st;
+    p.smem_bytes = (uint32_t)p.stages * stage_bytes + 1024 + 256;
     if (const char* e = getenv("GMLP_SKINNY_STAGES")) { int v = atoi(e); if (v >= 2 && v < p.stages) p.stages = v; }   // tuning override
     uint32_t cols = (uint32_t)(2 * nmat * p.NH * p.Mpad);
     uint32_t pow2 = 32;
@@ -458,7 +467,7 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);
     cfg.blockDim = dim3(gmlp::kSkinnyThreads);
-    cfg.dynamicSmemBytes = gmlp::kSkinnySmemBudget;
+    cfg.dynamicSmemBytes = p.smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
