@@ -160,6 +160,15 @@ int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);
  */
 int gmlp_device_status(void);
 
+/*
+ * Self-test of the device-side failure path: launches one tiny kernel whose bounded wait is bound to run
+ * out (it waits, for about a millisecond at most, on a barrier that nothing completes), synchronises, and
+ * checks that the device status word names that wait.  Nothing faults, traps or hangs; the context stays
+ * usable.  Returns GMLP_ERR_TIMEOUT when the time-out was detected and reported as designed (the
+ * expected outcome), GMLP_OK if the wait unexpectedly did not run out, or another GMLP_ERR_*.
+ */
+int gmlp_selftest_wait_timeout(void* stream);
+
 /* Number of kernels the library launched on this host thread since the last reset. */
 uint64_t gmlp_launch_count(void);
 void gmlp_reset_launch_count(void);

@@ -804,6 +804,22 @@ const char* gmlp_profile_kernel_name(int index) {
     return last.names[index];
 }
 
+int gmlp_selftest_wait_timeout(void* stream) {
+    int rc = GMLP_OK;
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    int s = read_device_status();                       // start from a clean status word
+    if (s < 0) return s;
+    gmlp::wait_timeout_probe_kernel<<<1, 32, 0, st>>>(2000000LL);      // about a millisecond
+    if (cudaPeekAtLastError() != cudaSuccess) return GMLP_ERR_LAUNCH;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    s = read_device_status();
+    if (s < 0) return s;
+    return s == ((99 << 16) | 1) ? GMLP_ERR_TIMEOUT : (s == 0 ? GMLP_OK : GMLP_ERR_LAUNCH);
+}
+
 uint64_t gmlp_launch_count(void) { return t_launches; }
 void gmlp_reset_launch_count(void) { t_launches = 0; }
 

@@ -45,18 +45,36 @@ __host__ __device__ constexpr int umma_stages(int nb) {
 constexpr long long kWaitLimitCycles = 2000000000LL;             // about a second
 
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                             int kernel_id, int site) {
+                                             int kernel_id, int site, long long limit_cycles = kWaitLimitCycles) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
     while (!ptx::mbar_try_wait(bar, parity)) {
         if (*abort_flag) return false;
-        if (clock64() - start > kWaitLimitCycles) {
+        if (clock64() - start > limit_cycles) {
             *abort_flag = 1;
             report_timeout(kernel_id, site);
             return false;
         }
     }
     return true;
+}
+
+// Self-test of the bounded wait: one warp waits on an mbarrier that nothing will ever complete, with a
+// short limit.  The wait gives up, records (kernel id 99, site 1) in the device status word and the kernel
+// returns normally; nothing traps, faults or spins without bound.
+__global__ void wait_timeout_probe_kernel(long long limit_cycles)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_addr(&bar), 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0)
+        (void)wait_bounded(ptx::smem_addr(&bar), 0u, &abort_flag, 99, 1, limit_cycles);
+    __syncthreads();
 }
 
 // NB = 64-column weight boxes per stage: 4 -> MMA N = 256 (the default), 2 -> MMA N = 128 (smaller tiles for

@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.gmlp_pick_variant.argtypes = [i64, i64, i64, u32]
         L.gmlp_device_status.restype = ctypes.c_int
         L.gmlp_device_status.argtypes = []
+        L.gmlp_selftest_wait_timeout.restype = ctypes.c_int
+        L.gmlp_selftest_wait_timeout.argtypes = [vp]
         L.gmlp_launch_count.restype = u64
         L.gmlp_launch_count.argtypes = []
         L.gmlp_reset_launch_count.restype = None
@@ -104,6 +106,12 @@ def pick_variant(M: int, d_model: int, d_ff: int, flags: int = 0) -> int:
 
 def device_status() -> int:
     return int(lib().gmlp_device_status())
+
+
+def selftest_wait_timeout() -> int:
+    """Runs the bounded-wait self-test on torch's current stream; ERR_TIMEOUT is the expected result."""
+    st = torch.cuda.current_stream()
+    return int(lib().gmlp_selftest_wait_timeout(st.cuda_stream))
 
 
 def launch_count() -> int:

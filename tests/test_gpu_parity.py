@@ -227,6 +227,45 @@ def test_silu_on_device_over_a_dense_sweep():
         assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -7 + 1e-30)
 
 
+def test_bounded_wait_reports_a_timeout_and_leaves_the_context_usable():
+    # failure detection without a fault: a wait that nothing will satisfy gives up after about a
+    # millisecond, the status word names it, and the next real call works and reports a clean status
+    assert gmlp.selftest_wait_timeout() == gmlp.ERR_TIMEOUT
+    assert gmlp.device_status() == 0
+    inp = I.make_inputs(I.WORKLOADS["tiny"])
+    check_case(inp, gmlp.VARIANT_AUTO, "after-timeout")
+    assert gmlp.device_status() == 0
+
+
+@pytest.mark.parametrize("variant,M", [(SKINNY, 7), (SKINNY, 100), (UMMA, 130), (UMMA, 300), (PAIR, 300), (PAIR, 1030),
+                                       (STREAM, 5), (SIMT, 70)])
+@pytest.mark.parametrize("rmsnorm", [False, True])
+def test_no_write_outside_y_and_workspace(variant, M, rmsnorm):
+    # Y and the workspace are carved out of one buffer with guard bands around them; the bands must be
+    # untouched after the call (ragged shapes: partial tiles in M, N and K).
+    dm, dff = 328, 712
+    inp = I.custom_inputs(M, dm, dff, 600 + M, rmsnorm=rmsnorm)
+    t = to_device(inp)
+    ws_bytes = gmlp.workspace_bytes(M, dm, dff, gmlp.FLAG_RMSNORM if rmsnorm else 0, variant)
+    guard = 4096
+    y_bytes = M * dm * 2
+    y_off = guard
+    ws_off = (y_off + y_bytes + guard + 255) // 256 * 256
+    total = ws_off + ws_bytes + guard
+    buf = torch.full((total,), 0x5A, dtype=torch.uint8, device="cuda")
+    Y = buf[y_off:y_off + y_bytes].view(torch.bfloat16).view(M, dm)
+    ws = buf[ws_off:ws_off + ws_bytes]
+    gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], Y, gamma=t["gamma"] if rmsnorm else None, eps=inp.workload.eps,
+                 rmsnorm=rmsnorm, variant=variant, workspace=ws, checked=True)
+    torch.cuda.synchronize()
+    assert bool((buf[:y_off] == 0x5A).all())
+    assert bool((buf[y_off + y_bytes:ws_off] == 0x5A).all())
+    assert bool((buf[ws_off + ws_bytes:] == 0x5A).all())
+    rows = np.arange(M)
+    e, _ = err_over_tol(Y, oracle_rows(inp, rows), rows)
+    assert e.max() <= 1.0
+
+
 # ---------------------------------------------------------------- the five stated configurations at full size
 @pytest.mark.parametrize("name", ["llama3-8b-decode-M8",
                                   "ragged-M1-plain", "ragged-M1-norm", "ragged-M7-plain", "ragged-M7-norm",
