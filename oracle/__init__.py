@@ -80,6 +80,10 @@ def _load():
         lib.gmlp_oracle_rows.argtypes = [u16p, u16p, u16p, u16p, u16p, ctypes.c_float, ctypes.c_int,
                                          ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                          i64p, ctypes.c_int64, f64p, u16p, u16p, ctypes.c_int]
+        lib.gmlp_oracle_gate_up_rows.restype = ctypes.c_int
+        lib.gmlp_oracle_gate_up_rows.argtypes = [u16p, u16p, u16p, u16p, ctypes.c_float, ctypes.c_int,
+                                                 ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                                 i64p, ctypes.c_int64, f64p, ctypes.c_int]
         lib.gmlp_oracle_bf16_rn_array.restype = None
         lib.gmlp_oracle_bf16_rn_array.argtypes = [f64p, u16p, ctypes.c_int64]
         lib.gmlp_oracle_silu_array.restype = None
@@ -181,6 +185,33 @@ def gmlp_rows(X, Wg, Wu, Wd, rows=None, gamma=None, eps: float = 1e-5, rmsnorm: 
     if want_xn:
         out.append(Xn)
     return out[0] if len(out) == 1 else tuple(out)
+
+
+def gate_up_rows(X, Wg, Wu, rows=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False,
+                 num_threads: int = 0) -> np.ndarray:
+    """Reference silu(Xn Wg) * (Xn Wu) (float64, not rounded) for the selected rows: the gate/up half alone."""
+    lib = _load()
+    X, Wg, Wu = _u16(X, "X"), _u16(Wg, "Wg"), _u16(Wu, "Wu")
+    M, d_model = X.shape
+    d_ff = Wg.shape[1]
+    if Wg.shape != (d_model, d_ff) or Wu.shape != (d_model, d_ff):
+        raise ValueError("shape mismatch")
+    if rows is None:
+        rows = np.arange(M, dtype=np.int64)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    g = None
+    if gamma is not None:
+        g = _u16(gamma, "gamma").reshape(-1)
+        if g.size != d_model:
+            raise ValueError("gamma size")
+    P = np.zeros((rows.size, d_ff), dtype=np.float64)
+    rc = lib.gmlp_oracle_gate_up_rows(_p(X, ctypes.c_uint16), _p(Wg, ctypes.c_uint16), _p(Wu, ctypes.c_uint16),
+                                      None if g is None else _p(g, ctypes.c_uint16), ctypes.c_float(eps),
+                                      int(bool(rmsnorm)), M, d_model, d_ff, _p(rows, ctypes.c_int64), rows.size,
+                                      _p(P, ctypes.c_double), int(num_threads))
+    if rc != 0:
+        raise RuntimeError(f"gmlp_oracle_gate_up_rows failed ({rc})")
+    return P
 
 
 def naive_matmul(A, B) -> np.ndarray:

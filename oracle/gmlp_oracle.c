@@ -180,6 +180,60 @@ int gmlp_oracle_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu, 
     return failed ? -1 : 0;
 }
 
+/*
+ * The gate/up half on its own ("Matmul+Matmul+SiLU+Mul" of the paper's benchmark list, Section 6.1):
+ *   P[i, n] = silu(sum_k xn[k] Wg[k, n]) * (sum_k xn[k] Wu[k, n])      for the selected rows,
+ * returned in fp64 WITHOUT the final rounding (the GPU rounds P once to bf16; the tolerance is taken
+ * around this value).  Same conventions as gmlp_oracle_rows; the optional RMSNorm prologue rounds Xn.
+ */
+int gmlp_oracle_gate_up_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu,
+                             const uint16_t* gamma, float eps, int rmsnorm,
+                             int64_t M, int64_t d_model, int64_t d_ff,
+                             const int64_t* rows, int64_t n_rows, double* P, int num_threads)
+{
+    if (!X || !Wg || !Wu || !rows || !P || M < 0 || d_model <= 0 || d_ff <= 0 || n_rows < 0) return -1;
+    for (int64_t i = 0; i < n_rows; ++i)
+        if (rows[i] < 0 || rows[i] >= M) return -1;
+    int failed = 0;
+#ifdef _OPENMP
+    if (num_threads > 0) omp_set_num_threads(num_threads);
+#else
+    (void)num_threads;
+#endif
+#pragma omp parallel
+    {
+        double* xn = (double*)malloc(sizeof(double) * (size_t)d_model);
+        uint16_t* xnb = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)d_model);
+        double* g = (double*)malloc(sizeof(double) * (size_t)d_ff);
+        double* u = (double*)malloc(sizeof(double) * (size_t)d_ff);
+        if (!xn || !xnb || !g || !u) {
+#pragma omp atomic write
+            failed = 1;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int64_t i = 0; i < n_rows; ++i) {
+                const uint16_t* x = X + rows[i] * d_model;
+                if (rmsnorm) gmlp_oracle_rmsnorm_row(x, gamma, eps, d_model, xnb, NULL);
+                else memcpy(xnb, x, sizeof(uint16_t) * (size_t)d_model);
+                for (int64_t k = 0; k < d_model; ++k) xn[k] = gmlp_oracle_bf16_to_double(xnb[k]);
+                for (int64_t n = 0; n < d_ff; ++n) { g[n] = 0.0; u[n] = 0.0; }
+                for (int64_t k = 0; k < d_model; ++k) {
+                    const double xk = xn[k];
+                    const uint16_t* wg = Wg + k * d_ff;
+                    const uint16_t* wu = Wu + k * d_ff;
+                    for (int64_t n = 0; n < d_ff; ++n) {
+                        g[n] += xk * gmlp_oracle_bf16_to_double(wg[n]);
+                        u[n] += xk * gmlp_oracle_bf16_to_double(wu[n]);
+                    }
+                }
+                for (int64_t n = 0; n < d_ff; ++n) P[i * d_ff + n] = gmlp_oracle_silu(g[n]) * u[n];
+            }
+        }
+        free(xn); free(xnb); free(g); free(u);
+    }
+    return failed ? -1 : 0;
+}
+
 /* Array forms of the two scalar helpers (plain loops), for the tests. */
 void gmlp_oracle_bf16_rn_array(const double* v, uint16_t* out, int64_t n)
 {

@@ -261,3 +261,35 @@ def test_bad_arguments_are_rejected():
     with pytest.raises(TypeError):
         oracle.gmlp_rows(X.astype(np.float32), Wg, Wu, Wd)
     assert oracle.gmlp_rows(X, Wg, Wu, Wd, rows=np.zeros(0, dtype=np.int64)).shape == (0, 16)
+
+
+# ---------------------------------------------------------------- the gate/up half on its own
+def test_gate_up_alone_against_naive_loops_torch_and_closed_form():
+    # "Matmul+Matmul+SiLU+Mul" (Section 6.1 benchmark list): silu(X Wg) * (X Wu), not rounded
+    inp = _rand(7, 40, 56, 71, rmsnorm=True, eps=1e-6)
+    X, Wg, Wu, gam = (inp.bits(n) for n in ("X", "Wg", "Wu", "gamma"))
+    P = oracle.gate_up_rows(X, Wg, Wu, gamma=gam, eps=1e-6, rmsnorm=True)
+    xd = oracle.bf16_to_double(X)
+    gd = oracle.bf16_to_double(gam)
+    eps = float(np.float32(1e-6))
+    xn = []
+    for m in range(7):
+        r = 1.0 / math.sqrt(sum(v * v for v in xd[m]) / 40 + eps)
+        xn.append([_round_bf16_py(xd[m, k] * r * gd[k]) for k in range(40)])
+    xn = oracle.bf16_to_double(np.array(xn, dtype=np.uint16))
+    G = oracle.naive_matmul(xn, oracle.bf16_to_double(Wg))
+    U = oracle.naive_matmul(xn, oracle.bf16_to_double(Wu))
+    want = np.vectorize(_py_silu)(G) * U
+    assert np.array_equal(P, want)
+    # library routine (no norm)
+    P2 = oracle.gate_up_rows(X, Wg, Wu)
+    t = torch.nn.functional.silu(inp.X.double() @ inp.Wg.double()) * (inp.X.double() @ inp.Wu.double())
+    assert np.allclose(P2, t.numpy(), rtol=1e-12, atol=1e-13)
+    # its bf16 rounding is exactly the H of the full pipeline; zero gate or zero up gives zero
+    _, H = oracle.gmlp_rows(X, Wg, Wu, inp.bits("Wd"), want_h=True)
+    assert np.array_equal(oracle.bf16_rn(P2), H)
+    z = np.zeros_like(Wg)
+    assert np.all(oracle.gate_up_rows(X, z, Wu) == 0.0) and np.all(oracle.gate_up_rows(X, Wg, z) == 0.0)
+    # rows subset and swapped roles
+    assert np.array_equal(oracle.gate_up_rows(X, Wg, Wu, rows=np.array([5, 1])), P2[[5, 1]])
+    assert not np.array_equal(oracle.gate_up_rows(X, Wu, Wg), P2)
