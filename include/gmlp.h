@@ -102,6 +102,16 @@ int gmlp_forward(const void* X, const void* Wg, const void* Wu, const void* Wd, 
 int gmlp_forward_ex(const gmlp_args* args);
 
 /*
+ * The gate/up half on its own: H = bf16( silu(Xn Wg) (.) (Xn Wu) ), the four-operator kernel
+ * "Matmul+Matmul+SiLU+Mul" of the paper's benchmark list (Section 6.1).  Uses args->X, Wg, Wu, the
+ * prologue options, stream, workspace and variant exactly as gmlp_forward_ex does; args->Wd is ignored
+ * (may be NULL) and args->Y receives H, row-major [M, d_ff] bf16 (d_ff columns, not d_model).
+ * Workspace: gmlp_workspace_bytes() of the same shape is sufficient.  GMLP_VARIANT_SIMT and _STREAM are
+ * not offered for this call (GMLP_ERR_UNSUPPORTED).
+ */
+int gmlp_gate_up(const gmlp_args* args);
+
+/*
  * The same call for a caller whose activations live in HOST memory: copies X_host
  * (M*d_model bf16, ideally pinned) to args->X, runs gmlp_forward_ex, and copies args->Y
  * to Y_host, all asynchronously on args->stream.  args->X and args->Y are device staging

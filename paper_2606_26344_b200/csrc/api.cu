@@ -680,9 +680,97 @@ int forward_static_impl(const void* Xp, const void* Wgp, const void* Wup, const 
                                 static_cast<bf16*>(Yp), M, d_ff, d_model, st);
 }
 
+// The gate/up half alone: same checks and schedules as forward_impl, output H to args->Y.
+int gate_up_impl(const gmlp_args* a) {
+    if (a == nullptr) return GMLP_ERR_NULL;
+    if (a->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
+    if (a->flags & ~kKnownFlags) return GMLP_ERR_FLAGS;
+    if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_PAIR) return GMLP_ERR_FLAGS;
+    int rc = check_shape(a->M, a->d_model, a->d_ff);
+    if (rc != GMLP_OK) return rc;
+    if (a->M == 0) return GMLP_OK;
+    if (!a->X || !a->Wg || !a->Wu || !a->Y) return GMLP_ERR_NULL;
+    if (!aligned16(a->X) || !aligned16(a->Wg) || !aligned16(a->Wu) || !aligned16(a->Y) || !aligned16(a->rms_gain))
+        return GMLP_ERR_ALIGN;
+    if (a->workspace != nullptr && (reinterpret_cast<uintptr_t>(a->workspace) & 255u)) return GMLP_ERR_ALIGN;
+    const int variant = resolve_variant(a->M, a->variant);
+    if (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM) return GMLP_ERR_UNSUPPORTED;
+    if (variant == GMLP_VARIANT_SKINNY && a->M > 128) return GMLP_ERR_UNSUPPORTED;
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    const Layout L = make_layout(a->M, a->d_model, a->d_ff, a->flags, variant, dev->sm_count);
+    uint8_t* ws = static_cast<uint8_t*>(a->workspace);
+    if (ws == nullptr) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (dev->workspace_bytes < L.total) {
+            if (dev->workspace != nullptr) {
+                if (cudaDeviceSynchronize() != cudaSuccess || cudaFree(dev->workspace) != cudaSuccess) return GMLP_ERR_LAUNCH;
+                dev->workspace = nullptr;
+                dev->workspace_bytes = 0;
+                dev->clean_counters = nullptr;
+                dev->clean_counters_bytes = 0;
+            }
+            void* p = nullptr;
+            if (cudaMalloc(&p, L.total) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return GMLP_ERR_WORKSPACE;
+            }
+            dev->workspace = p;
+            dev->workspace_bytes = L.total;
+        }
+        ws = static_cast<uint8_t*>(dev->workspace);
+    } else if (a->workspace_bytes < L.total) {
+        return GMLP_ERR_WORKSPACE;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(a->stream);
+    const bf16* A = static_cast<const bf16*>(a->X);
+    const bf16* Wg = static_cast<const bf16*>(a->Wg);
+    const bf16* Wu = static_cast<const bf16*>(a->Wu);
+    bf16* Hout = static_cast<bf16*>(a->Y);
+    prof_begin(st);
+    if (a->flags & GMLP_FLAG_RMSNORM) {
+        bf16* Xn = reinterpret_cast<bf16*>(ws + L.xn_off);
+        rc = launch_rmsnorm(A, static_cast<const bf16*>(a->rms_gain), Xn, a->M, a->d_model, a->rms_eps, st);
+        if (rc != GMLP_OK) return rc;
+        prof_mark("rmsnorm", st);
+        A = Xn;
+    }
+    if (variant == GMLP_VARIANT_SKINNY) {
+        float* scratch = reinterpret_cast<float*>(ws + L.partial_off);
+        unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
+        rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
+        if (rc == GMLP_OK) rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, Hout, a->M, a->d_model, a->d_ff, st);
+    } else if (variant == GMLP_VARIANT_PAIR) {
+        rc = launch_umma_pair<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st);
+    } else {
+        rc = launch_umma<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st);
+    }
+    if (rc != GMLP_OK) {
+        forget_counters(dev);
+        return rc;
+    }
+    prof_mark("gate_up", st);
+    if (a->flags & GMLP_FLAG_CHECKED) {
+        if (cudaStreamSynchronize(st) != cudaSuccess) { forget_counters(dev); return GMLP_ERR_LAUNCH; }
+        const int s = read_device_status();
+        if (s != 0) forget_counters(dev);
+        if (s < 0) return s;
+        if (s != 0) return GMLP_ERR_TIMEOUT;
+    }
+    return GMLP_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+int gmlp_gate_up(const gmlp_args* args) {
+    try {
+        return gate_up_impl(args);
+    } catch (...) {
+        return GMLP_ERR_LAUNCH;
+    }
+}
 
 int gmlp_forward_static(const void* X, const void* Wg, const void* Wu, const void* Wd, void* Y,
                         int64_t M, int64_t d_model, int64_t d_ff, void* stream) {

@@ -56,6 +56,8 @@ def lib() -> ctypes.CDLL:
         L.gmlp_forward.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, u32]
         L.gmlp_forward_ex.restype = ctypes.c_int
         L.gmlp_forward_ex.argtypes = [ctypes.POINTER(GmlpArgs)]
+        L.gmlp_gate_up.restype = ctypes.c_int
+        L.gmlp_gate_up.argtypes = [ctypes.POINTER(GmlpArgs)]
         L.gmlp_forward_host.restype = ctypes.c_int
         L.gmlp_forward_host.argtypes = [ctypes.POINTER(GmlpArgs), vp, vp]
         L.gmlp_forward_static.restype = ctypes.c_int
@@ -222,3 +224,36 @@ def forward_static(X, Wg, Wu, Wd, Y, stream=None) -> None:
                                        M, d_model, Wg.shape[1], st.cuda_stream)
     if rc != OK:
         raise GmlpError(rc)
+
+
+def gate_up(X, Wg, Wu, H=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, variant: int = VARIANT_AUTO,
+            workspace=None, stream=None, checked: bool = False) -> torch.Tensor:
+    """gmlp_gate_up: H = bf16(silu(Xn Wg) * (Xn Wu)), the gate/up half alone; H is [M, d_ff]."""
+    for t, n in ((X, "X"), (Wg, "Wg"), (Wu, "Wu")):
+        _check_bf16_cuda(t, n)
+    M, d_model = X.shape
+    d_ff = Wg.shape[1]
+    if Wg.shape != (d_model, d_ff) or Wu.shape != (d_model, d_ff):
+        raise ValueError("shape mismatch")
+    if H is None:
+        H = torch.empty(M, d_ff, dtype=torch.bfloat16, device=X.device)
+    _check_bf16_cuda(H, "H")
+    if gamma is not None:
+        _check_bf16_cuda(gamma, "gamma")
+    st = stream if stream is not None else torch.cuda.current_stream(X.device)
+    a = GmlpArgs()
+    a.struct_bytes = ctypes.sizeof(GmlpArgs)
+    a.flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0)
+    a.X, a.Wg, a.Wu, a.Wd, a.Y = X.data_ptr(), Wg.data_ptr(), Wu.data_ptr(), None, H.data_ptr()
+    a.M, a.d_model, a.d_ff = M, d_model, d_ff
+    a.rms_gain = gamma.data_ptr() if gamma is not None else None
+    a.rms_eps = eps
+    a.variant = variant
+    a.stream = st.cuda_stream
+    a.workspace = workspace.data_ptr() if workspace is not None else None
+    a.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    with torch.cuda.device(X.device):
+        rc = lib().gmlp_gate_up(ctypes.byref(a))
+    if rc != OK:
+        raise GmlpError(rc)
+    return H
