@@ -84,6 +84,9 @@ def _load():
         lib.gmlp_oracle_gate_up_rows.argtypes = [u16p, u16p, u16p, u16p, ctypes.c_float, ctypes.c_int,
                                                  ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                                  i64p, ctypes.c_int64, f64p, ctypes.c_int]
+        lib.gmlp_oracle_rmsnorm_matmul_rows.restype = ctypes.c_int
+        lib.gmlp_oracle_rmsnorm_matmul_rows.argtypes = [u16p, u16p, u16p, ctypes.c_float, ctypes.c_int64, ctypes.c_int64,
+                                                        ctypes.c_int64, i64p, ctypes.c_int64, f64p, ctypes.c_int]
         lib.gmlp_oracle_bf16_rn_array.restype = None
         lib.gmlp_oracle_bf16_rn_array.argtypes = [f64p, u16p, ctypes.c_int64]
         lib.gmlp_oracle_silu_array.restype = None
@@ -212,6 +215,32 @@ def gate_up_rows(X, Wg, Wu, rows=None, gamma=None, eps: float = 1e-5, rmsnorm: b
     if rc != 0:
         raise RuntimeError(f"gmlp_oracle_gate_up_rows failed ({rc})")
     return P
+
+
+def rmsnorm_matmul_rows(X, W, rows=None, gamma=None, eps: float = 1e-5, num_threads: int = 0) -> np.ndarray:
+    """Reference RMSNorm(X) @ W (float64, no intermediate rounding) for the selected rows."""
+    lib = _load()
+    X, W = _u16(X, "X"), _u16(W, "W")
+    M, K = X.shape
+    if W.shape[0] != K:
+        raise ValueError("shape mismatch")
+    N = W.shape[1]
+    if rows is None:
+        rows = np.arange(M, dtype=np.int64)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    g = None
+    if gamma is not None:
+        g = _u16(gamma, "gamma").reshape(-1)
+        if g.size != K:
+            raise ValueError("gamma size")
+    Z = np.zeros((rows.size, N), dtype=np.float64)
+    rc = lib.gmlp_oracle_rmsnorm_matmul_rows(_p(X, ctypes.c_uint16), _p(W, ctypes.c_uint16),
+                                             None if g is None else _p(g, ctypes.c_uint16), ctypes.c_float(eps),
+                                             M, K, N, _p(rows, ctypes.c_int64), rows.size, _p(Z, ctypes.c_double),
+                                             int(num_threads))
+    if rc != 0:
+        raise RuntimeError(f"gmlp_oracle_rmsnorm_matmul_rows failed ({rc})")
+    return Z
 
 
 def naive_matmul(A, B) -> np.ndarray:

@@ -234,6 +234,61 @@ int gmlp_oracle_gate_up_rows(const uint16_t* X, const uint16_t* Wg, const uint16
     return failed ? -1 : 0;
 }
 
+/*
+ * RMSNorm followed by a matrix multiplication, the paper's running example (Section 2, Eq. 1 and
+ * figure "rmsnorm-matmul-comp-graph" (a)):   Z = RMSNorm(X) * W,
+ *   r_i = 1/sqrt(mean_k X[i,k]^2 + eps),   Z[i, n] = sum_k (X[i,k] * r_i * gamma[k]) * W[k, n].
+ * Plain definition in fp64 with no intermediate rounding; gamma == NULL is the paper's gain-less form.
+ * X [M, K], W [K, N] bf16 bit patterns; Z [n_rows, N] fp64 for the selected rows.
+ */
+int gmlp_oracle_rmsnorm_matmul_rows(const uint16_t* X, const uint16_t* W, const uint16_t* gamma, float eps,
+                                    int64_t M, int64_t K, int64_t N, const int64_t* rows, int64_t n_rows,
+                                    double* Z, int num_threads)
+{
+    if (!X || !W || !rows || !Z || M < 0 || K <= 0 || N <= 0 || n_rows < 0) return -1;
+    for (int64_t i = 0; i < n_rows; ++i)
+        if (rows[i] < 0 || rows[i] >= M) return -1;
+    int failed = 0;
+#ifdef _OPENMP
+    if (num_threads > 0) omp_set_num_threads(num_threads);
+#else
+    (void)num_threads;
+#endif
+#pragma omp parallel
+    {
+        double* xn = (double*)malloc(sizeof(double) * (size_t)K);
+        if (!xn) {
+#pragma omp atomic write
+            failed = 1;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int64_t i = 0; i < n_rows; ++i) {
+                const uint16_t* x = X + rows[i] * K;
+                double ss = 0.0;
+                for (int64_t k = 0; k < K; ++k) {
+                    const double v = gmlp_oracle_bf16_to_double(x[k]);
+                    ss += v * v;
+                }
+                const double r = 1.0 / sqrt(ss / (double)K + (double)eps);
+                for (int64_t k = 0; k < K; ++k) {
+                    double v = gmlp_oracle_bf16_to_double(x[k]) * r;
+                    if (gamma) v *= gmlp_oracle_bf16_to_double(gamma[k]);
+                    xn[k] = v;
+                }
+                double* z = Z + i * N;
+                for (int64_t n = 0; n < N; ++n) z[n] = 0.0;
+                for (int64_t k = 0; k < K; ++k) {
+                    const double xk = xn[k];
+                    const uint16_t* w = W + k * N;
+                    for (int64_t n = 0; n < N; ++n) z[n] += xk * gmlp_oracle_bf16_to_double(w[n]);
+                }
+            }
+        }
+        free(xn);
+    }
+    return failed ? -1 : 0;
+}
+
 /* Array forms of the two scalar helpers (plain loops), for the tests. */
 void gmlp_oracle_bf16_rn_array(const double* v, uint16_t* out, int64_t n)
 {
