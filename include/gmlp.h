@@ -112,6 +112,34 @@ int gmlp_forward_ex(const gmlp_args* args);
 int gmlp_gate_up(const gmlp_args* args);
 
 /*
+ * RMSNorm followed by a matrix multiplication, the paper's running example (Section 2):
+ *     Z = RMSNorm(X) * W,     X [M, K], W [K, N], Z [M, N], row-major bf16, K and N multiples of 8.
+ * Default schedule = the paper's algebraic rewrite (X*W) (.) r: the row scale r = 1/sqrt(mean(X^2)+eps)
+ * does not depend on k, so the GEMM runs on the raw X and applies r in its epilogue, while a small
+ * kernel computes r; the two are chained by programmatic dependent launch and only the GEMM's epilogue
+ * waits for r, so the RMS branch runs in parallel with the matmul's main loop.  No normalised copy of X
+ * is stored.  A gain (rms_gain != NULL, along K) does not commute with the matmul: such calls, and calls
+ * with GMLP_RMSMM_UNFUSED, run the RMSNorm kernel into the workspace and then the plain GEMM.
+ * workspace (256-byte aligned, required): M*4 bytes for the rewritten schedule, M*K*2 for the unfused one.
+ */
+enum { GMLP_RMSMM_UNFUSED = 1u << 4 };   /* flag for gmlp_rmsmm_args.flags, next to GMLP_FLAG_CHECKED */
+typedef struct gmlp_rmsmm_args {
+    uint32_t struct_bytes;    /* sizeof(gmlp_rmsmm_args) */
+    uint32_t flags;           /* GMLP_FLAG_CHECKED | GMLP_RMSMM_UNFUSED */
+    const void* X;            /* device, [M, K] bf16 */
+    const void* W;            /* device, [K, N] bf16 */
+    void* Z;                  /* device, [M, N] bf16, written */
+    int64_t M, K, N;
+    const void* rms_gain;     /* device, [K] bf16, or NULL (the paper's form) */
+    float rms_eps;
+    int32_t reserved;         /* must be 0 */
+    void* stream;
+    void* workspace;
+    uint64_t workspace_bytes;
+} gmlp_rmsmm_args;
+int gmlp_rmsnorm_matmul(const gmlp_rmsmm_args* args);
+
+/*
  * The same call for a caller whose activations live in HOST memory: copies X_host
  * (M*d_model bf16, ideally pinned) to args->X, runs gmlp_forward_ex, and copies args->Y
  * to Y_host, all asynchronously on args->stream.  args->X and args->Y are device staging

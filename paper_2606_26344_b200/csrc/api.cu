@@ -76,6 +76,7 @@ struct DeviceState {
     uint64_t workspace_bytes = 0;
     bool umma_attr_set = false;
     bool pair_attr_set = false;
+    bool rowscale_attr_set = false;
     bool skinny_attr_set = false;
     // arrival counters last zeroed by the library (the kernels leave them zero after every call)
     const void* clean_counters = nullptr;
@@ -386,8 +387,8 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
-    if (cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles) !=
-        cudaSuccess)
+    if (cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m,
+                           num_tiles, (const float*)nullptr) != cudaSuccess)
         return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -431,11 +432,14 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
     cudaError_t err;
     if (GATEUP)
-        err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles);
+        err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
+                                 (const float*)nullptr);
     else if (nb == 4)
-        err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles);
+        err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
+                                 (const float*)nullptr);
     else
-        err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles);
+        err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
+                                 (const float*)nullptr);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -760,9 +764,105 @@ int gate_up_impl(const gmlp_args* a) {
     return GMLP_OK;
 }
 
+// RMSNorm+MatMul.  Rewritten schedule: one GEMM kernel with row-square reducer warps and an epilogue row scale.
+int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
+    if (a == nullptr) return GMLP_ERR_NULL;
+    if (a->struct_bytes != sizeof(gmlp_rmsmm_args)) return GMLP_ERR_FLAGS;
+    if ((a->flags & ~(uint32_t)(GMLP_FLAG_CHECKED | GMLP_RMSMM_UNFUSED)) || a->reserved != 0) return GMLP_ERR_FLAGS;
+    int rc = check_shape(a->M, a->K, a->N);
+    if (rc != GMLP_OK) return rc;
+    if (a->M == 0) return GMLP_OK;
+    if (!a->X || !a->W || !a->Z) return GMLP_ERR_NULL;
+    if (!aligned16(a->X) || !aligned16(a->W) || !aligned16(a->Z) || !aligned16(a->rms_gain)) return GMLP_ERR_ALIGN;
+    if (a->workspace != nullptr && (reinterpret_cast<uintptr_t>(a->workspace) & 255u)) return GMLP_ERR_ALIGN;
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(a->stream);
+    const bf16* X = static_cast<const bf16*>(a->X);
+    const bf16* W = static_cast<const bf16*>(a->W);
+    bf16* Z = static_cast<bf16*>(a->Z);
+    const bool unfused = (a->flags & GMLP_RMSMM_UNFUSED) != 0 || a->rms_gain != nullptr;
+    prof_begin(st);
+    if (unfused) {
+        const uint64_t need = align256((uint64_t)a->M * a->K * 2);
+        if (a->workspace == nullptr || a->workspace_bytes < need) return GMLP_ERR_WORKSPACE;
+        bf16* Xn = static_cast<bf16*>(a->workspace);
+        rc = launch_rmsnorm(X, static_cast<const bf16*>(a->rms_gain), Xn, a->M, a->K, a->rms_eps, st);
+        if (rc != GMLP_OK) return rc;
+        prof_mark("rmsnorm", st);
+        rc = a->M >= 1024 ? launch_umma_pair<false>(dev, Xn, W, nullptr, Z, a->M, a->K, a->N, st)
+                          : launch_umma<false>(dev, Xn, W, nullptr, Z, a->M, a->K, a->N, st);
+        if (rc != GMLP_OK) return rc;
+        prof_mark("matmul", st);
+    } else {
+        // rewritten: r = rsqrt(mean(x^2) + eps) per row (tiny kernel), then the GEMM on the raw X with the row scale
+        // in its epilogue; programmatic dependent launch lets the GEMM's main loop overlap the RMS branch
+        const uint64_t need = align256((uint64_t)a->M * 4);
+        if (a->workspace == nullptr || a->workspace_bytes < need) return GMLP_ERR_WORKSPACE;
+        float* r = static_cast<float*>(a->workspace);
+        gmlp::row_rsqrt_kernel<<<(unsigned)a->M, gmlp::kRmsThreads, 0, st>>>(X, r, a->M, (int)a->K, a->rms_eps);
+        GMLP_CHECK_LAUNCH();
+        prof_mark("row_rsqrt", st);
+        const bool pair = a->M >= 1024;
+        CUtensorMap tmA, tmB;
+        if (!encode_2d(&tmA, X, (uint64_t)a->K, (uint64_t)a->M, gmlp::kUmmaBK, 128) ||
+            !encode_2d(&tmB, W, (uint64_t)a->N, (uint64_t)a->K, 64, gmlp::kUmmaBK))
+            return GMLP_ERR_LAUNCH;
+        if (!dev->rowscale_attr_set) {
+            if (cudaFuncSetAttribute(gmlp::umma_gemm_kernel<false, 4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)gmlp::kUmmaSmemBytes) != cudaSuccess ||
+                cudaFuncSetAttribute(gmlp::umma_pair_gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)gmlp::kPairSmemBytes) != cudaSuccess)
+                return GMLP_ERR_LAUNCH;
+            dev->rowscale_attr_set = true;
+        }
+        const int sms = dev->sm_count > 0 ? dev->sm_count : 148;
+        const int num_m = (int)((a->M + (pair ? 255 : 127)) / (pair ? 256 : 128));
+        const int num_tiles = num_m * (int)((a->N + 255) / 256);
+        const int ctas = pair ? 2 * (num_tiles < sms / 2 ? num_tiles : sms / 2) : (num_tiles < sms ? num_tiles : sms);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)ctas);
+        cfg.blockDim = dim3(gmlp::kUmmaThreads);
+        cfg.dynamicSmemBytes = pair ? gmlp::kPairSmemBytes : gmlp::kUmmaSmemBytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = 2;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pair ? 2 : 1;
+        const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
+        const float* rc_ptr = r;
+        cudaError_t err = pair
+            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr)
+            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr);
+        if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
+        GMLP_CHECK_LAUNCH();
+        prof_mark("matmul_rowscale", st);
+    }
+    if (a->flags & GMLP_FLAG_CHECKED) {
+        if (cudaStreamSynchronize(st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+        const int s = read_device_status();
+        if (s < 0) return s;
+        if (s != 0) return GMLP_ERR_TIMEOUT;
+    }
+    return GMLP_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+int gmlp_rmsnorm_matmul(const gmlp_rmsmm_args* args) {
+    try {
+        return rmsnorm_matmul_impl(args);
+    } catch (...) {
+        return GMLP_ERR_LAUNCH;
+    }
+}
 
 int gmlp_gate_up(const gmlp_args* args) {
     try {

@@ -64,4 +64,39 @@ rmsnorm_kernel(const bf16* __restrict__ X, const bf16* __restrict__ gamma, bf16*
     }
 }
 
+// The RMS branch alone: r[m] = rsqrt(mean_k X[m,k]^2 + eps) in fp32, one CTA per row.  Used by the rewritten
+// RMSNorm+MatMul, whose GEMM applies r in its epilogue; the kernel lets its dependent start at once, so the
+// GEMM's main loop runs while the row scales are being computed.
+__global__ void __launch_bounds__(kRmsThreads)
+row_rsqrt_kernel(const bf16* __restrict__ X, float* __restrict__ r, int64_t M, int K, float eps)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int64_t row = blockIdx.x;
+    if (row >= M) return;
+    const uint4* x = reinterpret_cast<const uint4*>(X + row * K);
+    const int nvec = K >> 3;
+    float ss = 0.0f;
+    for (int i = threadIdx.x; i < nvec; i += kRmsThreads) {
+        const uint4 v = x[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float a = bf16_lo(w[j]), b = bf16_hi(w[j]);
+            ss = fmaf(a, a, ss);
+            ss = fmaf(b, b, ss);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+    __shared__ float warp_sums[kRmsThreads / 32];
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kRmsThreads / 32; ++w) t += warp_sums[w];
+        r[row] = rsqrtf(t / (float)K + eps);
+    }
+}
+
 }  // namespace gmlp

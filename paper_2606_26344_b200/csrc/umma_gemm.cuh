@@ -79,12 +79,19 @@ __global__ void wait_timeout_probe_kernel(long long limit_cycles)
 
 // NB = 64-column weight boxes per stage: 4 -> MMA N = 256 (the default), 2 -> MMA N = 128 (smaller tiles for
 // shapes that would otherwise leave most SMs without a tile; more stages, lower arithmetic intensity).
-template <bool GATEUP, int NB>
+//
+// ROWSCALE = true turns the plain GEMM into the paper's rewritten RMSNorm+MatMul (Section 2):
+// Z = (X * W) (.) r with r_m = 1/sqrt(mean_k X[m,k]^2 + eps) applied in the epilogue (legal because r does
+// not depend on k).  r comes from row_rsqrt_kernel, the kernel launched just before this one: the two
+// are chained by programmatic dependent launch and ONLY the epilogue warps wait for it, so the main loop
+// (which reads the raw X) runs in parallel with the RMS branch.
+template <bool GATEUP, int NB, bool ROWSCALE = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
-                 int M, int K, int N, int num_m_tiles, int num_tiles)
+                 int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale)
 {
+    static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
     constexpr int KERNEL_ID = GATEUP ? 1 : 2;
     constexpr int N_MMA = 64 * NB;
     constexpr int BN_OUT = GATEUP ? N_MMA / 2 : N_MMA;
@@ -140,7 +147,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            ptx::grid_dependency_wait();                          // A (X, Xn or H) may come from the previous kernel
+            if (!ROWSCALE) ptx::grid_dependency_wait();           // A (Xn or H) may come from the previous kernel
             int it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
@@ -213,6 +220,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             ptx::tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * kUmmaN);
             bf16* crow = C + (size_t)row * N + n0;
+            const float rscale = (ROWSCALE && row < M) ? __ldcg(row_scale + row) : 1.0f;
 #pragma unroll 1
             for (int c = 0; c < BN_OUT; c += 32) {
                 uint32_t g[32];
@@ -233,7 +241,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     ptx::tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        packed[j] = pack_bf16x2(__uint_as_float(g[2 * j]), __uint_as_float(g[2 * j + 1]));
+                        packed[j] = pack_bf16x2(__uint_as_float(g[2 * j]) * rscale, __uint_as_float(g[2 * j + 1]) * rscale);
                 }
                 if (row < M) {
 #pragma unroll

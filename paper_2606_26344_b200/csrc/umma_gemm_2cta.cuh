@@ -83,12 +83,14 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 }
 }  // namespace ptx
 
-template <bool GATEUP>
+// ROWSCALE: see umma_gemm.cuh (epilogue row scale from row_rsqrt_kernel; only the epilogue waits for it).
+template <bool GATEUP, bool ROWSCALE = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                       const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
-                      int M, int K, int N, int num_m_tiles, int num_tiles)
+                      int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale)
 {
+    static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
     constexpr int KERNEL_ID = GATEUP ? 6 : 7;
     constexpr int BN_OUT = GATEUP ? 128 : 256;
     // D = fp32, A = B = bf16, A K-major, B MN-major, M = 256 (128 per CTA), N = 256
@@ -142,7 +144,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs) ----------------
         if (lane == 0) {
-            ptx::grid_dependency_wait();
+            if (!ROWSCALE) ptx::grid_dependency_wait();
             const uint32_t leader_full0 = ptx::map_to_cta(full0, 0);
             int it = 0;
             bool ok = true;
@@ -211,6 +213,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             ptx::tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256);
             bf16* crow = C + (size_t)row * N + n0;
+            const float rscale = (ROWSCALE && row < M) ? __ldcg(row_scale + row) : 1.0f;
 #pragma unroll 1
             for (int c = 0; c < BN_OUT; c += 32) {
                 uint32_t g[32];
@@ -231,7 +234,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     ptx::tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        packed[j] = pack_bf16x2(__uint_as_float(g[2 * j]), __uint_as_float(g[2 * j + 1]));
+                        packed[j] = pack_bf16x2(__uint_as_float(g[2 * j]) * rscale, __uint_as_float(g[2 * j + 1]) * rscale);
                 }
                 if (row < M) {
 #pragma unroll

@@ -37,6 +37,19 @@ class GmlpArgs(ctypes.Structure):
     ]
 
 
+class GmlpRmsmmArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_bytes", ctypes.c_uint32), ("flags", ctypes.c_uint32),
+        ("X", ctypes.c_void_p), ("W", ctypes.c_void_p), ("Z", ctypes.c_void_p),
+        ("M", ctypes.c_int64), ("K", ctypes.c_int64), ("N", ctypes.c_int64),
+        ("rms_gain", ctypes.c_void_p), ("rms_eps", ctypes.c_float), ("reserved", ctypes.c_int32),
+        ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_uint64),
+    ]
+
+
+RMSMM_UNFUSED = 1 << 4
+
+
 class GmlpError(RuntimeError):
     def __init__(self, status: int):
         self.status = status
@@ -56,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.gmlp_forward.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, u32]
         L.gmlp_forward_ex.restype = ctypes.c_int
         L.gmlp_forward_ex.argtypes = [ctypes.POINTER(GmlpArgs)]
+        L.gmlp_rmsnorm_matmul.restype = ctypes.c_int
+        L.gmlp_rmsnorm_matmul.argtypes = [ctypes.POINTER(GmlpRmsmmArgs)]
         L.gmlp_gate_up.restype = ctypes.c_int
         L.gmlp_gate_up.argtypes = [ctypes.POINTER(GmlpArgs)]
         L.gmlp_forward_host.restype = ctypes.c_int
@@ -257,3 +272,36 @@ def gate_up(X, Wg, Wu, H=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = Fa
     if rc != OK:
         raise GmlpError(rc)
     return H
+
+
+def rmsnorm_matmul(X, W, Z=None, gamma=None, eps: float = 1e-5, unfused: bool = False, stream=None,
+                   checked: bool = False) -> torch.Tensor:
+    """gmlp_rmsnorm_matmul: Z = RMSNorm(X) @ W.  Default: the rewritten schedule (row scale in the GEMM epilogue)."""
+    for t, n in ((X, "X"), (W, "W")):
+        _check_bf16_cuda(t, n)
+    M, K = X.shape
+    N = W.shape[1]
+    if W.shape[0] != K:
+        raise ValueError("shape mismatch")
+    if Z is None:
+        Z = torch.empty(M, N, dtype=torch.bfloat16, device=X.device)
+    _check_bf16_cuda(Z, "Z")
+    nbytes = M * K * 2 if (unfused or gamma is not None) else M * 4
+    ws = torch.empty(((nbytes + 255) // 256 + 1) * 256, dtype=torch.uint8, device=X.device)
+    st = stream if stream is not None else torch.cuda.current_stream(X.device)
+    a = GmlpRmsmmArgs()
+    a.struct_bytes = ctypes.sizeof(GmlpRmsmmArgs)
+    a.flags = (FLAG_CHECKED if checked else 0) | (RMSMM_UNFUSED if unfused else 0)
+    a.X, a.W, a.Z = X.data_ptr(), W.data_ptr(), Z.data_ptr()
+    a.M, a.K, a.N = M, K, N
+    a.rms_gain = gamma.data_ptr() if gamma is not None else None
+    a.rms_eps = eps
+    a.reserved = 0
+    a.stream = st.cuda_stream
+    a.workspace = ws.data_ptr() if ws is not None else None
+    a.workspace_bytes = ws.numel() if ws is not None else 0
+    with torch.cuda.device(X.device):
+        rc = lib().gmlp_rmsnorm_matmul(ctypes.byref(a))
+    if rc != OK:
+        raise GmlpError(rc)
+    return Z
