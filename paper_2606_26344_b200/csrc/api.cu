@@ -210,9 +210,13 @@ struct Layout {
     SkinnyPlan s1, s2;
 };
 
-int resolve_variant(int64_t M, int32_t variant) {
+// Schedule choice, from measurements on B200: the operand-swapped stream-K schedule wins while the split-K
+// partials (which grow with M) stay small next to the weights: always up to 32 tokens, up to 96 tokens when the
+// three weight matrices are at least 200 MB; CTA pairs from 1024 rows on; single-CTA tiles in between.
+int resolve_variant(int64_t M, int64_t d_model, int64_t d_ff, int32_t variant) {
     if (variant != GMLP_VARIANT_AUTO) return variant;
-    if (M <= 128) return GMLP_VARIANT_SKINNY;
+    const double weight_bytes = 6.0 * (double)d_model * (double)d_ff;
+    if (M <= 32 || (M <= 96 && weight_bytes >= 200e6)) return GMLP_VARIANT_SKINNY;
     return M < 1024 ? GMLP_VARIANT_UMMA : GMLP_VARIANT_PAIR;
 }
 
@@ -537,7 +541,7 @@ int forward_impl(const gmlp_args* a) {
     DeviceState* dev = current_device(&rc);
     if (dev == nullptr) return rc;
 
-    const int variant = resolve_variant(a->M, a->variant);
+    const int variant = resolve_variant(a->M, a->d_model, a->d_ff, a->variant);
     if (variant == GMLP_VARIANT_SKINNY && a->M > 128) return GMLP_ERR_UNSUPPORTED;
     const Layout L = make_layout(a->M, a->d_model, a->d_ff, a->flags, variant, dev->sm_count);
 
@@ -697,7 +701,7 @@ int gate_up_impl(const gmlp_args* a) {
     if (!aligned16(a->X) || !aligned16(a->Wg) || !aligned16(a->Wu) || !aligned16(a->Y) || !aligned16(a->rms_gain))
         return GMLP_ERR_ALIGN;
     if (a->workspace != nullptr && (reinterpret_cast<uintptr_t>(a->workspace) & 255u)) return GMLP_ERR_ALIGN;
-    const int variant = resolve_variant(a->M, a->variant);
+    const int variant = resolve_variant(a->M, a->d_model, a->d_ff, a->variant);
     if (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM) return GMLP_ERR_UNSUPPORTED;
     if (variant == GMLP_VARIANT_SKINNY && a->M > 128) return GMLP_ERR_UNSUPPORTED;
     DeviceState* dev = current_device(&rc);
@@ -932,14 +936,14 @@ uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) sm_count = sms;
     }
     (void)cudaGetLastError();
-    const Layout L = make_layout(M, d_model, d_ff, flags, resolve_variant(M, variant), sm_count);
+    const Layout L = make_layout(M, d_model, d_ff, flags, resolve_variant(M, d_model, d_ff, variant), sm_count);
     return L.total > 256 ? L.total : 256;
 }
 
 int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags) {
     (void)flags;
     if (check_shape(M, d_model, d_ff) != GMLP_OK) return GMLP_ERR_SHAPE;
-    return resolve_variant(M, GMLP_VARIANT_AUTO);
+    return resolve_variant(M, d_model, d_ff, GMLP_VARIANT_AUTO);
 }
 
 int gmlp_device_status(void) {

@@ -96,7 +96,10 @@ def test_workspace_sizes_and_variant_choice(lib):
     assert wb(8, dm, dff, 0, gmlp.VARIANT_STREAM) < 64 << 20
     assert gmlp.pick_variant(8, dm, dff) == gmlp.VARIANT_SKINNY
     assert gmlp.pick_variant(1, 2048, 5632) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(128, 2048, 5632) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(32, 2048, 5632) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(64, 2048, 5632) == gmlp.VARIANT_UMMA
+    assert gmlp.pick_variant(64, dm, dff) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(128, dm, dff) == gmlp.VARIANT_UMMA
     assert gmlp.pick_variant(129, 2048, 5632) == gmlp.VARIANT_UMMA
     assert gmlp.pick_variant(1000, 2048, 5632) == gmlp.VARIANT_UMMA
     assert gmlp.pick_variant(2048, dm, dff) == gmlp.VARIANT_PAIR
