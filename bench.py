@@ -281,21 +281,39 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
                                "peak_source": peaks["source"] + " (copy)"}
 
     if want_e2e:
-        Xh, Yh = inp.X.pin_memory(), torch.empty_like(inp.X).pin_memory()
-        for _ in range(3):
-            gmlp.forward_host(a, Xh, Yh)
+        # End to end through the host-buffer entry point: every step copies its X from pinned host memory and its Y
+        # back.  Two lanes (stream + staging buffers + workspace each) alternate, so that a step's copies overlap the
+        # other lane's kernels, as a server with two batches in flight would run it.
+        lanes = []
+        for _ in range(2):
+            st_l = torch.cuda.Stream(device=dev)
+            Xs, Ys = torch.empty_like(X), torch.empty_like(X)
+            ws_l = gmlp.alloc_workspace(w.M, w.d_model, w.d_ff, w.rmsnorm)
+            lanes.append({"stream": st_l, "Xh": inp.X.clone().pin_memory(), "Yh": torch.empty_like(inp.X).pin_memory(),
+                          "keep": (Xs, Ys, ws_l),
+                          "args": gmlp.make_args(Xs, Wg, Wu, Wd, Ys, gamma, w.eps, w.rmsnorm, gmlp.VARIANT_AUTO, ws_l, st_l)})
+        for i in range(6):
+            ln = lanes[i % 2]
+            gmlp.forward_host(ln["args"], ln["Xh"], ln["Yh"])
         barrier()
+        n_e2e = max(4, min(steps, 50))
         t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
-        n_e2e = max(3, min(steps, 50))
         t0.record(stream)
-        for _ in range(n_e2e):
-            gmlp.forward_host(a, Xh, Yh)
+        for ln in lanes:
+            ln["stream"].wait_event(t0)
+        for i in range(n_e2e):
+            ln = lanes[i % 2]
+            gmlp.forward_host(ln["args"], ln["Xh"], ln["Yh"])
+        for ln in lanes:
+            done = torch.cuda.Event()
+            done.record(ln["stream"])
+            stream.wait_event(done)
         t1.record(stream)
         barrier()
         e2e_ms = t0.elapsed_time(t1) / n_e2e
         nb = w.M * w.d_model * 2
         res["e2e"] = {"value": w.M / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
-                      "h2d_bytes_per_step": nb, "d2h_bytes_per_step": nb, "steps": n_e2e}
+                      "h2d_bytes_per_step": nb, "d2h_bytes_per_step": nb, "steps": n_e2e, "lanes": 2}
     res["_inputs"] = inp
     return res
 

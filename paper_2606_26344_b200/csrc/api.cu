@@ -78,9 +78,12 @@ struct DeviceState {
     bool pair_attr_set = false;
     bool rowscale_attr_set = false;
     bool skinny_attr_set = false;
-    // arrival counters last zeroed by the library (the kernels leave them zero after every call)
-    const void* clean_counters = nullptr;
-    uint64_t clean_counters_bytes = 0;
+    // arrival-counter regions zeroed by the library (the kernels leave them zero after every call); a few are
+    // remembered so that callers alternating between workspaces (one per stream) do not pay a memset per call
+    static constexpr int kCleanSlots = 4;
+    const void* clean_counters[kCleanSlots] = {};
+    uint64_t clean_counters_bytes[kCleanSlots] = {};
+    int clean_next = 0;
 };
 std::mutex g_mutex;
 DeviceState g_dev[kMaxDevices];
@@ -273,17 +276,25 @@ bool encode_2d(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer
 // need clearing the first time a given counter region is used (or after a failed call).
 int ensure_counters_zero(DeviceState* dev, void* ptr, uint64_t bytes, cudaStream_t st) {
     std::lock_guard<std::mutex> lock(g_mutex);
-    if (dev->clean_counters == ptr && dev->clean_counters_bytes == bytes) return GMLP_OK;
+    for (int i = 0; i < DeviceState::kCleanSlots; ++i)
+        if (dev->clean_counters[i] == ptr && dev->clean_counters_bytes[i] == bytes) return GMLP_OK;
     if (cudaMemsetAsync(ptr, 0, bytes, st) != cudaSuccess) return GMLP_ERR_LAUNCH;
-    dev->clean_counters = ptr;
-    dev->clean_counters_bytes = bytes;
+    dev->clean_counters[dev->clean_next] = ptr;
+    dev->clean_counters_bytes[dev->clean_next] = bytes;
+    dev->clean_next = (dev->clean_next + 1) % DeviceState::kCleanSlots;
     return GMLP_OK;
+}
+
+void forget_counters_locked(DeviceState* dev) {
+    for (int i = 0; i < DeviceState::kCleanSlots; ++i) {
+        dev->clean_counters[i] = nullptr;
+        dev->clean_counters_bytes[i] = 0;
+    }
 }
 
 void forget_counters(DeviceState* dev) {
     std::lock_guard<std::mutex> lock(g_mutex);
-    dev->clean_counters = nullptr;
-    dev->clean_counters_bytes = 0;
+    forget_counters_locked(dev);
 }
 
 // ------------------------------------------------------------------ launches
@@ -554,8 +565,7 @@ int forward_impl(const gmlp_args* a) {
                 if (cudaDeviceSynchronize() != cudaSuccess || cudaFree(dev->workspace) != cudaSuccess) return GMLP_ERR_LAUNCH;
                 dev->workspace = nullptr;
                 dev->workspace_bytes = 0;
-                dev->clean_counters = nullptr;
-                dev->clean_counters_bytes = 0;
+                forget_counters_locked(dev);
             }
             void* p = nullptr;
             if (cudaMalloc(&p, L.total) != cudaSuccess) {
@@ -715,8 +725,7 @@ int gate_up_impl(const gmlp_args* a) {
                 if (cudaDeviceSynchronize() != cudaSuccess || cudaFree(dev->workspace) != cudaSuccess) return GMLP_ERR_LAUNCH;
                 dev->workspace = nullptr;
                 dev->workspace_bytes = 0;
-                dev->clean_counters = nullptr;
-                dev->clean_counters_bytes = 0;
+                forget_counters_locked(dev);
             }
             void* p = nullptr;
             if (cudaMalloc(&p, L.total) != cudaSuccess) {
