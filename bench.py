@@ -251,7 +251,7 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
     gmlp.profile_enable(False)
 
     res = {"name": w.name, "M": w.M, "d_model": w.d_model, "d_ff": w.d_ff, "rmsnorm": w.rmsnorm,
-           "variant": {1: "simt", 2: "stream", 3: "umma", 4: "skinny", 5: "pair"}[variant], "ms_per_step": ms,
+           "variant": {1: "simt", 2: "stream", 3: "umma", 4: "skinny", 5: "pair", 6: "tensor"}[variant], "ms_per_step": ms,
            "ms_min": min(per_step), "tokens_per_s": w.M / (ms * 1e-3), "tflops": w.flops / (ms * 1e-3) / 1e12,
            "gbps_min_bytes": w.min_bytes / (ms * 1e-3) / 1e9, "launches": launches, "clocks": clocks,
            "kernel_ms": kern_ms,

@@ -69,7 +69,10 @@ enum {
     GMLP_VARIANT_STREAM = 2, /* small M: weight-streaming split-K kernels on CUDA cores (HBM-bound regime) */
     GMLP_VARIANT_UMMA = 3,   /* medium M: tcgen05 tensor-core GEMMs fed by TMA, accumulators in TMEM, one CTA per tile */
     GMLP_VARIANT_SKINNY = 4, /* M <= 128: operand-swapped tcgen05 GEMMs, stream-K over all SMs (HBM-bound regime) */
-    GMLP_VARIANT_PAIR = 5    /* large M: the same GEMMs on CTA pairs (tcgen05 cta_group::2, 256-row tiles) */
+    GMLP_VARIANT_PAIR = 5,   /* large M: the same GEMMs on CTA pairs (tcgen05 cta_group::2, 256-row tiles) */
+    GMLP_VARIANT_TENSOR = 6  /* what AUTO takes outside SKINNY: each of the two GEMMs picks, by its number of
+                                128-row blocks, the CTA-pair kernel or the single-CTA kernel (whose down projection
+                                splits K over a thread-block cluster when there are few output tiles) */
 };
 
 typedef struct gmlp_args {
@@ -188,7 +191,7 @@ int gmlp_forward_static(const void* X, const void* Wg, const void* Wu, const voi
  */
 uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant);
 
-/* The schedule AUTO resolves to for this shape (GMLP_VARIANT_SKINNY, _UMMA or _PAIR). */
+/* The schedule AUTO resolves to for this shape (GMLP_VARIANT_SKINNY or _TENSOR). */
 int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);
 
 /*

@@ -14,6 +14,7 @@
 #include "stream_small_m.cuh"
 #include "umma_gemm.cuh"
 #include "umma_gemm_2cta.cuh"
+#include "umma_gemm_splitk.cuh"
 #include "umma_skinny.cuh"
 
 namespace {
@@ -74,6 +75,7 @@ struct DeviceState {
     int sm_count = 0;
     void* workspace = nullptr;
     uint64_t workspace_bytes = 0;
+    bool splitk_attr_set = false;
     bool umma_attr_set = false;
     bool pair_attr_set = false;
     bool rowscale_attr_set = false;
@@ -213,15 +215,28 @@ struct Layout {
     SkinnyPlan s1, s2;
 };
 
-// Schedule choice, from measurements on B200: the operand-swapped stream-K schedule wins while the split-K
-// partials (which grow with M) stay small next to the weights: always up to 32 tokens, up to 96 tokens when the
-// three weight matrices are at least 200 MB; CTA pairs from 1024 rows on; single-CTA tiles in between.
+// Schedule choice for AUTO, from A/B timings on B200.  SKINNY (operand-swapped stream-K) only pays for a
+// handful of tokens: on small and medium layers the one-CTA-per-tile kernels have too few tiles to fill the
+// GPU, and on large layers the two are within a few percent (the 128-row tiles are ahead in short bursts,
+// SKINNY in long runs under the power cap, where issuing 128-row MMAs for 8 real rows costs clock).  From 9
+// tokens on the 128-row tcgen05 tiles win everywhere, because their down projection splits K over a cluster
+// and reduces on chip.  TENSOR then picks, per GEMM, between single-CTA tiles and CTA pairs.
 int resolve_variant(int64_t M, int64_t d_model, int64_t d_ff, int32_t variant) {
+    (void)d_model;
+    (void)d_ff;
     if (variant != GMLP_VARIANT_AUTO) return variant;
-    const double weight_bytes = 6.0 * (double)d_model * (double)d_ff;
-    if (M <= 32 || (M <= 96 && weight_bytes >= 200e6)) return GMLP_VARIANT_SKINNY;
-    return M < 1024 ? GMLP_VARIANT_UMMA : GMLP_VARIANT_PAIR;
+    return M <= 8 ? GMLP_VARIANT_SKINNY : GMLP_VARIANT_TENSOR;
 }
+
+// TENSOR: which kernel each GEMM takes, by the number of 128-row blocks.  A CTA pair works on 256 rows, so an
+// odd block count leaves half a pair idle (measured: 3 blocks run faster on single CTAs, 2 and 4 on pairs);
+// from 8 blocks on the pair kernel's higher rate outweighs that.  The down projection has few output tiles
+// at small M and prefers the single-CTA kernel, which can split K over a cluster, until 8 blocks.
+bool gate_up_uses_pair(int64_t M) {
+    const int64_t mt = (M + 127) / 128;
+    return mt >= 8 || (mt >= 2 && mt % 2 == 0);
+}
+bool down_uses_pair(int64_t M) { return (M + 127) / 128 >= 8; }
 
 Layout make_layout(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int variant, int sm_count) {
     Layout L{};
@@ -409,11 +424,67 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     return GMLP_OK;
 }
 
+// Cluster size of the split-K schedule for a plain GEMM with num_m x ceil(N/128) output tiles, or 0 when the
+// ordinary one-CTA-per-tile schedule is to be used: the largest S in {4, 3, 2} whose tiles x S CTAs still fit
+// the SMs in one wave, provided every CTA keeps at least 8 k-blocks.
+int pick_split_k(int num_m, int64_t K, int64_t N, int sms) {
+    if (const char* e = getenv("GMLP_UMMA_SPLITK")) {               // tuning override: 0 disables, 2..4 forces
+        const int v = atoi(e);
+        if (v == 0) return 0;
+        if (v >= 2 && v <= 4 && (K + 63) / 64 >= v) return v;
+    }
+    const int64_t tiles = (int64_t)num_m * ((N + 127) / 128);
+    const int64_t nkb = (K + gmlp::kUmmaBK - 1) / gmlp::kUmmaBK;
+    for (int S = 4; S >= 2; --S)
+        if (tiles * S <= sms && nkb / S >= 8) return S;
+    return 0;
+}
+
+int launch_umma_splitk(DeviceState* dev, int S, const CUtensorMap& tmA, const CUtensorMap& tmB, bf16* C,
+                       int64_t M, int64_t K, int64_t N, int num_m, int a_box_rows, cudaStream_t st) {
+    if (!dev->splitk_attr_set) {
+        const int b = (int)gmlp::kSplitSmemBytes;
+        if (cudaFuncSetAttribute(gmlp::umma_splitk_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::umma_splitk_gemm_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::umma_splitk_gemm_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess)
+            return GMLP_ERR_LAUNCH;
+        dev->splitk_attr_set = true;
+    }
+    const int num_tiles = num_m * (int)((N + 127) / 128);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(num_tiles * S));
+    cfg.blockDim = dim3(gmlp::kUmmaThreads);
+    cfg.dynamicSmemBytes = gmlp::kSplitSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
+    cudaError_t err;
+    if (S == 4) err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<4>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows);
+    else if (S == 3) err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<3>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows);
+    else err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<2>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows);
+    if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
+    GMLP_CHECK_LAUNCH();
+    return GMLP_OK;
+}
+
 template <bool GATEUP>
 int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
                 int64_t M, int64_t K, int64_t N, cudaStream_t st) {
     CUtensorMap tmA, tmB0, tmB1;
-    if (!encode_2d(&tmA, A, (uint64_t)K, (uint64_t)M, gmlp::kUmmaBK, gmlp::kUmmaBM)) return GMLP_ERR_LAUNCH;
+    // TMA is markedly slower when a box has fewer than 16 rows inside the tensor; with so few rows in all, the
+    // box is made exactly M rows high instead (no out-of-range rows to fill)
+    int exact_below = 16;
+    if (const char* e = getenv("GMLP_UMMA_EXACT_BOX_BELOW")) exact_below = atoi(e);      // tuning override
+    const int a_box_rows = (M < exact_below && M < gmlp::kUmmaBM) ? (int)M : gmlp::kUmmaBM;
+    if (!encode_2d(&tmA, A, (uint64_t)K, (uint64_t)M, gmlp::kUmmaBK, (uint32_t)a_box_rows)) return GMLP_ERR_LAUNCH;
     if (!encode_2d(&tmB0, W0, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
     if (GATEUP) {
         if (!encode_2d(&tmB1, W1, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
@@ -423,6 +494,7 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     if (!dev->umma_attr_set) {
         const int b = (int)gmlp::kUmmaSmemBytes;
         if (cudaFuncSetAttribute(gmlp::umma_gemm_kernel<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::umma_gemm_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
             cudaFuncSetAttribute(gmlp::umma_gemm_kernel<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
             cudaFuncSetAttribute(gmlp::umma_gemm_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess)
             return GMLP_ERR_LAUNCH;
@@ -430,8 +502,16 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     }
     const int sms = dev->sm_count > 0 ? dev->sm_count : 148;
     const int num_m = (int)((M + gmlp::kUmmaBM - 1) / gmlp::kUmmaBM);
-    const int nb = GATEUP ? 4 : pick_umma_boxes(num_m, N, sms);
-    const int bn = GATEUP ? 128 : 64 * nb;
+    if (!GATEUP) {
+        // few output tiles: a cluster of S CTAs per tile splits K and reduces through distributed shared memory
+        const int S = pick_split_k(num_m, K, N, sms);
+        if (S >= 2) return launch_umma_splitk(dev, S, tmA, tmB0, C, M, K, N, num_m, a_box_rows, st);
+    }
+    // gate/up: 128 output columns per tile (two boxes of gate + two of up), or 64 when that still fits one wave
+    int gu_nb = (int64_t)num_m * ((N + 63) / 64) <= sms ? 2 : 4;
+    if (const char* e = getenv("GMLP_UMMA_GATEUP_NB")) gu_nb = atoi(e) == 2 ? 2 : 4;    // tuning override
+    const int nb = GATEUP ? gu_nb : pick_umma_boxes(num_m, N, sms);
+    const int bn = GATEUP ? 32 * nb : 64 * nb;
     const int num_n = (int)((N + bn - 1) / bn);
     const int num_tiles = num_m * num_n;
     cudaLaunchConfig_t cfg = {};
@@ -446,15 +526,18 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     cfg.numAttrs = 1;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
     cudaError_t err;
-    if (GATEUP)
+    if (GATEUP && nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr);
+                                 (const float*)nullptr, a_box_rows);
+    else if (GATEUP)
+        err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
+                                 (const float*)nullptr, a_box_rows);
     else if (nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr);
+                                 (const float*)nullptr, a_box_rows);
     else
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr);
+                                 (const float*)nullptr, a_box_rows);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -538,7 +621,7 @@ int forward_impl(const gmlp_args* a) {
     if (a == nullptr) return GMLP_ERR_NULL;
     if (a->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
     if (a->flags & ~kKnownFlags) return GMLP_ERR_FLAGS;
-    if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_PAIR) return GMLP_ERR_FLAGS;
+    if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_TENSOR) return GMLP_ERR_FLAGS;
     int rc = check_shape(a->M, a->d_model, a->d_ff);
     if (rc != GMLP_OK) return rc;
     if (a->M == 0) return GMLP_OK;              // nothing to compute; pointers may be NULL
@@ -613,6 +696,16 @@ int forward_impl(const gmlp_args* a) {
             if (rc == GMLP_OK) {
                 prof_mark("gate_up", st);
                 rc = launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st);
+                if (rc == GMLP_OK) prof_mark("down", st);
+            }
+            break;
+        case GMLP_VARIANT_TENSOR:
+            rc = gate_up_uses_pair(a->M) ? launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st)
+                                         : launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st);
+            if (rc == GMLP_OK) {
+                prof_mark("gate_up", st);
+                rc = down_uses_pair(a->M) ? launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st)
+                                          : launch_umma<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st);
                 if (rc == GMLP_OK) prof_mark("down", st);
             }
             break;
@@ -703,7 +796,7 @@ int gate_up_impl(const gmlp_args* a) {
     if (a == nullptr) return GMLP_ERR_NULL;
     if (a->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
     if (a->flags & ~kKnownFlags) return GMLP_ERR_FLAGS;
-    if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_PAIR) return GMLP_ERR_FLAGS;
+    if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_TENSOR) return GMLP_ERR_FLAGS;
     int rc = check_shape(a->M, a->d_model, a->d_ff);
     if (rc != GMLP_OK) return rc;
     if (a->M == 0) return GMLP_OK;
@@ -757,7 +850,7 @@ int gate_up_impl(const gmlp_args* a) {
         unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
         rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
         if (rc == GMLP_OK) rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, Hout, a->M, a->d_model, a->d_ff, st);
-    } else if (variant == GMLP_VARIANT_PAIR) {
+    } else if (variant == GMLP_VARIANT_PAIR || (variant == GMLP_VARIANT_TENSOR && gate_up_uses_pair(a->M))) {
         rc = launch_umma_pair<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st);
     } else {
         rc = launch_umma<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st);
@@ -851,7 +944,7 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
         const float* rc_ptr = r;
         cudaError_t err = pair
             ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr)
-            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr);
+            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("matmul_rowscale", st);
@@ -937,7 +1030,7 @@ int gmlp_forward_host(const gmlp_args* args, const void* X_host, void* Y_host) {
 
 uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant) {
     if (check_shape(M, d_model, d_ff) != GMLP_OK) return 0;
-    if (variant < GMLP_VARIANT_AUTO || variant > GMLP_VARIANT_PAIR) return 0;
+    if (variant < GMLP_VARIANT_AUTO || variant > GMLP_VARIANT_TENSOR) return 0;
     int sm_count = 148;
     int dev = -1;
     if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) {

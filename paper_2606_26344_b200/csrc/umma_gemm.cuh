@@ -89,7 +89,7 @@ template <bool GATEUP, int NB, bool ROWSCALE = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
-                 int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale)
+                 int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, int a_box_rows)
 {
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
     constexpr int KERNEL_ID = GATEUP ? 1 : 2;
@@ -150,6 +150,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (!ROWSCALE) ptx::grid_dependency_wait();           // A (Xn or H) may come from the previous kernel
             int it = 0;
             bool ok = true;
+            // the A box holds a_box_rows rows of 128 B (fewer than 128 only when the whole problem has fewer rows:
+            // the rest of the 128-row operand tile is never written and feeds accumulator rows nobody stores)
+            const uint32_t a_tx_bytes = (uint32_t)a_box_rows * 128u;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 const int m0 = (tile % num_m_tiles) * kUmmaBM;
                 const int n0 = (tile / num_m_tiles) * BN_OUT;
@@ -160,7 +163,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const uint32_t full = full0 + 8 * s;
                     const uint32_t a_dst = base + s * kStageBytes;
                     const uint32_t b_dst = a_dst + kUmmaABytes;
-                    ptx::mbar_arrive_expect_tx(full, kStageBytes);
+                    ptx::mbar_arrive_expect_tx(full, a_tx_bytes + NB * kUmmaBoxBBytes);
                     ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
 #pragma unroll
                     for (int i = 0; i < NB; ++i) {

@@ -1,0 +1,203 @@
+// Down-projection GEMM for medium M when there are far fewer output tiles than SMs.
+//
+// With one or two 128-row blocks, Y = H * Wd has only a few dozen 128 x 128 output tiles, and one
+// CTA per tile cannot pull its whole weight panel from HBM fast enough (a single SM sustains roughly
+// 50 GB/s through a TMA ring).  Here a thread-block cluster of S CTAs shares one output tile: CTA r
+// of the cluster runs the tcgen05 main loop over the r-th share of the K range, so S times as many
+// SMs stream the weights.  The partial accumulators are then reduced ON CHIP: after a cluster
+// barrier (every CTA's MMAs are done, the TMA rings are free) the non-leader CTAs copy their fp32
+// accumulators from TMEM into the leader's shared memory through distributed shared memory
+// (st.shared::cluster), a second cluster barrier publishes them, and the leader adds them to its own
+// accumulator in rank order (deterministic), rounds once and stores Y.  No partial ever touches
+// global memory and nothing waits on global flags.
+//
+// Tile 128 x 128, BK = 64, six stages of 32 KB (A 16 KB + two 64-column weight boxes), one tile per
+// cluster (the grid is tiles x S CTAs).  Operand layouts and descriptors as in umma_gemm.cuh.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+#include "umma_gemm.cuh"
+#include "umma_gemm_2cta.cuh"
+
+namespace gmlp {
+
+constexpr int kSplitStages = 6;
+constexpr uint32_t kSplitStageBytes = kUmmaABytes + 2 * kUmmaBoxBBytes;          // 32 KB
+constexpr uint32_t kSplitSmemBytes = kSplitStages * kSplitStageBytes + 1024 + 256;
+constexpr uint32_t kSplitPartialBytes = 128 * 128 * 4;                           // one CTA's fp32 tile: 64 KB
+
+__device__ __forceinline__ void st_cluster_f32x4(uint32_t cluster_addr, float a, float b, float c, float d) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "f"(a), "f"(b), "f"(c), "f"(d)
+                 : "memory");
+}
+
+template <int S>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                        bf16* __restrict__ C, int M, int K, int N, int num_m_tiles, int a_box_rows)
+{
+    static_assert(S >= 2 && (S - 1) * kSplitPartialBytes <= kSplitStages * kSplitStageBytes, "staging must fit the ring");
+    constexpr int KERNEL_ID = 9;
+    // D = fp32, A = B = bf16, A K-major, B MN-major, M = 128, N = 128
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                                ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - raw_addr);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + kSplitStages * kSplitStageBytes);
+    const uint32_t full0 = ptx::smem_addr(bars);
+    const uint32_t empty0 = ptx::smem_addr(bars + kSplitStages);
+    const uint32_t tfull = ptx::smem_addr(bars + 2 * kSplitStages);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kSplitStages + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();
+    const int tile = blockIdx.x / S;
+    const int m0 = (tile % num_m_tiles) * 128;
+    const int n0 = (tile / num_m_tiles) * 128;
+    const int nkb = (K + kUmmaBK - 1) / kUmmaBK;
+    const int kb0 = (int)(((long long)rank * nkb) / S), kb1 = (int)(((long long)(rank + 1) * nkb) / S);
+
+    ptx::launch_dependents();
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kSplitStages; ++s) {
+            ptx::mbar_init(full0 + 8 * s, 1);
+            ptx::mbar_init(empty0 + 8 * s, 1);
+        }
+        ptx::mbar_init(tfull, 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::fence_proxy_async_smem();
+        ptx::prefetch_tensormap(&tmA);
+        ptx::prefetch_tensormap(&tmB);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_addr(tmem_slot), 128);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            ptx::grid_dependency_wait();
+            int it = 0;
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                const int s = it % kSplitStages;
+                const uint32_t ph = (uint32_t)(it / kSplitStages) & 1u;
+                if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
+                const uint32_t full = full0 + 8 * s;
+                const uint32_t a_dst = base + s * kSplitStageBytes;
+                const uint32_t b_dst = a_dst + kUmmaABytes;
+                ptx::mbar_arrive_expect_tx(full, (uint32_t)a_box_rows * 128u + 2 * kUmmaBoxBBytes);
+                ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
+                ptx::tma_load_2d(b_dst, &tmB, n0, kb * kUmmaBK, full);
+                ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, n0 + 64, kb * kUmmaBK, full);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                const int s = it % kSplitStages;
+                const uint32_t ph = (uint32_t)(it / kSplitStages) & 1u;
+                if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
+                ptx::tc_fence_after_sync();
+                const uint32_t a_base = base + s * kSplitStageBytes;
+                const uint32_t b_base = a_base + kUmmaABytes;
+#pragma unroll
+                for (int k = 0; k < kUmmaBK / 16; ++k) {
+                    const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
+                    const uint64_t b_desc = ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
+                    ptx::umma_bf16(tmem_base, a_desc, b_desc, kIdesc, (it | k) != 0 ? 1u : 0u);
+                }
+                ptx::umma_commit(empty0 + 8 * s);
+            }
+            if (ok) ptx::umma_commit(tfull);
+        }
+        __syncwarp();
+    }
+
+    // every thread: wait until this CTA's accumulator is complete (which also means its MMAs no longer read the ring)
+    const bool acc_ok = wait_bounded(tfull, 0u, abort_flag, KERNEL_ID, 3);
+    ptx::tc_fence_after_sync();
+    __syncthreads();
+    ptx::cluster_sync();                                   // all rings of the cluster are free from here on
+
+    const int q = warp & 3;
+    const int rloc = q * 32 + lane;                        // row within the tile = TMEM lane (epilogue warps 2..5)
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    if (warp >= 2 && rank > 0) {
+        // copy this CTA's fp32 accumulator into the leader's ring: float4 (c4, row) at index c4 * 128 + row
+        const uint32_t remote = ptx::map_to_cta(base, 0) + (rank - 1) * kSplitPartialBytes;
+#pragma unroll 1
+        for (int c = 0; c < 128; c += 32) {
+            uint32_t v[32];
+            ptx::tmem_ld_32x32(taddr + c, v);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const bool z = !acc_ok;
+                st_cluster_f32x4(remote + (uint32_t)(((c >> 2) + j) * 128 + rloc) * 16u,
+                                 z ? 0.f : __uint_as_float(v[4 * j]), z ? 0.f : __uint_as_float(v[4 * j + 1]),
+                                 z ? 0.f : __uint_as_float(v[4 * j + 2]), z ? 0.f : __uint_as_float(v[4 * j + 3]));
+            }
+        }
+    }
+    __syncthreads();
+    ptx::cluster_sync();                                   // the partials are in the leader's shared memory
+    if (warp >= 2 && rank == 0) {
+        ptx::grid_dependency_wait();                       // C may still be read by the previous kernel
+        const int row = m0 + rloc;
+        bf16* crow = C + (size_t)row * N + n0;
+        const float4* stage = reinterpret_cast<const float4*>(base_ptr);
+#pragma unroll 1
+        for (int c = 0; c < 128; c += 32) {
+            uint32_t v[32];
+            ptx::tmem_ld_32x32(taddr + c, v);
+            ptx::tmem_ld_wait();
+            uint32_t packed[16];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                float4 acc = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                         __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+#pragma unroll
+                for (int s = 1; s < S; ++s) {                // fixed rank order
+                    const float4 p = stage[(size_t)(s - 1) * (kSplitPartialBytes / 16) + ((c >> 2) + j) * 128 + rloc];
+                    acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+                }
+                packed[2 * j] = pack_bf16x2(acc.x, acc.y);
+                packed[2 * j + 1] = pack_bf16x2(acc.z, acc.w);
+            }
+            if (row < M && acc_ok) {
+#pragma unroll
+                for (int v4 = 0; v4 < 4; ++v4) {
+                    if (n0 + c + v4 * 8 < N)
+                        *reinterpret_cast<uint4*>(crow + c + v4 * 8) =
+                            make_uint4(packed[4 * v4], packed[4 * v4 + 1], packed[4 * v4 + 2], packed[4 * v4 + 3]);
+                }
+            }
+        }
+    }
+
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, 128);
+    }
+}
+
+}  // namespace gmlp

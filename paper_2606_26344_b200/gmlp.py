@@ -20,7 +20,7 @@ STATIC_MAX_M = 16
 STATIC_SCRATCH_BYTES = 12 << 20
 FLAG_RMSNORM = 1 << 0
 FLAG_CHECKED = 1 << 2
-VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA, VARIANT_SKINNY, VARIANT_PAIR = 0, 1, 2, 3, 4, 5
+VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA, VARIANT_SKINNY, VARIANT_PAIR, VARIANT_TENSOR = 0, 1, 2, 3, 4, 5, 6
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgmlp.so")
 _lib = None

@@ -94,16 +94,17 @@ def test_workspace_sizes_and_variant_choice(lib):
     assert wb(M, dm, dff, 0, gmlp.VARIANT_UMMA) < h + 4096
     assert wb(8, dm, dff, 0, gmlp.VARIANT_STREAM) > wb(8, dm, dff, 0, gmlp.VARIANT_SIMT)     # split-K partials
     assert wb(8, dm, dff, 0, gmlp.VARIANT_STREAM) < 64 << 20
-    assert gmlp.pick_variant(8, dm, dff) == gmlp.VARIANT_SKINNY
+    # AUTO: the operand-swapped stream-K schedule for a handful of tokens, else the 128-row tensor-core tiles
+    # with a per-GEMM kernel choice
     assert gmlp.pick_variant(1, 2048, 5632) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(32, 2048, 5632) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(64, 2048, 5632) == gmlp.VARIANT_UMMA
-    assert gmlp.pick_variant(64, dm, dff) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(128, dm, dff) == gmlp.VARIANT_UMMA
-    assert gmlp.pick_variant(129, 2048, 5632) == gmlp.VARIANT_UMMA
-    assert gmlp.pick_variant(1000, 2048, 5632) == gmlp.VARIANT_UMMA
-    assert gmlp.pick_variant(2048, dm, dff) == gmlp.VARIANT_PAIR
-    assert gmlp.pick_variant(4096, 8192, 28672) == gmlp.VARIANT_PAIR
+    assert gmlp.pick_variant(8, 2048, 5632) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(9, 2048, 5632) == gmlp.VARIANT_TENSOR
+    assert gmlp.pick_variant(8, dm, dff) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(16, dm, dff) == gmlp.VARIANT_TENSOR
+    assert gmlp.pick_variant(129, 2048, 5632) == gmlp.VARIANT_TENSOR
+    assert gmlp.pick_variant(2048, dm, dff) == gmlp.VARIANT_TENSOR
+    assert gmlp.pick_variant(4096, 8192, 28672) == gmlp.VARIANT_TENSOR
+    assert wb(300, dm, dff, 0, gmlp.VARIANT_TENSOR) == wb(300, dm, dff, 0, gmlp.VARIANT_UMMA)
     assert gmlp.pick_variant(4, 60, 128) == gmlp.ERR_SHAPE
 
 

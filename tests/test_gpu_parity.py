@@ -15,10 +15,11 @@ pytestmark = pytest.mark.gpu
 
 SIMT, STREAM, UMMA, SKINNY, PAIR = (gmlp.VARIANT_SIMT, gmlp.VARIANT_STREAM, gmlp.VARIANT_UMMA, gmlp.VARIANT_SKINNY,
                                      gmlp.VARIANT_PAIR)
+TENSOR = gmlp.VARIANT_TENSOR
 
 
 # ---------------------------------------------------------------- small cases, every schedule
-@pytest.mark.parametrize("variant", [SIMT, STREAM, UMMA, SKINNY, PAIR])
+@pytest.mark.parametrize("variant", [SIMT, STREAM, UMMA, SKINNY, PAIR, TENSOR])
 def test_tiny_config_all_rows(variant):
     inp = I.make_inputs(I.WORKLOADS["tiny"])
     check_case(inp, variant, f"tiny/v{variant}")
@@ -59,6 +60,27 @@ def test_skinny_schedule_small_m(shape, rmsnorm):
     # stream-K contributors per tile (short K: tiles owned whole; long K: tiles split over several CTAs)
     M, dm, dff = shape
     check_case(I.custom_inputs(M, dm, dff, 400 + M, rmsnorm=rmsnorm, eps=1e-6), SKINNY, f"skinny{shape}")
+
+
+@pytest.mark.parametrize("rmsnorm", [False, True])
+@pytest.mark.parametrize("shape", [(77, 1024, 4096), (129, 2048, 2240), (100, 5120, 2048), (200, 3840, 1536),
+                                   (128, 4096, 1664), (1, 1024, 512 * 4 + 8)])
+def test_umma_down_projection_split_over_a_cluster(shape, rmsnorm):
+    """Few output tiles in the down projection: clusters of 4, 4 (uneven K shares), 3 and 2 CTAs split K and
+    reduce through distributed shared memory; last two: exactly 8 k-blocks per CTA, ragged K tail."""
+    M, dm, dff = shape
+    check_case(I.custom_inputs(M, dm, dff, 350 + M, rmsnorm=rmsnorm, eps=1e-5), UMMA, f"umma-splitk{shape}")
+
+
+@pytest.mark.parametrize("rmsnorm", [False, True])
+@pytest.mark.parametrize("shape", [(1, 1024, 2048), (9, 2048, 5632), (15, 520, 1096), (128, 512, 1024), (129, 1024, 1536),
+                                   (256, 512, 1088), (300, 1024, 2048), (512, 264, 520), (800, 512, 1024),
+                                   (897, 512, 1024), (1030, 320, 392)])
+def test_tensor_schedule_per_gemm_kernel_choice(shape, rmsnorm):
+    """1, 2, 3, 4, 7, 8 and 9 row blocks: single-CTA and CTA-pair kernels mixed between the two GEMMs; fewer than
+    16 rows: the operand box is exactly M rows high."""
+    M, dm, dff = shape
+    check_case(I.custom_inputs(M, dm, dff, 700 + M, rmsnorm=rmsnorm, eps=1e-5), TENSOR, f"tensor{shape}")
 
 
 def test_small_m_path_is_stable_over_many_back_to_back_calls():
@@ -238,7 +260,8 @@ def test_bounded_wait_reports_a_timeout_and_leaves_the_context_usable():
 
 
 @pytest.mark.parametrize("variant,M", [(SKINNY, 7), (SKINNY, 100), (UMMA, 130), (UMMA, 300), (PAIR, 300), (PAIR, 1030),
-                                       (STREAM, 5), (SIMT, 70)])
+                                       (STREAM, 5), (SIMT, 70), (UMMA, 9), (TENSOR, 9), (TENSOR, 300),
+                                       (TENSOR, 1030)])
 @pytest.mark.parametrize("rmsnorm", [False, True])
 def test_no_write_outside_y_and_workspace(variant, M, rmsnorm):
     # Y and the workspace are carved out of one buffer with guard bands around them; the bands must be
