@@ -203,6 +203,14 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
     const int64_t total = (int64_t)p.num_tiles * p.KB;
     const int sms = sm_count > 0 ? sm_count : 148;
     p.grid = (int)(total < sms ? total : sms);
+    // gate/up with half-size rings: two CTAs per SM keep more loads in flight (about 2 % on a large layer), as
+    // long as every CTA still gets 16 or more units, which also bounds the contributors of a tile
+    if (small && nmat == 2 && total >= (int64_t)32 * sms && p.KB / 16 + 2 <= gmlp::kSkinnyMaxContrib) p.grid = 2 * sms;
+    if (const char* e = getenv(nmat == 2 ? "GMLP_SKINNY_GRID1" : "GMLP_SKINNY_GRID2")) {   // tuning override
+        const int v = atoi(e);
+        if (v == -1) p.grid = (int)(p.num_tiles < total ? p.num_tiles : total);          // one CTA per tile
+        else if (v >= 1 && v <= total) p.grid = v;
+    }
     p.scratch_bytes = (uint64_t)p.grid * 2 * nmat * p.NH * p.Mpad * 128 * 4;
     return p;
 }
