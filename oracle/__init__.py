@@ -80,10 +80,18 @@ def _load():
         lib.gmlp_oracle_rows.argtypes = [u16p, u16p, u16p, u16p, u16p, ctypes.c_float, ctypes.c_int,
                                          ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                          i64p, ctypes.c_int64, f64p, u16p, u16p, ctypes.c_int]
+        lib.gmlp_oracle_rows_act.restype = ctypes.c_int
+        lib.gmlp_oracle_rows_act.argtypes = lib.gmlp_oracle_rows.argtypes + [ctypes.c_int, ctypes.c_double]
+        lib.gmlp_oracle_gate_act.restype = ctypes.c_double
+        lib.gmlp_oracle_gate_act.argtypes = [ctypes.c_double, ctypes.c_int, ctypes.c_double]
+        lib.gmlp_oracle_gate_act_array.restype = None
+        lib.gmlp_oracle_gate_act_array.argtypes = [f64p, f64p, ctypes.c_int64, ctypes.c_int, ctypes.c_double]
         lib.gmlp_oracle_gate_up_rows.restype = ctypes.c_int
         lib.gmlp_oracle_gate_up_rows.argtypes = [u16p, u16p, u16p, u16p, ctypes.c_float, ctypes.c_int,
                                                  ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                                  i64p, ctypes.c_int64, f64p, ctypes.c_int]
+        lib.gmlp_oracle_gate_up_rows_act.restype = ctypes.c_int
+        lib.gmlp_oracle_gate_up_rows_act.argtypes = lib.gmlp_oracle_gate_up_rows.argtypes + [ctypes.c_int, ctypes.c_double]
         lib.gmlp_oracle_rmsnorm_matmul_rows.restype = ctypes.c_int
         lib.gmlp_oracle_rmsnorm_matmul_rows.argtypes = [u16p, u16p, u16p, ctypes.c_float, ctypes.c_int64, ctypes.c_int64,
                                                         ctypes.c_int64, i64p, ctypes.c_int64, f64p, ctypes.c_int]
@@ -133,6 +141,18 @@ def silu(values) -> np.ndarray:
     return out
 
 
+ACT_KINDS = {"silu": 0, "swish": 1, "glu": 2}
+
+
+def gate_act(values, act: str = "silu", beta: float = 1.0) -> np.ndarray:
+    """The gate activation of the gated unit: silu g*sigmoid(g), swish g*sigmoid(beta*g), glu sigmoid(g)."""
+    lib = _load()
+    v = np.ascontiguousarray(values, dtype=np.float64)
+    out = np.empty_like(v)
+    lib.gmlp_oracle_gate_act_array(_p(v, ctypes.c_double), _p(out, ctypes.c_double), v.size, ACT_KINDS[act], float(beta))
+    return out
+
+
 def rmsnorm_row(x_bits, gamma_bits=None, eps: float = 1e-5):
     """One row of the RMSNorm prologue.  Returns (xn bf16 bits, r as float64)."""
     lib = _load()
@@ -150,7 +170,7 @@ def max_threads() -> int:
 
 
 def gmlp_rows(X, Wg, Wu, Wd, rows=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False,
-              num_threads: int = 0, want_h: bool = False, want_xn: bool = False):
+              num_threads: int = 0, want_h: bool = False, want_xn: bool = False, act: str = "silu", beta: float = 1.0):
     """Reference Y (float64, not rounded) for the selected rows of X.
 
     X [M, d_model], Wg/Wu [d_model, d_ff], Wd [d_ff, d_model]: uint16 bf16 bit patterns.
@@ -174,12 +194,16 @@ def gmlp_rows(X, Wg, Wu, Wd, rows=None, gamma=None, eps: float = 1e-5, rmsnorm: 
     Y = np.zeros((R, d_model), dtype=np.float64)
     H = np.zeros((R, d_ff), dtype=np.uint16) if want_h else None
     Xn = np.zeros((R, d_model), dtype=np.uint16) if want_xn else None
-    rc = lib.gmlp_oracle_rows(_p(X, ctypes.c_uint16), _p(Wg, ctypes.c_uint16), _p(Wu, ctypes.c_uint16),
-                              _p(Wd, ctypes.c_uint16), None if g is None else _p(g, ctypes.c_uint16),
-                              ctypes.c_float(eps), int(bool(rmsnorm)), M, d_model, d_ff,
-                              _p(rows, ctypes.c_int64), R, _p(Y, ctypes.c_double),
-                              None if H is None else _p(H, ctypes.c_uint16),
-                              None if Xn is None else _p(Xn, ctypes.c_uint16), int(num_threads))
+    common = (_p(X, ctypes.c_uint16), _p(Wg, ctypes.c_uint16), _p(Wu, ctypes.c_uint16),
+              _p(Wd, ctypes.c_uint16), None if g is None else _p(g, ctypes.c_uint16),
+              ctypes.c_float(eps), int(bool(rmsnorm)), M, d_model, d_ff,
+              _p(rows, ctypes.c_int64), R, _p(Y, ctypes.c_double),
+              None if H is None else _p(H, ctypes.c_uint16),
+              None if Xn is None else _p(Xn, ctypes.c_uint16), int(num_threads))
+    if act == "silu":
+        rc = lib.gmlp_oracle_rows(*common)
+    else:
+        rc = lib.gmlp_oracle_rows_act(*common, ACT_KINDS[act], float(beta))
     if rc != 0:
         raise RuntimeError(f"gmlp_oracle_rows failed ({rc})")
     out = [Y]
@@ -191,7 +215,7 @@ def gmlp_rows(X, Wg, Wu, Wd, rows=None, gamma=None, eps: float = 1e-5, rmsnorm: 
 
 
 def gate_up_rows(X, Wg, Wu, rows=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False,
-                 num_threads: int = 0) -> np.ndarray:
+                 num_threads: int = 0, act: str = "silu", beta: float = 1.0) -> np.ndarray:
     """Reference silu(Xn Wg) * (Xn Wu) (float64, not rounded) for the selected rows: the gate/up half alone."""
     lib = _load()
     X, Wg, Wu = _u16(X, "X"), _u16(Wg, "Wg"), _u16(Wu, "Wu")
@@ -208,10 +232,14 @@ def gate_up_rows(X, Wg, Wu, rows=None, gamma=None, eps: float = 1e-5, rmsnorm: b
         if g.size != d_model:
             raise ValueError("gamma size")
     P = np.zeros((rows.size, d_ff), dtype=np.float64)
-    rc = lib.gmlp_oracle_gate_up_rows(_p(X, ctypes.c_uint16), _p(Wg, ctypes.c_uint16), _p(Wu, ctypes.c_uint16),
-                                      None if g is None else _p(g, ctypes.c_uint16), ctypes.c_float(eps),
-                                      int(bool(rmsnorm)), M, d_model, d_ff, _p(rows, ctypes.c_int64), rows.size,
-                                      _p(P, ctypes.c_double), int(num_threads))
+    common = (_p(X, ctypes.c_uint16), _p(Wg, ctypes.c_uint16), _p(Wu, ctypes.c_uint16),
+              None if g is None else _p(g, ctypes.c_uint16), ctypes.c_float(eps),
+              int(bool(rmsnorm)), M, d_model, d_ff, _p(rows, ctypes.c_int64), rows.size,
+              _p(P, ctypes.c_double), int(num_threads))
+    if act == "silu":
+        rc = lib.gmlp_oracle_gate_up_rows(*common)
+    else:
+        rc = lib.gmlp_oracle_gate_up_rows_act(*common, ACT_KINDS[act], float(beta))
     if rc != 0:
         raise RuntimeError(f"gmlp_oracle_gate_up_rows failed ({rc})")
     return P

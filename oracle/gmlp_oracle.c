@@ -79,6 +79,22 @@ double gmlp_oracle_silu(double g)
 }
 
 /*
+ * Gate activation of the gated unit h = act(g) * u.  The paper's Gated MLP uses SiLU; its benchmark list
+ * (Section 6.1) also names SwiGLU- and GLU-gated forms without defining them.  Reading taken (the
+ * definitions of the GLU-variants literature): kind 0 SiLU g*sigmoid(g); kind 1 Swish-beta
+ * g*sigmoid(beta*g) (beta = 1 is SiLU); kind 2 GLU sigmoid(g).  Anything else: NaN.
+ */
+double gmlp_oracle_gate_act(double g, int kind, double beta)
+{
+    switch (kind) {
+        case 0: return gmlp_oracle_silu(g);
+        case 1: return g / (1.0 + exp(-(beta * g)));
+        case 2: return 1.0 / (1.0 + exp(-g));
+        default: return NAN;
+    }
+}
+
+/*
  * RMSNorm of one row (Eq. 1; graph order square, mean, add eps, rsqrt, multiply):
  *   ms = (1/d) sum_k x[k]^2 ;  r = 1/sqrt(ms + eps) ;  xn[k] = bf16_rn(x[k] * r * gamma[k]).
  * Also returns r through *r_out when non-NULL.
@@ -109,11 +125,12 @@ void gmlp_oracle_rmsnorm_row(const uint16_t* x, const uint16_t* gamma, float eps
  * (may be NULL); Xn_bits [n_rows, d_model] (may be NULL; the row as fed to the matmuls).
  * Returns 0, or -1 on a bad argument / allocation failure.
  */
-int gmlp_oracle_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu, const uint16_t* Wd,
-                     const uint16_t* gamma, float eps, int rmsnorm,
-                     int64_t M, int64_t d_model, int64_t d_ff,
-                     const int64_t* rows, int64_t n_rows,
-                     double* Y_ref, uint16_t* H_bits, uint16_t* Xn_bits, int num_threads)
+int gmlp_oracle_rows_act(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu, const uint16_t* Wd,
+                         const uint16_t* gamma, float eps, int rmsnorm,
+                         int64_t M, int64_t d_model, int64_t d_ff,
+                         const int64_t* rows, int64_t n_rows,
+                         double* Y_ref, uint16_t* H_bits, uint16_t* Xn_bits, int num_threads,
+                         int act_kind, double act_beta)
 {
     if (!X || !Wg || !Wu || !Wd || !rows || !Y_ref || M < 0 || d_model <= 0 || d_ff <= 0 || n_rows < 0)
         return -1;
@@ -160,7 +177,7 @@ int gmlp_oracle_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu, 
                 }
                 /* a3, a4: H = bf16_rn(silu(G) * U), rounding R1 */
                 for (int64_t n = 0; n < d_ff; ++n) {
-                    uint16_t hb = gmlp_oracle_bf16_rn(gmlp_oracle_silu(g[n]) * u[n]);
+                    uint16_t hb = gmlp_oracle_bf16_rn(gmlp_oracle_gate_act(g[n], act_kind, act_beta) * u[n]);
                     if (H_bits) H_bits[i * d_ff + n] = hb;
                     h[n] = gmlp_oracle_bf16_to_double(hb);
                 }
@@ -180,16 +197,28 @@ int gmlp_oracle_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu, 
     return failed ? -1 : 0;
 }
 
+/* The operator as the paper states it: SiLU gate. */
+int gmlp_oracle_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu, const uint16_t* Wd,
+                     const uint16_t* gamma, float eps, int rmsnorm,
+                     int64_t M, int64_t d_model, int64_t d_ff,
+                     const int64_t* rows, int64_t n_rows,
+                     double* Y_ref, uint16_t* H_bits, uint16_t* Xn_bits, int num_threads)
+{
+    return gmlp_oracle_rows_act(X, Wg, Wu, Wd, gamma, eps, rmsnorm, M, d_model, d_ff, rows, n_rows,
+                                Y_ref, H_bits, Xn_bits, num_threads, 0, 1.0);
+}
+
 /*
  * The gate/up half on its own ("Matmul+Matmul+SiLU+Mul" of the paper's benchmark list, Section 6.1):
  *   P[i, n] = silu(sum_k xn[k] Wg[k, n]) * (sum_k xn[k] Wu[k, n])      for the selected rows,
  * returned in fp64 WITHOUT the final rounding (the GPU rounds P once to bf16; the tolerance is taken
  * around this value).  Same conventions as gmlp_oracle_rows; the optional RMSNorm prologue rounds Xn.
  */
-int gmlp_oracle_gate_up_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu,
-                             const uint16_t* gamma, float eps, int rmsnorm,
-                             int64_t M, int64_t d_model, int64_t d_ff,
-                             const int64_t* rows, int64_t n_rows, double* P, int num_threads)
+int gmlp_oracle_gate_up_rows_act(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu,
+                                 const uint16_t* gamma, float eps, int rmsnorm,
+                                 int64_t M, int64_t d_model, int64_t d_ff,
+                                 const int64_t* rows, int64_t n_rows, double* P, int num_threads,
+                                 int act_kind, double act_beta)
 {
     if (!X || !Wg || !Wu || !rows || !P || M < 0 || d_model <= 0 || d_ff <= 0 || n_rows < 0) return -1;
     for (int64_t i = 0; i < n_rows; ++i)
@@ -226,12 +255,21 @@ int gmlp_oracle_gate_up_rows(const uint16_t* X, const uint16_t* Wg, const uint16
                         u[n] += xk * gmlp_oracle_bf16_to_double(wu[n]);
                     }
                 }
-                for (int64_t n = 0; n < d_ff; ++n) P[i * d_ff + n] = gmlp_oracle_silu(g[n]) * u[n];
+                for (int64_t n = 0; n < d_ff; ++n) P[i * d_ff + n] = gmlp_oracle_gate_act(g[n], act_kind, act_beta) * u[n];
             }
         }
         free(xn); free(xnb); free(g); free(u);
     }
     return failed ? -1 : 0;
+}
+
+int gmlp_oracle_gate_up_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu,
+                             const uint16_t* gamma, float eps, int rmsnorm,
+                             int64_t M, int64_t d_model, int64_t d_ff,
+                             const int64_t* rows, int64_t n_rows, double* P, int num_threads)
+{
+    return gmlp_oracle_gate_up_rows_act(X, Wg, Wu, gamma, eps, rmsnorm, M, d_model, d_ff, rows, n_rows, P,
+                                        num_threads, 0, 1.0);
 }
 
 /*
@@ -293,6 +331,11 @@ int gmlp_oracle_rmsnorm_matmul_rows(const uint16_t* X, const uint16_t* W, const 
 void gmlp_oracle_bf16_rn_array(const double* v, uint16_t* out, int64_t n)
 {
     for (int64_t i = 0; i < n; ++i) out[i] = gmlp_oracle_bf16_rn(v[i]);
+}
+
+void gmlp_oracle_gate_act_array(const double* v, double* out, int64_t n, int kind, double beta)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = gmlp_oracle_gate_act(v[i], kind, beta);
 }
 
 void gmlp_oracle_silu_array(const double* v, double* out, int64_t n)
