@@ -90,6 +90,10 @@ def _load():
         lib.gmlp_oracle_gate_up_rows.argtypes = [u16p, u16p, u16p, u16p, ctypes.c_float, ctypes.c_int,
                                                  ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                                  i64p, ctypes.c_int64, f64p, ctypes.c_int]
+        lib.gmlp_oracle_matmul_add_rmsnorm_rows.restype = ctypes.c_int
+        lib.gmlp_oracle_matmul_add_rmsnorm_rows.argtypes = [u16p, u16p, u16p, u16p, ctypes.c_float, ctypes.c_int64,
+                                                            ctypes.c_int64, ctypes.c_int64, i64p, ctypes.c_int64,
+                                                            u16p, f64p, f64p, ctypes.c_int]
         lib.gmlp_oracle_gate_up_rows_act.restype = ctypes.c_int
         lib.gmlp_oracle_gate_up_rows_act.argtypes = lib.gmlp_oracle_gate_up_rows.argtypes + [ctypes.c_int, ctypes.c_double]
         lib.gmlp_oracle_rmsnorm_matmul_rows.restype = ctypes.c_int
@@ -269,6 +273,37 @@ def rmsnorm_matmul_rows(X, W, rows=None, gamma=None, eps: float = 1e-5, num_thre
     if rc != 0:
         raise RuntimeError(f"gmlp_oracle_rmsnorm_matmul_rows failed ({rc})")
     return Z
+
+
+def matmul_add_rmsnorm_rows(X, W, R, rows=None, gamma=None, eps: float = 1e-5, num_threads: int = 0):
+    """Reference for S = X @ W + R, Z = RMSNorm(bf16(S)) on the selected rows.
+
+    Returns (S_bits uint16 [rows, N], S_ref float64 unrounded, Z float64)."""
+    lib = _load()
+    X, W, R = _u16(X, "X"), _u16(W, "W"), _u16(R, "R")
+    M, K = X.shape
+    N = W.shape[1]
+    if W.shape[0] != K or R.shape != (M, N):
+        raise ValueError("shape mismatch")
+    if rows is None:
+        rows = np.arange(M, dtype=np.int64)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    g = None
+    if gamma is not None:
+        g = _u16(gamma, "gamma").reshape(-1)
+        if g.size != N:
+            raise ValueError("gamma size")
+    Sb = np.zeros((rows.size, N), dtype=np.uint16)
+    Sr = np.zeros((rows.size, N), dtype=np.float64)
+    Z = np.zeros((rows.size, N), dtype=np.float64)
+    rc = lib.gmlp_oracle_matmul_add_rmsnorm_rows(_p(X, ctypes.c_uint16), _p(W, ctypes.c_uint16), _p(R, ctypes.c_uint16),
+                                                 None if g is None else _p(g, ctypes.c_uint16), ctypes.c_float(eps),
+                                                 M, K, N, _p(rows, ctypes.c_int64), rows.size,
+                                                 _p(Sb, ctypes.c_uint16), _p(Sr, ctypes.c_double), _p(Z, ctypes.c_double),
+                                                 int(num_threads))
+    if rc != 0:
+        raise RuntimeError(f"gmlp_oracle_matmul_add_rmsnorm_rows failed ({rc})")
+    return Sb, Sr, Z
 
 
 def naive_matmul(A, B) -> np.ndarray:

@@ -327,6 +327,71 @@ int gmlp_oracle_rmsnorm_matmul_rows(const uint16_t* X, const uint16_t* W, const 
     return failed ? -1 : 0;
 }
 
+/*
+ * A matrix multiplication, a residual addition and RMSNorm ("Matmul+Add+RMSNorm" of the paper's
+ * benchmark list, Section 6.1; the paper names the chain and does not spell out the graph):
+ *     S = X * W + R,     Z = RMSNorm(S)      (Eq. 1 along the last dimension, N)
+ * Readings taken: S is an output as well (the updated residual stream), stored in bf16 with ONE
+ * rounding of the fp64 sum; the RMSNorm is the one of Eq. (1) applied to the STORED S (what a
+ * following operator would read), in fp64, with the optional per-column gain gamma [N]; Z is left in
+ * fp64 (the value the tolerance is taken around).
+ * X [M, K], W [K, N], R [M, N], gamma [N] or NULL: bf16 bit patterns.  For the selected rows:
+ * S_bits [n_rows, N] bf16 bits (may be NULL), S_ref [n_rows, N] fp64 unrounded sums (may be NULL),
+ * Z [n_rows, N] fp64.
+ */
+int gmlp_oracle_matmul_add_rmsnorm_rows(const uint16_t* X, const uint16_t* W, const uint16_t* R,
+                                        const uint16_t* gamma, float eps, int64_t M, int64_t K, int64_t N,
+                                        const int64_t* rows, int64_t n_rows,
+                                        uint16_t* S_bits, double* S_ref, double* Z, int num_threads)
+{
+    if (!X || !W || !R || !rows || !Z || M < 0 || K <= 0 || N <= 0 || n_rows < 0) return -1;
+    for (int64_t i = 0; i < n_rows; ++i)
+        if (rows[i] < 0 || rows[i] >= M) return -1;
+    int failed = 0;
+#ifdef _OPENMP
+    if (num_threads > 0) omp_set_num_threads(num_threads);
+#else
+    (void)num_threads;
+#endif
+#pragma omp parallel
+    {
+        double* s = (double*)malloc(sizeof(double) * (size_t)N);
+        if (!s) {
+#pragma omp atomic write
+            failed = 1;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int64_t i = 0; i < n_rows; ++i) {
+                const uint16_t* x = X + rows[i] * K;
+                const uint16_t* res = R + rows[i] * N;
+                for (int64_t n = 0; n < N; ++n) s[n] = 0.0;
+                for (int64_t k = 0; k < K; ++k) {
+                    const double xk = gmlp_oracle_bf16_to_double(x[k]);
+                    const uint16_t* w = W + k * N;
+                    for (int64_t n = 0; n < N; ++n) s[n] += xk * gmlp_oracle_bf16_to_double(w[n]);
+                }
+                double ss = 0.0;
+                for (int64_t n = 0; n < N; ++n) {
+                    s[n] += gmlp_oracle_bf16_to_double(res[n]);
+                    if (S_ref) S_ref[i * N + n] = s[n];
+                    const uint16_t sb = gmlp_oracle_bf16_rn(s[n]);
+                    if (S_bits) S_bits[i * N + n] = sb;
+                    s[n] = gmlp_oracle_bf16_to_double(sb);
+                    ss += s[n] * s[n];
+                }
+                const double r = 1.0 / sqrt(ss / (double)N + (double)eps);
+                for (int64_t n = 0; n < N; ++n) {
+                    double v = s[n] * r;
+                    if (gamma) v *= gmlp_oracle_bf16_to_double(gamma[n]);
+                    Z[i * N + n] = v;
+                }
+            }
+        }
+        free(s);
+    }
+    return failed ? -1 : 0;
+}
+
 /* Array forms of the two scalar helpers (plain loops), for the tests. */
 void gmlp_oracle_bf16_rn_array(const double* v, uint16_t* out, int64_t n)
 {
