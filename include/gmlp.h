@@ -59,7 +59,15 @@ typedef enum gmlp_status {
 
 enum {
     GMLP_FLAG_RMSNORM = 1u << 0, /* apply the RMSNorm prologue to X */
-    GMLP_FLAG_CHECKED = 1u << 2  /* synchronise the stream and report the device status before returning */
+    GMLP_FLAG_CHECKED = 1u << 2, /* synchronise the stream and report the device status before returning */
+    /* Gate activation of the gated unit H = act(G) (.) U.  The paper's operator uses SiLU (no flag); its
+     * benchmark list (Section 6.1) also names SwiGLU- and GLU-gated forms, which differ only in act:
+     *   none             act(g) = g * sigmoid(g)              (SiLU)
+     *   ACT_SWISH        act(g) = g * sigmoid(act_beta * g)   (Swish-beta; beta = 1 is SiLU bit for bit)
+     *   ACT_GLU          act(g) = sigmoid(g)                  (GLU)
+     * Setting both is GMLP_ERR_FLAGS, and so is a NaN or infinite act_beta with ACT_SWISH. */
+    GMLP_FLAG_ACT_SWISH = 1u << 5,
+    GMLP_FLAG_ACT_GLU = 1u << 6
 };
 
 /* Kernel schedule.  AUTO picks by shape; the others force one schedule (tests, benchmarks). */
@@ -90,13 +98,16 @@ typedef struct gmlp_args {
     void* stream;             /* cudaStream_t; NULL = the legacy default stream */
     void* workspace;          /* device scratch of >= gmlp_workspace_bytes(...) bytes, 256-byte aligned, or NULL */
     uint64_t workspace_bytes;
+    float act_beta;           /* beta of GMLP_FLAG_ACT_SWISH; ignored without that flag */
+    uint32_t reserved;        /* must be 0 */
 } gmlp_args;
 
 /*
  * The operator as the paper states it: Y = (silu(X Wg) (.) (X Wu)) Wd.
  * Runs on the stream set by gmlp_set_stream (default: legacy default stream) with the
  * library-owned workspace.  With GMLP_FLAG_RMSNORM the prologue has no gain and uses the eps
- * set by gmlp_set_default_eps (default 1e-5).  Asynchronous; returns a gmlp_status.
+ * set by gmlp_set_default_eps (default 1e-5); GMLP_FLAG_ACT_SWISH here means beta = 1 (use
+ * gmlp_forward_ex for another beta).  Asynchronous; returns a gmlp_status.
  */
 int gmlp_forward(const void* X, const void* Wg, const void* Wu, const void* Wd, void* Y,
                  int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);

@@ -24,7 +24,21 @@ using gmlp::bf16;
 constexpr int kVersion = 100;
 constexpr int kMaxDevices = 64;
 constexpr int64_t kMaxDim = (int64_t)1 << 30;      // per-dimension limit (TMA coordinates are int32)
-constexpr uint32_t kKnownFlags = GMLP_FLAG_RMSNORM | GMLP_FLAG_CHECKED;
+constexpr uint32_t kKnownFlags = GMLP_FLAG_RMSNORM | GMLP_FLAG_CHECKED | GMLP_FLAG_ACT_SWISH | GMLP_FLAG_ACT_GLU;
+constexpr gmlp::GateAct kSilu = {1.0f, 0};
+
+// Gate activation named by the flags (SiLU when none is set); false for a contradictory or non-finite request.
+bool gate_act_from(uint32_t flags, float beta, gmlp::GateAct* out) {
+    const bool swish = flags & GMLP_FLAG_ACT_SWISH, glu = flags & GMLP_FLAG_ACT_GLU;
+    if (swish && glu) return false;
+    *out = kSilu;
+    if (swish) {
+        if (!(beta == beta) || beta - beta != 0.0f) return false;      // NaN or infinite
+        out->beta = beta;
+    }
+    if (glu) out->glu = 1;
+    return true;
+}
 
 thread_local cudaStream_t t_stream = nullptr;
 thread_local float t_default_eps = 1e-5f;
@@ -334,14 +348,14 @@ int launch_rmsnorm(const bf16* X, const bf16* gain, bf16* Xn, int64_t M, int64_t
 }
 
 int run_simt(const bf16* A, const bf16* Wg, const bf16* Wu, const bf16* Wd, bf16* H, bf16* Y,
-             int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st) {
+             int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st, gmlp::GateAct act) {
     const int T = gmlp::kSimtTile;
     dim3 g1((unsigned)((d_ff + T - 1) / T), (unsigned)((M + T - 1) / T));
-    gmlp::simt_gemm_kernel<true><<<g1, 256, 0, st>>>(A, Wg, Wu, H, M, (int)d_model, (int)d_ff);
+    gmlp::simt_gemm_kernel<true><<<g1, 256, 0, st>>>(A, Wg, Wu, H, M, (int)d_model, (int)d_ff, act);
     GMLP_CHECK_LAUNCH();
     prof_mark("gate_up", st);
     dim3 g2((unsigned)((d_model + T - 1) / T), (unsigned)((M + T - 1) / T));
-    gmlp::simt_gemm_kernel<false><<<g2, 256, 0, st>>>(H, Wd, nullptr, Y, M, (int)d_ff, (int)d_model);
+    gmlp::simt_gemm_kernel<false><<<g2, 256, 0, st>>>(H, Wd, nullptr, Y, M, (int)d_ff, (int)d_model, kSilu);
     GMLP_CHECK_LAUNCH();
     prof_mark("down", st);
     return GMLP_OK;
@@ -349,27 +363,28 @@ int run_simt(const bf16* A, const bf16* Wg, const bf16* Wu, const bf16* Wd, bf16
 
 template <bool GATEUP>
 int launch_stream(const StreamPlan& p, const bf16* A, const bf16* W0, const bf16* W1, float* partial,
-                  unsigned int* counters, bf16* out, int64_t M, int64_t K, int64_t N, cudaStream_t st) {
+                  unsigned int* counters, bf16* out, int64_t M, int64_t K, int64_t N, cudaStream_t st,
+                  gmlp::GateAct act = kSilu) {
     dim3 grid((unsigned)p.slabs, (unsigned)(p.KS * (GATEUP ? 2 : 1)), (unsigned)p.row_tiles);
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
     switch (p.MT) {
-        case 1: gmlp::stream_gemm_kernel<1, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS); break;
-        case 2: gmlp::stream_gemm_kernel<2, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS); break;
-        case 4: gmlp::stream_gemm_kernel<4, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS); break;
-        default: gmlp::stream_gemm_kernel<8, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS); break;
+        case 1: gmlp::stream_gemm_kernel<1, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS, act); break;
+        case 2: gmlp::stream_gemm_kernel<2, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS, act); break;
+        case 4: gmlp::stream_gemm_kernel<4, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS, act); break;
+        default: gmlp::stream_gemm_kernel<8, GATEUP><<<grid, gmlp::kStreamThreads, 0, st>>>(A, W0, W1, partial, counters, out, Mi, Ki, Ni, p.kchunk, p.KS, act); break;
     }
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
 }
 
 int run_stream(DeviceState* dev, const Layout& L, uint8_t* ws, const bf16* A, const bf16* Wg, const bf16* Wu, const bf16* Wd, bf16* H,
-               bf16* Y, int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st) {
+               bf16* Y, int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st, gmlp::GateAct act) {
     float* partial = reinterpret_cast<float*>(ws + L.partial_off);
     unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
     unsigned int* c2 = c1 + L.p1.row_tiles * L.p1.slabs;
     int rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
     if (rc != GMLP_OK) return rc;
-    rc = launch_stream<true>(L.p1, A, Wg, Wu, partial, c1, H, M, d_model, d_ff, st);
+    rc = launch_stream<true>(L.p1, A, Wg, Wu, partial, c1, H, M, d_model, d_ff, st, act);
     if (rc != GMLP_OK) return rc;
     prof_mark("gate_up", st);
     rc = launch_stream<false>(L.p2, H, Wd, nullptr, partial, c2, Y, M, d_ff, d_model, st);
@@ -389,7 +404,7 @@ int pick_umma_boxes(int64_t num_m, int64_t N, int sms) {
 
 template <bool GATEUP>
 int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
-                     int64_t M, int64_t K, int64_t N, cudaStream_t st) {
+                     int64_t M, int64_t K, int64_t N, cudaStream_t st, gmlp::GateAct act = kSilu) {
     CUtensorMap tmA, tmB0, tmB1;
     if (!encode_2d(&tmA, A, (uint64_t)K, (uint64_t)M, gmlp::kUmmaBK, 128)) return GMLP_ERR_LAUNCH;
     if (!encode_2d(&tmB0, W0, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
@@ -426,7 +441,7 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
     if (cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m,
-                           num_tiles, (const float*)nullptr) != cudaSuccess)
+                           num_tiles, (const float*)nullptr, act) != cudaSuccess)
         return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -485,7 +500,7 @@ int launch_umma_splitk(DeviceState* dev, int S, const CUtensorMap& tmA, const CU
 
 template <bool GATEUP>
 int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
-                int64_t M, int64_t K, int64_t N, cudaStream_t st) {
+                int64_t M, int64_t K, int64_t N, cudaStream_t st, gmlp::GateAct act = kSilu) {
     CUtensorMap tmA, tmB0, tmB1;
     // TMA is markedly slower when a box has fewer than 16 rows inside the tensor; with so few rows in all, the
     // box is made exactly M rows high instead (no out-of-range rows to fill)
@@ -536,16 +551,16 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     cudaError_t err;
     if (GATEUP && nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows);
+                                 (const float*)nullptr, a_box_rows, act);
     else if (GATEUP)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows);
+                                 (const float*)nullptr, a_box_rows, act);
     else if (nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows);
+                                 (const float*)nullptr, a_box_rows, act);
     else
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows);
+                                 (const float*)nullptr, a_box_rows, act);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -553,7 +568,8 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
 
 template <bool GATEUP>
 int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf16* W0, const bf16* W1, float* scratch,
-                  unsigned int* counters, bf16* out, int64_t M, int64_t K, int64_t N, cudaStream_t st) {
+                  unsigned int* counters, bf16* out, int64_t M, int64_t K, int64_t N, cudaStream_t st,
+                  gmlp::GateAct act = kSilu) {
     if (p.stages < 2 || p.tmem_cols > 512) return GMLP_ERR_UNSUPPORTED;
     CUtensorMap tmX, tmW0, tmW1;
     if (!encode_2d(&tmX, X, (uint64_t)K, (uint64_t)M, 64, (uint32_t)p.Mpad)) return GMLP_ERR_LAUNCH;
@@ -590,23 +606,24 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
     cudaError_t err;
     if (p.NH == 2)
         err = cudaLaunchKernelEx(&cfg, gmlp::skinny_gemm_kernel<GATEUP, 2>, tmX, tmW0, tmW1, scratch, counters, out,
-                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first);
+                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first, act);
     else
         err = cudaLaunchKernelEx(&cfg, gmlp::skinny_gemm_kernel<GATEUP, 1>, tmX, tmW0, tmW1, scratch, counters, out,
-                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first);
+                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first, act);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
 }
 
 int run_skinny(DeviceState* dev, const Layout& L, uint8_t* ws, const bf16* A, const bf16* Wg, const bf16* Wu,
-               const bf16* Wd, bf16* H, bf16* Y, int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st) {
+               const bf16* Wd, bf16* H, bf16* Y, int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st,
+               gmlp::GateAct act) {
     float* scratch = reinterpret_cast<float*>(ws + L.partial_off);
     unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
     unsigned int* c2 = c1 + L.s1.num_tiles;
     int rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
     if (rc != GMLP_OK) return rc;
-    rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, H, M, d_model, d_ff, st);
+    rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, H, M, d_model, d_ff, st, act);
     if (rc != GMLP_OK) return rc;
     prof_mark("gate_up", st);
     rc = launch_skinny<false>(dev, L.s2, H, Wd, nullptr, scratch, c2, Y, M, d_ff, d_model, st);
@@ -629,6 +646,8 @@ int forward_impl(const gmlp_args* a) {
     if (a == nullptr) return GMLP_ERR_NULL;
     if (a->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
     if (a->flags & ~kKnownFlags) return GMLP_ERR_FLAGS;
+    gmlp::GateAct act;
+    if (a->reserved != 0 || !gate_act_from(a->flags, a->act_beta, &act)) return GMLP_ERR_FLAGS;
     if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_TENSOR) return GMLP_ERR_FLAGS;
     int rc = check_shape(a->M, a->d_model, a->d_ff);
     if (rc != GMLP_OK) return rc;
@@ -691,16 +710,16 @@ int forward_impl(const gmlp_args* a) {
 
     switch (variant) {
         case GMLP_VARIANT_SIMT:
-            rc = run_simt(A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
+            rc = run_simt(A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st, act);
             break;
         case GMLP_VARIANT_STREAM:
-            rc = run_stream(dev, L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
+            rc = run_stream(dev, L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st, act);
             break;
         case GMLP_VARIANT_SKINNY:
-            rc = run_skinny(dev, L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st);
+            rc = run_skinny(dev, L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st, act);
             break;
         case GMLP_VARIANT_PAIR:
-            rc = launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st);
+            rc = launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act);
             if (rc == GMLP_OK) {
                 prof_mark("gate_up", st);
                 rc = launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st);
@@ -708,8 +727,8 @@ int forward_impl(const gmlp_args* a) {
             }
             break;
         case GMLP_VARIANT_TENSOR:
-            rc = gate_up_uses_pair(a->M) ? launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st)
-                                         : launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st);
+            rc = gate_up_uses_pair(a->M) ? launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act)
+                                         : launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act);
             if (rc == GMLP_OK) {
                 prof_mark("gate_up", st);
                 rc = down_uses_pair(a->M) ? launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st)
@@ -718,7 +737,7 @@ int forward_impl(const gmlp_args* a) {
             }
             break;
         default:
-            rc = launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st);
+            rc = launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act);
             if (rc == GMLP_OK) {
                 prof_mark("gate_up", st);
                 rc = launch_umma<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st);
@@ -804,6 +823,8 @@ int gate_up_impl(const gmlp_args* a) {
     if (a == nullptr) return GMLP_ERR_NULL;
     if (a->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
     if (a->flags & ~kKnownFlags) return GMLP_ERR_FLAGS;
+    gmlp::GateAct act;
+    if (a->reserved != 0 || !gate_act_from(a->flags, a->act_beta, &act)) return GMLP_ERR_FLAGS;
     if (a->variant < GMLP_VARIANT_AUTO || a->variant > GMLP_VARIANT_TENSOR) return GMLP_ERR_FLAGS;
     int rc = check_shape(a->M, a->d_model, a->d_ff);
     if (rc != GMLP_OK) return rc;
@@ -857,11 +878,11 @@ int gate_up_impl(const gmlp_args* a) {
         float* scratch = reinterpret_cast<float*>(ws + L.partial_off);
         unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
         rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
-        if (rc == GMLP_OK) rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, Hout, a->M, a->d_model, a->d_ff, st);
+        if (rc == GMLP_OK) rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, Hout, a->M, a->d_model, a->d_ff, st, act);
     } else if (variant == GMLP_VARIANT_PAIR || (variant == GMLP_VARIANT_TENSOR && gate_up_uses_pair(a->M))) {
-        rc = launch_umma_pair<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st);
+        rc = launch_umma_pair<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st, act);
     } else {
-        rc = launch_umma<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st);
+        rc = launch_umma<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st, act);
     }
     if (rc != GMLP_OK) {
         forget_counters(dev);
@@ -951,8 +972,8 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         const float* rc_ptr = r;
         cudaError_t err = pair
-            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr)
-            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128);
+            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu)
+            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("matmul_rowscale", st);
@@ -1016,6 +1037,7 @@ int gmlp_forward(const void* X, const void* Wg, const void* Wu, const void* Wd, 
     a.stream = t_stream;
     a.workspace = nullptr;
     a.workspace_bytes = 0;
+    a.act_beta = 1.0f;
     return gmlp_forward_ex(&a);
 }
 

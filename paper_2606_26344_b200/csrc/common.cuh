@@ -21,6 +21,19 @@ __device__ __forceinline__ float silu_f32(float g) {
     return __fdividef(g, 1.0f + __expf(-g));
 }
 
+// Gate activation of the gated unit, h = act(g) * u (Section 6.1 lists SiLU-, SwiGLU- and GLU-gated forms):
+//   SiLU      act(g) = g * sigmoid(g)            beta = 1, glu = 0
+//   Swish     act(g) = g * sigmoid(beta * g)     beta free, glu = 0
+//   GLU       act(g) = sigmoid(g)                beta = 1, glu = 1
+// one expression, numerator g or 1 over 1 + e^(-beta g); with beta = 1, glu = 0 it is silu_f32 bit for bit.
+struct GateAct {
+    float beta;
+    int glu;
+};
+__device__ __forceinline__ float gate_act_f32(float g, const GateAct a) {
+    return __fdividef(a.glu ? 1.0f : g, 1.0f + __expf(-(a.beta * g)));
+}
+
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 

@@ -15,7 +15,7 @@ constexpr int kSimtBK = 16;
 template <bool GATEUP>
 __global__ void __launch_bounds__(256)
 simt_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ B0, const bf16* __restrict__ B1,
-                 bf16* __restrict__ C, int64_t M, int K, int N)
+                 bf16* __restrict__ C, int64_t M, int K, int N, GateAct act)
 {
     __shared__ float As[kSimtBK][kSimtTile + 4];
     __shared__ float Bs0[kSimtBK][kSimtTile];
@@ -83,7 +83,7 @@ simt_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ B0, const 
         if (m >= M) continue;
         float o[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) o[j] = GATEUP ? silu_f32(acc0[i][j]) * acc1[i][j] : acc0[i][j];
+        for (int j = 0; j < 4; ++j) o[j] = GATEUP ? gate_act_f32(acc0[i][j], act) * acc1[i][j] : acc0[i][j];
         *reinterpret_cast<uint2*>(C + m * N + n) = make_uint2(pack_bf16x2(o[0], o[1]), pack_bf16x2(o[2], o[3]));
     }
 }

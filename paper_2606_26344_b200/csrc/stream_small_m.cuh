@@ -26,7 +26,7 @@ template <int MT, bool GATEUP>
 __global__ void __launch_bounds__(kStreamThreads, 4)
 stream_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W0, const bf16* __restrict__ W1,
                    float* __restrict__ partial, unsigned int* __restrict__ counters, bf16* __restrict__ out,
-                   int M, int K, int N, int kchunk, int KS)
+                   int M, int K, int N, int kchunk, int KS, GateAct act)
 {
     constexpr int NMAT = GATEUP ? 2 : 1;
     __shared__ __align__(16) float xs[kStreamMaxChunk][MT];
@@ -133,8 +133,8 @@ stream_gemm_kernel(const bf16* __restrict__ A, const bf16* __restrict__ W0, cons
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
             if (m < rows) {
-                const float o0 = GATEUP ? silu_f32(g[m].x) * u[m].x : g[m].x;
-                const float o1 = GATEUP ? silu_f32(g[m].y) * u[m].y : g[m].y;
+                const float o0 = GATEUP ? gate_act_f32(g[m].x, act) * u[m].x : g[m].x;
+                const float o1 = GATEUP ? gate_act_f32(g[m].y, act) * u[m].y : g[m].y;
                 *reinterpret_cast<uint32_t*>(out + (size_t)(m0 + m) * N + nc) = pack_bf16x2(o0, o1);
             }
         }

@@ -88,7 +88,7 @@ template <bool GATEUP, bool ROWSCALE = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                       const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
-                      int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale)
+                      int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, GateAct act)
 {
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
     constexpr int KERNEL_ID = GATEUP ? 6 : 7;
@@ -225,8 +225,8 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     ptx::tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const float h0 = silu_f32(__uint_as_float(g[2 * j])) * __uint_as_float(u[2 * j]);
-                        const float h1 = silu_f32(__uint_as_float(g[2 * j + 1])) * __uint_as_float(u[2 * j + 1]);
+                        const float h0 = gate_act_f32(__uint_as_float(g[2 * j]), act) * __uint_as_float(u[2 * j]);
+                        const float h1 = gate_act_f32(__uint_as_float(g[2 * j + 1]), act) * __uint_as_float(u[2 * j + 1]);
                         packed[j] = pack_bf16x2(h0, h1);
                     }
                 } else {

@@ -69,7 +69,8 @@ template <bool GATEUP, int NH>
 __device__ __forceinline__ bool skinny_epilogue_segment(
     uint32_t acc0, uint32_t tempty_bar, int tile, bool first_segment_of_cta, int cta, long long total, long long parts,
     int KB, int M, int Mpad, int N, float* __restrict__ scratch, unsigned int* __restrict__ counters,
-    bf16* __restrict__ out, unsigned long long* slot_off, volatile int* last_flag, int et, int nl, int lane)
+    bf16* __restrict__ out, unsigned long long* slot_off, volatile int* last_flag, int et, int nl, int lane,
+    const GateAct act)
 {
     constexpr int NMAT = GATEUP ? 2 : 1;
     constexpr int TILE_N = 128 * NH;
@@ -94,7 +95,7 @@ __device__ __forceinline__ bool skinny_epilogue_segment(
                     for (int i = 0; i < 16; ++i) {
                         const int m = c0 + i;
                         if (m < M) {
-                            const float v = GATEUP ? silu_f32(__uint_as_float(g[i])) * __uint_as_float(uu[i])
+                            const float v = GATEUP ? gate_act_f32(__uint_as_float(g[i]), act) * __uint_as_float(uu[i])
                                                    : __uint_as_float(g[i]);
                             out[(size_t)m * N + n] = __float2bfloat16_rn(v);
                         }
@@ -191,8 +192,8 @@ __device__ __forceinline__ bool skinny_epilogue_segment(
             auto finish = [&](const float4& g, const float4& uu, int mm) {
                 float v[4] = {g.x, g.y, g.z, g.w};
                 if (GATEUP) {
-                    v[0] = silu_f32(g.x) * uu.x; v[1] = silu_f32(g.y) * uu.y;
-                    v[2] = silu_f32(g.z) * uu.z; v[3] = silu_f32(g.w) * uu.w;
+                    v[0] = gate_act_f32(g.x, act) * uu.x; v[1] = gate_act_f32(g.y, act) * uu.y;
+                    v[2] = gate_act_f32(g.z, act) * uu.z; v[3] = gate_act_f32(g.w, act) * uu.w;
                 }
                 // N is a multiple of 8 and n of 4: the four columns are all inside or all outside
                 *reinterpret_cast<uint2*>(out + (size_t)mm * N + n) =
@@ -211,7 +212,8 @@ __global__ void __launch_bounds__(kSkinnyThreads, 1)
 skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW0,
                    const __grid_constant__ CUtensorMap tmW1, float* __restrict__ scratch,
                    unsigned int* __restrict__ counters, bf16* __restrict__ out,
-                   int M, int Mpad, int N, int num_tiles, int KB, int stages, uint32_t tmem_cols, int evict_first)
+                   int M, int Mpad, int N, int num_tiles, int KB, int stages, uint32_t tmem_cols, int evict_first,
+                   GateAct act)
 {
     constexpr int KERNEL_ID = GATEUP ? 3 : 4;
     constexpr int NMAT = GATEUP ? 2 : 1;
@@ -370,7 +372,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             if (!ok) break;
             skinny_epilogue_segment<GATEUP, NH>(tmem_base + lane_base + acc_col(buf, 0, 0), tempty0 + 8 * buf, tile,
                                                 tile == (int)(u_begin / KB), blockIdx.x, total, parts, KB, M, Mpad, N,
-                                                scratch, counters, out, slot_off, last_flag, et, nl, lane);
+                                                scratch, counters, out, slot_off, last_flag, et, nl, lane, act);
             u = seg_end;
         }
     }

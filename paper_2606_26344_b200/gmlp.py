@@ -20,6 +20,9 @@ STATIC_MAX_M = 16
 STATIC_SCRATCH_BYTES = 12 << 20
 FLAG_RMSNORM = 1 << 0
 FLAG_CHECKED = 1 << 2
+FLAG_ACT_SWISH = 1 << 5
+FLAG_ACT_GLU = 1 << 6
+ACT_FLAGS = {"silu": 0, "swish": FLAG_ACT_SWISH, "glu": FLAG_ACT_GLU}
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA, VARIANT_SKINNY, VARIANT_PAIR, VARIANT_TENSOR = 0, 1, 2, 3, 4, 5, 6
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgmlp.so")
@@ -34,6 +37,7 @@ class GmlpArgs(ctypes.Structure):
         ("M", ctypes.c_int64), ("d_model", ctypes.c_int64), ("d_ff", ctypes.c_int64),
         ("rms_gain", ctypes.c_void_p), ("rms_eps", ctypes.c_float), ("variant", ctypes.c_int32),
         ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_uint64),
+        ("act_beta", ctypes.c_float), ("reserved", ctypes.c_uint32),
     ]
 
 
@@ -160,14 +164,14 @@ def _check_bf16_cuda(t: torch.Tensor, name: str) -> None:
 
 def make_args(X, Wg, Wu, Wd, Y, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, variant: int = VARIANT_AUTO,
               workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
-              checked: bool = False) -> GmlpArgs:
+              checked: bool = False, act: str = "silu", beta: float = 1.0) -> GmlpArgs:
     for t, n in ((X, "X"), (Wg, "Wg"), (Wu, "Wu"), (Wd, "Wd"), (Y, "Y")):
         _check_bf16_cuda(t, n)
     M, d_model = X.shape
     d_ff = Wg.shape[1]
     if Wg.shape != (d_model, d_ff) or Wu.shape != (d_model, d_ff) or Wd.shape != (d_ff, d_model) or Y.shape != X.shape:
         raise ValueError("shape mismatch")
-    flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0)
+    flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0) | ACT_FLAGS[act]
     if gamma is not None:
         _check_bf16_cuda(gamma, "gamma")
     st = stream if stream is not None else torch.cuda.current_stream(X.device)
@@ -182,6 +186,8 @@ def make_args(X, Wg, Wu, Wd, Y, gamma=None, eps: float = 1e-5, rmsnorm: bool = F
     a.stream = st.cuda_stream
     a.workspace = workspace.data_ptr() if workspace is not None else None
     a.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    a.act_beta = beta
+    a.reserved = 0
     return a
 
 
@@ -198,12 +204,15 @@ def forward_ex(args: GmlpArgs) -> None:
 
 
 def forward(X, Wg, Wu, Wd, Y=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False,
-            variant: int = VARIANT_AUTO, workspace=None, stream=None, checked: bool = False) -> torch.Tensor:
-    """Y = (silu(Xn Wg) * (Xn Wu)) Wd on the GPU; asynchronous on ``stream`` (default: torch's current stream)."""
+            variant: int = VARIANT_AUTO, workspace=None, stream=None, checked: bool = False,
+            act: str = "silu", beta: float = 1.0) -> torch.Tensor:
+    """Y = (act(Xn Wg) * (Xn Wu)) Wd on the GPU; asynchronous on ``stream`` (default: torch's current stream).
+
+    ``act``: "silu" (the paper's operator), "swish" (g * sigmoid(beta * g)) or "glu" (sigmoid(g))."""
     if Y is None:
         Y = torch.empty_like(X)
     with torch.cuda.device(X.device):
-        forward_ex(make_args(X, Wg, Wu, Wd, Y, gamma, eps, rmsnorm, variant, workspace, stream, checked))
+        forward_ex(make_args(X, Wg, Wu, Wd, Y, gamma, eps, rmsnorm, variant, workspace, stream, checked, act, beta))
     return Y
 
 
@@ -242,8 +251,8 @@ def forward_static(X, Wg, Wu, Wd, Y, stream=None) -> None:
 
 
 def gate_up(X, Wg, Wu, H=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, variant: int = VARIANT_AUTO,
-            workspace=None, stream=None, checked: bool = False) -> torch.Tensor:
-    """gmlp_gate_up: H = bf16(silu(Xn Wg) * (Xn Wu)), the gate/up half alone; H is [M, d_ff]."""
+            workspace=None, stream=None, checked: bool = False, act: str = "silu", beta: float = 1.0) -> torch.Tensor:
+    """gmlp_gate_up: H = bf16(act(Xn Wg) * (Xn Wu)), the gate/up half alone; H is [M, d_ff]."""
     for t, n in ((X, "X"), (Wg, "Wg"), (Wu, "Wu")):
         _check_bf16_cuda(t, n)
     M, d_model = X.shape
@@ -258,7 +267,8 @@ def gate_up(X, Wg, Wu, H=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = Fa
     st = stream if stream is not None else torch.cuda.current_stream(X.device)
     a = GmlpArgs()
     a.struct_bytes = ctypes.sizeof(GmlpArgs)
-    a.flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0)
+    a.flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0) | ACT_FLAGS[act]
+    a.act_beta = beta
     a.X, a.Wg, a.Wu, a.Wd, a.Y = X.data_ptr(), Wg.data_ptr(), Wu.data_ptr(), None, H.data_ptr()
     a.M, a.d_model, a.d_ff = M, d_model, d_ff
     a.rms_gain = gamma.data_ptr() if gamma is not None else None

@@ -35,8 +35,8 @@ def test_header_symbols_are_exported(lib):
 
 
 def test_struct_layout_matches_header(lib):
-    # 2 x u32, 5 pointers, 3 x i64, pointer, float, i32, 2 pointers, u64 on LP64
-    assert ctypes.sizeof(gmlp.GmlpArgs) == 8 + 5 * 8 + 3 * 8 + 8 + 4 + 4 + 8 + 8 + 8
+    # 2 x u32, 5 pointers, 3 x i64, pointer, float, i32, 2 pointers, u64, float, u32 on LP64
+    assert ctypes.sizeof(gmlp.GmlpArgs) == 8 + 5 * 8 + 3 * 8 + 8 + 4 + 4 + 8 + 8 + 8 + 4 + 4
 
 
 def test_version_and_status_strings(lib):
@@ -62,6 +62,10 @@ def test_argument_validation_happens_before_device_work(lib):
     assert f(_args(struct_bytes=8)) == gmlp.ERR_FLAGS
     assert f(_args(flags=1 << 7)) == gmlp.ERR_FLAGS
     assert f(_args(variant=17)) == gmlp.ERR_FLAGS
+    assert f(_args(flags=gmlp.FLAG_ACT_SWISH | gmlp.FLAG_ACT_GLU, act_beta=1.0)) == gmlp.ERR_FLAGS
+    assert f(_args(flags=gmlp.FLAG_ACT_SWISH, act_beta=float("nan"))) == gmlp.ERR_FLAGS
+    assert f(_args(flags=gmlp.FLAG_ACT_SWISH, act_beta=float("inf"))) == gmlp.ERR_FLAGS
+    assert f(_args(reserved=1)) == gmlp.ERR_FLAGS
     assert f(_args(variant=-1)) == gmlp.ERR_FLAGS
     assert f(_args(M=-1)) == gmlp.ERR_SHAPE
     assert f(_args(d_model=60)) == gmlp.ERR_SHAPE

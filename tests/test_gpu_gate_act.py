@@ -1,0 +1,89 @@
+"""GPU parity of the gate-activation variants (Swish-beta, GLU) against the CPU oracle, every
+schedule, whole operator and gate/up half; and that beta = 1 reproduces the SiLU path bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2606_26344_b200 import gmlp, inputs as I
+
+from _parity import to_device
+
+pytestmark = pytest.mark.gpu
+
+V = gmlp
+CASES = [(V.VARIANT_SIMT, 70, 200, 328), (V.VARIANT_STREAM, 5, 264, 520), (V.VARIANT_SKINNY, 8, 1024, 2056),
+         (V.VARIANT_UMMA, 129, 320, 392), (V.VARIANT_PAIR, 300, 512, 1024), (V.VARIANT_TENSOR, 9, 1024, 2048),
+         (V.VARIANT_TENSOR, 520, 512, 1088), (V.VARIANT_AUTO, 16, 256, 512)]
+
+
+def _run(inp, variant, act, beta, rmsnorm):
+    w = inp.workload
+    t = to_device(inp)
+    ws = gmlp.alloc_workspace(w.M, w.d_model, w.d_ff, rmsnorm, variant)
+    Y = torch.full_like(t["X"], float("nan"))
+    gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], Y, gamma=t["gamma"] if rmsnorm else None, eps=w.eps,
+                 rmsnorm=rmsnorm, variant=variant, workspace=ws, checked=True, act=act, beta=beta)
+    torch.cuda.synchronize()
+    return Y
+
+
+@pytest.mark.parametrize("act,beta", [("swish", 1.702), ("swish", 0.5), ("swish", -1.0), ("glu", 1.0)])
+@pytest.mark.parametrize("case", CASES)
+def test_whole_operator(case, act, beta):
+    variant, M, dm, dff = case
+    rmsnorm = (M % 2 == 1)
+    inp = I.custom_inputs(M, dm, dff, 900 + M, rmsnorm=rmsnorm, eps=1e-5)
+    Y = _run(inp, variant, act, beta, rmsnorm)
+    rows = I.sample_rows(inp.workload, inp.outlier_rows)
+    y_ref = oracle.gmlp_rows(inp.bits("X"), inp.bits("Wg"), inp.bits("Wu"), inp.bits("Wd"), rows=rows,
+                             gamma=inp.bits("gamma") if rmsnorm else None, eps=inp.workload.eps, rmsnorm=rmsnorm,
+                             act=act, beta=beta)
+    y = Y[torch.as_tensor(rows, device=Y.device)].float().cpu().numpy().astype(np.float64)
+    e = np.abs(y - y_ref) / oracle.tolerance(y_ref)
+    assert np.isfinite(y).all() and float(e.max()) <= 1.0, f"{case} {act} {beta}: max err/tol {float(e.max()):.3f}"
+
+
+@pytest.mark.parametrize("case", CASES)
+def test_swish_with_beta_one_is_the_silu_path_bit_for_bit(case):
+    variant, M, dm, dff = case
+    inp = I.custom_inputs(M, dm, dff, 950 + M)
+    a = _run(inp, variant, "silu", 1.0, False)
+    b = _run(inp, variant, "swish", 1.0, False)
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+@pytest.mark.parametrize("act,beta", [("swish", 1.702), ("glu", 1.0)])
+@pytest.mark.parametrize("variant,M", [(V.VARIANT_SKINNY, 8), (V.VARIANT_UMMA, 100), (V.VARIANT_PAIR, 260),
+                                       (V.VARIANT_TENSOR, 300)])
+def test_gate_up_half_alone(variant, M, act, beta):
+    dm, dff = 512, 1096
+    inp = I.custom_inputs(M, dm, dff, 970 + M)
+    t = to_device(inp)
+    H = gmlp.gate_up(t["X"], t["Wg"], t["Wu"], variant=variant, checked=True, act=act, beta=beta)
+    torch.cuda.synchronize()
+    rows = I.sample_rows(inp.workload, inp.outlier_rows)
+    p_ref = oracle.gate_up_rows(inp.bits("X"), inp.bits("Wg"), inp.bits("Wu"), rows=rows, act=act, beta=beta)
+    h = H[torch.as_tensor(rows, device=H.device)].float().cpu().numpy().astype(np.float64)
+    e = np.abs(h - p_ref) / oracle.tolerance(p_ref)
+    assert float(e.max()) <= 1.0, f"max err/tol {float(e.max()):.3f}"
+
+
+def test_gate_values_on_device_over_a_dense_sweep():
+    """One-hot weights make G[m, n] = X[m, n] and U = 1, Wd = identity, so Y[m, n] = bf16(bf16(act(x)))."""
+    M, d = 64, 256
+    xs = torch.linspace(-30, 30, M * d).reshape(M, d).to(torch.bfloat16)
+    eye = torch.eye(d, dtype=torch.bfloat16)
+    ones_row = torch.zeros(d, d, dtype=torch.bfloat16)
+    ones_row[0, :] = 1                                   # U[m, n] = X[m, 0]
+    X = xs.clone()
+    X[:, 0] = 1                                          # so U = 1 everywhere
+    dev = "cuda"
+    xd = X.double().numpy()
+    for act, beta in (("swish", 1.702), ("swish", 0.25), ("glu", 1.0)):
+        Y = gmlp.forward(X.to(dev), eye.to(dev), ones_row.to(dev), eye.to(dev), variant=V.VARIANT_UMMA, checked=True,
+                         act=act, beta=beta)
+        want = oracle.bf16_to_double(oracle.bf16_rn(oracle.gate_act(xd, act, beta)))
+        got = Y.float().cpu().numpy().astype(np.float64)
+        # one bf16 ulp: the device evaluates exp and the division with fast fp32 approximations
+        assert np.all(np.abs(got - want) <= np.maximum(np.abs(want), 2.0 ** -120) * 2.0 ** -7), (act, beta)
