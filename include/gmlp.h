@@ -154,6 +154,38 @@ typedef struct gmlp_rmsmm_args {
 int gmlp_rmsnorm_matmul(const gmlp_rmsmm_args* args);
 
 /*
+ * A matrix multiplication, a residual addition and RMSNorm, "Matmul+Add+RMSNorm" of the paper's benchmark
+ * list (Section 6.1; the paper names the chain, the graph below is the reading taken):
+ *     S = bf16( X * W + R ),     Z = bf16( RMSNorm(S) ) = bf16( S * rsqrt(mean_n S^2 + eps) * gain ),
+ * X [M, K], W [K, N], R, S, Z [M, N] row-major bf16, gain [N] bf16 or NULL; K and N multiples of 8.  S (the
+ * updated residual stream) is an output too and is rounded once from the fp32 sum; the statistic of Eq. (1)
+ * is taken over the stored S.  R and S may be the same buffer (in-place residual update); Z must not alias.
+ * Default schedule: the GEMM's epilogue adds R, stores S and leaves one sum of squares per row and column
+ * tile; a light second kernel (chained by programmatic dependent launch) adds those in fixed order and
+ * writes Z with one read of S.  GMLP_MMADDNORM_UNFUSED runs the three operators one after the other
+ * (GEMM -> T, T + R -> S, RMSNorm(S) -> Z; T is rounded to bf16 on the way, so S may differ by an ulp).
+ * workspace (256-byte aligned, required): ceil(N/256)*M*4 bytes fused, M*N*2 bytes unfused.
+ */
+enum { GMLP_MMADDNORM_UNFUSED = 1u << 4 };
+typedef struct gmlp_mmaddnorm_args {
+    uint32_t struct_bytes;    /* sizeof(gmlp_mmaddnorm_args) */
+    uint32_t flags;           /* GMLP_FLAG_CHECKED | GMLP_MMADDNORM_UNFUSED */
+    const void* X;            /* device, [M, K] bf16 */
+    const void* W;            /* device, [K, N] bf16 */
+    const void* R;            /* device, [M, N] bf16 residual */
+    void* S;                  /* device, [M, N] bf16, written */
+    void* Z;                  /* device, [M, N] bf16, written */
+    int64_t M, K, N;
+    const void* rms_gain;     /* device, [N] bf16, or NULL */
+    float rms_eps;
+    int32_t reserved;         /* must be 0 */
+    void* stream;             /* cudaStream_t */
+    void* workspace;
+    uint64_t workspace_bytes;
+} gmlp_mmaddnorm_args;
+int gmlp_matmul_add_rmsnorm(const gmlp_mmaddnorm_args* args);
+
+/*
  * The same call for a caller whose activations live in HOST memory: copies X_host
  * (M*d_model bf16, ideally pinned) to args->X, runs gmlp_forward_ex, and copies args->Y
  * to Y_host, all asynchronously on args->stream.  args->X and args->Y are device staging

@@ -90,6 +90,7 @@ struct DeviceState {
     void* workspace = nullptr;
     uint64_t workspace_bytes = 0;
     bool splitk_attr_set = false;
+    bool addss_attr_set = false;
     bool umma_attr_set = false;
     bool pair_attr_set = false;
     bool rowscale_attr_set = false;
@@ -441,7 +442,7 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
     if (cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m,
-                           num_tiles, (const float*)nullptr, act) != cudaSuccess)
+                           num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr) != cudaSuccess)
         return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -551,16 +552,16 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     cudaError_t err;
     if (GATEUP && nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr);
     else if (GATEUP)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr);
     else if (nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr);
     else
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -972,8 +973,8 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         const float* rc_ptr = r;
         cudaError_t err = pair
-            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu)
-            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu);
+            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr)
+            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("matmul_rowscale", st);
@@ -987,9 +988,126 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
     return GMLP_OK;
 }
 
+// "Matmul+Add+RMSNorm" (Section 6.1): S = X W + R, Z = RMSNorm(S).
+int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
+    if (a == nullptr) return GMLP_ERR_NULL;
+    if (a->struct_bytes != sizeof(gmlp_mmaddnorm_args)) return GMLP_ERR_FLAGS;
+    if ((a->flags & ~(uint32_t)(GMLP_FLAG_CHECKED | GMLP_MMADDNORM_UNFUSED)) || a->reserved != 0) return GMLP_ERR_FLAGS;
+    int rc = check_shape(a->M, a->K, a->N);
+    if (rc != GMLP_OK) return rc;
+    if (a->M == 0) return GMLP_OK;
+    if (!a->X || !a->W || !a->R || !a->S || !a->Z) return GMLP_ERR_NULL;
+    if (!aligned16(a->X) || !aligned16(a->W) || !aligned16(a->R) || !aligned16(a->S) || !aligned16(a->Z) ||
+        !aligned16(a->rms_gain))
+        return GMLP_ERR_ALIGN;
+    if (a->workspace != nullptr && (reinterpret_cast<uintptr_t>(a->workspace) & 255u)) return GMLP_ERR_ALIGN;
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(a->stream);
+    const bf16* X = static_cast<const bf16*>(a->X);
+    const bf16* W = static_cast<const bf16*>(a->W);
+    const bf16* R = static_cast<const bf16*>(a->R);
+    const bf16* gain = static_cast<const bf16*>(a->rms_gain);
+    bf16* S = static_cast<bf16*>(a->S);
+    bf16* Z = static_cast<bf16*>(a->Z);
+    const bool pair = a->M >= 1024;
+    prof_begin(st);
+    if (a->flags & GMLP_MMADDNORM_UNFUSED) {
+        // three separate operators: T = X W (bf16), S = T + R, Z = RMSNorm(S)
+        const uint64_t need = align256((uint64_t)a->M * a->N * 2);
+        if (a->workspace == nullptr || a->workspace_bytes < need) return GMLP_ERR_WORKSPACE;
+        bf16* T = static_cast<bf16*>(a->workspace);
+        rc = pair ? launch_umma_pair<false>(dev, X, W, nullptr, T, a->M, a->K, a->N, st)
+                  : launch_umma<false>(dev, X, W, nullptr, T, a->M, a->K, a->N, st);
+        if (rc != GMLP_OK) return rc;
+        prof_mark("matmul", st);
+        const size_t nvec = (size_t)a->M * (size_t)a->N / 8;
+        gmlp::add_bf16_kernel<<<(unsigned)((nvec + 255) / 256), 256, 0, st>>>(T, R, S, nvec);
+        GMLP_CHECK_LAUNCH();
+        prof_mark("add", st);
+        rc = launch_rmsnorm(S, gain, Z, a->M, a->N, a->rms_eps, st);
+        if (rc != GMLP_OK) return rc;
+        prof_mark("rmsnorm", st);
+    } else {
+        // fused: the GEMM's epilogue adds R, stores S and leaves per-tile sums of squares; one light pass normalises
+        const int n_tiles = (int)((a->N + 255) / 256);
+        const uint64_t need = align256((uint64_t)n_tiles * a->M * 4);
+        if (a->workspace == nullptr || a->workspace_bytes < need) return GMLP_ERR_WORKSPACE;
+        float* sumsq = static_cast<float*>(a->workspace);
+        CUtensorMap tmA, tmB;
+        if (!encode_2d(&tmA, X, (uint64_t)a->K, (uint64_t)a->M, gmlp::kUmmaBK, 128) ||
+            !encode_2d(&tmB, W, (uint64_t)a->N, (uint64_t)a->K, 64, gmlp::kUmmaBK))
+            return GMLP_ERR_LAUNCH;
+        if (!dev->addss_attr_set) {
+            if (cudaFuncSetAttribute(gmlp::umma_gemm_kernel<false, 4, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)gmlp::kUmmaSmemBytes) != cudaSuccess ||
+                cudaFuncSetAttribute(gmlp::umma_pair_gemm_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)gmlp::kPairSmemBytes) != cudaSuccess)
+                return GMLP_ERR_LAUNCH;
+            dev->addss_attr_set = true;
+        }
+        const int sms = dev->sm_count > 0 ? dev->sm_count : 148;
+        const int num_m = (int)((a->M + (pair ? 255 : 127)) / (pair ? 256 : 128));
+        const int num_tiles = num_m * n_tiles;
+        const int ctas = pair ? 2 * (num_tiles < sms / 2 ? num_tiles : sms / 2) : (num_tiles < sms ? num_tiles : sms);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)ctas);
+        cfg.blockDim = dim3(gmlp::kUmmaThreads);
+        cfg.dynamicSmemBytes = pair ? gmlp::kPairSmemBytes : gmlp::kUmmaSmemBytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = 2;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pair ? 2 : 1;
+        const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
+        cudaError_t err = pair
+            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
+                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq)
+            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
+                                 num_tiles, (const float*)nullptr, 128, kSilu, R, sumsq);
+        if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
+        GMLP_CHECK_LAUNCH();
+        prof_mark("matmul_add", st);
+        cudaLaunchConfig_t c2 = {};
+        c2.gridDim = dim3((unsigned)a->M);
+        c2.blockDim = dim3(gmlp::kRmsThreads);
+        c2.stream = st;
+        c2.attrs = attr;                                   // programmatic stream serialization only
+        c2.numAttrs = 1;
+        const int64_t M64 = a->M;
+        const float eps = a->rms_eps;
+        const bf16* Sc = S;
+        const float* ssc = sumsq;
+        if (cudaLaunchKernelEx(&c2, gmlp::rmsnorm_apply_kernel, Sc, ssc, n_tiles, gain, Z, M64, Ni, eps) != cudaSuccess)
+            return GMLP_ERR_LAUNCH;
+        GMLP_CHECK_LAUNCH();
+        prof_mark("rmsnorm_apply", st);
+    }
+    if (a->flags & GMLP_FLAG_CHECKED) {
+        if (cudaStreamSynchronize(st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+        const int s = read_device_status();
+        if (s < 0) return s;
+        if (s != 0) return GMLP_ERR_TIMEOUT;
+    }
+    return GMLP_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+int gmlp_matmul_add_rmsnorm(const gmlp_mmaddnorm_args* args) {
+    try {
+        return matmul_add_rmsnorm_impl(args);
+    } catch (...) {
+        return GMLP_ERR_LAUNCH;
+    }
+}
 
 int gmlp_rmsnorm_matmul(const gmlp_rmsmm_args* args) {
     try {

@@ -99,4 +99,55 @@ row_rsqrt_kernel(const bf16* __restrict__ X, float* __restrict__ r, int64_t M, i
     }
 }
 
+// Second half of "Matmul+Add+RMSNorm": the GEMM's epilogue has stored S and, per row and column tile, the sum
+// of squares of the stored values (sumsq [n_tiles][M]); this kernel adds a row's partials in tile order
+// (every thread the same order: deterministic), forms r = rsqrt(sum / N + eps) and writes
+// Z[m, n] = bf16_rn(S[m, n] * r * gamma[n]).  One CTA per row, one read of S.
+__global__ void __launch_bounds__(kRmsThreads)
+rmsnorm_apply_kernel(const bf16* __restrict__ S, const float* __restrict__ sumsq, int n_tiles,
+                     const bf16* __restrict__ gamma, bf16* __restrict__ Z, int64_t M, int N, float eps)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");            // S and sumsq come from the previous kernel
+    const int64_t row = blockIdx.x;
+    if (row >= M) return;
+    float t = 0.0f;
+    for (int i = 0; i < n_tiles; ++i) t += __ldcg(sumsq + (size_t)i * M + row);
+    const float r = rsqrtf(t / (float)N + eps);
+    const uint4* x = reinterpret_cast<const uint4*>(S + row * N);
+    const uint4* g = reinterpret_cast<const uint4*>(gamma);
+    uint4* out = reinterpret_cast<uint4*>(Z + row * N);
+    const int nvec = N >> 3;
+    for (int i = threadIdx.x; i < nvec; i += kRmsThreads) {
+        const uint4 v = __ldcg(x + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t gw[4] = {0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u};   // bf16 ones
+        if (gamma != nullptr) {
+            const uint4 gv = g[i];
+            gw[0] = gv.x; gw[1] = gv.y; gw[2] = gv.z; gw[3] = gv.w;
+        }
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float a = bf16_lo(w[j]) * r * bf16_lo(gw[j]);
+            const float b = bf16_hi(w[j]) * r * bf16_hi(gw[j]);
+            o[j] = pack_bf16x2(a, b);
+        }
+        out[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// Unfused schedule of the same chain: S = bf16_rn(T + R) elementwise, T the bf16 product of a plain GEMM.
+__global__ void __launch_bounds__(256)
+add_bf16_kernel(const bf16* __restrict__ T, const bf16* __restrict__ R, bf16* __restrict__ S, size_t nvec)
+{
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= nvec) return;
+    const uint4 a = reinterpret_cast<const uint4*>(T)[i], b = reinterpret_cast<const uint4*>(R)[i];
+    const uint32_t x[4] = {a.x, a.y, a.z, a.w}, y[4] = {b.x, b.y, b.z, b.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) o[j] = pack_bf16x2(bf16_lo(x[j]) + bf16_lo(y[j]), bf16_hi(x[j]) + bf16_hi(y[j]));
+    reinterpret_cast<uint4*>(S)[i] = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 }  // namespace gmlp

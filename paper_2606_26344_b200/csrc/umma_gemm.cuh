@@ -77,6 +77,29 @@ __global__ void wait_timeout_probe_kernel(long long limit_cycles)
     __syncthreads();
 }
 
+// Residual epilogue of "Matmul+Add+RMSNorm" (Section 6.1) for 32 accumulator columns of one row:
+// s = acc + R, stored value = bf16_rn(s), and ss += (stored value)^2 - the statistic of Eq. (1) is taken over
+// what is stored.  rrow points at the row's residual for the chunk's first column; columns at or beyond
+// cols_left do not exist (their accumulators are zero and they add nothing).
+__device__ __forceinline__ void add_residual_chunk(const uint32_t (&acc)[32], uint32_t (&packed)[16],
+                                                   const bf16* rrow, int cols_left, bool row_ok, float& ss) {
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+        uint4 rr = make_uint4(0u, 0u, 0u, 0u);
+        if (row_ok && v * 8 < cols_left) rr = __ldcg(reinterpret_cast<const uint4*>(rrow + v * 8));   // R may be the buffer S is written to
+        const uint32_t w[4] = {rr.x, rr.y, rr.z, rr.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t p = pack_bf16x2(__uint_as_float(acc[v * 8 + 2 * j]) + bf16_lo(w[j]),
+                                           __uint_as_float(acc[v * 8 + 2 * j + 1]) + bf16_hi(w[j]));
+            packed[4 * v + j] = p;
+            const float a = bf16_lo(p), b = bf16_hi(p);
+            ss = fmaf(a, a, ss);
+            ss = fmaf(b, b, ss);
+        }
+    }
+}
+
 // NB = 64-column weight boxes per stage: 4 -> MMA N = 256 (the default), 2 -> MMA N = 128 (smaller tiles for
 // shapes that would otherwise leave most SMs without a tile; more stages, lower arithmetic intensity).
 //
@@ -85,13 +108,15 @@ __global__ void wait_timeout_probe_kernel(long long limit_cycles)
 // not depend on k).  r comes from row_rsqrt_kernel, the kernel launched just before this one: the two
 // are chained by programmatic dependent launch and ONLY the epilogue warps wait for it, so the main loop
 // (which reads the raw X) runs in parallel with the RMS branch.
-template <bool GATEUP, int NB, bool ROWSCALE = false>
+template <bool GATEUP, int NB, bool ROWSCALE = false, bool ADDSS = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
-                 int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, int a_box_rows, GateAct act)
+                 int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, int a_box_rows, GateAct act,
+                 const bf16* residual, float* __restrict__ sumsq)
 {
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
+    static_assert(!(ADDSS && (GATEUP || ROWSCALE)), "the residual epilogue is for the plain GEMM");
     constexpr int KERNEL_ID = GATEUP ? 1 : 2;
     constexpr int N_MMA = 64 * NB;
     constexpr int BN_OUT = GATEUP ? N_MMA / 2 : N_MMA;
@@ -224,6 +249,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * kUmmaN);
             bf16* crow = C + (size_t)row * N + n0;
             const float rscale = (ROWSCALE && row < M) ? __ldcg(row_scale + row) : 1.0f;
+            float ss = 0.0f;                                       // ADDSS: sum of squares of this row's stored values
 #pragma unroll 1
             for (int c = 0; c < BN_OUT; c += 32) {
                 uint32_t g[32];
@@ -239,6 +265,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         const float h1 = gate_act_f32(__uint_as_float(g[2 * j + 1]), act) * __uint_as_float(u[2 * j + 1]);
                         packed[j] = pack_bf16x2(h0, h1);
                     }
+                } else if (ADDSS) {
+                    ptx::tmem_ld_32x32(taddr + c, g);
+                    ptx::tmem_ld_wait();
+                    add_residual_chunk(g, packed, residual + (size_t)row * N + n0 + c, N - (n0 + c), row < M, ss);
                 } else {
                     ptx::tmem_ld_32x32(taddr + c, g);
                     ptx::tmem_ld_wait();
@@ -255,6 +285,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                 }
             }
+            if (ADDSS && row < M) sumsq[(size_t)(tile / num_m_tiles) * M + row] = ss;
             // all of this warp's TMEM reads of the buffer are done: hand it back to the MMA issuer
             ptx::tc_fence_before_sync();
             __syncwarp();

@@ -84,13 +84,15 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 }  // namespace ptx
 
 // ROWSCALE: see umma_gemm.cuh (epilogue row scale from row_rsqrt_kernel; only the epilogue waits for it).
-template <bool GATEUP, bool ROWSCALE = false>
+template <bool GATEUP, bool ROWSCALE = false, bool ADDSS = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                       const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
-                      int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, GateAct act)
+                      int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, GateAct act,
+                      const bf16* residual, float* __restrict__ sumsq)
 {
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
+    static_assert(!(ADDSS && (GATEUP || ROWSCALE)), "the residual epilogue is for the plain GEMM");
     constexpr int KERNEL_ID = GATEUP ? 6 : 7;
     constexpr int BN_OUT = GATEUP ? 128 : 256;
     // D = fp32, A = B = bf16, A K-major, B MN-major, M = 256 (128 per CTA), N = 256
@@ -214,6 +216,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256);
             bf16* crow = C + (size_t)row * N + n0;
             const float rscale = (ROWSCALE && row < M) ? __ldcg(row_scale + row) : 1.0f;
+            float ss = 0.0f;                                       // ADDSS: sum of squares of this row's stored values
 #pragma unroll 1
             for (int c = 0; c < BN_OUT; c += 32) {
                 uint32_t g[32];
@@ -229,6 +232,10 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                         const float h1 = gate_act_f32(__uint_as_float(g[2 * j + 1]), act) * __uint_as_float(u[2 * j + 1]);
                         packed[j] = pack_bf16x2(h0, h1);
                     }
+                } else if (ADDSS) {
+                    ptx::tmem_ld_32x32(taddr + c, g);
+                    ptx::tmem_ld_wait();
+                    add_residual_chunk(g, packed, residual + (size_t)row * N + n0 + c, N - (n0 + c), row < M, ss);
                 } else {
                     ptx::tmem_ld_32x32(taddr + c, g);
                     ptx::tmem_ld_wait();
@@ -245,6 +252,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     }
                 }
             }
+            if (ADDSS && row < M) sumsq[(size_t)(tile / num_m_tiles) * M + row] = ss;
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty0 + 8 * buf);

@@ -52,6 +52,18 @@ class GmlpRmsmmArgs(ctypes.Structure):
 
 
 RMSMM_UNFUSED = 1 << 4
+MMADDNORM_UNFUSED = 1 << 4
+
+
+class GmlpMmAddNormArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_bytes", ctypes.c_uint32), ("flags", ctypes.c_uint32),
+        ("X", ctypes.c_void_p), ("W", ctypes.c_void_p), ("R", ctypes.c_void_p), ("S", ctypes.c_void_p),
+        ("Z", ctypes.c_void_p),
+        ("M", ctypes.c_int64), ("K", ctypes.c_int64), ("N", ctypes.c_int64),
+        ("rms_gain", ctypes.c_void_p), ("rms_eps", ctypes.c_float), ("reserved", ctypes.c_int32),
+        ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_uint64),
+    ]
 
 
 class GmlpError(RuntimeError):
@@ -83,6 +95,8 @@ def lib() -> ctypes.CDLL:
         L.gmlp_forward_static.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.gmlp_workspace_bytes.restype = u64
         L.gmlp_workspace_bytes.argtypes = [i64, i64, i64, u32, i32]
+        L.gmlp_matmul_add_rmsnorm.restype = ctypes.c_int
+        L.gmlp_matmul_add_rmsnorm.argtypes = [ctypes.POINTER(GmlpMmAddNormArgs)]
         L.gmlp_pick_variant.restype = ctypes.c_int
         L.gmlp_pick_variant.argtypes = [i64, i64, i64, u32]
         L.gmlp_device_status.restype = ctypes.c_int
@@ -315,3 +329,51 @@ def rmsnorm_matmul(X, W, Z=None, gamma=None, eps: float = 1e-5, unfused: bool = 
     if rc != OK:
         raise GmlpError(rc)
     return Z
+
+
+def make_mmaddnorm_args(X, W, R, S, Z, gamma=None, eps: float = 1e-5, unfused: bool = False, workspace=None,
+                        stream=None, checked: bool = False) -> GmlpMmAddNormArgs:
+    for t, n in ((X, "X"), (W, "W"), (R, "R"), (S, "S"), (Z, "Z")):
+        _check_bf16_cuda(t, n)
+    M, K = X.shape
+    N = W.shape[1]
+    if W.shape[0] != K or R.shape != (M, N) or S.shape != (M, N) or Z.shape != (M, N):
+        raise ValueError("shape mismatch")
+    st = stream if stream is not None else torch.cuda.current_stream(X.device)
+    a = GmlpMmAddNormArgs()
+    a.struct_bytes = ctypes.sizeof(GmlpMmAddNormArgs)
+    a.flags = (FLAG_CHECKED if checked else 0) | (MMADDNORM_UNFUSED if unfused else 0)
+    a.X, a.W, a.R, a.S, a.Z = X.data_ptr(), W.data_ptr(), R.data_ptr(), S.data_ptr(), Z.data_ptr()
+    a.M, a.K, a.N = M, K, N
+    a.rms_gain = gamma.data_ptr() if gamma is not None else None
+    a.rms_eps = eps
+    a.reserved = 0
+    a.stream = st.cuda_stream
+    a.workspace = workspace.data_ptr() if workspace is not None else None
+    a.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    return a
+
+
+def mmaddnorm_workspace(M: int, N: int, unfused: bool = False, device="cuda") -> torch.Tensor:
+    nbytes = M * N * 2 if unfused else ((N + 255) // 256) * M * 4
+    return torch.empty(((nbytes + 255) // 256 + 1) * 256, dtype=torch.uint8, device=device)
+
+
+def matmul_add_rmsnorm_ex(args: GmlpMmAddNormArgs) -> None:
+    rc = lib().gmlp_matmul_add_rmsnorm(ctypes.byref(args))
+    if rc != OK:
+        raise GmlpError(rc)
+
+
+def matmul_add_rmsnorm(X, W, R, S=None, Z=None, gamma=None, eps: float = 1e-5, unfused: bool = False, stream=None,
+                       checked: bool = False):
+    """gmlp_matmul_add_rmsnorm: S = X @ W + R, Z = RMSNorm(S) * gamma.  Returns (S, Z); S may be R (in place)."""
+    M, N = X.shape[0], W.shape[1]
+    if S is None:
+        S = torch.empty(M, N, dtype=torch.bfloat16, device=X.device)
+    if Z is None:
+        Z = torch.empty(M, N, dtype=torch.bfloat16, device=X.device)
+    ws = mmaddnorm_workspace(M, N, unfused, X.device)
+    with torch.cuda.device(X.device):
+        matmul_add_rmsnorm_ex(make_mmaddnorm_args(X, W, R, S, Z, gamma, eps, unfused, ws, stream, checked))
+    return S, Z
