@@ -356,6 +356,48 @@ def measure_rmsnorm_matmul(dev, sizes=(2048, 4096, 8192), iters=10):
             "best_rewritten_tflops": max(r["rewritten_tflops"] for r in rows), "table": rows}
 
 
+def measure_matmul_add_rmsnorm(dev, sizes=(2048, 4096, 8192), iters=10):
+    """MatMul+Add+RMSNorm over the paper's {2K,4K,8K}^3 sweep: fused schedule (residual and sum of squares in the
+    GEMM epilogue, light normalise pass) against the three operators run one after the other.  Microseconds."""
+    import math
+    import torch
+    from paper_2606_26344_b200 import gmlp
+    g = torch.Generator(device="cpu").manual_seed(0)
+    rows = []
+    for M in sizes:
+        for K in sizes:
+            X = torch.randn(M, K, generator=g).bfloat16().to(dev)
+            for N in sizes:
+                W = (torch.randn(K, N, generator=g) * K ** -0.5).bfloat16().to(dev)
+                R = torch.randn(M, N, generator=g).bfloat16().to(dev)
+                gam = (0.5 + torch.rand(N, generator=g)).bfloat16().to(dev)
+                S, Z = torch.empty_like(R), torch.empty_like(R)
+                t = {}
+                for name, unf in (("fused", False), ("unfused", True)):
+                    ws = gmlp.mmaddnorm_workspace(M, N, unf, dev)
+                    a = gmlp.make_mmaddnorm_args(X, W, R, S, Z, gam, 1e-5, unf, ws)
+                    for _ in range(3):
+                        gmlp.matmul_add_rmsnorm_ex(a)
+                    torch.cuda.synchronize(dev)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    for _ in range(iters):
+                        gmlp.matmul_add_rmsnorm_ex(a)
+                    e1.record()
+                    torch.cuda.synchronize(dev)
+                    t[name] = e0.elapsed_time(e1) / iters * 1e3
+                    del ws
+                rows.append({"M": M, "K": K, "N": N, "fused_us": t["fused"], "unfused_us": t["unfused"],
+                             "speedup": t["unfused"] / t["fused"], "fused_tflops": 2.0 * M * K * N / t["fused"] / 1e6})
+                del W, R, S, Z
+            del X
+    sp = [r["speedup"] for r in rows]
+    return {"shapes": "{2K,4K,8K}^3 as MxKxN", "timing": "back-to-back calls, operands may stay in L2",
+            "geomean_speedup_fused_over_unfused": math.exp(sum(math.log(v) for v in sp) / len(sp)),
+            "min_speedup": min(sp), "max_speedup": max(sp),
+            "best_fused_tflops": max(r["fused_tflops"] for r in rows), "table": rows}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -364,8 +406,9 @@ def main():
     ap.add_argument("--impl", default="gmlp", choices=["gmlp", "reference"])
     ap.add_argument("--workload", default=PRIMARY)
     ap.add_argument("--no-extra", action="store_true", help="time only the primary workload")
-    ap.add_argument("--op", default="gmlp", choices=["gmlp", "rmsnorm_matmul"],
-                    help="rmsnorm_matmul: print only the RMSNorm+MatMul sweep (one JSON line) and exit")
+    ap.add_argument("--op", default="gmlp", choices=["gmlp", "rmsnorm_matmul", "matmul_add_rmsnorm"],
+                    help="rmsnorm_matmul / matmul_add_rmsnorm: print only that operator's {2K,4K,8K}^3 sweep "
+                         "(one JSON line) and exit")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time spent on the oracle baseline (0 = skip)")
     ap.add_argument("--clock-roll", type=float, default=0.6,
                     help="seconds of untimed identical steps before and after the timed region while clocks are "
@@ -399,9 +442,10 @@ def main():
     peaks = load_peaks()
     warmup = max(args.warmup, 3)
 
-    if args.op == "rmsnorm_matmul":
+    if args.op in ("rmsnorm_matmul", "matmul_add_rmsnorm"):
         if rank == 0:
-            print(json.dumps({"op": "rmsnorm_matmul", **measure_rmsnorm_matmul(dev)}))
+            fn = measure_rmsnorm_matmul if args.op == "rmsnorm_matmul" else measure_matmul_add_rmsnorm
+            print(json.dumps({"op": args.op, **fn(dev)}))
         if dist is not None:
             dist.barrier()
             dist.destroy_process_group()
