@@ -153,7 +153,8 @@ def run_reference(args):
     }))
 
 
-def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sample_clocks=True, clock_roll=0.6):
+def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sample_clocks=True, clock_roll=0.6,
+                     autotune=False):
     """Times one workload on this rank's GPU.  Returns a dict of measurements."""
     import torch
     from paper_2606_26344_b200 import gmlp, inputs as I
@@ -162,9 +163,14 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
     X, Wg, Wu, Wd = (t.to(dev) for t in (inp.X, inp.Wg, inp.Wu, inp.Wd))
     gamma = inp.gamma.to(dev) if inp.gamma is not None else None
     Y = torch.empty_like(X)
+    stream = torch.cuda.current_stream(dev)
+    tuned = None
+    if autotune:
+        # empirical schedule selection on this shape first (library-owned workspace), then AUTO follows it
+        gmlp.autotune(gmlp.make_args(X, Wg, Wu, Wd, Y, gamma, w.eps, w.rmsnorm, gmlp.VARIANT_AUTO, None, stream), 20)
+        tuned = gmlp.autotune_query(w.M, w.d_model, w.d_ff)
     variant = gmlp.pick_variant(w.M, w.d_model, w.d_ff)
     ws = gmlp.alloc_workspace(w.M, w.d_model, w.d_ff, w.rmsnorm)
-    stream = torch.cuda.current_stream(dev)
     a = gmlp.make_args(X, Wg, Wu, Wd, Y, gamma, w.eps, w.rmsnorm, gmlp.VARIANT_AUTO, ws, stream)
     weight_bytes = 3 * w.d_model * w.d_ff * 2
     fits_l2 = weight_bytes < L2_BYTES
@@ -255,6 +261,7 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
            "ms_min": min(per_step), "tokens_per_s": w.M / (ms * 1e-3), "tflops": w.flops / (ms * 1e-3) / 1e12,
            "gbps_min_bytes": w.min_bytes / (ms * 1e-3) / 1e9, "launches": launches, "clocks": clocks,
            "kernel_ms": kern_ms,
+           "autotuned": None if tuned is None else {"variant": tuned[0], "gate_up_pair": tuned[1], "down_pair": tuned[2]},
            "l2": "L2 overwritten between steps (weights fit L2); each step timed alone" if fits_l2
                  else "inputs larger than L2; steps back to back"}
 
@@ -409,6 +416,8 @@ def main():
     ap.add_argument("--op", default="gmlp", choices=["gmlp", "rmsnorm_matmul", "matmul_add_rmsnorm"],
                     help="rmsnorm_matmul / matmul_add_rmsnorm: print only that operator's {2K,4K,8K}^3 sweep "
                          "(one JSON line) and exit")
+    ap.add_argument("--autotune", action="store_true",
+                    help="run gmlp_autotune on each workload's shape before timing it (default: the built-in rule)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time spent on the oracle baseline (0 = skip)")
     ap.add_argument("--clock-roll", type=float, default=0.6,
                     help="seconds of untimed identical steps before and after the timed region while clocks are "
@@ -452,7 +461,8 @@ def main():
         return
 
     w = I.WORKLOADS[args.workload]
-    res = measure_workload(w, args.steps, warmup, dev, peaks, dist=dist, clock_roll=args.clock_roll)
+    res = measure_workload(w, args.steps, warmup, dev, peaks, dist=dist, clock_roll=args.clock_roll,
+                           autotune=args.autotune)
     from paper_2606_26344_b200 import sharding
     ms = sharding.max_over_ranks(res["ms_per_step"], dist, dev)          # the slowest rank bounds the step
     res["e2e"]["ms_per_step"] = sharding.max_over_ranks(res["e2e"]["ms_per_step"], dist, dev)
@@ -464,7 +474,7 @@ def main():
         for name in EXTRA:
             try:
                 r = measure_workload(I.WORKLOADS[name], max(5, min(args.steps, 30)), 3, dev, peaks,
-                                     want_e2e=False, sample_clocks=False)
+                                     want_e2e=False, sample_clocks=False, autotune=args.autotune)
                 r.pop("_inputs", None)
                 extras.append(r)
             except Exception as exc:  # a failed extra must not hide the primary number

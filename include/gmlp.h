@@ -234,7 +234,27 @@ int gmlp_forward_static(const void* X, const void* Wg, const void* Wu, const voi
  */
 uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant);
 
-/* The schedule AUTO resolves to for this shape (GMLP_VARIANT_SKINNY or _TENSOR). */
+/*
+ * Empirical schedule selection for one shape (the paper's extraction phase keeps, among the candidate kernels
+ * its search produced, the one that measures fastest, Sections 3 and 6): runs args (a complete, valid
+ * gmlp_forward_ex call; Y is overwritten with the correct result) with each tensor-core schedule that can run
+ * the shape (SKINNY up to 128 rows, and TENSOR with each of the four combinations of single-CTA or CTA-pair
+ * kernel for the gate/up and for the down GEMM; those that do not fit a caller-supplied workspace are
+ * skipped), about `iters` (1..10000) timed back-to-back calls each, in four interleaved rounds after a warm-up
+ * round so that clock drift falls on all candidates alike, CUDA events on args->stream, and
+ * remembers the fastest for (current device, M, d_model, d_ff): GMLP_VARIANT_AUTO, gmlp_pick_variant and
+ * gmlp_workspace_bytes use it from then on (size workspaces after tuning).  Synchronises the stream.
+ * best_variant (GMLP_VARIANT_SKINNY or _TENSOR) / best_us (microseconds per call) may be NULL.
+ * gmlp_autotune_query returns 1 and the kept choice if the shape was tuned on the current device (gate_up_pair /
+ * down_pair: 1 = CTA pairs, 0 = single CTAs, -1 = not applicable), else 0.  gmlp_autotune_clear forgets every
+ * tuned shape.
+ */
+int gmlp_autotune(const gmlp_args* args, int iters, int32_t* best_variant, float* best_us);
+int gmlp_autotune_query(int64_t M, int64_t d_model, int64_t d_ff, int32_t* variant, int32_t* gate_up_pair,
+                        int32_t* down_pair);
+void gmlp_autotune_clear(void);
+
+/* The schedule AUTO resolves to for this shape (GMLP_VARIANT_SKINNY or _TENSOR, or what gmlp_autotune kept). */
 int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);
 
 /*

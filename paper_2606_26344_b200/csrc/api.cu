@@ -3,8 +3,11 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstdio>
 #include <cstdlib>
+#include <atomic>
 #include <mutex>
+#include <vector>
 #include <new>
 
 #include "../../include/gmlp.h"
@@ -244,22 +247,71 @@ struct Layout {
 // SKINNY in long runs under the power cap, where issuing 128-row MMAs for 8 real rows costs clock).  From 9
 // tokens on the 128-row tcgen05 tiles win everywhere, because their down projection splits K over a cluster
 // and reduces on chip.  TENSOR then picks, per GEMM, between single-CTA tiles and CTA pairs.
+struct TunedShape {
+    int device;
+    int64_t M, d_model, d_ff;
+    int variant;
+    int gu_pair, down_pair;                      // TENSOR: kernel of each GEMM (1 = CTA pairs, 0 = single CTAs)
+};
+std::vector<TunedShape> g_tuned;                 // written by gmlp_autotune, under g_mutex
+std::atomic<int> g_tuned_count{0};               // lets untuned processes skip the lock
+
+bool tuned_lookup(int64_t M, int64_t d_model, int64_t d_ff, TunedShape* out) {
+    if (g_tuned_count.load(std::memory_order_acquire) == 0) return false;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+    std::lock_guard<std::mutex> lock(g_mutex);
+    for (const TunedShape& t : g_tuned)
+        if (t.device == dev && t.M == M && t.d_model == d_model && t.d_ff == d_ff) { *out = t; return true; }
+    return false;
+}
+
+int tuned_variant(int64_t M, int64_t d_model, int64_t d_ff) {
+    TunedShape t;
+    return tuned_lookup(M, d_model, d_ff, &t) ? t.variant : GMLP_VARIANT_AUTO;
+}
+
 int resolve_variant(int64_t M, int64_t d_model, int64_t d_ff, int32_t variant) {
-    (void)d_model;
-    (void)d_ff;
     if (variant != GMLP_VARIANT_AUTO) return variant;
+    const int tuned = tuned_variant(M, d_model, d_ff);
+    if (tuned != GMLP_VARIANT_AUTO) return tuned;
     return M <= 8 ? GMLP_VARIANT_SKINNY : GMLP_VARIANT_TENSOR;
 }
 
-// TENSOR: which kernel each GEMM takes, by the number of 128-row blocks.  A CTA pair works on 256 rows, so an
-// odd block count leaves half a pair idle (measured: 3 blocks run faster on single CTAs, 2 and 4 on pairs);
-// from 8 blocks on the pair kernel's higher rate outweighs that.  The down projection has few output tiles
-// at small M and prefers the single-CTA kernel, which can split K over a cluster, until 8 blocks.
+// TENSOR: which kernel each GEMM takes, by the number of 128-row blocks mt.  A CTA pair works on 256 rows, so an
+// odd block count leaves half a pair idle in the last row tile; measured on B200 (8B and 70B layer shapes):
+//   gate/up: pairs for even mt (mt = 2: 55.7 vs 63.3 us, 4: 97 vs 109, 6: 127 vs 135); single CTAs for odd mt
+//            (3: 85 vs 96 us, 9: 296 vs 306, 11 / 13 / 15 / 19: single ahead by 10-30 us) until the idle half
+//            is a few percent of the work (mt >= 24), where the pair kernel's higher rate wins again;
+//   down:    few output tiles at small M, so single CTAs (which can split K over a cluster) until mt = 8, then
+//            pairs, except mt = 9 (358 vs 296 us).
+// gmlp_autotune measures the four combinations for a given shape and overrides this rule.
 bool gate_up_uses_pair(int64_t M) {
     const int64_t mt = (M + 127) / 128;
-    return mt >= 8 || (mt >= 2 && mt % 2 == 0);
+    return mt >= 24 || (mt >= 2 && mt % 2 == 0);
 }
-bool down_uses_pair(int64_t M) { return (M + 127) / 128 >= 8; }
+bool down_uses_pair(int64_t M) {
+    const int64_t mt = (M + 127) / 128;
+    return mt == 8 || mt >= 10;
+}
+
+// The TENSOR plan of a shape: the rule above, unless gmlp_autotune measured the four combinations for this
+// shape and kept another one; t_force_* is how the tuner runs a combination of its choosing.
+struct TensorPlan {
+    bool gu_pair, down_pair;
+};
+thread_local int t_force_gu = -1, t_force_down = -1;
+TensorPlan tensor_plan(int64_t M, int64_t d_model, int64_t d_ff) {
+    TensorPlan p = {gate_up_uses_pair(M), down_uses_pair(M)};
+    TunedShape t;
+    if (tuned_lookup(M, d_model, d_ff, &t) && t.variant == GMLP_VARIANT_TENSOR) {
+        p.gu_pair = t.gu_pair != 0;
+        p.down_pair = t.down_pair != 0;
+    }
+    if (t_force_gu >= 0) p.gu_pair = t_force_gu != 0;
+    if (t_force_down >= 0) p.down_pair = t_force_down != 0;
+    return p;
+}
 
 Layout make_layout(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int variant, int sm_count) {
     Layout L{};
@@ -727,16 +779,18 @@ int forward_impl(const gmlp_args* a) {
                 if (rc == GMLP_OK) prof_mark("down", st);
             }
             break;
-        case GMLP_VARIANT_TENSOR:
-            rc = gate_up_uses_pair(a->M) ? launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act)
-                                         : launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act);
+        case GMLP_VARIANT_TENSOR: {
+            const TensorPlan plan = tensor_plan(a->M, a->d_model, a->d_ff);
+            rc = plan.gu_pair ? launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act)
+                              : launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act);
             if (rc == GMLP_OK) {
                 prof_mark("gate_up", st);
-                rc = down_uses_pair(a->M) ? launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st)
-                                          : launch_umma<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st);
+                rc = plan.down_pair ? launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st)
+                                    : launch_umma<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st);
                 if (rc == GMLP_OK) prof_mark("down", st);
             }
             break;
+        }
         default:
             rc = launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act);
             if (rc == GMLP_OK) {
@@ -880,7 +934,8 @@ int gate_up_impl(const gmlp_args* a) {
         unsigned int* c1 = reinterpret_cast<unsigned int*>(ws + L.counters_off);
         rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
         if (rc == GMLP_OK) rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, Hout, a->M, a->d_model, a->d_ff, st, act);
-    } else if (variant == GMLP_VARIANT_PAIR || (variant == GMLP_VARIANT_TENSOR && gate_up_uses_pair(a->M))) {
+    } else if (variant == GMLP_VARIANT_PAIR ||
+               (variant == GMLP_VARIANT_TENSOR && tensor_plan(a->M, a->d_model, a->d_ff).gu_pair)) {
         rc = launch_umma_pair<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st, act);
     } else {
         rc = launch_umma<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st, act);
@@ -1097,9 +1152,129 @@ int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
     return GMLP_OK;
 }
 
+// Empirical schedule selection for one shape: time every tensor-core schedule that can run it, keep the fastest.
+int autotune_impl(const gmlp_args* a, int iters, int32_t* best_variant, float* best_us) {
+    if (a == nullptr) return GMLP_ERR_NULL;
+    if (a->struct_bytes != sizeof(gmlp_args)) return GMLP_ERR_FLAGS;
+    if (iters < 1 || iters > 10000) return GMLP_ERR_FLAGS;
+    int rc = check_shape(a->M, a->d_model, a->d_ff);
+    if (rc != GMLP_OK) return rc;
+    if (a->M == 0) return GMLP_ERR_SHAPE;
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    cudaStream_t st = static_cast<cudaStream_t>(a->stream);
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        if (e0) (void)cudaEventDestroy(e0);
+        return GMLP_ERR_LAUNCH;
+    }
+    // candidates: SKINNY, and TENSOR with each of the four (gate/up kernel, down kernel) combinations
+    struct Cand { int variant, gu, down; };
+    const Cand candidates[5] = {{GMLP_VARIANT_SKINNY, -1, -1}, {GMLP_VARIANT_TENSOR, 0, 0}, {GMLP_VARIANT_TENSOR, 0, 1},
+                                {GMLP_VARIANT_TENSOR, 1, 0}, {GMLP_VARIANT_TENSOR, 1, 1}};
+    // The candidates are timed in interleaved rounds (each round runs every candidate for a share of the
+    // iterations; the first round is a warm-up and is not counted), so that clock and power drift over the
+    // tuning run falls on all of them alike instead of favouring whoever runs first.
+    constexpr int kRounds = 4;
+    const int per_round = (iters + kRounds - 1) / kRounds;
+    bool usable[5];
+    float total_ms[5] = {0, 0, 0, 0, 0};
+    int n_usable = 0;
+    for (int c = 0; c < 5; ++c) {
+        const int v = candidates[c].variant;
+        usable[c] = !(v == GMLP_VARIANT_SKINNY && a->M > 128) &&
+                    !(a->workspace != nullptr &&      // the caller's workspace must hold the schedule
+                      make_layout(a->M, a->d_model, a->d_ff, a->flags, v, dev->sm_count).total > a->workspace_bytes);
+        n_usable += usable[c] ? 1 : 0;
+    }
+    rc = GMLP_OK;
+    for (int round = 0; round <= kRounds && rc == GMLP_OK && n_usable > 0; ++round) {
+        for (int c = 0; c < 5 && rc == GMLP_OK; ++c) {
+            if (!usable[c]) continue;
+            gmlp_args t = *a;
+            t.variant = candidates[c].variant;
+            t.flags &= ~(uint32_t)GMLP_FLAG_CHECKED;
+            t_force_gu = candidates[c].gu;
+            t_force_down = candidates[c].down;
+            rc = forward_impl(&t);                          // not timed: the switch of schedule itself
+            float ms = 0.0f;
+            if (rc == GMLP_OK && cudaEventRecord(e0, st) != cudaSuccess) rc = GMLP_ERR_LAUNCH;
+            for (int i = 0; i < per_round && rc == GMLP_OK; ++i) rc = forward_impl(&t);
+            t_force_gu = t_force_down = -1;
+            if (rc != GMLP_OK) break;
+            if (cudaEventRecord(e1, st) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess ||
+                cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) { rc = GMLP_ERR_LAUNCH; break; }
+            if (round > 0) total_ms[c] += ms;
+        }
+    }
+    if (rc == GMLP_OK) {
+        const int s = read_device_status();
+        if (s < 0) rc = s;
+        else if (s != 0) rc = GMLP_ERR_TIMEOUT;
+    }
+    int best = -1;
+    for (int c = 0; c < 5; ++c)
+        if (usable[c] && (best < 0 || total_ms[c] < total_ms[best])) best = c;
+    const float best_ms = best >= 0 ? total_ms[best] : 0.0f;
+    const int timed_calls = kRounds * per_round;
+    if (getenv("GMLP_TUNE_VERBOSE")) {                       // the measurements behind the choice, on stderr
+        fprintf(stderr, "gmlp_autotune M=%lld d_model=%lld d_ff=%lld:", (long long)a->M, (long long)a->d_model, (long long)a->d_ff);
+        for (int c = 0; c < 5; ++c)
+            if (usable[c])
+                fprintf(stderr, " [variant %d gate_up_pair %d down_pair %d: %.1f us]%s", candidates[c].variant, candidates[c].gu,
+                        candidates[c].down, total_ms[c] * 1000.0f / (float)timed_calls, c == best ? "*" : "");
+        fprintf(stderr, "\n");
+    }
+    (void)cudaEventDestroy(e0);
+    (void)cudaEventDestroy(e1);
+    if (rc != GMLP_OK) return rc;
+    if (best < 0) return GMLP_ERR_WORKSPACE;                        // no candidate fitted the workspace
+    const Cand w = candidates[best];
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        bool found = false;
+        for (TunedShape& t : g_tuned)
+            if (t.device == device && t.M == a->M && t.d_model == a->d_model && t.d_ff == a->d_ff) {
+                t.variant = w.variant; t.gu_pair = w.gu; t.down_pair = w.down;
+                found = true;
+            }
+        if (!found) g_tuned.push_back({device, a->M, a->d_model, a->d_ff, w.variant, w.gu, w.down});
+        g_tuned_count.store((int)g_tuned.size(), std::memory_order_release);
+    }
+    if (best_variant) *best_variant = w.variant;
+    if (best_us) *best_us = best_ms * 1000.0f / (float)timed_calls;
+    return GMLP_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+int gmlp_autotune(const gmlp_args* args, int iters, int32_t* best_variant, float* best_us) {
+    try {
+        return autotune_impl(args, iters, best_variant, best_us);
+    } catch (...) {
+        return GMLP_ERR_LAUNCH;
+    }
+}
+
+int gmlp_autotune_query(int64_t M, int64_t d_model, int64_t d_ff, int32_t* variant, int32_t* gate_up_pair,
+                        int32_t* down_pair) {
+    TunedShape t;
+    if (!tuned_lookup(M, d_model, d_ff, &t)) return 0;
+    if (variant) *variant = t.variant;
+    if (gate_up_pair) *gate_up_pair = t.gu_pair;
+    if (down_pair) *down_pair = t.down_pair;
+    return 1;
+}
+
+void gmlp_autotune_clear(void) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_tuned.clear();
+    g_tuned_count.store(0, std::memory_order_release);
+}
 
 int gmlp_matmul_add_rmsnorm(const gmlp_mmaddnorm_args* args) {
     try {

@@ -97,6 +97,13 @@ def lib() -> ctypes.CDLL:
         L.gmlp_workspace_bytes.argtypes = [i64, i64, i64, u32, i32]
         L.gmlp_matmul_add_rmsnorm.restype = ctypes.c_int
         L.gmlp_matmul_add_rmsnorm.argtypes = [ctypes.POINTER(GmlpMmAddNormArgs)]
+        L.gmlp_autotune.restype = ctypes.c_int
+        L.gmlp_autotune.argtypes = [ctypes.POINTER(GmlpArgs), ctypes.c_int, ctypes.POINTER(ctypes.c_int32),
+                                    ctypes.POINTER(ctypes.c_float)]
+        L.gmlp_autotune_query.restype = ctypes.c_int
+        L.gmlp_autotune_query.argtypes = [i64, i64, i64] + [ctypes.POINTER(ctypes.c_int32)] * 3
+        L.gmlp_autotune_clear.restype = None
+        L.gmlp_autotune_clear.argtypes = []
         L.gmlp_pick_variant.restype = ctypes.c_int
         L.gmlp_pick_variant.argtypes = [i64, i64, i64, u32]
         L.gmlp_device_status.restype = ctypes.c_int
@@ -377,3 +384,25 @@ def matmul_add_rmsnorm(X, W, R, S=None, Z=None, gamma=None, eps: float = 1e-5, u
     with torch.cuda.device(X.device):
         matmul_add_rmsnorm_ex(make_mmaddnorm_args(X, W, R, S, Z, gamma, eps, unfused, ws, stream, checked))
     return S, Z
+
+
+def autotune(args: GmlpArgs, iters: int = 20):
+    """gmlp_autotune: time every schedule that can run args' shape, remember the fastest for AUTO.
+    Returns (variant, microseconds per call)."""
+    v, us = ctypes.c_int32(0), ctypes.c_float(0.0)
+    rc = lib().gmlp_autotune(ctypes.byref(args), iters, ctypes.byref(v), ctypes.byref(us))
+    if rc != OK:
+        raise GmlpError(rc)
+    return int(v.value), float(us.value)
+
+
+def autotune_clear() -> None:
+    lib().gmlp_autotune_clear()
+
+
+def autotune_query(M: int, d_model: int, d_ff: int):
+    """(variant, gate_up_pair, down_pair) kept by autotune for this shape on the current device, or None."""
+    v, g, d = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+    if not lib().gmlp_autotune_query(M, d_model, d_ff, ctypes.byref(v), ctypes.byref(g), ctypes.byref(d)):
+        return None
+    return int(v.value), int(g.value), int(d.value)

@@ -78,6 +78,11 @@ def test_argument_validation_happens_before_device_work(lib):
     assert lib.gmlp_forward(None, 0x1000, 0x1000, 0x1000, 0x1000, 4, 64, 128, 0) == gmlp.ERR_NULL
     assert lib.gmlp_forward_host(None, 0x1000, 0x1000) == gmlp.ERR_NULL
     assert lib.gmlp_forward_host(ctypes.byref(_args()), None, 0x1000) == gmlp.ERR_NULL
+    assert lib.gmlp_autotune(None, 5, None, None) == gmlp.ERR_NULL
+    assert lib.gmlp_autotune(ctypes.byref(_args()), 0, None, None) == gmlp.ERR_FLAGS
+    assert lib.gmlp_autotune(ctypes.byref(_args(M=0)), 5, None, None) == gmlp.ERR_SHAPE
+    lib.gmlp_autotune_clear()
+    assert lib.gmlp_matmul_add_rmsnorm(None) == gmlp.ERR_NULL
     assert lib.gmlp_set_default_eps(-1.0) == gmlp.ERR_FLAGS
     assert lib.gmlp_set_default_eps(1e-5) == gmlp.OK
 
