@@ -32,7 +32,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 PRIMARY = "llama3-8b-decode-M8"
-EXTRA = ["llama3-8b-prefill-M2048-rmsnorm", "llama3-70b-prefill-M4096-outliers", "ragged-M8192-plain",
+EXTRA = ["llama3-8b-batch-M64", "llama3-8b-prefill-M2048-rmsnorm", "llama3-70b-prefill-M4096-outliers", "ragged-M8192-plain",
          "ragged-M1000-plain", "ragged-M129-plain", "ragged-M7-plain", "ragged-M1-plain"]
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures

@@ -54,6 +54,7 @@ WORKLOADS = {
     w.name: w for w in [
         Workload("tiny", 16, 256, 512, 0),
         Workload("llama3-8b-decode-M8", 8, 4096, 14336, 0),
+        Workload("llama3-8b-batch-M64", 64, 4096, 14336, 0),      # not a stated config: the mid-M schedule on the same layer
         Workload("llama3-8b-prefill-M2048-rmsnorm", 2048, 4096, 14336, 0, rmsnorm=True, eps=1e-5),
         Workload("llama3-70b-prefill-M4096-outliers", 4096, 8192, 28672, 0, outlier_frac=0.01),
         *[_ragged(M, s, n) for (M, s) in zip((1, 7, 129, 1000, 8192), (1, 2, 3, 4, 5)) for n in (False, True)],

@@ -290,7 +290,7 @@ def test_no_write_outside_y_and_workspace(variant, M, rmsnorm):
 
 
 # ---------------------------------------------------------------- the five stated configurations at full size
-@pytest.mark.parametrize("name", ["llama3-8b-decode-M8",
+@pytest.mark.parametrize("name", ["llama3-8b-decode-M8", "llama3-8b-batch-M64",
                                   "ragged-M1-plain", "ragged-M1-norm", "ragged-M7-plain", "ragged-M7-norm",
                                   "ragged-M129-plain", "ragged-M129-norm", "ragged-M1000-plain", "ragged-M1000-norm",
                                   "ragged-M8192-plain", "ragged-M8192-norm",
