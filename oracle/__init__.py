@@ -94,6 +94,9 @@ def _load():
         lib.gmlp_oracle_matmul_add_rmsnorm_rows.argtypes = [u16p, u16p, u16p, u16p, ctypes.c_float, ctypes.c_int64,
                                                             ctypes.c_int64, ctypes.c_int64, i64p, ctypes.c_int64,
                                                             u16p, f64p, f64p, ctypes.c_int]
+        lib.gmlp_oracle_matmul_rows.restype = ctypes.c_int
+        lib.gmlp_oracle_matmul_rows.argtypes = [u16p, u16p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, i64p,
+                                                ctypes.c_int64, f64p, ctypes.c_int]
         lib.gmlp_oracle_gate_up_rows_act.restype = ctypes.c_int
         lib.gmlp_oracle_gate_up_rows_act.argtypes = lib.gmlp_oracle_gate_up_rows.argtypes + [ctypes.c_int, ctypes.c_double]
         lib.gmlp_oracle_rmsnorm_matmul_rows.restype = ctypes.c_int
@@ -304,6 +307,30 @@ def matmul_add_rmsnorm_rows(X, W, R, rows=None, gamma=None, eps: float = 1e-5, n
     if rc != 0:
         raise RuntimeError(f"gmlp_oracle_matmul_add_rmsnorm_rows failed ({rc})")
     return Sb, Sr, Z
+
+
+def matmul_rows(X, W, rows=None, num_threads: int = 0) -> np.ndarray:
+    """Reference X @ W (float64) for the selected rows; bf16 bit patterns in."""
+    lib = _load()
+    X, W = _u16(X, "X"), _u16(W, "W")
+    M, K = X.shape
+    if W.shape[0] != K:
+        raise ValueError("shape mismatch")
+    N = W.shape[1]
+    if rows is None:
+        rows = np.arange(M, dtype=np.int64)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    Z = np.zeros((rows.size, N), dtype=np.float64)
+    rc = lib.gmlp_oracle_matmul_rows(_p(X, ctypes.c_uint16), _p(W, ctypes.c_uint16), M, K, N, _p(rows, ctypes.c_int64),
+                                     rows.size, _p(Z, ctypes.c_double), int(num_threads))
+    if rc != 0:
+        raise RuntimeError(f"gmlp_oracle_matmul_rows failed ({rc})")
+    return Z
+
+
+def qkv_rows(X, Wq, Wk, Wv, rows=None, num_threads: int = 0):
+    """Reference (Q, K, V) = (X @ Wq, X @ Wk, X @ Wv) for the selected rows: the QKV projection."""
+    return tuple(matmul_rows(X, W, rows, num_threads) for W in (Wq, Wk, Wv))
 
 
 def naive_matmul(A, B) -> np.ndarray:

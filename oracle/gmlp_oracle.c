@@ -392,6 +392,36 @@ int gmlp_oracle_matmul_add_rmsnorm_rows(const uint16_t* X, const uint16_t* W, co
     return failed ? -1 : 0;
 }
 
+/*
+ * A plain matrix multiplication on selected rows, Z[i, n] = sum_k X[rows[i], k] * W[k, n] in fp64 (the granular
+ * definition of matmul in Section 5's operation table).  It is the reference for each of the three products of
+ * the QKV projection (Section 6.1), which share X and nothing else.  X [M, K], W [K, N] bf16 bit patterns.
+ */
+int gmlp_oracle_matmul_rows(const uint16_t* X, const uint16_t* W, int64_t M, int64_t K, int64_t N,
+                            const int64_t* rows, int64_t n_rows, double* Z, int num_threads)
+{
+    if (!X || !W || !rows || !Z || M < 0 || K <= 0 || N <= 0 || n_rows < 0) return -1;
+    for (int64_t i = 0; i < n_rows; ++i)
+        if (rows[i] < 0 || rows[i] >= M) return -1;
+#ifdef _OPENMP
+    if (num_threads > 0) omp_set_num_threads(num_threads);
+#else
+    (void)num_threads;
+#endif
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < n_rows; ++i) {
+        const uint16_t* x = X + rows[i] * K;
+        double* z = Z + i * N;
+        for (int64_t n = 0; n < N; ++n) z[n] = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            const double xk = gmlp_oracle_bf16_to_double(x[k]);
+            const uint16_t* w = W + k * N;
+            for (int64_t n = 0; n < N; ++n) z[n] += xk * gmlp_oracle_bf16_to_double(w[n]);
+        }
+    }
+    return 0;
+}
+
 /* Array forms of the two scalar helpers (plain loops), for the tests. */
 void gmlp_oracle_bf16_rn_array(const double* v, uint16_t* out, int64_t n)
 {
