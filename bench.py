@@ -36,10 +36,11 @@ EXTRA = ["llama3-8b-batch-M64", "llama3-8b-prefill-M2048-rmsnorm", "llama3-70b-p
          "ragged-M1000-plain", "ragged-M129-plain", "ragged-M7-plain", "ragged-M1-plain"]
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
-# summarised under profiles/ (skinny_gemm_decode_M8.md, umma_gemm_prefill8b_M2048.md)
+# summarised under profiles/ (skinny_gemm_decode_M8.md, umma_pair_gemm_prefill8b_M2048.md, umma_gemm_batch64_M64.md)
 NCU_TRAFFIC_BYTES = {
-    ("llama3-8b-decode-M8", "gate_up"): 235.5e6 + 4.0e6,
-    ("llama3-8b-prefill-M2048-rmsnorm", "gate_up"): 255.4e6 + 51.2e6,
+    ("llama3-8b-decode-M8", "gate_up"): 235.0e6 + 4.2e6,
+    ("llama3-8b-prefill-M2048-rmsnorm", "gate_up"): 253.6e6 + 52.0e6,
+    ("llama3-8b-batch-M64", "gate_up"): 235.5e6 + 4.1e6,
 }
 
 
@@ -405,6 +406,46 @@ def measure_matmul_add_rmsnorm(dev, sizes=(2048, 4096, 8192), iters=10):
             "best_fused_tflops": max(r["fused_tflops"] for r in rows), "table": rows}
 
 
+def measure_qkv(dev, iters=10):
+    """QKV projection on grouped-query attention shapes: one launch over the three weight matrices against three
+    GEMM launches.  Microseconds, CUDA events."""
+    import math
+    import torch
+    from paper_2606_26344_b200 import gmlp
+    g = torch.Generator(device="cpu").manual_seed(0)
+    rows = []
+    for (K, Nq, Nkv, label) in ((2048, 2048, 512, "2048-wide, 4:1 groups"), (4096, 4096, 1024, "8B attention block"),
+                                (8192, 8192, 1024, "70B attention block")):
+        Ws = [(torch.randn(K, n, generator=g) * K ** -0.5).bfloat16().to(dev) for n in (Nq, Nkv, Nkv)]
+        for M in (128, 512, 2048, 4096, 8192):
+            X = torch.randn(M, K, generator=g).bfloat16().to(dev)
+            Q = torch.empty(M, Nq, dtype=torch.bfloat16, device=dev)
+            Ko, V = (torch.empty(M, Nkv, dtype=torch.bfloat16, device=dev) for _ in range(2))
+            t = {}
+            for name, sep in (("fused", False), ("separate", True)):
+                a = gmlp.make_qkv_args(X, Ws[0], Ws[1], Ws[2], Q, Ko, V, sep)
+                for _ in range(3):
+                    gmlp.qkv_proj_ex(a)
+                torch.cuda.synchronize(dev)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(iters):
+                    gmlp.qkv_proj_ex(a)
+                e1.record()
+                torch.cuda.synchronize(dev)
+                t[name] = e0.elapsed_time(e1) / iters * 1e3
+            rows.append({"shape": label, "M": M, "K": K, "Nq": Nq, "Nkv": Nkv, "fused_us": t["fused"],
+                         "separate_us": t["separate"], "speedup": t["separate"] / t["fused"],
+                         "fused_tflops": 2.0 * M * K * (Nq + 2 * Nkv) / t["fused"] / 1e6})
+            del X, Q, Ko, V
+        del Ws
+    sp = [r["speedup"] for r in rows]
+    return {"timing": "back-to-back calls, operands may stay in L2",
+            "geomean_speedup_fused_over_separate": math.exp(sum(math.log(v) for v in sp) / len(sp)),
+            "min_speedup": min(sp), "max_speedup": max(sp),
+            "best_fused_tflops": max(r["fused_tflops"] for r in rows), "table": rows}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -413,8 +454,8 @@ def main():
     ap.add_argument("--impl", default="gmlp", choices=["gmlp", "reference"])
     ap.add_argument("--workload", default=PRIMARY)
     ap.add_argument("--no-extra", action="store_true", help="time only the primary workload")
-    ap.add_argument("--op", default="gmlp", choices=["gmlp", "rmsnorm_matmul", "matmul_add_rmsnorm"],
-                    help="rmsnorm_matmul / matmul_add_rmsnorm: print only that operator's {2K,4K,8K}^3 sweep "
+    ap.add_argument("--op", default="gmlp", choices=["gmlp", "rmsnorm_matmul", "matmul_add_rmsnorm", "qkv"],
+                    help="rmsnorm_matmul / matmul_add_rmsnorm / qkv: print only that operator's sweep "
                          "(one JSON line) and exit")
     ap.add_argument("--autotune", action="store_true",
                     help="run gmlp_autotune on each workload's shape before timing it (default: the built-in rule)")
@@ -451,9 +492,10 @@ def main():
     peaks = load_peaks()
     warmup = max(args.warmup, 3)
 
-    if args.op in ("rmsnorm_matmul", "matmul_add_rmsnorm"):
+    if args.op != "gmlp":
         if rank == 0:
-            fn = measure_rmsnorm_matmul if args.op == "rmsnorm_matmul" else measure_matmul_add_rmsnorm
+            fn = {"rmsnorm_matmul": measure_rmsnorm_matmul, "matmul_add_rmsnorm": measure_matmul_add_rmsnorm,
+                  "qkv": measure_qkv}[args.op]
             print(json.dumps({"op": args.op, **fn(dev)}))
         if dist is not None:
             dist.barrier()

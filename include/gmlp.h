@@ -186,6 +186,32 @@ typedef struct gmlp_mmaddnorm_args {
 int gmlp_matmul_add_rmsnorm(const gmlp_mmaddnorm_args* args);
 
 /*
+ * QKV projection, one of the paper's multi-operator kernels (Section 6.1): three matmuls that share X,
+ *     Q = X * Wq  [M, Nq],     K = X * Wk  [M, Nkv],     V = X * Wv  [M, Nkv]       (grouped-query shapes: Nkv <= Nq),
+ * X [M, K], W* [K, N*], outputs row-major bf16, fp32 accumulation, one rounding; K, Nq, Nkv multiples of 8.
+ * Default: ONE launch of the tensor-core GEMM whose column tiles run through the three weight matrices end to end
+ * (the same sharing of the X strip that fuses the gate and up matmuls), each tile written to its own output.
+ * GMLP_QKV_SEPARATE runs three GEMMs one after the other (for comparison).  No workspace.  The attention that
+ * follows (GQA) is not part of this library.
+ */
+enum { GMLP_QKV_SEPARATE = 1u << 4 };
+typedef struct gmlp_qkv_args {
+    uint32_t struct_bytes;    /* sizeof(gmlp_qkv_args) */
+    uint32_t flags;           /* GMLP_FLAG_CHECKED | GMLP_QKV_SEPARATE */
+    const void* X;            /* device, [M, K] bf16 */
+    const void* Wq;           /* device, [K, Nq] bf16 */
+    const void* Wk;           /* device, [K, Nkv] bf16 */
+    const void* Wv;           /* device, [K, Nkv] bf16 */
+    void* Q;                  /* device, [M, Nq] bf16, written */
+    void* Kout;               /* device, [M, Nkv] bf16, written */
+    void* V;                  /* device, [M, Nkv] bf16, written */
+    int64_t M, K, Nq, Nkv;
+    void* stream;             /* cudaStream_t */
+    uint64_t reserved;        /* must be 0 */
+} gmlp_qkv_args;
+int gmlp_qkv_proj(const gmlp_qkv_args* args);
+
+/*
  * The same call for a caller whose activations live in HOST memory: copies X_host
  * (M*d_model bf16, ideally pinned) to args->X, runs gmlp_forward_ex, and copies args->Y
  * to Y_host, all asynchronously on args->stream.  args->X and args->Y are device staging

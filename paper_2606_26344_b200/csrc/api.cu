@@ -29,6 +29,7 @@ constexpr int kMaxDevices = 64;
 constexpr int64_t kMaxDim = (int64_t)1 << 30;      // per-dimension limit (TMA coordinates are int32)
 constexpr uint32_t kKnownFlags = GMLP_FLAG_RMSNORM | GMLP_FLAG_CHECKED | GMLP_FLAG_ACT_SWISH | GMLP_FLAG_ACT_GLU;
 constexpr gmlp::GateAct kSilu = {1.0f, 0};
+const gmlp::MultiB kNoMulti = {};
 
 // Gate activation named by the flags (SiLU when none is set); false for a contradictory or non-finite request.
 bool gate_act_from(uint32_t flags, float beta, gmlp::GateAct* out) {
@@ -94,6 +95,7 @@ struct DeviceState {
     uint64_t workspace_bytes = 0;
     bool splitk_attr_set = false;
     bool addss_attr_set = false;
+    bool multi_attr_set = false;
     bool umma_attr_set = false;
     bool pair_attr_set = false;
     bool rowscale_attr_set = false;
@@ -494,7 +496,7 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
     if (cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m,
-                           num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr) != cudaSuccess)
+                           num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti) != cudaSuccess)
         return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -604,16 +606,16 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     cudaError_t err;
     if (GATEUP && nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti);
     else if (GATEUP)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti);
     else if (nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti);
     else
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -1028,8 +1030,8 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         const float* rc_ptr = r;
         cudaError_t err = pair
-            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr)
-            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr);
+            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti)
+            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("matmul_rowscale", st);
@@ -1122,9 +1124,9 @@ int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         cudaError_t err = pair
             ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
-                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq)
+                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq, kNoMulti)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
-                                 num_tiles, (const float*)nullptr, 128, kSilu, R, sumsq);
+                                 num_tiles, (const float*)nullptr, 128, kSilu, R, sumsq, kNoMulti);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("matmul_add", st);
@@ -1142,6 +1144,103 @@ int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
             return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("rmsnorm_apply", st);
+    }
+    if (a->flags & GMLP_FLAG_CHECKED) {
+        if (cudaStreamSynchronize(st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+        const int s = read_device_status();
+        if (s < 0) return s;
+        if (s != 0) return GMLP_ERR_TIMEOUT;
+    }
+    return GMLP_OK;
+}
+
+// QKV projection (Section 6.1): Q = X Wq, K = X Wk, V = X Wv in one launch of the multi-matrix GEMM.
+int qkv_proj_impl(const gmlp_qkv_args* a) {
+    if (a == nullptr) return GMLP_ERR_NULL;
+    if (a->struct_bytes != sizeof(gmlp_qkv_args)) return GMLP_ERR_FLAGS;
+    if ((a->flags & ~(uint32_t)(GMLP_FLAG_CHECKED | GMLP_QKV_SEPARATE)) || a->reserved != 0) return GMLP_ERR_FLAGS;
+    int rc = check_shape(a->M, a->K, a->Nq);
+    if (rc == GMLP_OK) rc = check_shape(a->M, a->K, a->Nkv);
+    if (rc != GMLP_OK) return rc;
+    if (a->M == 0) return GMLP_OK;
+    if (!a->X || !a->Wq || !a->Wk || !a->Wv || !a->Q || !a->Kout || !a->V) return GMLP_ERR_NULL;
+    if (!aligned16(a->X) || !aligned16(a->Wq) || !aligned16(a->Wk) || !aligned16(a->Wv) || !aligned16(a->Q) ||
+        !aligned16(a->Kout) || !aligned16(a->V))
+        return GMLP_ERR_ALIGN;
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(a->stream);
+    const bf16* X = static_cast<const bf16*>(a->X);
+    const bf16* Wq = static_cast<const bf16*>(a->Wq);
+    const bf16* Wk = static_cast<const bf16*>(a->Wk);
+    const bf16* Wv = static_cast<const bf16*>(a->Wv);
+    bf16* Q = static_cast<bf16*>(a->Q);
+    bf16* Ko = static_cast<bf16*>(a->Kout);
+    bf16* V = static_cast<bf16*>(a->V);
+    const int64_t mt = (a->M + 127) / 128;
+    const bool pair = mt >= 24 || (mt >= 2 && mt % 2 == 0);          // as for the gate/up GEMM
+    prof_begin(st);
+    if (a->flags & GMLP_QKV_SEPARATE) {
+        // three plain GEMMs, one after the other
+        const bf16* Ws[3] = {Wq, Wk, Wv};
+        bf16* Os[3] = {Q, Ko, V};
+        const int64_t Ns[3] = {a->Nq, a->Nkv, a->Nkv};
+        const char* names[3] = {"q", "k", "v"};
+        for (int i = 0; i < 3; ++i) {
+            rc = pair ? launch_umma_pair<false>(dev, X, Ws[i], nullptr, Os[i], a->M, a->K, Ns[i], st)
+                      : launch_umma<false>(dev, X, Ws[i], nullptr, Os[i], a->M, a->K, Ns[i], st);
+            if (rc != GMLP_OK) return rc;
+            prof_mark(names[i], st);
+        }
+    } else {
+        CUtensorMap tmA, tmB0, tmB1;
+        gmlp::MultiB multi = {};
+        if (!encode_2d(&tmA, X, (uint64_t)a->K, (uint64_t)a->M, gmlp::kUmmaBK, 128) ||
+            !encode_2d(&tmB0, Wq, (uint64_t)a->Nq, (uint64_t)a->K, 64, gmlp::kUmmaBK) ||
+            !encode_2d(&tmB1, Wk, (uint64_t)a->Nkv, (uint64_t)a->K, 64, gmlp::kUmmaBK) ||
+            !encode_2d(&multi.tmB2, Wv, (uint64_t)a->Nkv, (uint64_t)a->K, 64, gmlp::kUmmaBK))
+            return GMLP_ERR_LAUNCH;
+        multi.C1 = Ko;
+        multi.C2 = V;
+        multi.N1 = multi.N2 = (int)a->Nkv;
+        multi.tiles0 = (int)((a->Nq + 255) / 256);
+        multi.tiles1 = (int)((a->Nkv + 255) / 256);
+        if (!dev->multi_attr_set) {
+            if (cudaFuncSetAttribute(gmlp::umma_gemm_kernel<false, 4, false, false, true>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gmlp::kUmmaSmemBytes) != cudaSuccess ||
+                cudaFuncSetAttribute(gmlp::umma_pair_gemm_kernel<false, false, false, true>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gmlp::kPairSmemBytes) != cudaSuccess)
+                return GMLP_ERR_LAUNCH;
+            dev->multi_attr_set = true;
+        }
+        const int sms = dev->sm_count > 0 ? dev->sm_count : 148;
+        const int num_m = (int)((a->M + (pair ? 255 : 127)) / (pair ? 256 : 128));
+        const int num_tiles = num_m * (multi.tiles0 + 2 * multi.tiles1);
+        const int ctas = pair ? 2 * (num_tiles < sms / 2 ? num_tiles : sms / 2) : (num_tiles < sms ? num_tiles : sms);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)ctas);
+        cfg.blockDim = dim3(gmlp::kUmmaThreads);
+        cfg.dynamicSmemBytes = pair ? gmlp::kPairSmemBytes : gmlp::kUmmaSmemBytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = 2;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pair ? 2 : 1;
+        const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->Nq;
+        cudaError_t err = pair
+            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, false, true>, tmA, tmB0, tmB1, Q, Mi, Ki, Ni,
+                                 num_m, num_tiles, (const float*)nullptr, kSilu, (const bf16*)nullptr, (float*)nullptr, multi)
+            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, false, true>, tmA, tmB0, tmB1, Q, Mi, Ki, Ni,
+                                 num_m, num_tiles, (const float*)nullptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr,
+                                 multi);
+        if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
+        GMLP_CHECK_LAUNCH();
+        prof_mark("qkv", st);
     }
     if (a->flags & GMLP_FLAG_CHECKED) {
         if (cudaStreamSynchronize(st) != cudaSuccess) return GMLP_ERR_LAUNCH;
@@ -1251,6 +1350,14 @@ int autotune_impl(const gmlp_args* a, int iters, int32_t* best_variant, float* b
 }  // namespace
 
 extern "C" {
+
+int gmlp_qkv_proj(const gmlp_qkv_args* args) {
+    try {
+        return qkv_proj_impl(args);
+    } catch (...) {
+        return GMLP_ERR_LAUNCH;
+    }
+}
 
 int gmlp_autotune(const gmlp_args* args, int iters, int32_t* best_variant, float* best_us) {
     try {

@@ -77,6 +77,25 @@ __global__ void wait_timeout_probe_kernel(long long limit_cycles)
     __syncthreads();
 }
 
+// Several weight matrices behind one A operand in ONE launch (the QKV projection of Section 6.1: three matmuls
+// that share X).  The column tiles of the matrices are laid end to end: tiles [0, tiles0) belong to the first
+// matrix (tensor map tmB0, output C, N columns), [tiles0, tiles0 + tiles1) to the second (tmB1, C1, N1), the rest
+// to the third (tmB2, C2, N2).  Row tiles vary fastest, so a round of CTAs shares A panels in L2.
+struct alignas(64) MultiB {
+    CUtensorMap tmB2;
+    bf16* C1;
+    bf16* C2;
+    int N1, N2;
+    int tiles0, tiles1;
+};
+// which matrix a column tile belongs to (0, 1, 2) and its tile index inside that matrix
+__device__ __forceinline__ int multi_segment(const MultiB& m, int n_tile, int* local) {
+    if (n_tile < m.tiles0) { *local = n_tile; return 0; }
+    if (n_tile < m.tiles0 + m.tiles1) { *local = n_tile - m.tiles0; return 1; }
+    *local = n_tile - m.tiles0 - m.tiles1;
+    return 2;
+}
+
 // Residual epilogue of "Matmul+Add+RMSNorm" (Section 6.1) for 32 accumulator columns of one row:
 // s = acc + R, stored value = bf16_rn(s), and ss += (stored value)^2 - the statistic of Eq. (1) is taken over
 // what is stored.  rrow points at the row's residual for the chunk's first column; columns at or beyond
@@ -108,15 +127,16 @@ __device__ __forceinline__ void add_residual_chunk(const uint32_t (&acc)[32], ui
 // not depend on k).  r comes from row_rsqrt_kernel, the kernel launched just before this one: the two
 // are chained by programmatic dependent launch and ONLY the epilogue warps wait for it, so the main loop
 // (which reads the raw X) runs in parallel with the RMS branch.
-template <bool GATEUP, int NB, bool ROWSCALE = false, bool ADDSS = false>
+template <bool GATEUP, int NB, bool ROWSCALE = false, bool ADDSS = false, bool MULTI = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
                  int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, int a_box_rows, GateAct act,
-                 const bf16* residual, float* __restrict__ sumsq)
+                 const bf16* residual, float* __restrict__ sumsq, const __grid_constant__ MultiB multi)
 {
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
     static_assert(!(ADDSS && (GATEUP || ROWSCALE)), "the residual epilogue is for the plain GEMM");
+    static_assert(!(MULTI && (GATEUP || ROWSCALE || ADDSS)), "several weight matrices: plain GEMM only");
     constexpr int KERNEL_ID = GATEUP ? 1 : 2;
     constexpr int N_MMA = 64 * NB;
     constexpr int BN_OUT = GATEUP ? N_MMA / 2 : N_MMA;
@@ -156,7 +176,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ptx::fence_proxy_async_smem();
         ptx::prefetch_tensormap(&tmA);
         ptx::prefetch_tensormap(&tmB0);
-        if (GATEUP) ptx::prefetch_tensormap(&tmB1);
+        if (GATEUP || MULTI) ptx::prefetch_tensormap(&tmB1);
+        if (MULTI) ptx::prefetch_tensormap(&multi.tmB2);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_addr(tmem_slot), kUmmaTmemCols);
@@ -180,7 +201,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t a_tx_bytes = (uint32_t)a_box_rows * 128u;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 const int m0 = (tile % num_m_tiles) * kUmmaBM;
-                const int n0 = (tile / num_m_tiles) * BN_OUT;
+                int n0 = (tile / num_m_tiles) * BN_OUT;
+                const CUtensorMap* plain_map = &tmB0;
+                if (MULTI) {
+                    int local;
+                    const int seg = multi_segment(multi, tile / num_m_tiles, &local);
+                    n0 = local * BN_OUT;
+                    plain_map = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &multi.tmB2);
+                }
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (uint32_t)(it / kStages) & 1u;
@@ -193,7 +221,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                     for (int i = 0; i < NB; ++i) {
                         // gate/up: the first NB/2 boxes are gate columns, the rest the same columns of up
-                        const CUtensorMap* map = (GATEUP && i >= NB / 2) ? &tmB1 : &tmB0;
+                        const CUtensorMap* map = (GATEUP && i >= NB / 2) ? &tmB1 : plain_map;
                         const int x = GATEUP ? n0 + (i % (NB / 2)) * 64 : n0 + i * 64;
                         ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
                     }
@@ -242,12 +270,21 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++t) {
             const int buf = t & 1;
             const int m0 = (tile % num_m_tiles) * kUmmaBM;
-            const int n0 = (tile / num_m_tiles) * BN_OUT;
+            int n0 = (tile / num_m_tiles) * BN_OUT;
             const int row = m0 + q * 32 + lane;
             if (!wait_bounded(tfull0 + 8 * buf, ((uint32_t)t >> 1) & 1u, abort_flag, KERNEL_ID, 3)) break;
             ptx::tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * kUmmaN);
-            bf16* crow = C + (size_t)row * N + n0;
+            bf16* Cseg = C;
+            int Nseg = N;
+            if (MULTI) {                                           // this tile's matrix: its output and width
+                int local;
+                const int seg = multi_segment(multi, tile / num_m_tiles, &local);
+                n0 = local * BN_OUT;
+                if (seg == 1) { Cseg = multi.C1; Nseg = multi.N1; }
+                else if (seg == 2) { Cseg = multi.C2; Nseg = multi.N2; }
+            }
+            bf16* crow = Cseg + (size_t)row * Nseg + n0;
             const float rscale = (ROWSCALE && row < M) ? __ldcg(row_scale + row) : 1.0f;
             float ss = 0.0f;                                       // ADDSS: sum of squares of this row's stored values
 #pragma unroll 1
@@ -279,7 +316,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (row < M) {
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
-                        if (n0 + c + v * 8 < N)
+                        if (n0 + c + v * 8 < Nseg)
                             *reinterpret_cast<uint4*>(crow + c + v * 8) =
                                 make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
                     }

@@ -84,15 +84,16 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 }  // namespace ptx
 
 // ROWSCALE: see umma_gemm.cuh (epilogue row scale from row_rsqrt_kernel; only the epilogue waits for it).
-template <bool GATEUP, bool ROWSCALE = false, bool ADDSS = false>
+template <bool GATEUP, bool ROWSCALE = false, bool ADDSS = false, bool MULTI = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                       const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
                       int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, GateAct act,
-                      const bf16* residual, float* __restrict__ sumsq)
+                      const bf16* residual, float* __restrict__ sumsq, const __grid_constant__ MultiB multi)
 {
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
     static_assert(!(ADDSS && (GATEUP || ROWSCALE)), "the residual epilogue is for the plain GEMM");
+    static_assert(!(MULTI && (GATEUP || ROWSCALE || ADDSS)), "several weight matrices: plain GEMM only");
     constexpr int KERNEL_ID = GATEUP ? 6 : 7;
     constexpr int BN_OUT = GATEUP ? 128 : 256;
     // D = fp32, A = B = bf16, A K-major, B MN-major, M = 256 (128 per CTA), N = 256
@@ -131,7 +132,8 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         ptx::fence_proxy_async_smem();
         ptx::prefetch_tensormap(&tmA);
         ptx::prefetch_tensormap(&tmB0);
-        if (GATEUP) ptx::prefetch_tensormap(&tmB1);
+        if (GATEUP || MULTI) ptx::prefetch_tensormap(&tmB1);
+        if (MULTI) ptx::prefetch_tensormap(&multi.tmB2);
     }
     if (warp == 1) {
         ptx::tmem_alloc_pair(ptx::smem_addr(tmem_slot), kUmmaTmemCols);
@@ -152,9 +154,15 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
                 const int m0 = (tile % num_m_tiles) * 256 + (int)rank * 128;
-                const int n0 = (tile / num_m_tiles) * BN_OUT;
+                int n0 = (tile / num_m_tiles) * BN_OUT;
                 // this CTA's half of the B columns: gate/up -> gate (rank 0) or up (rank 1) columns n0..n0+127
                 const CUtensorMap* bmap = (GATEUP && rank == 1) ? &tmB1 : &tmB0;
+                if (MULTI) {
+                    int local;
+                    const int seg = multi_segment(multi, tile / num_m_tiles, &local);
+                    n0 = local * BN_OUT;
+                    bmap = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &multi.tmB2);
+                }
                 const int bx = GATEUP ? n0 : n0 + (int)rank * 128;
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % kPairStages;
@@ -209,12 +217,21 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++t) {
             const int buf = t & 1;
             const int m0 = (tile % num_m_tiles) * 256 + (int)rank * 128;
-            const int n0 = (tile / num_m_tiles) * BN_OUT;
+            int n0 = (tile / num_m_tiles) * BN_OUT;
             const int row = m0 + q * 32 + lane;
             if (!wait_bounded(tfull0 + 8 * buf, ((uint32_t)t >> 1) & 1u, abort_flag, KERNEL_ID, 3)) break;
             ptx::tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256);
-            bf16* crow = C + (size_t)row * N + n0;
+            bf16* Cseg = C;
+            int Nseg = N;
+            if (MULTI) {                                           // this tile's matrix: its output and width
+                int local;
+                const int seg = multi_segment(multi, tile / num_m_tiles, &local);
+                n0 = local * BN_OUT;
+                if (seg == 1) { Cseg = multi.C1; Nseg = multi.N1; }
+                else if (seg == 2) { Cseg = multi.C2; Nseg = multi.N2; }
+            }
+            bf16* crow = Cseg + (size_t)row * Nseg + n0;
             const float rscale = (ROWSCALE && row < M) ? __ldcg(row_scale + row) : 1.0f;
             float ss = 0.0f;                                       // ADDSS: sum of squares of this row's stored values
 #pragma unroll 1
@@ -246,7 +263,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 if (row < M) {
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
-                        if (n0 + c + v * 8 < N)
+                        if (n0 + c + v * 8 < Nseg)
                             *reinterpret_cast<uint4*>(crow + c + v * 8) =
                                 make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
                     }

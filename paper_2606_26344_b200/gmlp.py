@@ -53,6 +53,17 @@ class GmlpRmsmmArgs(ctypes.Structure):
 
 RMSMM_UNFUSED = 1 << 4
 MMADDNORM_UNFUSED = 1 << 4
+QKV_SEPARATE = 1 << 4
+
+
+class GmlpQkvArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_bytes", ctypes.c_uint32), ("flags", ctypes.c_uint32),
+        ("X", ctypes.c_void_p), ("Wq", ctypes.c_void_p), ("Wk", ctypes.c_void_p), ("Wv", ctypes.c_void_p),
+        ("Q", ctypes.c_void_p), ("Kout", ctypes.c_void_p), ("V", ctypes.c_void_p),
+        ("M", ctypes.c_int64), ("K", ctypes.c_int64), ("Nq", ctypes.c_int64), ("Nkv", ctypes.c_int64),
+        ("stream", ctypes.c_void_p), ("reserved", ctypes.c_uint64),
+    ]
 
 
 class GmlpMmAddNormArgs(ctypes.Structure):
@@ -97,6 +108,8 @@ def lib() -> ctypes.CDLL:
         L.gmlp_workspace_bytes.argtypes = [i64, i64, i64, u32, i32]
         L.gmlp_matmul_add_rmsnorm.restype = ctypes.c_int
         L.gmlp_matmul_add_rmsnorm.argtypes = [ctypes.POINTER(GmlpMmAddNormArgs)]
+        L.gmlp_qkv_proj.restype = ctypes.c_int
+        L.gmlp_qkv_proj.argtypes = [ctypes.POINTER(GmlpQkvArgs)]
         L.gmlp_autotune.restype = ctypes.c_int
         L.gmlp_autotune.argtypes = [ctypes.POINTER(GmlpArgs), ctypes.c_int, ctypes.POINTER(ctypes.c_int32),
                                     ctypes.POINTER(ctypes.c_float)]
@@ -406,3 +419,40 @@ def autotune_query(M: int, d_model: int, d_ff: int):
     if not lib().gmlp_autotune_query(M, d_model, d_ff, ctypes.byref(v), ctypes.byref(g), ctypes.byref(d)):
         return None
     return int(v.value), int(g.value), int(d.value)
+
+
+def make_qkv_args(X, Wq, Wk, Wv, Q, K, V, separate: bool = False, stream=None, checked: bool = False) -> GmlpQkvArgs:
+    for t, n in ((X, "X"), (Wq, "Wq"), (Wk, "Wk"), (Wv, "Wv"), (Q, "Q"), (K, "K"), (V, "V")):
+        _check_bf16_cuda(t, n)
+    M, Kd = X.shape
+    Nq, Nkv = Wq.shape[1], Wk.shape[1]
+    if Wq.shape[0] != Kd or Wk.shape != (Kd, Nkv) or Wv.shape != (Kd, Nkv) or Q.shape != (M, Nq) or K.shape != (M, Nkv) \
+            or V.shape != (M, Nkv):
+        raise ValueError("shape mismatch")
+    st = stream if stream is not None else torch.cuda.current_stream(X.device)
+    a = GmlpQkvArgs()
+    a.struct_bytes = ctypes.sizeof(GmlpQkvArgs)
+    a.flags = (FLAG_CHECKED if checked else 0) | (QKV_SEPARATE if separate else 0)
+    a.X, a.Wq, a.Wk, a.Wv = X.data_ptr(), Wq.data_ptr(), Wk.data_ptr(), Wv.data_ptr()
+    a.Q, a.Kout, a.V = Q.data_ptr(), K.data_ptr(), V.data_ptr()
+    a.M, a.K, a.Nq, a.Nkv = M, Kd, Nq, Nkv
+    a.stream = st.cuda_stream
+    a.reserved = 0
+    return a
+
+
+def qkv_proj_ex(args: GmlpQkvArgs) -> None:
+    rc = lib().gmlp_qkv_proj(ctypes.byref(args))
+    if rc != OK:
+        raise GmlpError(rc)
+
+
+def qkv_proj(X, Wq, Wk, Wv, separate: bool = False, stream=None, checked: bool = False):
+    """gmlp_qkv_proj: (Q, K, V) = (X @ Wq, X @ Wk, X @ Wv), one launch unless ``separate``."""
+    M = X.shape[0]
+    Q = torch.empty(M, Wq.shape[1], dtype=torch.bfloat16, device=X.device)
+    K = torch.empty(M, Wk.shape[1], dtype=torch.bfloat16, device=X.device)
+    V = torch.empty(M, Wv.shape[1], dtype=torch.bfloat16, device=X.device)
+    with torch.cuda.device(X.device):
+        qkv_proj_ex(make_qkv_args(X, Wq, Wk, Wv, Q, K, V, separate, stream, checked))
+    return Q, K, V
