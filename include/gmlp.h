@@ -67,7 +67,15 @@ enum {
      *   ACT_GLU          act(g) = sigmoid(g)                  (GLU)
      * Setting both is GMLP_ERR_FLAGS, and so is a NaN or infinite act_beta with ACT_SWISH. */
     GMLP_FLAG_ACT_SWISH = 1u << 5,
-    GMLP_FLAG_ACT_GLU = 1u << 6
+    GMLP_FLAG_ACT_GLU = 1u << 6,
+    /* The three weight matrices are stored [out, in] (the layout of a linear layer's weight in the common
+     * frameworks): Wg, Wu [d_ff, d_model], Wd [d_model, d_ff], row-major.  The operator is unchanged
+     * (Y = (act(X Wg^T) (.) (X Wu^T)) Wd^T in that storage); the tensor-core kernels read such a matrix as a
+     * K-major operand straight from its TMA tile, so no transposed copy is made and the results are the same
+     * bit for bit as with the [in, out] storage.  gmlp_forward_ex and gmlp_gate_up with the tensor-core
+     * schedules only (GMLP_VARIANT_SIMT / _STREAM: GMLP_ERR_UNSUPPORTED); gmlp_forward_static and the other
+     * operators take [in, out] weights. */
+    GMLP_FLAG_WEIGHTS_OUT_IN = 1u << 7
 };
 
 /* Kernel schedule.  AUTO picks by shape; the others force one schedule (tests, benchmarks). */

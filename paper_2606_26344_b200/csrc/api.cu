@@ -27,8 +27,19 @@ using gmlp::bf16;
 constexpr int kVersion = 100;
 constexpr int kMaxDevices = 64;
 constexpr int64_t kMaxDim = (int64_t)1 << 30;      // per-dimension limit (TMA coordinates are int32)
-constexpr uint32_t kKnownFlags = GMLP_FLAG_RMSNORM | GMLP_FLAG_CHECKED | GMLP_FLAG_ACT_SWISH | GMLP_FLAG_ACT_GLU;
+constexpr uint32_t kKnownFlags = GMLP_FLAG_RMSNORM | GMLP_FLAG_CHECKED | GMLP_FLAG_ACT_SWISH | GMLP_FLAG_ACT_GLU |
+                                 GMLP_FLAG_WEIGHTS_OUT_IN;
 constexpr gmlp::GateAct kSilu = {1.0f, 0};
+// weights of the call in flight are stored [out, in] (set by the entry points around their launches)
+thread_local bool t_w_out_in = false;
+struct WeightLayoutScope {                       // sets the switch for one call, restores it on every exit path
+    bool prev;
+    explicit WeightLayoutScope(bool out_in) : prev(t_w_out_in) { t_w_out_in = out_in; }
+    ~WeightLayoutScope() { t_w_out_in = prev; }
+};
+// tensor map of a weight matrix with `n` output columns and `k` input rows, 64 x 64 boxes either way
+#define GMLP_ENCODE_W(map, ptr, n, k) \
+    (t_w_out_in ? encode_2d(map, ptr, (uint64_t)(k), (uint64_t)(n), 64, 64) : encode_2d(map, ptr, (uint64_t)(n), (uint64_t)(k), 64, 64))
 const gmlp::MultiB kNoMulti = {};
 
 // Gate activation named by the flags (SiLU when none is set); false for a contradictory or non-finite request.
@@ -460,11 +471,12 @@ int pick_umma_boxes(int64_t num_m, int64_t N, int sms) {
 template <bool GATEUP>
 int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
                      int64_t M, int64_t K, int64_t N, cudaStream_t st, gmlp::GateAct act = kSilu) {
+    const int wkm = t_w_out_in ? 1 : 0;
     CUtensorMap tmA, tmB0, tmB1;
     if (!encode_2d(&tmA, A, (uint64_t)K, (uint64_t)M, gmlp::kUmmaBK, 128)) return GMLP_ERR_LAUNCH;
-    if (!encode_2d(&tmB0, W0, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
+    if (!GMLP_ENCODE_W(&tmB0, W0, N, K)) return GMLP_ERR_LAUNCH;
     if (GATEUP) {
-        if (!encode_2d(&tmB1, W1, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
+        if (!GMLP_ENCODE_W(&tmB1, W1, N, K)) return GMLP_ERR_LAUNCH;
     } else {
         tmB1 = tmB0;
     }
@@ -496,7 +508,7 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
     if (cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m,
-                           num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti) != cudaSuccess)
+                           num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm) != cudaSuccess)
         return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -520,6 +532,7 @@ int pick_split_k(int num_m, int64_t K, int64_t N, int sms) {
 
 int launch_umma_splitk(DeviceState* dev, int S, const CUtensorMap& tmA, const CUtensorMap& tmB, bf16* C,
                        int64_t M, int64_t K, int64_t N, int num_m, int a_box_rows, cudaStream_t st) {
+    const int wkm = t_w_out_in ? 1 : 0;
     if (!dev->splitk_attr_set) {
         const int b = (int)gmlp::kSplitSmemBytes;
         if (cudaFuncSetAttribute(gmlp::umma_splitk_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
@@ -545,9 +558,9 @@ int launch_umma_splitk(DeviceState* dev, int S, const CUtensorMap& tmA, const CU
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
     cudaError_t err;
-    if (S == 4) err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<4>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows);
-    else if (S == 3) err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<3>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows);
-    else err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<2>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows);
+    if (S == 4) err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<4>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows, wkm);
+    else if (S == 3) err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<3>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows, wkm);
+    else err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<2>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows, wkm);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -556,6 +569,7 @@ int launch_umma_splitk(DeviceState* dev, int S, const CUtensorMap& tmA, const CU
 template <bool GATEUP>
 int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
                 int64_t M, int64_t K, int64_t N, cudaStream_t st, gmlp::GateAct act = kSilu) {
+    const int wkm = t_w_out_in ? 1 : 0;
     CUtensorMap tmA, tmB0, tmB1;
     // TMA is markedly slower when a box has fewer than 16 rows inside the tensor; with so few rows in all, the
     // box is made exactly M rows high instead (no out-of-range rows to fill)
@@ -563,9 +577,9 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     if (const char* e = getenv("GMLP_UMMA_EXACT_BOX_BELOW")) exact_below = atoi(e);      // tuning override
     const int a_box_rows = (M < exact_below && M < gmlp::kUmmaBM) ? (int)M : gmlp::kUmmaBM;
     if (!encode_2d(&tmA, A, (uint64_t)K, (uint64_t)M, gmlp::kUmmaBK, (uint32_t)a_box_rows)) return GMLP_ERR_LAUNCH;
-    if (!encode_2d(&tmB0, W0, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
+    if (!GMLP_ENCODE_W(&tmB0, W0, N, K)) return GMLP_ERR_LAUNCH;
     if (GATEUP) {
-        if (!encode_2d(&tmB1, W1, (uint64_t)N, (uint64_t)K, 64, gmlp::kUmmaBK)) return GMLP_ERR_LAUNCH;
+        if (!GMLP_ENCODE_W(&tmB1, W1, N, K)) return GMLP_ERR_LAUNCH;
     } else {
         tmB1 = tmB0;
     }
@@ -606,16 +620,16 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     cudaError_t err;
     if (GATEUP && nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm);
     else if (GATEUP)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm);
     else if (nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm);
     else
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -625,12 +639,13 @@ template <bool GATEUP>
 int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf16* W0, const bf16* W1, float* scratch,
                   unsigned int* counters, bf16* out, int64_t M, int64_t K, int64_t N, cudaStream_t st,
                   gmlp::GateAct act = kSilu) {
+    const int wkm = t_w_out_in ? 1 : 0;
     if (p.stages < 2 || p.tmem_cols > 512) return GMLP_ERR_UNSUPPORTED;
     CUtensorMap tmX, tmW0, tmW1;
     if (!encode_2d(&tmX, X, (uint64_t)K, (uint64_t)M, 64, (uint32_t)p.Mpad)) return GMLP_ERR_LAUNCH;
-    if (!encode_2d(&tmW0, W0, (uint64_t)N, (uint64_t)K, 64, 64)) return GMLP_ERR_LAUNCH;
+    if (!GMLP_ENCODE_W(&tmW0, W0, N, K)) return GMLP_ERR_LAUNCH;
     if (GATEUP) {
-        if (!encode_2d(&tmW1, W1, (uint64_t)N, (uint64_t)K, 64, 64)) return GMLP_ERR_LAUNCH;
+        if (!GMLP_ENCODE_W(&tmW1, W1, N, K)) return GMLP_ERR_LAUNCH;
     } else {
         tmW1 = tmW0;
     }
@@ -661,10 +676,10 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
     cudaError_t err;
     if (p.NH == 2)
         err = cudaLaunchKernelEx(&cfg, gmlp::skinny_gemm_kernel<GATEUP, 2>, tmX, tmW0, tmW1, scratch, counters, out,
-                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first, act);
+                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first, act, wkm);
     else
         err = cudaLaunchKernelEx(&cfg, gmlp::skinny_gemm_kernel<GATEUP, 1>, tmX, tmW0, tmW1, scratch, counters, out,
-                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first, act);
+                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first, act, wkm);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -719,6 +734,9 @@ int forward_impl(const gmlp_args* a) {
 
     const int variant = resolve_variant(a->M, a->d_model, a->d_ff, a->variant);
     if (variant == GMLP_VARIANT_SKINNY && a->M > 128) return GMLP_ERR_UNSUPPORTED;
+    const bool w_out_in = (a->flags & GMLP_FLAG_WEIGHTS_OUT_IN) != 0;
+    if (w_out_in && (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM)) return GMLP_ERR_UNSUPPORTED;
+    const WeightLayoutScope layout_scope(w_out_in);
     const Layout L = make_layout(a->M, a->d_model, a->d_ff, a->flags, variant, dev->sm_count);
 
     uint8_t* ws = static_cast<uint8_t*>(a->workspace);
@@ -893,6 +911,7 @@ int gate_up_impl(const gmlp_args* a) {
     const int variant = resolve_variant(a->M, a->d_model, a->d_ff, a->variant);
     if (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM) return GMLP_ERR_UNSUPPORTED;
     if (variant == GMLP_VARIANT_SKINNY && a->M > 128) return GMLP_ERR_UNSUPPORTED;
+    const WeightLayoutScope layout_scope((a->flags & GMLP_FLAG_WEIGHTS_OUT_IN) != 0);
     DeviceState* dev = current_device(&rc);
     if (dev == nullptr) return rc;
     const Layout L = make_layout(a->M, a->d_model, a->d_ff, a->flags, variant, dev->sm_count);
@@ -1030,8 +1049,8 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         const float* rc_ptr = r;
         cudaError_t err = pair
-            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti)
-            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti);
+            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0)
+            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("matmul_rowscale", st);
@@ -1124,9 +1143,9 @@ int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         cudaError_t err = pair
             ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
-                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq, kNoMulti)
+                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq, kNoMulti, 0)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
-                                 num_tiles, (const float*)nullptr, 128, kSilu, R, sumsq, kNoMulti);
+                                 num_tiles, (const float*)nullptr, 128, kSilu, R, sumsq, kNoMulti, 0);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("matmul_add", st);
@@ -1234,10 +1253,10 @@ int qkv_proj_impl(const gmlp_qkv_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->Nq;
         cudaError_t err = pair
             ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, false, true>, tmA, tmB0, tmB1, Q, Mi, Ki, Ni,
-                                 num_m, num_tiles, (const float*)nullptr, kSilu, (const bf16*)nullptr, (float*)nullptr, multi)
+                                 num_m, num_tiles, (const float*)nullptr, kSilu, (const bf16*)nullptr, (float*)nullptr, multi, 0)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, false, true>, tmA, tmB0, tmB1, Q, Mi, Ki, Ni,
                                  num_m, num_tiles, (const float*)nullptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr,
-                                 multi);
+                                 multi, 0);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("qkv", st);

@@ -132,7 +132,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
                  int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, int a_box_rows, GateAct act,
-                 const bf16* residual, float* __restrict__ sumsq, const __grid_constant__ MultiB multi)
+                 const bf16* residual, float* __restrict__ sumsq, const __grid_constant__ MultiB multi,
+                 int w_kmajor)
 {
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
     static_assert(!(ADDSS && (GATEUP || ROWSCALE)), "the residual epilogue is for the plain GEMM");
@@ -143,8 +144,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     constexpr int kStages = umma_stages(NB);
     constexpr uint32_t kStageBytes = kUmmaABytes + NB * kUmmaBoxBBytes;
     // kind::f16 instruction descriptor: D = fp32, A = B = bf16, A K-major, B MN-major, M = 128, N = N_MMA
-    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
-                                ((uint32_t)(N_MMA >> 3) << 17) | ((uint32_t)(kUmmaBM >> 4) << 24);
+    // (bit 16 = B is MN-major: weights stored [K, N]; with w_kmajor they are stored [N, K] and B is K-major like A)
+    const uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | ((w_kmajor ? 0u : 1u) << 16) |
+                            ((uint32_t)(N_MMA >> 3) << 17) | ((uint32_t)(kUmmaBM >> 4) << 24);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
@@ -223,7 +225,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         // gate/up: the first NB/2 boxes are gate columns, the rest the same columns of up
                         const CUtensorMap* map = (GATEUP && i >= NB / 2) ? &tmB1 : plain_map;
                         const int x = GATEUP ? n0 + (i % (NB / 2)) * 64 : n0 + i * 64;
-                        ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
+                        // [K, N] weights: box of 64 columns x 64 k; [N, K] weights: box of 64 k x 64 rows of N
+                        if (w_kmajor) ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, kb * kUmmaBK, x, full);
+                        else ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
                     }
                 }
             }
@@ -253,7 +257,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         // B: MN-major, 64-column chunks 8 KB apart (LBO), 8-row k-groups 1024 B apart (SBO);
                         //    K = 16 is two k-groups: +2048 B per step.
                         const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
-                        const uint64_t b_desc = ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
+                        //    K-major B ([N, K] weights): the boxes stack to N_MMA rows of 128 B, same form as A.
+                        const uint64_t b_desc = w_kmajor ? ptx::make_smem_desc_sw128(b_base + k * 32, 16, 1024)
+                                                         : ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
                         ptx::umma_bf16(d_tmem, a_desc, b_desc, kIdesc, (kb | k) != 0 ? 1u : 0u);
                     }
                     ptx::umma_commit(empty0 + 8 * s);      // stage is free once these MMAs have read it

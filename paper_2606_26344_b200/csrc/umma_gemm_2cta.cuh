@@ -89,7 +89,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                       const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
                       int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, GateAct act,
-                      const bf16* residual, float* __restrict__ sumsq, const __grid_constant__ MultiB multi)
+                      const bf16* residual, float* __restrict__ sumsq, const __grid_constant__ MultiB multi,
+                      int w_kmajor)
 {
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
     static_assert(!(ADDSS && (GATEUP || ROWSCALE)), "the residual epilogue is for the plain GEMM");
@@ -97,8 +98,9 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     constexpr int KERNEL_ID = GATEUP ? 6 : 7;
     constexpr int BN_OUT = GATEUP ? 128 : 256;
     // D = fp32, A = B = bf16, A K-major, B MN-major, M = 256 (128 per CTA), N = 256
-    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
-                                ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+    // (with w_kmajor the weights are stored [N, K] and B is K-major like A: bit 16 clear)
+    const uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | ((w_kmajor ? 0u : 1u) << 16) |
+                            ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
@@ -173,8 +175,13 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     const uint32_t b_dst = a_dst + kPairABytes;
                     ptx::mbar_arrive_expect_tx_cluster(full, kPairStageBytes);
                     ptx::tma_load_2d_pair(a_dst, &tmA, kb * kUmmaBK, m0, full);
-                    ptx::tma_load_2d_pair(b_dst, bmap, bx, kb * kUmmaBK, full);
-                    ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, bx + 64, kb * kUmmaBK, full);
+                    if (w_kmajor) {                        // [N, K] weights: boxes of 64 k x 64 rows of N
+                        ptx::tma_load_2d_pair(b_dst, bmap, kb * kUmmaBK, bx, full);
+                        ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, kb * kUmmaBK, bx + 64, full);
+                    } else {                               // [K, N] weights: boxes of 64 columns x 64 k
+                        ptx::tma_load_2d_pair(b_dst, bmap, bx, kb * kUmmaBK, full);
+                        ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, bx + 64, kb * kUmmaBK, full);
+                    }
                 }
             }
         }
@@ -199,7 +206,8 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 #pragma unroll
                     for (int k = 0; k < kUmmaBK / 16; ++k) {
                         const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
-                        const uint64_t b_desc = ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
+                        const uint64_t b_desc = w_kmajor ? ptx::make_smem_desc_sw128(b_base + k * 32, 16, 1024)
+                                                         : ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
                         ptx::umma_bf16_pair(d_tmem, a_desc, b_desc, kIdesc, (kb | k) != 0 ? 1u : 0u);
                     }
                     ptx::umma_commit_pair(empty0 + 8 * s);

@@ -36,13 +36,14 @@ __device__ __forceinline__ void st_cluster_f32x4(uint32_t cluster_addr, float a,
 template <int S>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                        bf16* __restrict__ C, int M, int K, int N, int num_m_tiles, int a_box_rows)
+                        bf16* __restrict__ C, int M, int K, int N, int num_m_tiles, int a_box_rows, int w_kmajor)
 {
     static_assert(S >= 2 && (S - 1) * kSplitPartialBytes <= kSplitStages * kSplitStageBytes, "staging must fit the ring");
     constexpr int KERNEL_ID = 9;
     // D = fp32, A = B = bf16, A K-major, B MN-major, M = 128, N = 128
-    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
-                                ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    // (with w_kmajor the weights are stored [N, K] and B is K-major like A: bit 16 clear)
+    const uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | ((w_kmajor ? 0u : 1u) << 16) |
+                            ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
@@ -98,8 +99,13 @@ umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 const uint32_t b_dst = a_dst + kUmmaABytes;
                 ptx::mbar_arrive_expect_tx(full, (uint32_t)a_box_rows * 128u + 2 * kUmmaBoxBBytes);
                 ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
-                ptx::tma_load_2d(b_dst, &tmB, n0, kb * kUmmaBK, full);
-                ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, n0 + 64, kb * kUmmaBK, full);
+                if (w_kmajor) {
+                    ptx::tma_load_2d(b_dst, &tmB, kb * kUmmaBK, n0, full);
+                    ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, kb * kUmmaBK, n0 + 64, full);
+                } else {
+                    ptx::tma_load_2d(b_dst, &tmB, n0, kb * kUmmaBK, full);
+                    ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, n0 + 64, kb * kUmmaBK, full);
+                }
             }
         }
         __syncwarp();
@@ -117,7 +123,8 @@ umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 #pragma unroll
                 for (int k = 0; k < kUmmaBK / 16; ++k) {
                     const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
-                    const uint64_t b_desc = ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
+                    const uint64_t b_desc = w_kmajor ? ptx::make_smem_desc_sw128(b_base + k * 32, 16, 1024)
+                                                     : ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
                     ptx::umma_bf16(tmem_base, a_desc, b_desc, kIdesc, (it | k) != 0 ? 1u : 0u);
                 }
                 ptx::umma_commit(empty0 + 8 * s);

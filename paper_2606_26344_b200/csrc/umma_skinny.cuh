@@ -213,7 +213,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                    const __grid_constant__ CUtensorMap tmW1, float* __restrict__ scratch,
                    unsigned int* __restrict__ counters, bf16* __restrict__ out,
                    int M, int Mpad, int N, int num_tiles, int KB, int stages, uint32_t tmem_cols, int evict_first,
-                   GateAct act)
+                   GateAct act, int w_kmajor)
 {
     constexpr int KERNEL_ID = GATEUP ? 3 : 4;
     constexpr int NMAT = GATEUP ? 2 : 1;
@@ -284,12 +284,16 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 for (int j = 0; j < NMAT; ++j)
 #pragma unroll
                     for (int hb = 0; hb < NH * 2; ++hb)
+                    {
+                        // [K, N] weights: box of 64 columns x 64 k at (n, k); [N, K] weights: 64 k x 64 rows at (k, n)
+                        const int n = tile * TILE_N + hb * 64;
+                        const int cx = w_kmajor ? kb * 64 : n, cy = w_kmajor ? n : kb * 64;
                         if (evict_first)
-                            ptx::tma_load_2d_hint(st + (j * NH * 2 + hb) * kSkinnyBoxBytes, j ? &tmW1 : &tmW0,
-                                                  tile * TILE_N + hb * 64, kb * 64, full, policy);
+                            ptx::tma_load_2d_hint(st + (j * NH * 2 + hb) * kSkinnyBoxBytes, j ? &tmW1 : &tmW0, cx, cy, full,
+                                                  policy);
                         else
-                            ptx::tma_load_2d(st + (j * NH * 2 + hb) * kSkinnyBoxBytes, j ? &tmW1 : &tmW0,
-                                             tile * TILE_N + hb * 64, kb * 64, full);
+                            ptx::tma_load_2d(st + (j * NH * 2 + hb) * kSkinnyBoxBytes, j ? &tmW1 : &tmW0, cx, cy, full);
+                    }
             };
             auto load_tokens = [&](long long u, int s) {
                 ptx::tma_load_2d(base + s * stage_bytes + W_BYTES, &tmX, (int)(u % KB) * 64, 0, full0 + 8 * s);
@@ -314,7 +318,8 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             // D = fp32, A = B = bf16, A (weights) MN-major, B (tokens) K-major, M = 128, N = Mpad
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (0u << 16) |
+            // (weights stored [N, K]: A is K-major too, bit 15 clear)
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((w_kmajor ? 0u : 1u) << 15) | (0u << 16) |
                                    ((uint32_t)(Mpad >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
             int it = 0, seg = 0;
             bool fresh = true;
@@ -338,8 +343,10 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     for (int j = 0; j < NMAT; ++j)
 #pragma unroll
                         for (int h = 0; h < NH; ++h) {
-                            const uint64_t a_desc = ptx::make_smem_desc_sw128(
-                                st + (j * NH + h) * 2 * kSkinnyBoxBytes + k * 2048, kSkinnyBoxBytes, 1024);
+                            // weights stored [N, K]: the two boxes stack to 128 rows of 128 B, K-major like the tokens
+                            const uint32_t w_base = st + (j * NH + h) * 2 * kSkinnyBoxBytes;
+                            const uint64_t a_desc = w_kmajor ? ptx::make_smem_desc_sw128(w_base + k * 32, 16, 1024)
+                                                             : ptx::make_smem_desc_sw128(w_base + k * 2048, kSkinnyBoxBytes, 1024);
                             ptx::umma_bf16(tmem_base + acc_col(buf, j, h), a_desc, b_desc, idesc,
                                            (fresh && k == 0) ? 0u : 1u);
                         }

@@ -22,6 +22,7 @@ FLAG_RMSNORM = 1 << 0
 FLAG_CHECKED = 1 << 2
 FLAG_ACT_SWISH = 1 << 5
 FLAG_ACT_GLU = 1 << 6
+FLAG_WEIGHTS_OUT_IN = 1 << 7
 ACT_FLAGS = {"silu": 0, "swish": FLAG_ACT_SWISH, "glu": FLAG_ACT_GLU}
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA, VARIANT_SKINNY, VARIANT_PAIR, VARIANT_TENSOR = 0, 1, 2, 3, 4, 5, 6
 
@@ -198,14 +199,16 @@ def _check_bf16_cuda(t: torch.Tensor, name: str) -> None:
 
 def make_args(X, Wg, Wu, Wd, Y, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, variant: int = VARIANT_AUTO,
               workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
-              checked: bool = False, act: str = "silu", beta: float = 1.0) -> GmlpArgs:
+              checked: bool = False, act: str = "silu", beta: float = 1.0, weights_out_in: bool = False) -> GmlpArgs:
     for t, n in ((X, "X"), (Wg, "Wg"), (Wu, "Wu"), (Wd, "Wd"), (Y, "Y")):
         _check_bf16_cuda(t, n)
     M, d_model = X.shape
-    d_ff = Wg.shape[1]
-    if Wg.shape != (d_model, d_ff) or Wu.shape != (d_model, d_ff) or Wd.shape != (d_ff, d_model) or Y.shape != X.shape:
+    d_ff = Wg.shape[0] if weights_out_in else Wg.shape[1]
+    w_up, w_down = ((d_ff, d_model), (d_model, d_ff)) if weights_out_in else ((d_model, d_ff), (d_ff, d_model))
+    if Wg.shape != w_up or Wu.shape != w_up or Wd.shape != w_down or Y.shape != X.shape:
         raise ValueError("shape mismatch")
-    flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0) | ACT_FLAGS[act]
+    flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0) | ACT_FLAGS[act] | \
+        (FLAG_WEIGHTS_OUT_IN if weights_out_in else 0)
     if gamma is not None:
         _check_bf16_cuda(gamma, "gamma")
     st = stream if stream is not None else torch.cuda.current_stream(X.device)
@@ -239,14 +242,16 @@ def forward_ex(args: GmlpArgs) -> None:
 
 def forward(X, Wg, Wu, Wd, Y=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False,
             variant: int = VARIANT_AUTO, workspace=None, stream=None, checked: bool = False,
-            act: str = "silu", beta: float = 1.0) -> torch.Tensor:
+            act: str = "silu", beta: float = 1.0, weights_out_in: bool = False) -> torch.Tensor:
     """Y = (act(Xn Wg) * (Xn Wu)) Wd on the GPU; asynchronous on ``stream`` (default: torch's current stream).
 
-    ``act``: "silu" (the paper's operator), "swish" (g * sigmoid(beta * g)) or "glu" (sigmoid(g))."""
+    ``act``: "silu" (the paper's operator), "swish" (g * sigmoid(beta * g)) or "glu" (sigmoid(g)).
+    ``weights_out_in``: the weights are stored [out, in] (Wg, Wu [d_ff, d_model], Wd [d_model, d_ff])."""
     if Y is None:
         Y = torch.empty_like(X)
     with torch.cuda.device(X.device):
-        forward_ex(make_args(X, Wg, Wu, Wd, Y, gamma, eps, rmsnorm, variant, workspace, stream, checked, act, beta))
+        forward_ex(make_args(X, Wg, Wu, Wd, Y, gamma, eps, rmsnorm, variant, workspace, stream, checked, act, beta,
+                             weights_out_in))
     return Y
 
 
@@ -285,13 +290,15 @@ def forward_static(X, Wg, Wu, Wd, Y, stream=None) -> None:
 
 
 def gate_up(X, Wg, Wu, H=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, variant: int = VARIANT_AUTO,
-            workspace=None, stream=None, checked: bool = False, act: str = "silu", beta: float = 1.0) -> torch.Tensor:
+            workspace=None, stream=None, checked: bool = False, act: str = "silu", beta: float = 1.0,
+            weights_out_in: bool = False) -> torch.Tensor:
     """gmlp_gate_up: H = bf16(act(Xn Wg) * (Xn Wu)), the gate/up half alone; H is [M, d_ff]."""
     for t, n in ((X, "X"), (Wg, "Wg"), (Wu, "Wu")):
         _check_bf16_cuda(t, n)
     M, d_model = X.shape
-    d_ff = Wg.shape[1]
-    if Wg.shape != (d_model, d_ff) or Wu.shape != (d_model, d_ff):
+    d_ff = Wg.shape[0] if weights_out_in else Wg.shape[1]
+    w_up = (d_ff, d_model) if weights_out_in else (d_model, d_ff)
+    if Wg.shape != w_up or Wu.shape != w_up:
         raise ValueError("shape mismatch")
     if H is None:
         H = torch.empty(M, d_ff, dtype=torch.bfloat16, device=X.device)
@@ -301,7 +308,8 @@ def gate_up(X, Wg, Wu, H=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = Fa
     st = stream if stream is not None else torch.cuda.current_stream(X.device)
     a = GmlpArgs()
     a.struct_bytes = ctypes.sizeof(GmlpArgs)
-    a.flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0) | ACT_FLAGS[act]
+    a.flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0) | ACT_FLAGS[act] | \
+        (FLAG_WEIGHTS_OUT_IN if weights_out_in else 0)
     a.act_beta = beta
     a.X, a.Wg, a.Wu, a.Wd, a.Y = X.data_ptr(), Wg.data_ptr(), Wu.data_ptr(), None, H.data_ptr()
     a.M, a.d_model, a.d_ff = M, d_model, d_ff
