@@ -97,6 +97,8 @@ def _load():
         lib.gmlp_oracle_matmul_rows.restype = ctypes.c_int
         lib.gmlp_oracle_matmul_rows.argtypes = [u16p, u16p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, i64p,
                                                 ctypes.c_int64, f64p, ctypes.c_int]
+        lib.gmlp_oracle_gqa_rows.restype = ctypes.c_int
+        lib.gmlp_oracle_gqa_rows.argtypes = [u16p, u16p, u16p] + [ctypes.c_int64] * 5 + [i64p, ctypes.c_int64, f64p, ctypes.c_int]
         lib.gmlp_oracle_gate_up_rows_act.restype = ctypes.c_int
         lib.gmlp_oracle_gate_up_rows_act.argtypes = lib.gmlp_oracle_gate_up_rows.argtypes + [ctypes.c_int, ctypes.c_double]
         lib.gmlp_oracle_rmsnorm_matmul_rows.restype = ctypes.c_int
@@ -331,6 +333,30 @@ def matmul_rows(X, W, rows=None, num_threads: int = 0) -> np.ndarray:
 def qkv_rows(X, Wq, Wk, Wv, rows=None, num_threads: int = 0):
     """Reference (Q, K, V) = (X @ Wq, X @ Wk, X @ Wv) for the selected rows: the QKV projection."""
     return tuple(matmul_rows(X, W, rows, num_threads) for W in (Wq, Wk, Wv))
+
+
+def gqa_rows(Q, K, V, n_q_heads: int, n_kv_heads: int, rows=None, num_threads: int = 0) -> np.ndarray:
+    """Reference group query attention (float64) for the selected query rows.
+
+    Q [M, Hq*D], K and V [S, Hkv*D] bf16 bit patterns; returns O_ref [len(rows), Hq*D]."""
+    lib = _load()
+    Q, K, V = _u16(Q, "Q"), _u16(K, "K"), _u16(V, "V")
+    M, S = Q.shape[0], K.shape[0]
+    if Q.shape[1] % n_q_heads:
+        raise ValueError("Q width is not a multiple of the head count")
+    D = Q.shape[1] // n_q_heads
+    if K.shape != (S, n_kv_heads * D) or V.shape != K.shape:
+        raise ValueError("shape mismatch")
+    if rows is None:
+        rows = np.arange(M, dtype=np.int64)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    O = np.zeros((rows.size, n_q_heads * D), dtype=np.float64)
+    rc = lib.gmlp_oracle_gqa_rows(_p(Q, ctypes.c_uint16), _p(K, ctypes.c_uint16), _p(V, ctypes.c_uint16), M, S,
+                                  n_q_heads, n_kv_heads, D, _p(rows, ctypes.c_int64), rows.size, _p(O, ctypes.c_double),
+                                  int(num_threads))
+    if rc != 0:
+        raise RuntimeError(f"gmlp_oracle_gqa_rows failed ({rc})")
+    return O
 
 
 def naive_matmul(A, B) -> np.ndarray:

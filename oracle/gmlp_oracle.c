@@ -422,6 +422,71 @@ int gmlp_oracle_matmul_rows(const uint16_t* X, const uint16_t* W, int64_t M, int
     return 0;
 }
 
+/*
+ * Group Query Attention (one of the paper's multi-operator kernels, Section 6.1; the paper names it and gives no
+ * graph).  Reading taken - the standard definition, no mask:
+ *     for query head h (0 <= h < Hq), with key/value head g = h / (Hq / Hkv):
+ *         P = softmax_s( Q_h K_g^T / sqrt(D) ),      O_h = P V_g
+ * Q [M, Hq*D], K and V [S, Hkv*D], O [M, Hq*D] row-major (head h occupies columns [h*D, (h+1)*D)); bf16 bit
+ * patterns in, everything in fp64, softmax written out as max-subtracted exponentials over their sum, O left in
+ * fp64.  For the selected query rows: O_ref [n_rows, Hq*D].
+ */
+int gmlp_oracle_gqa_rows(const uint16_t* Q, const uint16_t* K, const uint16_t* V, int64_t M, int64_t S,
+                         int64_t Hq, int64_t Hkv, int64_t D, const int64_t* rows, int64_t n_rows,
+                         double* O_ref, int num_threads)
+{
+    if (!Q || !K || !V || !rows || !O_ref || M < 0 || S <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || n_rows < 0) return -1;
+    if (Hq % Hkv != 0) return -1;
+    for (int64_t i = 0; i < n_rows; ++i)
+        if (rows[i] < 0 || rows[i] >= M) return -1;
+    const int64_t group = Hq / Hkv;
+    const double scale = 1.0 / sqrt((double)D);
+    int failed = 0;
+#ifdef _OPENMP
+    if (num_threads > 0) omp_set_num_threads(num_threads);
+#else
+    (void)num_threads;
+#endif
+#pragma omp parallel
+    {
+        double* p = (double*)malloc(sizeof(double) * (size_t)S);
+        if (!p) {
+#pragma omp atomic write
+            failed = 1;
+        } else {
+#pragma omp for collapse(2) schedule(dynamic, 1)
+            for (int64_t i = 0; i < n_rows; ++i) {
+                for (int64_t h = 0; h < Hq; ++h) {
+                    const uint16_t* q = Q + rows[i] * Hq * D + h * D;
+                    const int64_t g = h / group;
+                    double mx = -INFINITY;
+                    for (int64_t s = 0; s < S; ++s) {
+                        const uint16_t* k = K + s * Hkv * D + g * D;
+                        double dot = 0.0;
+                        for (int64_t d = 0; d < D; ++d) dot += gmlp_oracle_bf16_to_double(q[d]) * gmlp_oracle_bf16_to_double(k[d]);
+                        p[s] = dot * scale;
+                        if (p[s] > mx) mx = p[s];
+                    }
+                    double sum = 0.0;
+                    for (int64_t s = 0; s < S; ++s) {
+                        p[s] = exp(p[s] - mx);
+                        sum += p[s];
+                    }
+                    double* o = O_ref + i * Hq * D + h * D;
+                    for (int64_t d = 0; d < D; ++d) o[d] = 0.0;
+                    for (int64_t s = 0; s < S; ++s) {
+                        const double w = p[s] / sum;
+                        const uint16_t* v = V + s * Hkv * D + g * D;
+                        for (int64_t d = 0; d < D; ++d) o[d] += w * gmlp_oracle_bf16_to_double(v[d]);
+                    }
+                }
+            }
+        }
+        free(p);
+    }
+    return failed ? -1 : 0;
+}
+
 /* Array forms of the two scalar helpers (plain loops), for the tests. */
 void gmlp_oracle_bf16_rn_array(const double* v, uint16_t* out, int64_t n)
 {
