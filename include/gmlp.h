@@ -220,6 +220,31 @@ typedef struct gmlp_qkv_args {
 int gmlp_qkv_proj(const gmlp_qkv_args* args);
 
 /*
+ * Group Query Attention, forward, no mask - the kernel that follows the QKV projection in the paper's benchmark
+ * list (Section 6.1; the paper names it, the definition below is the standard one):
+ *     for query head h, with key/value head g = h / (n_q_heads / n_kv_heads):
+ *         O_h = softmax( Q_h K_g^T / sqrt(head_dim) ) V_g
+ * Q [M, n_q_heads*head_dim], K and V [S, n_kv_heads*head_dim], O [M, n_q_heads*head_dim], row-major bf16 (head h in
+ * columns [h*head_dim, (h+1)*head_dim) - the layout gmlp_qkv_proj writes); fp32 scores and accumulation, the
+ * probabilities are rounded to bf16 for the second matmul, O is rounded once.  head_dim must be 128
+ * (GMLP_ERR_UNSUPPORTED otherwise); n_q_heads a multiple of n_kv_heads.  One tcgen05 kernel, online softmax, the
+ * scores never leave the SM.  No workspace.
+ */
+typedef struct gmlp_gqa_args {
+    uint32_t struct_bytes;    /* sizeof(gmlp_gqa_args) */
+    uint32_t flags;           /* GMLP_FLAG_CHECKED */
+    const void* Q;            /* device, [M, n_q_heads*head_dim] bf16 */
+    const void* K;            /* device, [S, n_kv_heads*head_dim] bf16 */
+    const void* V;            /* device, [S, n_kv_heads*head_dim] bf16 */
+    void* O;                  /* device, [M, n_q_heads*head_dim] bf16, written */
+    int64_t M, S;             /* query rows, key/value rows */
+    int32_t n_q_heads, n_kv_heads, head_dim;
+    int32_t reserved;         /* must be 0 */
+    void* stream;             /* cudaStream_t */
+} gmlp_gqa_args;
+int gmlp_gqa_attention(const gmlp_gqa_args* args);
+
+/*
  * The same call for a caller whose activations live in HOST memory: copies X_host
  * (M*d_model bf16, ideally pinned) to args->X, runs gmlp_forward_ex, and copies args->Y
  * to Y_host, all asynchronously on args->stream.  args->X and args->Y are device staging

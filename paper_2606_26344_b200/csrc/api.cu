@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <atomic>
@@ -19,6 +20,7 @@
 #include "umma_gemm_2cta.cuh"
 #include "umma_gemm_splitk.cuh"
 #include "umma_skinny.cuh"
+#include "gqa_attention.cuh"
 
 namespace {
 
@@ -107,6 +109,7 @@ struct DeviceState {
     bool splitk_attr_set = false;
     bool addss_attr_set = false;
     bool multi_attr_set = false;
+    bool gqa_attr_set = false;
     bool umma_attr_set = false;
     bool pair_attr_set = false;
     bool rowscale_attr_set = false;
@@ -1270,6 +1273,60 @@ int qkv_proj_impl(const gmlp_qkv_args* a) {
     return GMLP_OK;
 }
 
+// Group Query Attention forward (Section 6.1), no mask, head dimension 128.
+int gqa_attention_impl(const gmlp_gqa_args* a) {
+    if (a == nullptr) return GMLP_ERR_NULL;
+    if (a->struct_bytes != sizeof(gmlp_gqa_args)) return GMLP_ERR_FLAGS;
+    if ((a->flags & ~(uint32_t)GMLP_FLAG_CHECKED) || a->reserved != 0) return GMLP_ERR_FLAGS;
+    if (a->M < 0 || a->S <= 0 || a->n_q_heads <= 0 || a->n_kv_heads <= 0 || a->n_q_heads % a->n_kv_heads != 0 ||
+        a->M > (1 << 30) || a->S > (1 << 30) || a->n_q_heads > 65535)
+        return GMLP_ERR_SHAPE;
+    if (a->head_dim != gmlp::kGqaD) return GMLP_ERR_UNSUPPORTED;
+    if (a->M == 0) return GMLP_OK;
+    if (!a->Q || !a->K || !a->V || !a->O) return GMLP_ERR_NULL;
+    if (!aligned16(a->Q) || !aligned16(a->K) || !aligned16(a->V) || !aligned16(a->O)) return GMLP_ERR_ALIGN;
+    int rc = GMLP_OK;
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(a->stream);
+    const uint64_t qw = (uint64_t)a->n_q_heads * gmlp::kGqaD, kvw = (uint64_t)a->n_kv_heads * gmlp::kGqaD;
+    CUtensorMap tmQ, tmK, tmV;
+    if (!encode_2d(&tmQ, a->Q, qw, (uint64_t)a->M, 64, 128) || !encode_2d(&tmK, a->K, kvw, (uint64_t)a->S, 64, 128) ||
+        !encode_2d(&tmV, a->V, kvw, (uint64_t)a->S, 64, 64))
+        return GMLP_ERR_LAUNCH;
+    if (!dev->gqa_attr_set) {
+        if (cudaFuncSetAttribute(gmlp::gqa_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)gmlp::kGqaSmemBytes) != cudaSuccess)
+            return GMLP_ERR_LAUNCH;
+        dev->gqa_attr_set = true;
+    }
+    prof_begin(st);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((a->M + gmlp::kGqaBM - 1) / gmlp::kGqaBM), (unsigned)a->n_q_heads);
+    cfg.blockDim = dim3(gmlp::kUmmaThreads);
+    cfg.dynamicSmemBytes = gmlp::kGqaSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int Mi = (int)a->M, Si = (int)a->S, Hq = (int)a->n_q_heads, group = (int)(a->n_q_heads / a->n_kv_heads);
+    const float scale_log2 = 1.4426950408889634f / sqrtf((float)gmlp::kGqaD);      // log2(e) / sqrt(D)
+    bf16* O = static_cast<bf16*>(a->O);
+    if (cudaLaunchKernelEx(&cfg, gmlp::gqa_attention_kernel, tmQ, tmK, tmV, O, Mi, Si, Hq, group, scale_log2) != cudaSuccess)
+        return GMLP_ERR_LAUNCH;
+    GMLP_CHECK_LAUNCH();
+    prof_mark("gqa", st);
+    if (a->flags & GMLP_FLAG_CHECKED) {
+        if (cudaStreamSynchronize(st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+        const int s = read_device_status();
+        if (s < 0) return s;
+        if (s != 0) return GMLP_ERR_TIMEOUT;
+    }
+    return GMLP_OK;
+}
+
 // Empirical schedule selection for one shape: time every tensor-core schedule that can run it, keep the fastest.
 int autotune_impl(const gmlp_args* a, int iters, int32_t* best_variant, float* best_us) {
     if (a == nullptr) return GMLP_ERR_NULL;
@@ -1369,6 +1426,14 @@ int autotune_impl(const gmlp_args* a, int iters, int32_t* best_variant, float* b
 }  // namespace
 
 extern "C" {
+
+int gmlp_gqa_attention(const gmlp_gqa_args* args) {
+    try {
+        return gqa_attention_impl(args);
+    } catch (...) {
+        return GMLP_ERR_LAUNCH;
+    }
+}
 
 int gmlp_qkv_proj(const gmlp_qkv_args* args) {
     try {

@@ -57,6 +57,16 @@ MMADDNORM_UNFUSED = 1 << 4
 QKV_SEPARATE = 1 << 4
 
 
+class GmlpGqaArgs(ctypes.Structure):
+    _fields_ = [
+        ("struct_bytes", ctypes.c_uint32), ("flags", ctypes.c_uint32),
+        ("Q", ctypes.c_void_p), ("K", ctypes.c_void_p), ("V", ctypes.c_void_p), ("O", ctypes.c_void_p),
+        ("M", ctypes.c_int64), ("S", ctypes.c_int64),
+        ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+        ("reserved", ctypes.c_int32), ("stream", ctypes.c_void_p),
+    ]
+
+
 class GmlpQkvArgs(ctypes.Structure):
     _fields_ = [
         ("struct_bytes", ctypes.c_uint32), ("flags", ctypes.c_uint32),
@@ -109,6 +119,8 @@ def lib() -> ctypes.CDLL:
         L.gmlp_workspace_bytes.argtypes = [i64, i64, i64, u32, i32]
         L.gmlp_matmul_add_rmsnorm.restype = ctypes.c_int
         L.gmlp_matmul_add_rmsnorm.argtypes = [ctypes.POINTER(GmlpMmAddNormArgs)]
+        L.gmlp_gqa_attention.restype = ctypes.c_int
+        L.gmlp_gqa_attention.argtypes = [ctypes.POINTER(GmlpGqaArgs)]
         L.gmlp_qkv_proj.restype = ctypes.c_int
         L.gmlp_qkv_proj.argtypes = [ctypes.POINTER(GmlpQkvArgs)]
         L.gmlp_autotune.restype = ctypes.c_int
@@ -464,3 +476,36 @@ def qkv_proj(X, Wq, Wk, Wv, separate: bool = False, stream=None, checked: bool =
     with torch.cuda.device(X.device):
         qkv_proj_ex(make_qkv_args(X, Wq, Wk, Wv, Q, K, V, separate, stream, checked))
     return Q, K, V
+
+
+def make_gqa_args(Q, K, V, O, n_q_heads: int, n_kv_heads: int, stream=None, checked: bool = False) -> GmlpGqaArgs:
+    for t, n in ((Q, "Q"), (K, "K"), (V, "V"), (O, "O")):
+        _check_bf16_cuda(t, n)
+    M, S = Q.shape[0], K.shape[0]
+    D = Q.shape[1] // n_q_heads
+    if Q.shape[1] != n_q_heads * D or K.shape != (S, n_kv_heads * D) or V.shape != K.shape or O.shape != Q.shape:
+        raise ValueError("shape mismatch")
+    st = stream if stream is not None else torch.cuda.current_stream(Q.device)
+    a = GmlpGqaArgs()
+    a.struct_bytes = ctypes.sizeof(GmlpGqaArgs)
+    a.flags = FLAG_CHECKED if checked else 0
+    a.Q, a.K, a.V, a.O = Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr()
+    a.M, a.S = M, S
+    a.n_q_heads, a.n_kv_heads, a.head_dim, a.reserved = n_q_heads, n_kv_heads, D, 0
+    a.stream = st.cuda_stream
+    return a
+
+
+def gqa_attention_ex(args: GmlpGqaArgs) -> None:
+    rc = lib().gmlp_gqa_attention(ctypes.byref(args))
+    if rc != OK:
+        raise GmlpError(rc)
+
+
+def gqa_attention(Q, K, V, n_q_heads: int, n_kv_heads: int, O=None, stream=None, checked: bool = False) -> torch.Tensor:
+    """gmlp_gqa_attention: O_h = softmax(Q_h K_g^T / sqrt(D)) V_g, no mask, D = 128."""
+    if O is None:
+        O = torch.empty_like(Q)
+    with torch.cuda.device(Q.device):
+        gqa_attention_ex(make_gqa_args(Q, K, V, O, n_q_heads, n_kv_heads, stream, checked))
+    return O

@@ -1,0 +1,97 @@
+"""GPU parity of gmlp_gqa_attention (Group Query Attention, Section 6.1) against the CPU oracle:
+|o - o_ref| <= 2e-2 * max(1, |o_ref|), ragged M and S, several group sizes, and closed-form cases."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2606_26344_b200 import gmlp
+
+pytestmark = pytest.mark.gpu
+D = 128
+
+
+def _bits(t):
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def _case(M, S, Hq, Hkv, seed, q_scale=1.0):
+    g = torch.Generator().manual_seed(seed)
+    Q = (torch.randn(M, Hq * D, generator=g) * q_scale).to(torch.bfloat16)
+    K = torch.randn(S, Hkv * D, generator=g).to(torch.bfloat16)
+    V = torch.randn(S, Hkv * D, generator=g).to(torch.bfloat16)
+    return Q, K, V
+
+
+def _check(M, S, Hq, Hkv, seed, q_scale=1.0, max_rows=64):
+    Q, K, V = _case(M, S, Hq, Hkv, seed, q_scale)
+    dev = torch.device("cuda")
+    O = torch.full((M, Hq * D), float("nan"), dtype=torch.bfloat16, device=dev)
+    gmlp.gqa_attention(Q.to(dev), K.to(dev), V.to(dev), Hq, Hkv, O=O, checked=True)
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(O.float()).all())
+    rows = np.arange(M) if M <= max_rows else np.sort(np.random.default_rng(seed).choice(M, max_rows, replace=False))
+    ref = oracle.gqa_rows(_bits(Q), _bits(K), _bits(V), Hq, Hkv, rows=rows)
+    got = O[torch.as_tensor(rows, device=dev)].float().cpu().numpy().astype(np.float64)
+    e = np.abs(got - ref) / oracle.tolerance(ref)
+    assert e.max() <= 1.0, f"max err/tol {e.max():.3f}"
+    return e.max()
+
+
+@pytest.mark.parametrize("shape", [(128, 128, 2, 1), (1, 1, 1, 1), (1, 300, 4, 4), (17, 200, 4, 2), (300, 129, 8, 2),
+                                   (129, 1000, 6, 3), (256, 1024, 4, 1), (1030, 64, 2, 2)])
+def test_small_and_ragged(shape):
+    _check(*shape, seed=50 + shape[0])
+
+
+def test_peaked_softmax_and_large_scores():
+    # queries scaled up: scores of +-100 and a softmax concentrated on a few keys (the running maximum moves a lot)
+    _check(200, 700, 4, 2, seed=7, q_scale=6.0)
+
+
+def test_llama_like_block():
+    # 8B attention block: 32 query heads, 8 key/value heads of 128; 2048 tokens; 64 sampled query rows
+    _check(2048, 2048, 32, 8, seed=3)
+
+
+def test_closed_forms_on_device():
+    dev = torch.device("cuda")
+    Q, K, V = _case(70, 333, 4, 2, 9)
+    # zero queries: every output row is the mean of its group's values
+    O = gmlp.gqa_attention(torch.zeros_like(Q).to(dev), K.to(dev), V.to(dev), 4, 2, checked=True).float().cpu()
+    vm = V.float().view(333, 2, D).mean(dim=0).repeat_interleave(2, dim=0).reshape(1, 4 * D)
+    assert bool(((O - vm).abs() <= 2e-2).all())
+    # a single key: the output is that key's value exactly (P = 1, one rounding of a bf16 value)
+    O1 = gmlp.gqa_attention(Q.to(dev), K[:1].to(dev), V[:1].to(dev), 4, 2, checked=True).cpu()
+    want = V[:1].view(1, 2, D).repeat_interleave(2, dim=1).reshape(1, 4 * D).expand(70, 4 * D)
+    assert torch.equal(O1.view(torch.int16), want.contiguous().view(torch.int16))
+    # deterministic
+    a = gmlp.gqa_attention(Q.to(dev), K.to(dev), V.to(dev), 4, 2, checked=True)
+    b = gmlp.gqa_attention(Q.to(dev), K.to(dev), V.to(dev), 4, 2, checked=True)
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+def test_argument_checks():
+    dev = torch.device("cuda")
+    Q, K, V = _case(40, 50, 4, 2, 2)
+    Qd, Kd, Vd = Q.to(dev), K.to(dev), V.to(dev)
+    O = torch.empty_like(Qd)
+    a = gmlp.make_gqa_args(Qd, Kd, Vd, O, 4, 2)
+    f = lambda: gmlp.lib().gmlp_gqa_attention(ctypes.byref(a))
+    assert f() == gmlp.OK
+    a.head_dim = 64
+    assert f() == gmlp.ERR_UNSUPPORTED
+    a.head_dim = 128
+    a.n_kv_heads = 3
+    assert f() == gmlp.ERR_SHAPE
+    a.n_kv_heads = 2
+    a.flags = 1 << 9
+    assert f() == gmlp.ERR_FLAGS
+    a.flags = 0
+    a.V = None
+    assert f() == gmlp.ERR_NULL
+    assert gmlp.lib().gmlp_gqa_attention(None) == gmlp.ERR_NULL
+    torch.cuda.synchronize()
+    assert gmlp.device_status() == 0
