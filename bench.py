@@ -446,6 +446,37 @@ def measure_qkv(dev, iters=10):
             "best_fused_tflops": max(r["fused_tflops"] for r in rows), "table": rows}
 
 
+def measure_gqa(dev, peaks, iters=10):
+    """Group Query Attention forward (no mask, head dimension 128) on grouped-query blocks; 4*M*S*D*Hq flops."""
+    import torch
+    from paper_2606_26344_b200 import gmlp
+    g = torch.Generator(device="cpu").manual_seed(0)
+    rows = []
+    for (Hq, Hkv, label) in ((32, 8, "8B attention block"), (64, 8, "70B attention block")):
+        for T in (512, 2048, 4096, 8192):
+            Q = torch.randn(T, Hq * 128, generator=g).bfloat16().to(dev)
+            K = torch.randn(T, Hkv * 128, generator=g).bfloat16().to(dev)
+            V = torch.randn(T, Hkv * 128, generator=g).bfloat16().to(dev)
+            O = torch.empty_like(Q)
+            a = gmlp.make_gqa_args(Q, K, V, O, Hq, Hkv)
+            for _ in range(3):
+                gmlp.gqa_attention_ex(a)
+            torch.cuda.synchronize(dev)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(iters):
+                gmlp.gqa_attention_ex(a)
+            e1.record()
+            torch.cuda.synchronize(dev)
+            us = e0.elapsed_time(e1) / iters * 1e3
+            tf = 4.0 * T * T * 128 * Hq / us / 1e6
+            rows.append({"shape": label, "M": T, "S": T, "n_q_heads": Hq, "n_kv_heads": Hkv, "us": us, "tflops": tf,
+                         "frac_of_bf16_peak": tf / peaks["bf16_tflops"]})
+            del Q, K, V, O
+    return {"timing": "back-to-back calls", "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst bf16)",
+            "best_tflops": max(r["tflops"] for r in rows), "table": rows}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -454,8 +485,8 @@ def main():
     ap.add_argument("--impl", default="gmlp", choices=["gmlp", "reference"])
     ap.add_argument("--workload", default=PRIMARY)
     ap.add_argument("--no-extra", action="store_true", help="time only the primary workload")
-    ap.add_argument("--op", default="gmlp", choices=["gmlp", "rmsnorm_matmul", "matmul_add_rmsnorm", "qkv"],
-                    help="rmsnorm_matmul / matmul_add_rmsnorm / qkv: print only that operator's sweep "
+    ap.add_argument("--op", default="gmlp", choices=["gmlp", "rmsnorm_matmul", "matmul_add_rmsnorm", "qkv", "gqa"],
+                    help="rmsnorm_matmul / matmul_add_rmsnorm / qkv / gqa: print only that operator's sweep "
                          "(one JSON line) and exit")
     ap.add_argument("--autotune", action="store_true",
                     help="run gmlp_autotune on each workload's shape before timing it (default: the built-in rule)")
@@ -495,7 +526,7 @@ def main():
     if args.op != "gmlp":
         if rank == 0:
             fn = {"rmsnorm_matmul": measure_rmsnorm_matmul, "matmul_add_rmsnorm": measure_matmul_add_rmsnorm,
-                  "qkv": measure_qkv}[args.op]
+                  "qkv": measure_qkv, "gqa": lambda d: measure_gqa(d, peaks)}[args.op]
             print(json.dumps({"op": args.op, **fn(dev)}))
         if dist is not None:
             dist.barrier()

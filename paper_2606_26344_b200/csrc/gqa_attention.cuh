@@ -5,11 +5,16 @@
 // leave the SM: both matmuls run on tcgen05 with their accumulators in TMEM and the probabilities go from
 // registers to shared memory as the second matmul's A operand.
 //
-//   warp 0      TMA producer: Q tile once, then (K block, V block) into a two-stage ring
-//   warp 1      MMA issuer:   S = Q K^T (TMEM columns [0,128)), then O += P V (TMEM columns [128,256))
+//   warp 0      TMA producer: Q tile once, then K blocks and V blocks into two two-stage rings of their own
+//   warp 1      MMA issuer:   S = Q K^T into one of two TMEM score buffers (columns [0,128) / [128,256)), so the
+//                             scores of block j+1 are computed while block j is in the softmax; then
+//                             O += P V (TMEM columns [256,384))
 //   warps 2..5  softmax:      thread t owns query row t (its TMEM lane), so row maxima and sums need no shuffles;
-//                             reads S, rescales O in TMEM when the maximum moves, writes P (bf16) into the
-//                             128-byte-swizzled K-major layout the MMA expects, and at the end stores O / l
+//                             reads its 128 scores once into registers, writes P (bf16) into the
+//                             128-byte-swizzled K-major layout the MMA expects, and at the end stores O / l.
+//                             The exponent base is a running maximum that is only moved when a block's maximum
+//                             exceeds it by more than 8 (probabilities stay below 2^8), so O in TMEM is rescaled
+//                             rarely instead of once per block.
 //
 // Operand forms: Q and P are K-major A operands (rows of 128 B, two 64-wide swizzle atoms side by side); a K block
 // [128 keys, D] is a K-major B operand (keys are the N dimension); a V block [128 keys, D] is an MN-major B
@@ -28,9 +33,9 @@ constexpr int kGqaD = 128;                       // head dimension
 constexpr int kGqaBM = 128;                      // query rows per CTA
 constexpr int kGqaBS = 128;                      // keys per block
 constexpr uint32_t kGqaTileBytes = 128 * 128 * 2;                         // one 128 x 128 bf16 tile: 32 KB
-constexpr uint32_t kGqaStageBytes = 2 * kGqaTileBytes;                    // K block + V block
-constexpr int kGqaStages = 2;
-constexpr uint32_t kGqaSmemBytes = 2 * kGqaTileBytes + kGqaStages * kGqaStageBytes + 1024 + 256;   // Q, P, ring
+constexpr int kGqaStages = 2;                                             // per ring (K blocks, V blocks)
+constexpr uint32_t kGqaSmemBytes = (2 + 2 * kGqaStages) * kGqaTileBytes + 1024 + 256;   // Q, P, K ring, V ring
+constexpr float kGqaLazyLog2 = 8.0f;                                      // move the exponent base only beyond this
 
 __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
     asm volatile(
@@ -66,16 +71,19 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - raw_addr);
-    const uint32_t q_smem = base, p_smem = base + kGqaTileBytes, ring = base + 2 * kGqaTileBytes;
+    const uint32_t q_smem = base, p_smem = base + kGqaTileBytes;
+    const uint32_t k_ring = base + 2 * kGqaTileBytes, v_ring = k_ring + kGqaStages * kGqaTileBytes;
     uint8_t* p_ptr = base_ptr + kGqaTileBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + 2 * kGqaTileBytes + kGqaStages * kGqaStageBytes);
-    const uint32_t kv_full0 = ptx::smem_addr(bars);                  // [2]
-    const uint32_t kv_empty0 = ptx::smem_addr(bars + 2);             // [2]
-    const uint32_t q_full = ptx::smem_addr(bars + 4);
-    const uint32_t s_full = ptx::smem_addr(bars + 5);                // the scores of a block are in TMEM
-    const uint32_t p_full = ptx::smem_addr(bars + 6);                // P is in shared memory and O has been rescaled
-    const uint32_t o_full = ptx::smem_addr(bars + 7);                // O += P V of a block is done
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + (2 + 2 * kGqaStages) * kGqaTileBytes);
+    const uint32_t k_full0 = ptx::smem_addr(bars);                   // [2]
+    const uint32_t k_empty0 = ptx::smem_addr(bars + 2);              // [2]
+    const uint32_t v_full0 = ptx::smem_addr(bars + 4);               // [2]
+    const uint32_t v_empty0 = ptx::smem_addr(bars + 6);              // [2]
+    const uint32_t s_full0 = ptx::smem_addr(bars + 8);               // [2] the scores of a block are in TMEM buffer b
+    const uint32_t q_full = ptx::smem_addr(bars + 10);
+    const uint32_t p_full = ptx::smem_addr(bars + 11);               // P is in shared memory (and O rescaled if need be)
+    const uint32_t o_full = ptx::smem_addr(bars + 12);               // O += P V of a block is done
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -86,12 +94,8 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     ptx::launch_dependents();
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kGqaStages; ++i) {
-            ptx::mbar_init(kv_full0 + 8 * i, 1);
-            ptx::mbar_init(kv_empty0 + 8 * i, 1);
-        }
+        for (int i = 0; i < 10; ++i) ptx::mbar_init(k_full0 + 8 * i, 1);      // the five two-entry barrier arrays
         ptx::mbar_init(q_full, 1);
-        ptx::mbar_init(s_full, 1);
         ptx::mbar_init(p_full, 4);                                   // one arrival per softmax warp
         ptx::mbar_init(o_full, 1);
         *abort_flag = 0;
@@ -102,14 +106,14 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         ptx::prefetch_tensormap(&tmV);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_addr(tmem_slot), 256);
+        ptx::tmem_alloc(ptx::smem_addr(tmem_slot), 512);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 128;
+    const uint32_t tmem_o = tmem_base + 256;                         // scores: tmem_base + 128 * (block & 1)
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -121,44 +125,57 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             for (int j = 0; j < n_blocks; ++j) {
                 const int s = j % kGqaStages;
                 const uint32_t ph = (uint32_t)(j / kGqaStages) & 1u;
-                if (!wait_bounded(kv_empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
-                const uint32_t full = kv_full0 + 8 * s;
-                const uint32_t k_dst = ring + s * kGqaStageBytes, v_dst = k_dst + kGqaTileBytes;
                 const int s0 = j * kGqaBS;
-                ptx::mbar_arrive_expect_tx(full, kGqaStageBytes);
                 // K block: two boxes of 64 d x 128 keys (K-major: a key's d values are contiguous)
-                ptx::tma_load_2d(k_dst, &tmK, g * kGqaD, s0, full);
-                ptx::tma_load_2d(k_dst + 16384, &tmK, g * kGqaD + 64, s0, full);
+                if (!wait_bounded(k_empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
+                const uint32_t k_dst = k_ring + s * kGqaTileBytes;
+                ptx::mbar_arrive_expect_tx(k_full0 + 8 * s, kGqaTileBytes);
+                ptx::tma_load_2d(k_dst, &tmK, g * kGqaD, s0, k_full0 + 8 * s);
+                ptx::tma_load_2d(k_dst + 16384, &tmK, g * kGqaD + 64, s0, k_full0 + 8 * s);
                 // V block: four boxes of 64 d x 64 keys; (key half, d half) at (2 * key half + d half) * 8 KB
+                if (!wait_bounded(v_empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 8)) break;
+                const uint32_t v_dst = v_ring + s * kGqaTileBytes;
+                ptx::mbar_arrive_expect_tx(v_full0 + 8 * s, kGqaTileBytes);
 #pragma unroll
                 for (int sh = 0; sh < 2; ++sh)
 #pragma unroll
                     for (int nh = 0; nh < 2; ++nh)
-                        ptx::tma_load_2d(v_dst + (sh * 2 + nh) * 8192, &tmV, g * kGqaD + nh * 64, s0 + sh * 64, full);
+                        ptx::tma_load_2d(v_dst + (sh * 2 + nh) * 8192, &tmV, g * kGqaD + nh * 64, s0 + sh * 64,
+                                         v_full0 + 8 * s);
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            bool ok = wait_bounded(q_full, 0u, abort_flag, KERNEL_ID, 5);
-            for (int j = 0; j < n_blocks && ok; ++j) {
+            // S(j) = Q K(j)^T over D = 128: eight K = 16 steps, four per 64-wide swizzle atom
+            auto issue_scores = [&](int j) -> bool {
                 const int s = j % kGqaStages;
-                const uint32_t ph = (uint32_t)(j / kGqaStages) & 1u;
-                if (!wait_bounded(kv_full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) break;
+                if (!wait_bounded(k_full0 + 8 * s, (uint32_t)(j / kGqaStages) & 1u, abort_flag, KERNEL_ID, 2)) return false;
                 ptx::tc_fence_after_sync();
-                const uint32_t k_smem = ring + s * kGqaStageBytes, v_smem = k_smem + kGqaTileBytes;
-                // S = Q K^T over D = 128: eight K = 16 steps, four per 64-wide swizzle atom
+                const uint32_t k_smem = k_ring + s * kGqaTileBytes;
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     const uint32_t off = (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u;
-                    ptx::umma_bf16(tmem_s, ptx::make_smem_desc_sw128(q_smem + off, 16, 1024),
+                    ptx::umma_bf16(tmem_base + 128u * (uint32_t)(j & 1), ptx::make_smem_desc_sw128(q_smem + off, 16, 1024),
                                    ptx::make_smem_desc_sw128(k_smem + off, 16, 1024), kIdescQK, k != 0 ? 1u : 0u);
                 }
-                ptx::umma_commit(s_full);
-                // the softmax warps turn S into P (and rescale O); then O += P V over the block's 128 keys
+                ptx::umma_commit(s_full0 + 8 * (j & 1));
+                ptx::umma_commit(k_empty0 + 8 * s);
+                return true;
+            };
+            bool ok = wait_bounded(q_full, 0u, abort_flag, KERNEL_ID, 5);
+            ok = ok && issue_scores(0);
+            for (int j = 0; j < n_blocks && ok; ++j) {
+                // the scores of the next block are computed while this block is in the softmax: its score buffer
+                // was last read for block j-1, whose probabilities the wait below (one iteration ago) has seen
+                if (j + 1 < n_blocks && !issue_scores(j + 1)) break;
+                const int s = j % kGqaStages;
                 if (!wait_bounded(p_full, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 6)) break;
+                if (!wait_bounded(v_full0 + 8 * s, (uint32_t)(j / kGqaStages) & 1u, abort_flag, KERNEL_ID, 9)) break;
                 ptx::tc_fence_after_sync();
+                const uint32_t v_smem = v_ring + s * kGqaTileBytes;
+                // O += P V over the block's 128 keys
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     const uint64_t a_desc = ptx::make_smem_desc_sw128(
@@ -167,7 +184,7 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         v_smem + (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 2048u, 8192, 1024);
                     ptx::umma_bf16(tmem_o, a_desc, b_desc, kIdescPV, (j | k) != 0 ? 1u : 0u);
                 }
-                ptx::umma_commit(kv_empty0 + 8 * s);
+                ptx::umma_commit(v_empty0 + 8 * s);
                 ptx::umma_commit(o_full);
             }
         }
@@ -177,29 +194,36 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         const int q = warp & 3;
         const int r = q * 32 + lane;                                 // row within the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-        float m_run = -INFINITY, l_run = 0.0f;
+        float m_use = 0.0f, l_run = 0.0f;                            // exponent base (set on the first block), row sum
         bool ok = true;
         for (int j = 0; j < n_blocks && ok; ++j) {
-            if (!wait_bounded(s_full, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 3)) { ok = false; break; }
+            if (!wait_bounded(s_full0 + 8 * (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag, KERNEL_ID, 3)) { ok = false; break; }
             ptx::tc_fence_after_sync();
             const int valid = min(kGqaBS, S - j * kGqaBS);           // keys of this block that exist
-            // pass 1: row maximum of the scaled scores
+            const uint32_t s_addr = tmem_base + 128u * (uint32_t)(j & 1) + lane_addr;
+            uint32_t sv[4][32];                                      // this row's 128 scores
+#pragma unroll
+            for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(s_addr + 32 * c, sv[c]);
+            ptx::tmem_ld_wait();
             float m_blk = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < kGqaBS; c += 32) {
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(tmem_s + lane_addr + c, v);
-                ptx::tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
-                    if (c + i < valid) m_blk = fmaxf(m_blk, __uint_as_float(v[i]) * scale_log2);
-            }
-            const float m_new = fmaxf(m_run, m_blk);
-            const float alpha = ex2_approx(m_run - m_new);           // 0 on the first block (m_run = -inf)
-            // O += P V of the previous block must be complete before O is rescaled and P overwritten
+                    if (32 * c + i < valid) m_blk = fmaxf(m_blk, __uint_as_float(sv[c][i]) * scale_log2);
+            // P of the previous block must have been consumed (and O complete) before P is overwritten
             if (j > 0) {
                 if (!wait_bounded(o_full, (uint32_t)(j - 1) & 1u, abort_flag, KERNEL_ID, 4)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
+            }
+            if (j == 0) {
+                m_use = m_blk;                                       // finite: the first block has at least one key
+            } else if (__any_sync(0xFFFFFFFFu, m_blk > m_use + kGqaLazyLog2)) {
+                // some row's maximum moved far: rescale this warp's rows of O (and l) to the new base
+                const float m_new = fmaxf(m_use, m_blk);
+                const float alpha = ex2_approx(m_use - m_new);
+                m_use = m_new;
+                l_run *= alpha;
 #pragma unroll 1
                 for (int c = 0; c < kGqaD; c += 32) {
                     uint32_t v[32];
@@ -211,32 +235,28 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 }
                 tmem_st_wait();
             }
-            // pass 2: p = 2^(x - m_new), row sum, P as bf16 into the swizzled K-major tile
+            // p = 2^(x - base), row sum, P as bf16 into the swizzled K-major tile
             float l_blk = 0.0f;
-#pragma unroll 1
-            for (int c = 0; c < kGqaBS; c += 32) {
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(tmem_s + lane_addr + c, v);
-                ptx::tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
                 uint32_t packed[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const float p0 = (c + 2 * i < valid) ? ex2_approx(__uint_as_float(v[2 * i]) * scale_log2 - m_new) : 0.0f;
-                    const float p1 = (c + 2 * i + 1 < valid) ? ex2_approx(__uint_as_float(v[2 * i + 1]) * scale_log2 - m_new) : 0.0f;
+                    const float p0 = (32 * c + 2 * i < valid) ? ex2_approx(__uint_as_float(sv[c][2 * i]) * scale_log2 - m_use) : 0.0f;
+                    const float p1 = (32 * c + 2 * i + 1 < valid) ? ex2_approx(__uint_as_float(sv[c][2 * i + 1]) * scale_log2 - m_use) : 0.0f;
                     l_blk += p0 + p1;
                     packed[i] = pack_bf16x2(p0, p1);
                 }
-                // columns c .. c+31 of row r: four 16-byte chunks of the 64-wide atom (c / 64)
-                uint8_t* atom = p_ptr + (size_t)(c >> 6) * 16384 + (size_t)r * 128;
+                // columns 32c .. 32c+31 of row r: four 16-byte chunks of the 64-wide atom (c / 2)
+                uint8_t* atom = p_ptr + (size_t)(c >> 1) * 16384 + (size_t)r * 128;
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
-                    const int chunk = ((c & 63) >> 3) + ch;                          // 0..7 within the 128-byte row
+                    const int chunk = (c & 1) * 4 + ch;                              // 0..7 within the 128-byte row
                     *reinterpret_cast<uint4*>(atom + ((chunk ^ (r & 7)) << 4)) =
                         make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
                 }
             }
-            m_run = m_new;
-            l_run = l_run * alpha + l_blk;
+            l_run += l_blk;
             ptx::fence_proxy_async_smem();                           // P (generic writes) -> visible to the MMA
             ptx::tc_fence_before_sync();
             __syncwarp();
@@ -274,7 +294,7 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, 256);
+        ptx::tmem_dealloc(tmem_base, 512);
     }
 }
 
