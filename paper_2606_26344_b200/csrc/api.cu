@@ -1303,7 +1303,7 @@ int gqa_attention_impl(const gmlp_gqa_args* a) {
     prof_begin(st);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)((a->M + gmlp::kGqaBM - 1) / gmlp::kGqaBM), (unsigned)a->n_q_heads);
-    cfg.blockDim = dim3(gmlp::kUmmaThreads);
+    cfg.blockDim = dim3(gmlp::kGqaThreads);
     cfg.dynamicSmemBytes = gmlp::kGqaSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

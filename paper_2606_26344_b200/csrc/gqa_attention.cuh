@@ -1,20 +1,21 @@
 // Group Query Attention (one of the paper's multi-operator kernels, Section 6.1), forward, no mask:
 //     O_h = softmax( Q_h K_g^T / sqrt(D) ) V_g,      g = h / (Hq / Hkv),      D = 128,
-// Q [M, Hq*D], K and V [S, Hkv*D], O [M, Hq*D] row-major bf16.  One CTA per (128 query rows, query head); the
-// key/value sequence is walked in blocks of 128 with the running-maximum (online) softmax, so the scores never
-// leave the SM: both matmuls run on tcgen05 with their accumulators in TMEM and the probabilities go from
-// registers to shared memory as the second matmul's A operand.
+// Q [M, Hq*D], K and V [S, Hkv*D], O [M, Hq*D] row-major bf16.  One CTA per (256 query rows, query head), as TWO
+// query tiles of 128 rows that take turns on the tensor pipe: while one tile's scores are in the softmax, the
+// other tile's matmuls run.  The key/value sequence is walked in blocks of 128 with the running-maximum (online)
+// softmax, so the scores never leave the SM: both matmuls run on tcgen05 with their accumulators in TMEM and the
+// probabilities go from registers to shared memory as the second matmul's A operand.
 //
-//   warp 0      TMA producer: Q tile once, then K blocks and V blocks into two two-stage rings of their own
-//   warp 1      MMA issuer:   S = Q K^T into one of two TMEM score buffers (columns [0,128) / [128,256)), so the
-//                             scores of block j+1 are computed while block j is in the softmax; then
-//                             O += P V (TMEM columns [256,384))
-//   warps 2..5  softmax:      thread t owns query row t (its TMEM lane), so row maxima and sums need no shuffles;
-//                             reads its 128 scores once into registers, writes P (bf16) into the
-//                             128-byte-swizzled K-major layout the MMA expects, and at the end stores O / l.
-//                             The exponent base is a running maximum that is only moved when a block's maximum
-//                             exceeds it by more than 8 (probabilities stay below 2^8), so O in TMEM is rescaled
-//                             rarely instead of once per block.
+//   warp 0      TMA producer: both Q tiles once, then K(0), V(0), K(1), V(1), ... through one three-slot FIFO
+//   warp 1      MMA issuer:   per tile t, S_t = Q_t K^T (TMEM columns 128 t) and O_t += P_t V (columns 256 + 128 t),
+//                             in the order PV_A(j), S_A(j+1), PV_B(j), S_B(j+1)
+//   warps 2..5  softmax of tile A, warps 6..9 of tile B: thread = query row (its TMEM lane), so row maxima and sums
+//                             need no shuffles.  The exponent base is a running maximum that is only moved when a
+//                             block's maximum exceeds it by more than 8 (probabilities stay below 2^8): a block is
+//                             normally ONE pass over its scores (exponentials with the current base while the
+//                             maximum is tracked); only if the base has to move is O in TMEM rescaled and the
+//                             block's probabilities recomputed.  P (bf16) is written in the 128-byte-swizzled
+//                             K-major layout the MMA expects; at the end O / l is stored.
 //
 // Operand forms: Q and P are K-major A operands (rows of 128 B, two 64-wide swizzle atoms side by side); a K block
 // [128 keys, D] is a K-major B operand (keys are the N dimension); a V block [128 keys, D] is an MN-major B
@@ -30,11 +31,12 @@
 namespace gmlp {
 
 constexpr int kGqaD = 128;                       // head dimension
-constexpr int kGqaBM = 128;                      // query rows per CTA
+constexpr int kGqaBM = 256;                      // query rows per CTA (two tiles of 128)
 constexpr int kGqaBS = 128;                      // keys per block
+constexpr int kGqaThreads = 320;                 // producer warp, MMA warp, 2 x 4 softmax warps
 constexpr uint32_t kGqaTileBytes = 128 * 128 * 2;                         // one 128 x 128 bf16 tile: 32 KB
-constexpr int kGqaStages = 2;                                             // per ring (K blocks, V blocks)
-constexpr uint32_t kGqaSmemBytes = (2 + 2 * kGqaStages) * kGqaTileBytes + 1024 + 256;   // Q, P, K ring, V ring
+constexpr int kGqaSlots = 3;                                              // K/V FIFO slots
+constexpr uint32_t kGqaSmemBytes = (4 + kGqaSlots) * kGqaTileBytes + 1024 + 256;   // Q_A Q_B P_A P_B, FIFO
 constexpr float kGqaLazyLog2 = 8.0f;                                      // move the exponent base only beyond this
 
 __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -55,7 +57,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-__global__ void __launch_bounds__(kUmmaThreads, 1)
+__global__ void __launch_bounds__(kGqaThreads, 1)
 gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, bf16* __restrict__ O,
                      int M, int S, int n_q_heads, int group, float scale_log2)
@@ -71,18 +73,16 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - raw_addr);
-    const uint32_t q_smem = base, p_smem = base + kGqaTileBytes;
-    const uint32_t k_ring = base + 2 * kGqaTileBytes, v_ring = k_ring + kGqaStages * kGqaTileBytes;
-    uint8_t* p_ptr = base_ptr + kGqaTileBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + (2 + 2 * kGqaStages) * kGqaTileBytes);
-    const uint32_t k_full0 = ptx::smem_addr(bars);                   // [2]
-    const uint32_t k_empty0 = ptx::smem_addr(bars + 2);              // [2]
-    const uint32_t v_full0 = ptx::smem_addr(bars + 4);               // [2]
-    const uint32_t v_empty0 = ptx::smem_addr(bars + 6);              // [2]
-    const uint32_t s_full0 = ptx::smem_addr(bars + 8);               // [2] the scores of a block are in TMEM buffer b
-    const uint32_t q_full = ptx::smem_addr(bars + 10);
-    const uint32_t p_full = ptx::smem_addr(bars + 11);               // P is in shared memory (and O rescaled if need be)
-    const uint32_t o_full = ptx::smem_addr(bars + 12);               // O += P V of a block is done
+    const uint32_t q_smem = base;                                    // + tile * 32 KB
+    const uint32_t p_smem = base + 2 * kGqaTileBytes;                // + tile * 32 KB
+    const uint32_t fifo = base + 4 * kGqaTileBytes;                  // + slot * 32 KB
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + (4 + kGqaSlots) * kGqaTileBytes);
+    const uint32_t kv_full0 = ptx::smem_addr(bars);                  // [3]
+    const uint32_t kv_empty0 = ptx::smem_addr(bars + 3);             // [3]
+    const uint32_t s_full0 = ptx::smem_addr(bars + 6);               // [2] tile t: the scores of a block are in TMEM
+    const uint32_t p_full0 = ptx::smem_addr(bars + 8);               // [2] tile t: P is in shared memory
+    const uint32_t o_full0 = ptx::smem_addr(bars + 10);              // [2] tile t: O += P V of a block is done
+    const uint32_t q_full = ptx::smem_addr(bars + 12);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -94,10 +94,12 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     ptx::launch_dependents();
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 10; ++i) ptx::mbar_init(k_full0 + 8 * i, 1);      // the five two-entry barrier arrays
+        for (int i = 0; i < 8; ++i) ptx::mbar_init(kv_full0 + 8 * i, 1);       // kv_full, kv_empty, s_full
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(p_full0 + 8 * i, 4);                      // one arrival per softmax warp of the tile
+            ptx::mbar_init(o_full0 + 8 * i, 1);
+        }
         ptx::mbar_init(q_full, 1);
-        ptx::mbar_init(p_full, 4);                                   // one arrival per softmax warp
-        ptx::mbar_init(o_full, 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
@@ -112,166 +114,203 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_o = tmem_base + 256;                         // scores: tmem_base + 128 * (block & 1)
+    const uint32_t tmem_base = *tmem_slot;                           // S_t at + 128 t, O_t at + 256 + 128 t
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             ptx::grid_dependency_wait();                             // Q, K, V may come from the previous kernel
-            ptx::mbar_arrive_expect_tx(q_full, kGqaTileBytes);
-            ptx::tma_load_2d(q_smem, &tmQ, h * kGqaD, m0, q_full);
-            ptx::tma_load_2d(q_smem + 16384, &tmQ, h * kGqaD + 64, m0, q_full);
-            for (int j = 0; j < n_blocks; ++j) {
-                const int s = j % kGqaStages;
-                const uint32_t ph = (uint32_t)(j / kGqaStages) & 1u;
-                const int s0 = j * kGqaBS;
-                // K block: two boxes of 64 d x 128 keys (K-major: a key's d values are contiguous)
-                if (!wait_bounded(k_empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
-                const uint32_t k_dst = k_ring + s * kGqaTileBytes;
-                ptx::mbar_arrive_expect_tx(k_full0 + 8 * s, kGqaTileBytes);
-                ptx::tma_load_2d(k_dst, &tmK, g * kGqaD, s0, k_full0 + 8 * s);
-                ptx::tma_load_2d(k_dst + 16384, &tmK, g * kGqaD + 64, s0, k_full0 + 8 * s);
-                // V block: four boxes of 64 d x 64 keys; (key half, d half) at (2 * key half + d half) * 8 KB
-                if (!wait_bounded(v_empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 8)) break;
-                const uint32_t v_dst = v_ring + s * kGqaTileBytes;
-                ptx::mbar_arrive_expect_tx(v_full0 + 8 * s, kGqaTileBytes);
+            ptx::mbar_arrive_expect_tx(q_full, 2 * kGqaTileBytes);
 #pragma unroll
-                for (int sh = 0; sh < 2; ++sh)
+            for (int t = 0; t < 2; ++t) {
+                ptx::tma_load_2d(q_smem + t * kGqaTileBytes, &tmQ, h * kGqaD, m0 + 128 * t, q_full);
+                ptx::tma_load_2d(q_smem + t * kGqaTileBytes + 16384, &tmQ, h * kGqaD + 64, m0 + 128 * t, q_full);
+            }
+            for (int i = 0; i < 2 * n_blocks; ++i) {                 // item 2j = K(j), item 2j+1 = V(j)
+                const int slot = i % kGqaSlots;
+                if (!wait_bounded(kv_empty0 + 8 * slot, ((uint32_t)(i / kGqaSlots) & 1u) ^ 1u, abort_flag, KERNEL_ID, 1)) break;
+                const uint32_t full = kv_full0 + 8 * slot;
+                const uint32_t dst = fifo + slot * kGqaTileBytes;
+                const int s0 = (i >> 1) * kGqaBS;
+                ptx::mbar_arrive_expect_tx(full, kGqaTileBytes);
+                if ((i & 1) == 0) {
+                    // K block: two boxes of 64 d x 128 keys (K-major: a key's d values are contiguous)
+                    ptx::tma_load_2d(dst, &tmK, g * kGqaD, s0, full);
+                    ptx::tma_load_2d(dst + 16384, &tmK, g * kGqaD + 64, s0, full);
+                } else {
+                    // V block: four boxes of 64 d x 64 keys; (key half, d half) at (2 * key half + d half) * 8 KB
 #pragma unroll
-                    for (int nh = 0; nh < 2; ++nh)
-                        ptx::tma_load_2d(v_dst + (sh * 2 + nh) * 8192, &tmV, g * kGqaD + nh * 64, s0 + sh * 64,
-                                         v_full0 + 8 * s);
+                    for (int sh = 0; sh < 2; ++sh)
+#pragma unroll
+                        for (int nh = 0; nh < 2; ++nh)
+                            ptx::tma_load_2d(dst + (sh * 2 + nh) * 8192, &tmV, g * kGqaD + nh * 64, s0 + sh * 64, full);
+                }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            // S(j) = Q K(j)^T over D = 128: eight K = 16 steps, four per 64-wide swizzle atom
-            auto issue_scores = [&](int j) -> bool {
-                const int s = j % kGqaStages;
-                if (!wait_bounded(k_full0 + 8 * s, (uint32_t)(j / kGqaStages) & 1u, abort_flag, KERNEL_ID, 2)) return false;
+            auto item_ready = [&](int i, int site) -> bool {
+                const bool ok = wait_bounded(kv_full0 + 8 * (i % kGqaSlots), (uint32_t)(i / kGqaSlots) & 1u, abort_flag, KERNEL_ID, site);
                 ptx::tc_fence_after_sync();
-                const uint32_t k_smem = k_ring + s * kGqaTileBytes;
+                return ok;
+            };
+            // S_t(j) = Q_t K(j)^T over D = 128: eight K = 16 steps, four per 64-wide swizzle atom
+            auto issue_scores = [&](int t, int j) {
+                const uint32_t k_smem = fifo + ((2 * j) % kGqaSlots) * kGqaTileBytes;
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     const uint32_t off = (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u;
-                    ptx::umma_bf16(tmem_base + 128u * (uint32_t)(j & 1), ptx::make_smem_desc_sw128(q_smem + off, 16, 1024),
+                    ptx::umma_bf16(tmem_base + 128u * (uint32_t)t,
+                                   ptx::make_smem_desc_sw128(q_smem + t * kGqaTileBytes + off, 16, 1024),
                                    ptx::make_smem_desc_sw128(k_smem + off, 16, 1024), kIdescQK, k != 0 ? 1u : 0u);
                 }
-                ptx::umma_commit(s_full0 + 8 * (j & 1));
-                ptx::umma_commit(k_empty0 + 8 * s);
-                return true;
+                ptx::umma_commit(s_full0 + 8 * t);
+                if (t == 1) ptx::umma_commit(kv_empty0 + 8 * ((2 * j) % kGqaSlots));      // both tiles have used K(j)
             };
-            bool ok = wait_bounded(q_full, 0u, abort_flag, KERNEL_ID, 5);
-            ok = ok && issue_scores(0);
+            bool ok = wait_bounded(q_full, 0u, abort_flag, KERNEL_ID, 5) && item_ready(0, 2);
+            if (ok) {
+                issue_scores(0, 0);
+                issue_scores(1, 0);
+            }
             for (int j = 0; j < n_blocks && ok; ++j) {
-                // the scores of the next block are computed while this block is in the softmax: its score buffer
-                // was last read for block j-1, whose probabilities the wait below (one iteration ago) has seen
-                if (j + 1 < n_blocks && !issue_scores(j + 1)) break;
-                const int s = j % kGqaStages;
-                if (!wait_bounded(p_full, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 6)) break;
-                if (!wait_bounded(v_full0 + 8 * s, (uint32_t)(j / kGqaStages) & 1u, abort_flag, KERNEL_ID, 9)) break;
-                ptx::tc_fence_after_sync();
-                const uint32_t v_smem = v_ring + s * kGqaTileBytes;
-                // O += P V over the block's 128 keys
+                for (int t = 0; t < 2 && ok; ++t) {
+                    // tile t's probabilities of block j are in shared memory; V(j) has landed
+                    if (!wait_bounded(p_full0 + 8 * t, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 6)) { ok = false; break; }
+                    if (t == 0 && !item_ready(2 * j + 1, 9)) { ok = false; break; }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t v_smem = fifo + ((2 * j + 1) % kGqaSlots) * kGqaTileBytes;
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const uint64_t a_desc = ptx::make_smem_desc_sw128(
-                        p_smem + (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u, 16, 1024);
-                    const uint64_t b_desc = ptx::make_smem_desc_sw128(
-                        v_smem + (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 2048u, 8192, 1024);
-                    ptx::umma_bf16(tmem_o, a_desc, b_desc, kIdescPV, (j | k) != 0 ? 1u : 0u);
+                    for (int k = 0; k < 8; ++k) {
+                        const uint64_t a_desc = ptx::make_smem_desc_sw128(
+                            p_smem + t * kGqaTileBytes + (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u, 16, 1024);
+                        const uint64_t b_desc = ptx::make_smem_desc_sw128(
+                            v_smem + (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 2048u, 8192, 1024);
+                        ptx::umma_bf16(tmem_base + 256u + 128u * (uint32_t)t, a_desc, b_desc, kIdescPV, (j | k) != 0 ? 1u : 0u);
+                    }
+                    ptx::umma_commit(o_full0 + 8 * t);
+                    if (t == 1) ptx::umma_commit(kv_empty0 + 8 * ((2 * j + 1) % kGqaSlots));   // both tiles have used V(j)
+                    // the tile's next scores follow at once: its score buffer was consumed before p_full
+                    if (j + 1 < n_blocks) {
+                        if (t == 0 && !item_ready(2 * j + 2, 2)) { ok = false; break; }
+                        issue_scores(t, j + 1);
+                    }
                 }
-                ptx::umma_commit(v_empty0 + 8 * s);
-                ptx::umma_commit(o_full);
             }
         }
         __syncwarp();
     } else {
-        // ---------------- softmax and epilogue: thread = query row ----------------
+        // ---------------- softmax and epilogue: one group of four warps per tile, thread = query row ----------------
+        const int t = (warp - 2) >> 2;                               // tile
         const int q = warp & 3;
         const int r = q * 32 + lane;                                 // row within the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-        float m_use = 0.0f, l_run = 0.0f;                            // exponent base (set on the first block), row sum
+        const uint32_t s_addr = tmem_base + 128u * (uint32_t)t + lane_addr;
+        const uint32_t o_addr = tmem_base + 256u + 128u * (uint32_t)t + lane_addr;
+        uint8_t* p_row = base_ptr + (2 + t) * kGqaTileBytes + (size_t)r * 128;
+        float m_use = -INFINITY, l_run = 0.0f;                       // exponent base, row sum
         bool ok = true;
-        for (int j = 0; j < n_blocks && ok; ++j) {
-            if (!wait_bounded(s_full0 + 8 * (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag, KERNEL_ID, 3)) { ok = false; break; }
-            ptx::tc_fence_after_sync();
-            const int valid = min(kGqaBS, S - j * kGqaBS);           // keys of this block that exist
-            const uint32_t s_addr = tmem_base + 128u * (uint32_t)(j & 1) + lane_addr;
-            uint32_t sv[4][32];                                      // this row's 128 scores
-#pragma unroll
-            for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(s_addr + 32 * c, sv[c]);
+
+        // one pass over the block's scores with base m_use: P to shared memory, row sum and row maximum.  The
+        // next 32 scores are on their way from TMEM while the current 32 are processed; the scale is folded into
+        // the exponent's FMA; only a block with missing keys (the last one) pays for the masking.
+        auto block_pass = [&](int valid, float& l_blk, float& m_blk) {
+            const bool masked = valid < kGqaBS;
+            const float neg_base = -m_use;
+            float l_acc = 0.0f, m_raw = -INFINITY;
+            uint32_t v[2][32];
+            ptx::tmem_ld_32x32(s_addr, v[0]);
             ptx::tmem_ld_wait();
-            float m_blk = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (32 * c + i < valid) m_blk = fmaxf(m_blk, __uint_as_float(sv[c][i]) * scale_log2);
-            // P of the previous block must have been consumed (and O complete) before P is overwritten
-            if (j > 0) {
-                if (!wait_bounded(o_full, (uint32_t)(j - 1) & 1u, abort_flag, KERNEL_ID, 4)) { ok = false; break; }
-                ptx::tc_fence_after_sync();
-            }
-            if (j == 0) {
-                m_use = m_blk;                                       // finite: the first block has at least one key
-            } else if (__any_sync(0xFFFFFFFFu, m_blk > m_use + kGqaLazyLog2)) {
-                // some row's maximum moved far: rescale this warp's rows of O (and l) to the new base
-                const float m_new = fmaxf(m_use, m_blk);
-                const float alpha = ex2_approx(m_use - m_new);
-                m_use = m_new;
-                l_run *= alpha;
-#pragma unroll 1
-                for (int c = 0; c < kGqaD; c += 32) {
-                    uint32_t v[32];
-                    ptx::tmem_ld_32x32(tmem_o + lane_addr + c, v);
-                    ptx::tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                    tmem_st_32x32(tmem_o + lane_addr + c, v);
-                }
-                tmem_st_wait();
-            }
-            // p = 2^(x - base), row sum, P as bf16 into the swizzled K-major tile
-            float l_blk = 0.0f;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
+                if (c + 1 < 4) ptx::tmem_ld_32x32(s_addr + 32 * (c + 1), v[(c + 1) & 1]);
                 uint32_t packed[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const float p0 = (32 * c + 2 * i < valid) ? ex2_approx(__uint_as_float(sv[c][2 * i]) * scale_log2 - m_use) : 0.0f;
-                    const float p1 = (32 * c + 2 * i + 1 < valid) ? ex2_approx(__uint_as_float(sv[c][2 * i + 1]) * scale_log2 - m_use) : 0.0f;
-                    l_blk += p0 + p1;
+                    float x0 = __uint_as_float(v[c & 1][2 * i]), x1 = __uint_as_float(v[c & 1][2 * i + 1]);
+                    if (masked) {
+                        if (32 * c + 2 * i >= valid) x0 = -INFINITY;
+                        if (32 * c + 2 * i + 1 >= valid) x1 = -INFINITY;
+                    }
+                    m_raw = fmaxf(m_raw, fmaxf(x0, x1));
+                    const float p0 = ex2_approx(fmaf(x0, scale_log2, neg_base));
+                    const float p1 = ex2_approx(fmaf(x1, scale_log2, neg_base));
+                    l_acc += p0 + p1;
                     packed[i] = pack_bf16x2(p0, p1);
                 }
                 // columns 32c .. 32c+31 of row r: four 16-byte chunks of the 64-wide atom (c / 2)
-                uint8_t* atom = p_ptr + (size_t)(c >> 1) * 16384 + (size_t)r * 128;
+                uint8_t* atom = p_row + (size_t)(c >> 1) * 16384;
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
                     const int chunk = (c & 1) * 4 + ch;                              // 0..7 within the 128-byte row
                     *reinterpret_cast<uint4*>(atom + ((chunk ^ (r & 7)) << 4)) =
                         make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
                 }
+                if (c + 1 < 4) ptx::tmem_ld_wait();
+            }
+            l_blk = l_acc;
+            m_blk = m_raw * scale_log2;                              // the scale is positive
+        };
+
+        for (int j = 0; j < n_blocks && ok; ++j) {
+            if (!wait_bounded(s_full0 + 8 * t, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 3)) { ok = false; break; }
+            // P of the previous block must have been consumed (and O complete) before P is overwritten
+            if (j > 0 && !wait_bounded(o_full0 + 8 * t, (uint32_t)(j - 1) & 1u, abort_flag, KERNEL_ID, 4)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            const int valid = min(kGqaBS, S - j * kGqaBS);           // keys of this block that exist
+            float l_blk, m_blk;
+            if (j == 0) {
+                // first block: find the base first (finite: the block has at least one key)
+                float m0v = -INFINITY;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    ptx::tmem_ld_32x32(s_addr + 32 * c, v);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (32 * c + i < valid) m0v = fmaxf(m0v, __uint_as_float(v[i]) * scale_log2);
+                }
+                m_use = m0v;
+                block_pass(valid, l_blk, m_blk);
+            } else {
+                block_pass(valid, l_blk, m_blk);
+                if (__any_sync(0xFFFFFFFFu, m_blk > m_use + kGqaLazyLog2)) {
+                    // some row's maximum moved far: new base, rescale this warp's rows of O and l, redo the block
+                    const float m_new = fmaxf(m_use, m_blk);
+                    const float alpha = ex2_approx(m_use - m_new);
+                    m_use = m_new;
+                    l_run *= alpha;
+#pragma unroll 1
+                    for (int c = 0; c < kGqaD; c += 32) {
+                        uint32_t v[32];
+                        ptx::tmem_ld_32x32(o_addr + c, v);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                        tmem_st_32x32(o_addr + c, v);
+                    }
+                    tmem_st_wait();
+                    block_pass(valid, l_blk, m_blk);
+                }
             }
             l_run += l_blk;
             ptx::fence_proxy_async_smem();                           // P (generic writes) -> visible to the MMA
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(p_full);
+            if (lane == 0) ptx::mbar_arrive(p_full0 + 8 * t);
         }
         // epilogue: O / l, one rounding, 256 contiguous bytes per row
-        if (ok && wait_bounded(o_full, (uint32_t)(n_blocks - 1) & 1u, abort_flag, KERNEL_ID, 7)) {
+        if (ok && wait_bounded(o_full0 + 8 * t, (uint32_t)(n_blocks - 1) & 1u, abort_flag, KERNEL_ID, 7)) {
             ptx::tc_fence_after_sync();
             const float inv_l = 1.0f / l_run;
-            const int row = m0 + r;
+            const int row = m0 + 128 * t + r;
             bf16* orow = O + (size_t)row * ((size_t)n_q_heads * kGqaD) + (size_t)h * kGqaD;
 #pragma unroll 1
             for (int c = 0; c < kGqaD; c += 32) {
                 uint32_t v[32];
-                ptx::tmem_ld_32x32(tmem_o + lane_addr + c, v);
+                ptx::tmem_ld_32x32(o_addr + c, v);
                 ptx::tmem_ld_wait();
                 if (row < M) {
 #pragma unroll
