@@ -411,7 +411,17 @@ void forget_counters(DeviceState* dev) {
     } while (0)
 
 int launch_rmsnorm(const bf16* X, const bf16* gain, bf16* Xn, int64_t M, int64_t d_model, float eps, cudaStream_t st) {
-    gmlp::rmsnorm_kernel<<<(unsigned)M, gmlp::kRmsThreads, 0, st>>>(X, gain, Xn, M, (int)d_model, eps);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)M);
+    cfg.blockDim = dim3(gmlp::kRmsThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int dm = (int)d_model;
+    if (cudaLaunchKernelEx(&cfg, gmlp::rmsnorm_kernel, X, gain, Xn, M, dm, eps) != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
 }

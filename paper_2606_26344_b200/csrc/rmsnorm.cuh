@@ -12,6 +12,11 @@ __global__ void __launch_bounds__(kRmsThreads)
 rmsnorm_kernel(const bf16* __restrict__ X, const bf16* __restrict__ gamma, bf16* __restrict__ Xn,
                int64_t M, int d_model, float eps)
 {
+    // launched with programmatic stream serialization: the GEMM that follows may become resident (barriers, TMEM,
+    // tensor-map prefetch) while this kernel runs; X may be the previous kernel's output, so nothing is read
+    // before that kernel is complete
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t row = blockIdx.x;
     if (row >= M) return;
     const uint4* x = reinterpret_cast<const uint4*>(X + row * d_model);
