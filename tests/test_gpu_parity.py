@@ -300,6 +300,24 @@ def test_stated_configs_in_the_benchmarked_launch_configuration(name):
     check_case(inp, gmlp.VARIANT_AUTO, name)
 
 
+def test_h_with_more_than_two_to_the_31_elements():
+    """Maximum sizes: 140,000 x 16,384 intermediate values (2.29e9 elements, 4.6 GB) - element offsets no longer
+    fit 32 bits; rows from the whole range, the last one included, are compared with the oracle."""
+    M, dm, dff = 140000, 256, 16384
+    assert M * dff > 2 ** 31
+    inp = I.custom_inputs(M, dm, dff, 31)
+    t = to_device(inp)
+    Y = gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], checked=True)
+    torch.cuda.synchronize()
+    rows = np.unique(np.concatenate([np.array([0, 1, 2 ** 17 - 1, 2 ** 17, 131071 + 128, M - 129, M - 2, M - 1]),
+                                     np.random.default_rng(5).choice(M, 40, replace=False)]))
+    y_ref = oracle_rows(inp, rows)
+    e, _ = err_over_tol(Y, y_ref, rows)
+    assert float(e.max()) <= 1.0, f"max err/tol {float(e.max()):.3f}"
+    del Y, t
+    torch.cuda.empty_cache()
+
+
 def test_llama70b_prefill_with_outlier_rows():
     # Rows scaled x20 reach |h| ~ 2000, where ONE bf16 rounding flip of h (an effect of fp32 versus
     # fp64 accumulation of g, u that any fp32-accumulating data path has) moves a y element by ~0.05,
