@@ -75,7 +75,12 @@ enum {
      * bit for bit as with the [in, out] storage.  gmlp_forward_ex and gmlp_gate_up with the tensor-core
      * schedules only (GMLP_VARIANT_SIMT / _STREAM: GMLP_ERR_UNSUPPORTED); gmlp_forward_static and the other
      * operators take [in, out] weights. */
-    GMLP_FLAG_WEIGHTS_OUT_IN = 1u << 7
+    GMLP_FLAG_WEIGHTS_OUT_IN = 1u << 7,
+    /* Y is left in fp32: args->Y is a float matrix [M, d_model] and receives the down projection's fp32
+     * accumulator without the final rounding (rounding it to bf16 gives the default output bit for bit).
+     * gmlp_forward_ex / gmlp_forward_host with the tensor-core schedules only (SIMT / STREAM:
+     * GMLP_ERR_UNSUPPORTED); gmlp_gate_up rejects it (GMLP_ERR_FLAGS). */
+    GMLP_FLAG_Y_FP32 = 1u << 8
 };
 
 /* Kernel schedule.  AUTO picks by shape; the others force one schedule (tests, benchmarks). */

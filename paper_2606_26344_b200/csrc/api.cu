@@ -30,10 +30,17 @@ constexpr int kVersion = 100;
 constexpr int kMaxDevices = 64;
 constexpr int64_t kMaxDim = (int64_t)1 << 30;      // per-dimension limit (TMA coordinates are int32)
 constexpr uint32_t kKnownFlags = GMLP_FLAG_RMSNORM | GMLP_FLAG_CHECKED | GMLP_FLAG_ACT_SWISH | GMLP_FLAG_ACT_GLU |
-                                 GMLP_FLAG_WEIGHTS_OUT_IN;
+                                 GMLP_FLAG_WEIGHTS_OUT_IN | GMLP_FLAG_Y_FP32;
 constexpr gmlp::GateAct kSilu = {1.0f, 0};
 // weights of the call in flight are stored [out, in] (set by the entry points around their launches)
 thread_local bool t_w_out_in = false;
+// the down projection of the call in flight leaves Y in fp32 (set by gmlp_forward_ex around its second GEMM)
+thread_local bool t_y_fp32 = false;
+struct OutputTypeScope {
+    bool prev;
+    explicit OutputTypeScope(bool fp32) : prev(t_y_fp32) { t_y_fp32 = fp32; }
+    ~OutputTypeScope() { t_y_fp32 = prev; }
+};
 struct WeightLayoutScope {                       // sets the switch for one call, restores it on every exit path
     bool prev;
     explicit WeightLayoutScope(bool out_in) : prev(t_w_out_in) { t_w_out_in = out_in; }
@@ -485,6 +492,7 @@ template <bool GATEUP>
 int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
                      int64_t M, int64_t K, int64_t N, cudaStream_t st, gmlp::GateAct act = kSilu) {
     const int wkm = t_w_out_in ? 1 : 0;
+    const int yf32 = (!GATEUP && t_y_fp32) ? 1 : 0;
     CUtensorMap tmA, tmB0, tmB1;
     if (!encode_2d(&tmA, A, (uint64_t)K, (uint64_t)M, gmlp::kUmmaBK, 128)) return GMLP_ERR_LAUNCH;
     if (!GMLP_ENCODE_W(&tmB0, W0, N, K)) return GMLP_ERR_LAUNCH;
@@ -521,7 +529,7 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
     if (cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m,
-                           num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm) != cudaSuccess)
+                           num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm, yf32) != cudaSuccess)
         return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -546,6 +554,7 @@ int pick_split_k(int num_m, int64_t K, int64_t N, int sms) {
 int launch_umma_splitk(DeviceState* dev, int S, const CUtensorMap& tmA, const CUtensorMap& tmB, bf16* C,
                        int64_t M, int64_t K, int64_t N, int num_m, int a_box_rows, cudaStream_t st) {
     const int wkm = t_w_out_in ? 1 : 0;
+    const int yf32 = t_y_fp32 ? 1 : 0;
     if (!dev->splitk_attr_set) {
         const int b = (int)gmlp::kSplitSmemBytes;
         if (cudaFuncSetAttribute(gmlp::umma_splitk_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
@@ -571,9 +580,9 @@ int launch_umma_splitk(DeviceState* dev, int S, const CUtensorMap& tmA, const CU
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
     cudaError_t err;
-    if (S == 4) err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<4>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows, wkm);
-    else if (S == 3) err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<3>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows, wkm);
-    else err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<2>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows, wkm);
+    if (S == 4) err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<4>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows, wkm, yf32);
+    else if (S == 3) err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<3>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows, wkm, yf32);
+    else err = cudaLaunchKernelEx(&cfg, gmlp::umma_splitk_gemm_kernel<2>, tmA, tmB, C, Mi, Ki, Ni, num_m, a_box_rows, wkm, yf32);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -583,6 +592,7 @@ template <bool GATEUP>
 int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
                 int64_t M, int64_t K, int64_t N, cudaStream_t st, gmlp::GateAct act = kSilu) {
     const int wkm = t_w_out_in ? 1 : 0;
+    const int yf32 = (!GATEUP && t_y_fp32) ? 1 : 0;
     CUtensorMap tmA, tmB0, tmB1;
     // TMA is markedly slower when a box has fewer than 16 rows inside the tensor; with so few rows in all, the
     // box is made exactly M rows high instead (no out-of-range rows to fill)
@@ -633,16 +643,16 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     cudaError_t err;
     if (GATEUP && nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm, yf32);
     else if (GATEUP)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<true, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm, yf32);
     else if (nb == 4)
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm, yf32);
     else
         err = cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 2>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m, num_tiles,
-                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm);
+                                 (const float*)nullptr, a_box_rows, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm, yf32);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -653,6 +663,7 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
                   unsigned int* counters, bf16* out, int64_t M, int64_t K, int64_t N, cudaStream_t st,
                   gmlp::GateAct act = kSilu) {
     const int wkm = t_w_out_in ? 1 : 0;
+    const int yf32 = (!GATEUP && t_y_fp32) ? 1 : 0;
     if (p.stages < 2 || p.tmem_cols > 512) return GMLP_ERR_UNSUPPORTED;
     CUtensorMap tmX, tmW0, tmW1;
     if (!encode_2d(&tmX, X, (uint64_t)K, (uint64_t)M, 64, (uint32_t)p.Mpad)) return GMLP_ERR_LAUNCH;
@@ -689,10 +700,10 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
     cudaError_t err;
     if (p.NH == 2)
         err = cudaLaunchKernelEx(&cfg, gmlp::skinny_gemm_kernel<GATEUP, 2>, tmX, tmW0, tmW1, scratch, counters, out,
-                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first, act, wkm);
+                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first, act, wkm, yf32);
     else
         err = cudaLaunchKernelEx(&cfg, gmlp::skinny_gemm_kernel<GATEUP, 1>, tmX, tmW0, tmW1, scratch, counters, out,
-                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first, act, wkm);
+                                 Mi, p.Mpad, Ni, p.num_tiles, p.KB, p.stages, p.tmem_cols, evict_first, act, wkm, yf32);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -748,8 +759,10 @@ int forward_impl(const gmlp_args* a) {
     const int variant = resolve_variant(a->M, a->d_model, a->d_ff, a->variant);
     if (variant == GMLP_VARIANT_SKINNY && a->M > 128) return GMLP_ERR_UNSUPPORTED;
     const bool w_out_in = (a->flags & GMLP_FLAG_WEIGHTS_OUT_IN) != 0;
-    if (w_out_in && (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM)) return GMLP_ERR_UNSUPPORTED;
+    const bool y_fp32 = (a->flags & GMLP_FLAG_Y_FP32) != 0;
+    if ((w_out_in || y_fp32) && (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM)) return GMLP_ERR_UNSUPPORTED;
     const WeightLayoutScope layout_scope(w_out_in);
+    const OutputTypeScope output_scope(y_fp32);
     const Layout L = make_layout(a->M, a->d_model, a->d_ff, a->flags, variant, dev->sm_count);
 
     uint8_t* ws = static_cast<uint8_t*>(a->workspace);
@@ -924,6 +937,7 @@ int gate_up_impl(const gmlp_args* a) {
     const int variant = resolve_variant(a->M, a->d_model, a->d_ff, a->variant);
     if (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM) return GMLP_ERR_UNSUPPORTED;
     if (variant == GMLP_VARIANT_SKINNY && a->M > 128) return GMLP_ERR_UNSUPPORTED;
+    if (a->flags & GMLP_FLAG_Y_FP32) return GMLP_ERR_FLAGS;          // H is the bf16 operand of the next GEMM
     const WeightLayoutScope layout_scope((a->flags & GMLP_FLAG_WEIGHTS_OUT_IN) != 0);
     DeviceState* dev = current_device(&rc);
     if (dev == nullptr) return rc;
@@ -1062,8 +1076,8 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         const float* rc_ptr = r;
         cudaError_t err = pair
-            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0)
-            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0);
+            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0, 0)
+            : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0, 0);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("matmul_rowscale", st);
@@ -1156,9 +1170,9 @@ int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         cudaError_t err = pair
             ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
-                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq, kNoMulti, 0)
+                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq, kNoMulti, 0, 0)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
-                                 num_tiles, (const float*)nullptr, 128, kSilu, R, sumsq, kNoMulti, 0);
+                                 num_tiles, (const float*)nullptr, 128, kSilu, R, sumsq, kNoMulti, 0, 0);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("matmul_add", st);
@@ -1266,10 +1280,10 @@ int qkv_proj_impl(const gmlp_qkv_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->Nq;
         cudaError_t err = pair
             ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, false, true>, tmA, tmB0, tmB1, Q, Mi, Ki, Ni,
-                                 num_m, num_tiles, (const float*)nullptr, kSilu, (const bf16*)nullptr, (float*)nullptr, multi, 0)
+                                 num_m, num_tiles, (const float*)nullptr, kSilu, (const bf16*)nullptr, (float*)nullptr, multi, 0, 0)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, false, true>, tmA, tmB0, tmB1, Q, Mi, Ki, Ni,
                                  num_m, num_tiles, (const float*)nullptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr,
-                                 multi, 0);
+                                 multi, 0, 0);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
         prof_mark("qkv", st);
@@ -1543,12 +1557,13 @@ int gmlp_forward_host(const gmlp_args* args, const void* X_host, void* Y_host) {
     if (args->M == 0) return gmlp_forward_ex(args);
     if (!args->X || !args->Y) return GMLP_ERR_NULL;
     const size_t bytes = (size_t)args->M * (size_t)args->d_model * 2;
+    const size_t y_bytes = (args->flags & GMLP_FLAG_Y_FP32) ? 2 * bytes : bytes;
     cudaStream_t st = static_cast<cudaStream_t>(args->stream);
     if (cudaMemcpyAsync(const_cast<void*>(args->X), X_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return GMLP_ERR_LAUNCH;
     rc = gmlp_forward_ex(args);
     if (rc != GMLP_OK) return rc;
-    if (cudaMemcpyAsync(Y_host, args->Y, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GMLP_ERR_LAUNCH;
+    if (cudaMemcpyAsync(Y_host, args->Y, y_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GMLP_ERR_LAUNCH;
     return GMLP_OK;
 }
 

@@ -133,7 +133,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
                  int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, int a_box_rows, GateAct act,
                  const bf16* residual, float* __restrict__ sumsq, const __grid_constant__ MultiB multi,
-                 int w_kmajor)
+                 int w_kmajor, int out_fp32)
 {
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
     static_assert(!(ADDSS && (GATEUP || ROWSCALE)), "the residual epilogue is for the plain GEMM");
@@ -319,7 +319,18 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     for (int j = 0; j < 16; ++j)
                         packed[j] = pack_bf16x2(__uint_as_float(g[2 * j]) * rscale, __uint_as_float(g[2 * j + 1]) * rscale);
                 }
-                if (row < M) {
+                if (!GATEUP && !ADDSS && !MULTI && out_fp32) {
+                    // the plain product left in fp32 (C is a float matrix): 128 bytes of this row per chunk
+                    if (row < M) {
+                        float* frow = reinterpret_cast<float*>(C) + (size_t)row * N + n0 + c;
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            if (n0 + c + v * 4 < N)
+                                *reinterpret_cast<float4*>(frow + v * 4) =
+                                    make_float4(__uint_as_float(g[4 * v]) * rscale, __uint_as_float(g[4 * v + 1]) * rscale,
+                                                __uint_as_float(g[4 * v + 2]) * rscale, __uint_as_float(g[4 * v + 3]) * rscale);
+                    }
+                } else if (row < M) {
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
                         if (n0 + c + v * 8 < Nseg)

@@ -36,7 +36,7 @@ __device__ __forceinline__ void st_cluster_f32x4(uint32_t cluster_addr, float a,
 template <int S>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                        bf16* __restrict__ C, int M, int K, int N, int num_m_tiles, int a_box_rows, int w_kmajor)
+                        bf16* __restrict__ C, int M, int K, int N, int num_m_tiles, int a_box_rows, int w_kmajor, int out_fp32)
 {
     static_assert(S >= 2 && (S - 1) * kSplitPartialBytes <= kSplitStages * kSplitStageBytes, "staging must fit the ring");
     constexpr int KERNEL_ID = 9;
@@ -173,6 +173,7 @@ umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             ptx::tmem_ld_32x32(taddr + c, v);
             ptx::tmem_ld_wait();
             uint32_t packed[16];
+            float* frow = reinterpret_cast<float*>(C) + (size_t)row * N + n0 + c;     // used when Y is kept in fp32
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 float4 acc = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
@@ -184,8 +185,9 @@ umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 }
                 packed[2 * j] = pack_bf16x2(acc.x, acc.y);
                 packed[2 * j + 1] = pack_bf16x2(acc.z, acc.w);
+                if (out_fp32 && row < M && acc_ok && n0 + c + j * 4 < N) *reinterpret_cast<float4*>(frow + j * 4) = acc;
             }
-            if (row < M && acc_ok) {
+            if (!out_fp32 && row < M && acc_ok) {
 #pragma unroll
                 for (int v4 = 0; v4 < 4; ++v4) {
                     if (n0 + c + v4 * 8 < N)

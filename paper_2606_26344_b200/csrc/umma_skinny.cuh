@@ -70,7 +70,7 @@ __device__ __forceinline__ bool skinny_epilogue_segment(
     uint32_t acc0, uint32_t tempty_bar, int tile, bool first_segment_of_cta, int cta, long long total, long long parts,
     int KB, int M, int Mpad, int N, float* __restrict__ scratch, unsigned int* __restrict__ counters,
     bf16* __restrict__ out, unsigned long long* slot_off, volatile int* last_flag, int et, int nl, int lane,
-    const GateAct act)
+    const GateAct act, const int out_fp32)
 {
     constexpr int NMAT = GATEUP ? 2 : 1;
     constexpr int TILE_N = 128 * NH;
@@ -97,7 +97,8 @@ __device__ __forceinline__ bool skinny_epilogue_segment(
                         if (m < M) {
                             const float v = GATEUP ? gate_act_f32(__uint_as_float(g[i]), act) * __uint_as_float(uu[i])
                                                    : __uint_as_float(g[i]);
-                            out[(size_t)m * N + n] = __float2bfloat16_rn(v);
+                            if (!GATEUP && out_fp32) reinterpret_cast<float*>(out)[(size_t)m * N + n] = v;
+                            else out[(size_t)m * N + n] = __float2bfloat16_rn(v);
                         }
                     }
                 }
@@ -196,8 +197,11 @@ __device__ __forceinline__ bool skinny_epilogue_segment(
                     v[2] = gate_act_f32(g.z, act) * uu.z; v[3] = gate_act_f32(g.w, act) * uu.w;
                 }
                 // N is a multiple of 8 and n of 4: the four columns are all inside or all outside
-                *reinterpret_cast<uint2*>(out + (size_t)mm * N + n) =
-                    make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+                if (!GATEUP && out_fp32)
+                    *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + (size_t)mm * N + n) = make_float4(v[0], v[1], v[2], v[3]);
+                else
+                    *reinterpret_cast<uint2*>(out + (size_t)mm * N + n) =
+                        make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
             };
             finish(g0, u0, m);
             if (two) finish(g1, u1, m + 4);
@@ -213,7 +217,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                    const __grid_constant__ CUtensorMap tmW1, float* __restrict__ scratch,
                    unsigned int* __restrict__ counters, bf16* __restrict__ out,
                    int M, int Mpad, int N, int num_tiles, int KB, int stages, uint32_t tmem_cols, int evict_first,
-                   GateAct act, int w_kmajor)
+                   GateAct act, int w_kmajor, int out_fp32)
 {
     constexpr int KERNEL_ID = GATEUP ? 3 : 4;
     constexpr int NMAT = GATEUP ? 2 : 1;
@@ -379,7 +383,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             if (!ok) break;
             skinny_epilogue_segment<GATEUP, NH>(tmem_base + lane_base + acc_col(buf, 0, 0), tempty0 + 8 * buf, tile,
                                                 tile == (int)(u_begin / KB), blockIdx.x, total, parts, KB, M, Mpad, N,
-                                                scratch, counters, out, slot_off, last_flag, et, nl, lane, act);
+                                                scratch, counters, out, slot_off, last_flag, et, nl, lane, act, out_fp32);
             u = seg_end;
         }
     }

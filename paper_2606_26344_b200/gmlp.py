@@ -23,6 +23,7 @@ FLAG_CHECKED = 1 << 2
 FLAG_ACT_SWISH = 1 << 5
 FLAG_ACT_GLU = 1 << 6
 FLAG_WEIGHTS_OUT_IN = 1 << 7
+FLAG_Y_FP32 = 1 << 8
 ACT_FLAGS = {"silu": 0, "swish": FLAG_ACT_SWISH, "glu": FLAG_ACT_GLU}
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA, VARIANT_SKINNY, VARIANT_PAIR, VARIANT_TENSOR = 0, 1, 2, 3, 4, 5, 6
 
@@ -212,15 +213,18 @@ def _check_bf16_cuda(t: torch.Tensor, name: str) -> None:
 def make_args(X, Wg, Wu, Wd, Y, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, variant: int = VARIANT_AUTO,
               workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
               checked: bool = False, act: str = "silu", beta: float = 1.0, weights_out_in: bool = False) -> GmlpArgs:
-    for t, n in ((X, "X"), (Wg, "Wg"), (Wu, "Wu"), (Wd, "Wd"), (Y, "Y")):
+    for t, n in ((X, "X"), (Wg, "Wg"), (Wu, "Wu"), (Wd, "Wd")):
         _check_bf16_cuda(t, n)
+    y_fp32 = Y.dtype == torch.float32              # a float32 Y asks for the unrounded down projection
+    if not (Y.is_cuda and Y.is_contiguous() and Y.dtype in (torch.bfloat16, torch.float32)):
+        raise TypeError("Y: expected a contiguous CUDA bfloat16 or float32 tensor")
     M, d_model = X.shape
     d_ff = Wg.shape[0] if weights_out_in else Wg.shape[1]
     w_up, w_down = ((d_ff, d_model), (d_model, d_ff)) if weights_out_in else ((d_model, d_ff), (d_ff, d_model))
     if Wg.shape != w_up or Wu.shape != w_up or Wd.shape != w_down or Y.shape != X.shape:
         raise ValueError("shape mismatch")
     flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0) | ACT_FLAGS[act] | \
-        (FLAG_WEIGHTS_OUT_IN if weights_out_in else 0)
+        (FLAG_WEIGHTS_OUT_IN if weights_out_in else 0) | (FLAG_Y_FP32 if y_fp32 else 0)
     if gamma is not None:
         _check_bf16_cuda(gamma, "gamma")
     st = stream if stream is not None else torch.cuda.current_stream(X.device)
