@@ -279,8 +279,9 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             const uint64_t policy = ptx::l2_policy_evict_first();
-            auto load_weights = [&](long long u, int s) {
-                const int tile = (int)(u / KB), kb = (int)(u % KB);
+            // (tile, k-block) of a unit are carried along and stepped, never recomputed: 64-bit divisions by a
+            // run-time KB cost this single thread hundreds of cycles per unit, as much as the unit's share of time
+            auto load_weights = [&](int tile, int kb, int s) {
                 const uint32_t full = full0 + 8 * s;
                 const uint32_t st = base + s * stage_bytes;
                 ptx::mbar_arrive_expect_tx(full, stage_bytes);
@@ -299,22 +300,26 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                             ptx::tma_load_2d(st + (j * NH * 2 + hb) * kSkinnyBoxBytes, j ? &tmW1 : &tmW0, cx, cy, full);
                     }
             };
-            auto load_tokens = [&](long long u, int s) {
-                ptx::tma_load_2d(base + s * stage_bytes + W_BYTES, &tmX, (int)(u % KB) * 64, 0, full0 + 8 * s);
+            auto load_tokens = [&](int kb, int s) {
+                ptx::tma_load_2d(base + s * stage_bytes + W_BYTES, &tmX, kb * 64, 0, full0 + 8 * s);
             };
+            auto step = [&](int& tile, int& kb) { if (++kb == KB) { kb = 0; ++tile; } };
+            const int tile0 = (int)(u_begin / KB), kb0 = (int)(u_begin % KB);
             // weights of the first ring-full of units do not depend on the previous kernel
             const long long n_units = u_end - u_begin;
             const int head = (int)(n_units < stages ? n_units : stages);
-            for (int i = 0; i < head; ++i) load_weights(u_begin + i, i);
+            int tile = tile0, kb = kb0;
+            for (int i = 0; i < head; ++i) { load_weights(tile, kb, i); step(tile, kb); }
             ptx::grid_dependency_wait();
-            for (int i = 0; i < head; ++i) load_tokens(u_begin + i, i);
-            int it = head;
-            for (long long u = u_begin + head; u < u_end; ++u, ++it) {
-                const int s = it % stages;
-                const uint32_t ph = (uint32_t)(it / stages) & 1u;
+            { int t2 = tile0, k2 = kb0; for (int i = 0; i < head; ++i) { load_tokens(k2, i); step(t2, k2); } }
+            int s = head == stages ? 0 : head;                     // ring slot and its phase, stepped as well
+            uint32_t ph = head == stages ? 1u : 0u;
+            for (long long u = u_begin + head; u < u_end; ++u) {
                 if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
-                load_weights(u, s);
-                load_tokens(u, s);
+                load_weights(tile, kb, s);
+                load_tokens(kb, s);
+                step(tile, kb);
+                if (++s == stages) { s = 0; ph ^= 1u; }
             }
         }
         __syncwarp();
@@ -325,12 +330,10 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             // (weights stored [N, K]: A is K-major too, bit 15 clear)
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((w_kmajor ? 0u : 1u) << 15) | (0u << 16) |
                                    ((uint32_t)(Mpad >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-            int it = 0, seg = 0;
+            int seg = 0, s = 0, kb = (int)(u_begin % KB);           // ring slot, its phase and the k-block are stepped
+            uint32_t ph = 0u;
             bool fresh = true;
-            for (long long u = u_begin; u < u_end; ++u, ++it) {
-                const int s = it % stages;
-                const uint32_t ph = (uint32_t)(it / stages) & 1u;
-                const int kb = (int)(u % KB);
+            for (long long u = u_begin; u < u_end; ++u) {
                 const int buf = seg & 1;
                 if (fresh) {
                     // the accumulator buffer must have been drained by the epilogue two segments ago
@@ -362,6 +365,8 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     ++seg;
                     fresh = true;
                 }
+                if (++kb == KB) kb = 0;
+                if (++s == stages) { s = 0; ph ^= 1u; }
             }
         }
         __syncwarp();
