@@ -265,12 +265,13 @@ struct Layout {
     SkinnyPlan s1, s2;
 };
 
-// Schedule choice for AUTO, from A/B timings on B200.  SKINNY (operand-swapped stream-K) only pays for a
-// handful of tokens: on small and medium layers the one-CTA-per-tile kernels have too few tiles to fill the
-// GPU, and on large layers the two are within a few percent (the 128-row tiles are ahead in short bursts,
-// SKINNY in long runs under the power cap, where issuing 128-row MMAs for 8 real rows costs clock).  From 9
-// tokens on the 128-row tcgen05 tiles win everywhere, because their down projection splits K over a cluster
-// and reduces on chip.  TENSOR then picks, per GEMM, between single-CTA tiles and CTA pairs.
+// Schedule choice for AUTO, from A/B timings on B200.  SKINNY (operand-swapped stream-K) pays for up to 16
+// tokens: on small and medium layers the one-CTA-per-tile kernels have too few tiles to fill the GPU (2048 x 5632,
+// M = 16: 26 vs 34 us), on large layers the two are within a few percent (8B layer, M = 16: 65.5 vs 66.2 us; 70B
+// layer: 219 vs 227 us).  Beyond that SKINNY's partial-sum traffic and last-arriver reduction grow with M and the
+// 128-row tcgen05 tiles win, because their down projection splits K over a cluster and reduces on chip (8B layer,
+// M = 32: 72 vs 67 us).  TENSOR then picks, per GEMM, between single-CTA tiles and CTA pairs.  gmlp_autotune
+// replaces this rule by a measurement for a given shape.
 struct TunedShape {
     int device;
     int64_t M, d_model, d_ff;
@@ -299,7 +300,7 @@ int resolve_variant(int64_t M, int64_t d_model, int64_t d_ff, int32_t variant) {
     if (variant != GMLP_VARIANT_AUTO) return variant;
     const int tuned = tuned_variant(M, d_model, d_ff);
     if (tuned != GMLP_VARIANT_AUTO) return tuned;
-    return M <= 8 ? GMLP_VARIANT_SKINNY : GMLP_VARIANT_TENSOR;
+    return M <= 16 ? GMLP_VARIANT_SKINNY : GMLP_VARIANT_TENSOR;
 }
 
 // TENSOR: which kernel each GEMM takes, by the number of 128-row blocks mt.  A CTA pair works on 256 rows, so an

@@ -51,11 +51,16 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16])
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Flat work sequence of `total` units cut into `parts` ranges: range c = [c*total/parts, (c+1)*total/parts).
+// (64-bit division is a long instruction sequence on the GPU; the products fit 32 bits for every realistic shape)
 __device__ __forceinline__ long long range_start(long long c, long long total, long long parts) {
-    return (c * total) / parts;
+    const unsigned long long num = (unsigned long long)c * (unsigned long long)total;
+    if ((num >> 32) == 0 && ((unsigned long long)parts >> 32) == 0) return (long long)((uint32_t)num / (uint32_t)parts);
+    return (long long)(num / (unsigned long long)parts);
 }
 __device__ __forceinline__ int range_owner(long long unit, long long total, long long parts) {
-    return (int)(((unit + 1) * parts - 1) / total);
+    const unsigned long long num = (unsigned long long)(unit + 1) * (unsigned long long)parts - 1;
+    if ((num >> 32) == 0 && ((unsigned long long)total >> 32) == 0) return (int)((uint32_t)num / (uint32_t)total);
+    return (int)(num / (unsigned long long)total);
 }
 
 // One segment (this CTA's share of one column tile's K range) as seen by the 128 epilogue threads:
@@ -67,7 +72,8 @@ __device__ __forceinline__ int range_owner(long long unit, long long total, long
 //   total/parts/KB  the flat work sequence (see range_start / range_owner) this phase was cut from
 template <bool GATEUP, int NH>
 __device__ __forceinline__ bool skinny_epilogue_segment(
-    uint32_t acc0, uint32_t tempty_bar, int tile, bool first_segment_of_cta, int cta, long long total, long long parts,
+    uint32_t acc0, uint32_t tempty_bar, int tile, int first_c, int last_c, bool first_segment_of_cta, int cta,
+    long long total, long long parts,
     int KB, int M, int Mpad, int N, float* __restrict__ scratch, unsigned int* __restrict__ counters,
     bf16* __restrict__ out, unsigned long long* slot_off, volatile int* last_flag, int et, int nl, int lane,
     const GateAct act, const int out_fp32)
@@ -75,9 +81,6 @@ __device__ __forceinline__ bool skinny_epilogue_segment(
     constexpr int NMAT = GATEUP ? 2 : 1;
     constexpr int TILE_N = 128 * NH;
     const size_t slot_floats = (size_t)NMAT * NH * Mpad * 128;
-    const long long tile_first = (long long)tile * KB;
-    const int first_c = range_owner(tile_first, total, parts);
-    const int last_c = range_owner(tile_first + KB - 1, total, parts);
     const int n_base = tile * TILE_N;
 
     if (first_c == last_c) {
@@ -377,17 +380,21 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         const int et = threadIdx.x - 64;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         int seg = 0;
+        int tile = (int)(u_begin / KB);
+        const int first_tile = tile;
         ptx::grid_dependency_wait();          // scratch, counters and `out` may still be in use by the previous kernel
-        for (long long u = u_begin; u < u_end; ++seg) {
-            const int tile = (int)(u / KB);
+        for (long long u = u_begin; u < u_end; ++seg, ++tile) {
             const long long tile_first = (long long)tile * KB;
             const long long seg_end = (tile_first + KB < u_end) ? tile_first + KB : u_end;
+            // who shares this tile: worked out while the accumulator is still being produced
+            const int first_c = range_owner(tile_first, total, parts);
+            const int last_c = range_owner(tile_first + KB - 1, total, parts);
             const int buf = seg & 1;
             const bool ok = wait_bounded(tfull0 + 8 * buf, ((uint32_t)seg >> 1) & 1u, abort_flag, KERNEL_ID, 3);
             ptx::tc_fence_after_sync();
             if (!ok) break;
             skinny_epilogue_segment<GATEUP, NH>(tmem_base + lane_base + acc_col(buf, 0, 0), tempty0 + 8 * buf, tile,
-                                                tile == (int)(u_begin / KB), blockIdx.x, total, parts, KB, M, Mpad, N,
+                                                first_c, last_c, tile == first_tile, blockIdx.x, total, parts, KB, M, Mpad, N,
                                                 scratch, counters, out, slot_off, last_flag, et, nl, lane, act, out_fp32);
             u = seg_end;
         }

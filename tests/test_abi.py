@@ -106,10 +106,10 @@ def test_workspace_sizes_and_variant_choice(lib):
     # AUTO: the operand-swapped stream-K schedule for a handful of tokens, else the 128-row tensor-core tiles
     # with a per-GEMM kernel choice
     assert gmlp.pick_variant(1, 2048, 5632) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(8, 2048, 5632) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(9, 2048, 5632) == gmlp.VARIANT_TENSOR
+    assert gmlp.pick_variant(16, 2048, 5632) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(17, 2048, 5632) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(8, dm, dff) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(16, dm, dff) == gmlp.VARIANT_TENSOR
+    assert gmlp.pick_variant(32, dm, dff) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(129, 2048, 5632) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(2048, dm, dff) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(4096, 8192, 28672) == gmlp.VARIANT_TENSOR
