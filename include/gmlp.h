@@ -27,6 +27,11 @@
  * workspace is passed; with workspace == NULL it uses a library-owned buffer that grows on
  * demand (cudaMalloc on the calling thread's current device) and is freed by
  * gmlp_shutdown().
+ * A caller-made workspace belongs to the library between calls: the small-M schedules keep arrival
+ * counters in it, which the library zeroes the first time it sees a (pointer, size) and which its kernels
+ * leave zero after every call, so later calls with the same workspace start without a memset.  If
+ * anything else writes to that memory between two calls (the buffer was freed and handed out again by an
+ * allocator, reused as scratch, ...), tell the library with gmlp_workspace_forget() before the next call.
  *
  * Errors: every entry point returns a gmlp_status code; nothing throws, aborts or prints.
  * Calls are asynchronous on the given stream: device-side problems (a bounded wait that
@@ -297,6 +302,14 @@ int gmlp_forward_static(const void* X, const void* Wg, const void* Wu, const voi
  * the small-M schedule.  Returns 0 for invalid shapes.
  */
 uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant);
+
+/*
+ * Drop what the library remembers about the contents of caller-made workspaces on the current device (the
+ * arrival counters it believes to be zero; see "Ownership" above): those inside [workspace, workspace + bytes),
+ * or all of them when `workspace` is NULL.  The next call that uses such a workspace zeroes its counters again
+ * (one cudaMemsetAsync on the call's stream).  Host-side bookkeeping only; returns GMLP_OK or GMLP_ERR_ARCH.
+ */
+int gmlp_workspace_forget(const void* workspace, uint64_t bytes);
 
 /*
  * Empirical schedule selection for one shape (the paper's extraction phase keeps, among the candidate kernels

@@ -1487,6 +1487,22 @@ int gmlp_autotune_query(int64_t M, int64_t d_model, int64_t d_ff, int32_t* varia
     return 1;
 }
 
+int gmlp_workspace_forget(const void* workspace, uint64_t bytes) {
+    int rc = GMLP_OK;
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const uint8_t* w = static_cast<const uint8_t*>(workspace);
+    for (int i = 0; i < DeviceState::kCleanSlots; ++i) {
+        const uint8_t* c = static_cast<const uint8_t*>(dev->clean_counters[i]);
+        if (c != nullptr && (w == nullptr || (c >= w && (uint64_t)(c - w) < bytes))) {
+            dev->clean_counters[i] = nullptr;
+            dev->clean_counters_bytes[i] = 0;
+        }
+    }
+    return GMLP_OK;
+}
+
 void gmlp_autotune_clear(void) {
     std::lock_guard<std::mutex> lock(g_mutex);
     g_tuned.clear();

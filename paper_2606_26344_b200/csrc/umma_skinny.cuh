@@ -52,6 +52,10 @@ __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;"
 
 // Flat work sequence of `total` units cut into `parts` ranges: range c = [c*total/parts, (c+1)*total/parts).
 // (64-bit division is a long instruction sequence on the GPU; the products fit 32 bits for every realistic shape)
+__device__ __forceinline__ long long div_fast(long long a, int b) {          // a >= 0, b > 0
+    if (((unsigned long long)a >> 32) == 0) return (long long)((uint32_t)a / (uint32_t)b);
+    return a / b;
+}
 __device__ __forceinline__ long long range_start(long long c, long long total, long long parts) {
     const unsigned long long num = (unsigned long long)c * (unsigned long long)total;
     if ((num >> 32) == 0 && ((unsigned long long)parts >> 32) == 0) return (long long)((uint32_t)num / (uint32_t)parts);
@@ -148,7 +152,7 @@ __device__ __forceinline__ bool skinny_epilogue_segment(
     const int ncontrib = last_c - first_c + 1;
     for (int i = et; i < ncontrib; i += 128) {
         const int c = first_c + i;
-        const int cslot = ((int)(range_start(c, total, parts) / KB) == tile) ? 0 : 1;
+        const int cslot = ((int)div_fast(range_start(c, total, parts), KB) == tile) ? 0 : 1;
         slot_off[i] = ((unsigned long long)c * 2 + cslot) * slot_floats;
     }
     epi_bar_sync();
@@ -307,7 +311,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 ptx::tma_load_2d(base + s * stage_bytes + W_BYTES, &tmX, kb * 64, 0, full0 + 8 * s);
             };
             auto step = [&](int& tile, int& kb) { if (++kb == KB) { kb = 0; ++tile; } };
-            const int tile0 = (int)(u_begin / KB), kb0 = (int)(u_begin % KB);
+            const int tile0 = (int)div_fast(u_begin, KB), kb0 = (int)(u_begin - (long long)tile0 * KB);
             // weights of the first ring-full of units do not depend on the previous kernel
             const long long n_units = u_end - u_begin;
             const int head = (int)(n_units < stages ? n_units : stages);
@@ -333,7 +337,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             // (weights stored [N, K]: A is K-major too, bit 15 clear)
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((w_kmajor ? 0u : 1u) << 15) | (0u << 16) |
                                    ((uint32_t)(Mpad >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-            int seg = 0, s = 0, kb = (int)(u_begin % KB);           // ring slot, its phase and the k-block are stepped
+            int seg = 0, s = 0, kb = (int)(u_begin - div_fast(u_begin, KB) * KB);   // ring slot, its phase and the k-block are stepped
             uint32_t ph = 0u;
             bool fresh = true;
             for (long long u = u_begin; u < u_end; ++u) {
@@ -380,7 +384,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         const int et = threadIdx.x - 64;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         int seg = 0;
-        int tile = (int)(u_begin / KB);
+        int tile = (int)div_fast(u_begin, KB);
         const int first_tile = tile;
         ptx::grid_dependency_wait();          // scratch, counters and `out` may still be in use by the previous kernel
         for (long long u = u_begin; u < u_end; ++seg, ++tile) {

@@ -131,6 +131,8 @@ def lib() -> ctypes.CDLL:
         L.gmlp_autotune_query.argtypes = [i64, i64, i64] + [ctypes.POINTER(ctypes.c_int32)] * 3
         L.gmlp_autotune_clear.restype = None
         L.gmlp_autotune_clear.argtypes = []
+        L.gmlp_workspace_forget.restype = ctypes.c_int
+        L.gmlp_workspace_forget.argtypes = [ctypes.c_void_p, ctypes.c_uint64]
         L.gmlp_pick_variant.restype = ctypes.c_int
         L.gmlp_pick_variant.argtypes = [i64, i64, i64, u32]
         L.gmlp_device_status.restype = ctypes.c_int
@@ -247,7 +249,12 @@ def make_args(X, Wg, Wu, Wd, Y, gamma=None, eps: float = 1e-5, rmsnorm: bool = F
 def alloc_workspace(M: int, d_model: int, d_ff: int, rmsnorm: bool = False, variant: int = VARIANT_AUTO,
                     device="cuda") -> torch.Tensor:
     n = workspace_bytes(M, d_model, d_ff, FLAG_RMSNORM if rmsnorm else 0, variant)
-    return torch.empty(n + 256, dtype=torch.uint8, device=device)[:n] if n else torch.empty(256, dtype=torch.uint8, device=device)
+    ws = torch.empty(n + 256, dtype=torch.uint8, device=device)[:n] if n else torch.empty(256, dtype=torch.uint8, device=device)
+    # the caching allocator may hand out memory the library saw as a workspace before and that other tensors have
+    # written since: what the library remembers about it (counters it left at zero) no longer holds
+    with torch.cuda.device(ws.device):
+        lib().gmlp_workspace_forget(ws.data_ptr(), ws.numel())
+    return ws
 
 
 def forward_ex(args: GmlpArgs) -> None:

@@ -206,6 +206,28 @@ def test_workspace_too_small_is_rejected_and_results_are_deterministic():
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
 
 
+def test_workspace_written_by_someone_else_is_usable_again_after_forget():
+    # the small-M schedules keep arrival counters in the workspace and rely on finding them zero; a caller that
+    # lets other work write to the workspace says so with gmlp_workspace_forget, and the next call re-zeroes them
+    inp = I.custom_inputs(8, 512, 1024, 77)
+    t = to_device(inp)
+    n = gmlp.workspace_bytes(8, 512, 1024, 0, SKINNY)
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+    gmlp.lib().gmlp_workspace_forget(ws.data_ptr(), n)
+    Y0 = gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], variant=SKINNY, workspace=ws, checked=True)
+    ws.fill_(0xFF)                                           # foreign writes
+    assert gmlp.lib().gmlp_workspace_forget(ws.data_ptr(), n) == gmlp.OK
+    Y1 = gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], variant=SKINNY, workspace=ws, checked=True)
+    torch.cuda.synchronize()
+    assert torch.equal(Y0.view(torch.int16), Y1.view(torch.int16))
+    ws.fill_(0x5A)
+    assert gmlp.lib().gmlp_workspace_forget(None, 0) == gmlp.OK          # NULL: every remembered workspace
+    Y2 = gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], variant=SKINNY, workspace=ws, checked=True)
+    torch.cuda.synchronize()
+    assert torch.equal(Y0.view(torch.int16), Y2.view(torch.int16))
+    assert gmlp.device_status() == 0
+
+
 def test_host_buffer_entry_point_matches_device_entry_point():
     inp = I.custom_inputs(33, 256, 512, 6)
     t = to_device(inp)
