@@ -98,7 +98,8 @@ def _load():
         lib.gmlp_oracle_matmul_rows.argtypes = [u16p, u16p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, i64p,
                                                 ctypes.c_int64, f64p, ctypes.c_int]
         lib.gmlp_oracle_gqa_rows.restype = ctypes.c_int
-        lib.gmlp_oracle_gqa_rows.argtypes = [u16p, u16p, u16p] + [ctypes.c_int64] * 5 + [i64p, ctypes.c_int64, f64p, ctypes.c_int]
+        lib.gmlp_oracle_gqa_rows.argtypes = [u16p, u16p, u16p] + [ctypes.c_int64] * 5 + [i64p, ctypes.c_int64, f64p, ctypes.c_int,
+                                             ctypes.c_int]
         lib.gmlp_oracle_gate_up_rows_act.restype = ctypes.c_int
         lib.gmlp_oracle_gate_up_rows_act.argtypes = lib.gmlp_oracle_gate_up_rows.argtypes + [ctypes.c_int, ctypes.c_double]
         lib.gmlp_oracle_rmsnorm_matmul_rows.restype = ctypes.c_int
@@ -335,7 +336,7 @@ def qkv_rows(X, Wq, Wk, Wv, rows=None, num_threads: int = 0):
     return tuple(matmul_rows(X, W, rows, num_threads) for W in (Wq, Wk, Wv))
 
 
-def gqa_rows(Q, K, V, n_q_heads: int, n_kv_heads: int, rows=None, num_threads: int = 0) -> np.ndarray:
+def gqa_rows(Q, K, V, n_q_heads: int, n_kv_heads: int, rows=None, num_threads: int = 0, causal: bool = False) -> np.ndarray:
     """Reference group query attention (float64) for the selected query rows.
 
     Q [M, Hq*D], K and V [S, Hkv*D] bf16 bit patterns; returns O_ref [len(rows), Hq*D]."""
@@ -353,7 +354,7 @@ def gqa_rows(Q, K, V, n_q_heads: int, n_kv_heads: int, rows=None, num_threads: i
     O = np.zeros((rows.size, n_q_heads * D), dtype=np.float64)
     rc = lib.gmlp_oracle_gqa_rows(_p(Q, ctypes.c_uint16), _p(K, ctypes.c_uint16), _p(V, ctypes.c_uint16), M, S,
                                   n_q_heads, n_kv_heads, D, _p(rows, ctypes.c_int64), rows.size, _p(O, ctypes.c_double),
-                                  int(num_threads))
+                                  int(num_threads), int(bool(causal)))
     if rc != 0:
         raise RuntimeError(f"gmlp_oracle_gqa_rows failed ({rc})")
     return O

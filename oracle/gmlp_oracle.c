@@ -430,13 +430,17 @@ int gmlp_oracle_matmul_rows(const uint16_t* X, const uint16_t* W, int64_t M, int
  * Q [M, Hq*D], K and V [S, Hkv*D], O [M, Hq*D] row-major (head h occupies columns [h*D, (h+1)*D)); bf16 bit
  * patterns in, everything in fp64, softmax written out as max-subtracted exponentials over their sum, O left in
  * fp64.  For the selected query rows: O_ref [n_rows, Hq*D].
+ * causal != 0 (an extension; decoder models use it): query row m sees keys s <= m + (S - M) only, i.e. the
+ * queries are the LAST M positions of the S-long sequence (needs S >= M); masked scores take no part in the
+ * softmax.
  */
 int gmlp_oracle_gqa_rows(const uint16_t* Q, const uint16_t* K, const uint16_t* V, int64_t M, int64_t S,
                          int64_t Hq, int64_t Hkv, int64_t D, const int64_t* rows, int64_t n_rows,
-                         double* O_ref, int num_threads)
+                         double* O_ref, int num_threads, int causal)
 {
     if (!Q || !K || !V || !rows || !O_ref || M < 0 || S <= 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || n_rows < 0) return -1;
     if (Hq % Hkv != 0) return -1;
+    if (causal && S < M) return -1;
     for (int64_t i = 0; i < n_rows; ++i)
         if (rows[i] < 0 || rows[i] >= M) return -1;
     const int64_t group = Hq / Hkv;
@@ -459,8 +463,9 @@ int gmlp_oracle_gqa_rows(const uint16_t* Q, const uint16_t* K, const uint16_t* V
                 for (int64_t h = 0; h < Hq; ++h) {
                     const uint16_t* q = Q + rows[i] * Hq * D + h * D;
                     const int64_t g = h / group;
+                    const int64_t S_vis = causal ? rows[i] + (S - M) + 1 : S;      /* keys this row may see */
                     double mx = -INFINITY;
-                    for (int64_t s = 0; s < S; ++s) {
+                    for (int64_t s = 0; s < S_vis; ++s) {
                         const uint16_t* k = K + s * Hkv * D + g * D;
                         double dot = 0.0;
                         for (int64_t d = 0; d < D; ++d) dot += gmlp_oracle_bf16_to_double(q[d]) * gmlp_oracle_bf16_to_double(k[d]);
@@ -468,13 +473,13 @@ int gmlp_oracle_gqa_rows(const uint16_t* Q, const uint16_t* K, const uint16_t* V
                         if (p[s] > mx) mx = p[s];
                     }
                     double sum = 0.0;
-                    for (int64_t s = 0; s < S; ++s) {
+                    for (int64_t s = 0; s < S_vis; ++s) {
                         p[s] = exp(p[s] - mx);
                         sum += p[s];
                     }
                     double* o = O_ref + i * Hq * D + h * D;
                     for (int64_t d = 0; d < D; ++d) o[d] = 0.0;
-                    for (int64_t s = 0; s < S; ++s) {
+                    for (int64_t s = 0; s < S_vis; ++s) {
                         const double w = p[s] / sum;
                         const uint16_t* v = V + s * Hkv * D + g * D;
                         for (int64_t d = 0; d < D; ++d) o[d] += w * gmlp_oracle_bf16_to_double(v[d]);

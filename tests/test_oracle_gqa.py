@@ -100,3 +100,41 @@ def test_head_to_group_mapping_and_bad_arguments():
         oracle.gqa_rows(_bits(Q), _bits(K[:, :D]), _bits(V[:, :D]), 4, 3 if False else 1, rows=np.array([9]))
     with pytest.raises(ValueError):
         oracle.gqa_rows(_bits(Q), _bits(K), _bits(V[:, :D]), Hq, Hkv)
+
+
+def _torch_ref_causal(Q, K, V, Hq, Hkv):
+    M, S = Q.shape[0], K.shape[0]
+    D = Q.shape[1] // Hq
+    q = Q.double().view(M, Hq, D).transpose(0, 1)
+    k = K.double().view(S, Hkv, D).transpose(0, 1).repeat_interleave(Hq // Hkv, dim=0)
+    v = V.double().view(S, Hkv, D).transpose(0, 1).repeat_interleave(Hq // Hkv, dim=0)
+    mask = torch.arange(S)[None, :] <= (torch.arange(M)[:, None] + (S - M))          # bottom-right aligned
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v, attn_mask=mask)
+    return o.transpose(0, 1).reshape(M, Hq * D).numpy()
+
+
+@pytest.mark.parametrize("shape", [(6, 6, 4, 2, 8), (3, 11, 2, 1, 16), (1, 5, 2, 2, 8)])
+def test_causal_against_the_library_attention_and_closed_forms(shape):
+    M, S, Hq, Hkv, D = shape
+    Q, K, V = _case(*shape, seed=21)
+    O = oracle.gqa_rows(_bits(Q), _bits(K), _bits(V), Hq, Hkv, causal=True)
+    assert np.allclose(O, _torch_ref_causal(Q, K, V, Hq, Hkv), rtol=1e-12, atol=1e-13)
+    if M == S:
+        # the first query sees the first key only: its output is that key's value; the last one sees everything
+        want0 = V[:1].double().view(1, Hkv, D).repeat_interleave(Hq // Hkv, dim=1).reshape(Hq * D).numpy()
+        assert np.allclose(O[0], want0, rtol=1e-15, atol=0)
+        full = oracle.gqa_rows(_bits(Q), _bits(K), _bits(V), Hq, Hkv)
+        assert np.array_equal(O[-1], full[-1]) and not np.allclose(O[0], full[0], rtol=1e-3, atol=1e-3)
+    # keys beyond a row's horizon do not matter to it
+    K2, V2 = K.clone(), V.clone()
+    K2[-1] += 3.0
+    V2[-1] -= 5.0
+    O2 = oracle.gqa_rows(_bits(Q), _bits(K2), _bits(V2), Hq, Hkv, causal=True)
+    if M > 1:
+        assert np.array_equal(O2[:-1], O[:-1])
+
+
+def test_causal_needs_at_least_as_many_keys_as_queries():
+    Q, K, V = _case(4, 3, 2, 1, 8, seed=22)
+    with pytest.raises(RuntimeError):
+        oracle.gqa_rows(_bits(Q), _bits(K), _bits(V), 2, 1, causal=True)
