@@ -458,20 +458,25 @@ def measure_gqa(dev, peaks, iters=10):
             K = torch.randn(T, Hkv * 128, generator=g).bfloat16().to(dev)
             V = torch.randn(T, Hkv * 128, generator=g).bfloat16().to(dev)
             O = torch.empty_like(Q)
-            a = gmlp.make_gqa_args(Q, K, V, O, Hq, Hkv)
-            for _ in range(3):
-                gmlp.gqa_attention_ex(a)
-            torch.cuda.synchronize(dev)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(iters):
-                gmlp.gqa_attention_ex(a)
-            e1.record()
-            torch.cuda.synchronize(dev)
-            us = e0.elapsed_time(e1) / iters * 1e3
+            res = {}
+            for causal in (False, True):
+                a = gmlp.make_gqa_args(Q, K, V, O, Hq, Hkv, causal=causal)
+                for _ in range(3):
+                    gmlp.gqa_attention_ex(a)
+                torch.cuda.synchronize(dev)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(iters):
+                    gmlp.gqa_attention_ex(a)
+                e1.record()
+                torch.cuda.synchronize(dev)
+                res[causal] = e0.elapsed_time(e1) / iters * 1e3
+            us = res[False]
             tf = 4.0 * T * T * 128 * Hq / us / 1e6
+            tf_causal = 4.0 * (T * (T + 1) / 2) * 128 * Hq / res[True] / 1e6        # visible (query, key) pairs only
             rows.append({"shape": label, "M": T, "S": T, "n_q_heads": Hq, "n_kv_heads": Hkv, "us": us, "tflops": tf,
-                         "frac_of_bf16_peak": tf / peaks["bf16_tflops"]})
+                         "frac_of_bf16_peak": tf / peaks["bf16_tflops"], "causal_us": res[True],
+                         "causal_tflops": tf_causal})
             del Q, K, V, O
     return {"timing": "back-to-back calls", "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst bf16)",
             "best_tflops": max(r["tflops"] for r in rows), "table": rows}

@@ -239,10 +239,14 @@ int gmlp_qkv_proj(const gmlp_qkv_args* args);
  * probabilities are rounded to bf16 for the second matmul, O is rounded once.  head_dim must be 128
  * (GMLP_ERR_UNSUPPORTED otherwise); n_q_heads a multiple of n_kv_heads.  One tcgen05 kernel, online softmax, the
  * scores never leave the SM.  No workspace.
+ * GMLP_GQA_CAUSAL (an extension; the paper's kernel has no mask): query row m sees keys s <= m + (S - M) only -
+ * the queries are the last M positions of the S-long sequence; needs S >= M (GMLP_ERR_SHAPE otherwise).  Key
+ * blocks beyond a query tile's horizon are skipped.
  */
+enum { GMLP_GQA_CAUSAL = 1u << 4 };
 typedef struct gmlp_gqa_args {
     uint32_t struct_bytes;    /* sizeof(gmlp_gqa_args) */
-    uint32_t flags;           /* GMLP_FLAG_CHECKED */
+    uint32_t flags;           /* GMLP_FLAG_CHECKED | GMLP_GQA_CAUSAL */
     const void* Q;            /* device, [M, n_q_heads*head_dim] bf16 */
     const void* K;            /* device, [S, n_kv_heads*head_dim] bf16 */
     const void* V;            /* device, [S, n_kv_heads*head_dim] bf16 */

@@ -1303,7 +1303,8 @@ int qkv_proj_impl(const gmlp_qkv_args* a) {
 int gqa_attention_impl(const gmlp_gqa_args* a) {
     if (a == nullptr) return GMLP_ERR_NULL;
     if (a->struct_bytes != sizeof(gmlp_gqa_args)) return GMLP_ERR_FLAGS;
-    if ((a->flags & ~(uint32_t)GMLP_FLAG_CHECKED) || a->reserved != 0) return GMLP_ERR_FLAGS;
+    if ((a->flags & ~(uint32_t)(GMLP_FLAG_CHECKED | GMLP_GQA_CAUSAL)) || a->reserved != 0) return GMLP_ERR_FLAGS;
+    if ((a->flags & GMLP_GQA_CAUSAL) && a->S < a->M) return GMLP_ERR_SHAPE;
     if (a->M < 0 || a->S <= 0 || a->n_q_heads <= 0 || a->n_kv_heads <= 0 || a->n_q_heads % a->n_kv_heads != 0 ||
         a->M > (1 << 30) || a->S > (1 << 30) || a->n_q_heads > 65535)
         return GMLP_ERR_SHAPE;
@@ -1340,7 +1341,9 @@ int gqa_attention_impl(const gmlp_gqa_args* a) {
     const int Mi = (int)a->M, Si = (int)a->S, Hq = (int)a->n_q_heads, group = (int)(a->n_q_heads / a->n_kv_heads);
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)gmlp::kGqaD);      // log2(e) / sqrt(D)
     bf16* O = static_cast<bf16*>(a->O);
-    if (cudaLaunchKernelEx(&cfg, gmlp::gqa_attention_kernel, tmQ, tmK, tmV, O, Mi, Si, Hq, group, scale_log2) != cudaSuccess)
+    const int causal_off = (a->flags & GMLP_GQA_CAUSAL) ? (int)(a->S - a->M) : -1;
+    if (cudaLaunchKernelEx(&cfg, gmlp::gqa_attention_kernel, tmQ, tmK, tmV, O, Mi, Si, Hq, group, scale_log2, causal_off) !=
+        cudaSuccess)
         return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     prof_mark("gqa", st);

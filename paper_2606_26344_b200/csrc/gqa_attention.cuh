@@ -60,7 +60,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
 __global__ void __launch_bounds__(kGqaThreads, 1)
 gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, bf16* __restrict__ O,
-                     int M, int S, int n_q_heads, int group, float scale_log2)
+                     int M, int S, int n_q_heads, int group, float scale_log2, int causal_off)
 {
     constexpr int KERNEL_ID = 10;
     // S = Q K^T: A and B K-major;  O += P V: A K-major, B MN-major;  both M = 128, N = 128, fp32 accumulate
@@ -87,10 +87,14 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kGqaBM;
+    // causal: the query tiles with the longest horizons (the most key blocks) are started first
+    const int m0 = (causal_off >= 0 ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x) * kGqaBM;
     const int h = blockIdx.y;
     const int g = h / group;
-    const int n_blocks = (S + kGqaBS - 1) / kGqaBS;
+    // causal_off >= 0: causal attention, query row m sees keys s <= m + causal_off (causal_off = S - M: the queries
+    // are the last M positions); blocks entirely beyond the horizon of this CTA's last row are not visited
+    int n_blocks = (S + kGqaBS - 1) / kGqaBS;
+    if (causal_off >= 0) n_blocks = min(n_blocks, (m0 + kGqaBM - 1 + causal_off) / kGqaBS + 1);
 
     ptx::launch_dependents();
     if (threadIdx.x == 0) {
@@ -211,6 +215,8 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         uint8_t* p_row = base_ptr + (2 + t) * kGqaTileBytes + (size_t)r * 128;
         float m_use = -INFINITY, l_run = 0.0f;                       // exponent base, row sum
         bool ok = true;
+        // last key this row may see (causal), or none of that
+        const int horizon = causal_off >= 0 ? m0 + 128 * t + r + causal_off : 0x7FFFFFFF - kGqaBS;
 
         // one pass over the block's scores with base m_use: P to shared memory, row sum and row maximum.  The
         // next 32 scores are on their way from TMEM while the current 32 are processed; the scale is folded into
@@ -258,10 +264,11 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             // P of the previous block must have been consumed (and O complete) before P is overwritten
             if (j > 0 && !wait_bounded(o_full0 + 8 * t, (uint32_t)(j - 1) & 1u, abort_flag, KERNEL_ID, 4)) { ok = false; break; }
             ptx::tc_fence_after_sync();
-            const int valid = min(kGqaBS, S - j * kGqaBS);           // keys of this block that exist
+            // keys of this block that exist and that this row may see (0 when the whole block is beyond its horizon)
+            const int valid = max(0, min(min(kGqaBS, S - j * kGqaBS), horizon - j * kGqaBS + 1));
             float l_blk, m_blk;
             if (j == 0) {
-                // first block: find the base first (finite: the block has at least one key)
+                // first block: find the base first (finite: every row sees at least key 0)
                 float m0v = -INFINITY;
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {

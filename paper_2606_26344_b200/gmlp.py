@@ -56,6 +56,7 @@ class GmlpRmsmmArgs(ctypes.Structure):
 RMSMM_UNFUSED = 1 << 4
 MMADDNORM_UNFUSED = 1 << 4
 QKV_SEPARATE = 1 << 4
+GQA_CAUSAL = 1 << 4
 
 
 class GmlpGqaArgs(ctypes.Structure):
@@ -489,7 +490,8 @@ def qkv_proj(X, Wq, Wk, Wv, separate: bool = False, stream=None, checked: bool =
     return Q, K, V
 
 
-def make_gqa_args(Q, K, V, O, n_q_heads: int, n_kv_heads: int, stream=None, checked: bool = False) -> GmlpGqaArgs:
+def make_gqa_args(Q, K, V, O, n_q_heads: int, n_kv_heads: int, stream=None, checked: bool = False,
+                  causal: bool = False) -> GmlpGqaArgs:
     for t, n in ((Q, "Q"), (K, "K"), (V, "V"), (O, "O")):
         _check_bf16_cuda(t, n)
     M, S = Q.shape[0], K.shape[0]
@@ -499,7 +501,7 @@ def make_gqa_args(Q, K, V, O, n_q_heads: int, n_kv_heads: int, stream=None, chec
     st = stream if stream is not None else torch.cuda.current_stream(Q.device)
     a = GmlpGqaArgs()
     a.struct_bytes = ctypes.sizeof(GmlpGqaArgs)
-    a.flags = FLAG_CHECKED if checked else 0
+    a.flags = (FLAG_CHECKED if checked else 0) | (GQA_CAUSAL if causal else 0)
     a.Q, a.K, a.V, a.O = Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr()
     a.M, a.S = M, S
     a.n_q_heads, a.n_kv_heads, a.head_dim, a.reserved = n_q_heads, n_kv_heads, D, 0
@@ -513,10 +515,11 @@ def gqa_attention_ex(args: GmlpGqaArgs) -> None:
         raise GmlpError(rc)
 
 
-def gqa_attention(Q, K, V, n_q_heads: int, n_kv_heads: int, O=None, stream=None, checked: bool = False) -> torch.Tensor:
-    """gmlp_gqa_attention: O_h = softmax(Q_h K_g^T / sqrt(D)) V_g, no mask, D = 128."""
+def gqa_attention(Q, K, V, n_q_heads: int, n_kv_heads: int, O=None, stream=None, checked: bool = False,
+                  causal: bool = False) -> torch.Tensor:
+    """gmlp_gqa_attention: O_h = softmax(Q_h K_g^T / sqrt(D)) V_g, D = 128; no mask, or causal (queries = last M positions)."""
     if O is None:
         O = torch.empty_like(Q)
     with torch.cuda.device(Q.device):
-        gqa_attention_ex(make_gqa_args(Q, K, V, O, n_q_heads, n_kv_heads, stream, checked))
+        gqa_attention_ex(make_gqa_args(Q, K, V, O, n_q_heads, n_kv_heads, stream, checked, causal))
     return O

@@ -25,15 +25,17 @@ def _case(M, S, Hq, Hkv, seed, q_scale=1.0):
     return Q, K, V
 
 
-def _check(M, S, Hq, Hkv, seed, q_scale=1.0, max_rows=64):
+def _check(M, S, Hq, Hkv, seed, q_scale=1.0, max_rows=64, causal=False):
     Q, K, V = _case(M, S, Hq, Hkv, seed, q_scale)
     dev = torch.device("cuda")
     O = torch.full((M, Hq * D), float("nan"), dtype=torch.bfloat16, device=dev)
-    gmlp.gqa_attention(Q.to(dev), K.to(dev), V.to(dev), Hq, Hkv, O=O, checked=True)
+    gmlp.gqa_attention(Q.to(dev), K.to(dev), V.to(dev), Hq, Hkv, O=O, checked=True, causal=causal)
     torch.cuda.synchronize()
     assert bool(torch.isfinite(O.float()).all())
     rows = np.arange(M) if M <= max_rows else np.sort(np.random.default_rng(seed).choice(M, max_rows, replace=False))
-    ref = oracle.gqa_rows(_bits(Q), _bits(K), _bits(V), Hq, Hkv, rows=rows)
+    if causal and M > max_rows:          # the first and the last rows of the mask matter most
+        rows = np.unique(np.concatenate([rows, np.arange(4), np.arange(M - 4, M), np.array([127, 128, 255, 256])[:0 if M < 257 else 4]]))
+    ref = oracle.gqa_rows(_bits(Q), _bits(K), _bits(V), Hq, Hkv, rows=rows, causal=causal)
     got = O[torch.as_tensor(rows, device=dev)].float().cpu().numpy().astype(np.float64)
     e = np.abs(got - ref) / oracle.tolerance(ref)
     assert e.max() <= 1.0, f"max err/tol {e.max():.3f}"
@@ -44,6 +46,26 @@ def _check(M, S, Hq, Hkv, seed, q_scale=1.0, max_rows=64):
                                    (129, 1000, 6, 3), (256, 1024, 4, 1), (1030, 64, 2, 2)])
 def test_small_and_ragged(shape):
     _check(*shape, seed=50 + shape[0])
+
+
+@pytest.mark.parametrize("shape", [(128, 128, 2, 1), (1, 1, 1, 1), (1, 300, 4, 4), (17, 200, 4, 2), (300, 300, 8, 2),
+                                   (129, 1000, 6, 3), (256, 256, 4, 1), (700, 700, 2, 2), (1030, 1100, 2, 1)])
+def test_causal_small_and_ragged(shape):
+    _check(*shape, seed=150 + shape[0], causal=True)
+
+
+def test_causal_llama_like_block_and_first_rows_exact():
+    _check(2048, 2048, 32, 8, seed=4, causal=True)
+    # row 0 sees key 0 only: its output is V[0] of its group exactly
+    dev = torch.device("cuda")
+    Q, K, V = _case(300, 300, 4, 2, 8)
+    O = gmlp.gqa_attention(Q.to(dev), K.to(dev), V.to(dev), 4, 2, checked=True, causal=True).cpu()
+    want = V[:1].view(1, 2, D).repeat_interleave(2, dim=1).reshape(4 * D)
+    assert torch.equal(O[0].view(torch.int16), want.contiguous().view(torch.int16))
+    # S < M is refused
+    with pytest.raises(gmlp.GmlpError) as e:
+        gmlp.gqa_attention(Q.to(dev), K[:200].to(dev), V[:200].to(dev), 4, 2, causal=True)
+    assert e.value.status == gmlp.ERR_SHAPE
 
 
 def test_peaked_softmax_and_large_scores():
