@@ -228,6 +228,33 @@ def test_workspace_written_by_someone_else_is_usable_again_after_forget():
     assert gmlp.device_status() == 0
 
 
+@pytest.mark.parametrize("variant,M", [(SKINNY, 8), (TENSOR, 100)])
+def test_two_streams_with_their_own_workspaces_do_not_disturb_each_other(variant, M):
+    # two lanes (stream + workspace + buffers each) with different inputs, calls interleaved and overlapping on
+    # the GPU; every result must equal the one the same lane produces when it runs alone
+    dm, dff = 1024, 2816
+    lanes = []
+    for seed in (21, 22):
+        inp = I.custom_inputs(M, dm, dff, seed)
+        t = to_device(inp)
+        st = torch.cuda.Stream()
+        ws = gmlp.alloc_workspace(M, dm, dff, False, variant)
+        Y = torch.empty_like(t["X"])
+        alone = gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], variant=variant, checked=True).clone()
+        lanes.append((gmlp.make_args(t["X"], t["Wg"], t["Wu"], t["Wd"], Y, variant=variant, workspace=ws, stream=st), t, Y, alone, ws))
+    torch.cuda.synchronize()
+    for it in range(40):
+        for args, _, Y, alone, _ in lanes:
+            gmlp.forward_ex(args)
+        if it % 10 == 9:
+            torch.cuda.synchronize()
+            for _, _, Y, alone, _ in lanes:
+                assert torch.equal(Y.view(torch.int16), alone.view(torch.int16))
+                Y.fill_(float("nan"))
+    torch.cuda.synchronize()
+    assert gmlp.device_status() == 0
+
+
 def test_host_buffer_entry_point_matches_device_entry_point():
     inp = I.custom_inputs(33, 256, 512, 6)
     t = to_device(inp)
