@@ -225,16 +225,16 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             const bool masked = valid < kGqaBS;
             const float neg_base = -m_use;
             float l_acc = 0.0f, m_raw = -INFINITY;
-            uint32_t v[2][32];
-            ptx::tmem_ld_32x32(s_addr, v[0]);
+            uint32_t v[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(s_addr + 32 * c, v[c]);
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                if (c + 1 < 4) ptx::tmem_ld_32x32(s_addr + 32 * (c + 1), v[(c + 1) & 1]);
                 uint32_t packed[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    float x0 = __uint_as_float(v[c & 1][2 * i]), x1 = __uint_as_float(v[c & 1][2 * i + 1]);
+                    float x0 = __uint_as_float(v[c][2 * i]), x1 = __uint_as_float(v[c][2 * i + 1]);
                     if (masked) {
                         if (32 * c + 2 * i >= valid) x0 = -INFINITY;
                         if (32 * c + 2 * i + 1 >= valid) x1 = -INFINITY;
@@ -253,7 +253,6 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     *reinterpret_cast<uint4*>(atom + ((chunk ^ (r & 7)) << 4)) =
                         make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
                 }
-                if (c + 1 < 4) ptx::tmem_ld_wait();
             }
             l_blk = l_acc;
             m_blk = m_raw * scale_log2;                              // the scale is positive
