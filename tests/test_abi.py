@@ -122,3 +122,14 @@ def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(gmlp, "_LIB_PATH", str(tmp_path / "libgmlp.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         gmlp.lib()
+
+
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C header: it must compile as C99 on its own (no C++, no CUDA, no torch types)."""
+    import subprocess
+    src = tmp_path / "t.c"
+    src.write_text('#include "gmlp.h"\nint main(void) { gmlp_args a; gmlp_qkv_args q; gmlp_gqa_args g; (void)a; (void)q; (void)g; '
+                   'return GMLP_OK + GMLP_VARIANT_TENSOR - GMLP_VARIANT_TENSOR; }\n')
+    r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-fsyntax-only",
+                        "-I", os.path.join(ROOT, "include"), str(src)], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
