@@ -29,7 +29,8 @@
  * gmlp_shutdown().
  * A caller-made workspace belongs to the library between calls: the small-M schedules keep arrival
  * counters in it, which the library zeroes the first time it sees a (pointer, size) and which its kernels
- * leave zero after every call, so later calls with the same workspace start without a memset.  If
+ * leave zero after every call, so later calls with the same workspace start without a memset (calls of other
+ * shapes or schedules through the same buffer are noticed: what they overwrite is forgotten by itself).  If
  * anything else writes to that memory between two calls (the buffer was freed and handed out again by an
  * allocator, reused as scratch, ...), tell the library with gmlp_workspace_forget() before the next call.
  *

@@ -400,6 +400,23 @@ int ensure_counters_zero(DeviceState* dev, void* ptr, uint64_t bytes, cudaStream
     return GMLP_OK;
 }
 
+// A call is about to use [ws, ws + total) as its workspace.  Counter regions remembered as zero that lie in that
+// range were put there by calls with another layout (another shape or schedule in the same buffer) and are about to
+// be overwritten by this call's intermediates - except the region this call itself keeps its counters in.
+void claim_workspace(DeviceState* dev, const uint8_t* ws, uint64_t total, const void* keep_ptr, uint64_t keep_bytes) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    for (int i = 0; i < DeviceState::kCleanSlots; ++i) {
+        const uint8_t* c = static_cast<const uint8_t*>(dev->clean_counters[i]);
+        if (c == nullptr) continue;
+        const bool same = dev->clean_counters[i] == keep_ptr && dev->clean_counters_bytes[i] == keep_bytes;
+        const bool overlaps = c < ws + total && c + dev->clean_counters_bytes[i] > ws;
+        if (overlaps && !same) {
+            dev->clean_counters[i] = nullptr;
+            dev->clean_counters_bytes[i] = 0;
+        }
+    }
+}
+
 void forget_counters_locked(DeviceState* dev) {
     for (int i = 0; i < DeviceState::kCleanSlots; ++i) {
         dev->clean_counters[i] = nullptr;
@@ -790,6 +807,7 @@ int forward_impl(const gmlp_args* a) {
     } else if (a->workspace_bytes < L.total) {
         return GMLP_ERR_WORKSPACE;
     }
+    claim_workspace(dev, ws, L.total, L.counters_bytes ? ws + L.counters_off : nullptr, L.counters_bytes);
 
     cudaStream_t st = static_cast<cudaStream_t>(a->stream);
     const bf16* X = static_cast<const bf16*>(a->X);
@@ -966,6 +984,7 @@ int gate_up_impl(const gmlp_args* a) {
     } else if (a->workspace_bytes < L.total) {
         return GMLP_ERR_WORKSPACE;
     }
+    claim_workspace(dev, ws, L.total, L.counters_bytes ? ws + L.counters_off : nullptr, L.counters_bytes);
     cudaStream_t st = static_cast<cudaStream_t>(a->stream);
     const bf16* A = static_cast<const bf16*>(a->X);
     const bf16* Wg = static_cast<const bf16*>(a->Wg);
@@ -1027,6 +1046,7 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
     if (unfused) {
         const uint64_t need = align256((uint64_t)a->M * a->K * 2);
         if (a->workspace == nullptr || a->workspace_bytes < need) return GMLP_ERR_WORKSPACE;
+        claim_workspace(dev, static_cast<const uint8_t*>(a->workspace), need, nullptr, 0);
         bf16* Xn = static_cast<bf16*>(a->workspace);
         rc = launch_rmsnorm(X, static_cast<const bf16*>(a->rms_gain), Xn, a->M, a->K, a->rms_eps, st);
         if (rc != GMLP_OK) return rc;
@@ -1040,6 +1060,7 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
         // in its epilogue; programmatic dependent launch lets the GEMM's main loop overlap the RMS branch
         const uint64_t need = align256((uint64_t)a->M * 4);
         if (a->workspace == nullptr || a->workspace_bytes < need) return GMLP_ERR_WORKSPACE;
+        claim_workspace(dev, static_cast<const uint8_t*>(a->workspace), need, nullptr, 0);
         float* r = static_cast<float*>(a->workspace);
         gmlp::row_rsqrt_kernel<<<(unsigned)a->M, gmlp::kRmsThreads, 0, st>>>(X, r, a->M, (int)a->K, a->rms_eps);
         GMLP_CHECK_LAUNCH();
@@ -1121,6 +1142,7 @@ int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
         // three separate operators: T = X W (bf16), S = T + R, Z = RMSNorm(S)
         const uint64_t need = align256((uint64_t)a->M * a->N * 2);
         if (a->workspace == nullptr || a->workspace_bytes < need) return GMLP_ERR_WORKSPACE;
+        claim_workspace(dev, static_cast<const uint8_t*>(a->workspace), need, nullptr, 0);
         bf16* T = static_cast<bf16*>(a->workspace);
         rc = pair ? launch_umma_pair<false>(dev, X, W, nullptr, T, a->M, a->K, a->N, st)
                   : launch_umma<false>(dev, X, W, nullptr, T, a->M, a->K, a->N, st);
@@ -1138,6 +1160,7 @@ int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
         const int n_tiles = (int)((a->N + 255) / 256);
         const uint64_t need = align256((uint64_t)n_tiles * a->M * 4);
         if (a->workspace == nullptr || a->workspace_bytes < need) return GMLP_ERR_WORKSPACE;
+        claim_workspace(dev, static_cast<const uint8_t*>(a->workspace), need, nullptr, 0);
         float* sumsq = static_cast<float*>(a->workspace);
         CUtensorMap tmA, tmB;
         if (!encode_2d(&tmA, X, (uint64_t)a->K, (uint64_t)a->M, gmlp::kUmmaBK, 128) ||

@@ -206,6 +206,34 @@ def test_workspace_too_small_is_rejected_and_results_are_deterministic():
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
 
 
+def test_one_workspace_shared_by_calls_of_different_shapes():
+    # the library-owned workspace (and any caller buffer used for several shapes) holds every call's intermediates
+    # at shape-dependent offsets: the arrival counters one shape left at zero get overwritten by another shape's H,
+    # and the library must notice (regression: it used to trust what it remembered about the first shape)
+    a = I.custom_inputs(5, 1024, 128, 1, rmsnorm=True)
+    b = I.custom_inputs(300, 512, 1024, 2)
+    c = I.custom_inputs(8, 256, 512, 3)
+    for inp, variant in ((a, SKINNY), (b, TENSOR), (a, SKINNY), (c, SKINNY), (b, PAIR), (c, SKINNY), (a, SKINNY)):
+        w = inp.workload
+        t = to_device(inp)
+        Y = gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], gamma=t["gamma"] if w.rmsnorm else None, eps=w.eps,
+                         rmsnorm=w.rmsnorm, variant=variant, checked=True)          # workspace=None: the library's own
+        rows = I.sample_rows(w, inp.outlier_rows)
+        e, _ = err_over_tol(Y, oracle_rows(inp, rows), rows)
+        assert float(e.max()) <= 1.0, f"M={w.M} variant {variant}: max err/tol {float(e.max()):.2f}"
+    # the same with one caller-made buffer big enough for all of them
+    big = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    gmlp.lib().gmlp_workspace_forget(big.data_ptr(), big.numel())
+    for inp, variant in ((a, SKINNY), (b, TENSOR), (a, SKINNY), (c, SKINNY), (a, SKINNY)):
+        w = inp.workload
+        t = to_device(inp)
+        Y = gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], gamma=t["gamma"] if w.rmsnorm else None, eps=w.eps,
+                         rmsnorm=w.rmsnorm, variant=variant, workspace=big, checked=True)
+        rows = I.sample_rows(w, inp.outlier_rows)
+        e, _ = err_over_tol(Y, oracle_rows(inp, rows), rows)
+        assert float(e.max()) <= 1.0, f"caller buffer, M={w.M} variant {variant}: max err/tol {float(e.max()):.2f}"
+
+
 def test_workspace_written_by_someone_else_is_usable_again_after_forget():
     # the small-M schedules keep arrival counters in the workspace and rely on finding them zero; a caller that
     # lets other work write to the workspace says so with gmlp_workspace_forget, and the next call re-zeroes them
