@@ -22,6 +22,7 @@
 // operand (keys are the K dimension, D the N dimension) read as it lies in memory - no transposed copy of K or V.
 // Every wait is bounded (see umma_gemm.cuh).
 #pragma once
+#include <type_traits>
 #include <cuda.h>
 
 #include "common.cuh"
@@ -53,9 +54,58 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
-    asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+
+// Two fp32 values in one 64-bit register pair: sm_100 adds, multiplies and fuses them two at a time, which halves
+// the instruction count of the softmax's scaling and summing (the softmax warps are bound by instruction issue
+// and by the special-function unit, not by arithmetic).
+__device__ __forceinline__ uint64_t pack_f32x2(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3_f32(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// 2^x on the FMA pipe for part of the exponentials, so that the special-function unit (16 results per cycle
+// and SM) is not the only source: x is split into the nearest integer n (taken from the mantissa of
+// x + 1.5 * 2^23) and f in [-1/2, 1/2]; 2^f is a cubic fitted for minimum relative error (7.5e-5, a twenty-
+// fifth of the bf16 rounding that P gets next); n is added to the exponent field.  Both values of a pair at once.
+__device__ __forceinline__ void ex2_poly_x2(float x0, float x1, float& p0, float& p1) {
+    const uint64_t x = pack_f32x2(fmaxf(x0, -125.0f), fmaxf(x1, -125.0f));
+    const uint64_t magic = pack_f32x2(12582912.0f, 12582912.0f);
+    const uint64_t t = add_f32x2(x, magic);
+    const uint64_t n = add_f32x2(t, pack_f32x2(-12582912.0f, -12582912.0f));
+    const uint64_t f = fma_f32x2(n, pack_f32x2(-1.0f, -1.0f), x);
+    uint64_t p = fma_f32x2(pack_f32x2(0.0551716685f, 0.0551716685f), f, pack_f32x2(0.2426111400f, 0.2426111400f));
+    p = fma_f32x2(p, f, pack_f32x2(0.6932609677f, 0.6932609677f));
+    p = fma_f32x2(p, f, pack_f32x2(0.9999280572f, 0.9999280572f));
+    float q0, q1, t0, t1;
+    unpack_f32x2(p, q0, q1);
+    unpack_f32x2(t, t0, t1);
+    p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+    p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
+}
+#ifndef GMLP_GQA_POLY_MASK
+#define GMLP_GQA_POLY_MASK 0
+#endif
 
 __global__ void __launch_bounds__(kGqaThreads, 1)
 gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -221,10 +271,11 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         // one pass over the block's scores with base m_use: P to shared memory, row sum and row maximum.  The
         // next 32 scores are on their way from TMEM while the current 32 are processed; the scale is folded into
         // the exponent's FMA; only a block with missing keys (the last one) pays for the masking.
-        auto block_pass = [&](int valid, float& l_blk, float& m_blk) {
-            const bool masked = valid < kGqaBS;
-            const float neg_base = -m_use;
-            float l_acc = 0.0f, m_raw = -INFINITY;
+        auto block_pass = [&](auto masked_tag, int valid, float& l_blk, float& m_blk) {
+            constexpr bool masked = decltype(masked_tag)::value;
+            const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2), neg_base2 = pack_f32x2(-m_use, -m_use);
+            uint64_t l_acc2 = pack_f32x2(0.0f, 0.0f);
+            float m_raw = -INFINITY;
             uint32_t v[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(s_addr + 32 * c, v[c]);
@@ -235,14 +286,20 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     float x0 = __uint_as_float(v[c][2 * i]), x1 = __uint_as_float(v[c][2 * i + 1]);
-                    if (masked) {
+                    if constexpr (masked) {
                         if (32 * c + 2 * i >= valid) x0 = -INFINITY;
                         if (32 * c + 2 * i + 1 >= valid) x1 = -INFINITY;
                     }
-                    m_raw = fmaxf(m_raw, fmaxf(x0, x1));
-                    const float p0 = ex2_approx(fmaf(x0, scale_log2, neg_base));
-                    const float p1 = ex2_approx(fmaf(x1, scale_log2, neg_base));
-                    l_acc += p0 + p1;
+                    m_raw = max3_f32(m_raw, x0, x1);
+                    float e0, e1, p0, p1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(x0, x1), scale2, neg_base2), e0, e1);
+                    if ((GMLP_GQA_POLY_MASK >> (i & 7)) & 1) {       // an unrolled constant: which pairs take the polynomial
+                        ex2_poly_x2(e0, e1, p0, p1);
+                    } else {
+                        p0 = ex2_approx(e0);
+                        p1 = ex2_approx(e1);
+                    }
+                    l_acc2 = add_f32x2(l_acc2, pack_f32x2(p0, p1));
                     packed[i] = pack_bf16x2(p0, p1);
                 }
                 // columns 32c .. 32c+31 of row r: four 16-byte chunks of the 64-wide atom (c / 2)
@@ -254,8 +311,16 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
                 }
             }
-            l_blk = l_acc;
+            float l0, l1;
+            unpack_f32x2(l_acc2, l0, l1);
+            l_blk = l0 + l1;
             m_blk = m_raw * scale_log2;                              // the scale is positive
+        };
+        // the pass holds warp-wide TMEM loads, so the choice between its two forms is made for the warp as a whole
+        // (under a causal mask the rows of a warp see different numbers of keys)
+        auto block_pass_any = [&](int valid, float& l_blk, float& m_blk) {
+            if (__any_sync(0xFFFFFFFFu, valid < kGqaBS)) block_pass(std::true_type{}, valid, l_blk, m_blk);
+            else block_pass(std::false_type{}, valid, l_blk, m_blk);
         };
 
         for (int j = 0; j < n_blocks && ok; ++j) {
@@ -279,9 +344,9 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         if (32 * c + i < valid) m0v = fmaxf(m0v, __uint_as_float(v[i]) * scale_log2);
                 }
                 m_use = m0v;
-                block_pass(valid, l_blk, m_blk);
+                block_pass_any(valid, l_blk, m_blk);
             } else {
-                block_pass(valid, l_blk, m_blk);
+                block_pass_any(valid, l_blk, m_blk);
                 if (__any_sync(0xFFFFFFFFu, m_blk > m_use + kGqaLazyLog2)) {
                     // some row's maximum moved far: new base, rescale this warp's rows of O and l, redo the block
                     const float m_new = fmaxf(m_use, m_blk);
@@ -298,7 +363,7 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         tmem_st_32x32(o_addr + c, v);
                     }
                     tmem_st_wait();
-                    block_pass(valid, l_blk, m_blk);
+                    block_pass_any(valid, l_blk, m_blk);
                 }
             }
             l_run += l_blk;
