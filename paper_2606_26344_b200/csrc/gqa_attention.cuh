@@ -9,7 +9,7 @@
 //   warp 0      TMA producer: both Q tiles once, then K(0), V(0), K(1), V(1), ... through one three-slot FIFO
 //   warp 1      MMA issuer:   per tile t, S_t = Q_t K^T (TMEM columns 128 t) and O_t += P_t V (columns 256 + 128 t),
 //                             in the order PV_A(j), S_A(j+1), PV_B(j), S_B(j+1)
-//   warps 2..5  softmax of tile A, warps 6..9 of tile B: thread = query row (its TMEM lane), so row maxima and sums
+//   warps 4..7  softmax of tile A, warps 8..11 of tile B: thread = query row (its TMEM lane), so row maxima and sums
 //                             need no shuffles.  The exponent base is a running maximum that is only moved when a
 //                             block's maximum exceeds it by more than 8 (probabilities stay below 2^8): a block is
 //                             normally ONE pass over its scores (exponentials with the current base while the
@@ -34,10 +34,11 @@ namespace gmlp {
 constexpr int kGqaD = 128;                       // head dimension
 constexpr int kGqaBM = 256;                      // query rows per CTA (two tiles of 128)
 constexpr int kGqaBS = 128;                      // keys per block
-constexpr int kGqaThreads = 320;                 // producer warp, MMA warp, 2 x 4 softmax warps
+constexpr int kGqaThreads = 384;                 // warp group 0: producer warp, MMA warp, two idle; groups 1, 2: softmax
+constexpr int kGqaRegsLight = 56, kGqaRegsSoftmax = 224;   // registers per thread after the groups trade (sum kept)
 constexpr uint32_t kGqaTileBytes = 128 * 128 * 2;                         // one 128 x 128 bf16 tile: 32 KB
-constexpr int kGqaSlots = 3;                                              // K/V FIFO slots
-constexpr uint32_t kGqaSmemBytes = (4 + kGqaSlots) * kGqaTileBytes + 1024 + 256;   // Q_A Q_B P_A P_B, FIFO
+constexpr int kGqaSlots = 5;                                              // K/V FIFO slots
+constexpr uint32_t kGqaSmemBytes = (2 + kGqaSlots) * kGqaTileBytes + 1024 + 256;   // Q_A Q_B, FIFO
 constexpr float kGqaLazyLog2 = 8.0f;                                      // move the exponent base only beyond this
 
 __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -50,6 +51,16 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r
           "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
           "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]: the A operand (M = 128 rows = lanes, K = 16 per instruction as 8 columns of
+// packed 16-bit pairs) is read from tensor memory.
+__device__ __forceinline__ void umma_bf16_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -84,29 +95,6 @@ __device__ __forceinline__ float max3_f32(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
-// 2^x on the FMA pipe for part of the exponentials, so that the special-function unit (16 results per cycle
-// and SM) is not the only source: x is split into the nearest integer n (taken from the mantissa of
-// x + 1.5 * 2^23) and f in [-1/2, 1/2]; 2^f is a cubic fitted for minimum relative error (7.5e-5, a twenty-
-// fifth of the bf16 rounding that P gets next); n is added to the exponent field.  Both values of a pair at once.
-__device__ __forceinline__ void ex2_poly_x2(float x0, float x1, float& p0, float& p1) {
-    const uint64_t x = pack_f32x2(fmaxf(x0, -125.0f), fmaxf(x1, -125.0f));
-    const uint64_t magic = pack_f32x2(12582912.0f, 12582912.0f);
-    const uint64_t t = add_f32x2(x, magic);
-    const uint64_t n = add_f32x2(t, pack_f32x2(-12582912.0f, -12582912.0f));
-    const uint64_t f = fma_f32x2(n, pack_f32x2(-1.0f, -1.0f), x);
-    uint64_t p = fma_f32x2(pack_f32x2(0.0551716685f, 0.0551716685f), f, pack_f32x2(0.2426111400f, 0.2426111400f));
-    p = fma_f32x2(p, f, pack_f32x2(0.6932609677f, 0.6932609677f));
-    p = fma_f32x2(p, f, pack_f32x2(0.9999280572f, 0.9999280572f));
-    float q0, q1, t0, t1;
-    unpack_f32x2(p, q0, q1);
-    unpack_f32x2(t, t0, t1);
-    p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
-    p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
-}
-#ifndef GMLP_GQA_POLY_MASK
-#define GMLP_GQA_POLY_MASK 0
-#endif
-
 __global__ void __launch_bounds__(kGqaThreads, 1)
 gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, bf16* __restrict__ O,
@@ -124,16 +112,15 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - raw_addr);
     const uint32_t q_smem = base;                                    // + tile * 32 KB
-    const uint32_t p_smem = base + 2 * kGqaTileBytes;                // + tile * 32 KB
-    const uint32_t fifo = base + 4 * kGqaTileBytes;                  // + slot * 32 KB
-    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + (4 + kGqaSlots) * kGqaTileBytes);
-    const uint32_t kv_full0 = ptx::smem_addr(bars);                  // [3]
-    const uint32_t kv_empty0 = ptx::smem_addr(bars + 3);             // [3]
-    const uint32_t s_full0 = ptx::smem_addr(bars + 6);               // [2] tile t: the scores of a block are in TMEM
-    const uint32_t p_full0 = ptx::smem_addr(bars + 8);               // [2] tile t: P is in shared memory
-    const uint32_t o_full0 = ptx::smem_addr(bars + 10);              // [2] tile t: O += P V of a block is done
-    const uint32_t q_full = ptx::smem_addr(bars + 12);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+    const uint32_t fifo = base + 2 * kGqaTileBytes;                  // + slot * 32 KB
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + (2 + kGqaSlots) * kGqaTileBytes);
+    const uint32_t kv_full0 = ptx::smem_addr(bars);                  // [slots]
+    const uint32_t kv_empty0 = ptx::smem_addr(bars + kGqaSlots);     // [slots]
+    const uint32_t s_full0 = ptx::smem_addr(bars + 2 * kGqaSlots);   // [2] tile t: the scores of a block are in TMEM
+    const uint32_t p_full0 = ptx::smem_addr(bars + 2 * kGqaSlots + 2);   // [2] tile t: P is in TMEM
+    const uint32_t o_full0 = ptx::smem_addr(bars + 2 * kGqaSlots + 4);   // [2] tile t: O += P V of a block is done
+    const uint32_t q_full = ptx::smem_addr(bars + 2 * kGqaSlots + 6);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kGqaSlots + 7);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -148,7 +135,7 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     ptx::launch_dependents();
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 8; ++i) ptx::mbar_init(kv_full0 + 8 * i, 1);       // kv_full, kv_empty, s_full
+        for (int i = 0; i < 2 * kGqaSlots + 2; ++i) ptx::mbar_init(kv_full0 + 8 * i, 1);   // kv_full, kv_empty, s_full
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(p_full0 + 8 * i, 4);                      // one arrival per softmax warp of the tile
             ptx::mbar_init(o_full0 + 8 * i, 1);
@@ -170,7 +157,13 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;                           // S_t at + 128 t, O_t at + 256 + 128 t
 
-    if (warp == 0) {
+    // The launch gives every thread 168 registers (65536 / 384); the softmax threads hold a block's 128 scores and
+    // want more, the producer, the MMA issuer and the two idle warps need few: warp group 0 hands registers back
+    // and the two softmax groups take them (56 * 128 + 224 * 256 = 168 * 384).  Each form of the instruction sits
+    // inside its own branch, so that the compiler knows the budget of the code that follows it.
+    if (warp < 4) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kGqaRegsLight));
+      if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             ptx::grid_dependency_wait();                             // Q, K, V may come from the previous kernel
@@ -237,11 +230,11 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     const uint32_t v_smem = fifo + ((2 * j + 1) % kGqaSlots) * kGqaTileBytes;
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
-                        const uint64_t a_desc = ptx::make_smem_desc_sw128(
-                            p_smem + t * kGqaTileBytes + (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u, 16, 1024);
+                        // A = P_t from TMEM: 16 keys of a K step are 8 columns of packed bf16 pairs
                         const uint64_t b_desc = ptx::make_smem_desc_sw128(
                             v_smem + (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 2048u, 8192, 1024);
-                        ptx::umma_bf16(tmem_base + 256u + 128u * (uint32_t)t, a_desc, b_desc, kIdescPV, (j | k) != 0 ? 1u : 0u);
+                        umma_bf16_tmem_a(tmem_base + 256u + 128u * (uint32_t)t, tmem_base + 128u * (uint32_t)t + 8u * (uint32_t)k,
+                                         b_desc, kIdescPV, (j | k) != 0 ? 1u : 0u);
                     }
                     ptx::umma_commit(o_full0 + 8 * t);
                     if (t == 1) ptx::umma_commit(kv_empty0 + 8 * ((2 * j + 1) % kGqaSlots));   // both tiles have used V(j)
@@ -254,120 +247,97 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             }
         }
         __syncwarp();
+      }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kGqaRegsSoftmax));
         // ---------------- softmax and epilogue: one group of four warps per tile, thread = query row ----------------
-        const int t = (warp - 2) >> 2;                               // tile
+        const int t = (warp - 4) >> 2;                               // tile
         const int q = warp & 3;
         const int r = q * 32 + lane;                                 // row within the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const uint32_t s_addr = tmem_base + 128u * (uint32_t)t + lane_addr;
         const uint32_t o_addr = tmem_base + 256u + 128u * (uint32_t)t + lane_addr;
-        uint8_t* p_row = base_ptr + (2 + t) * kGqaTileBytes + (size_t)r * 128;
         float m_use = -INFINITY, l_run = 0.0f;                       // exponent base, row sum
         bool ok = true;
         // last key this row may see (causal), or none of that
         const int horizon = causal_off >= 0 ? m0 + 128 * t + r + causal_off : 0x7FFFFFFF - kGqaBS;
 
-        // one pass over the block's scores with base m_use: P to shared memory, row sum and row maximum.  The
-        // next 32 scores are on their way from TMEM while the current 32 are processed; the scale is folded into
-        // the exponent's FMA; only a block with missing keys (the last one) pays for the masking.
-        auto block_pass = [&](auto masked_tag, int valid, float& l_blk, float& m_blk) {
+        // One block: the scores come from TMEM into registers once; the row maximum decides (for the warp as a
+        // whole, the rescale holds warp-wide TMEM accesses) whether the exponent base has to move, and if so O and
+        // l are rescaled first; then one pass of exponentials with the scale folded into the exponent's FMA, two
+        // values per instruction where sm_100 has packed fp32 forms.  P goes back to TMEM as packed bf16 pairs
+        // over the first 64 columns of the tile's own score buffer (its scores are in registers by then): the
+        // second matmul reads its A operand from there, so P never crosses shared memory.  Only a block with
+        // keys a row may not see (the last one, or the diagonal under a causal mask) pays for the masking.
+        auto block_pass = [&](auto masked_tag, int j, int valid) {
             constexpr bool masked = decltype(masked_tag)::value;
-            const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2), neg_base2 = pack_f32x2(-m_use, -m_use);
-            uint64_t l_acc2 = pack_f32x2(0.0f, 0.0f);
-            float m_raw = -INFINITY;
             uint32_t v[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(s_addr + 32 * c, v[c]);
             ptx::tmem_ld_wait();
+            float m_raw = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t packed[16];
+            for (int c = 0; c < 4; ++c)
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    float x0 = __uint_as_float(v[c][2 * i]), x1 = __uint_as_float(v[c][2 * i + 1]);
                     if constexpr (masked) {
-                        if (32 * c + 2 * i >= valid) x0 = -INFINITY;
-                        if (32 * c + 2 * i + 1 >= valid) x1 = -INFINITY;
+                        if (32 * c + 2 * i >= valid) v[c][2 * i] = 0xFF800000u;          // -inf
+                        if (32 * c + 2 * i + 1 >= valid) v[c][2 * i + 1] = 0xFF800000u;
                     }
-                    m_raw = max3_f32(m_raw, x0, x1);
-                    float e0, e1, p0, p1;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(x0, x1), scale2, neg_base2), e0, e1);
-                    if ((GMLP_GQA_POLY_MASK >> (i & 7)) & 1) {       // an unrolled constant: which pairs take the polynomial
-                        ex2_poly_x2(e0, e1, p0, p1);
-                    } else {
-                        p0 = ex2_approx(e0);
-                        p1 = ex2_approx(e1);
-                    }
-                    l_acc2 = add_f32x2(l_acc2, pack_f32x2(p0, p1));
-                    packed[i] = pack_bf16x2(p0, p1);
+                    m_raw = max3_f32(m_raw, __uint_as_float(v[c][2 * i]), __uint_as_float(v[c][2 * i + 1]));
                 }
-                // columns 32c .. 32c+31 of row r: four 16-byte chunks of the 64-wide atom (c / 2)
-                uint8_t* atom = p_row + (size_t)(c >> 1) * 16384;
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    const int chunk = (c & 1) * 4 + ch;                              // 0..7 within the 128-byte row
-                    *reinterpret_cast<uint4*>(atom + ((chunk ^ (r & 7)) << 4)) =
-                        make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
-                }
-            }
-            float l0, l1;
-            unpack_f32x2(l_acc2, l0, l1);
-            l_blk = l0 + l1;
-            m_blk = m_raw * scale_log2;                              // the scale is positive
-        };
-        // the pass holds warp-wide TMEM loads, so the choice between its two forms is made for the warp as a whole
-        // (under a causal mask the rows of a warp see different numbers of keys)
-        auto block_pass_any = [&](int valid, float& l_blk, float& m_blk) {
-            if (__any_sync(0xFFFFFFFFu, valid < kGqaBS)) block_pass(std::true_type{}, valid, l_blk, m_blk);
-            else block_pass(std::false_type{}, valid, l_blk, m_blk);
-        };
-
-        for (int j = 0; j < n_blocks && ok; ++j) {
-            if (!wait_bounded(s_full0 + 8 * t, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 3)) { ok = false; break; }
-            // P of the previous block must have been consumed (and O complete) before P is overwritten
-            if (j > 0 && !wait_bounded(o_full0 + 8 * t, (uint32_t)(j - 1) & 1u, abort_flag, KERNEL_ID, 4)) { ok = false; break; }
-            ptx::tc_fence_after_sync();
-            // keys of this block that exist and that this row may see (0 when the whole block is beyond its horizon)
-            const int valid = max(0, min(min(kGqaBS, S - j * kGqaBS), horizon - j * kGqaBS + 1));
-            float l_blk, m_blk;
-            if (j == 0) {
-                // first block: find the base first (finite: every row sees at least key 0)
-                float m0v = -INFINITY;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    ptx::tmem_ld_32x32(s_addr + 32 * c, v);
-                    ptx::tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (32 * c + i < valid) m0v = fmaxf(m0v, __uint_as_float(v[i]) * scale_log2);
-                }
-                m_use = m0v;
-                block_pass_any(valid, l_blk, m_blk);
-            } else {
-                block_pass_any(valid, l_blk, m_blk);
-                if (__any_sync(0xFFFFFFFFu, m_blk > m_use + kGqaLazyLog2)) {
-                    // some row's maximum moved far: new base, rescale this warp's rows of O and l, redo the block
-                    const float m_new = fmaxf(m_use, m_blk);
+            const float m_blk = m_raw * scale_log2;                  // the scale is positive
+            if (__any_sync(0xFFFFFFFFu, m_blk > m_use + kGqaLazyLog2)) {
+                // some row's maximum moved far (always so in the first block, whose rows all see key 0): new base;
+                // O of the blocks so far is complete, because this block's scores were issued after their matmuls
+                const float m_new = fmaxf(m_use, m_blk);
+                if (j > 0) {
                     const float alpha = ex2_approx(m_use - m_new);
-                    m_use = m_new;
                     l_run *= alpha;
 #pragma unroll 1
                     for (int c = 0; c < kGqaD; c += 32) {
-                        uint32_t v[32];
-                        ptx::tmem_ld_32x32(o_addr + c, v);
+                        uint32_t o[32];
+                        ptx::tmem_ld_32x32(o_addr + c, o);
                         ptx::tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                        tmem_st_32x32(o_addr + c, v);
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st_32x32(o_addr + c, o);
                     }
-                    tmem_st_wait();
-                    block_pass_any(valid, l_blk, m_blk);
                 }
+                m_use = m_new;
             }
-            l_run += l_blk;
-            ptx::fence_proxy_async_smem();                           // P (generic writes) -> visible to the MMA
+            const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2), neg_base2 = pack_f32x2(-m_use, -m_use);
+            uint64_t l_acc2 = pack_f32x2(0.0f, 0.0f);
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                uint32_t packed[32];
+#pragma unroll
+                for (int ci = 0; ci < 32; ++ci) {
+                    const int c = 2 * hh + (ci >> 4), i = ci & 15;
+                    float e0, e1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[c][2 * i]), __uint_as_float(v[c][2 * i + 1])),
+                                           scale2, neg_base2), e0, e1);
+                    const float p0 = ex2_approx(e0), p1 = ex2_approx(e1);
+                    l_acc2 = add_f32x2(l_acc2, pack_f32x2(p0, p1));
+                    packed[ci] = pack_bf16x2(p0, p1);
+                }
+                tmem_st_32x32(s_addr + 32 * hh, packed);             // P columns 64 hh .. 64 hh + 63 as 32 pairs
+            }
+            float l0, l1;
+            unpack_f32x2(l_acc2, l0, l1);
+            l_run += l0 + l1;
+            tmem_st_wait();
+        };
+
+        for (int j = 0; j < n_blocks && ok; ++j) {
+            // the scores of block j are complete, and with them every matmul issued before them: O += P V of block
+            // j - 1 is done and has read its P
+            if (!wait_bounded(s_full0 + 8 * t, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 3)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            // keys of this block that exist and that this row may see (0 when the whole block is beyond its horizon)
+            const int valid = max(0, min(min(kGqaBS, S - j * kGqaBS), horizon - j * kGqaBS + 1));
+            if (__any_sync(0xFFFFFFFFu, valid < kGqaBS)) block_pass(std::true_type{}, j, valid);
+            else block_pass(std::false_type{}, j, valid);
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(p_full0 + 8 * t);
