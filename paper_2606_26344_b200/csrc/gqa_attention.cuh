@@ -3,21 +3,22 @@
 // Q [M, Hq*D], K and V [S, Hkv*D], O [M, Hq*D] row-major bf16.  One CTA per (256 query rows, query head), as TWO
 // query tiles of 128 rows that take turns on the tensor pipe: while one tile's scores are in the softmax, the
 // other tile's matmuls run.  The key/value sequence is walked in blocks of 128 with the running-maximum (online)
-// softmax, so the scores never leave the SM: both matmuls run on tcgen05 with their accumulators in TMEM and the
-// probabilities go from registers to shared memory as the second matmul's A operand.
+// softmax, so the scores never leave the SM: both matmuls run on tcgen05 with their accumulators in TMEM, and the
+// probabilities go from registers back to TMEM, where the second matmul reads them as its A operand.
 //
-//   warp 0      TMA producer: both Q tiles once, then K(0), V(0), K(1), V(1), ... through one three-slot FIFO
+//   warp 0      TMA producer: both Q tiles once, then K(0), V(0), K(1), V(1), ... through one five-slot FIFO
 //   warp 1      MMA issuer:   per tile t, S_t = Q_t K^T (TMEM columns 128 t) and O_t += P_t V (columns 256 + 128 t),
 //                             in the order PV_A(j), S_A(j+1), PV_B(j), S_B(j+1)
+//   warps 2, 3  idle (they fill warp group 0, which gives most of its registers to the softmax groups)
 //   warps 4..7  softmax of tile A, warps 8..11 of tile B: thread = query row (its TMEM lane), so row maxima and sums
-//                             need no shuffles.  The exponent base is a running maximum that is only moved when a
-//                             block's maximum exceeds it by more than 8 (probabilities stay below 2^8): a block is
-//                             normally ONE pass over its scores (exponentials with the current base while the
-//                             maximum is tracked); only if the base has to move is O in TMEM rescaled and the
-//                             block's probabilities recomputed.  P (bf16) is written in the 128-byte-swizzled
-//                             K-major layout the MMA expects; at the end O / l is stored.
+//                             need no shuffles.  A block's 128 scores are read into registers once.  The exponent
+//                             base is a running maximum that is only moved when a block's maximum exceeds it by more
+//                             than 8 (probabilities stay below 2^8), and then O in TMEM and l are rescaled BEFORE the
+//                             block's exponentials, so a block is always one pass.  P (bf16 pairs) overwrites the
+//                             first 64 columns of the tile's own score buffer; at the end O / l is stored.
 //
-// Operand forms: Q and P are K-major A operands (rows of 128 B, two 64-wide swizzle atoms side by side); a K block
+// Operand forms: Q is a K-major A operand in shared memory (rows of 128 B, two 64-wide swizzle atoms side by side),
+// P an A operand in TMEM (lane = query row, 8 columns of packed pairs per K step of 16 keys); a K block
 // [128 keys, D] is a K-major B operand (keys are the N dimension); a V block [128 keys, D] is an MN-major B
 // operand (keys are the K dimension, D the N dimension) read as it lies in memory - no transposed copy of K or V.
 // Every wait is bounded (see umma_gemm.cuh).
