@@ -11,11 +11,14 @@
 //                             in the order PV_A(j), S_A(j+1), PV_B(j), S_B(j+1)
 //   warps 2, 3  idle (they fill warp group 0, which gives most of its registers to the softmax groups)
 //   warps 4..7  softmax of tile A, warps 8..11 of tile B: thread = query row (its TMEM lane), so row maxima and sums
-//                             need no shuffles.  A block's 128 scores are read into registers once.  The exponent
-//                             base is a running maximum that is only moved when a block's maximum exceeds it by more
-//                             than 8 (probabilities stay below 2^8), and then O in TMEM and l are rescaled BEFORE the
-//                             block's exponentials, so a block is always one pass.  P (bf16 pairs) overwrites the
-//                             first 64 columns of the tile's own score buffer; at the end O / l is stored.
+//                             need no shuffles.  A block's 128 scores are read into registers once and go
+//                             through ONE pass of exponentials with the current base (scale folded into the
+//                             exponent's FMA, packed fp32 pairs, a quarter of the exponentials as a cubic on the
+//                             FMA pipe).  The base is a running maximum that is only moved when some row's sum of
+//                             a block exceeds 2^10: only then is the block's row maximum taken, O in TMEM and l
+//                             rescaled and the pass repeated (in the first block the maximum comes first).  P (bf16
+//                             pairs) overwrites the first 64 columns of the tile's own score buffer; at the end
+//                             O / l is stored.
 //
 // Operand forms: Q is a K-major A operand in shared memory (rows of 128 B, two 64-wide swizzle atoms side by side),
 // P an A operand in TMEM (lane = query row, 8 columns of packed pairs per K step of 16 keys); a K block
@@ -36,11 +39,11 @@ constexpr int kGqaD = 128;                       // head dimension
 constexpr int kGqaBM = 256;                      // query rows per CTA (two tiles of 128)
 constexpr int kGqaBS = 128;                      // keys per block
 constexpr int kGqaThreads = 384;                 // warp group 0: producer warp, MMA warp, two idle; groups 1, 2: softmax
-constexpr int kGqaRegsLight = 56, kGqaRegsSoftmax = 224;   // registers per thread after the groups trade (sum kept)
+constexpr int kGqaRegsLight = 72, kGqaRegsSoftmax = 216;   // registers per thread after the groups trade (sum kept)
 constexpr uint32_t kGqaTileBytes = 128 * 128 * 2;                         // one 128 x 128 bf16 tile: 32 KB
 constexpr int kGqaSlots = 5;                                              // K/V FIFO slots
 constexpr uint32_t kGqaSmemBytes = (2 + kGqaSlots) * kGqaTileBytes + 1024 + 256;   // Q_A Q_B, FIFO
-constexpr float kGqaLazyLog2 = 8.0f;                                      // move the exponent base only beyond this
+constexpr float kGqaLazySum = 1024.0f;          // move the exponent base only when a row of a block sums to more
 
 __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
     asm volatile(
@@ -62,6 +65,27 @@ __device__ __forceinline__ void umma_bf16_tmem_a(uint32_t d_tmem, uint32_t a_tme
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The same two instructions with each shared-memory descriptor given as its two 32-bit words (the upper word is
+// shared by all descriptors of this kernel, so the issuing thread keeps one register per descriptor).
+__device__ __forceinline__ void umma_bf16_halves(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                                 uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_tmem_a_halves(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
+                                                        uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -96,6 +120,31 @@ __device__ __forceinline__ float max3_f32(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
+// 2^x on the FMA pipe for part of the exponentials: x is split into the nearest integer n (taken from the mantissa
+// of x + 1.5 * 2^23) and f in [-1/2, 1/2]; 2^f is a cubic fitted for minimum relative error (7.5e-5, a twenty-fifth
+// of the bf16 rounding that P gets next); n is added to the exponent field.  Both values of a pair at once.
+__device__ __forceinline__ void ex2_poly_x2(float x0, float x1, float& p0, float& p1) {
+    const uint64_t x = pack_f32x2(fmaxf(x0, -125.0f), fmaxf(x1, -125.0f));
+    const uint64_t t = add_f32x2(x, pack_f32x2(12582912.0f, 12582912.0f));
+    const uint64_t n = add_f32x2(t, pack_f32x2(-12582912.0f, -12582912.0f));
+    const uint64_t f = fma_f32x2(n, pack_f32x2(-1.0f, -1.0f), x);
+    uint64_t p = fma_f32x2(pack_f32x2(0.0551716685f, 0.0551716685f), f, pack_f32x2(0.2426111400f, 0.2426111400f));
+    p = fma_f32x2(p, f, pack_f32x2(0.6932609677f, 0.6932609677f));
+    p = fma_f32x2(p, f, pack_f32x2(0.9999280572f, 0.9999280572f));
+    float q0, q1, t0, t1;
+    unpack_f32x2(p, q0, q1);
+    unpack_f32x2(t, t0, t1);
+    p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+    p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
+}
+// Which column pairs take the polynomial: bit (i & 7) for pair i of a 32-column chunk, i.e. two pairs in eight, a
+// quarter of the exponentials (measured at 8K tokens: none 1278, an eighth 1294, a quarter 1318, three eighths
+// 1250-1269, a half 1152 TFLOP/s - the softmax warps are bound by instruction issue as much as by the
+// special-function unit, and a polynomial pair costs five times the instructions of a hardware pair).
+#ifndef GMLP_GQA_POLY_MASK
+#define GMLP_GQA_POLY_MASK 0x11
+#endif
+
 __global__ void __launch_bounds__(kGqaThreads, 1)
 gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, bf16* __restrict__ O,
@@ -160,7 +209,7 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     // The launch gives every thread 168 registers (65536 / 384); the softmax threads hold a block's 128 scores and
     // want more, the producer, the MMA issuer and the two idle warps need few: warp group 0 hands registers back
-    // and the two softmax groups take them (56 * 128 + 224 * 256 = 168 * 384).  Each form of the instruction sits
+    // and the two softmax groups take them (72 * 128 + 216 * 256 = 168 * 384).  Each form of the instruction sits
     // inside its own branch, so that the compiler knows the budget of the code that follows it.
     if (warp < 4) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kGqaRegsLight));
@@ -199,50 +248,72 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            auto item_ready = [&](int i, int site) -> bool {
-                const bool ok = wait_bounded(kv_full0 + 8 * (i % kGqaSlots), (uint32_t)(i / kGqaSlots) & 1u, abort_flag, KERNEL_ID, site);
+            // The issuing thread is a single dependent instruction stream with a budget of 64 cycles per MMA, so
+            // nothing is derived per MMA: the FIFO position is stepped, not divided, and the descriptors of a group
+            // of eight K = 16 steps are formed (base + constant, independent of one another) before its first MMA.
+            // In 16-byte units a step advances a K-major operand by 2 within a 64-wide swizzle atom and by 1024 to
+            // the next atom of 128 rows; the MN-major V operand by 128 per 16 keys and by 1024 per 64 keys.
+            uint32_t it_slot = 0, it_phase = 0;                      // next K/V item (K(0), V(0), K(1), ...) to wait for
+            auto wait_next = [&](int site, uint32_t& slot_out) -> bool {
+                const bool ok = wait_bounded(kv_full0 + 8 * it_slot, it_phase, abort_flag, KERNEL_ID, site);
                 ptx::tc_fence_after_sync();
+                slot_out = it_slot;
+                if (++it_slot == (uint32_t)kGqaSlots) { it_slot = 0; it_phase ^= 1u; }
                 return ok;
             };
-            // S_t(j) = Q_t K(j)^T over D = 128: eight K = 16 steps, four per 64-wide swizzle atom
-            auto issue_scores = [&](int t, int j) {
-                const uint32_t k_smem = fifo + ((2 * j) % kGqaSlots) * kGqaTileBytes;
+            // (the upper word of every descriptor here is the same: stride 1024 B, version 1, 128-byte swizzle; only
+            // the lower words, start address and leading offset, are kept per step)
+            const uint32_t desc_hi = (uint32_t)(ptx::make_smem_desc_sw128(0, 0, 1024) >> 32);
+            const uint32_t q_lo0 = (uint32_t)ptx::make_smem_desc_sw128(q_smem, 16, 1024);
+            const uint32_t q_lo1 = (uint32_t)ptx::make_smem_desc_sw128(q_smem + kGqaTileBytes, 16, 1024);
+            const uint32_t k_lo_base = (uint32_t)ptx::make_smem_desc_sw128(fifo, 16, 1024);
+            const uint32_t v_lo_base = (uint32_t)ptx::make_smem_desc_sw128(fifo, 8192, 1024);
+            // S_t = Q_t K^T over D = 128 with the K block in FIFO slot `slot`
+            auto issue_scores = [&](int t, uint32_t slot) {
+                const uint32_t a0 = t ? q_lo1 : q_lo0;
+                const uint32_t b0 = k_lo_base + slot * (kGqaTileBytes >> 4);
+                uint32_t ad[8], bd[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                    const uint32_t off = (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u;
-                    ptx::umma_bf16(tmem_base + 128u * (uint32_t)t,
-                                   ptx::make_smem_desc_sw128(q_smem + t * kGqaTileBytes + off, 16, 1024),
-                                   ptx::make_smem_desc_sw128(k_smem + off, 16, 1024), kIdescQK, k != 0 ? 1u : 0u);
+                    ad[k] = a0 + (uint32_t)((k >> 2) * 1024 + (k & 3) * 2);
+                    bd[k] = b0 + (uint32_t)((k >> 2) * 1024 + (k & 3) * 2);
                 }
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16_halves(tmem_base + 128u * (uint32_t)t, ad[k], bd[k], desc_hi, kIdescQK, k != 0 ? 1u : 0u);
                 ptx::umma_commit(s_full0 + 8 * t);
-                if (t == 1) ptx::umma_commit(kv_empty0 + 8 * ((2 * j) % kGqaSlots));      // both tiles have used K(j)
+                if (t == 1) ptx::umma_commit(kv_empty0 + 8 * slot);              // both tiles have used this K block
             };
-            bool ok = wait_bounded(q_full, 0u, abort_flag, KERNEL_ID, 5) && item_ready(0, 2);
+            uint32_t k_slot = 0, v_slot = 0;
+            bool ok = wait_bounded(q_full, 0u, abort_flag, KERNEL_ID, 5) && wait_next(2, k_slot);
             if (ok) {
-                issue_scores(0, 0);
-                issue_scores(1, 0);
+                issue_scores(0, k_slot);
+                issue_scores(1, k_slot);
             }
             for (int j = 0; j < n_blocks && ok; ++j) {
                 for (int t = 0; t < 2 && ok; ++t) {
-                    // tile t's probabilities of block j are in shared memory; V(j) has landed
+                    // tile t's probabilities of block j are in TMEM; V(j) has landed
                     if (!wait_bounded(p_full0 + 8 * t, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 6)) { ok = false; break; }
-                    if (t == 0 && !item_ready(2 * j + 1, 9)) { ok = false; break; }
+                    if (t == 0 && !wait_next(9, v_slot)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
-                    const uint32_t v_smem = fifo + ((2 * j + 1) % kGqaSlots) * kGqaTileBytes;
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
+                    {
                         // A = P_t from TMEM: 16 keys of a K step are 8 columns of packed bf16 pairs
-                        const uint64_t b_desc = ptx::make_smem_desc_sw128(
-                            v_smem + (uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 2048u, 8192, 1024);
-                        umma_bf16_tmem_a(tmem_base + 256u + 128u * (uint32_t)t, tmem_base + 128u * (uint32_t)t + 8u * (uint32_t)k,
-                                         b_desc, kIdescPV, (j | k) != 0 ? 1u : 0u);
+                        const uint32_t v0 = v_lo_base + v_slot * (kGqaTileBytes >> 4);
+                        const uint32_t d_tmem = tmem_base + 256u + 128u * (uint32_t)t, p_tmem = tmem_base + 128u * (uint32_t)t;
+                        uint32_t bd[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) bd[k] = v0 + (uint32_t)((k >> 2) * 1024 + (k & 3) * 128);
+                        umma_bf16_tmem_a_halves(d_tmem, p_tmem, bd[0], desc_hi, kIdescPV, j != 0 ? 1u : 0u);
+#pragma unroll
+                        for (int k = 1; k < 8; ++k)
+                            umma_bf16_tmem_a_halves(d_tmem, p_tmem + 8u * (uint32_t)k, bd[k], desc_hi, kIdescPV, 1u);
                     }
                     ptx::umma_commit(o_full0 + 8 * t);
-                    if (t == 1) ptx::umma_commit(kv_empty0 + 8 * ((2 * j + 1) % kGqaSlots));   // both tiles have used V(j)
+                    if (t == 1) ptx::umma_commit(kv_empty0 + 8 * v_slot);        // both tiles have used V(j)
                     // the tile's next scores follow at once: its score buffer was consumed before p_full
                     if (j + 1 < n_blocks) {
-                        if (t == 0 && !item_ready(2 * j + 2, 2)) { ok = false; break; }
-                        issue_scores(t, j + 1);
+                        if (t == 0 && !wait_next(2, k_slot)) { ok = false; break; }
+                        issue_scores(t, k_slot);
                     }
                 }
             }
@@ -263,36 +334,72 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         // last key this row may see (causal), or none of that
         const int horizon = causal_off >= 0 ? m0 + 128 * t + r + causal_off : 0x7FFFFFFF - kGqaBS;
 
-        // One block: the scores come from TMEM into registers once; the row maximum decides (for the warp as a
-        // whole, the rescale holds warp-wide TMEM accesses) whether the exponent base has to move, and if so O and
-        // l are rescaled first; then one pass of exponentials with the scale folded into the exponent's FMA, two
-        // values per instruction where sm_100 has packed fp32 forms.  P goes back to TMEM as packed bf16 pairs
-        // over the first 64 columns of the tile's own score buffer (its scores are in registers by then): the
-        // second matmul reads its A operand from there, so P never crosses shared memory.  Only a block with
-        // keys a row may not see (the last one, or the diagonal under a causal mask) pays for the masking.
+        // One block: the scores come from TMEM into registers once; P goes back to TMEM as packed bf16 pairs over
+        // the first 64 columns of the tile's own score buffer (its scores are in registers by then): the second
+        // matmul reads its A operand from there, so P never crosses shared memory.  Only a block with keys a row
+        // may not see (the last one, or the diagonal under a causal mask) pays for the masking.
         auto block_pass = [&](auto masked_tag, int j, int valid) {
             constexpr bool masked = decltype(masked_tag)::value;
             uint32_t v[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(s_addr + 32 * c, v[c]);
             ptx::tmem_ld_wait();
-            float m_raw = -INFINITY;
+            if constexpr (masked) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    if constexpr (masked) {
-                        if (32 * c + 2 * i >= valid) v[c][2 * i] = 0xFF800000u;          // -inf
-                        if (32 * c + 2 * i + 1 >= valid) v[c][2 * i + 1] = 0xFF800000u;
+                    for (int i = 0; i < 32; ++i)
+                        if (32 * c + i >= valid) v[c][i] = 0xFF800000u;                  // -inf
+            }
+            // exponentials of the block with the current base: P to TMEM, returns the row's sum
+            auto exp_pass = [&]() -> float {
+                const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2), neg_base2 = pack_f32x2(-m_use, -m_use);
+                uint64_t l_acc2 = pack_f32x2(0.0f, 0.0f);
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    uint32_t packed[32];
+#pragma unroll
+                    for (int ci = 0; ci < 32; ++ci) {
+                        const int c = 2 * hh + (ci >> 4), i = ci & 15;
+                        float e0, e1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[c][2 * i]), __uint_as_float(v[c][2 * i + 1])),
+                                               scale2, neg_base2), e0, e1);
+                        float p0, p1;
+                        if ((GMLP_GQA_POLY_MASK >> (i & 7)) & 1) {
+                            ex2_poly_x2(e0, e1, p0, p1);
+                        } else {
+                            p0 = ex2_approx(e0);
+                            p1 = ex2_approx(e1);
+                        }
+                        l_acc2 = add_f32x2(l_acc2, pack_f32x2(p0, p1));
+                        packed[ci] = pack_bf16x2(p0, p1);
                     }
-                    m_raw = max3_f32(m_raw, __uint_as_float(v[c][2 * i]), __uint_as_float(v[c][2 * i + 1]));
+                    tmem_st_32x32(s_addr + 32 * hh, packed);         // P columns 64 hh .. 64 hh + 63 as 32 pairs
                 }
-            const float m_blk = m_raw * scale_log2;                  // the scale is positive
-            if (__any_sync(0xFFFFFFFFu, m_blk > m_use + kGqaLazyLog2)) {
-                // some row's maximum moved far (always so in the first block, whose rows all see key 0): new base;
-                // O of the blocks so far is complete, because this block's scores were issued after their matmuls
-                const float m_new = fmaxf(m_use, m_blk);
+                float l0, l1;
+                unpack_f32x2(l_acc2, l0, l1);
+                return l0 + l1;
+            };
+            // The row maximum (64 three-input maxima, 290 cycles of a half-rate pipe, on the critical path of the
+            // tile) is only taken when it is needed: in the first block, and when some row's sum of exponentials
+            // with the current base says that the base is far too low.  The sum bounds every term: below
+            // kGqaLazySum nothing can overflow and P keeps its relative precision, whatever the base.
+            float l_blk = 0.0f;
+            bool moved = j == 0;
+            if (j > 0) {
+                l_blk = exp_pass();
+                moved = __any_sync(0xFFFFFFFFu, !(l_blk <= kGqaLazySum));        // also catches inf and NaN
+            }
+            if (moved) {
+                float m_raw = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        m_raw = max3_f32(m_raw, __uint_as_float(v[c][2 * i]), __uint_as_float(v[c][2 * i + 1]));
+                const float m_new = fmaxf(m_use, m_raw * scale_log2);            // the scale is positive
                 if (j > 0) {
+                    // O of the blocks so far is complete: this block's scores were issued after their matmuls
                     const float alpha = ex2_approx(m_use - m_new);
                     l_run *= alpha;
 #pragma unroll 1
@@ -306,27 +413,9 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     }
                 }
                 m_use = m_new;
+                l_blk = exp_pass();
             }
-            const uint64_t scale2 = pack_f32x2(scale_log2, scale_log2), neg_base2 = pack_f32x2(-m_use, -m_use);
-            uint64_t l_acc2 = pack_f32x2(0.0f, 0.0f);
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                uint32_t packed[32];
-#pragma unroll
-                for (int ci = 0; ci < 32; ++ci) {
-                    const int c = 2 * hh + (ci >> 4), i = ci & 15;
-                    float e0, e1;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[c][2 * i]), __uint_as_float(v[c][2 * i + 1])),
-                                           scale2, neg_base2), e0, e1);
-                    const float p0 = ex2_approx(e0), p1 = ex2_approx(e1);
-                    l_acc2 = add_f32x2(l_acc2, pack_f32x2(p0, p1));
-                    packed[ci] = pack_bf16x2(p0, p1);
-                }
-                tmem_st_32x32(s_addr + 32 * hh, packed);             // P columns 64 hh .. 64 hh + 63 as 32 pairs
-            }
-            float l0, l1;
-            unpack_f32x2(l_acc2, l0, l1);
-            l_run += l0 + l1;
+            l_run += l_blk;
             tmem_st_wait();
         };
 
