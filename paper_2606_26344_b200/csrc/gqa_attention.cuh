@@ -66,18 +66,7 @@ __device__ __forceinline__ void umma_bf16_tmem_a(uint32_t d_tmem, uint32_t a_tme
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// The same two instructions with each shared-memory descriptor given as its two 32-bit words (the upper word is
-// shared by all descriptors of this kernel, so the issuing thread keeps one register per descriptor).
-__device__ __forceinline__ void umma_bf16_halves(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
-                                                 uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "mov.b64 da, {%1, %3};\n\t"
-        "mov.b64 db, {%2, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
-}
+// The TMEM-operand form with the shared-memory descriptor given as its two 32-bit words (see ptx::umma_bf16_halves).
 __device__ __forceinline__ void umma_bf16_tmem_a_halves(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
                                                         uint32_t idesc, uint32_t accumulate) {
     asm volatile(
@@ -280,7 +269,7 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 }
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    umma_bf16_halves(tmem_base + 128u * (uint32_t)t, ad[k], bd[k], desc_hi, kIdescQK, k != 0 ? 1u : 0u);
+                    ptx::umma_bf16_halves(tmem_base + 128u * (uint32_t)t, ad[k], bd[k], desc_hi, kIdescQK, k != 0 ? 1u : 0u);
                 ptx::umma_commit(s_full0 + 8 * t);
                 if (t == 1) ptx::umma_commit(kv_empty0 + 8 * slot);              // both tiles have used this K block
             };

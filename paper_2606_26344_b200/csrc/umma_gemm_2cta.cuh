@@ -76,6 +76,17 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc,
         "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// descriptors as 32-bit halves (see umma_bf16_halves)
+__device__ __forceinline__ void umma_bf16_pair_halves(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                                      uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
 // one arrival on the barrier at this shared-memory offset in BOTH CTAs once the MMAs issued so far are done
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -152,7 +163,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         if (lane == 0) {
             if (!ROWSCALE) ptx::grid_dependency_wait();
             const uint32_t leader_full0 = ptx::map_to_cta(full0, 0);
-            int it = 0;
+            uint32_t s = 0, ph = 0;                              // ring position of the next k-block
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
                 const int m0 = (tile % num_m_tiles) * 256 + (int)rank * 128;
@@ -166,9 +177,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     bmap = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &multi.tmB2);
                 }
                 const int bx = GATEUP ? n0 : n0 + (int)rank * 128;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % kPairStages;
-                    const uint32_t ph = (uint32_t)(it / kPairStages) & 1u;
+                for (int kb = 0; kb < num_kb; ++kb) {
                     if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) { ok = false; break; }
                     const uint32_t full = leader_full0 + 8 * s;
                     const uint32_t a_dst = base + s * kPairStageBytes;
@@ -182,6 +191,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                         ptx::tma_load_2d_pair(b_dst, bmap, bx, kb * kUmmaBK, full);
                         ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, bx + 64, kb * kUmmaBK, full);
                     }
+                    if (++s == (uint32_t)kPairStages) { s = 0; ph ^= 1u; }
                 }
             }
         }
@@ -189,28 +199,32 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader only) ----------------
         if (lane == 0 && rank == 0) {
-            int it = 0, t = 0;
+            // Nothing is derived per MMA: the ring position is stepped, not divided, and a step's descriptors are
+            // the stage's first ones plus a constant (in 16-byte units: 2 per K = 16 step of a K-major operand,
+            // 128 of the MN-major weights); only the lower descriptor word changes.
+            const uint32_t desc_hi = (uint32_t)(ptx::make_smem_desc_sw128(0, 0, 1024) >> 32);
+            const uint32_t a_lo0 = (uint32_t)ptx::make_smem_desc_sw128(base, 16, 1024);
+            const uint32_t b_lo0 = w_kmajor ? (uint32_t)ptx::make_smem_desc_sw128(base + kPairABytes, 16, 1024)
+                                            : (uint32_t)ptx::make_smem_desc_sw128(base + kPairABytes, kUmmaBoxBBytes, 1024);
+            const uint32_t b_step = w_kmajor ? 2u : 128u;
+            uint32_t s = 0, ph = 0;                              // ring position of the next k-block
+            int t = 0;
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++t) {
                 const int buf = t & 1;
                 if (!wait_bounded(tempty0 + 8 * buf, (((uint32_t)t >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4)) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % kPairStages;
-                    const uint32_t ph = (uint32_t)(it / kPairStages) & 1u;
+                for (int kb = 0; kb < num_kb; ++kb) {
                     if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
-                    const uint32_t a_base = base + s * kPairStageBytes;
-                    const uint32_t b_base = a_base + kPairABytes;
+                    const uint32_t a_lo = a_lo0 + s * (kPairStageBytes >> 4), b_lo = b_lo0 + s * (kPairStageBytes >> 4);
+                    ptx::umma_bf16_pair_halves(d_tmem, a_lo, b_lo, desc_hi, kIdesc, kb != 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k = 0; k < kUmmaBK / 16; ++k) {
-                        const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
-                        const uint64_t b_desc = w_kmajor ? ptx::make_smem_desc_sw128(b_base + k * 32, 16, 1024)
-                                                         : ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
-                        ptx::umma_bf16_pair(d_tmem, a_desc, b_desc, kIdesc, (kb | k) != 0 ? 1u : 0u);
-                    }
+                    for (int k = 1; k < kUmmaBK / 16; ++k)
+                        ptx::umma_bf16_pair_halves(d_tmem, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
                     ptx::umma_commit_pair(empty0 + 8 * s);
+                    if (++s == (uint32_t)kPairStages) { s = 0; ph ^= 1u; }
                 }
                 if (ok) ptx::umma_commit_pair(tfull0 + 8 * buf);
             }
