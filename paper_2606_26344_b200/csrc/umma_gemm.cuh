@@ -196,7 +196,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             if (!ROWSCALE) ptx::grid_dependency_wait();           // A (Xn or H) may come from the previous kernel
-            int it = 0;
+            uint32_t s = 0, ph = 0;                                // ring position of the next k-block (stepped, not divided)
             bool ok = true;
             // the A box holds a_box_rows rows of 128 B (fewer than 128 only when the whole problem has fewer rows:
             // the rest of the 128-row operand tile is never written and feeds accumulator rows nobody stores)
@@ -211,9 +211,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     n0 = local * BN_OUT;
                     plain_map = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &multi.tmB2);
                 }
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                for (int kb = 0; kb < num_kb; ++kb) {
                     if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) { ok = false; break; }
                     const uint32_t full = full0 + 8 * s;
                     const uint32_t a_dst = base + s * kStageBytes;
@@ -229,6 +227,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         if (w_kmajor) ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, kb * kUmmaBK, x, full);
                         else ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
                     }
+                    if (++s == (uint32_t)kStages) { s = 0; ph ^= 1u; }
                 }
             }
         }
@@ -236,7 +235,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            int it = 0, t = 0;
+            // Nothing is derived per MMA: the ring position is stepped, not divided, and a step's descriptors are the
+            // stage's first ones plus a constant, added to the lower descriptor word only (the single issuing thread
+            // is a dependent instruction stream; with everything derived per MMA it ran at about ten cycles per
+            // instruction and bounded the kernel).  In 16-byte units a K = 16 step advances
+            //   A, K-major (rows of 128 B, 8-row groups 1024 B apart): 2;
+            //   B, MN-major (64-column chunks 8 KB apart (LBO), 8-row k-groups 1024 B apart (SBO); K = 16 is two
+            //      k-groups): 128;  B, K-major ([N, K] weights: the boxes stack to N_MMA rows of 128 B, like A): 2.
+            const uint32_t desc_hi = (uint32_t)(ptx::make_smem_desc_sw128(0, 0, 1024) >> 32);
+            const uint32_t a_lo0 = (uint32_t)ptx::make_smem_desc_sw128(base, 16, 1024);
+            const uint32_t b_lo0 = w_kmajor ? (uint32_t)ptx::make_smem_desc_sw128(base + kUmmaABytes, 16, 1024)
+                                            : (uint32_t)ptx::make_smem_desc_sw128(base + kUmmaABytes, kUmmaBoxBBytes, 1024);
+            const uint32_t b_step = w_kmajor ? 2u : 128u;
+            uint32_t s = 0, ph = 0;
+            int t = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
                 const int buf = t & 1;
@@ -244,25 +256,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (!wait_bounded(tempty0 + 8 * buf, (((uint32_t)t >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4)) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kUmmaN);
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (uint32_t)(it / kStages) & 1u;
+                for (int kb = 0; kb < num_kb; ++kb) {
                     if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
-                    const uint32_t a_base = base + s * kStageBytes;
-                    const uint32_t b_base = a_base + kUmmaABytes;
+                    const uint32_t a_lo = a_lo0 + s * (kStageBytes >> 4), b_lo = b_lo0 + s * (kStageBytes >> 4);
+                    ptx::umma_bf16_halves(d_tmem, a_lo, b_lo, desc_hi, kIdesc, kb != 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k = 0; k < kUmmaBK / 16; ++k) {
-                        // A: K-major, rows of 128 B, 8-row groups 1024 B apart; +32 B per K = 16 step.
-                        // B: MN-major, 64-column chunks 8 KB apart (LBO), 8-row k-groups 1024 B apart (SBO);
-                        //    K = 16 is two k-groups: +2048 B per step.
-                        const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
-                        //    K-major B ([N, K] weights): the boxes stack to N_MMA rows of 128 B, same form as A.
-                        const uint64_t b_desc = w_kmajor ? ptx::make_smem_desc_sw128(b_base + k * 32, 16, 1024)
-                                                         : ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
-                        ptx::umma_bf16(d_tmem, a_desc, b_desc, kIdesc, (kb | k) != 0 ? 1u : 0u);
-                    }
+                    for (int k = 1; k < kUmmaBK / 16; ++k)
+                        ptx::umma_bf16_halves(d_tmem, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
                     ptx::umma_commit(empty0 + 8 * s);      // stage is free once these MMAs have read it
+                    if (++s == (uint32_t)kStages) { s = 0; ph ^= 1u; }
                 }
                 if (ok) ptx::umma_commit(tfull0 + 8 * buf);   // accumulator complete
             }

@@ -89,10 +89,8 @@ umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (warp == 0) {
         if (lane == 0) {
             ptx::grid_dependency_wait();
-            int it = 0;
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                const int s = it % kSplitStages;
-                const uint32_t ph = (uint32_t)(it / kSplitStages) & 1u;
+            uint32_t s = 0, ph = 0;                                // ring position, stepped
+            for (int kb = kb0; kb < kb1; ++kb) {
                 if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
                 const uint32_t full = full0 + 8 * s;
                 const uint32_t a_dst = base + s * kSplitStageBytes;
@@ -106,28 +104,30 @@ umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     ptx::tma_load_2d(b_dst, &tmB, n0, kb * kUmmaBK, full);
                     ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, n0 + 64, kb * kUmmaBK, full);
                 }
+                if (++s == (uint32_t)kSplitStages) { s = 0; ph ^= 1u; }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
-            int it = 0;
+            // lean issue loop: see umma_gemm.cuh (stepped ring position, one addition per descriptor)
+            const uint32_t desc_hi = (uint32_t)(ptx::make_smem_desc_sw128(0, 0, 1024) >> 32);
+            const uint32_t a_lo0 = (uint32_t)ptx::make_smem_desc_sw128(base, 16, 1024);
+            const uint32_t b_lo0 = w_kmajor ? (uint32_t)ptx::make_smem_desc_sw128(base + kUmmaABytes, 16, 1024)
+                                            : (uint32_t)ptx::make_smem_desc_sw128(base + kUmmaABytes, kUmmaBoxBBytes, 1024);
+            const uint32_t b_step = w_kmajor ? 2u : 128u;
+            uint32_t s = 0, ph = 0;
             bool ok = true;
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                const int s = it % kSplitStages;
-                const uint32_t ph = (uint32_t)(it / kSplitStages) & 1u;
+            for (int kb = kb0; kb < kb1; ++kb) {
                 if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
-                const uint32_t a_base = base + s * kSplitStageBytes;
-                const uint32_t b_base = a_base + kUmmaABytes;
+                const uint32_t a_lo = a_lo0 + s * (kSplitStageBytes >> 4), b_lo = b_lo0 + s * (kSplitStageBytes >> 4);
+                ptx::umma_bf16_halves(tmem_base, a_lo, b_lo, desc_hi, kIdesc, kb != kb0 ? 1u : 0u);
 #pragma unroll
-                for (int k = 0; k < kUmmaBK / 16; ++k) {
-                    const uint64_t a_desc = ptx::make_smem_desc_sw128(a_base + k * 32, 16, 1024);
-                    const uint64_t b_desc = w_kmajor ? ptx::make_smem_desc_sw128(b_base + k * 32, 16, 1024)
-                                                     : ptx::make_smem_desc_sw128(b_base + k * 2048, kUmmaBoxBBytes, 1024);
-                    ptx::umma_bf16(tmem_base, a_desc, b_desc, kIdesc, (it | k) != 0 ? 1u : 0u);
-                }
+                for (int k = 1; k < kUmmaBK / 16; ++k)
+                    ptx::umma_bf16_halves(tmem_base, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
                 ptx::umma_commit(empty0 + 8 * s);
+                if (++s == (uint32_t)kSplitStages) { s = 0; ph ^= 1u; }
             }
             if (ok) ptx::umma_commit(tfull);
         }
