@@ -236,7 +236,11 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         __syncwarp();
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        // All 32 lanes run the loop, its waits and its arithmetic, so that everything the MMAs take is warp-uniform
+        // (the tensor-core instructions read their operands from uniform registers; inside a one-lane branch every
+        // operand has to be moved there per MMA); only the instructions themselves sit under the elected lane.
+        {
+            const bool leader = ptx::elect_one();
             // The issuing thread is a single dependent instruction stream with a budget of 64 cycles per MMA, so
             // nothing is derived per MMA: the FIFO position is stepped, not divided, and the descriptors of a group
             // of eight K = 16 steps are formed (base + constant, independent of one another) before its first MMA.
@@ -244,7 +248,7 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             // the next atom of 128 rows; the MN-major V operand by 128 per 16 keys and by 1024 per 64 keys.
             uint32_t it_slot = 0, it_phase = 0;                      // next K/V item (K(0), V(0), K(1), ...) to wait for
             auto wait_next = [&](int site, uint32_t& slot_out) -> bool {
-                const bool ok = wait_bounded(kv_full0 + 8 * it_slot, it_phase, abort_flag, KERNEL_ID, site);
+                const bool ok = __all_sync(0xFFFFFFFFu, wait_bounded(kv_full0 + 8 * it_slot, it_phase, abort_flag, KERNEL_ID, site));
                 ptx::tc_fence_after_sync();
                 slot_out = it_slot;
                 if (++it_slot == (uint32_t)kGqaSlots) { it_slot = 0; it_phase ^= 1u; }
@@ -267,14 +271,17 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     ad[k] = a0 + (uint32_t)((k >> 2) * 1024 + (k & 3) * 2);
                     bd[k] = b0 + (uint32_t)((k >> 2) * 1024 + (k & 3) * 2);
                 }
+                if (leader) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    ptx::umma_bf16_halves(tmem_base + 128u * (uint32_t)t, ad[k], bd[k], desc_hi, kIdescQK, k != 0 ? 1u : 0u);
-                ptx::umma_commit(s_full0 + 8 * t);
-                if (t == 1) ptx::umma_commit(kv_empty0 + 8 * slot);              // both tiles have used this K block
+                    for (int k = 0; k < 8; ++k)
+                        ptx::umma_bf16_halves(tmem_base + 128u * (uint32_t)t, ad[k], bd[k], desc_hi, kIdescQK, k != 0 ? 1u : 0u);
+                    ptx::umma_commit(s_full0 + 8 * t);
+                    if (t == 1) ptx::umma_commit(kv_empty0 + 8 * slot);          // both tiles have used this K block
+                }
+                __syncwarp();
             };
             uint32_t k_slot = 0, v_slot = 0;
-            bool ok = wait_bounded(q_full, 0u, abort_flag, KERNEL_ID, 5) && wait_next(2, k_slot);
+            bool ok = __all_sync(0xFFFFFFFFu, wait_bounded(q_full, 0u, abort_flag, KERNEL_ID, 5)) && wait_next(2, k_slot);
             if (ok) {
                 issue_scores(0, k_slot);
                 issue_scores(1, k_slot);
@@ -282,7 +289,7 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             for (int j = 0; j < n_blocks && ok; ++j) {
                 for (int t = 0; t < 2 && ok; ++t) {
                     // tile t's probabilities of block j are in TMEM; V(j) has landed
-                    if (!wait_bounded(p_full0 + 8 * t, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 6)) { ok = false; break; }
+                    if (!__all_sync(0xFFFFFFFFu, wait_bounded(p_full0 + 8 * t, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 6))) { ok = false; break; }
                     if (t == 0 && !wait_next(9, v_slot)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
                     {
@@ -292,13 +299,16 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         uint32_t bd[8];
 #pragma unroll
                         for (int k = 0; k < 8; ++k) bd[k] = v0 + (uint32_t)((k >> 2) * 1024 + (k & 3) * 128);
-                        umma_bf16_tmem_a_halves(d_tmem, p_tmem, bd[0], desc_hi, kIdescPV, j != 0 ? 1u : 0u);
+                        if (leader) {
+                            umma_bf16_tmem_a_halves(d_tmem, p_tmem, bd[0], desc_hi, kIdescPV, j != 0 ? 1u : 0u);
 #pragma unroll
-                        for (int k = 1; k < 8; ++k)
-                            umma_bf16_tmem_a_halves(d_tmem, p_tmem + 8u * (uint32_t)k, bd[k], desc_hi, kIdescPV, 1u);
+                            for (int k = 1; k < 8; ++k)
+                                umma_bf16_tmem_a_halves(d_tmem, p_tmem + 8u * (uint32_t)k, bd[k], desc_hi, kIdescPV, 1u);
+                            ptx::umma_commit(o_full0 + 8 * t);
+                            if (t == 1) ptx::umma_commit(kv_empty0 + 8 * v_slot);    // both tiles have used V(j)
+                        }
+                        __syncwarp();
                     }
-                    ptx::umma_commit(o_full0 + 8 * t);
-                    if (t == 1) ptx::umma_commit(kv_empty0 + 8 * v_slot);        // both tiles have used V(j)
                     // the tile's next scores follow at once: its score buffer was consumed before p_full
                     if (j + 1 < n_blocks) {
                         if (t == 0 && !wait_next(2, k_slot)) { ok = false; break; }
