@@ -234,7 +234,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         __syncwarp();
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        // All 32 lanes run the loop, its waits and its arithmetic, so that everything the MMAs take is warp-uniform
+        // (the tensor-core instructions read their operands from uniform registers; inside a one-lane branch every
+        // operand would have to be moved there per MMA); only the instructions themselves sit under the elected lane.
+        {
+            const bool leader = ptx::elect_one();
             // Nothing is derived per MMA: the ring position is stepped, not divided, and a step's descriptors are the
             // stage's first ones plus a constant, added to the lower descriptor word only (the single issuing thread
             // is a dependent instruction stream; with everything derived per MMA it ran at about ten cycles per
@@ -253,21 +257,25 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
                 const int buf = t & 1;
                 // the epilogue must have drained this accumulator buffer (two tiles ago)
-                if (!wait_bounded(tempty0 + 8 * buf, (((uint32_t)t >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4)) break;
+                if (!__all_sync(0xFFFFFFFFu, wait_bounded(tempty0 + 8 * buf, (((uint32_t)t >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4))) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kUmmaN);
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
+                    if (!__all_sync(0xFFFFFFFFu, wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2))) { ok = false; break; }
                     ptx::tc_fence_after_sync();
                     const uint32_t a_lo = a_lo0 + s * (kStageBytes >> 4), b_lo = b_lo0 + s * (kStageBytes >> 4);
-                    ptx::umma_bf16_halves(d_tmem, a_lo, b_lo, desc_hi, kIdesc, kb != 0 ? 1u : 0u);
+                    if (leader) {
+                        ptx::umma_bf16_halves(d_tmem, a_lo, b_lo, desc_hi, kIdesc, kb != 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k = 1; k < kUmmaBK / 16; ++k)
-                        ptx::umma_bf16_halves(d_tmem, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
-                    ptx::umma_commit(empty0 + 8 * s);      // stage is free once these MMAs have read it
+                        for (int k = 1; k < kUmmaBK / 16; ++k)
+                            ptx::umma_bf16_halves(d_tmem, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
+                        ptx::umma_commit(empty0 + 8 * s);  // stage is free once these MMAs have read it
+                    }
+                    __syncwarp();
                     if (++s == (uint32_t)kStages) { s = 0; ph ^= 1u; }
                 }
-                if (ok) ptx::umma_commit(tfull0 + 8 * buf);   // accumulator complete
+                if (ok && leader) ptx::umma_commit(tfull0 + 8 * buf);   // accumulator complete
+                __syncwarp();
             }
         }
         __syncwarp();

@@ -197,8 +197,12 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ---------------- MMA issuer (leader only) ----------------
-        if (lane == 0 && rank == 0) {
+        // ---------------- MMA issuer (leader CTA only) ----------------
+        // All 32 lanes run the loop, its waits and its arithmetic, so that everything the MMAs take is warp-uniform
+        // (the tensor-core instructions read their operands from uniform registers; inside a one-lane branch every
+        // operand would have to be moved there per MMA); only the instructions themselves sit under the elected lane.
+        if (rank == 0) {
+            const bool leader = ptx::elect_one();
             // Nothing is derived per MMA: the ring position is stepped, not divided, and a step's descriptors are
             // the stage's first ones plus a constant (in 16-byte units: 2 per K = 16 step of a K-major operand,
             // 128 of the MN-major weights); only the lower descriptor word changes.
@@ -212,21 +216,25 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++t) {
                 const int buf = t & 1;
-                if (!wait_bounded(tempty0 + 8 * buf, (((uint32_t)t >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4)) break;
+                if (!__all_sync(0xFFFFFFFFu, wait_bounded(tempty0 + 8 * buf, (((uint32_t)t >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4))) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 256);
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
+                    if (!__all_sync(0xFFFFFFFFu, wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2))) { ok = false; break; }
                     ptx::tc_fence_after_sync();
                     const uint32_t a_lo = a_lo0 + s * (kPairStageBytes >> 4), b_lo = b_lo0 + s * (kPairStageBytes >> 4);
-                    ptx::umma_bf16_pair_halves(d_tmem, a_lo, b_lo, desc_hi, kIdesc, kb != 0 ? 1u : 0u);
+                    if (leader) {
+                        ptx::umma_bf16_pair_halves(d_tmem, a_lo, b_lo, desc_hi, kIdesc, kb != 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k = 1; k < kUmmaBK / 16; ++k)
-                        ptx::umma_bf16_pair_halves(d_tmem, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
-                    ptx::umma_commit_pair(empty0 + 8 * s);
+                        for (int k = 1; k < kUmmaBK / 16; ++k)
+                            ptx::umma_bf16_pair_halves(d_tmem, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
+                        ptx::umma_commit_pair(empty0 + 8 * s);
+                    }
+                    __syncwarp();
                     if (++s == (uint32_t)kPairStages) { s = 0; ph ^= 1u; }
                 }
-                if (ok) ptx::umma_commit_pair(tfull0 + 8 * buf);
+                if (ok && leader) ptx::umma_commit_pair(tfull0 + 8 * buf);
+                __syncwarp();
             }
         }
         __syncwarp();
