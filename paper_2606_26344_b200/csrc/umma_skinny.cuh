@@ -332,11 +332,23 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         __syncwarp();
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        // All 32 lanes run the loop, its waits and its arithmetic, so that everything the MMAs take is warp-uniform
+        // (the tensor-core instructions read their operands from uniform registers); only the instructions
+        // themselves sit under the elected lane.  Nothing is derived per MMA: a descriptor is the stage's first one
+        // plus a constant, added to the lower descriptor word (the upper word is the same for all).
+        {
+            const bool leader = ptx::elect_one();
             // D = fp32, A = B = bf16, A (weights) MN-major, B (tokens) K-major, M = 128, N = Mpad
             // (weights stored [N, K]: A is K-major too, bit 15 clear)
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((w_kmajor ? 0u : 1u) << 15) | (0u << 16) |
                                    ((uint32_t)(Mpad >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+            const uint32_t desc_hi = (uint32_t)(ptx::make_smem_desc_sw128(0, 0, 1024) >> 32);
+            const uint32_t tok_lo0 = (uint32_t)ptx::make_smem_desc_sw128(base + W_BYTES, 16, 1024);
+            // weights stored [N, K]: the two boxes stack to 128 rows of 128 B, K-major like the tokens
+            const uint32_t w_lo0 = w_kmajor ? (uint32_t)ptx::make_smem_desc_sw128(base, 16, 1024)
+                                            : (uint32_t)ptx::make_smem_desc_sw128(base, kSkinnyBoxBytes, 1024);
+            const uint32_t w_step = w_kmajor ? 2u : 128u;            // 16-byte units per K = 16 step
+            const uint32_t stage16 = stage_bytes >> 4;
             int seg = 0, s = 0, kb = (int)(u_begin - div_fast(u_begin, KB) * KB);   // ring slot, its phase and the k-block are stepped
             uint32_t ph = 0u;
             bool fresh = true;
@@ -344,31 +356,30 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 const int buf = seg & 1;
                 if (fresh) {
                     // the accumulator buffer must have been drained by the epilogue two segments ago
-                    if (!wait_bounded(tempty0 + 8 * buf, (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4)) break;
+                    if (!__all_sync(0xFFFFFFFFu, wait_bounded(tempty0 + 8 * buf, (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4))) break;
                     ptx::tc_fence_after_sync();
                 }
-                if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) break;
+                if (!__all_sync(0xFFFFFFFFu, wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2))) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t st = base + s * stage_bytes;
+                const uint32_t tok_lo = tok_lo0 + (uint32_t)s * stage16, w_lo = w_lo0 + (uint32_t)s * stage16;
+                const bool last_of_segment = kb == KB - 1 || u == u_end - 1;
+                if (leader) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const uint64_t b_desc = ptx::make_smem_desc_sw128(st + W_BYTES + k * 32, 16, 1024);
+                    for (int k = 0; k < 4; ++k) {
 #pragma unroll
-                    for (int j = 0; j < NMAT; ++j)
+                        for (int j = 0; j < NMAT; ++j)
 #pragma unroll
-                        for (int h = 0; h < NH; ++h) {
-                            // weights stored [N, K]: the two boxes stack to 128 rows of 128 B, K-major like the tokens
-                            const uint32_t w_base = st + (j * NH + h) * 2 * kSkinnyBoxBytes;
-                            const uint64_t a_desc = w_kmajor ? ptx::make_smem_desc_sw128(w_base + k * 32, 16, 1024)
-                                                             : ptx::make_smem_desc_sw128(w_base + k * 2048, kSkinnyBoxBytes, 1024);
-                            ptx::umma_bf16(tmem_base + acc_col(buf, j, h), a_desc, b_desc, idesc,
-                                           (fresh && k == 0) ? 0u : 1u);
-                        }
+                            for (int h = 0; h < NH; ++h)
+                                ptx::umma_bf16_halves(tmem_base + acc_col(buf, j, h),
+                                                      w_lo + (uint32_t)((j * NH + h) * ((2 * kSkinnyBoxBytes) >> 4)) + w_step * (uint32_t)k,
+                                                      tok_lo + 2u * (uint32_t)k, desc_hi, idesc, (fresh && k == 0) ? 0u : 1u);
+                    }
+                    ptx::umma_commit(empty0 + 8 * s);
+                    if (last_of_segment) ptx::umma_commit(tfull0 + 8 * buf);
                 }
+                __syncwarp();
                 fresh = false;
-                ptx::umma_commit(empty0 + 8 * s);
-                if (kb == KB - 1 || u == u_end - 1) {
-                    ptx::umma_commit(tfull0 + 8 * buf);
+                if (last_of_segment) {
                     ++seg;
                     fresh = true;
                 }
