@@ -160,7 +160,9 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs) ----------------
-        if (lane == 0) {
+        // (warp-uniform like the MMA issuer: coordinates and addresses by all lanes, the copies by the elected one)
+        {
+            const bool leader = ptx::elect_one();
             if (!ROWSCALE) ptx::grid_dependency_wait();
             const uint32_t leader_full0 = ptx::map_to_cta(full0, 0);
             uint32_t s = 0, ph = 0;                              // ring position of the next k-block
@@ -178,19 +180,22 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 }
                 const int bx = GATEUP ? n0 : n0 + (int)rank * 128;
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) { ok = false; break; }
+                    if (!__all_sync(0xFFFFFFFFu, wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1))) { ok = false; break; }
                     const uint32_t full = leader_full0 + 8 * s;
                     const uint32_t a_dst = base + s * kPairStageBytes;
                     const uint32_t b_dst = a_dst + kPairABytes;
-                    ptx::mbar_arrive_expect_tx_cluster(full, kPairStageBytes);
-                    ptx::tma_load_2d_pair(a_dst, &tmA, kb * kUmmaBK, m0, full);
-                    if (w_kmajor) {                        // [N, K] weights: boxes of 64 k x 64 rows of N
-                        ptx::tma_load_2d_pair(b_dst, bmap, kb * kUmmaBK, bx, full);
-                        ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, kb * kUmmaBK, bx + 64, full);
-                    } else {                               // [K, N] weights: boxes of 64 columns x 64 k
-                        ptx::tma_load_2d_pair(b_dst, bmap, bx, kb * kUmmaBK, full);
-                        ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, bx + 64, kb * kUmmaBK, full);
+                    if (leader) {
+                        ptx::mbar_arrive_expect_tx_cluster(full, kPairStageBytes);
+                        ptx::tma_load_2d_pair(a_dst, &tmA, kb * kUmmaBK, m0, full);
+                        if (w_kmajor) {                    // [N, K] weights: boxes of 64 k x 64 rows of N
+                            ptx::tma_load_2d_pair(b_dst, bmap, kb * kUmmaBK, bx, full);
+                            ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, kb * kUmmaBK, bx + 64, full);
+                        } else {                           // [K, N] weights: boxes of 64 columns x 64 k
+                            ptx::tma_load_2d_pair(b_dst, bmap, bx, kb * kUmmaBK, full);
+                            ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, bx + 64, kb * kUmmaBK, full);
+                        }
                     }
+                    __syncwarp();
                     if (++s == (uint32_t)kPairStages) { s = 0; ph ^= 1u; }
                 }
             }

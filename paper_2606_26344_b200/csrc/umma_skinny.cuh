@@ -284,13 +284,17 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        if (lane == 0) {
+        // (warp-uniform like the MMA issuer: coordinates and addresses are computed by all lanes, the copies are
+        // issued by the elected one)
+        {
+            const bool leader = ptx::elect_one();
             const uint64_t policy = ptx::l2_policy_evict_first();
             // (tile, k-block) of a unit are carried along and stepped, never recomputed: 64-bit divisions by a
             // run-time KB cost this single thread hundreds of cycles per unit, as much as the unit's share of time
             auto load_weights = [&](int tile, int kb, int s) {
                 const uint32_t full = full0 + 8 * s;
                 const uint32_t st = base + s * stage_bytes;
+                if (!leader) return;
                 ptx::mbar_arrive_expect_tx(full, stage_bytes);
 #pragma unroll
                 for (int j = 0; j < NMAT; ++j)
@@ -308,7 +312,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     }
             };
             auto load_tokens = [&](int kb, int s) {
-                ptx::tma_load_2d(base + s * stage_bytes + W_BYTES, &tmX, kb * 64, 0, full0 + 8 * s);
+                if (leader) ptx::tma_load_2d(base + s * stage_bytes + W_BYTES, &tmX, kb * 64, 0, full0 + 8 * s);
             };
             auto step = [&](int& tile, int& kb) { if (++kb == KB) { kb = 0; ++tile; } };
             const int tile0 = (int)div_fast(u_begin, KB), kb0 = (int)(u_begin - (long long)tile0 * KB);
@@ -322,9 +326,10 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             int s = head == stages ? 0 : head;                     // ring slot and its phase, stepped as well
             uint32_t ph = head == stages ? 1u : 0u;
             for (long long u = u_begin + head; u < u_end; ++u) {
-                if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
+                if (!__all_sync(0xFFFFFFFFu, wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1))) break;
                 load_weights(tile, kb, s);
                 load_tokens(kb, s);
+                __syncwarp();
                 step(tile, kb);
                 if (++s == stages) { s = 0; ph ^= 1u; }
             }
