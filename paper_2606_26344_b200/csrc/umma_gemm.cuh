@@ -194,7 +194,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // one round work on the same few weight panels (L2 reuse).
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        if (lane == 0) {
+        // (warp-uniform like the MMA issuer: coordinates and addresses by all lanes, the copies by the elected one)
+        {
+            const bool leader = ptx::elect_one();
             if (!ROWSCALE) ptx::grid_dependency_wait();           // A (Xn or H) may come from the previous kernel
             uint32_t s = 0, ph = 0;                                // ring position of the next k-block (stepped, not divided)
             bool ok = true;
@@ -212,21 +214,24 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     plain_map = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &multi.tmB2);
                 }
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) { ok = false; break; }
+                    if (!__all_sync(0xFFFFFFFFu, wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1))) { ok = false; break; }
                     const uint32_t full = full0 + 8 * s;
                     const uint32_t a_dst = base + s * kStageBytes;
                     const uint32_t b_dst = a_dst + kUmmaABytes;
-                    ptx::mbar_arrive_expect_tx(full, a_tx_bytes + NB * kUmmaBoxBBytes);
-                    ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
+                    if (leader) {
+                        ptx::mbar_arrive_expect_tx(full, a_tx_bytes + NB * kUmmaBoxBBytes);
+                        ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
 #pragma unroll
-                    for (int i = 0; i < NB; ++i) {
-                        // gate/up: the first NB/2 boxes are gate columns, the rest the same columns of up
-                        const CUtensorMap* map = (GATEUP && i >= NB / 2) ? &tmB1 : plain_map;
-                        const int x = GATEUP ? n0 + (i % (NB / 2)) * 64 : n0 + i * 64;
-                        // [K, N] weights: box of 64 columns x 64 k; [N, K] weights: box of 64 k x 64 rows of N
-                        if (w_kmajor) ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, kb * kUmmaBK, x, full);
-                        else ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
+                        for (int i = 0; i < NB; ++i) {
+                            // gate/up: the first NB/2 boxes are gate columns, the rest the same columns of up
+                            const CUtensorMap* map = (GATEUP && i >= NB / 2) ? &tmB1 : plain_map;
+                            const int x = GATEUP ? n0 + (i % (NB / 2)) * 64 : n0 + i * 64;
+                            // [K, N] weights: box of 64 columns x 64 k; [N, K] weights: box of 64 k x 64 rows of N
+                            if (w_kmajor) ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, kb * kUmmaBK, x, full);
+                            else ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
+                        }
                     }
+                    __syncwarp();
                     if (++s == (uint32_t)kStages) { s = 0; ph ^= 1u; }
                 }
             }

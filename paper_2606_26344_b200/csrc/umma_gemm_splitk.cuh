@@ -86,30 +86,37 @@ umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
+    // producer and MMA issuer run their loops warp-uniformly; the copies and the tensor-core instructions sit under the
+    // elected lane (see umma_gemm.cuh)
     if (warp == 0) {
-        if (lane == 0) {
+        {
+            const bool leader = ptx::elect_one();
             ptx::grid_dependency_wait();
             uint32_t s = 0, ph = 0;                                // ring position, stepped
             for (int kb = kb0; kb < kb1; ++kb) {
-                if (!wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1)) break;
+                if (!__all_sync(0xFFFFFFFFu, wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1))) break;
                 const uint32_t full = full0 + 8 * s;
                 const uint32_t a_dst = base + s * kSplitStageBytes;
                 const uint32_t b_dst = a_dst + kUmmaABytes;
-                ptx::mbar_arrive_expect_tx(full, (uint32_t)a_box_rows * 128u + 2 * kUmmaBoxBBytes);
-                ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
-                if (w_kmajor) {
-                    ptx::tma_load_2d(b_dst, &tmB, kb * kUmmaBK, n0, full);
-                    ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, kb * kUmmaBK, n0 + 64, full);
-                } else {
-                    ptx::tma_load_2d(b_dst, &tmB, n0, kb * kUmmaBK, full);
-                    ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, n0 + 64, kb * kUmmaBK, full);
+                if (leader) {
+                    ptx::mbar_arrive_expect_tx(full, (uint32_t)a_box_rows * 128u + 2 * kUmmaBoxBBytes);
+                    ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
+                    if (w_kmajor) {
+                        ptx::tma_load_2d(b_dst, &tmB, kb * kUmmaBK, n0, full);
+                        ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, kb * kUmmaBK, n0 + 64, full);
+                    } else {
+                        ptx::tma_load_2d(b_dst, &tmB, n0, kb * kUmmaBK, full);
+                        ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, n0 + 64, kb * kUmmaBK, full);
+                    }
                 }
+                __syncwarp();
                 if (++s == (uint32_t)kSplitStages) { s = 0; ph ^= 1u; }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
+        {
+            const bool leader = ptx::elect_one();
             // lean issue loop: see umma_gemm.cuh (stepped ring position, one addition per descriptor)
             const uint32_t desc_hi = (uint32_t)(ptx::make_smem_desc_sw128(0, 0, 1024) >> 32);
             const uint32_t a_lo0 = (uint32_t)ptx::make_smem_desc_sw128(base, 16, 1024);
@@ -119,17 +126,21 @@ umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             uint32_t s = 0, ph = 0;
             bool ok = true;
             for (int kb = kb0; kb < kb1; ++kb) {
-                if (!wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2)) { ok = false; break; }
+                if (!__all_sync(0xFFFFFFFFu, wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2))) { ok = false; break; }
                 ptx::tc_fence_after_sync();
                 const uint32_t a_lo = a_lo0 + s * (kSplitStageBytes >> 4), b_lo = b_lo0 + s * (kSplitStageBytes >> 4);
-                ptx::umma_bf16_halves(tmem_base, a_lo, b_lo, desc_hi, kIdesc, kb != kb0 ? 1u : 0u);
+                if (leader) {
+                    ptx::umma_bf16_halves(tmem_base, a_lo, b_lo, desc_hi, kIdesc, kb != kb0 ? 1u : 0u);
 #pragma unroll
-                for (int k = 1; k < kUmmaBK / 16; ++k)
-                    ptx::umma_bf16_halves(tmem_base, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
-                ptx::umma_commit(empty0 + 8 * s);
+                    for (int k = 1; k < kUmmaBK / 16; ++k)
+                        ptx::umma_bf16_halves(tmem_base, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
+                    ptx::umma_commit(empty0 + 8 * s);
+                }
+                __syncwarp();
                 if (++s == (uint32_t)kSplitStages) { s = 0; ph ^= 1u; }
             }
-            if (ok) ptx::umma_commit(tfull);
+            if (ok && leader) ptx::umma_commit(tfull);
+            __syncwarp();
         }
         __syncwarp();
     }
