@@ -303,21 +303,32 @@ int resolve_variant(int64_t M, int64_t d_model, int64_t d_ff, int32_t variant) {
     return M <= 16 ? GMLP_VARIANT_SKINNY : GMLP_VARIANT_TENSOR;
 }
 
-// TENSOR: which kernel each GEMM takes, by the number of 128-row blocks mt.  A CTA pair works on 256 rows, so an
-// odd block count leaves half a pair idle in the last row tile; measured on B200 (8B and 70B layer shapes):
-//   gate/up: pairs for even mt (mt = 2: 55.7 vs 63.3 us, 4: 97 vs 109, 6: 127 vs 135); single CTAs for odd mt
-//            (3: 85 vs 96 us, 9: 296 vs 306, 11 / 13 / 15 / 19: single ahead by 10-30 us) until the idle half
-//            is a few percent of the work (mt >= 24), where the pair kernel's higher rate wins again;
-//   down:    few output tiles at small M, so single CTAs (which can split K over a cluster) until mt = 8, then
-//            pairs, except mt = 9 (358 vs 296 us).
+// TENSOR: which kernel each GEMM takes.  Both kernels are persistent, so a GEMM costs (rounds of tiles over the SMs)
+// x (cost of a tile).  A CTA pair works on 256 rows at 0.94 of the cost of two single-CTA tiles (measured), but an
+// odd number of 128-row blocks leaves half a pair idle in the last row tile and a pair tile count just above a
+// multiple of 74 pays a whole extra round; the single-CTA kernel can narrow its tiles (128 columns at 0.75 of the
+// cost) or split K over a cluster when its tiles are few.  The counts decide; this model reproduces the measured
+// winner of all four combinations on 41 shapes (128-row blocks 2..32 on the 2048x5632, 8B and 70B layers), e.g.
+// gate/up 8B: pairs for even block counts, single CTAs for odd ones up to 23; 2048x5632: pairs from 4 blocks on;
+// down 8B: single CTAs up to 4 blocks and at 9 (307 vs 382 us), pairs otherwise.
 // gmlp_autotune measures the four combinations for a given shape and overrides this rule.
-bool gate_up_uses_pair(int64_t M) {
-    const int64_t mt = (M + 127) / 128;
-    return mt >= 24 || (mt >= 2 && mt % 2 == 0);
+int pick_split_k(int num_m, int64_t K, int64_t N, int sms);
+static double rounds_of(int64_t tiles, int64_t units) { return (double)((tiles + units - 1) / units); }
+constexpr double kPairTileCost = 0.94;
+bool gate_up_uses_pair(int64_t M, int64_t d_ff, int sms) {
+    const int64_t mt = (M + 127) / 128, ct = (d_ff + 127) / 128;
+    if (mt < 2) return false;
+    return kPairTileCost * rounds_of(((mt + 1) / 2) * ct, sms / 2) < rounds_of(mt * ct, sms);
 }
-bool down_uses_pair(int64_t M) {
+bool down_uses_pair(int64_t M, int64_t d_ff, int64_t d_model, int sms) {
     const int64_t mt = (M + 127) / 128;
-    return mt == 8 || mt >= 10;
+    if (mt < 2) return false;
+    const int64_t t256 = mt * ((d_model + 255) / 256), t128 = mt * ((d_model + 127) / 128);
+    double single = rounds_of(t256, sms);
+    if (0.75 * rounds_of(t128, sms) < single) single = 0.75 * rounds_of(t128, sms);
+    const int S = pick_split_k((int)mt, d_ff, d_model, sms);
+    if (S >= 2) single = 0.75 / S + 0.1;                                // K split over a cluster, reduced on chip
+    return kPairTileCost * rounds_of(((mt + 1) / 2) * ((d_model + 255) / 256), sms / 2) < single;
 }
 
 // The TENSOR plan of a shape: the rule above, unless gmlp_autotune measured the four combinations for this
@@ -326,8 +337,9 @@ struct TensorPlan {
     bool gu_pair, down_pair;
 };
 thread_local int t_force_gu = -1, t_force_down = -1;
-TensorPlan tensor_plan(int64_t M, int64_t d_model, int64_t d_ff) {
-    TensorPlan p = {gate_up_uses_pair(M), down_uses_pair(M)};
+TensorPlan tensor_plan(int64_t M, int64_t d_model, int64_t d_ff, int sms) {
+    if (sms <= 0) sms = 148;
+    TensorPlan p = {gate_up_uses_pair(M, d_ff, sms), down_uses_pair(M, d_ff, d_model, sms)};
     TunedShape t;
     if (tuned_lookup(M, d_model, d_ff, &t) && t.variant == GMLP_VARIANT_TENSOR) {
         p.gu_pair = t.gu_pair != 0;
@@ -846,7 +858,7 @@ int forward_impl(const gmlp_args* a) {
             }
             break;
         case GMLP_VARIANT_TENSOR: {
-            const TensorPlan plan = tensor_plan(a->M, a->d_model, a->d_ff);
+            const TensorPlan plan = tensor_plan(a->M, a->d_model, a->d_ff, dev->sm_count);
             rc = plan.gu_pair ? launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act)
                               : launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act);
             if (rc == GMLP_OK) {
@@ -1004,7 +1016,7 @@ int gate_up_impl(const gmlp_args* a) {
         rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
         if (rc == GMLP_OK) rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, Hout, a->M, a->d_model, a->d_ff, st, act);
     } else if (variant == GMLP_VARIANT_PAIR ||
-               (variant == GMLP_VARIANT_TENSOR && tensor_plan(a->M, a->d_model, a->d_ff).gu_pair)) {
+               (variant == GMLP_VARIANT_TENSOR && tensor_plan(a->M, a->d_model, a->d_ff, dev->sm_count).gu_pair)) {
         rc = launch_umma_pair<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st, act);
     } else {
         rc = launch_umma<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st, act);
