@@ -73,6 +73,40 @@ def test_peaked_softmax_and_large_scores():
     _check(200, 700, 4, 2, seed=7, q_scale=6.0)
 
 
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("slope", [0.02, 1.0, 20.0])
+def test_scores_that_rise_along_the_keys_move_the_base_in_every_block(slope, causal):
+    """Key j is (1 + slope * j) times one direction and every query is a multiple of it, so a row's scores rise along the
+    keys: gently (a block's sum of exponentials with the old base stays moderate), by hundreds or by thousands of
+    binary orders per block (the exponentials with the old base overflow and the block has to be redone with a new
+    one).  Against the oracle, and against the closed form for the steepest case: the softmax is one-hot on the last
+    key a row may see."""
+    M, S, Hq, Hkv = 300, 700, 4, 2
+    g = torch.Generator().manual_seed(11)
+    u = torch.randn(D, generator=g)
+    u = u / u.norm() * 4.0
+    ramp = 1.0 + slope * torch.arange(S, dtype=torch.float32)
+    K = (ramp[:, None] * u[None, :]).repeat(1, Hkv).to(torch.bfloat16)
+    Q = ((1.0 + torch.rand(M, 1, generator=g)) * u[None, :]).repeat(1, Hq).to(torch.bfloat16)
+    V = torch.randn(S, Hkv * D, generator=g).to(torch.bfloat16)
+    dev = torch.device("cuda")
+    O = torch.full((M, Hq * D), float("nan"), dtype=torch.bfloat16, device=dev)
+    gmlp.gqa_attention(Q.to(dev), K.to(dev), V.to(dev), Hq, Hkv, O=O, checked=True, causal=causal)
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(O.float()).all())
+    rows = np.array([0, 1, 127, 128, 129, 255, 256, 257, 298, 299])
+    ref = oracle.gqa_rows(_bits(Q), _bits(K), _bits(V), Hq, Hkv, rows=rows, causal=causal)
+    got = O[torch.as_tensor(rows, device=dev)].float().cpu().numpy().astype(np.float64)
+    e = np.abs(got - ref) / oracle.tolerance(ref)
+    assert e.max() <= 1.0, f"max err/tol {e.max():.3f}"
+    if slope == 20.0:                                    # adjacent keys differ by more than 40 nats
+        last = (rows + (S - M)) if causal else np.full(len(rows), S - 1)
+        want = V.float().numpy().astype(np.float64)[last]                        # [rows, Hkv * D]
+        for h in range(Hq):
+            gsel = slice((h // (Hq // Hkv)) * D, (h // (Hq // Hkv)) * D + D)
+            assert np.abs(got[:, h * D:(h + 1) * D] - want[:, gsel]).max() <= 2e-2 * max(1.0, np.abs(want).max())
+
+
 def test_llama_like_block():
     # 8B attention block: 32 query heads, 8 key/value heads of 128; 2048 tokens; 64 sampled query rows
     _check(2048, 2048, 32, 8, seed=3)
