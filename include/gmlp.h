@@ -309,6 +309,21 @@ int gmlp_forward_static(const void* X, const void* Wg, const void* Wu, const voi
 uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int32_t variant);
 
 /*
+ * The last step of a d_ff-sharded Gated MLP.  Y = H W_down sums over d_ff (Section 2), so the layer may be cut into
+ * shards of d_ff - the matching columns of W_gate and W_up and rows of W_down - each of which is a complete call of
+ * this library with GMLP_FLAG_Y_FP32 that leaves an fp32 partial product [M, d_model] (H, and with it the rounding
+ * of H, is per element of d_ff and does not depend on the cut).  gmlp_sum_partials adds n_partials (1..8) such
+ * buffers in the order given - fixed, so the result does not depend on scheduling - rounds once and stores bf16:
+ *   Y[i] = bf16_rn(partials[0][i] + partials[1][i] + ...),   i < count.
+ * partials is a HOST array of DEVICE pointers (fp32, 16-byte aligned, count elements each); Y is a device pointer
+ * (bf16, 16-byte aligned); count must be a multiple of 8.  With one process per GPU the partials are first summed
+ * across ranks by the caller's collective (one all-reduce of M * d_model floats) and n_partials is 1.
+ * Asynchronous on `stream` (a cudaStream_t, NULL = the default stream).  Returns GMLP_OK, GMLP_ERR_NULL,
+ * GMLP_ERR_SHAPE (n_partials or count), GMLP_ERR_ALIGN, GMLP_ERR_ARCH or GMLP_ERR_LAUNCH.
+ */
+int gmlp_sum_partials(const void* const* partials, int32_t n_partials, void* Y, uint64_t count, void* stream);
+
+/*
  * Drop what the library remembers about the contents of caller-made workspaces on the current device (the
  * arrival counters it believes to be zero; see "Ownership" above): those inside [workspace, workspace + bytes),
  * or all of them when `workspace` is NULL.  The next call that uses such a workspace zeroes its counters again

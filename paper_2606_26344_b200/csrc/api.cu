@@ -1525,6 +1525,38 @@ int gmlp_autotune_query(int64_t M, int64_t d_model, int64_t d_ff, int32_t* varia
     return 1;
 }
 
+int gmlp_sum_partials(const void* const* partials, int32_t n_partials, void* Y, uint64_t count, void* stream) {
+    if (partials == nullptr || Y == nullptr) return GMLP_ERR_NULL;
+    if (n_partials < 1 || n_partials > gmlp::kMaxPartials) return GMLP_ERR_SHAPE;
+    if (count % 8 != 0) return GMLP_ERR_SHAPE;
+    if (!aligned16(Y)) return GMLP_ERR_ALIGN;
+    gmlp::PartialList list = {};
+    list.n = n_partials;
+    for (int i = 0; i < n_partials; ++i) {
+        if (partials[i] == nullptr) return GMLP_ERR_NULL;
+        if (!aligned16(partials[i])) return GMLP_ERR_ALIGN;
+        list.p[i] = static_cast<const float*>(partials[i]);
+    }
+    int rc = GMLP_OK;
+    DeviceState* dev = current_device(&rc);
+    if (dev == nullptr) return rc;
+    if (count == 0) return GMLP_OK;
+    const size_t nvec4 = (size_t)(count / 4);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((nvec4 + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, gmlp::sum_partials_bf16_kernel, list, static_cast<bf16*>(Y), nvec4) != cudaSuccess)
+        return GMLP_ERR_LAUNCH;
+    GMLP_CHECK_LAUNCH();
+    return GMLP_OK;
+}
+
 int gmlp_workspace_forget(const void* workspace, uint64_t bytes) {
     int rc = GMLP_OK;
     DeviceState* dev = current_device(&rc);

@@ -155,4 +155,27 @@ add_bf16_kernel(const bf16* __restrict__ T, const bf16* __restrict__ R, bf16* __
     reinterpret_cast<uint4*>(S)[i] = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
+// d_ff-sharded Gated MLP: each shard (a slice of d_ff: the matching columns of W_gate / W_up and rows of W_down)
+// yields an fp32 partial product of the down projection, Y = sum over shards of H_s W_down,s.  This kernel adds up to
+// kMaxPartials partials in the order given (fixed: the result does not depend on scheduling), rounds once and
+// stores bf16.  count is a multiple of 4; 16 bytes loaded per partial and thread.
+constexpr int kMaxPartials = 8;
+struct PartialList {
+    const float* p[kMaxPartials];
+    int n;
+};
+__global__ void __launch_bounds__(256)
+sum_partials_bf16_kernel(PartialList parts, bf16* __restrict__ Y, size_t nvec4)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");           // the partials may come from the previous kernel
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= nvec4) return;
+    float4 acc = reinterpret_cast<const float4*>(parts.p[0])[i];
+    for (int s = 1; s < parts.n; ++s) {
+        const float4 v = reinterpret_cast<const float4*>(parts.p[s])[i];
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    reinterpret_cast<uint2*>(Y)[i] = make_uint2(pack_bf16x2(acc.x, acc.y), pack_bf16x2(acc.z, acc.w));
+}
+
 }  // namespace gmlp

@@ -132,6 +132,9 @@ def lib() -> ctypes.CDLL:
         L.gmlp_autotune_query.argtypes = [i64, i64, i64] + [ctypes.POINTER(ctypes.c_int32)] * 3
         L.gmlp_autotune_clear.restype = None
         L.gmlp_autotune_clear.argtypes = []
+        L.gmlp_sum_partials.restype = ctypes.c_int
+        L.gmlp_sum_partials.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int32, ctypes.c_void_p, ctypes.c_uint64,
+                                        ctypes.c_void_p]
         L.gmlp_workspace_forget.restype = ctypes.c_int
         L.gmlp_workspace_forget.argtypes = [ctypes.c_void_p, ctypes.c_uint64]
         L.gmlp_pick_variant.restype = ctypes.c_int
@@ -523,3 +526,23 @@ def gqa_attention(Q, K, V, n_q_heads: int, n_kv_heads: int, O=None, stream=None,
     with torch.cuda.device(Q.device):
         gqa_attention_ex(make_gqa_args(Q, K, V, O, n_q_heads, n_kv_heads, stream, checked, causal))
     return O
+
+
+def sum_partials(parts, Y=None, stream=None) -> "torch.Tensor":
+    """gmlp_sum_partials: Y = bf16(parts[0] + parts[1] + ...) over fp32 partial products of equal shape (the last
+    step of a d_ff-sharded Gated MLP); the sum runs in the order given."""
+    if not parts:
+        raise ValueError("no partial products")
+    for t in parts:
+        if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and t.shape == parts[0].shape):
+            raise ValueError("partial products must be contiguous float32 CUDA tensors of one shape")
+    if Y is None:
+        Y = torch.empty(parts[0].shape, dtype=torch.bfloat16, device=parts[0].device)
+    _check_bf16_cuda(Y, "Y")
+    ptrs = (ctypes.c_void_p * len(parts))(*[t.data_ptr() for t in parts])
+    st = stream.cuda_stream if stream is not None else torch.cuda.current_stream(Y.device).cuda_stream
+    with torch.cuda.device(Y.device):
+        rc = lib().gmlp_sum_partials(ptrs, len(parts), Y.data_ptr(), Y.numel(), st)
+    if rc != OK:
+        raise GmlpError(rc)
+    return Y
