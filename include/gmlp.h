@@ -340,7 +340,10 @@ int gmlp_workspace_forget(const void* workspace, uint64_t bytes);
  * skipped), about `iters` (1..10000) timed back-to-back calls each, in four interleaved rounds after a warm-up
  * round so that clock drift falls on all candidates alike, CUDA events on args->stream, and
  * remembers the fastest for (current device, M, d_model, d_ff): GMLP_VARIANT_AUTO, gmlp_pick_variant and
- * gmlp_workspace_bytes use it from then on (size workspaces after tuning).  Synchronises the stream.
+ * gmlp_workspace_bytes use it from then on (size workspaces after tuning).  When a single-CTA kernel is part of
+ * the winner, a second stage measures its tile forms the same way (gate/up: 64- or 128-column tiles; down: K split
+ * over a cluster of 2, 3 or 4 CTAs, or 128- or 256-column tiles without a split) and keeps a form that beats the
+ * library's own rule by more than 1 %.  Synchronises the stream.
  * best_variant (GMLP_VARIANT_SKINNY or _TENSOR) / best_us (microseconds per call) may be NULL.
  * gmlp_autotune_query returns 1 and the kept choice if the shape was tuned on the current device (gate_up_pair /
  * down_pair: 1 = CTA pairs, 0 = single CTAs, -1 = not applicable), else 0.  gmlp_autotune_clear forgets every

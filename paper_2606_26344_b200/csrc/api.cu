@@ -277,6 +277,7 @@ struct TunedShape {
     int64_t M, d_model, d_ff;
     int variant;
     int gu_pair, down_pair;                      // TENSOR: kernel of each GEMM (1 = CTA pairs, 0 = single CTAs)
+    int gu_nb, down_form;                        // single-CTA kernels: tile form (see t_force_gu_nb / t_force_down_form)
 };
 std::vector<TunedShape> g_tuned;                 // written by gmlp_autotune, under g_mutex
 std::atomic<int> g_tuned_count{0};               // lets untuned processes skip the lock
@@ -335,15 +336,35 @@ bool down_uses_pair(int64_t M, int64_t d_ff, int64_t d_model, int sms) {
 // shape and kept another one; t_force_* is how the tuner runs a combination of its choosing.
 struct TensorPlan {
     bool gu_pair, down_pair;
+    int gu_nb, down_form;
 };
 thread_local int t_force_gu = -1, t_force_down = -1;
+// Form of the single-CTA kernels, 0 = the library's own choice (pick_split_k / pick_umma_boxes / one-wave rule):
+//   gate/up: 2 = 64-column tiles, 4 = 128-column tiles;
+//   down:    2, 3, 4 = K split over a cluster of that many CTAs; 12 = 128-column tiles, 14 = 256-column tiles, no split.
+// Set by gmlp_autotune while it measures, and from its result around the launches of a tuned shape.
+thread_local int t_force_gu_nb = 0, t_force_down_form = 0;
+constexpr int kDownForms[6] = {0, 2, 3, 4, 12, 14};
+struct UmmaFormScope {
+    int prev_gu, prev_down;
+    UmmaFormScope(int gu_nb, int down_form) : prev_gu(t_force_gu_nb), prev_down(t_force_down_form) {
+        t_force_gu_nb = gu_nb;
+        t_force_down_form = down_form;
+    }
+    ~UmmaFormScope() {
+        t_force_gu_nb = prev_gu;
+        t_force_down_form = prev_down;
+    }
+};
 TensorPlan tensor_plan(int64_t M, int64_t d_model, int64_t d_ff, int sms) {
     if (sms <= 0) sms = 148;
-    TensorPlan p = {gate_up_uses_pair(M, d_ff, sms), down_uses_pair(M, d_ff, d_model, sms)};
+    TensorPlan p = {gate_up_uses_pair(M, d_ff, sms), down_uses_pair(M, d_ff, d_model, sms), t_force_gu_nb, t_force_down_form};
     TunedShape t;
     if (tuned_lookup(M, d_model, d_ff, &t) && t.variant == GMLP_VARIANT_TENSOR) {
         p.gu_pair = t.gu_pair != 0;
         p.down_pair = t.down_pair != 0;
+        if (t_force_gu_nb == 0) p.gu_nb = t.gu_nb;
+        if (t_force_down_form == 0) p.down_form = t.down_form;
     }
     if (t_force_gu >= 0) p.gu_pair = t_force_gu != 0;
     if (t_force_down >= 0) p.down_pair = t_force_down != 0;
@@ -650,13 +671,20 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     const int num_m = (int)((M + gmlp::kUmmaBM - 1) / gmlp::kUmmaBM);
     if (!GATEUP) {
         // few output tiles: a cluster of S CTAs per tile splits K and reduces through distributed shared memory
-        const int S = pick_split_k(num_m, K, N, sms);
+        int S = pick_split_k(num_m, K, N, sms);
+        const int form = t_force_down_form;
+        if (form >= 2 && form <= 4 && (K + gmlp::kUmmaBK - 1) / gmlp::kUmmaBK >= form) S = form;
+        else if (form == 12 || form == 14) S = 0;
         if (S >= 2) return launch_umma_splitk(dev, S, tmA, tmB0, C, M, K, N, num_m, a_box_rows, st);
     }
     // gate/up: 128 output columns per tile (two boxes of gate + two of up), or 64 when that still fits one wave
     int gu_nb = (int64_t)num_m * ((N + 63) / 64) <= sms ? 2 : 4;
     if (const char* e = getenv("GMLP_UMMA_GATEUP_NB")) gu_nb = atoi(e) == 2 ? 2 : 4;    // tuning override
-    const int nb = GATEUP ? gu_nb : pick_umma_boxes(num_m, N, sms);
+    if (t_force_gu_nb == 2 || t_force_gu_nb == 4) gu_nb = t_force_gu_nb;
+    int down_nb = pick_umma_boxes(num_m, N, sms);
+    if (t_force_down_form == 12) down_nb = 2;
+    if (t_force_down_form == 14) down_nb = 4;
+    const int nb = GATEUP ? gu_nb : down_nb;
     const int bn = GATEUP ? 32 * nb : 64 * nb;
     const int num_n = (int)((N + bn - 1) / bn);
     const int num_tiles = num_m * num_n;
@@ -859,6 +887,7 @@ int forward_impl(const gmlp_args* a) {
             break;
         case GMLP_VARIANT_TENSOR: {
             const TensorPlan plan = tensor_plan(a->M, a->d_model, a->d_ff, dev->sm_count);
+            UmmaFormScope forms(plan.gu_nb, plan.down_form);
             rc = plan.gu_pair ? launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act)
                               : launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act);
             if (rc == GMLP_OK) {
@@ -1466,20 +1495,84 @@ int autotune_impl(const gmlp_args* a, int iters, int32_t* best_variant, float* b
                         candidates[c].down, total_ms[c] * 1000.0f / (float)timed_calls, c == best ? "*" : "");
         fprintf(stderr, "\n");
     }
-    (void)cudaEventDestroy(e0);
-    (void)cudaEventDestroy(e1);
+    if (rc != GMLP_OK || best < 0) {
+        (void)cudaEventDestroy(e0);
+        (void)cudaEventDestroy(e1);
+    }
     if (rc != GMLP_OK) return rc;
     if (best < 0) return GMLP_ERR_WORKSPACE;                        // no candidate fitted the workspace
     const Cand w = candidates[best];
+    // Second stage, for the single-CTA kernels of a TENSOR winner: their tile form (gate/up: 64- or 128-column
+    // tiles; down: K split over a cluster of 2 to 4 CTAs, or 128- or 256-column tiles without a split) is otherwise
+    // picked by rule.  One GEMM at a time, the other left as chosen so far; the same interleaved rounds.
+    int best_gu_nb = 0, best_down_form = 0;
+    if (w.variant == GMLP_VARIANT_TENSOR && (w.gu == 0 || w.down == 0)) {
+        const int64_t mt = (a->M + 127) / 128, nkb = (a->d_ff + 63) / 64;
+        for (int which = 0; which < 2 && rc == GMLP_OK; ++which) {       // 0: gate/up forms, 1: down forms
+            if ((which == 0 ? w.gu : w.down) != 0) continue;
+            int forms[6], n_forms = 0;
+            if (which == 0) { forms[0] = 0; forms[1] = 2; forms[2] = 4; n_forms = 3; }
+            else
+                for (int f : kDownForms) {
+                    const bool split = f >= 2 && f <= 4;
+                    if (split && (nkb / f < 8 || mt * ((a->d_model + 127) / 128) * f > 2 * (int64_t)dev->sm_count)) continue;
+                    forms[n_forms++] = f;
+                }
+            float form_ms[6] = {0, 0, 0, 0, 0, 0};
+            for (int round = 0; round <= kRounds && rc == GMLP_OK; ++round)
+                for (int c = 0; c < n_forms && rc == GMLP_OK; ++c) {
+                    gmlp_args t = *a;
+                    t.variant = GMLP_VARIANT_TENSOR;
+                    t.flags &= ~(uint32_t)GMLP_FLAG_CHECKED;
+                    t_force_gu = w.gu;
+                    t_force_down = w.down;
+                    t_force_gu_nb = which == 0 ? forms[c] : best_gu_nb;
+                    t_force_down_form = which == 1 ? forms[c] : 0;
+                    rc = forward_impl(&t);
+                    float ms = 0.0f;
+                    if (rc == GMLP_OK && cudaEventRecord(e0, st) != cudaSuccess) rc = GMLP_ERR_LAUNCH;
+                    for (int i = 0; i < per_round && rc == GMLP_OK; ++i) rc = forward_impl(&t);
+                    t_force_gu = t_force_down = -1;
+                    t_force_gu_nb = t_force_down_form = 0;
+                    if (rc != GMLP_OK) break;
+                    if (cudaEventRecord(e1, st) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess ||
+                        cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) { rc = GMLP_ERR_LAUNCH; break; }
+                    if (round > 0) form_ms[c] += ms;
+                }
+            if (rc != GMLP_OK) break;
+            int bf = 0;
+            for (int c = 1; c < n_forms; ++c)
+                if (form_ms[c] < form_ms[bf]) bf = c;
+            // the rule's own choice (form 0) is kept unless another form is measurably (1 %) faster
+            if (form_ms[bf] < 0.99f * form_ms[0]) (which == 0 ? best_gu_nb : best_down_form) = forms[bf];
+            if (getenv("GMLP_TUNE_VERBOSE")) {
+                fprintf(stderr, "gmlp_autotune   %s forms:", which == 0 ? "gate/up" : "down");
+                for (int c = 0; c < n_forms; ++c)
+                    fprintf(stderr, " [%d: %.1f us]%s", forms[c], form_ms[c] * 1000.0f / (float)timed_calls,
+                            forms[c] == (which == 0 ? best_gu_nb : best_down_form) ? "*" : "");
+                fprintf(stderr, "\n");
+            }
+        }
+        if (rc == GMLP_OK) {
+            const int s2 = read_device_status();
+            if (s2 < 0) rc = s2;
+            else if (s2 != 0) rc = GMLP_ERR_TIMEOUT;
+        }
+        if (rc != GMLP_OK) { (void)0; }
+    }
+    (void)cudaEventDestroy(e0);
+    (void)cudaEventDestroy(e1);
+    if (rc != GMLP_OK) return rc;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
         bool found = false;
         for (TunedShape& t : g_tuned)
             if (t.device == device && t.M == a->M && t.d_model == a->d_model && t.d_ff == a->d_ff) {
                 t.variant = w.variant; t.gu_pair = w.gu; t.down_pair = w.down;
+                t.gu_nb = best_gu_nb; t.down_form = best_down_form;
                 found = true;
             }
-        if (!found) g_tuned.push_back({device, a->M, a->d_model, a->d_ff, w.variant, w.gu, w.down});
+        if (!found) g_tuned.push_back({device, a->M, a->d_model, a->d_ff, w.variant, w.gu, w.down, best_gu_nb, best_down_form});
         g_tuned_count.store((int)g_tuned.size(), std::memory_order_release);
     }
     if (best_variant) *best_variant = w.variant;
