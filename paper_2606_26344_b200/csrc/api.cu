@@ -1048,6 +1048,8 @@ int gate_up_impl(const gmlp_args* a) {
                (variant == GMLP_VARIANT_TENSOR && tensor_plan(a->M, a->d_model, a->d_ff, dev->sm_count).gu_pair)) {
         rc = launch_umma_pair<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st, act);
     } else {
+        // (a tuned shape's tile form applies to the gate/up half alone as well)
+        UmmaFormScope forms(variant == GMLP_VARIANT_TENSOR ? tensor_plan(a->M, a->d_model, a->d_ff, dev->sm_count).gu_nb : 0, 0);
         rc = launch_umma<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st, act);
     }
     if (rc != GMLP_OK) {
