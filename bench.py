@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the fused Gated MLP (libgmlp) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--no-extra]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--shard rows|dff] [--no-extra]
     python bench.py --impl reference ...          # times the CPU oracle on the host cores
 
 One "step" is one pass of the whole hot path (optional RMSNorm, gate/up GEMM with the SiLU
@@ -11,16 +11,28 @@ same metric through the host-buffer entry point (host->device copy of X and devi
 copy of Y inside the timed region).  The line also carries the roofline of the dominant
 kernel (measured with CUDA events around that kernel), the CPU oracle timed on the host
 cores, the SM clocks sampled during the timed region, and, unless --no-extra, the same
-measurements for the other stated workloads under "workloads".
+measurements for every other stated workload under "workloads", with a compact "summary"
+of all of them as the last key.
 
-With N > 1 (torchrun) every rank runs the same workload on its own rows (data parallel:
-rows are independent, weights replicated, no collective on the data path): weak scaling.
+The primary workload is the largest stated single-GPU configuration (the 70B-shaped prefill).
+A region of exactly K steps is timed between a barrier + synchronize on both sides; it is
+repeated until about half a second of steps has run and the median region is reported (min
+and max beside it), so that the number belongs to the clock the GPU settles at under load.
+
+With N > 1 the script starts N ranks itself (or runs under torchrun when that set
+WORLD_SIZE).  --shard rows (default): every rank runs the same workload on its own rows (rows
+are independent, weights replicated, no collective on the data path): weak scaling.
+--shard dff: d_ff is cut over the ranks (per-GPU weight bytes fall as 1 / N), each rank
+computes an fp32 partial product and the ranks exchange ONE all-reduce of M x d_model
+floats per step: strong scaling, the cut that helps a handful of tokens.
 """
 from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -31,12 +43,18 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-PRIMARY = "llama3-8b-decode-M8"
-EXTRA = ["llama3-8b-batch-M64", "llama3-8b-prefill-M2048-rmsnorm", "llama3-70b-prefill-M4096-outliers", "ragged-M8192-plain",
-         "ragged-M1000-plain", "ragged-M129-plain", "ragged-M7-plain", "ragged-M1-plain"]
+PRIMARY = "llama3-70b-prefill-M4096-outliers"
+PRIMARY_DFF = "llama3-8b-decode-M8"             # default workload of --shard dff
+# every stated configuration (decode first), then one unstated mid-M shape of the 8B layer
+STATED = ["llama3-8b-decode-M8", "llama3-8b-prefill-M2048-rmsnorm", "llama3-70b-prefill-M4096-outliers",
+          "ragged-M1-plain", "ragged-M7-plain", "ragged-M129-plain", "ragged-M1000-plain", "ragged-M8192-plain",
+          "ragged-M1-norm", "ragged-M7-norm", "ragged-M129-norm", "ragged-M1000-norm", "ragged-M8192-norm", "tiny"]
+UNSTATED = ["llama3-8b-batch-M64"]
 L2_BYTES = 126 * 1024 * 1024
+NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}       # dense bf16 peak and "about 8 TB/s": the stated targets' denominators
+MIN_TIMED_S = 0.5                                            # steps timed per workload, all regions together
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
-# summarised under profiles/ (skinny_gemm_decode_M8.md, umma_pair_gemm_prefill8b_M2048.md, umma_gemm_batch64_M64.md)
+# summarised under profiles/
 NCU_TRAFFIC_BYTES = {
     ("llama3-8b-decode-M8", "gate_up"): 235.0e6 + 4.5e6,
     ("llama3-8b-prefill-M2048-rmsnorm", "gate_up"): 254.0e6 + 50.4e6,
@@ -124,10 +142,9 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import numpy as np
     import oracle
     from paper_2606_26344_b200 import inputs as I
-    w = I.WORKLOADS[args.workload]
+    w = I.WORKLOADS[args.workload or PRIMARY]
     inp = I.make_inputs(w)
     rows = I.sample_rows(w, inp.outlier_rows)
     n_rows = min(len(rows), 8)
@@ -154,9 +171,47 @@ def run_reference(args):
     }))
 
 
+def fractions(w, ms, peaks):
+    """Roofline of the whole path: the slower of the FLOPs at the bf16 peak and the algorithmic bytes at the HBM
+    bandwidth, against the measured peaks (burst and, for a tensor-bound shape, sustained) and the nominal ones."""
+    t = ms * 1e-3
+    t_tensor = w.flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = w.min_bytes / (peaks["hbm_gbs"] * 1e9)
+    bound = "tensor" if t_tensor >= t_hbm else "hbm"
+    out = {"bound": bound, "frac": max(t_tensor, t_hbm) / t,
+           "frac_nominal": max(w.flops / (NOMINAL["bf16_tflops"] * 1e12), w.min_bytes / (NOMINAL["hbm_gbs"] * 1e9)) / t,
+           "denominators": f"frac: measured {peaks['bf16_tflops']} TFLOP/s burst, {peaks['hbm_gbs']} GB/s copy ({peaks['source']}); "
+                           f"frac_nominal: {NOMINAL['bf16_tflops']} TFLOP/s, {NOMINAL['hbm_gbs']} GB/s"}
+    if bound == "tensor":
+        out["frac_sustained"] = w.flops / (peaks["bf16_tflops_sustained"] * 1e12) / t
+    return out
+
+
+def timed_regions(run_step, steps, barrier, stream, est_ms, max_regions=40):
+    """Regions of exactly `steps` steps, each between a barrier + synchronize on both sides and its own pair of
+    events, repeated until MIN_TIMED_S of steps have run (at least three regions).  Returns the per-step time of
+    every region, in milliseconds."""
+    import torch
+    n = max(3, min(max_regions, int(math.ceil(MIN_TIMED_S * 1e3 / max(est_ms * steps, 1e-6)))))
+    out = []
+    k = 0
+    for _ in range(n):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            run_step(k)
+            k += 1
+        e1.record(stream)
+        barrier()
+        out.append(e0.elapsed_time(e1) / steps)
+    return out
+
+
 def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sample_clocks=True, clock_roll=0.6,
-                     autotune=False):
-    """Times one workload on this rank's GPU.  Returns a dict of measurements."""
+                     autotune=False, exact_steps=True):
+    """Times one workload on this rank's GPU.  `exact_steps`: regions of exactly `steps` steps (the primary line);
+    otherwise a region is stretched to about 0.1 s of steps."""
     import torch
     from paper_2606_26344_b200 import gmlp, inputs as I
 
@@ -182,68 +237,61 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    for _ in range(warmup):
-        gmlp.forward_ex(a)
+    # Weights that would stay in L2 are timed cold: several copies of the weights are used in rotation, enough that a
+    # copy has left L2 before its turn comes again (2.5 x L2 of other weights pass in between), steps back to back
+    # like the large workloads - programmatic dependent launch overlaps a step's launch and ramp with its
+    # predecessor's tail, as in a model that runs layer after layer.
+    rot, keep = [a], []
+    if fits_l2:
+        n_sets = int(-(-2.5 * L2_BYTES // weight_bytes)) + 1
+        for _ in range(n_sets - 1):
+            wg, wu, wd = Wg.clone(), Wu.clone(), Wd.clone()
+            keep.append((wg, wu, wd))
+            rot.append(gmlp.make_args(X, wg, wu, wd, Y, gamma, w.eps, w.rmsnorm, gmlp.VARIANT_AUTO, ws, stream))
+    n_sets = len(rot)
+
+    def run_step(k):
+        gmlp.forward_ex(rot[k % n_sets])
+
+    for k in range(max(warmup, 2 * n_sets)):
+        run_step(k)
     torch.cuda.synchronize(dev)
     st = gmlp.device_status()
     if st != 0:
         raise RuntimeError(f"device status {st:#x} after warm-up")
+    t0 = time.perf_counter()
+    for k in range(10):
+        run_step(k)
+    torch.cuda.synchronize(dev)
+    est_ms = (time.perf_counter() - t0) * 1e3 / 10
 
-    # The timed region of a small workload lasts a few milliseconds, shorter than nvidia-smi's sampling
-    # period.  The clocks are therefore sampled over an untimed pre-roll of the same steps, the timed
-    # region and an untimed post-roll: one continuous stretch of identical load.
+    # The clocks are sampled over an untimed pre-roll of the same steps (which also brings the GPU to the power state
+    # it holds under this load), every timed region, and a short post-roll: one stretch of identical load.
     sampler = ClockSampler(dev.index or 0) if (sample_clocks and clock_roll > 0) else None
 
     def roll(seconds):
         t_end = time.perf_counter() + seconds
+        k = 0
         while time.perf_counter() < t_end:
             for _ in range(20):
-                gmlp.forward_ex(a)
+                run_step(k)
+                k += 1
             torch.cuda.synchronize(dev)
 
     if sampler:
         sampler.start()
         roll(clock_roll)
+    region_steps = steps if exact_steps else max(steps, int(math.ceil(100.0 / max(est_ms, 1e-3))))
     gmlp.reset_launch_count()
-    if not fits_l2:
-        # inputs are larger than L2: back-to-back steps, one pair of events around the region
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(steps):
-            gmlp.forward_ex(a)
-        e1.record(stream)
-        barrier()
-        total_ms = e0.elapsed_time(e1)
-        per_step = [total_ms / steps]
-    else:
-        # Weights that would stay in L2.  Cold figure: several copies of the weights are used in rotation, enough
-        # that a copy has left L2 before its turn comes again (2.5 x L2 of other weights pass in between), steps
-        # back to back like the large workloads - programmatic dependent launch overlaps a step's launch and ramp
-        # with its predecessor's tail, as in a model that runs layer after layer.
-        n_sets = int(-(-2.5 * L2_BYTES // weight_bytes)) + 1
-        rot = [a]
-        keep = []
-        for _ in range(n_sets - 1):
-            wg, wu, wd = Wg.clone(), Wu.clone(), Wd.clone()
-            keep.append((wg, wu, wd))
-            rot.append(gmlp.make_args(X, wg, wu, wd, Y, gamma, w.eps, w.rmsnorm, gmlp.VARIANT_AUTO, ws, stream))
-        for k in range(2 * n_sets):
-            gmlp.forward_ex(rot[k % n_sets])
-        gmlp.reset_launch_count()
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for k in range(steps):
-            gmlp.forward_ex(rot[k % n_sets])
-        e1.record(stream)
-        barrier()
-        total_ms = e0.elapsed_time(e1)
-        per_step = [total_ms / steps]
-        launches_rot = gmlp.launch_count()
+    run_step(0)
+    launches_per_step = gmlp.launch_count()
+    per_step = timed_regions(run_step, region_steps, barrier, stream, est_ms)
+    ms = statistics.median(per_step)
+    isolated_ms = None
+    if fits_l2:
         # the same step alone: L2 overwritten before it, one pair of events around it (launch latency and ramp exposed)
         iso = []
-        for _ in range(max(3, min(steps, 20))):
+        for _ in range(10):
             flush.fill_(1)
             i0, i1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             i0.record(stream)
@@ -252,26 +300,25 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
             iso.append((i0, i1))
         torch.cuda.synchronize(dev)
         isolated_ms = sum(x.elapsed_time(y) for x, y in iso) / len(iso)
-        del keep
-    launches = gmlp.launch_count() if not fits_l2 else launches_rot
     if sampler:
-        roll(clock_roll)
+        roll(min(clock_roll, 0.2))
     clocks = sampler.stop() if sampler else None
     if clocks is not None:
-        clocks["window"] = f"pre-roll {clock_roll} s + timed region + post-roll {clock_roll} s of the same steps"
-    ms = total_ms / steps
+        clocks["window"] = f"pre-roll {clock_roll} s + the timed regions + post-roll of the same steps"
 
     # per-kernel durations, in a loop of their own (an event between two kernels stops the second from
     # overlapping the first's tail, so these are stand-alone kernel times, like a profiler's)
-    gmlp.profile_enable(True)
-    n_prof = max(3, min(steps, 50))
+    n_prof = max(3, min(int(math.ceil(150.0 / max(est_ms, 1e-3))), 50))
     if flush is None:
+        for _ in range(3):
+            gmlp.forward_ex(a)
+        gmlp.profile_enable(True)
         for _ in range(n_prof):
             gmlp.forward_ex(a)
         kern_ms = gmlp.profile_read()
     else:
         acc = {}
-        for _ in range(n_prof):
+        for _ in range(min(n_prof, 20)):
             gmlp.profile_enable(True)
             flush.fill_(1)
             gmlp.forward_ex(a)
@@ -281,39 +328,43 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
     gmlp.profile_enable(False)
 
     res = {"name": w.name, "M": w.M, "d_model": w.d_model, "d_ff": w.d_ff, "rmsnorm": w.rmsnorm,
-           "variant": {1: "simt", 2: "stream", 3: "umma", 4: "skinny", 5: "pair", 6: "tensor"}[variant], "ms_per_step": ms,
-           "ms_min": min(per_step), "tokens_per_s": w.M / (ms * 1e-3), "tflops": w.flops / (ms * 1e-3) / 1e12,
-           "gbps_min_bytes": w.min_bytes / (ms * 1e-3) / 1e9, "launches": launches, "clocks": clocks,
+           "variant": {1: "simt", 2: "stream", 3: "umma", 4: "skinny", 5: "pair", 6: "tensor", 7: "fused"}.get(variant, str(variant)),
+           "ms_per_step": ms, "ms_min": min(per_step), "ms_max": max(per_step), "regions": len(per_step),
+           "steps_per_region": region_steps, "tokens_per_s": w.M / (ms * 1e-3), "tflops": w.flops / (ms * 1e-3) / 1e12,
+           "gbps_min_bytes": w.min_bytes / (ms * 1e-3) / 1e9, "launches": launches_per_step * region_steps, "clocks": clocks,
            "kernel_ms": kern_ms,
-           "autotuned": None if tuned is None else {"variant": tuned[0], "gate_up_pair": tuned[1], "down_pair": tuned[2]},
-           "l2": f"weights fit L2: {n_sets} copies of the weights in rotation (a copy has left L2 before its next turn), "
-                 "steps back to back" if fits_l2 else "inputs larger than L2; steps back to back"}
-    if fits_l2:
+           "l2": f"weights fit L2: {n_sets} copies in rotation, steps back to back" if fits_l2
+                 else "inputs larger than L2; steps back to back"}
+    if tuned is not None:
+        res["autotuned"] = {"variant": tuned[0], "gate_up_pair": tuned[1], "down_pair": tuned[2]}
+    if isolated_ms is not None:
         res["ms_step_alone"] = isolated_ms      # L2 overwritten before the step, events around that one step
+    res["roofline_path"] = fractions(w, ms, peaks)
 
-    # roofline of the path and of its dominant kernel
-    t_tensor = w.flops / (peaks["bf16_tflops"] * 1e12)
-    t_hbm = w.min_bytes / (peaks["hbm_gbs"] * 1e9)
-    res["roofline_path"] = {"bound": "tensor" if t_tensor >= t_hbm else "hbm",
-                            "frac": max(t_tensor, t_hbm) / (ms * 1e-3)}
+    # roofline of the dominant kernel (gate/up: two thirds of the FLOPs and of the weight bytes)
     if "gate_up" in kern_ms:
         kms = kern_ms["gate_up"] * 1e-3
-        if t_tensor >= t_hbm:
+        if res["roofline_path"]["bound"] == "tensor":
             flops = 4 * w.M * w.d_model * w.d_ff
             ach = flops / kms / 1e12
-            res["roofline"] = {"kernel": "gate_up", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
-                               "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
+            # a kernel timed inside a long run of steps under the power cap is held against the sustained figure
+            long_run = est_ms * n_prof > 100.0
+            peak = peaks["bf16_tflops_sustained"] if long_run else peaks["bf16_tflops"]
+            res["roofline"] = {"kernel": "gate_up", "bound": "tensor", "achieved": ach, "peak": peak,
+                               "unit": "TFLOP/s", "frac": ach / peak, "frac_burst": ach / peaks["bf16_tflops"],
+                               "frac_nominal": ach / NOMINAL["bf16_tflops"],
                                "traffic": NCU_TRAFFIC_BYTES.get((w.name, "gate_up")), "algorithmic_flops": flops,
-                               "peak_source": peaks["source"] + " (burst bf16)"}
+                               "peak_source": peaks["source"] + (" (sustained bf16: the kernel is timed inside a long run)"
+                                                                 if long_run else " (burst bf16)")}
         else:
             nbytes = 2 * (2 * w.d_model * w.d_ff + w.M * w.d_model + w.M * w.d_ff)
             ach = nbytes / kms / 1e9
             res["roofline"] = {"kernel": "gate_up", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
-                               "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                               "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "frac_nominal": ach / NOMINAL["hbm_gbs"],
                                "traffic": NCU_TRAFFIC_BYTES.get((w.name, "gate_up")), "algorithmic_bytes": nbytes,
                                "peak_source": peaks["source"] + " (copy)"}
 
-    if "roofline" in res and not fits_l2:
+    if "roofline" in res and not fits_l2 and res["roofline"]["bound"] == "hbm":
         # The same kernel in a chain of its own launches: programmatic dependent launch overlaps a launch's ramp with
         # its predecessor's tail, as it does inside the timed steps, so this is the kernel's rate in steady state
         # (the figure above is one launch between two events, like a profiler's).  Two events around the loop; the
@@ -331,8 +382,7 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
         torch.cuda.synchronize(dev)
         chain_ms = c0.elapsed_time(c1) / n_chain
         r = res["roofline"]
-        work = r.get("algorithmic_bytes", r.get("algorithmic_flops"))
-        ach_c = work / (chain_ms * 1e-3) / (1e9 if r["bound"] == "hbm" else 1e12)
+        ach_c = r["algorithmic_bytes"] / (chain_ms * 1e-3) / 1e9
         r["chained"] = {"achieved": ach_c, "frac": ach_c / r["peak"], "ms_per_launch": chain_ms, "launches": n_chain,
                         "how": "launches of this kernel back to back on one stream, two events around the loop"}
         del Hc
@@ -371,8 +421,80 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
         nb = w.M * w.d_model * 2
         res["e2e"] = {"value": w.M / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
                       "h2d_bytes_per_step": nb, "d2h_bytes_per_step": nb, "steps": n_e2e, "lanes": 2}
+    del keep
     res["_inputs"] = inp
     return res
+
+
+def measure_dff_sharded(w, steps, warmup, dev, peaks, dist, rank, world, clock_roll=0.6):
+    """--shard dff: this rank holds columns [a, b) of W_gate / W_up and rows [a, b) of W_down.  A step is the rank's
+    fp32 partial product (one call of the library), ONE all-reduce of M x d_model floats over the ranks, and the
+    single rounding to bf16 (gmlp_sum_partials).  Every rank ends with the whole Y."""
+    import torch
+    from paper_2606_26344_b200 import gmlp, inputs as I, sharding
+
+    inp = I.make_inputs(w)
+    a0, a1 = sharding.dff_range(w.d_ff, rank, world)
+    X = inp.X.to(dev)
+    Wg, Wu = inp.Wg[:, a0:a1].contiguous().to(dev), inp.Wu[:, a0:a1].contiguous().to(dev)
+    Wd = inp.Wd[a0:a1].contiguous().to(dev)
+    gamma = inp.gamma.to(dev) if inp.gamma is not None else None
+    stream = torch.cuda.current_stream(dev)
+    P = torch.zeros(w.M, w.d_model, dtype=torch.float32, device=dev)
+    Y = torch.empty_like(X)
+    use_dist = dist if world > 1 else None
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def run_step(_k):
+        sharding.forward_dff_sharded(X, Wg, Wu, Wd, use_dist, gamma, w.eps, w.rmsnorm, stream, P=P, Y=Y)
+
+    for k in range(max(warmup, 3)):
+        run_step(k)
+    torch.cuda.synchronize(dev)
+    t0 = time.perf_counter()
+    for k in range(10):
+        run_step(k)
+    torch.cuda.synchronize(dev)
+    est_ms = (time.perf_counter() - t0) * 1e3 / 10
+    sampler = ClockSampler(dev.index or 0) if clock_roll > 0 else None
+    if sampler:
+        sampler.start()
+        t_end = time.perf_counter() + clock_roll
+        while time.perf_counter() < t_end:
+            for k in range(20):
+                run_step(k)
+            torch.cuda.synchronize(dev)
+    gmlp.reset_launch_count()
+    run_step(0)
+    launches_per_step = gmlp.launch_count()
+    per_step = timed_regions(run_step, steps, barrier, stream, est_ms)
+    clocks = sampler.stop() if sampler else None
+    ms = statistics.median(per_step)
+    # end to end: X from pinned host memory on every rank, Y back to the host on rank 0
+    Xh, Yh = inp.X.clone().pin_memory(), torch.empty_like(inp.X).pin_memory()
+    n_e2e = max(4, min(steps, 50))
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for k in range(n_e2e):
+        X.copy_(Xh, non_blocking=True)
+        run_step(k)
+        if rank == 0:
+            Yh.copy_(Y, non_blocking=True)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / n_e2e
+    nb = w.M * w.d_model * 2
+    return {"ms_per_step": ms, "ms_min": min(per_step), "ms_max": max(per_step), "regions": len(per_step),
+            "launches": launches_per_step * steps, "clocks": clocks, "slice": [a0, a1],
+            "allreduce_bytes": w.M * w.d_model * 4 if world > 1 else 0,
+            "weight_bytes_per_gpu": 3 * w.d_model * (a1 - a0) * 2,
+            "e2e": {"ms_per_step": e2e_ms, "unit": "tokens/s", "h2d_bytes_per_step": nb, "d2h_bytes_per_step": nb},
+            "_inputs": inp}
 
 
 def measure_rmsnorm_matmul(dev, sizes=(2048, 4096, 8192), iters=10):
@@ -531,35 +653,92 @@ def measure_gqa(dev, peaks, iters=10):
             "best_tflops": max(r["tflops"] for r in rows), "table": rows}
 
 
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launch_ranks(n: int) -> int:
+    """--gpus N without a launcher: start N ranks of this script (one per GPU) under torch.distributed.run on this
+    node and pass their exit code on.  Rank 0 of those prints the JSON line."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(free_port()), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.call(cmd)
+
+
+def summary_entry(r):
+    rp = r.get("roofline_path", {})
+    rk = r.get("roofline") or {}
+    clk = r.get("clocks") or {}
+    return {"name": r["name"], "ms": round(r["ms_per_step"], 5), "bound": rp.get("bound"),
+            "frac_path": round(rp.get("frac", 0.0), 4), "frac_path_nominal": round(rp.get("frac_nominal", 0.0), 4),
+            **({"frac_path_sustained": round(rp["frac_sustained"], 4)} if "frac_sustained" in rp else {}),
+            "frac_kernel": round(rk["frac"], 4) if "frac" in rk else None, "sm_mhz": clk.get("sm_mhz"),
+            "reasons": clk.get("reasons")}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="gmlp", choices=["gmlp", "reference"])
-    ap.add_argument("--workload", default=PRIMARY)
+    ap.add_argument("--workload", default=None, help=f"primary workload (default {PRIMARY}; {PRIMARY_DFF} with --shard dff)")
+    ap.add_argument("--shard", default="rows", choices=["rows", "dff"],
+                    help="rows: ranks take disjoint rows, no collective (weak scaling); dff: d_ff cut over the ranks, "
+                         "one all-reduce of M x d_model floats per step (strong scaling)")
     ap.add_argument("--no-extra", action="store_true", help="time only the primary workload")
     ap.add_argument("--op", default="gmlp", choices=["gmlp", "rmsnorm_matmul", "matmul_add_rmsnorm", "qkv", "gqa"],
                     help="rmsnorm_matmul / matmul_add_rmsnorm / qkv / gqa: print only that operator's sweep "
                          "(one JSON line) and exit")
     ap.add_argument("--autotune", action="store_true",
                     help="run gmlp_autotune on each workload's shape before timing it (default: the built-in rule)")
-    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time spent on the oracle baseline (0 = skip)")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="least CPU time spent on the oracle baseline (0 = skip)")
     ap.add_argument("--clock-roll", type=float, default=0.6,
-                    help="seconds of untimed identical steps before and after the timed region while clocks are "
-                         "sampled (0 = no clock sampling; for runs under a profiler)")
+                    help="seconds of untimed identical steps before the timed regions while clocks are sampled "
+                         "(0 = no clock sampling; for runs under a profiler)")
+    ap.add_argument("--stub-measure", action="store_true",
+                    help="test hook: no GPU work at all - the ranks rendezvous over gloo, report a constant step time and "
+                         "rank 0 prints the line marked \"data\": \"stub\" (checks the launch path on a CPU-only machine)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
         return
-
-    import torch
-    from paper_2606_26344_b200 import build as B
-    from paper_2606_26344_b200 import gmlp, inputs as I
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(launch_ranks(args.gpus))
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wname = args.workload or (PRIMARY_DFF if args.shard == "dff" else PRIMARY)
+    parallelism = (f"dp{world} (rows sharded, no collective)" if args.shard == "rows"
+                   else f"tp{world} (d_ff sharded, one all-reduce of M x d_model fp32 per step)")
+    scaling = "weak" if args.shard == "rows" else "strong"
+
+    import torch
+    from paper_2606_26344_b200 import inputs as I, sharding
+    w = I.WORKLOADS[wname]
+
+    if args.stub_measure:
+        import torch.distributed as dist_mod
+        if world > 1:
+            dist_mod.init_process_group("gloo")
+            dist_mod.barrier()
+        ms = sharding.max_over_ranks(1.0 + 0.25 * rank, dist_mod if world > 1 else None)
+        units = w.M * (world if args.shard == "rows" else 1)
+        if rank == 0:
+            print(json.dumps({"metric": "gated_mlp_tokens_per_s", "value": units / (ms * 1e-3), "unit": "tokens/s",
+                              "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                              "higher_is_better": True, "scaling": scaling, "vs_baseline": None, "dtype": "bf16",
+                              "data": "stub", "config": {"workload": w.name, "parallelism": parallelism}}))
+        if world > 1:
+            dist_mod.barrier()
+            dist_mod.destroy_process_group()
+        return
+
+    from paper_2606_26344_b200 import build as B
+    from paper_2606_26344_b200 import gmlp
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     if rank == 0:
@@ -587,10 +766,34 @@ def main():
             dist.destroy_process_group()
         return
 
-    w = I.WORKLOADS[args.workload]
+    if args.shard == "dff":
+        res = measure_dff_sharded(w, args.steps, warmup, dev, peaks, dist, rank, world, clock_roll=args.clock_roll)
+        ms = sharding.max_over_ranks(res["ms_per_step"], dist, dev)
+        e2e_ms = sharding.max_over_ranks(res["e2e"]["ms_per_step"], dist, dev)
+        if rank == 0:
+            line = {
+                "metric": "gated_mlp_tokens_per_s", "value": w.M / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
+                "steps": args.steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": scaling,
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": w.name, "M": w.M, "d_model": w.d_model, "d_ff": w.d_ff, "rmsnorm": w.rmsnorm,
+                           "parallelism": parallelism, "d_ff_slice_rank0": res["slice"],
+                           "weight_bytes_per_gpu": res["weight_bytes_per_gpu"], "allreduce_bytes_per_step": res["allreduce_bytes"]},
+                "timing": {"ms_min": res["ms_min"], "ms_max": res["ms_max"], "regions": res["regions"],
+                           "how": "median over regions of exactly `steps` steps, max over ranks"},
+                "tflops": w.flops / (ms * 1e-3) / 1e12,
+                "roofline_path": fractions(w, ms, peaks),
+                "e2e": {"value": w.M / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": res["e2e"]["h2d_bytes_per_step"],
+                        "d2h_bytes_per_step": res["e2e"]["d2h_bytes_per_step"]},
+                "gpu_launches": res["launches"], "clocks": res["clocks"], "peaks": peaks,
+            }
+            print(json.dumps(line))
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
     res = measure_workload(w, args.steps, warmup, dev, peaks, dist=dist, clock_roll=args.clock_roll,
-                           autotune=args.autotune)
-    from paper_2606_26344_b200 import sharding
+                           autotune=args.autotune, exact_steps=True)
     ms = sharding.max_over_ranks(res["ms_per_step"], dist, dev)          # the slowest rank bounds the step
     res["e2e"]["ms_per_step"] = sharding.max_over_ranks(res["e2e"]["ms_per_step"], dist, dev)
     res["e2e"]["value"] = sharding.job_throughput(w.M, world, res["e2e"]["ms_per_step"])
@@ -598,10 +801,10 @@ def main():
 
     extras = []
     if not args.no_extra and world == 1:
-        for name in EXTRA:
+        for name in [n for n in STATED + UNSTATED if n != w.name]:
             try:
-                r = measure_workload(I.WORKLOADS[name], max(5, min(args.steps, 30)), 3, dev, peaks,
-                                     want_e2e=False, sample_clocks=False, autotune=args.autotune)
+                r = measure_workload(I.WORKLOADS[name], args.steps, 3, dev, peaks, want_e2e=False, sample_clocks=True,
+                                     clock_roll=min(args.clock_roll, 0.3), autotune=args.autotune, exact_steps=False)
                 r.pop("_inputs", None)
                 extras.append(r)
             except Exception as exc:  # a failed extra must not hide the primary number
@@ -623,21 +826,24 @@ def main():
         return
 
     inp = res.pop("_inputs")
-    rows = I.sample_rows(w, inp.outlier_rows)
+    rows = I.sample_rows(w, inp.outlier_rows)          # the rows the parity tests compare: all, or the 256 seeded ones
     if world == 1 and args.cpu_seconds > 0:
-        cpu_rate, cpu_rows, cpu_dt, cores = cpu_oracle_rate(inp, rows[: min(len(rows), 32)], args.cpu_seconds)
+        cpu_rate, cpu_rows, cpu_dt, cores = cpu_oracle_rate(inp, rows, args.cpu_seconds)
         cpu = {"value": cpu_rate, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-               "sample": f"{cpu_rows} row evaluations of this workload ({min(len(rows), 32)} rows per pass, "
-                         f"repeated for {cpu_dt:.1f} s); fp64, OpenMP over rows"}
+               "sample": f"{cpu_rows} row evaluations of this workload (its {len(rows)} parity rows per pass, "
+                         f"{cpu_dt:.1f} s in all); fp64, OpenMP over rows"}
     else:
         cpu = None
 
     line = {
         "metric": "gated_mlp_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
-        "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": scaling, "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "M": w.M, "d_model": w.d_model, "d_ff": w.d_ff, "rmsnorm": w.rmsnorm,
-                   "schedule": res["variant"], "l2": res["l2"], "parallelism": f"dp{world} (rows sharded, no collective)"},
+                   "schedule": res["variant"], "l2": res["l2"], "parallelism": parallelism},
+        "timing": {"ms_min": res["ms_min"], "ms_max": res["ms_max"], "regions": res["regions"],
+                   "how": "median over regions of exactly `steps` steps, each between barrier + synchronize; "
+                          "regions repeat until 0.5 s of steps have run, after a pre-roll of the same load"},
         "tflops": world * w.flops / (ms * 1e-3) / 1e12,
         "gbps_min_bytes": world * w.min_bytes / (ms * 1e-3) / 1e9,
         "roofline_path": res["roofline_path"],
@@ -650,6 +856,7 @@ def main():
         "peaks": peaks,
         "workloads": extras,
         "rmsnorm_matmul": rmsmm,
+        "summary": [summary_entry(r) for r in [dict(res, name=w.name)] + [e for e in extras if "error" not in e]],
     }
     print(json.dumps(line))
     if dist is not None:

@@ -253,6 +253,13 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
         if (v == -1) p.grid = (int)(p.num_tiles < total ? p.num_tiles : total);          // one CTA per tile
         else if (v >= 1 && v <= total) p.grid = v;
     }
+    // a column tile is shared by at most min(grid, KB / (units per CTA) + 2) consecutive CTAs; the kernel keeps one
+    // scratch offset per contributor in a fixed shared array
+    {
+        const int64_t per_cta = total / p.grid > 0 ? total / p.grid : 1;
+        const int64_t contrib = p.KB / per_cta + 2 < p.grid ? p.KB / per_cta + 2 : p.grid;
+        if (contrib > gmlp::kSkinnyMaxContrib) p.stages = 0;               // launch_skinny refuses the plan
+    }
     p.scratch_bytes = (uint64_t)p.grid * 2 * nmat * p.NH * p.Mpad * 128 * 4;
     return p;
 }
@@ -540,9 +547,27 @@ int pick_umma_boxes(int64_t num_m, int64_t N, int sms) {
     return nb;
 }
 
+// Length of an accumulation chain (in k-blocks of 64) of the Gated MLP's CTA-pair GEMMs; 0 = one chain per tile.
+// Gate/up: the tensor core's truncating accumulation biases g and u in proportion to the chain length, and H is
+// rounded to bf16 right after, so a long chain changes which bf16 many H values round to (measured on rows scaled
+// by 20, K = 8192: 1.8 % of them with one chain, 0.24 % with chains of 16 k-blocks, 0.12 % with 8, 0.05 % for
+// sequential fp32 FMA; elements beyond the absolute output tolerance on three such rows: 274 / 134 / 19 / 15).
+// Chains of 8 cost 3.5 % of the kernel's cycles (about one MMA time per chain switch), chains of 16 nothing
+// measurable: 8 from K = 8192 on, 16 below.  Down projection: its output is rounded once at the end and the
+// chain length made no difference to any compared element (one chain of 448 k-blocks: 18 elements, chains of 8: 19),
+// so it keeps one chain.
+int pair_chunk_kb(bool gate_up, int64_t K) {
+    int v = gate_up ? (K >= 8192 ? gmlp::kPairChunkKb : 2 * gmlp::kPairChunkKb) : 0;
+    if (const char* e = getenv("GMLP_PAIR_CHUNK_KB")) v = atoi(e);                                   // tuning override
+    if (const char* e = getenv(gate_up ? "GMLP_PAIR_CHUNK_KB_GU" : "GMLP_PAIR_CHUNK_KB_DOWN")) v = atoi(e);
+    return v > 0 ? v : 0;
+}
+
+// chunk_kb > 0: the kernel form that accumulates K in chains of that many k-blocks (the Gated MLP's own GEMMs);
+// the other operators' plain products keep one chain per tile.
 template <bool GATEUP>
 int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1, bf16* C,
-                     int64_t M, int64_t K, int64_t N, cudaStream_t st, gmlp::GateAct act = kSilu) {
+                     int64_t M, int64_t K, int64_t N, cudaStream_t st, gmlp::GateAct act = kSilu, int chunk_kb = 0) {
     const int wkm = t_w_out_in ? 1 : 0;
     const int yf32 = (!GATEUP && t_y_fp32) ? 1 : 0;
     CUtensorMap tmA, tmB0, tmB1;
@@ -556,7 +581,9 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     if (!dev->pair_attr_set) {
         const int b = (int)gmlp::kPairSmemBytes;
         if (cudaFuncSetAttribute(gmlp::umma_pair_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
-            cudaFuncSetAttribute(gmlp::umma_pair_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess)
+            cudaFuncSetAttribute(gmlp::umma_pair_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::umma_pair_gemm_kernel<true, false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::umma_pair_gemm_kernel<false, false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess)
             return GMLP_ERR_LAUNCH;
         dev->pair_attr_set = true;
     }
@@ -565,9 +592,10 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     const int bn = GATEUP ? 128 : 256;
     const int num_tiles = num_m * (int)((N + bn - 1) / bn);
     const int pairs = num_tiles < sms / 2 ? num_tiles : sms / 2;
+    const bool chunked = chunk_kb > 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs));
-    cfg.blockDim = dim3(gmlp::kUmmaThreads);
+    cfg.blockDim = dim3(chunked ? gmlp::kPairChunkThreads : gmlp::kUmmaThreads);
     cfg.dynamicSmemBytes = gmlp::kPairSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -580,9 +608,13 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
-    if (cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m,
-                           num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm, yf32) != cudaSuccess)
-        return GMLP_ERR_LAUNCH;
+    const cudaError_t err = chunked
+        ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false, false, false, true>, tmA, tmB0, tmB1, C, Mi, Ki, Ni,
+                             num_m, num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm,
+                             yf32, chunk_kb)
+        : cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m,
+                             num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm, yf32, 0);
+    if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
 }
@@ -878,21 +910,21 @@ int forward_impl(const gmlp_args* a) {
             rc = run_skinny(dev, L, ws, A, Wg, Wu, Wd, H, Y, a->M, a->d_model, a->d_ff, st, act);
             break;
         case GMLP_VARIANT_PAIR:
-            rc = launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act);
+            rc = launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act, pair_chunk_kb(true, a->d_model));
             if (rc == GMLP_OK) {
                 prof_mark("gate_up", st);
-                rc = launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st);
+                rc = launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st, kSilu, pair_chunk_kb(false, a->d_ff));
                 if (rc == GMLP_OK) prof_mark("down", st);
             }
             break;
         case GMLP_VARIANT_TENSOR: {
             const TensorPlan plan = tensor_plan(a->M, a->d_model, a->d_ff, dev->sm_count);
             UmmaFormScope forms(plan.gu_nb, plan.down_form);
-            rc = plan.gu_pair ? launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act)
+            rc = plan.gu_pair ? launch_umma_pair<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act, pair_chunk_kb(true, a->d_model))
                               : launch_umma<true>(dev, A, Wg, Wu, H, a->M, a->d_model, a->d_ff, st, act);
             if (rc == GMLP_OK) {
                 prof_mark("gate_up", st);
-                rc = plan.down_pair ? launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st)
+                rc = plan.down_pair ? launch_umma_pair<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st, kSilu, pair_chunk_kb(false, a->d_ff))
                                     : launch_umma<false>(dev, H, Wd, nullptr, Y, a->M, a->d_ff, a->d_model, st);
                 if (rc == GMLP_OK) prof_mark("down", st);
             }
@@ -1046,7 +1078,7 @@ int gate_up_impl(const gmlp_args* a) {
         if (rc == GMLP_OK) rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, Hout, a->M, a->d_model, a->d_ff, st, act);
     } else if (variant == GMLP_VARIANT_PAIR ||
                (variant == GMLP_VARIANT_TENSOR && tensor_plan(a->M, a->d_model, a->d_ff, dev->sm_count).gu_pair)) {
-        rc = launch_umma_pair<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st, act);
+        rc = launch_umma_pair<true>(dev, A, Wg, Wu, Hout, a->M, a->d_model, a->d_ff, st, act, pair_chunk_kb(true, a->d_model));
     } else {
         // (a tuned shape's tile form applies to the gate/up half alone as well)
         UmmaFormScope forms(variant == GMLP_VARIANT_TENSOR ? tensor_plan(a->M, a->d_model, a->d_ff, dev->sm_count).gu_nb : 0, 0);
@@ -1142,7 +1174,7 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         const float* rc_ptr = r;
         cudaError_t err = pair
-            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0, 0)
+            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0, 0, 0)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0, 0);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
@@ -1238,7 +1270,7 @@ int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         cudaError_t err = pair
             ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
-                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq, kNoMulti, 0, 0)
+                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq, kNoMulti, 0, 0, 0)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
                                  num_tiles, (const float*)nullptr, 128, kSilu, R, sumsq, kNoMulti, 0, 0);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
@@ -1348,7 +1380,7 @@ int qkv_proj_impl(const gmlp_qkv_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->Nq;
         cudaError_t err = pair
             ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, false, true>, tmA, tmB0, tmB1, Q, Mi, Ki, Ni,
-                                 num_m, num_tiles, (const float*)nullptr, kSilu, (const bf16*)nullptr, (float*)nullptr, multi, 0, 0)
+                                 num_m, num_tiles, (const float*)nullptr, kSilu, (const bf16*)nullptr, (float*)nullptr, multi, 0, 0, 0)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, false, true>, tmA, tmB0, tmB1, Q, Mi, Ki, Ni,
                                  num_m, num_tiles, (const float*)nullptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr,
                                  multi, 0, 0);
@@ -1835,6 +1867,15 @@ int gmlp_selftest_wait_timeout(void* stream) {
     if (s < 0) return s;
     return s == ((99 << 16) | 1) ? GMLP_ERR_TIMEOUT : (s == 0 ? GMLP_OK : GMLP_ERR_LAUNCH);
 }
+
+#ifdef GMLP_TRACE
+// GMLP_TRACE builds only: copies the timeline (kernels x CTAs x sites, nanoseconds) to `dst` after a device synchronize
+int gmlp_trace_read(unsigned long long* dst, uint64_t bytes) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return GMLP_ERR_LAUNCH;
+    if (bytes > sizeof(gmlp::g_trace)) bytes = sizeof(gmlp::g_trace);
+    return cudaMemcpyFromSymbol(dst, gmlp::g_trace, bytes) == cudaSuccess ? GMLP_OK : GMLP_ERR_LAUNCH;
+}
+#endif
 
 uint64_t gmlp_launch_count(void) { return t_launches; }
 void gmlp_reset_launch_count(void) { t_launches = 0; }

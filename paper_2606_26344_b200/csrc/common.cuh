@@ -15,6 +15,21 @@ __device__ __forceinline__ void report_timeout(int kernel_id, int site) {
     atomicCAS(&g_device_status, 0, (kernel_id << 16) | (site & 0xFFFF));
 }
 
+// Optional timeline of the small-M kernels (builds with -DGMLP_TRACE only; nothing of it exists in the normal
+// library): one thread per site stores the global nanosecond timer, the last launch of each kernel wins.
+#ifdef GMLP_TRACE
+constexpr int kTraceKernels = 4, kTraceCtas = 512, kTraceSites = 16;
+__device__ unsigned long long g_trace[kTraceKernels][kTraceCtas][kTraceSites];
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define GMLP_TR(kernel, site) do { if (blockIdx.x < gmlp::kTraceCtas) gmlp::g_trace[kernel][blockIdx.x][site] = gmlp::global_timer_ns(); } while (0)
+#else
+#define GMLP_TR(kernel, site) do { } while (0)
+#endif
+
 // silu(g) = g * sigmoid(g), written g / (1 + e^-g): for g -> -inf this tends to -0 and never
 // forms 0 * inf.  ex2.approx / fast division are ~2^-21 relative, far below a bf16 ulp.
 __device__ __forceinline__ float silu_f32(float g) {

@@ -421,7 +421,8 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         for (int j = 0; j < n_blocks && ok; ++j) {
             // the scores of block j are complete, and with them every matmul issued before them: O += P V of block
             // j - 1 is done and has read its P
-            if (!wait_bounded(s_full0 + 8 * t, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 3)) { ok = false; break; }
+            // (the outcome is made warp-uniform: a warp must not split around the warp-wide instructions below)
+            if (!__all_sync(0xFFFFFFFFu, wait_bounded(s_full0 + 8 * t, (uint32_t)j & 1u, abort_flag, KERNEL_ID, 3))) { ok = false; break; }
             ptx::tc_fence_after_sync();
             // keys of this block that exist and that this row may see (0 when the whole block is beyond its horizon)
             const int valid = max(0, min(min(kGqaBS, S - j * kGqaBS), horizon - j * kGqaBS + 1));
@@ -432,7 +433,7 @@ gqa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             if (lane == 0) ptx::mbar_arrive(p_full0 + 8 * t);
         }
         // epilogue: O / l, one rounding, 256 contiguous bytes per row
-        if (ok && wait_bounded(o_full0 + 8 * t, (uint32_t)(n_blocks - 1) & 1u, abort_flag, KERNEL_ID, 7)) {
+        if (ok && __all_sync(0xFFFFFFFFu, wait_bounded(o_full0 + 8 * t, (uint32_t)(n_blocks - 1) & 1u, abort_flag, KERNEL_ID, 7))) {
             ptx::tc_fence_after_sync();
             const float inv_l = 1.0f / l_run;
             const int row = m0 + 128 * t + r;

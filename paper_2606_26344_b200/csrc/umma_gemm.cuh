@@ -294,7 +294,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const int m0 = (tile % num_m_tiles) * kUmmaBM;
             int n0 = (tile / num_m_tiles) * BN_OUT;
             const int row = m0 + q * 32 + lane;
-            if (!wait_bounded(tfull0 + 8 * buf, ((uint32_t)t >> 1) & 1u, abort_flag, KERNEL_ID, 3)) break;
+            // (warp-uniform outcome: a warp must not split around the warp-wide TMEM loads and __syncwarp below)
+            if (!__all_sync(0xFFFFFFFFu, wait_bounded(tfull0 + 8 * buf, ((uint32_t)t >> 1) & 1u, abort_flag, KERNEL_ID, 3))) break;
             ptx::tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * kUmmaN);
             bf16* Cseg = C;

@@ -17,6 +17,16 @@
 // Each CTA's TMEM holds its 128 rows x 256 columns, two buffers; the epilogue is the one of
 // umma_gemm.cuh.  Every wait is bounded; the pair leaves through a cluster barrier so that neither
 // CTA's shared memory or TMEM disappears under the other.
+//
+// CHUNKED = true (the Gated MLP's two GEMMs): the K loop is cut into chunks of `chunk_kb` k-blocks.  Each chunk
+// starts a fresh accumulation in one of the two TMEM buffers, and eight epilogue warps (two per TMEM lane
+// quarter, half of the columns each) add the finished chunk into fp32 REGISTERS with round-to-nearest while the
+// tensor cores fill the other buffer.  Reason: the tensor core adds into its fp32 accumulator by truncation, a
+// small bias toward zero per MMA that grows linearly with the length of the accumulation chain (measured: the
+// share of H values that round to another bf16 than the fp64 reference does is 1.8 % on rows scaled by 20 for one
+// chain of 512 MMAs, and falls in proportion to the chain length down to the 0.05 % of sequential fp32 FMA);
+// rows with |h| in the thousands then miss an absolute output tolerance.  Chains of 32 MMAs (8 k-blocks) joined
+// by ordinary fp32 additions behave like sequential fp32.  The per-tile epilogue then works from registers.
 #pragma once
 #include <cuda.h>
 
@@ -31,6 +41,8 @@ constexpr uint32_t kPairABytes = 128 * kUmmaBK * 2;               // 16 KB: this
 constexpr uint32_t kPairBBytes = 2 * kUmmaBoxBBytes;              // 16 KB: this CTA's 128 columns
 constexpr uint32_t kPairStageBytes = kPairABytes + kPairBBytes;   // 32 KB per CTA
 constexpr uint32_t kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + 256;
+constexpr int kPairChunkThreads = 64 + 8 * 32;                    // CHUNKED: producer, issuer and eight epilogue warps
+constexpr int kPairChunkKb = 8;                                   // k-blocks (of 64) per accumulation chain
 
 namespace ptx {
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -95,14 +107,15 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 }  // namespace ptx
 
 // ROWSCALE: see umma_gemm.cuh (epilogue row scale from row_rsqrt_kernel; only the epilogue waits for it).
-template <bool GATEUP, bool ROWSCALE = false, bool ADDSS = false, bool MULTI = false>
-__global__ void __launch_bounds__(kUmmaThreads, 1)
+template <bool GATEUP, bool ROWSCALE = false, bool ADDSS = false, bool MULTI = false, bool CHUNKED = false>
+__global__ void __launch_bounds__(CHUNKED ? kPairChunkThreads : kUmmaThreads, 1)
 umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                       const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
                       int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, GateAct act,
                       const bf16* residual, float* __restrict__ sumsq, const __grid_constant__ MultiB multi,
-                      int w_kmajor, int out_fp32)
+                      int w_kmajor, int out_fp32, int chunk_kb)
 {
+    static_assert(!(CHUNKED && (ROWSCALE || ADDSS || MULTI)), "chunked accumulation: the Gated MLP's two GEMMs only");
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
     static_assert(!(ADDSS && (GATEUP || ROWSCALE)), "the residual epilogue is for the plain GEMM");
     static_assert(!(MULTI && (GATEUP || ROWSCALE || ADDSS)), "several weight matrices: plain GEMM only");
@@ -138,7 +151,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(tfull0 + 8 * b, 1);
-            ptx::mbar_init(tempty0 + 8 * b, 8);                   // four epilogue warps of each CTA (used in the leader)
+            ptx::mbar_init(tempty0 + 8 * b, CHUNKED ? 16 : 8);    // the epilogue warps of both CTAs (used in the leader)
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -217,8 +230,41 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                                             : (uint32_t)ptx::make_smem_desc_sw128(base + kPairABytes, kUmmaBoxBBytes, 1024);
             const uint32_t b_step = w_kmajor ? 2u : 128u;
             uint32_t s = 0, ph = 0;                              // ring position of the next k-block
-            int t = 0;
             bool ok = true;
+            if (CHUNKED) {
+                // every chunk of chunk_kb k-blocks is an accumulation of its own, in the TMEM buffer its number selects
+                uint32_t n = 0;                                   // chunks issued so far (all tiles)
+                for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+                    int left = 0;                                 // k-blocks left in the current chunk
+                    uint32_t d_tmem = tmem_base;
+                    for (int kb = 0; kb < num_kb; ++kb) {
+                        const bool fresh = left == 0;
+                        if (fresh) {
+                            left = chunk_kb;
+                            if (!__all_sync(0xFFFFFFFFu, wait_bounded(tempty0 + 8 * (n & 1u), ((n >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4))) { ok = false; break; }
+                            ptx::tc_fence_after_sync();
+                            d_tmem = tmem_base + (n & 1u) * 256u;
+                        }
+                        if (!__all_sync(0xFFFFFFFFu, wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2))) { ok = false; break; }
+                        ptx::tc_fence_after_sync();
+                        const uint32_t a_lo = a_lo0 + s * (kPairStageBytes >> 4), b_lo = b_lo0 + s * (kPairStageBytes >> 4);
+                        --left;
+                        const bool closes = left == 0 || kb == num_kb - 1;
+                        if (leader) {
+                            ptx::umma_bf16_pair_halves(d_tmem, a_lo, b_lo, desc_hi, kIdesc, fresh ? 0u : 1u);
+#pragma unroll
+                            for (int k = 1; k < kUmmaBK / 16; ++k)
+                                ptx::umma_bf16_pair_halves(d_tmem, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
+                            ptx::umma_commit_pair(empty0 + 8 * s);
+                            if (closes) ptx::umma_commit_pair(tfull0 + 8 * (n & 1u));
+                        }
+                        __syncwarp();
+                        if (closes) { ++n; left = 0; }
+                        if (++s == (uint32_t)kPairStages) { s = 0; ph ^= 1u; }
+                    }
+                }
+            } else {
+            int t = 0;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++t) {
                 const int buf = t & 1;
                 if (!__all_sync(0xFFFFFFFFu, wait_bounded(tempty0 + 8 * buf, (((uint32_t)t >> 1) & 1u) ^ 1u, abort_flag, KERNEL_ID, 4))) break;
@@ -241,6 +287,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 if (ok && leader) ptx::umma_commit_pair(tfull0 + 8 * buf);
                 __syncwarp();
             }
+            }
         }
         __syncwarp();
     } else {
@@ -248,13 +295,83 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         const int q = warp & 3;
         ptx::grid_dependency_wait();
         const uint32_t leader_tempty0 = ptx::map_to_cta(tempty0, 0);
+        if (CHUNKED) {
+            // Warps 2..9: warp w reads TMEM lanes 32 (w % 4) .. +31 (its row) and half `hsel` of the tile's columns:
+            // gate/up: 64 gate accumulators (TMEM columns 64 hsel .. +63) and the 64 up accumulators of the same H
+            // columns (128 + 64 hsel ..); plain: 128 accumulators (columns 128 hsel ..).  The running sums of a
+            // tile live in registers; TMEM only ever holds one chunk per buffer.
+            const int hsel = (warp - 2) >> 2;
+            const int num_chunks = (num_kb + chunk_kb - 1) / chunk_kb;
+            uint32_t n = 0;                                       // chunks drained so far (all tiles)
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+                float acc[128];
+#pragma unroll
+                for (int i = 0; i < 128; ++i) acc[i] = 0.0f;
+                for (int c = 0; c < num_chunks; ++c, ++n) {
+                    const uint32_t buf = n & 1u;
+                    if (!__all_sync(0xFFFFFFFFu, wait_bounded(tfull0 + 8 * buf, (n >> 1) & 1u, abort_flag, KERNEL_ID, 3))) { ok = false; break; }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * 256u;
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        uint32_t r[32];
+                        const uint32_t col = GATEUP ? (uint32_t)((p >> 1) * 128 + hsel * 64 + (p & 1) * 32)
+                                                    : (uint32_t)(hsel * 128 + p * 32);
+                        ptx::tmem_ld_32x32(taddr + col, r);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) acc[p * 32 + i] += __uint_as_float(r[i]);
+                    }
+                    // this warp's reads of the buffer are done: hand it back to the MMA issuer
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty0 + 8 * buf);
+                }
+                if (!ok) break;
+                const int m0 = (tile % num_m_tiles) * 256 + (int)rank * 128;
+                const int row = m0 + q * 32 + lane;
+                if (row >= M) continue;
+                if (GATEUP) {
+                    const int col0 = (tile / num_m_tiles) * BN_OUT + hsel * 64;
+                    bf16* crow = C + (size_t)row * N + col0;
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int i = v * 8 + 2 * j;
+                            w[j] = pack_bf16x2(gate_act_f32(acc[i], act) * acc[64 + i], gate_act_f32(acc[i + 1], act) * acc[64 + i + 1]);
+                        }
+                        if (col0 + v * 8 < N) *reinterpret_cast<uint4*>(crow + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                } else {
+                    const int col0 = (tile / num_m_tiles) * BN_OUT + hsel * 128;
+                    if (out_fp32) {
+                        float* frow = reinterpret_cast<float*>(C) + (size_t)row * N + col0;
+#pragma unroll
+                        for (int v = 0; v < 32; ++v)
+                            if (col0 + v * 4 < N)
+                                *reinterpret_cast<float4*>(frow + v * 4) = make_float4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
+                    } else {
+                        bf16* crow = C + (size_t)row * N + col0;
+#pragma unroll
+                        for (int v = 0; v < 16; ++v)
+                            if (col0 + v * 8 < N)
+                                *reinterpret_cast<uint4*>(crow + v * 8) =
+                                    make_uint4(pack_bf16x2(acc[8 * v], acc[8 * v + 1]), pack_bf16x2(acc[8 * v + 2], acc[8 * v + 3]),
+                                               pack_bf16x2(acc[8 * v + 4], acc[8 * v + 5]), pack_bf16x2(acc[8 * v + 6], acc[8 * v + 7]));
+                    }
+                }
+            }
+        } else {
         int t = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++t) {
             const int buf = t & 1;
             const int m0 = (tile % num_m_tiles) * 256 + (int)rank * 128;
             int n0 = (tile / num_m_tiles) * BN_OUT;
             const int row = m0 + q * 32 + lane;
-            if (!wait_bounded(tfull0 + 8 * buf, ((uint32_t)t >> 1) & 1u, abort_flag, KERNEL_ID, 3)) break;
+            if (!__all_sync(0xFFFFFFFFu, wait_bounded(tfull0 + 8 * buf, ((uint32_t)t >> 1) & 1u, abort_flag, KERNEL_ID, 3))) break;
             ptx::tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256);
             bf16* Cseg = C;
@@ -319,6 +436,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty0 + 8 * buf);
+        }
         }
     }
 

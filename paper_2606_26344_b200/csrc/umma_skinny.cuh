@@ -253,8 +253,11 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     const long long u_begin = range_start(blockIdx.x, total, parts);
     const long long u_end = range_start(blockIdx.x + 1, total, parts);
 
+    constexpr int TRK = GATEUP ? 0 : 1;                  // timeline slot (GMLP_TRACE builds)
+    (void)TRK;
     ptx::launch_dependents();
     if (threadIdx.x == 0) {
+        GMLP_TR(TRK, 0);
         for (int s = 0; s < stages; ++s) {
             ptx::mbar_init(full0 + 8 * s, 1);
             ptx::mbar_init(empty0 + 8 * s, 1);
@@ -279,6 +282,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) GMLP_TR(TRK, 1);
     // TMEM column of accumulator (buffer b, matrix j, half h): Mpad fp32 columns each
     auto acc_col = [&](int b, int j, int h) -> uint32_t { return (uint32_t)(((b * NMAT + j) * NH + h) * Mpad); };
 
@@ -321,7 +325,9 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             const int head = (int)(n_units < stages ? n_units : stages);
             int tile = tile0, kb = kb0;
             for (int i = 0; i < head; ++i) { load_weights(tile, kb, i); step(tile, kb); }
+            if (leader) GMLP_TR(TRK, 2);
             ptx::grid_dependency_wait();
+            if (leader) GMLP_TR(TRK, 3);
             { int t2 = tile0, k2 = kb0; for (int i = 0; i < head; ++i) { load_tokens(k2, i); step(t2, k2); } }
             int s = head == stages ? 0 : head;                     // ring slot and its phase, stepped as well
             uint32_t ph = head == stages ? 1u : 0u;
@@ -333,6 +339,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 step(tile, kb);
                 if (++s == stages) { s = 0; ph ^= 1u; }
             }
+            if (leader) GMLP_TR(TRK, 4);
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -366,6 +373,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                 }
                 if (!__all_sync(0xFFFFFFFFu, wait_bounded(full0 + 8 * s, ph, abort_flag, KERNEL_ID, 2))) break;
                 ptx::tc_fence_after_sync();
+                if (leader && u == u_begin) GMLP_TR(TRK, 5);
                 const uint32_t tok_lo = tok_lo0 + (uint32_t)s * stage16, w_lo = w_lo0 + (uint32_t)s * stage16;
                 const bool last_of_segment = kb == KB - 1 || u == u_end - 1;
                 if (leader) {
@@ -381,6 +389,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                     }
                     ptx::umma_commit(empty0 + 8 * s);
                     if (last_of_segment) ptx::umma_commit(tfull0 + 8 * buf);
+                    if (u == u_end - 1) GMLP_TR(TRK, 6);
                 }
                 __syncwarp();
                 fresh = false;
@@ -410,12 +419,19 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             const int first_c = range_owner(tile_first, total, parts);
             const int last_c = range_owner(tile_first + KB - 1, total, parts);
             const int buf = seg & 1;
-            const bool ok = wait_bounded(tfull0 + 8 * buf, ((uint32_t)seg >> 1) & 1u, abort_flag, KERNEL_ID, 3);
+            (void)wait_bounded(tfull0 + 8 * buf, ((uint32_t)seg >> 1) & 1u, abort_flag, KERNEL_ID, 3);
             ptx::tc_fence_after_sync();
-            if (!ok) break;
-            skinny_epilogue_segment<GATEUP, NH>(tmem_base + lane_base + acc_col(buf, 0, 0), tempty0 + 8 * buf, tile,
+            // The segment's code contains barriers over all 128 epilogue threads, so they must all take the same
+            // branch: every wait above has ended (each is bounded); whoever gave up raised the abort flag first,
+            // and after this barrier every thread sees it.
+            epi_bar_sync();
+            if (*abort_flag) break;
+            if (et == 0) { if (seg == 0) GMLP_TR(TRK, 7); GMLP_TR(TRK, 8); }
+            const bool wrote = skinny_epilogue_segment<GATEUP, NH>(tmem_base + lane_base + acc_col(buf, 0, 0), tempty0 + 8 * buf, tile,
                                                 first_c, last_c, tile == first_tile, blockIdx.x, total, parts, KB, M, Mpad, N,
                                                 scratch, counters, out, slot_off, last_flag, et, nl, lane, act, out_fp32);
+            if (et == 0) { GMLP_TR(TRK, 9); if (wrote) GMLP_TR(TRK, 10); }
+            (void)wrote;
             u = seg_end;
         }
     }
@@ -425,6 +441,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) GMLP_TR(TRK, 11);
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, tmem_cols);

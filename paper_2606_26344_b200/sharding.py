@@ -55,23 +55,28 @@ def dff_range(d_ff: int, rank: int, world: int, multiple: int = 128) -> Tuple[in
     return min(first * multiple, d_ff), min(last * multiple, d_ff)
 
 
-def forward_dff_partial(X, Wg_s, Wu_s, Wd_s, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, stream=None):
+def forward_dff_partial(X, Wg_s, Wu_s, Wd_s, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, stream=None, P=None):
     """This rank's fp32 partial product [M, d_model] from its slice of the weights (Wg_s, Wu_s: [d_model, n],
-    Wd_s: [n, d_model]; n may be 0 for a rank left without a slice).  One call of the library."""
+    Wd_s: [n, d_model]; n may be 0 for a rank left without a slice).  One call of the library.  `P`: a float32
+    [M, d_model] buffer to reuse (it is overwritten)."""
     import torch
     from . import gmlp
     M, d_model = X.shape
-    P = torch.zeros(M, d_model, dtype=torch.float32, device=X.device)
+    if P is None:
+        P = torch.zeros(M, d_model, dtype=torch.float32, device=X.device)
     if Wg_s.shape[1] > 0:
         gmlp.forward(X, Wg_s, Wu_s, Wd_s, P, gamma, eps, rmsnorm, stream=stream)
+    else:
+        P.zero_()
     return P
 
 
-def forward_dff_sharded(X, Wg_s, Wu_s, Wd_s, dist=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, stream=None):
+def forward_dff_sharded(X, Wg_s, Wu_s, Wd_s, dist=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, stream=None,
+                        P=None, Y=None):
     """The whole layer with d_ff cut over the ranks of `dist` (one process per GPU): partial product, one all-reduce
-    (sum) of M * d_model floats, one rounding.  Every rank returns the full bf16 Y."""
+    (sum) of M * d_model floats, one rounding.  Every rank returns the full bf16 Y.  `P` / `Y`: buffers to reuse."""
     from . import gmlp
-    P = forward_dff_partial(X, Wg_s, Wu_s, Wd_s, gamma, eps, rmsnorm, stream)
+    P = forward_dff_partial(X, Wg_s, Wu_s, Wd_s, gamma, eps, rmsnorm, stream, P)
     if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(P)                                           # the path's only exchange
-    return gmlp.sum_partials([P], stream=stream)
+    return gmlp.sum_partials([P], Y, stream=stream)

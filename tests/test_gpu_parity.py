@@ -395,13 +395,42 @@ def test_h_with_more_than_two_to_the_31_elements():
     torch.cuda.empty_cache()
 
 
+# Bounds of the config-4 test, from the arithmetic of the data path (the derivation and the measured table are in the
+# design notes).  A tensor-core accumulation chain of L MMAs changes the bf16 that an H value rounds to, relative to the
+# fp64 reference, for a share of about 3.5e-5 * L of the values on rows scaled by 20 (half of that on ordinary rows):
+# measured linear from L = 512 (1.78e-2) down to L = 16 (5.7e-4).  The gate/up kernel keeps L = 32 at d_model = 8192:
+# 1.1e-3 expected; the bounds are 1.5 times that (the three sampled rows hold about a hundred flips, sigma = 10 %), rounded.
+H_FLIP_BOUND_OUTLIER_ROWS = 2.0e-3
+H_FLIP_BOUND_NORMAL_ROWS = 1.0e-3
+
+
+def expected_violations_upper(h_ref, y_ref, Wd_f64, flip_share):
+    """Elements of the given rows expected beyond 2e-2 * max(1, |y_ref|) when a share `flip_share` of the row's H
+    values, taken uniformly, is off by one bf16 step: the error of y[c] is then about normal with variance
+    flip_share * sum_n (step(h_n) * Wd[n, c])^2.  Uniform is pessimistic - flips favour small |h|, whose steps are
+    small - so this is an upper estimate (it gave 2 to 5 times the measured count over a range of flip shares)."""
+    from math import erfc, sqrt
+    step = np.where(h_ref != 0, 2.0 ** (np.floor(np.log2(np.abs(h_ref) + 1e-300)) - 7), 0.0)
+    sigma = np.sqrt(flip_share * (step ** 2) @ (Wd_f64 ** 2))
+    tol = oracle.tolerance(y_ref)
+    return float(sum(erfc(t / (s * sqrt(2.0))) for t, s in zip(tol.ravel(), sigma.ravel()) if s > 0))
+
+
 def test_llama70b_prefill_with_outlier_rows():
-    # Rows scaled x20 reach |h| ~ 2000, where ONE bf16 rounding flip of h (an effect of fp32 versus
-    # fp64 accumulation of g, u that any fp32-accumulating data path has) moves a y element by ~0.05,
-    # more than the absolute floor of the rule wherever |y_ref| is small (a CUDA-core fp32 FMA pipeline
-    # shows the same effect).  The strict rule is therefore applied to the 253 normal rows; on the 3
-    # sampled outlier rows the rule is applied with the row's own scale, 2e-2 * max(1, |y_ref|, rms(y_ref row)),
-    # H is checked against the oracle's H to one rounding step, and the strict count is printed.
+    # Rows scaled x20 reach |h| ~ 2000, where ONE bf16 rounding flip of h (an effect of fp32 versus fp64 accumulation
+    # of g and u that any fp32-accumulating data path has) moves every y of the row by ~0.05, more than the absolute
+    # floor of the rule wherever |y_ref| is small.  So the stated rule cannot hold on every element of such rows for
+    # any fp32 pipeline; what the test asserts:
+    #   normal rows (253): the stated rule, every element;
+    #   outlier rows (3): (a) the share of H values that differ from the oracle's H stays under the bound that the
+    #     kernel's accumulation-chain length implies, (b) the elements beyond the stated rule number no more than what
+    #     that share of one-step H errors can cause (an upper estimate computed here from the oracle's own H, y and
+    #     W_down) and no more than this library's sequential-fp32-FMA schedule leaves on the same rows plus one more
+    #     shifted row (the count comes in lumps: one flipped h of magnitude ~2000 shifts its whole row by ~0.05 and
+    #     puts every element with |y_ref| below about 2.5 out at once),
+    #     (c) the rule holds with the row's own scale, 2e-2 * max(1, |y_ref|, rms(y_ref row));
+    #   printed beside them: the same count for a CPU emulation of an fp32 data path (tests/_emulate.py).
+    from _emulate import fp32_path_rows
     w = I.WORKLOADS["llama3-70b-prefill-M4096-outliers"]
     inp = I.make_inputs(w)
     rows = I.sample_rows(w, inp.outlier_rows)
@@ -426,9 +455,24 @@ def test_llama70b_prefill_with_outlier_rows():
     h_ref = oracle.bf16_to_double(H_ref)
     h_rms = np.sqrt(np.mean(h_ref * h_ref, axis=1, keepdims=True))
     assert np.all(np.abs(h - h_ref) <= np.abs(h_ref) * 2.0 ** -7 + h_rms * 2.0 ** -10)
-    flips = float(np.mean(h != h_ref))
-    assert flips < 0.05
+    flips_out, flips_norm = float(np.mean(h[is_out] != h_ref[is_out])), float(np.mean(h[~is_out] != h_ref[~is_out]))
     strict_viol = int((e[is_out] > 1.0).sum())
-    print(f"70B: H flip fraction {flips:.4f}; outlier rows: {strict_viol} of {e[is_out].size} elements beyond the "
-          f"absolute-floor rule (max err/tol {e[is_out].max():.2f}), row-scaled max {np.max(np.abs(y - y_ref) / tol_row):.3f}; "
-          f"normal rows max err/tol {e[~is_out].max():.3f}")
+    # the yardsticks: this library's CUDA-core schedule (sequential fp32 FMA) and the CPU emulation, outlier rows only
+    out_rows = rows[is_out]
+    Xo = t["X"][torch.as_tensor(out_rows, device="cuda")].contiguous()
+    Yf = gmlp.forward(Xo, t["Wg"], t["Wu"], t["Wd"], variant=gmlp.VARIANT_STREAM, checked=True)
+    torch.cuda.synchronize()
+    fma_viol = int((np.abs(Yf.float().cpu().numpy().astype(np.float64) - y_ref[is_out]) > oracle.tolerance(y_ref[is_out])).sum())
+    y_emu, h_emu = fp32_path_rows(inp.bits("X"), inp.bits("Wg"), inp.bits("Wu"), inp.bits("Wd"), out_rows)
+    emu_viol = int((np.abs(y_emu - y_ref[is_out]) > oracle.tolerance(y_ref[is_out])).sum())
+    emu_flips = float(np.mean(h_emu != h_ref[is_out]))
+    upper = expected_violations_upper(h_ref[is_out], y_ref[is_out], inp.Wd.double().numpy(), H_FLIP_BOUND_OUTLIER_ROWS)
+    print(f"70B: H flip share {flips_out:.5f} on outlier rows (bound {H_FLIP_BOUND_OUTLIER_ROWS}), {flips_norm:.5f} on normal rows "
+          f"(bound {H_FLIP_BOUND_NORMAL_ROWS}); outlier rows: {strict_viol} of {e[is_out].size} elements beyond the absolute-floor "
+          f"rule (max err/tol {e[is_out].max():.2f}; upper estimate for the flip bound {upper:.0f}; sequential-FMA schedule "
+          f"{fma_viol}; CPU fp32 emulation {emu_viol} with flip share {emu_flips:.5f}), row-scaled max "
+          f"{np.max(np.abs(y - y_ref) / tol_row):.3f}; normal rows max err/tol {e[~is_out].max():.3f}")
+    assert flips_out <= H_FLIP_BOUND_OUTLIER_ROWS and flips_norm <= H_FLIP_BOUND_NORMAL_ROWS
+    assert strict_viol <= upper
+    one_row_shift = int((np.abs(y_ref[is_out]) < 2.5).sum(axis=1).max())
+    assert strict_viol <= fma_viol + one_row_shift
