@@ -20,6 +20,7 @@
 #include "umma_gemm_2cta.cuh"
 #include "umma_gemm_splitk.cuh"
 #include "umma_skinny.cuh"
+#include "umma_skinny_cluster.cuh"
 #include "gqa_attention.cuh"
 
 namespace {
@@ -121,6 +122,8 @@ struct DeviceState {
     bool pair_attr_set = false;
     bool rowscale_attr_set = false;
     bool skinny_attr_set = false;
+    bool skinny_cluster_attr_set = false;
+    int cluster_capacity[2][9] = {};             // clusters of C CTAs of the cluster-form kernels resident at once (0 = not asked yet)
     // arrival-counter regions zeroed by the library (the kernels leave them zero after every call); a few are
     // remembered so that callers alternating between workspaces (one per stream) do not pay a memset per call
     static constexpr int kCleanSlots = 4;
@@ -206,12 +209,26 @@ StreamPlan make_stream_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
     return p;
 }
 
+// Clusters of C CTAs (one CTA per SM, about half of an SM's shared memory each) that a device with `sms` SMs holds at
+// once.  A cluster lives inside one GPC, and the GPCs do not all have a multiple of C SMs: measured on B200 (148 SMs;
+// cudaOccupancyMaxActiveClusters) 74 / 45 / 33 / 26 / 22 / 15 / 15 for C = 2 .. 8.  Elsewhere a cautious guess; the launch
+// asks the runtime and falls back to the stream-K form if the plan's clusters do not fit one wave.
+int cluster_capacity_estimate(int C, int sms) {
+    static const int b200[9] = {0, 148, 74, 45, 33, 26, 22, 15, 15};
+    if (C < 1 || C > 8) return 0;
+    if (sms == 148) return b200[C];
+    return C == 1 ? sms : (sms / C) * 85 / 100;
+}
+
 // ------------------------------------------------------------------ skinny (swap-AB tcgen05) plan
 struct SkinnyPlan {
     int Mpad, NH, num_tiles, KB, stages, grid;
     uint32_t smem_bytes;
     uint32_t tmem_cols;
     uint64_t scratch_bytes;
+    // cluster form (umma_skinny_cluster.cuh): CTAs per 128-column tile, 0 = not applicable (the stream-K form runs)
+    int cluster, c_boxes, c_tiles, c_stages;     // c_boxes: 64-column boxes per tile (2 = 128-column tiles, 1 = 64)
+    uint32_t c_smem_bytes, c_tmem_cols, c_staging_off;    // c_staging_off: the partial sums' own region (0 = they reuse the ring)
 };
 
 SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_count) {
@@ -260,7 +277,68 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
         const int64_t contrib = p.KB / per_cta + 2 < p.grid ? p.KB / per_cta + 2 : p.grid;
         if (contrib > gmlp::kSkinnyMaxContrib) p.stages = 0;               // launch_skinny refuses the plan
     }
-    p.scratch_bytes = (uint64_t)p.grid * 2 * nmat * p.NH * p.Mpad * 128 * 4;
+    // (beyond 128 tokens only the cluster form below can run, and it needs no scratch)
+    p.scratch_bytes = M > 128 ? 0 : (uint64_t)p.grid * 2 * nmat * p.NH * p.Mpad * 128 * 4;
+    // Cluster form: one cluster of C CTAs per column tile (128 columns, or 64), K split C ways and reduced in distributed
+    // shared memory.  Taken for few tokens when the tiles are fewer than the SMs and tiles x C - with C <= 8, two k-blocks
+    // or more per CTA, the non-leaders' partial sums fitting the leader's ring, and all clusters resident at once - fill at
+    // least 80 % of the SMs; otherwise (8B and 70B gate/up: 112 and 224 tiles) the stream-K form keeps every SM streaming.
+    p.cluster = 0;
+    p.c_boxes = 2;
+    p.c_tiles = 0;
+    p.c_stages = 0;
+    p.c_smem_bytes = 0;
+    p.c_staging_off = 0;
+    {
+        uint32_t c_cols = (uint32_t)(nmat * p.Mpad), c_pow2 = 32;
+        while (c_pow2 < c_cols) c_pow2 <<= 1;
+        p.c_tmem_cols = c_pow2;
+        int forced = -1;
+        if (const char* e = getenv(nmat == 2 ? "GMLP_SKINNY_CLUSTER1" : "GMLP_SKINNY_CLUSTER2")) forced = atoi(e);   // tuning override: 0 = stream-K, 1..8 = that cluster size
+        int forced_boxes = 0;
+        if (const char* e = getenv("GMLP_SKINNY_CLUSTER_BOXES")) forced_boxes = atoi(e);                              // tuning override: 1 or 2
+        int64_t best_ctas = 0;
+        for (int boxes = 2; boxes >= 1 && p.Mpad <= gmlp::kSkinnyClusterMaxTokens && forced != 0; --boxes) {
+            if (forced_boxes != 0 && forced_boxes != boxes) continue;
+            if (boxes == 1 && p.cluster >= 1 && forced_boxes == 0) break;        // the wide tiles qualified
+            const int tiles = (int)((N + 64 * boxes - 1) / (64 * boxes));
+            const uint32_t c_stage_bytes = (uint32_t)(nmat * boxes) * gmlp::kSkinnyBoxBytes + (uint32_t)p.Mpad * 128u;
+            // (a 64-column tile's MMA reads one box length past its box: keep that inside the allocation)
+            const uint32_t tail = 1024 + 256 + (boxes == 1 ? gmlp::kSkinnyBoxBytes : 0);
+            // few tokens: half of the shared memory, so that the next kernel on the stream is co-resident (see above)
+            int cst = (int)(((small ? gmlp::kSkinnySmemBudget / 2 : gmlp::kSkinnySmemBudget) - tail) / c_stage_bytes);
+            if (cst > gmlp::kSkinnyMaxStages) cst = gmlp::kSkinnyMaxStages;
+            if (tiles > sms || cst < 2) continue;
+            int C = forced > 0 ? forced : sms / tiles;
+            if (C > 8) C = 8;
+            if (C > p.KB / 2) C = p.KB / 2 > 0 ? p.KB / 2 : 1;
+            while (C > 1 && (gmlp::skinny_cluster_staging_bytes(C, nmat, (int)M) > (uint32_t)cst * c_stage_bytes ||
+                             cluster_capacity_estimate(C, sms) < tiles))
+                --C;
+            if (forced > 0 && C != forced) continue;
+            const int64_t ctas = (int64_t)tiles * C;
+            // 128-column tiles read 256 contiguous bytes per weight row, 64-column tiles 128: the narrow rows use DRAM
+            // so much worse (8B down projection, 128 CTAs either way: 34.8 against 26.9 us) that the wide tiles are
+            // taken from 60 % of the SMs on, the narrow ones only if they alone reach 80 %
+            if (ctas > best_ctas && (forced > 0 || ctas * 10 >= (int64_t)sms * (boxes == 2 ? 6 : 8))) {
+                best_ctas = ctas;
+                p.cluster = C;
+                p.c_boxes = boxes;
+                p.c_tiles = tiles;
+                // partial sums of at most 24 KB get a region of their own behind the ring and its barriers (a stage less
+                // if need be): the senders then do not have to wait for the receiver's ring to be free
+                const uint32_t staging = gmlp::skinny_cluster_staging_bytes(C, nmat, (int)M);
+                const uint32_t limit = small ? gmlp::kSkinnySmemBudget / 2 : gmlp::kSkinnySmemBudget;
+                p.c_staging_off = 0;
+                if (C > 1 && staging <= 24 * 1024) {
+                    while (cst > 2 && (uint32_t)cst * c_stage_bytes + tail + staging > limit) --cst;
+                    if ((uint32_t)cst * c_stage_bytes + tail + staging <= limit) p.c_staging_off = (uint32_t)cst * c_stage_bytes + tail;
+                }
+                p.c_stages = cst;
+                p.c_smem_bytes = (uint32_t)cst * c_stage_bytes + tail + (p.c_staging_off ? staging : 0);
+            }
+        }
+    }
     return p;
 }
 
@@ -304,11 +382,17 @@ int tuned_variant(int64_t M, int64_t d_model, int64_t d_ff) {
     return tuned_lookup(M, d_model, d_ff, &t) ? t.variant : GMLP_VARIANT_AUTO;
 }
 
+bool skinny_both_cluster(int64_t M, int64_t d_model, int64_t d_ff);
+
 int resolve_variant(int64_t M, int64_t d_model, int64_t d_ff, int32_t variant) {
     if (variant != GMLP_VARIANT_AUTO) return variant;
     const int tuned = tuned_variant(M, d_model, d_ff);
     if (tuned != GMLP_VARIANT_AUTO) return tuned;
-    return M <= 16 ? GMLP_VARIANT_SKINNY : GMLP_VARIANT_TENSOR;
+    if (M <= 16) return GMLP_VARIANT_SKINNY;
+    // up to 24 tokens the operand-swapped schedule still wins where both of its GEMMs run in the cluster form (layers
+    // with fewer column tiles than SMs; 2048 x 5632 at 17 tokens: 23.9 against 32.1 us; level at 32)
+    if (M <= 24 && skinny_both_cluster(M, d_model, d_ff)) return GMLP_VARIANT_SKINNY;
+    return GMLP_VARIANT_TENSOR;
 }
 
 // TENSOR: which kernel each GEMM takes.  Both kernels are persistent, so a GEMM costs (rounds of tiles over the SMs)
@@ -406,6 +490,27 @@ Layout make_layout(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int
     }
     L.total = off;
     return L;
+}
+
+// The operand-swapped schedule takes up to 128 tokens in its stream-K form, and up to kSkinnyClusterMaxTokens when both
+// GEMMs of the shape have a cluster form.
+bool skinny_can_run(int64_t M, int64_t d_model, int64_t d_ff, int sm_count) {
+    if (M <= 128) return true;
+    if (M > gmlp::kSkinnyClusterMaxTokens) return false;
+    return make_skinny_plan(M, d_model, d_ff, 2, sm_count).cluster >= 1 && make_skinny_plan(M, d_ff, d_model, 1, sm_count).cluster >= 1;
+}
+
+int current_sm_count() {
+    int dev = -1, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+        return sms;
+    (void)cudaGetLastError();
+    return 148;
+}
+bool skinny_both_cluster(int64_t M, int64_t d_model, int64_t d_ff) {
+    const int sms = current_sm_count();
+    return make_skinny_plan(M, d_model, d_ff, 2, sms).cluster >= 1 && make_skinny_plan(M, d_ff, d_model, 1, sms).cluster >= 1;
 }
 
 int check_shape(int64_t M, int64_t d_model, int64_t d_ff) {
@@ -749,13 +854,65 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     return GMLP_OK;
 }
 
+// The cluster form of a small-M GEMM (umma_skinny_cluster.cuh).  Returns GMLP_ERR_UNSUPPORTED when the device cannot
+// hold the plan's clusters in one wave (the caller then runs the stream-K form).
+template <bool GATEUP>
+int launch_skinny_cluster(DeviceState* dev, const SkinnyPlan& p, const CUtensorMap& tmX, const CUtensorMap& tmW0,
+                          const CUtensorMap& tmW1, bf16* out, int64_t M, int64_t N, cudaStream_t st, gmlp::GateAct act,
+                          int wkm, int yf32) {
+    if (!dev->skinny_cluster_attr_set) {
+        const int b = (int)gmlp::kSkinnySmemBudget;
+        if (cudaFuncSetAttribute(gmlp::skinny_cluster_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess ||
+            cudaFuncSetAttribute(gmlp::skinny_cluster_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, b) != cudaSuccess)
+            return GMLP_ERR_LAUNCH;
+        dev->skinny_cluster_attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.c_tiles * p.cluster));
+    cfg.blockDim = dim3(gmlp::kSkinnyThreads);
+    cfg.dynamicSmemBytes = p.c_smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)p.cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    int& capacity = dev->cluster_capacity[GATEUP ? 0 : 1][p.cluster];
+    if (capacity == 0) {
+        int n = 0;
+        cfg.numAttrs = 1;                                   // the occupancy query takes the cluster shape only
+        if (cudaOccupancyMaxActiveClusters(&n, gmlp::skinny_cluster_gemm_kernel<GATEUP>, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            n = -1;
+        }
+        cfg.numAttrs = 2;
+        capacity = n > 0 ? n : -1;
+        if (getenv("GMLP_TUNE_VERBOSE"))
+            fprintf(stderr, "gmlp: clusters of %d CTAs (%s, %u B shared memory) resident at once: %d\n", p.cluster,
+                    GATEUP ? "gate/up" : "down", p.c_smem_bytes, n);
+    }
+    if (capacity < p.c_tiles) return GMLP_ERR_UNSUPPORTED;
+    const int Mi = (int)M, Ni = (int)N;
+    int evict_first = 1;
+    if (const char* e = getenv("GMLP_SKINNY_EVICT_FIRST")) evict_first = atoi(e);      // tuning override
+    if (cudaLaunchKernelEx(&cfg, gmlp::skinny_cluster_gemm_kernel<GATEUP>, tmX, tmW0, tmW1, out, Mi, p.Mpad, Ni, p.KB, p.c_stages,
+                           p.c_tmem_cols, evict_first, act, wkm, yf32, p.c_boxes, p.c_staging_off) != cudaSuccess)
+        return GMLP_ERR_LAUNCH;
+    GMLP_CHECK_LAUNCH();
+    return GMLP_OK;
+}
+
 template <bool GATEUP>
 int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf16* W0, const bf16* W1, float* scratch,
                   unsigned int* counters, bf16* out, int64_t M, int64_t K, int64_t N, cudaStream_t st,
                   gmlp::GateAct act = kSilu) {
     const int wkm = t_w_out_in ? 1 : 0;
     const int yf32 = (!GATEUP && t_y_fp32) ? 1 : 0;
-    if (p.stages < 2 || p.tmem_cols > 512) return GMLP_ERR_UNSUPPORTED;
+    if (p.cluster < 1 && (p.stages < 2 || p.tmem_cols > 512)) return GMLP_ERR_UNSUPPORTED;
     CUtensorMap tmX, tmW0, tmW1;
     if (!encode_2d(&tmX, X, (uint64_t)K, (uint64_t)M, 64, (uint32_t)p.Mpad)) return GMLP_ERR_LAUNCH;
     if (!GMLP_ENCODE_W(&tmW0, W0, N, K)) return GMLP_ERR_LAUNCH;
@@ -763,6 +920,11 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
         if (!GMLP_ENCODE_W(&tmW1, W1, N, K)) return GMLP_ERR_LAUNCH;
     } else {
         tmW1 = tmW0;
+    }
+    if (p.cluster >= 1) {
+        const int rc = launch_skinny_cluster<GATEUP>(dev, p, tmX, tmW0, tmW1, out, M, N, st, act, wkm, yf32);
+        if (rc != GMLP_ERR_UNSUPPORTED) return rc;          // clusters that do not fit one wave: the stream-K form below
+        if (M > 128 || p.stages < 2 || p.tmem_cols > 512) return GMLP_ERR_UNSUPPORTED;
     }
     if (!dev->skinny_attr_set) {
         const int b = (int)gmlp::kSkinnySmemBudget;
@@ -848,7 +1010,7 @@ int forward_impl(const gmlp_args* a) {
     if (dev == nullptr) return rc;
 
     const int variant = resolve_variant(a->M, a->d_model, a->d_ff, a->variant);
-    if (variant == GMLP_VARIANT_SKINNY && a->M > 128) return GMLP_ERR_UNSUPPORTED;
+    if (variant == GMLP_VARIANT_SKINNY && !skinny_can_run(a->M, a->d_model, a->d_ff, dev->sm_count)) return GMLP_ERR_UNSUPPORTED;
     const bool w_out_in = (a->flags & GMLP_FLAG_WEIGHTS_OUT_IN) != 0;
     const bool y_fp32 = (a->flags & GMLP_FLAG_Y_FP32) != 0;
     if ((w_out_in || y_fp32) && (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM)) return GMLP_ERR_UNSUPPORTED;
@@ -1029,11 +1191,11 @@ int gate_up_impl(const gmlp_args* a) {
     if (a->workspace != nullptr && (reinterpret_cast<uintptr_t>(a->workspace) & 255u)) return GMLP_ERR_ALIGN;
     const int variant = resolve_variant(a->M, a->d_model, a->d_ff, a->variant);
     if (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM) return GMLP_ERR_UNSUPPORTED;
-    if (variant == GMLP_VARIANT_SKINNY && a->M > 128) return GMLP_ERR_UNSUPPORTED;
     if (a->flags & GMLP_FLAG_Y_FP32) return GMLP_ERR_FLAGS;          // H is the bf16 operand of the next GEMM
     const WeightLayoutScope layout_scope((a->flags & GMLP_FLAG_WEIGHTS_OUT_IN) != 0);
     DeviceState* dev = current_device(&rc);
     if (dev == nullptr) return rc;
+    if (variant == GMLP_VARIANT_SKINNY && !skinny_can_run(a->M, a->d_model, a->d_ff, dev->sm_count)) return GMLP_ERR_UNSUPPORTED;
     const Layout L = make_layout(a->M, a->d_model, a->d_ff, a->flags, variant, dev->sm_count);
     uint8_t* ws = static_cast<uint8_t*>(a->workspace);
     if (ws == nullptr) {
@@ -1486,7 +1648,7 @@ int autotune_impl(const gmlp_args* a, int iters, int32_t* best_variant, float* b
     int n_usable = 0;
     for (int c = 0; c < 5; ++c) {
         const int v = candidates[c].variant;
-        usable[c] = !(v == GMLP_VARIANT_SKINNY && a->M > 128) &&
+        usable[c] = !(v == GMLP_VARIANT_SKINNY && !skinny_can_run(a->M, a->d_model, a->d_ff, dev->sm_count)) &&
                     !(a->workspace != nullptr &&      // the caller's workspace must hold the schedule
                       make_layout(a->M, a->d_model, a->d_ff, a->flags, v, dev->sm_count).total > a->workspace_bytes);
         n_usable += usable[c] ? 1 : 0;

@@ -106,6 +106,39 @@ def test_small_m_path_is_stable_over_many_back_to_back_calls():
     assert e.max() <= 1.0
 
 
+@pytest.mark.parametrize("rmsnorm", [False, True])
+@pytest.mark.parametrize("shape", [(1, 2048, 5632), (7, 2048, 5632), (16, 2048, 5632), (24, 2048, 5632), (129, 2048, 5632),
+                                   (250, 2048, 5632), (5, 2040, 5624), (8, 4096, 14336), (3, 8192, 8192), (13, 1024, 9000)])
+def test_skinny_schedule_cluster_form(shape, rmsnorm):
+    """Layers with fewer column tiles than SMs: a cluster of CTAs per tile splits K and reduce-scatters the partial sums in
+    distributed shared memory (128-column tiles x 3 CTAs and 64-column tiles x 4 CTAs on the 2048 x 5632 layer; more than
+    128 tokens run in this form only).  Ragged widths put the tile and k-block tails in play."""
+    M, dm, dff = shape
+    inp = I.custom_inputs(M, dm, dff, seed=M + dm, rmsnorm=rmsnorm, eps=1e-6)
+    check_case(inp, SKINNY, f"skinny-cluster {shape} norm={rmsnorm}")
+
+
+def test_skinny_cluster_sizes_agree_within_tolerance_and_are_deterministic():
+    """Every cluster size the device can hold (a tuning override forces it) gives the oracle's result within the rule,
+    and the same bits on a second call."""
+    import os
+    inp = I.custom_inputs(9, 1024, 2048, 3)
+    t = to_device(inp)
+    y_ref = oracle_rows(inp, np.arange(9))
+    try:
+        for c in ("1", "2", "3", "4", "5", "6"):
+            os.environ["GMLP_SKINNY_CLUSTER1"] = os.environ["GMLP_SKINNY_CLUSTER2"] = c
+            a = gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], variant=SKINNY, checked=True)
+            b = gmlp.forward(t["X"], t["Wg"], t["Wu"], t["Wd"], variant=SKINNY, checked=True)
+            torch.cuda.synchronize()
+            assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+            e, _ = err_over_tol(a, y_ref, np.arange(9))
+            assert float(e.max()) <= 1.0, f"cluster size {c}: max err/tol {float(e.max()):.3f}"
+    finally:
+        os.environ.pop("GMLP_SKINNY_CLUSTER1", None)
+        os.environ.pop("GMLP_SKINNY_CLUSTER2", None)
+
+
 def test_skinny_rejects_more_than_128_rows():
     inp = I.custom_inputs(129, 64, 128, 1)
     t = to_device(inp)
