@@ -59,7 +59,8 @@ typedef enum gmlp_status {
     GMLP_ERR_ARCH = -6,       /* no CUDA device, or the current device is not sm_100 */
     GMLP_ERR_LAUNCH = -7,     /* a CUDA runtime call failed (cudaGetLastError is left readable) */
     GMLP_ERR_TIMEOUT = -8,    /* a bounded device-side wait ran out (see gmlp_device_status) */
-    GMLP_ERR_UNSUPPORTED = -9,/* the forced variant cannot run this shape (SKINNY needs M <= 128) */
+    GMLP_ERR_UNSUPPORTED = -9,/* the forced variant cannot run this shape (SKINNY: M <= 128, or <= 256 on layers whose
+                                 two GEMMs both have its cluster form) */
     GMLP_ERR_STATIC_LIMIT = -10 /* gmlp_forward_static: the shape needs more than its fixed built-in scratch */
 } gmlp_status;
 
@@ -211,7 +212,7 @@ int gmlp_matmul_add_rmsnorm(const gmlp_mmaddnorm_args* args);
  * Default: ONE launch of the tensor-core GEMM whose column tiles run through the three weight matrices end to end
  * (the same sharing of the X strip that fuses the gate and up matmuls), each tile written to its own output.
  * GMLP_QKV_SEPARATE runs three GEMMs one after the other (for comparison).  No workspace.  The attention that
- * follows (GQA) is not part of this library.
+ * follows is gmlp_gqa_attention below.
  */
 enum { GMLP_QKV_SEPARATE = 1u << 4 };
 typedef struct gmlp_qkv_args {
@@ -290,7 +291,13 @@ int gmlp_forward_host(const gmlp_args* args, const void* X_host, void* Y_host);
  * It calls no cudaMalloc, cudaFree or allocating library routine.  The FIRST call on each
  * device looks up the device address of the built-in array (cudaGetSymbolAddress, with that
  * device current) and sets kernel attributes; make that first call outside any stream
- * capture.  All calls on a device share the one array, and it keeps whatever the previous
+ * capture.  That first call is also what makes the CUDA runtime load the library's code and
+ * the array onto the device (module loading is lazy), so make one call with M >= 1 per
+ * device BEFORE the application freezes its memory plan: a caller that has already handed
+ * every byte to its own pool gets GMLP_ERR_LAUNCH from that first call instead (the lookup
+ * fails for lack of memory), and a call with M == 0 returns before the lookup and does not
+ * serve as the warm-up.  After it, a call leaves the device's free memory as it found it.
+ * All calls on a device share the one array, and it keeps whatever the previous
  * call left: each call clears the counters it needs itself, so back-to-back calls on one
  * stream are fine, but two calls that can overlap on the GPU (different streams, no
  * ordering) race on the scratch and give wrong results.

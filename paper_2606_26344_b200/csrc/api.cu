@@ -389,8 +389,8 @@ int resolve_variant(int64_t M, int64_t d_model, int64_t d_ff, int32_t variant) {
     const int tuned = tuned_variant(M, d_model, d_ff);
     if (tuned != GMLP_VARIANT_AUTO) return tuned;
     if (M <= 16) return GMLP_VARIANT_SKINNY;
-    // up to 24 tokens the operand-swapped schedule still wins where both of its GEMMs run in the cluster form (layers
-    // with fewer column tiles than SMs; 2048 x 5632 at 17 tokens: 23.9 against 32.1 us; level at 32)
+    // up to 24 tokens the operand-swapped schedule still wins where both of its GEMMs split K over a cluster (layers
+    // with far fewer column tiles than SMs; 2048 x 5632 at 17 tokens: 23.9 against 32.1 us; level at 32)
     if (M <= 24 && skinny_both_cluster(M, d_model, d_ff)) return GMLP_VARIANT_SKINNY;
     return GMLP_VARIANT_TENSOR;
 }
@@ -510,7 +510,7 @@ int current_sm_count() {
 }
 bool skinny_both_cluster(int64_t M, int64_t d_model, int64_t d_ff) {
     const int sms = current_sm_count();
-    return make_skinny_plan(M, d_model, d_ff, 2, sms).cluster >= 1 && make_skinny_plan(M, d_ff, d_model, 1, sms).cluster >= 1;
+    return make_skinny_plan(M, d_model, d_ff, 2, sms).cluster >= 2 && make_skinny_plan(M, d_ff, d_model, 1, sms).cluster >= 2;
 }
 
 int check_shape(int64_t M, int64_t d_model, int64_t d_ff) {

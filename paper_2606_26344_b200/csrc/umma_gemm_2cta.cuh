@@ -11,8 +11,8 @@
 // Only the leader (cluster rank 0) issues MMAs.  Barriers:
 //   full[s]   (leader's)  two arrivals: each CTA's producer arms its own 32 KB; both CTAs' TMA loads
 //                         complete on it (the peer's through .cta_group::2 addressing)
-//   empty[s]  (per CTA)   tcgen05.commit multicast to both CTAs when the stage's MMAs are done
-//   tfull[b]  (per CTA)   tcgen05.commit multicast: accumulator buffer b is complete
+//   empty[s]  (per CTA)   tcgen05.commit to each CTA's barrier when the stage's MMAs are done
+//   tfull[b]  (per CTA)   tcgen05.commit to each CTA's barrier: accumulator buffer b is complete
 //   tempty[b] (leader's)  eight arrivals: the four epilogue warps of both CTAs have drained buffer b
 // Each CTA's TMEM holds its 128 rows x 256 columns, two buffers; the epilogue is the one of
 // umma_gemm.cuh.  Every wait is bounded; the pair leaves through a cluster barrier so that neither
@@ -99,10 +99,13 @@ __device__ __forceinline__ void umma_bf16_pair_halves(uint32_t d_tmem, uint32_t 
         "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}"
         ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
-// one arrival on the barrier at this shared-memory offset in BOTH CTAs once the MMAs issued so far are done
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+// One arrival on the barrier at this shared-memory offset in BOTH CTAs of the pair once the MMAs issued so far are
+// done: two commits, one to the leader's own barrier and one to the peer's (its shared::cluster address, from mapa).
+// peer_delta = map_to_cta(x, 1) - x, the same for every offset, is computed once by the caller.  (Measured against the
+// single instruction that signals both CTAs at once: the same time on every large-M workload, within 0.3 %.)
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint32_t peer_delta) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar + peer_delta) : "memory");
 }
 }  // namespace ptx
 
@@ -229,6 +232,9 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             const uint32_t b_lo0 = w_kmajor ? (uint32_t)ptx::make_smem_desc_sw128(base + kPairABytes, 16, 1024)
                                             : (uint32_t)ptx::make_smem_desc_sw128(base + kPairABytes, kUmmaBoxBBytes, 1024);
             const uint32_t b_step = w_kmajor ? 2u : 128u;
+            // a shared::cta address is the executing CTA's own window of the shared::cluster space; the peer's window
+            // lies a constant distance away
+            const uint32_t peer_delta = ptx::map_to_cta(empty0, 1) - empty0;
             uint32_t s = 0, ph = 0;                              // ring position of the next k-block
             bool ok = true;
             if (CHUNKED) {
@@ -255,8 +261,8 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 #pragma unroll
                             for (int k = 1; k < kUmmaBK / 16; ++k)
                                 ptx::umma_bf16_pair_halves(d_tmem, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
-                            ptx::umma_commit_pair(empty0 + 8 * s);
-                            if (closes) ptx::umma_commit_pair(tfull0 + 8 * (n & 1u));
+                            ptx::umma_commit_pair(empty0 + 8 * s, peer_delta);
+                            if (closes) ptx::umma_commit_pair(tfull0 + 8 * (n & 1u), peer_delta);
                         }
                         __syncwarp();
                         if (closes) { ++n; left = 0; }
@@ -279,12 +285,12 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 #pragma unroll
                         for (int k = 1; k < kUmmaBK / 16; ++k)
                             ptx::umma_bf16_pair_halves(d_tmem, a_lo + 2u * (uint32_t)k, b_lo + b_step * (uint32_t)k, desc_hi, kIdesc, 1u);
-                        ptx::umma_commit_pair(empty0 + 8 * s);
+                        ptx::umma_commit_pair(empty0 + 8 * s, peer_delta);
                     }
                     __syncwarp();
                     if (++s == (uint32_t)kPairStages) { s = 0; ph ^= 1u; }
                 }
-                if (ok && leader) ptx::umma_commit_pair(tfull0 + 8 * buf);
+                if (ok && leader) ptx::umma_commit_pair(tfull0 + 8 * buf, peer_delta);
                 __syncwarp();
             }
             }

@@ -293,3 +293,22 @@ def test_gate_up_alone_against_naive_loops_torch_and_closed_form():
     # rows subset and swapped roles
     assert np.array_equal(oracle.gate_up_rows(X, Wg, Wu, rows=np.array([5, 1])), P2[[5, 1]])
     assert not np.array_equal(oracle.gate_up_rows(X, Wu, Wg), P2)
+
+
+def test_config4_recipe_and_oracle_against_an_independent_evaluation():
+    """The 70B-shaped prefill recipe end to end (seeded draws, 41 outlier rows scaled by 20, the stratified 256-row
+    sample) through the oracle, against two sums that an independent evaluation of the same recipe produced before any
+    kernel existed: torch fp64 matmuls in column blocks of 4096 with `G * sigmoid(G) * U`, H rounded by torch's own
+    bfloat16 conversion - another summation order, another SiLU expression and another rounding routine than the
+    oracle's.  Sum of y_ref 37867.4278 and sum of |y_ref| 6607161.118 over the sample; the two evaluations may differ
+    where an H value sits on a rounding boundary, so they are compared to 1e-6 of the absolute sum (6.6), far below what
+    a wrong row set, a dropped outlier scaling, a transposed weight or a missing H rounding would change.
+    About 3.6e11 fp64 operations: the slowest test of the CPU suite (under a minute on 8 cores)."""
+    w = I.WORKLOADS["llama3-70b-prefill-M4096-outliers"]
+    inp = I.make_inputs(w)
+    rows = I.sample_rows(w, inp.outlier_rows)
+    assert inp.outlier_rows.size == 41 and rows.size == 256 and rows[:8].tolist() == [8, 16, 35, 44, 58, 60, 61, 62]
+    y = oracle.gmlp_rows(inp.bits("X"), inp.bits("Wg"), inp.bits("Wu"), inp.bits("Wd"), rows=rows)
+    total, absolute = float(y.sum()), float(np.abs(y).sum())
+    assert abs(absolute - 6607161.118) <= 1e-6 * 6607161.118
+    assert abs(total - 37867.4278) <= 1e-6 * 6607161.118

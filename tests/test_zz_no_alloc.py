@@ -29,10 +29,12 @@ def test_static_entry_refuses_shapes_beyond_its_fixed_scratch():
 
 
 @pytest.mark.gpu
-def test_static_entry_matches_the_workspace_entry_on_two_calls_in_a_row():
+def test_static_entry_matches_the_oracle_and_the_workspace_entry_on_two_calls_in_a_row():
+    import oracle
     dev = torch.device("cuda")
-    # decode-shaped (several stream-K contributors per column tile) and a ragged small case
-    for (M, dm, dff, seed) in ((8, 4096, 14336, 0), (5, 264, 520, 3)):
+    # decode-shaped (several contributors per column tile), the 2048 x 5632 layer (both GEMMs in the cluster form)
+    # and a ragged small case
+    for (M, dm, dff, seed) in ((8, 4096, 14336, 0), (7, 2048, 5632, 2), (5, 264, 520, 3)):
         first = I.custom_inputs(M, dm, dff, seed)
         second = I.custom_inputs(M, dm, dff, seed + 100)
         Wg, Wu, Wd = first.Wg.to(dev), first.Wu.to(dev), first.Wd.to(dev)
@@ -45,9 +47,11 @@ def test_static_entry_matches_the_workspace_entry_on_two_calls_in_a_row():
             assert gmlp.device_status() == 0
             w, g = want.float().cpu().numpy().astype(np.float64), got.float().cpu().numpy().astype(np.float64)
             assert np.all(np.isfinite(g))
-            # the parity rule of the other GPU tests, taken around the existing entry point's output
+            # against the oracle (the weights are the first case's for both calls), by the rule of the other GPU tests
+            y_ref = oracle.gmlp_rows(inp.bits("X"), first.bits("Wg"), first.bits("Wu"), first.bits("Wd"))
+            assert np.all(np.abs(g - y_ref) <= oracle.tolerance(y_ref))
+            # and against the existing entry point: same kernels, same split - in fact bit-identical
             assert np.all(np.abs(g - w) <= 2e-2 * np.maximum(1.0, np.abs(w)))
-            # same kernels, same split: in fact bit-identical
             assert torch.equal(got.view(torch.int16), want.view(torch.int16))
     # a shape that is too large for the array is refused on the device as well, and nothing was written
     X = torch.zeros(gmlp.STATIC_MAX_M + 1, 64, dtype=torch.bfloat16, device=dev)
@@ -56,3 +60,22 @@ def test_static_entry_matches_the_workspace_entry_on_two_calls_in_a_row():
     with pytest.raises(gmlp.GmlpError) as ei:
         gmlp.forward_static(X, Wg, Wg, Wd, torch.empty_like(X))
     assert ei.value.status == gmlp.ERR_STATIC_LIMIT
+
+
+@pytest.mark.gpu
+def test_static_entry_leaves_the_free_device_memory_as_it_found_it():
+    """The point of the call: after one warm-up call per device (which loads the library's code and its built-in array)
+    further calls take nothing from the device.  Free memory as the driver reports it, before and after."""
+    dev = torch.device("cuda")
+    inp = I.custom_inputs(8, 4096, 14336, 0)
+    X, Wg, Wu, Wd = (t.to(dev) for t in (inp.X, inp.Wg, inp.Wu, inp.Wd))
+    Y = torch.empty_like(X)
+    gmlp.forward_static(X, Wg, Wu, Wd, Y)                # warm-up: first use on this device
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info(dev)
+    for _ in range(3):
+        gmlp.forward_static(X, Wg, Wu, Wd, Y)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info(dev)
+    assert free_after == free_before
+    assert gmlp.device_status() == 0
