@@ -698,6 +698,10 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     const int num_tiles = num_m * (int)((N + bn - 1) / bn);
     const int pairs = num_tiles < sms / 2 ? num_tiles : sms / 2;
     const bool chunked = chunk_kb > 0;
+    // Row tiles in groups of eight when there are two groups or more (70B prefill, 16 row tiles: 4.33 -> 4.22 ms;
+    // 2048 x 5632 at M = 8192: 0.441 -> 0.432 ms; on 8 row tiles groups of four cost 3 %)
+    int group_m = num_m >= 16 ? 8 : 0;
+    if (const char* e = getenv(GATEUP ? "GMLP_PAIR_GROUP_M_GU" : "GMLP_PAIR_GROUP_M_DOWN")) group_m = atoi(e);   // tuning override
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs));
     cfg.blockDim = dim3(chunked ? gmlp::kPairChunkThreads : gmlp::kUmmaThreads);
@@ -716,9 +720,10 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     const cudaError_t err = chunked
         ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false, false, false, true>, tmA, tmB0, tmB1, C, Mi, Ki, Ni,
                              num_m, num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm,
-                             yf32, chunk_kb)
+                             yf32, chunk_kb, group_m)
         : cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<GATEUP, false>, tmA, tmB0, tmB1, C, Mi, Ki, Ni, num_m,
-                             num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm, yf32, 0);
+                             num_tiles, (const float*)nullptr, act, (const bf16*)nullptr, (float*)nullptr, kNoMulti, wkm, yf32, 0,
+                             group_m);
     if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
     GMLP_CHECK_LAUNCH();
     return GMLP_OK;
@@ -1336,7 +1341,7 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         const float* rc_ptr = r;
         cudaError_t err = pair
-            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0, 0, 0)
+            ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0, 0, 0, 0)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, true>, tmA, tmB, tmB, Z, Mi, Ki, Ni, num_m, num_tiles, rc_ptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr, kNoMulti, 0, 0);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
         GMLP_CHECK_LAUNCH();
@@ -1432,7 +1437,7 @@ int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->N;
         cudaError_t err = pair
             ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
-                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq, kNoMulti, 0, 0, 0)
+                                 num_tiles, (const float*)nullptr, kSilu, R, sumsq, kNoMulti, 0, 0, 0, 0)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, true>, tmA, tmB, tmB, S, Mi, Ki, Ni, num_m,
                                  num_tiles, (const float*)nullptr, 128, kSilu, R, sumsq, kNoMulti, 0, 0);
         if (err != cudaSuccess) return GMLP_ERR_LAUNCH;
@@ -1542,7 +1547,7 @@ int qkv_proj_impl(const gmlp_qkv_args* a) {
         const int Mi = (int)a->M, Ki = (int)a->K, Ni = (int)a->Nq;
         cudaError_t err = pair
             ? cudaLaunchKernelEx(&cfg, gmlp::umma_pair_gemm_kernel<false, false, false, true>, tmA, tmB0, tmB1, Q, Mi, Ki, Ni,
-                                 num_m, num_tiles, (const float*)nullptr, kSilu, (const bf16*)nullptr, (float*)nullptr, multi, 0, 0, 0)
+                                 num_m, num_tiles, (const float*)nullptr, kSilu, (const bf16*)nullptr, (float*)nullptr, multi, 0, 0, 0, 0)
             : cudaLaunchKernelEx(&cfg, gmlp::umma_gemm_kernel<false, 4, false, false, true>, tmA, tmB0, tmB1, Q, Mi, Ki, Ni,
                                  num_m, num_tiles, (const float*)nullptr, 128, kSilu, (const bf16*)nullptr, (float*)nullptr,
                                  multi, 0, 0);

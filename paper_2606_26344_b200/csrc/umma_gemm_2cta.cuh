@@ -116,7 +116,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                       const __grid_constant__ CUtensorMap tmB1, bf16* __restrict__ C,
                       int M, int K, int N, int num_m_tiles, int num_tiles, const float* __restrict__ row_scale, GateAct act,
                       const bf16* residual, float* __restrict__ sumsq, const __grid_constant__ MultiB multi,
-                      int w_kmajor, int out_fp32, int chunk_kb)
+                      int w_kmajor, int out_fp32, int chunk_kb, int group_m)
 {
     static_assert(!(CHUNKED && (ROWSCALE || ADDSS || MULTI)), "chunked accumulation: the Gated MLP's two GEMMs only");
     static_assert(!(ROWSCALE && GATEUP), "row scaling is for the plain GEMM");
@@ -145,6 +145,18 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const uint32_t rank = ptx::cluster_ctarank();                 // 0 = leader
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     const int num_kb = (K + kUmmaBK - 1) / kUmmaBK;
+    // Order of the tiles: row tiles fastest, so that the pairs of one round work on few weight panels.  With
+    // 0 < group_m < num_m_tiles the row tiles are taken in groups of group_m: all column tiles of a group before the
+    // next group, so that the A rows of a group stay in L2 while the weights stream past (each weight panel is then
+    // read once per group instead of A once per round).
+    const int num_n_tiles = num_tiles / num_m_tiles;
+    auto tile_coords = [&](int tile, int& mt, int& nt) {
+        if (group_m <= 0 || group_m >= num_m_tiles) { mt = tile % num_m_tiles; nt = tile / num_m_tiles; return; }
+        const int per = group_m * num_n_tiles, g = tile / per, r = tile - g * per;
+        const int gs = num_m_tiles - g * group_m < group_m ? num_m_tiles - g * group_m : group_m;
+        mt = g * group_m + r % gs;
+        nt = r / gs;
+    };
 
     ptx::launch_dependents();
     if (threadIdx.x == 0) {
@@ -184,13 +196,15 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             uint32_t s = 0, ph = 0;                              // ring position of the next k-block
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-                const int m0 = (tile % num_m_tiles) * 256 + (int)rank * 128;
-                int n0 = (tile / num_m_tiles) * BN_OUT;
+                int mt, nt;
+                tile_coords(tile, mt, nt);
+                const int m0 = mt * 256 + (int)rank * 128;
+                int n0 = nt * BN_OUT;
                 // this CTA's half of the B columns: gate/up -> gate (rank 0) or up (rank 1) columns n0..n0+127
                 const CUtensorMap* bmap = (GATEUP && rank == 1) ? &tmB1 : &tmB0;
                 if (MULTI) {
                     int local;
-                    const int seg = multi_segment(multi, tile / num_m_tiles, &local);
+                    const int seg = multi_segment(multi, nt, &local);
                     n0 = local * BN_OUT;
                     bmap = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &multi.tmB2);
                 }
@@ -335,11 +349,13 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty0 + 8 * buf);
                 }
                 if (!ok) break;
-                const int m0 = (tile % num_m_tiles) * 256 + (int)rank * 128;
+                int mt, nt;
+                tile_coords(tile, mt, nt);
+                const int m0 = mt * 256 + (int)rank * 128;
                 const int row = m0 + q * 32 + lane;
                 if (row >= M) continue;
                 if (GATEUP) {
-                    const int col0 = (tile / num_m_tiles) * BN_OUT + hsel * 64;
+                    const int col0 = nt * BN_OUT + hsel * 64;
                     bf16* crow = C + (size_t)row * N + col0;
 #pragma unroll
                     for (int v = 0; v < 8; ++v) {
@@ -352,7 +368,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                         if (col0 + v * 8 < N) *reinterpret_cast<uint4*>(crow + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 } else {
-                    const int col0 = (tile / num_m_tiles) * BN_OUT + hsel * 128;
+                    const int col0 = nt * BN_OUT + hsel * 128;
                     if (out_fp32) {
                         float* frow = reinterpret_cast<float*>(C) + (size_t)row * N + col0;
 #pragma unroll
@@ -374,8 +390,10 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         int t = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++t) {
             const int buf = t & 1;
-            const int m0 = (tile % num_m_tiles) * 256 + (int)rank * 128;
-            int n0 = (tile / num_m_tiles) * BN_OUT;
+            int mt, nt;
+            tile_coords(tile, mt, nt);
+            const int m0 = mt * 256 + (int)rank * 128;
+            int n0 = nt * BN_OUT;
             const int row = m0 + q * 32 + lane;
             if (!__all_sync(0xFFFFFFFFu, wait_bounded(tfull0 + 8 * buf, ((uint32_t)t >> 1) & 1u, abort_flag, KERNEL_ID, 3))) break;
             ptx::tc_fence_after_sync();
@@ -384,7 +402,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             int Nseg = N;
             if (MULTI) {                                           // this tile's matrix: its output and width
                 int local;
-                const int seg = multi_segment(multi, tile / num_m_tiles, &local);
+                const int seg = multi_segment(multi, nt, &local);
                 n0 = local * BN_OUT;
                 if (seg == 1) { Cseg = multi.C1; Nseg = multi.N1; }
                 else if (seg == 2) { Cseg = multi.C2; Nseg = multi.N2; }
@@ -438,7 +456,7 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     }
                 }
             }
-            if (ADDSS && row < M) sumsq[(size_t)(tile / num_m_tiles) * M + row] = ss;
+            if (ADDSS && row < M) sumsq[(size_t)nt * M + row] = ss;
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty0 + 8 * buf);
