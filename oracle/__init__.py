@@ -151,11 +151,11 @@ def silu(values) -> np.ndarray:
     return out
 
 
-ACT_KINDS = {"silu": 0, "swish": 1, "glu": 2}
+ACT_KINDS = {"silu": 0, "swish": 1, "glu": 2, "gelu": 3}
 
 
 def gate_act(values, act: str = "silu", beta: float = 1.0) -> np.ndarray:
-    """The gate activation of the gated unit: silu g*sigmoid(g), swish g*sigmoid(beta*g), glu sigmoid(g)."""
+    """The gate activation of the gated unit: silu g*sigmoid(g), swish g*sigmoid(beta*g), glu sigmoid(g), gelu g*Phi(g)."""
     lib = _load()
     v = np.ascontiguousarray(values, dtype=np.float64)
     out = np.empty_like(v)

@@ -82,7 +82,9 @@ double gmlp_oracle_silu(double g)
  * Gate activation of the gated unit h = act(g) * u.  The paper's Gated MLP uses SiLU; its benchmark list
  * (Section 6.1) also names SwiGLU- and GLU-gated forms without defining them.  Reading taken (the
  * definitions of the GLU-variants literature): kind 0 SiLU g*sigmoid(g); kind 1 Swish-beta
- * g*sigmoid(beta*g) (beta = 1 is SiLU); kind 2 GLU sigmoid(g).  Anything else: NaN.
+ * g*sigmoid(beta*g) (beta = 1 is SiLU); kind 2 GLU sigmoid(g); kind 3 GELU g*Phi(g), Phi the standard normal
+ * distribution function (the exact form, not the tanh approximation), written g * erfc(-g / sqrt 2) / 2 so
+ * that the negative tail keeps its relative accuracy.  Anything else: NaN.
  */
 double gmlp_oracle_gate_act(double g, int kind, double beta)
 {
@@ -90,6 +92,7 @@ double gmlp_oracle_gate_act(double g, int kind, double beta)
         case 0: return gmlp_oracle_silu(g);
         case 1: return g / (1.0 + exp(-(beta * g)));
         case 2: return 1.0 / (1.0 + exp(-g));
+        case 3: return 0.5 * g * erfc(-g * 0.70710678118654752440);
         default: return NAN;
     }
 }

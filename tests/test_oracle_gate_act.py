@@ -104,3 +104,51 @@ def test_the_three_gates_differ_where_they_should():
     assert np.array_equal(oracle.gmlp_rows(X, Wg, Wu, Wd, act="swish", beta=1.0), y_silu)
     assert not np.allclose(oracle.gmlp_rows(X, Wg, Wu, Wd, act="swish", beta=2.0), y_silu, rtol=1e-3, atol=1e-3)
     assert not np.allclose(oracle.gmlp_rows(X, Wg, Wu, Wd, act="glu"), y_silu, rtol=1e-3, atol=1e-3)
+
+
+def test_gelu_closed_forms_identities_and_library_routines():
+    """GELU g * Phi(g), Phi the standard normal distribution function (the exact form)."""
+    gelu = lambda v: oracle.gate_act(np.asarray(v, dtype=np.float64), "gelu")
+    assert gelu([0.0])[0] == 0.0
+    # Phi(x) + Phi(-x) = 1  =>  gelu(x) - gelu(-x) = x
+    x = np.linspace(-12, 12, 4801)
+    assert np.allclose(gelu(x) - gelu(-x), x, rtol=0, atol=4e-16 * np.maximum(1.0, np.abs(x)))
+    # tabulated values of Phi: Phi(1) = 0.8413447460685429, Phi(-2) = 0.0227501319481792, Phi(3) = 0.9986501019683699
+    assert abs(gelu([1.0])[0] - 0.8413447460685429) < 2e-16
+    assert abs(gelu([-2.0])[0] + 2 * 0.0227501319481792) < 1e-16
+    assert abs(gelu([3.0])[0] - 3 * 0.9986501019683699) < 1e-15
+    # tails: gelu(x) -> x, gelu(-x) -> -0 with the relative accuracy of erfc kept (Phi(-10) = 7.619853024160527e-24)
+    assert gelu([40.0])[0] == 40.0 and gelu([-40.0])[0] == 0.0
+    assert abs(gelu([-10.0])[0] / (-10 * 7.619853024160527e-24) - 1.0) < 1e-13
+    # the one minimum: gelu'(x) = Phi(x) + x phi(x) = 0 at x* = -0.7517915...; there Phi(x*) = -x* phi(x*), so the
+    # minimum is -x*^2 phi(x*) with phi the normal density - an expression without erf
+    fine = np.linspace(-0.76, -0.74, 200001)
+    v = gelu(fine)
+    xs = fine[int(np.argmin(v))]
+    assert abs(xs + 0.751791524693564) < 2e-7
+    xstar = -0.751791524693564                      # (the grid point is within 1e-7 of it, and gelu is flat there)
+    assert abs(v.min() + xstar * xstar * math.exp(-xstar * xstar / 2.0) / math.sqrt(2.0 * math.pi)) < 1e-13
+    assert abs(v.min() + 0.1699712) < 1e-7
+    assert np.all(np.diff(gelu(np.linspace(-0.75, 12, 2000))) > 0) and np.all(np.diff(gelu(np.linspace(-12, -0.76, 2000))) < 0)
+    # library routines: math.erf / erfc and torch's gelu (exact form) in float64
+    pts = np.array([-6.5, -3.25, -1.0, -0.3, 0.002, 0.7, 2.5, 9.0])
+    want = np.array([0.5 * t * math.erfc(-t / math.sqrt(2.0)) for t in pts])
+    assert np.allclose(gelu(pts), want, rtol=1e-14, atol=0)
+    tg = torch.nn.functional.gelu(torch.tensor(x, dtype=torch.float64), approximate="none").numpy()
+    # (torch evaluates x (1 + erf(x / sqrt 2)) / 2, which is absolutely, not relatively, accurate in the negative tail)
+    assert np.all(np.abs(gelu(x) - tg) <= 1e-12 * np.abs(tg) + 2.3e-16 * np.maximum(1.0, np.abs(x)))
+    # and it is NOT the tanh approximation (which differs by up to 5e-4 around |x| = 2)
+    tt = torch.nn.functional.gelu(torch.tensor(x, dtype=torch.float64), approximate="tanh").numpy()
+    assert np.abs(gelu(x) - tt).max() > 1e-4
+
+
+def test_gelu_gated_operator_is_built_from_the_pinned_pieces():
+    X, Wg, Wu, Wd = _rand(5, 48, 80, 21)
+    y, H = oracle.gmlp_rows(X, Wg, Wu, Wd, want_h=True, act="gelu")
+    G = oracle.naive_matmul(oracle.bf16_to_double(X), oracle.bf16_to_double(Wg))
+    U = oracle.naive_matmul(oracle.bf16_to_double(X), oracle.bf16_to_double(Wu))
+    h = oracle.bf16_to_double(oracle.bf16_rn(oracle.gate_act(G, "gelu") * U))
+    assert np.array_equal(oracle.bf16_to_double(H), h)
+    assert np.array_equal(y, oracle.naive_matmul(h, oracle.bf16_to_double(Wd)))
+    # and differs from the SiLU-gated operator
+    assert np.abs(y - oracle.gmlp_rows(X, Wg, Wu, Wd)).max() > 1e-3
