@@ -72,9 +72,12 @@ enum {
      *   none             act(g) = g * sigmoid(g)              (SiLU)
      *   ACT_SWISH        act(g) = g * sigmoid(act_beta * g)   (Swish-beta; beta = 1 is SiLU bit for bit)
      *   ACT_GLU          act(g) = sigmoid(g)                  (GLU)
-     * Setting both is GMLP_ERR_FLAGS, and so is a NaN or infinite act_beta with ACT_SWISH. */
+     *   ACT_GELU         act(g) = g * Phi(g)                  (GELU gate; Phi the standard normal distribution function,
+     *                                                          the exact erf form, not the tanh approximation)
+     * Setting more than one is GMLP_ERR_FLAGS, and so is a NaN or infinite act_beta with ACT_SWISH. */
     GMLP_FLAG_ACT_SWISH = 1u << 5,
     GMLP_FLAG_ACT_GLU = 1u << 6,
+    GMLP_FLAG_ACT_GELU = 1u << 9,
     /* The three weight matrices are stored [out, in] (the layout of a linear layer's weight in the common
      * frameworks): Wg, Wu [d_ff, d_model], Wd [d_model, d_ff], row-major.  The operator is unchanged
      * (Y = (act(X Wg^T) (.) (X Wu^T)) Wd^T in that storage); the tensor-core kernels read such a matrix as a

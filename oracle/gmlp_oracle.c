@@ -141,7 +141,7 @@ int gmlp_oracle_rows_act(const uint16_t* X, const uint16_t* Wg, const uint16_t* 
         if (rows[i] < 0 || rows[i] >= M) return -1;
     int failed = 0;
 #ifdef _OPENMP
-    if (num_threads > 0) omp_set_num_threads(num_threads);
+    omp_set_num_threads(num_threads > 0 ? num_threads : omp_get_num_procs());   /* 0 = all cores, whatever an earlier call asked for */
 #else
     (void)num_threads;
 #endif
@@ -228,7 +228,7 @@ int gmlp_oracle_gate_up_rows_act(const uint16_t* X, const uint16_t* Wg, const ui
         if (rows[i] < 0 || rows[i] >= M) return -1;
     int failed = 0;
 #ifdef _OPENMP
-    if (num_threads > 0) omp_set_num_threads(num_threads);
+    omp_set_num_threads(num_threads > 0 ? num_threads : omp_get_num_procs());   /* 0 = all cores, whatever an earlier call asked for */
 #else
     (void)num_threads;
 #endif
@@ -291,7 +291,7 @@ int gmlp_oracle_rmsnorm_matmul_rows(const uint16_t* X, const uint16_t* W, const 
         if (rows[i] < 0 || rows[i] >= M) return -1;
     int failed = 0;
 #ifdef _OPENMP
-    if (num_threads > 0) omp_set_num_threads(num_threads);
+    omp_set_num_threads(num_threads > 0 ? num_threads : omp_get_num_procs());   /* 0 = all cores, whatever an earlier call asked for */
 #else
     (void)num_threads;
 #endif
@@ -352,7 +352,7 @@ int gmlp_oracle_matmul_add_rmsnorm_rows(const uint16_t* X, const uint16_t* W, co
         if (rows[i] < 0 || rows[i] >= M) return -1;
     int failed = 0;
 #ifdef _OPENMP
-    if (num_threads > 0) omp_set_num_threads(num_threads);
+    omp_set_num_threads(num_threads > 0 ? num_threads : omp_get_num_procs());   /* 0 = all cores, whatever an earlier call asked for */
 #else
     (void)num_threads;
 #endif
@@ -407,7 +407,7 @@ int gmlp_oracle_matmul_rows(const uint16_t* X, const uint16_t* W, int64_t M, int
     for (int64_t i = 0; i < n_rows; ++i)
         if (rows[i] < 0 || rows[i] >= M) return -1;
 #ifdef _OPENMP
-    if (num_threads > 0) omp_set_num_threads(num_threads);
+    omp_set_num_threads(num_threads > 0 ? num_threads : omp_get_num_procs());   /* 0 = all cores, whatever an earlier call asked for */
 #else
     (void)num_threads;
 #endif
@@ -450,7 +450,7 @@ int gmlp_oracle_gqa_rows(const uint16_t* Q, const uint16_t* K, const uint16_t* V
     const double scale = 1.0 / sqrt((double)D);
     int failed = 0;
 #ifdef _OPENMP
-    if (num_threads > 0) omp_set_num_threads(num_threads);
+    omp_set_num_threads(num_threads > 0 ? num_threads : omp_get_num_procs());   /* 0 = all cores, whatever an earlier call asked for */
 #else
     (void)num_threads;
 #endif

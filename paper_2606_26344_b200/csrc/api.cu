@@ -31,7 +31,7 @@ constexpr int kVersion = 100;
 constexpr int kMaxDevices = 64;
 constexpr int64_t kMaxDim = (int64_t)1 << 30;      // per-dimension limit (TMA coordinates are int32)
 constexpr uint32_t kKnownFlags = GMLP_FLAG_RMSNORM | GMLP_FLAG_CHECKED | GMLP_FLAG_ACT_SWISH | GMLP_FLAG_ACT_GLU |
-                                 GMLP_FLAG_WEIGHTS_OUT_IN | GMLP_FLAG_Y_FP32;
+                                 GMLP_FLAG_ACT_GELU | GMLP_FLAG_WEIGHTS_OUT_IN | GMLP_FLAG_Y_FP32;
 constexpr gmlp::GateAct kSilu = {1.0f, 0};
 // weights of the call in flight are stored [out, in] (set by the entry points around their launches)
 thread_local bool t_w_out_in = false;
@@ -54,14 +54,15 @@ const gmlp::MultiB kNoMulti = {};
 
 // Gate activation named by the flags (SiLU when none is set); false for a contradictory or non-finite request.
 bool gate_act_from(uint32_t flags, float beta, gmlp::GateAct* out) {
-    const bool swish = flags & GMLP_FLAG_ACT_SWISH, glu = flags & GMLP_FLAG_ACT_GLU;
-    if (swish && glu) return false;
+    const bool swish = flags & GMLP_FLAG_ACT_SWISH, glu = flags & GMLP_FLAG_ACT_GLU, gelu = flags & GMLP_FLAG_ACT_GELU;
+    if ((swish ? 1 : 0) + (glu ? 1 : 0) + (gelu ? 1 : 0) > 1) return false;
     *out = kSilu;
     if (swish) {
         if (!(beta == beta) || beta - beta != 0.0f) return false;      // NaN or infinite
         out->beta = beta;
     }
     if (glu) out->glu = 1;
+    if (gelu) out->glu = 2;
     return true;
 }
 

@@ -40,13 +40,18 @@ __device__ __forceinline__ float silu_f32(float g) {
 //   SiLU      act(g) = g * sigmoid(g)            beta = 1, glu = 0
 //   Swish     act(g) = g * sigmoid(beta * g)     beta free, glu = 0
 //   GLU       act(g) = sigmoid(g)                beta = 1, glu = 1
-// one expression, numerator g or 1 over 1 + e^(-beta g); with beta = 1, glu = 0 it is silu_f32 bit for bit.
+//   GELU      act(g) = g * Phi(g)                glu = 2   (Phi the standard normal distribution function: the exact
+//             form, g * erfc(-g / sqrt 2) / 2, not the tanh approximation, whose 5e-4 error would change the bf16 H
+//             rounds to far more often than anything else on the path)
+// the first three are one expression, numerator g or 1 over 1 + e^(-beta g); with beta = 1, glu = 0 it is silu_f32
+// bit for bit.  The choice is uniform over a launch.
 struct GateAct {
     float beta;
     int glu;
 };
 __device__ __forceinline__ float gate_act_f32(float g, const GateAct a) {
-    return __fdividef(a.glu ? 1.0f : g, 1.0f + __expf(-(a.beta * g)));
+    if (a.glu == 2) return 0.5f * g * erfcf(-0.70710678118654752f * g);
+    return __fdividef(a.glu == 1 ? 1.0f : g, 1.0f + __expf(-(a.beta * g)));
 }
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }

@@ -24,7 +24,8 @@ FLAG_ACT_SWISH = 1 << 5
 FLAG_ACT_GLU = 1 << 6
 FLAG_WEIGHTS_OUT_IN = 1 << 7
 FLAG_Y_FP32 = 1 << 8
-ACT_FLAGS = {"silu": 0, "swish": FLAG_ACT_SWISH, "glu": FLAG_ACT_GLU}
+FLAG_ACT_GELU = 1 << 9
+ACT_FLAGS = {"silu": 0, "swish": FLAG_ACT_SWISH, "glu": FLAG_ACT_GLU, "gelu": FLAG_ACT_GELU}
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA, VARIANT_SKINNY, VARIANT_PAIR, VARIANT_TENSOR = 0, 1, 2, 3, 4, 5, 6
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgmlp.so")

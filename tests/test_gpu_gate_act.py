@@ -1,4 +1,4 @@
-"""GPU parity of the gate-activation variants (Swish-beta, GLU) against the CPU oracle, every
+"""GPU parity of the gate-activation variants (Swish-beta, GLU, GELU) against the CPU oracle, every
 schedule, whole operator and gate/up half; and that beta = 1 reproduces the SiLU path bit for bit."""
 import numpy as np
 import pytest
@@ -28,7 +28,7 @@ def _run(inp, variant, act, beta, rmsnorm):
     return Y
 
 
-@pytest.mark.parametrize("act,beta", [("swish", 1.702), ("swish", 0.5), ("swish", -1.0), ("glu", 1.0)])
+@pytest.mark.parametrize("act,beta", [("swish", 1.702), ("swish", 0.5), ("swish", -1.0), ("glu", 1.0), ("gelu", 1.0)])
 @pytest.mark.parametrize("case", CASES)
 def test_whole_operator(case, act, beta):
     variant, M, dm, dff = case
@@ -53,7 +53,7 @@ def test_swish_with_beta_one_is_the_silu_path_bit_for_bit(case):
     assert torch.equal(a.view(torch.int16), b.view(torch.int16))
 
 
-@pytest.mark.parametrize("act,beta", [("swish", 1.702), ("glu", 1.0)])
+@pytest.mark.parametrize("act,beta", [("swish", 1.702), ("glu", 1.0), ("gelu", 1.0)])
 @pytest.mark.parametrize("variant,M", [(V.VARIANT_SKINNY, 8), (V.VARIANT_UMMA, 100), (V.VARIANT_PAIR, 260),
                                        (V.VARIANT_TENSOR, 300)])
 def test_gate_up_half_alone(variant, M, act, beta):
@@ -80,7 +80,7 @@ def test_gate_values_on_device_over_a_dense_sweep():
     X[:, 0] = 1                                          # so U = 1 everywhere
     dev = "cuda"
     xd = X.double().numpy()
-    for act, beta in (("swish", 1.702), ("swish", 0.25), ("glu", 1.0)):
+    for act, beta in (("swish", 1.702), ("swish", 0.25), ("glu", 1.0), ("gelu", 1.0)):
         Y = gmlp.forward(X.to(dev), eye.to(dev), ones_row.to(dev), eye.to(dev), variant=V.VARIANT_UMMA, checked=True,
                          act=act, beta=beta)
         want = oracle.bf16_to_double(oracle.bf16_rn(oracle.gate_act(xd, act, beta)))
