@@ -364,6 +364,24 @@ int gmlp_autotune_query(int64_t M, int64_t d_model, int64_t d_ff, int32_t* varia
                         int32_t* down_pair);
 void gmlp_autotune_clear(void);
 
+/*
+ * The tuned choices as a file (the scaled-down image of the paper's per-shape kernel cache, Section 6.5: a
+ * search result is kept and reused, not recomputed).  One text line per tuned shape, tab-separated:
+ *     gmlp-tune-v1  <library version>  <device name>  M  d_model  d_ff  variant  gate_up_pair  down_pair  gate_up_form  down_form
+ * Lines that start with '#' and empty lines are ignored.
+ * gmlp_autotune_save writes every choice the process holds (all devices) to `path`, through a temporary file that is
+ * renamed over it; returns the number of lines written or a negative status.
+ * gmlp_autotune_load reads `path` and keeps the lines whose library version is this library's and whose device name
+ * is `device_name` (NULL: the name of the current CUDA device), attached to the current device (device 0 when there is
+ * no CUDA device: loading and saving then still work, which is how the file format is tested on a machine without a
+ * GPU); malformed lines and lines with values no schedule has are skipped.  Returns the number of shapes taken, or
+ * GMLP_ERR_NULL / GMLP_ERR_LAUNCH (the file cannot be opened).  A shape loaded twice keeps the later line.
+ * With the environment variable GMLP_TUNE_CACHE set to a path, the file is loaded the first time the library touches a
+ * device and rewritten after every gmlp_autotune.
+ */
+int gmlp_autotune_save(const char* path);
+int gmlp_autotune_load(const char* path, const char* device_name);
+
 /* The schedule AUTO resolves to for this shape (GMLP_VARIANT_SKINNY or _TENSOR, or what gmlp_autotune kept). */
 int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);
 

@@ -7,7 +7,9 @@
 #include <cstdio>
 #include <cstdlib>
 #include <atomic>
+#include <cstring>
 #include <mutex>
+#include <string>
 #include <vector>
 #include <new>
 
@@ -143,6 +145,9 @@ EncodeTiledFn g_encode_tiled = nullptr;
 inline uint64_t align256(uint64_t v) { return (v + 255u) & ~(uint64_t)255u; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+int tune_cache_load(const char* path, const char* device_name);
+int tune_cache_save(const char* path);
+
 // Returns the state of the current device, probing it on first use; nullptr if there is none.
 DeviceState* current_device(int* status) {
     int dev = -1;
@@ -151,7 +156,8 @@ DeviceState* current_device(int* status) {
         *status = GMLP_ERR_ARCH;
         return nullptr;
     }
-    std::lock_guard<std::mutex> lock(g_mutex);
+    bool load_cache = false;                     // first touch of this device: read the tuned choices kept in a file
+    std::unique_lock<std::mutex> lock(g_mutex);
     DeviceState& d = g_dev[dev];
     if (!d.probed) {
         int major = 0, sms = 0;
@@ -164,6 +170,7 @@ DeviceState* current_device(int* status) {
         d.is_sm100 = (major == 10);
         d.sm_count = sms;
         d.probed = true;
+        load_cache = d.is_sm100;
     }
     if (!d.is_sm100) {
         *status = GMLP_ERR_ARCH;
@@ -180,6 +187,9 @@ DeviceState* current_device(int* status) {
         }
         g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
     }
+    lock.unlock();
+    if (load_cache)
+        if (const char* cache = getenv("GMLP_TUNE_CACHE")) (void)tune_cache_load(cache, nullptr);
     *status = GMLP_OK;
     return &d;
 }
@@ -358,15 +368,114 @@ struct Layout {
 // 128-row tcgen05 tiles win, because their down projection splits K over a cluster and reduces on chip (8B layer,
 // M = 32: 72 vs 67 us).  TENSOR then picks, per GEMM, between single-CTA tiles and CTA pairs.  gmlp_autotune
 // replaces this rule by a measurement for a given shape.
+int check_shape_values(int64_t M, int64_t d_model, int64_t d_ff);
+constexpr int kDownForms[6] = {0, 2, 3, 4, 12, 14};   // forms of the single-CTA down projection (see t_force_down_form)
 struct TunedShape {
     int device;
     int64_t M, d_model, d_ff;
     int variant;
     int gu_pair, down_pair;                      // TENSOR: kernel of each GEMM (1 = CTA pairs, 0 = single CTAs)
     int gu_nb, down_form;                        // single-CTA kernels: tile form (see t_force_gu_nb / t_force_down_form)
+    char device_name[64];                        // for the cache file: a choice belongs to the GPU model it was measured on
 };
 std::vector<TunedShape> g_tuned;                 // written by gmlp_autotune, under g_mutex
 std::atomic<int> g_tuned_count{0};               // lets untuned processes skip the lock
+
+// ---- the tuned choices as a text file (format: include/gmlp.h) ----
+void device_name_of(int device, char (&name)[64]) {
+    name[0] = 0;
+    cudaDeviceProp prop;
+    if (device >= 0 && cudaGetDeviceProperties(&prop, device) == cudaSuccess) {
+        snprintf(name, sizeof(name), "%s", prop.name);
+        for (char* c = name; *c; ++c)
+            if (*c == '\t' || *c == '\n') *c = ' ';
+    } else {
+        (void)cudaGetLastError();
+    }
+}
+
+bool tuned_values_valid(const TunedShape& t) {
+    if (t.M <= 0 || check_shape_values(t.M, t.d_model, t.d_ff) != GMLP_OK) return false;
+    if (t.variant != GMLP_VARIANT_SKINNY && t.variant != GMLP_VARIANT_TENSOR) return false;
+    if (t.gu_pair < -1 || t.gu_pair > 1 || t.down_pair < -1 || t.down_pair > 1) return false;
+    if (t.gu_nb != 0 && t.gu_nb != 2 && t.gu_nb != 4) return false;
+    bool form_ok = false;
+    for (int f : kDownForms) form_ok = form_ok || f == t.down_form;
+    return form_ok;
+}
+
+int tune_cache_save(const char* path) {
+    if (path == nullptr) return GMLP_ERR_NULL;
+    const std::string tmp = std::string(path) + ".tmp";
+    FILE* f = fopen(tmp.c_str(), "w");
+    if (f == nullptr) return GMLP_ERR_LAUNCH;
+    int n = 0;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        fprintf(f, "# libgmlp tuned schedule choices: version, device, M, d_model, d_ff, variant, gate_up_pair, down_pair, gate_up_form, down_form\n");
+        for (const TunedShape& t : g_tuned) {
+            fprintf(f, "gmlp-tune-v1\t%d\t%s\t%lld\t%lld\t%lld\t%d\t%d\t%d\t%d\t%d\n", kVersion, t.device_name, (long long)t.M,
+                    (long long)t.d_model, (long long)t.d_ff, t.variant, t.gu_pair, t.down_pair, t.gu_nb, t.down_form);
+            ++n;
+        }
+    }
+    if (fclose(f) != 0 || rename(tmp.c_str(), path) != 0) {
+        (void)remove(tmp.c_str());
+        return GMLP_ERR_LAUNCH;
+    }
+    return n;
+}
+
+int tune_cache_load(const char* path, const char* device_name) {
+    if (path == nullptr) return GMLP_ERR_NULL;
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0) { (void)cudaGetLastError(); device = 0; }
+    char own_name[64];
+    if (device_name == nullptr) {
+        device_name_of(device, own_name);
+        device_name = own_name;
+    }
+    FILE* f = fopen(path, "r");
+    if (f == nullptr) return GMLP_ERR_LAUNCH;
+    char line[512];
+    int taken = 0;
+    while (fgets(line, sizeof(line), f) != nullptr) {
+        if (line[0] == '#' || line[0] == '\n' || line[0] == 0) continue;
+        // tab-separated fields; the device name may contain spaces
+        char* field[11];
+        int nf = 0;
+        for (char* p = line; nf < 11; ++nf) {
+            field[nf] = p;
+            char* tab = strchr(p, '\t');
+            if (tab == nullptr) { ++nf; break; }
+            *tab = 0;
+            p = tab + 1;
+        }
+        if (nf != 11 || strcmp(field[0], "gmlp-tune-v1") != 0) continue;
+        if (char* nl = strchr(field[10], '\n')) *nl = 0;
+        char* end = nullptr;
+        long long v[10] = {};
+        bool ok = true;
+        for (int i = 1; i < 11 && ok; ++i) {
+            if (i == 2) continue;
+            v[i - 1] = strtoll(field[i], &end, 10);
+            ok = end != field[i] && *end == 0;
+        }
+        if (!ok || v[0] != kVersion || strcmp(field[2], device_name) != 0) continue;
+        TunedShape t = {device, v[2], v[3], v[4], (int)v[5], (int)v[6], (int)v[7], (int)v[8], (int)v[9], {0}};
+        snprintf(t.device_name, sizeof(t.device_name), "%s", device_name);
+        if (!tuned_values_valid(t)) continue;
+        std::lock_guard<std::mutex> lock(g_mutex);
+        bool found = false;
+        for (TunedShape& o : g_tuned)
+            if (o.device == device && o.M == t.M && o.d_model == t.d_model && o.d_ff == t.d_ff) { o = t; found = true; }
+        if (!found) g_tuned.push_back(t);
+        g_tuned_count.store((int)g_tuned.size(), std::memory_order_release);
+        ++taken;
+    }
+    fclose(f);
+    return taken;
+}
 
 bool tuned_lookup(int64_t M, int64_t d_model, int64_t d_ff, TunedShape* out) {
     if (g_tuned_count.load(std::memory_order_acquire) == 0) return false;
@@ -436,7 +545,6 @@ thread_local int t_force_gu = -1, t_force_down = -1;
 //   down:    2, 3, 4 = K split over a cluster of that many CTAs; 12 = 128-column tiles, 14 = 256-column tiles, no split.
 // Set by gmlp_autotune while it measures, and from its result around the launches of a tuned shape.
 thread_local int t_force_gu_nb = 0, t_force_down_form = 0;
-constexpr int kDownForms[6] = {0, 2, 3, 4, 12, 14};
 struct UmmaFormScope {
     int prev_gu, prev_down;
     UmmaFormScope(int gu_nb, int down_form) : prev_gu(t_force_gu_nb), prev_down(t_force_down_form) {
@@ -519,6 +627,7 @@ int check_shape(int64_t M, int64_t d_model, int64_t d_ff) {
     if (M > kMaxDim || d_model > kMaxDim || d_ff > kMaxDim) return GMLP_ERR_SHAPE;
     return GMLP_OK;
 }
+int check_shape_values(int64_t M, int64_t d_model, int64_t d_ff) { return check_shape(M, d_model, d_ff); }
 
 // ------------------------------------------------------------------ TMA descriptors
 // 2-D bf16 tensor, row-major [outer, inner]; box = box_outer rows x box_inner elements, 128-byte swizzle,
@@ -1774,9 +1883,14 @@ int autotune_impl(const gmlp_args* a, int iters, int32_t* best_variant, float* b
                 t.gu_nb = best_gu_nb; t.down_form = best_down_form;
                 found = true;
             }
-        if (!found) g_tuned.push_back({device, a->M, a->d_model, a->d_ff, w.variant, w.gu, w.down, best_gu_nb, best_down_form});
+        if (!found) {
+            TunedShape t = {device, a->M, a->d_model, a->d_ff, w.variant, w.gu, w.down, best_gu_nb, best_down_form, {0}};
+            device_name_of(device, t.device_name);
+            g_tuned.push_back(t);
+        }
         g_tuned_count.store((int)g_tuned.size(), std::memory_order_release);
     }
+    if (const char* cache = getenv("GMLP_TUNE_CACHE")) (void)tune_cache_save(cache);
     if (best_variant) *best_variant = w.variant;
     if (best_us) *best_us = best_ms * 1000.0f / (float)timed_calls;
     return GMLP_OK;
@@ -1866,6 +1980,22 @@ int gmlp_workspace_forget(const void* workspace, uint64_t bytes) {
         }
     }
     return GMLP_OK;
+}
+
+int gmlp_autotune_save(const char* path) {
+    try {
+        return tune_cache_save(path);
+    } catch (...) {
+        return GMLP_ERR_LAUNCH;
+    }
+}
+
+int gmlp_autotune_load(const char* path, const char* device_name) {
+    try {
+        return tune_cache_load(path, device_name);
+    } catch (...) {
+        return GMLP_ERR_LAUNCH;
+    }
 }
 
 void gmlp_autotune_clear(void) {

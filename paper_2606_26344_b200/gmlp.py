@@ -133,6 +133,10 @@ def lib() -> ctypes.CDLL:
         L.gmlp_autotune_query.argtypes = [i64, i64, i64] + [ctypes.POINTER(ctypes.c_int32)] * 3
         L.gmlp_autotune_clear.restype = None
         L.gmlp_autotune_clear.argtypes = []
+        L.gmlp_autotune_save.restype = ctypes.c_int
+        L.gmlp_autotune_save.argtypes = [ctypes.c_char_p]
+        L.gmlp_autotune_load.restype = ctypes.c_int
+        L.gmlp_autotune_load.argtypes = [ctypes.c_char_p, ctypes.c_char_p]
         L.gmlp_sum_partials.restype = ctypes.c_int
         L.gmlp_sum_partials.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int32, ctypes.c_void_p, ctypes.c_uint64,
                                         ctypes.c_void_p]
@@ -447,6 +451,23 @@ def autotune(args: GmlpArgs, iters: int = 20):
 
 def autotune_clear() -> None:
     lib().gmlp_autotune_clear()
+
+
+def autotune_save(path: str) -> int:
+    """gmlp_autotune_save: the tuned choices of this process as a text file; returns the number of shapes written."""
+    n = lib().gmlp_autotune_save(os.fsencode(path))
+    if n < 0:
+        raise GmlpError(n)
+    return n
+
+
+def autotune_load(path: str, device_name: Optional[str] = None) -> int:
+    """gmlp_autotune_load: takes the file's lines for this library version and `device_name` (default: the current
+    device's name); returns the number of shapes taken."""
+    n = lib().gmlp_autotune_load(os.fsencode(path), None if device_name is None else device_name.encode())
+    if n < 0:
+        raise GmlpError(n)
+    return n
 
 
 def autotune_query(M: int, d_model: int, d_ff: int):
