@@ -57,7 +57,8 @@ MIN_TIMED_S = 0.5                                            # steps timed per w
 # summarised under profiles/
 NCU_TRAFFIC_BYTES = {
     ("llama3-8b-decode-M8", "gate_up"): 235.0e6 + 4.5e6,
-    ("llama3-8b-prefill-M2048-rmsnorm", "gate_up"): 254.0e6 + 50.4e6,
+    ("llama3-8b-prefill-M2048-rmsnorm", "gate_up"): 256.8e6 + 52.6e6,
+    ("llama3-70b-prefill-M4096-outliers", "gate_up"): 3966.1e6 + 233.4e6,     # captured at full size (row tiles in groups of eight)
     ("llama3-8b-batch-M64", "gate_up"): 235.5e6 + 4.1e6,
 }
 
