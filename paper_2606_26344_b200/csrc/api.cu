@@ -386,7 +386,7 @@ void device_name_of(int device, char (&name)[64]) {
     name[0] = 0;
     cudaDeviceProp prop;
     if (device >= 0 && cudaGetDeviceProperties(&prop, device) == cudaSuccess) {
-        snprintf(name, sizeof(name), "%s", prop.name);
+        snprintf(name, sizeof(name), "%.63s", prop.name);
         for (char* c = name; *c; ++c)
             if (*c == '\t' || *c == '\n') *c = ' ';
     } else {
