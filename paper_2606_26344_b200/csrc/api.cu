@@ -498,10 +498,14 @@ int resolve_variant(int64_t M, int64_t d_model, int64_t d_ff, int32_t variant) {
     if (variant != GMLP_VARIANT_AUTO) return variant;
     const int tuned = tuned_variant(M, d_model, d_ff);
     if (tuned != GMLP_VARIANT_AUTO) return tuned;
-    if (M <= 16) return GMLP_VARIANT_SKINNY;
-    // up to 24 tokens the operand-swapped schedule still wins where both of its GEMMs split K over a cluster (layers
-    // with far fewer column tiles than SMs; 2048 x 5632 at 17 tokens: 23.9 against 32.1 us; level at 32)
-    if (M <= 24 && skinny_both_cluster(M, d_model, d_ff)) return GMLP_VARIANT_SKINNY;
+    // Measured, cold weights, us per step, operand-swapped / 128-row tiles:
+    //   2048 x 5632:   M = 8 18.9 / 29.4, 32 23.4 / 29.6, 64 24.7 / 30.1, 96 28.1 / 30.7, 128 37.2 / 31.3
+    //   4096 x 14336:  M = 8 59.3 / 70.1, 32 64.3 / 71.2, 64 63.4 / 72.0, 96 68.8 / 72.6, 128 74.2 / 73.8
+    //   8192 x 28672:  M = 8 212 / 232, 32 225 / 230, 48 237 / 231, 64 248 / 234, 128 258 / 243
+    // The operand-swapped schedule wins up to 32 tokens everywhere, and up to 96 where its gate/up GEMM has the cluster
+    // form (on the 70B layer it runs as stream-K, whose partial-sum traffic grows with M).
+    if (M <= 32) return GMLP_VARIANT_SKINNY;
+    if (M <= 96 && skinny_both_cluster(M, d_model, d_ff)) return GMLP_VARIANT_SKINNY;
     return GMLP_VARIANT_TENSOR;
 }
 
@@ -619,7 +623,7 @@ int current_sm_count() {
 }
 bool skinny_both_cluster(int64_t M, int64_t d_model, int64_t d_ff) {
     const int sms = current_sm_count();
-    return make_skinny_plan(M, d_model, d_ff, 2, sms).cluster >= 2 && make_skinny_plan(M, d_ff, d_model, 1, sms).cluster >= 2;
+    return make_skinny_plan(M, d_model, d_ff, 2, sms).cluster >= 1 && make_skinny_plan(M, d_ff, d_model, 1, sms).cluster >= 1;
 }
 
 int check_shape(int64_t M, int64_t d_model, int64_t d_ff) {

@@ -109,11 +109,12 @@ def test_workspace_sizes_and_variant_choice(lib):
     # with a per-GEMM kernel choice
     assert gmlp.pick_variant(1, 2048, 5632) == gmlp.VARIANT_SKINNY
     assert gmlp.pick_variant(16, 2048, 5632) == gmlp.VARIANT_SKINNY
-    # (up to 24 tokens on a layer whose two GEMMs both have the operand-swapped schedule's cluster form)
-    assert gmlp.pick_variant(17, 2048, 5632) == gmlp.VARIANT_SKINNY and gmlp.pick_variant(24, 2048, 5632) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(25, 2048, 5632) == gmlp.VARIANT_TENSOR and gmlp.pick_variant(17, 4096, 14336) == gmlp.VARIANT_TENSOR
+    # (up to 32 tokens everywhere; up to 96 on a layer whose two GEMMs both have the operand-swapped schedule's cluster form)
+    assert gmlp.pick_variant(32, 2048, 5632) == gmlp.VARIANT_SKINNY and gmlp.pick_variant(32, 8192, 28672) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(96, 2048, 5632) == gmlp.VARIANT_SKINNY and gmlp.pick_variant(96, 4096, 14336) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(33, 8192, 28672) == gmlp.VARIANT_TENSOR and gmlp.pick_variant(97, 4096, 14336) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(8, dm, dff) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(32, dm, dff) == gmlp.VARIANT_TENSOR
+    assert gmlp.pick_variant(128, dm, dff) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(129, 2048, 5632) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(2048, dm, dff) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(4096, 8192, 28672) == gmlp.VARIANT_TENSOR
