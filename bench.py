@@ -54,12 +54,13 @@ L2_BYTES = 126 * 1024 * 1024
 NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}       # dense bf16 peak and "about 8 TB/s": the stated targets' denominators
 MIN_TIMED_S = 0.5                                            # steps timed per workload, all regions together
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures
-# summarised under profiles/
+# summarised under profiles/ (skinny_cluster_gemm_decode_M8.md, umma_pair_gemm_chunked_prefill8b_M2048.md,
+# bench_prefill70b_launch_list.md; the M = 64 figure from the same two-counter capture as the decode one)
 NCU_TRAFFIC_BYTES = {
-    ("llama3-8b-decode-M8", "gate_up"): 235.0e6 + 4.5e6,
+    ("llama3-8b-decode-M8", "gate_up"): 235.0e6 + 3.2e6,
     ("llama3-8b-prefill-M2048-rmsnorm", "gate_up"): 256.8e6 + 52.6e6,
     ("llama3-70b-prefill-M4096-outliers", "gate_up"): 3966.1e6 + 233.4e6,     # captured at full size (row tiles in groups of eight)
-    ("llama3-8b-batch-M64", "gate_up"): 235.5e6 + 4.1e6,
+    ("llama3-8b-batch-M64", "gate_up"): 235.5e6 + 3.1e6,
 }
 
 
