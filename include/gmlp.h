@@ -99,7 +99,11 @@ enum {
     GMLP_VARIANT_SIMT = 1,   /* CUDA-core tiled GEMMs: any shape, slow; bring-up and cross-check */
     GMLP_VARIANT_STREAM = 2, /* small M: weight-streaming split-K kernels on CUDA cores (HBM-bound regime) */
     GMLP_VARIANT_UMMA = 3,   /* medium M: tcgen05 tensor-core GEMMs fed by TMA, accumulators in TMEM, one CTA per tile */
-    GMLP_VARIANT_SKINNY = 4, /* M <= 128: operand-swapped tcgen05 GEMMs, stream-K over all SMs (HBM-bound regime) */
+    GMLP_VARIANT_SKINNY = 4, /* few tokens (HBM-bound regime): operand-swapped tcgen05 GEMMs that stream the weights once; per
+                                GEMM either K split over a thread-block cluster per column tile and reduced on chip (layers
+                                with fewer column tiles than SMs; up to 256 tokens) or stream-K over all SMs with partial
+                                sums through the workspace (up to 128 tokens).  AUTO takes it up to 32 tokens, and up to
+                                96 where both GEMMs have the cluster form. */
     GMLP_VARIANT_PAIR = 5,   /* large M: the same GEMMs on CTA pairs (tcgen05 cta_group::2, 256-row tiles) */
     GMLP_VARIANT_TENSOR = 6  /* what AUTO takes outside SKINNY: each of the two GEMMs picks, by its number of
                                 128-row blocks, the CTA-pair kernel or the single-CTA kernel (whose down projection
@@ -345,7 +349,7 @@ int gmlp_workspace_forget(const void* workspace, uint64_t bytes);
  * Empirical schedule selection for one shape (the paper's extraction phase keeps, among the candidate kernels
  * its search produced, the one that measures fastest, Sections 3 and 6): runs args (a complete, valid
  * gmlp_forward_ex call; Y is overwritten with the correct result) with each tensor-core schedule that can run
- * the shape (SKINNY up to 128 rows, and TENSOR with each of the four combinations of single-CTA or CTA-pair
+ * the shape (SKINNY where it can run, and TENSOR with each of the four combinations of single-CTA or CTA-pair
  * kernel for the gate/up and for the down GEMM; those that do not fit a caller-supplied workspace are
  * skipped), about `iters` (1..10000) timed back-to-back calls each, in four interleaved rounds after a warm-up
  * round so that clock drift falls on all candidates alike, CUDA events on args->stream, and
