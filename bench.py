@@ -401,11 +401,14 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
             lanes.append({"stream": st_l, "Xh": inp.X.clone().pin_memory(), "Yh": torch.empty_like(inp.X).pin_memory(),
                           "keep": (Xs, Ys, ws_l),
                           "args": gmlp.make_args(Xs, Wg, Wu, Wd, Ys, gamma, w.eps, w.rmsnorm, gmlp.VARIANT_AUTO, ws_l, st_l)})
-        for i in range(6):
+        # the same regime as the resident number: an untimed pre-roll of the same host-buffer steps, then at least
+        # MIN_TIMED_S of them between the two events
+        n_e2e = max(4, steps, int(math.ceil(MIN_TIMED_S * 1e3 / max(ms, 1e-3))))
+        n_e2e = min(n_e2e, 20000)
+        for i in range(max(6, int(math.ceil(clock_roll * 1e3 / max(ms, 1e-3))))):
             ln = lanes[i % 2]
             gmlp.forward_host(ln["args"], ln["Xh"], ln["Yh"])
         barrier()
-        n_e2e = max(4, min(steps, 50))
         t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
         t0.record(stream)
         for ln in lanes:

@@ -386,6 +386,15 @@ void gmlp_autotune_clear(void);
 int gmlp_autotune_save(const char* path);
 int gmlp_autotune_load(const char* path, const char* device_name);
 
+/*
+ * How GMLP_VARIANT_SKINNY would run this shape on a device with `sm_count` SMs (0: the current device, 148 if there is
+ * none): for the gate/up GEMM in plan[0..2] and the down projection in plan[3..5], the CTAs per thread-block cluster
+ * that share a column tile (0: that GEMM runs as stream-K over all SMs, with partial sums through the workspace),
+ * the tile width in columns and the number of tiles.  Returns GMLP_OK, or GMLP_ERR_SHAPE / GMLP_ERR_NULL.
+ * Pure host arithmetic (the launch still asks the device whether the clusters fit one wave).
+ */
+int gmlp_small_m_plan(int64_t M, int64_t d_model, int64_t d_ff, int32_t sm_count, int32_t plan[6]);
+
 /* The schedule AUTO resolves to for this shape (GMLP_VARIANT_SKINNY or _TENSOR, or what gmlp_autotune kept). */
 int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);
 

@@ -2098,6 +2098,20 @@ uint64_t gmlp_workspace_bytes(int64_t M, int64_t d_model, int64_t d_ff, uint32_t
     return L.total > 256 ? L.total : 256;
 }
 
+int gmlp_small_m_plan(int64_t M, int64_t d_model, int64_t d_ff, int32_t sm_count, int32_t plan[6]) {
+    if (plan == nullptr) return GMLP_ERR_NULL;
+    if (check_shape(M, d_model, d_ff) != GMLP_OK || M < 1) return GMLP_ERR_SHAPE;
+    const int sms = sm_count > 0 ? sm_count : current_sm_count();
+    const SkinnyPlan a = make_skinny_plan(M, d_model, d_ff, 2, sms), b = make_skinny_plan(M, d_ff, d_model, 1, sms);
+    const SkinnyPlan* p[2] = {&a, &b};
+    for (int i = 0; i < 2; ++i) {
+        plan[3 * i] = p[i]->cluster;
+        plan[3 * i + 1] = p[i]->cluster >= 1 ? 64 * p[i]->c_boxes : 128 * p[i]->NH;
+        plan[3 * i + 2] = p[i]->cluster >= 1 ? p[i]->c_tiles : p[i]->num_tiles;
+    }
+    return GMLP_OK;
+}
+
 int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags) {
     (void)flags;
     if (check_shape(M, d_model, d_ff) != GMLP_OK) return GMLP_ERR_SHAPE;

@@ -180,6 +180,19 @@ def workspace_bytes(M: int, d_model: int, d_ff: int, flags: int = 0, variant: in
     return int(lib().gmlp_workspace_bytes(M, d_model, d_ff, flags, variant))
 
 
+def small_m_plan(M: int, d_model: int, d_ff: int, sm_count: int = 0):
+    """gmlp_small_m_plan: ((cluster, tile columns, tiles) of the gate/up GEMM, the same of the down projection) as
+    GMLP_VARIANT_SKINNY would run the shape; cluster 0 = stream-K."""
+    out = (ctypes.c_int32 * 6)()
+    L = lib()
+    L.gmlp_small_m_plan.restype = ctypes.c_int
+    L.gmlp_small_m_plan.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)]
+    rc = L.gmlp_small_m_plan(M, d_model, d_ff, sm_count, out)
+    if rc != OK:
+        raise GmlpError(rc)
+    return tuple(out[0:3]), tuple(out[3:6])
+
+
 def pick_variant(M: int, d_model: int, d_ff: int, flags: int = 0) -> int:
     return int(lib().gmlp_pick_variant(M, d_model, d_ff, flags))
 

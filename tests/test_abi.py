@@ -138,3 +138,26 @@ def test_header_is_plain_c(tmp_path):
     r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-fsyntax-only",
                         "-I", os.path.join(ROOT, "include"), str(src)], capture_output=True, text=True)
     assert r.returncode == 0, r.stderr
+
+
+def test_small_m_plan_per_gemm_form(lib):
+    """Host arithmetic of the operand-swapped schedule: which GEMMs split K over a cluster per column tile (and how), which
+    keep stream-K.  148 SMs (a B200 holds 74 / 45 / 33 / 26 / 22 / 15 / 15 clusters of 2 .. 8 CTAs at once)."""
+    plan = lambda *a: gmlp.small_m_plan(*a, 148)
+    # 2048 x 5632: gate/up 44 tiles x 3 CTAs (132 SMs); down 16 tiles x 6 (eight would need 16 clusters of 8: 15 fit)
+    assert plan(7, 2048, 5632) == ((3, 128, 44), (6, 128, 16))
+    # 8B: gate/up has 112 tiles, 76 % of the SMs with one CTA each (no reduction); down 32 tiles x 4
+    assert plan(8, 4096, 14336) == ((1, 128, 112), (4, 128, 32))
+    # 70B: 224 gate/up tiles exceed the SMs: stream-K; down 64 tiles x 2
+    gu, down = plan(8, 8192, 28672)
+    assert gu[0] == 0 and down == (2, 128, 64)
+    # every cluster plan fills at least 60 % of the SMs and fits one wave
+    capacity = {1: 148, 2: 74, 3: 45, 4: 33, 5: 26, 6: 22, 7: 15, 8: 15}
+    for (M, dm, dff) in ((1, 2048, 5632), (16, 1024, 4096), (24, 3072, 8192), (96, 4096, 11008), (5, 264, 520), (200, 2048, 5632)):
+        for c, cols, tiles in plan(M, dm, dff):
+            if c >= 1:
+                assert cols in (64, 128) and tiles * c <= 148 and tiles <= capacity[c]
+                assert tiles * c * 10 >= 148 * (6 if cols == 128 else 8)
+    # more than 128 tokens run only where both GEMMs have the cluster form; shapes are validated
+    assert lib.gmlp_small_m_plan(7, 60, 128, 148, (ctypes.c_int32 * 6)()) == gmlp.ERR_SHAPE
+    assert lib.gmlp_small_m_plan(7, 64, 128, 148, None) == gmlp.ERR_NULL
