@@ -366,6 +366,18 @@ def measure_workload(w, steps, warmup, dev, peaks, dist=None, want_e2e=True, sam
                                "traffic": NCU_TRAFFIC_BYTES.get((w.name, "gate_up")), "algorithmic_bytes": nbytes,
                                "peak_source": peaks["source"] + " (copy)"}
 
+    elif "fused" in kern_ms:
+        # the small-M schedule's one-kernel form: all three weight matrices stream through one kernel, which also writes
+        # the slices' partial Y (fp32); the sum over the slices is a second, tiny kernel
+        kms = kern_ms["fused"] * 1e-3
+        slices = (w.d_ff + 127) // 128
+        nbytes = 2 * (3 * w.d_model * w.d_ff + w.M * w.d_model) + 4 * slices * w.M * w.d_model
+        ach = nbytes / kms / 1e9
+        res["roofline"] = {"kernel": "fused", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                           "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "frac_nominal": ach / NOMINAL["hbm_gbs"],
+                           "traffic": NCU_TRAFFIC_BYTES.get((w.name, "fused")), "algorithmic_bytes": nbytes,
+                           "peak_source": peaks["source"] + " (copy)"}
+
     if "roofline" in res and not fits_l2 and res["roofline"]["bound"] == "hbm":
         # The same kernel in a chain of its own launches: programmatic dependent launch overlaps a launch's ramp with
         # its predecessor's tail, as it does inside the timed steps, so this is the kernel's rate in steady state

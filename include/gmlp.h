@@ -102,8 +102,10 @@ enum {
     GMLP_VARIANT_SKINNY = 4, /* few tokens (HBM-bound regime): operand-swapped tcgen05 GEMMs that stream the weights once; per
                                 GEMM either K split over a thread-block cluster per column tile and reduced on chip (layers
                                 with fewer column tiles than SMs; up to 256 tokens) or stream-K over all SMs with partial
-                                sums through the workspace (up to 128 tokens).  AUTO takes it up to 32 tokens, and up to
-                                96 where both GEMMs have the cluster form. */
+                                sums through the workspace (up to 128 tokens); on small layers with at most 16 tokens
+                                both GEMMs and the activation run in ONE kernel per 128-wide slice of d_ff (see
+                                gmlp_small_m_fused_plan).  AUTO takes it up to 32 tokens, and up to 96 where both GEMMs
+                                have the cluster form. */
     GMLP_VARIANT_PAIR = 5,   /* large M: the same GEMMs on CTA pairs (tcgen05 cta_group::2, 256-row tiles) */
     GMLP_VARIANT_TENSOR = 6  /* what AUTO takes outside SKINNY: each of the two GEMMs picks, by its number of
                                 128-row blocks, the CTA-pair kernel or the single-CTA kernel (whose down projection
@@ -395,6 +397,20 @@ int gmlp_autotune_load(const char* path, const char* device_name);
  */
 int gmlp_small_m_plan(int64_t M, int64_t d_model, int64_t d_ff, int32_t sm_count, int32_t plan[6]);
 
+/*
+ * The one-kernel ("fused") form of GMLP_VARIANT_SKINNY for this shape on a device with `sm_count` SMs (0: the current
+ * device, 148 if there is none).  In that form a thread-block cluster per 128-wide slice of d_ff computes its slice of
+ * H = act(X Wg) * (X Wu) on chip and multiplies it with its rows of W_down at once; the partial Y of the slices go
+ * through the workspace and a second, tiny kernel adds them in slice order.  plan[0] = CTAs per cluster (0: the form
+ * does not apply and the two kernels of gmlp_small_m_plan run), plan[1] = number of slices (= clusters), plan[2] =
+ * stages of the weight ring, plan[3] = TMEM columns per CTA, plan[4] = 1 if GMLP_VARIANT_SKINNY takes this form by
+ * default (small layers, where the hand-over between two kernels costs more than it; by measurement), else 0.
+ * The form needs at most 16 tokens, all clusters resident in one wave and the accumulators of gate, up
+ * and a CTA's share of the d_model / 128 partial-Y tiles in TMEM.  Returns GMLP_OK, or GMLP_ERR_SHAPE / GMLP_ERR_NULL.
+ * Pure host arithmetic.
+ */
+int gmlp_small_m_fused_plan(int64_t M, int64_t d_model, int64_t d_ff, int32_t sm_count, int32_t plan[5]);
+
 /* The schedule AUTO resolves to for this shape (GMLP_VARIANT_SKINNY or _TENSOR, or what gmlp_autotune kept). */
 int gmlp_pick_variant(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags);
 
@@ -425,7 +441,7 @@ void gmlp_reset_launch_count(void);
  * enqueued back to back.  gmlp_profile_read synchronises on those events and writes the
  * AVERAGE duration of each kernel over the recorded calls, in launch order, in milliseconds;
  * *count gets the number of kernels (at most max_count are written).
- * gmlp_profile_kernel_name(i) names the i-th kernel ("rmsnorm", "gate_up", "down").  An event
+ * gmlp_profile_kernel_name(i) names the i-th kernel ("rmsnorm", "gate_up", "down"; "fused", "sum" for the one-kernel small-M form).  An event
  * between two kernels keeps the second from overlapping the first's tail, so these are
  * stand-alone kernel durations; do not leave profiling on in a timed region.
  */

@@ -23,6 +23,7 @@
 #include "umma_gemm_splitk.cuh"
 #include "umma_skinny.cuh"
 #include "umma_skinny_cluster.cuh"
+#include "umma_skinny_fused.cuh"
 #include "gqa_attention.cuh"
 
 namespace {
@@ -126,6 +127,8 @@ struct DeviceState {
     bool rowscale_attr_set = false;
     bool skinny_attr_set = false;
     bool skinny_cluster_attr_set = false;
+    bool skinny_fused_attr_set = false;
+    int fused_capacity[9] = {};                  // the same for the fused small-M kernel
     int cluster_capacity[2][9] = {};             // clusters of C CTAs of the cluster-form kernels resident at once (0 = not asked yet)
     // arrival-counter regions zeroed by the library (the kernels leave them zero after every call); a few are
     // remembered so that callers alternating between workspaces (one per stream) do not pay a memset per call
@@ -353,12 +356,75 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
     return p;
 }
 
+// ------------------------------------------------------------------ fused small-M plan (umma_skinny_fused.cuh)
+// One cluster of C CTAs per 128-wide slice of d_ff; both GEMMs and the activation in one kernel, partial Y summed over
+// the slices through scratch by a second, tiny kernel.  Applicable when the slices x C fill at least 60 % of the SMs in
+// one wave, the accumulators fit TMEM - gate, up and this CTA's share of the d_model / 128
+// partial-Y tiles, each Mpad columns - and every CTA has two k-blocks or more.  cluster == 0: not applicable.
+struct FusedPlan {
+    int cluster, slices, Mpad, stages;
+    bool preferred;                             // faster than the two-kernel forms by measurement (see make_fused_plan)
+    uint32_t smem_bytes, tmem_cols, hbuf_off, staging_off, bars_off;
+    uint64_t scratch_bytes;
+};
+
+FusedPlan make_fused_plan(int64_t M, int64_t d_model, int64_t d_ff, int sm_count) {
+    FusedPlan p{};
+    if (M < 1 || M > gmlp::kFusedMaxTokens) return p;
+    const int sms = sm_count > 0 ? sm_count : 148;
+    p.Mpad = (int)((M + 15) / 16 * 16);
+    const int64_t S = (d_ff + 127) / 128, NT = (d_model + 127) / 128, KB = (d_model + 63) / 64;
+    if (S > sms) return p;
+    int forced = -1;
+    if (const char* e = getenv("GMLP_FUSED_CLUSTER")) forced = atoi(e);          // tuning override: that cluster size (0: none)
+    if (forced == 0) return p;
+    int best = 0;
+    for (int C = 1; C <= 8; ++C) {
+        if (forced > 0 && C != forced) continue;
+        if (S * C > sms || cluster_capacity_estimate(C, sms) < S) continue;
+        if (C > 1 && (KB / C < 2 || C > NT)) continue;
+        if ((2 + (NT + C - 1) / C) * p.Mpad > 512) continue;
+        best = C;                                                                 // the largest that fits: most SMs streaming
+    }
+    if (best == 0 || (forced <= 0 && S * best * 10 < (int64_t)sms * 6)) return p;
+    const uint32_t stage_bytes = gmlp::kFusedWeightBytes + (uint32_t)p.Mpad * 128u;
+    const uint32_t hbuf = 2u * (uint32_t)p.Mpad * 128u;
+    const uint32_t staging = gmlp::skinny_fused_staging_bytes(best, (int)M);
+    // all of the shared memory: a deep ring keeps W_down streaming through the exchange in the middle of the kernel, which
+    // is worth more than having the next kernel on the stream co-resident (2048 x 5632, M = 7: 18.8 against 22.6 us per step)
+    uint32_t budget = gmlp::kFusedSmemBudget;
+    if (const char* e = getenv("GMLP_FUSED_SMEM_KB")) { int v = atoi(e); if (v >= 48 && v <= 224) budget = (uint32_t)v * 1024u; }   // tuning override
+    const uint32_t fixed = 1024 + hbuf + staging + 256;
+    if (budget < fixed + 2 * stage_bytes) return p;
+    int st = (int)((budget - fixed) / stage_bytes);
+    if (st > gmlp::kSkinnyMaxStages) st = gmlp::kSkinnyMaxStages;
+    p.stages = st;
+    p.hbuf_off = (uint32_t)st * stage_bytes;
+    p.staging_off = p.hbuf_off + hbuf;
+    p.bars_off = p.staging_off + staging;
+    p.smem_bytes = p.bars_off + 256 + 1024;
+    uint32_t cols = (uint32_t)((2 + (NT + best - 1) / best) * p.Mpad), pow2 = 32;
+    while (pow2 < cols) pow2 <<= 1;
+    p.tmem_cols = pow2;
+    p.slices = (int)S;
+    p.cluster = best;
+    p.scratch_bytes = (uint64_t)S * (uint64_t)M * (uint64_t)d_model * 4u;
+    // Where it pays (B200, cold weights, steps back to back, us per step fused / two kernels): 1024 x 4096 10.1 / 14.7 (M = 1)
+    // to 12.2 / 17.7 (16); 2048 x 5632 16.5 / 18.4 (1), 18.0 / 18.9 (8), 20.9 / 21.3 (16); from about 80 MB of weights on the
+    // two forms are within 5 % of each other either way (1536 x 8960, 2048 x 8192, 2560 x 6912), and with more than six
+    // down-projection tiles per CTA, whose MMAs all come after the exchange, the fused form loses (4096 x 5632: 35.5 / 26.9;
+    // 3072 x 8192 at M = 8: 33.4 / 29.5).
+    p.preferred = 3 * d_model * d_ff * 2 <= (int64_t)72 << 20 && (NT + best - 1) / best <= 6;
+    return p;
+}
+
 // ------------------------------------------------------------------ workspace layout
 struct Layout {
     uint64_t xn_off, h_off, partial_off, counters_off, total;
     uint64_t counters_bytes;
     StreamPlan p1, p2;
     SkinnyPlan s1, s2;
+    FusedPlan sf;
 };
 
 // Schedule choice for AUTO, from A/B timings on B200.  SKINNY (operand-swapped stream-K) pays for up to 16
@@ -596,7 +662,10 @@ Layout make_layout(int64_t M, int64_t d_model, int64_t d_ff, uint32_t flags, int
     } else if (variant == GMLP_VARIANT_SKINNY) {
         L.s1 = make_skinny_plan(M, d_model, d_ff, 2, sm_count);
         L.s2 = make_skinny_plan(M, d_ff, d_model, 1, sm_count);
-        off += align256(L.s1.scratch_bytes > L.s2.scratch_bytes ? L.s1.scratch_bytes : L.s2.scratch_bytes);
+        L.sf = make_fused_plan(M, d_model, d_ff, sm_count);
+        uint64_t scratch = L.s1.scratch_bytes > L.s2.scratch_bytes ? L.s1.scratch_bytes : L.s2.scratch_bytes;
+        if (L.sf.cluster >= 1 && L.sf.scratch_bytes > scratch) scratch = L.sf.scratch_bytes;
+        off += align256(scratch);
         L.counters_off = off;
         L.counters_bytes = align256((uint64_t)(L.s1.num_tiles + L.s2.num_tiles) * 4);
         off += L.counters_bytes;
@@ -1081,6 +1150,78 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
     return GMLP_OK;
 }
 
+// The fused form of the small-M schedule (umma_skinny_fused.cuh): one launch for the whole layer.  Returns
+// GMLP_ERR_UNSUPPORTED when the device cannot hold all clusters at once (the caller then runs the two-kernel forms).
+int launch_skinny_fused(DeviceState* dev, const FusedPlan& p, const bf16* X, const bf16* Wg, const bf16* Wu, const bf16* Wd,
+                        float* scratch, bf16* Y, int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st, gmlp::GateAct act) {
+    if (!dev->skinny_fused_attr_set) {
+        if (cudaFuncSetAttribute(gmlp::skinny_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gmlp::kFusedSmemBudget) != cudaSuccess)
+            return GMLP_ERR_LAUNCH;
+        dev->skinny_fused_attr_set = true;
+    }
+    CUtensorMap tmX, tmWg, tmWu, tmWd;
+    if (!encode_2d(&tmX, X, (uint64_t)d_model, (uint64_t)M, 64, (uint32_t)p.Mpad)) return GMLP_ERR_LAUNCH;
+    if (!GMLP_ENCODE_W(&tmWg, Wg, d_ff, d_model)) return GMLP_ERR_LAUNCH;
+    if (!GMLP_ENCODE_W(&tmWu, Wu, d_ff, d_model)) return GMLP_ERR_LAUNCH;
+    if (!GMLP_ENCODE_W(&tmWd, Wd, d_model, d_ff)) return GMLP_ERR_LAUNCH;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.slices * p.cluster));
+    cfg.blockDim = dim3(gmlp::kSkinnyThreads);
+    cfg.dynamicSmemBytes = p.smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)p.cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    int& capacity = dev->fused_capacity[p.cluster];
+    if (capacity == 0) {
+        int n = 0;
+        cfg.numAttrs = 1;                                   // the occupancy query takes the cluster shape only
+        if (cudaOccupancyMaxActiveClusters(&n, gmlp::skinny_fused_kernel, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            n = -1;
+        }
+        cfg.numAttrs = 2;
+        capacity = n > 0 ? n : -1;
+        if (getenv("GMLP_TUNE_VERBOSE"))
+            fprintf(stderr, "gmlp: clusters of %d CTAs (fused small-M kernel, %u B shared memory) resident at once: %d\n", p.cluster, p.smem_bytes, n);
+    }
+    if (capacity < p.slices) return GMLP_ERR_UNSUPPORTED;
+    int evict_first = 1;
+    if (const char* e = getenv("GMLP_SKINNY_EVICT_FIRST")) evict_first = atoi(e);      // tuning override
+    if (cudaLaunchKernelEx(&cfg, gmlp::skinny_fused_kernel, tmX, tmWg, tmWu, tmWd, scratch, (int)M, p.Mpad, (int)d_model,
+                           p.stages, p.tmem_cols, evict_first, act, p.hbuf_off, p.staging_off, p.bars_off, t_w_out_in ? 1 : 0) != cudaSuccess)
+        return GMLP_ERR_LAUNCH;
+    GMLP_CHECK_LAUNCH();
+    prof_mark("fused", st);
+    // the sum over the slices: a programmatic dependent of the kernel above
+    cudaLaunchConfig_t sum = {};
+    const int64_t threads = M * (d_model / 4) * gmlp::kSumLanes;
+    sum.gridDim = dim3((unsigned)((threads + 255) / 256));
+    sum.blockDim = dim3(256);
+    sum.stream = st;
+    sum.attrs = attr + 1;
+    sum.numAttrs = 1;
+    if (cudaLaunchKernelEx(&sum, gmlp::sum_slices_kernel, (const float*)scratch, Y, (int)M, (int)d_model, p.slices, t_y_fp32 ? 1 : 0) != cudaSuccess)
+        return GMLP_ERR_LAUNCH;
+    GMLP_CHECK_LAUNCH();
+    prof_mark("sum", st);
+    return GMLP_OK;
+}
+
+// Whether the SKINNY schedule runs this layer as one fused kernel: where the plan applies and was measured to pay.
+// Tuning override GMLP_SKINNY_FUSED: 0 never, 1 wherever the plan applies.
+bool skinny_use_fused(const FusedPlan& f) {
+    if (f.cluster < 1) return false;
+    if (const char* e = getenv("GMLP_SKINNY_FUSED")) return atoi(e) != 0;
+    return f.preferred;
+}
+
 int run_skinny(DeviceState* dev, const Layout& L, uint8_t* ws, const bf16* A, const bf16* Wg, const bf16* Wu,
                const bf16* Wd, bf16* H, bf16* Y, int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st,
                gmlp::GateAct act) {
@@ -1089,6 +1230,10 @@ int run_skinny(DeviceState* dev, const Layout& L, uint8_t* ws, const bf16* A, co
     unsigned int* c2 = c1 + L.s1.num_tiles;
     int rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
     if (rc != GMLP_OK) return rc;
+    if (skinny_use_fused(L.sf)) {
+        rc = launch_skinny_fused(dev, L.sf, A, Wg, Wu, Wd, scratch, Y, M, d_model, d_ff, st, act);
+        if (rc != GMLP_ERR_UNSUPPORTED) return rc;          // clusters that do not fit one wave: the two-kernel forms below
+    }
     rc = launch_skinny<true>(dev, L.s1, A, Wg, Wu, scratch, c1, H, M, d_model, d_ff, st, act);
     if (rc != GMLP_OK) return rc;
     prof_mark("gate_up", st);
@@ -2109,6 +2254,18 @@ int gmlp_small_m_plan(int64_t M, int64_t d_model, int64_t d_ff, int32_t sm_count
         plan[3 * i + 1] = p[i]->cluster >= 1 ? 64 * p[i]->c_boxes : 128 * p[i]->NH;
         plan[3 * i + 2] = p[i]->cluster >= 1 ? p[i]->c_tiles : p[i]->num_tiles;
     }
+    return GMLP_OK;
+}
+
+int gmlp_small_m_fused_plan(int64_t M, int64_t d_model, int64_t d_ff, int32_t sm_count, int32_t plan[5]) {
+    if (plan == nullptr) return GMLP_ERR_NULL;
+    if (check_shape(M, d_model, d_ff) != GMLP_OK || M < 1) return GMLP_ERR_SHAPE;
+    const FusedPlan f = make_fused_plan(M, d_model, d_ff, sm_count > 0 ? sm_count : current_sm_count());
+    plan[0] = f.cluster;
+    plan[1] = f.cluster >= 1 ? f.slices : 0;
+    plan[2] = f.cluster >= 1 ? f.stages : 0;
+    plan[3] = f.cluster >= 1 ? (int32_t)f.tmem_cols : 0;
+    plan[4] = f.cluster >= 1 && f.preferred ? 1 : 0;
     return GMLP_OK;
 }
 

@@ -193,6 +193,19 @@ def small_m_plan(M: int, d_model: int, d_ff: int, sm_count: int = 0):
     return tuple(out[0:3]), tuple(out[3:6])
 
 
+def small_m_fused_plan(M: int, d_model: int, d_ff: int, sm_count: int = 0):
+    """gmlp_small_m_fused_plan: (CTAs per cluster, slices, ring stages, TMEM columns, taken by default) of the one-kernel
+    form of GMLP_VARIANT_SKINNY; cluster 0 = the form does not apply."""
+    out = (ctypes.c_int32 * 5)()
+    L = lib()
+    L.gmlp_small_m_fused_plan.restype = ctypes.c_int
+    L.gmlp_small_m_fused_plan.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)]
+    rc = L.gmlp_small_m_fused_plan(M, d_model, d_ff, sm_count, out)
+    if rc != OK:
+        raise GmlpError(rc)
+    return tuple(out[0:5])
+
+
 def pick_variant(M: int, d_model: int, d_ff: int, flags: int = 0) -> int:
     return int(lib().gmlp_pick_variant(M, d_model, d_ff, flags))
 

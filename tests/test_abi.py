@@ -161,3 +161,28 @@ def test_small_m_plan_per_gemm_form(lib):
     # more than 128 tokens run only where both GEMMs have the cluster form; shapes are validated
     assert lib.gmlp_small_m_plan(7, 60, 128, 148, (ctypes.c_int32 * 6)()) == gmlp.ERR_SHAPE
     assert lib.gmlp_small_m_plan(7, 64, 128, 148, None) == gmlp.ERR_NULL
+
+
+def test_small_m_fused_plan(lib):
+    """Host arithmetic of the one-kernel form of the operand-swapped schedule: one cluster per 128-wide slice of d_ff, the
+    largest cluster that fits one wave, TMEM for gate, up and a CTA's share of the partial-Y tiles."""
+    plan = lambda *a: gmlp.small_m_fused_plan(*a, 148)
+    # 2048 x 5632: 44 slices x 3 CTAs (132 SMs; four would need 176); (2 + ceil(16 / 3)) x 16 = 128 TMEM columns; the default
+    assert plan(7, 2048, 5632)[:2] == (3, 44) and plan(7, 2048, 5632)[3:] == (128, 1)
+    assert plan(1, 2048, 5632)[2] >= plan(16, 2048, 5632)[2] >= 4      # fewer tokens: smaller exchange area, more ring stages
+    # at most 16 tokens; 8B and 70B layers do not apply (the partial-Y tiles of a CTA would not fit TMEM / too many slices)
+    assert plan(17, 2048, 5632)[0] == 0 and plan(8, 4096, 14336)[0] == 0 and plan(8, 8192, 28672)[0] == 0
+    # applies but is not the default: more than 72 MB of weights, or more than six down tiles per CTA
+    assert plan(8, 1536, 8960)[0] == 2 and plan(8, 1536, 8960)[4] == 0
+    assert plan(8, 4096, 5632)[0] == 3 and plan(8, 4096, 5632)[4] == 0
+    assert plan(8, 1024, 4096) [:2] == (4, 32) and plan(8, 1024, 4096)[4] == 1
+    capacity = {1: 148, 2: 74, 3: 45, 4: 33, 5: 26, 6: 22, 7: 15, 8: 15}
+    for (M, dm, dff) in ((1, 2048, 5632), (16, 1024, 4096), (5, 3072, 8192), (8, 2560, 6912), (2, 1024, 16384), (16, 256, 512)):
+        c, slices, stages, cols, _ = plan(M, dm, dff)
+        if c >= 1:
+            assert slices == -(-dff // 128) and slices * c <= 148 and slices <= capacity[c] and slices * c * 10 >= 148 * 6
+            assert 2 <= stages <= 12 and cols in (32, 64, 128, 256, 512) and cols >= (2 + -(-(-(-dm // 128)) // c)) * 16
+    # the workspace holds the slices' partial Y
+    assert gmlp.workspace_bytes(7, 2048, 5632, 0, gmlp.VARIANT_SKINNY) >= 44 * 7 * 2048 * 4
+    assert lib.gmlp_small_m_fused_plan(7, 60, 128, 148, (ctypes.c_int32 * 5)()) == gmlp.ERR_SHAPE
+    assert lib.gmlp_small_m_fused_plan(7, 64, 128, 148, None) == gmlp.ERR_NULL
