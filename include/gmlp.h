@@ -104,8 +104,8 @@ enum {
                                 with fewer column tiles than SMs; up to 256 tokens) or stream-K over all SMs with partial
                                 sums through the workspace (up to 128 tokens); on small layers with at most 16 tokens
                                 both GEMMs and the activation run in ONE kernel per 128-wide slice of d_ff (see
-                                gmlp_small_m_fused_plan).  AUTO takes it up to 32 tokens, and up to 96 where both GEMMs
-                                have the cluster form. */
+                                gmlp_small_m_fused_plan).  AUTO takes it up to 32 tokens; where both GEMMs have the cluster
+                                form up to 96, and up to 200 on layers with d_model >= 3072. */
     GMLP_VARIANT_PAIR = 5,   /* large M: the same GEMMs on CTA pairs (tcgen05 cta_group::2, 256-row tiles) */
     GMLP_VARIANT_TENSOR = 6  /* what AUTO takes outside SKINNY: each of the two GEMMs picks, by its number of
                                 128-row blocks, the CTA-pair kernel or the single-CTA kernel (whose down projection

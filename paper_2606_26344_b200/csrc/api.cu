@@ -253,7 +253,9 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
     // programmatic stream serialization - is co-resident on every SM and has its weight ring full by the time
     // this one drains.  Both kernels then use 128-column tiles (more, smaller units balance better: measured
     // 1-17 % faster than 256-column tiles for the down projection on nine layer shapes).
-    const bool small = p.Mpad <= 32;
+    int small_max = 32;
+    if (const char* e = getenv("GMLP_SKINNY_SMALL_MPAD")) small_max = atoi(e);                      // tuning override
+    const bool small = p.Mpad <= small_max;
     p.NH = (N >= 256 && 2 * nmat * 2 * p.Mpad <= 512 && !small) ? 2 : 1;
     if (const char* e = getenv(nmat == 2 ? "GMLP_SKINNY_NH1" : "GMLP_SKINNY_NH2")) {      // tuning override
         if (e[0] == '1') p.NH = 1;
@@ -307,6 +309,12 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
         uint32_t c_cols = (uint32_t)(nmat * p.Mpad), c_pow2 = 32;
         while (c_pow2 < c_cols) c_pow2 <<= 1;
         p.c_tmem_cols = c_pow2;
+        // Half-size rings (co-residency with the next kernel, see above) in the cluster form: only with at most 16 tokens and a
+        // matrix of at most 28 MB.  A deep ring is worth more than the early start of the successor once the stream is long
+        // (us per step, half / full: 2048 x 5632 20.4 / 22.3 at M = 8, but 22.7 / 21.2 at M = 17; 2048 x 8192 25.2 / 23.7;
+        // 3072 x 8192 30.8 / 29.5; 8B layer 60.0 / 55.7; 5120 x 13824 71.8 / 66.0).
+        bool c_small = p.Mpad <= 16 && K * N * 2 <= (int64_t)28 << 20;
+        if (const char* e = getenv("GMLP_SKINNY_CLUSTER_SMALL")) { const int v = atoi(e); if (v == 0 || v == 1) c_small = v == 1; }   // tuning override
         int forced = -1;
         if (const char* e = getenv(nmat == 2 ? "GMLP_SKINNY_CLUSTER1" : "GMLP_SKINNY_CLUSTER2")) forced = atoi(e);   // tuning override: 0 = stream-K, 1..8 = that cluster size
         int forced_boxes = 0;
@@ -320,7 +328,7 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
             // (a 64-column tile's MMA reads one box length past its box: keep that inside the allocation)
             const uint32_t tail = 1024 + 256 + (boxes == 1 ? gmlp::kSkinnyBoxBytes : 0);
             // few tokens: half of the shared memory, so that the next kernel on the stream is co-resident (see above)
-            int cst = (int)(((small ? gmlp::kSkinnySmemBudget / 2 : gmlp::kSkinnySmemBudget) - tail) / c_stage_bytes);
+            int cst = (int)(((c_small ? gmlp::kSkinnySmemBudget / 2 : gmlp::kSkinnySmemBudget) - tail) / c_stage_bytes);
             if (cst > gmlp::kSkinnyMaxStages) cst = gmlp::kSkinnyMaxStages;
             if (tiles > sms || cst < 2) continue;
             int C = forced > 0 ? forced : sms / tiles;
@@ -342,7 +350,7 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
                 // partial sums of at most 24 KB get a region of their own behind the ring and its barriers (a stage less
                 // if need be): the senders then do not have to wait for the receiver's ring to be free
                 const uint32_t staging = gmlp::skinny_cluster_staging_bytes(C, nmat, (int)M);
-                const uint32_t limit = small ? gmlp::kSkinnySmemBudget / 2 : gmlp::kSkinnySmemBudget;
+                const uint32_t limit = c_small ? gmlp::kSkinnySmemBudget / 2 : gmlp::kSkinnySmemBudget;
                 p.c_staging_off = 0;
                 if (C > 1 && staging <= 24 * 1024) {
                     while (cst > 2 && (uint32_t)cst * c_stage_bytes + tail + staging > limit) --cst;
@@ -427,13 +435,11 @@ struct Layout {
     FusedPlan sf;
 };
 
-// Schedule choice for AUTO, from A/B timings on B200.  SKINNY (operand-swapped stream-K) pays for up to 16
-// tokens: on small and medium layers the one-CTA-per-tile kernels have too few tiles to fill the GPU (2048 x 5632,
-// M = 16: 26 vs 34 us), on large layers the two are within a few percent (8B layer, M = 16: 65.5 vs 66.2 us; 70B
-// layer: 219 vs 227 us).  Beyond that SKINNY's partial-sum traffic and last-arriver reduction grow with M and the
-// 128-row tcgen05 tiles win, because their down projection splits K over a cluster and reduces on chip (8B layer,
-// M = 32: 72 vs 67 us).  TENSOR then picks, per GEMM, between single-CTA tiles and CTA pairs.  gmlp_autotune
-// replaces this rule by a measurement for a given shape.
+// Schedule choice for AUTO, from A/B timings on B200 (resolve_variant below has the table).  The operand-swapped SKINNY
+// schedule streams every weight once with all SMs whatever the token count, where the 128-row tiles of TENSOR have too few
+// tiles to fill the GPU on small and medium layers; SKINNY's epilogue work and, in its stream-K form, its partial-sum
+// traffic grow with M, so TENSOR takes over from a token count that depends on the form.  TENSOR then picks, per GEMM,
+// between single-CTA tiles and CTA pairs.  gmlp_autotune replaces this rule by a measurement for a given shape.
 int check_shape_values(int64_t M, int64_t d_model, int64_t d_ff);
 constexpr int kDownForms[6] = {0, 2, 3, 4, 12, 14};   // forms of the single-CTA down projection (see t_force_down_form)
 struct TunedShape {
@@ -565,13 +571,18 @@ int resolve_variant(int64_t M, int64_t d_model, int64_t d_ff, int32_t variant) {
     const int tuned = tuned_variant(M, d_model, d_ff);
     if (tuned != GMLP_VARIANT_AUTO) return tuned;
     // Measured, cold weights, us per step, operand-swapped / 128-row tiles:
-    //   2048 x 5632:   M = 8 18.9 / 29.4, 32 23.4 / 29.6, 64 24.7 / 30.1, 96 28.1 / 30.7, 128 37.2 / 31.3
-    //   4096 x 14336:  M = 8 59.3 / 70.1, 32 64.3 / 71.2, 64 63.4 / 72.0, 96 68.8 / 72.6, 128 74.2 / 73.8
-    //   8192 x 28672:  M = 8 212 / 232, 32 225 / 230, 48 237 / 231, 64 248 / 234, 128 258 / 243
-    // The operand-swapped schedule wins up to 32 tokens everywhere, and up to 96 where its gate/up GEMM has the cluster
-    // form (on the 70B layer it runs as stream-K, whose partial-sum traffic grows with M).
+    //   2048 x 5632:   M = 33 21.5 / 28.8, 64 24.0 / 29.2, 96 28.2 / 29.8, 128 31.8 / 30.5, 160 33.9 / 30.9, 256 46.5 / 31.5
+    //   2048 x 8192:   M = 33 26.0 / 32.9, 96 29.9 / 33.9, 128 33.7 / 34.4, 160 36.2 / 34.6, 256 48.0 / 35.0
+    //   3072 x 8192:   M = 33 32.0 / 39.0, 128 39.7 / 40.8, 129 40.4 / 53.5, 200 49.0 / 53.7, 256 55.6 / 54.3
+    //   4096 x 14336:  M = 33 57.7 / 70.2, 128 66.1 / 72.1, 129 67.6 / 84.8, 200 81.2 / 87.7, 256 91.8 / 89.6
+    //   5120 x 13824:  M = 33 67.5 / 78.9, 128 78.2 / 81.9, 129 79.7 / 109.1, 200 96.1 / 112.1, 256 109.1 / 115.1
+    //   4096 x 11008:  M = 33 65.0 / 60.5, 64 79.3 / 61.2 (gate/up as stream-K: 86 tiles)
+    //   8192 x 28672:  M = 8 211 / 232, 33 230 / 229, 64 248 / 230, 128 257 / 240 (gate/up as stream-K)
+    // The operand-swapped schedule wins up to 32 tokens everywhere.  Where both of its GEMMs have the cluster form (no
+    // partial sums through global memory) it wins up to 96 tokens on the narrow layers and - because the 128-row tiles pay
+    // for a second row block from 129 tokens on - up to 200 on layers with d_model of 3072 or more.
     if (M <= 32) return GMLP_VARIANT_SKINNY;
-    if (M <= 96 && skinny_both_cluster(M, d_model, d_ff)) return GMLP_VARIANT_SKINNY;
+    if (M <= (d_model >= 3072 ? 200 : 96) && skinny_both_cluster(M, d_model, d_ff)) return GMLP_VARIANT_SKINNY;
     return GMLP_VARIANT_TENSOR;
 }
 

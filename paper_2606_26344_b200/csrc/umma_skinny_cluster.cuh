@@ -224,15 +224,39 @@ skinny_cluster_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid
                 if (p != rank && pnq > 0) {
                     const uint32_t slot = rank < p ? rank : rank - 1u;
                     const uint32_t remote = ptx::map_to_cta(base + staging_off, p) + (uint32_t)nl * 16u;
+                    // (eight, four or one quad per TMEM load: with many tokens a wait per quad was most of this loop)
 #pragma unroll
-                    for (int j = 0; j < NMAT; ++j)
-                        for (int quad = pq0; quad < pq1; ++quad) {
-                            uint32_t v[4];
-                            tmem_ld_32x4(taddr + (uint32_t)(j * Mpad + 4 * quad), v);
+                    for (int j = 0; j < NMAT; ++j) {
+                        const uint32_t dst = remote + (uint32_t)(((slot * NMAT + j) * pnq) * 128) * 16u;
+                        const uint32_t tcol = taddr + (uint32_t)(j * Mpad);
+                        int quad = pq0;
+                        for (; quad + 8 <= pq1; quad += 8) {
+                            uint32_t v[32];
+                            ptx::tmem_ld_32x32(tcol + (uint32_t)(4 * quad), v);
                             ptx::tmem_ld_wait();
-                            st_cluster_f32x4(remote + (uint32_t)(((slot * NMAT + j) * pnq + (quad - pq0)) * 128) * 16u,
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+                                st_cluster_f32x4(dst + (uint32_t)((quad - pq0 + k) * 128) * 16u, __uint_as_float(v[4 * k]), __uint_as_float(v[4 * k + 1]),
+                                                 __uint_as_float(v[4 * k + 2]), __uint_as_float(v[4 * k + 3]));
+                        }
+                        if (quad + 4 <= pq1) {
+                            uint32_t v[16];
+                            tmem_ld_32x16(tcol + (uint32_t)(4 * quad), v);
+                            ptx::tmem_ld_wait();
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                st_cluster_f32x4(dst + (uint32_t)((quad - pq0 + k) * 128) * 16u, __uint_as_float(v[4 * k]), __uint_as_float(v[4 * k + 1]),
+                                                 __uint_as_float(v[4 * k + 2]), __uint_as_float(v[4 * k + 3]));
+                            quad += 4;
+                        }
+                        for (; quad < pq1; ++quad) {
+                            uint32_t v[4];
+                            tmem_ld_32x4(tcol + (uint32_t)(4 * quad), v);
+                            ptx::tmem_ld_wait();
+                            st_cluster_f32x4(dst + (uint32_t)((quad - pq0) * 128) * 16u,
                                              __uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
                         }
+                    }
                 }
                 pq0 = pq1;
             }
@@ -246,38 +270,71 @@ skinny_cluster_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid
         ptx::grid_dependency_wait();                                  // `out` may still be read by the previous kernel
         const float4* stage = reinterpret_cast<const float4*>(base_ptr + staging_off);
         const int n = tile * TW + nl;
-        for (int quad = myq0; quad < myq1; ++quad) {
-            uint32_t g[4], uu[4];
-            tmem_ld_32x4(taddr + (uint32_t)(4 * quad), g);
-            if (GATEUP) tmem_ld_32x4(taddr + (uint32_t)(Mpad + 4 * quad), uu);
+        const bool gelu = act.glu == 2, glu = act.glu == 1;
+        const float beta = act.beta;
+        for (int q0 = myq0; q0 < myq1; q0 += 4) {                     // four quads (sixteen tokens) per round
+            const int nq = myq1 - q0 < 4 ? myq1 - q0 : 4;
+            uint32_t g[16], uu[16];
+            if (nq == 4) {
+                tmem_ld_32x16(taddr + (uint32_t)(4 * q0), g);
+                if (GATEUP) tmem_ld_32x16(taddr + (uint32_t)(Mpad + 4 * q0), uu);
+            } else {
+#pragma unroll
+                for (int k = 0; k < 3; ++k)
+                    if (k < nq) {
+                        tmem_ld_32x4(taddr + (uint32_t)(4 * (q0 + k)), *reinterpret_cast<uint32_t(*)[4]>(&g[4 * k]));
+                        if (GATEUP) tmem_ld_32x4(taddr + (uint32_t)(Mpad + 4 * (q0 + k)), *reinterpret_cast<uint32_t(*)[4]>(&uu[4 * k]));
+                    }
+            }
             ptx::tmem_ld_wait();
-            const float4 own_g = make_float4(__uint_as_float(g[0]), __uint_as_float(g[1]), __uint_as_float(g[2]), __uint_as_float(g[3]));
-            const float4 own_u = GATEUP ? make_float4(__uint_as_float(uu[0]), __uint_as_float(uu[1]), __uint_as_float(uu[2]), __uint_as_float(uu[3]))
-                                        : make_float4(0.f, 0.f, 0.f, 0.f);
-            float4 ga = make_float4(0.f, 0.f, 0.f, 0.f), ua = ga;
-            for (uint32_t r = 0; r < csize; ++r) {                    // fixed rank order, this CTA's own share in its place
-                float4 pg = own_g, pu = own_u;
+            // the C shares in rank order, this CTA's own in its place
+            float ga[16], ua[16];
+            for (uint32_t r = 0; r < csize; ++r) {
                 if (r != rank) {
                     const uint32_t slot = r < rank ? r : r - 1u;
-                    const size_t at = ((size_t)(slot * NMAT) * mynq + (quad - myq0)) * 128 + nl;
-                    pg = stage[at];
-                    if (GATEUP) pu = stage[at + (size_t)mynq * 128];
-                }
-                if (r == 0) { ga = pg; ua = pu; }
-                else {
-                    ga.x += pg.x; ga.y += pg.y; ga.z += pg.z; ga.w += pg.w;
-                    if (GATEUP) { ua.x += pu.x; ua.y += pu.y; ua.z += pu.z; ua.w += pu.w; }
+                    const float4* sg = stage + ((size_t)(slot * NMAT) * mynq + (q0 - myq0)) * 128 + nl;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (k < nq) {
+                            const float4 a = sg[(size_t)k * 128];
+                            const float4 b = GATEUP ? sg[((size_t)mynq + k) * 128] : make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (r == 0) {
+                                ga[4 * k] = a.x; ga[4 * k + 1] = a.y; ga[4 * k + 2] = a.z; ga[4 * k + 3] = a.w;
+                                ua[4 * k] = b.x; ua[4 * k + 1] = b.y; ua[4 * k + 2] = b.z; ua[4 * k + 3] = b.w;
+                            } else {
+                                ga[4 * k] += a.x; ga[4 * k + 1] += a.y; ga[4 * k + 2] += a.z; ga[4 * k + 3] += a.w;
+                                if (GATEUP) { ua[4 * k] += b.x; ua[4 * k + 1] += b.y; ua[4 * k + 2] += b.z; ua[4 * k + 3] += b.w; }
+                            }
+                        }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float og = __uint_as_float(g[i]), ou = GATEUP ? __uint_as_float(uu[i]) : 0.f;
+                        ga[i] = r == 0 ? og : ga[i] + og;
+                        ua[i] = r == 0 ? ou : ua[i] + ou;
+                    }
                 }
             }
-            const float gv[4] = {ga.x, ga.y, ga.z, ga.w}, uv[4] = {ua.x, ua.y, ua.z, ua.w};
+            // (the activation is chosen outside the loops: the GELU form is a call, and a possible call per element would
+            // keep the sixteen independent evaluations from overlapping)
+            float v[16];
+            if (!GATEUP) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = ga[i];
+            } else if (gelu) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = (i < 4 * nq) ? gelu_f32(ga[i]) * ua[i] : 0.f;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = __fdividef(glu ? 1.0f : ga[i], 1.0f + __expf(-(beta * ga[i]))) * ua[i];
+            }
             if (n < N) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int m = 4 * quad + i;
-                    if (m < M) {
-                        const float v = GATEUP ? gate_act_f32(gv[i], act) * uv[i] : gv[i];
-                        if (!GATEUP && out_fp32) reinterpret_cast<float*>(out)[(size_t)m * N + n] = v;
-                        else out[(size_t)m * N + n] = __float2bfloat16_rn(v);
+                for (int i = 0; i < 16; ++i) {
+                    const int m = 4 * q0 + i;
+                    if (i < 4 * nq && m < M) {
+                        if (!GATEUP && out_fp32) reinterpret_cast<float*>(out)[(size_t)m * N + n] = v[i];
+                        else out[(size_t)m * N + n] = __float2bfloat16_rn(v[i]);
                     }
                 }
             }

@@ -109,12 +109,14 @@ def test_workspace_sizes_and_variant_choice(lib):
     # with a per-GEMM kernel choice
     assert gmlp.pick_variant(1, 2048, 5632) == gmlp.VARIANT_SKINNY
     assert gmlp.pick_variant(16, 2048, 5632) == gmlp.VARIANT_SKINNY
-    # (up to 32 tokens everywhere; up to 96 on a layer whose two GEMMs both have the operand-swapped schedule's cluster form)
+    # (up to 32 tokens everywhere; on a layer whose two GEMMs both have the operand-swapped schedule's cluster form up to 96,
+    # and up to 200 where d_model >= 3072, because the 128-row tiles pay for a second row block from 129 tokens on)
     assert gmlp.pick_variant(32, 2048, 5632) == gmlp.VARIANT_SKINNY and gmlp.pick_variant(32, 8192, 28672) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(96, 2048, 5632) == gmlp.VARIANT_SKINNY and gmlp.pick_variant(96, 4096, 14336) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(33, 8192, 28672) == gmlp.VARIANT_TENSOR and gmlp.pick_variant(97, 4096, 14336) == gmlp.VARIANT_TENSOR
+    assert gmlp.pick_variant(96, 2048, 5632) == gmlp.VARIANT_SKINNY and gmlp.pick_variant(97, 2048, 5632) == gmlp.VARIANT_TENSOR
+    assert gmlp.pick_variant(33, 8192, 28672) == gmlp.VARIANT_TENSOR and gmlp.pick_variant(33, 4096, 11008) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(8, dm, dff) == gmlp.VARIANT_SKINNY
-    assert gmlp.pick_variant(128, dm, dff) == gmlp.VARIANT_TENSOR
+    assert gmlp.pick_variant(128, dm, dff) == gmlp.VARIANT_SKINNY and gmlp.pick_variant(200, dm, dff) == gmlp.VARIANT_SKINNY
+    assert gmlp.pick_variant(201, dm, dff) == gmlp.VARIANT_TENSOR and gmlp.pick_variant(129, 3072, 8192) == gmlp.VARIANT_SKINNY
     assert gmlp.pick_variant(129, 2048, 5632) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(2048, dm, dff) == gmlp.VARIANT_TENSOR
     assert gmlp.pick_variant(4096, 8192, 28672) == gmlp.VARIANT_TENSOR
