@@ -417,12 +417,13 @@ FusedPlan make_fused_plan(int64_t M, int64_t d_model, int64_t d_ff, int sm_count
     p.slices = (int)S;
     p.cluster = best;
     p.scratch_bytes = (uint64_t)S * (uint64_t)M * (uint64_t)d_model * 4u;
-    // Where it pays (B200, cold weights, steps back to back, us per step fused / two kernels): 1024 x 4096 10.1 / 14.7 (M = 1)
-    // to 12.2 / 17.7 (16); 2048 x 5632 16.5 / 18.4 (1), 18.0 / 18.9 (8), 20.9 / 21.3 (16); from about 80 MB of weights on the
-    // two forms are within 5 % of each other either way (1536 x 8960, 2048 x 8192, 2560 x 6912), and with more than six
-    // down-projection tiles per CTA, whose MMAs all come after the exchange, the fused form loses (4096 x 5632: 35.5 / 26.9;
-    // 3072 x 8192 at M = 8: 33.4 / 29.5).
-    p.preferred = 3 * d_model * d_ff * 2 <= (int64_t)72 << 20 && (NT + best - 1) / best <= 6;
+    // Where it pays (B200, cold weights, steps back to back, us per step fused / two kernels, M = 1 and M = 16):
+    // 1024 x 4096 10.0 / 15.5 and 12.5 / 18.5; 1536 x 6144 15.2 / 18.9 and 16.1 / 20.4; 2048 x 5632 16.4 / 18.6 and 20.7 / 21.7;
+    // 2048 x 6144 18.1 / 21.6 and 22.0 / 22.7; 1536 x 8960 19.8 / 22.2 and 22.8 / 23.3; from about 100 MB of weights on the
+    // two forms are within a few percent of each other either way (2048 x 8192 22.1 / 23.5 and 26.7 / 24.6; 2560 x 6912
+    // 22.9 / 23.8 and 27.8 / 25.2), and with more than six down-projection tiles per CTA, whose MMAs all come after the
+    // exchange, the fused form loses (4096 x 5632: 35.5 / 26.9; 3072 x 8192 at M = 8: 33.4 / 29.5).
+    p.preferred = 3 * d_model * d_ff * 2 <= (int64_t)90 << 20 && (NT + best - 1) / best <= 6;
     return p;
 }
 

@@ -272,20 +272,13 @@ skinny_cluster_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid
         const int n = tile * TW + nl;
         const bool gelu = act.glu == 2, glu = act.glu == 1;
         const float beta = act.beta;
-        for (int q0 = myq0; q0 < myq1; q0 += 4) {                     // four quads (sixteen tokens) per round
-            const int nq = myq1 - q0 < 4 ? myq1 - q0 : 4;
+        // Four quads (sixteen tokens) per round when this CTA has four or more; the last round then starts at the fourth quad
+        // from the end and repeats what the round before it has done of those (same values, same stores).
+        int q0 = myq0;
+        for (bool more = mynq >= 4; more; ) {
             uint32_t g[16], uu[16];
-            if (nq == 4) {
-                tmem_ld_32x16(taddr + (uint32_t)(4 * q0), g);
-                if (GATEUP) tmem_ld_32x16(taddr + (uint32_t)(Mpad + 4 * q0), uu);
-            } else {
-#pragma unroll
-                for (int k = 0; k < 3; ++k)
-                    if (k < nq) {
-                        tmem_ld_32x4(taddr + (uint32_t)(4 * (q0 + k)), *reinterpret_cast<uint32_t(*)[4]>(&g[4 * k]));
-                        if (GATEUP) tmem_ld_32x4(taddr + (uint32_t)(Mpad + 4 * (q0 + k)), *reinterpret_cast<uint32_t(*)[4]>(&uu[4 * k]));
-                    }
-            }
+            tmem_ld_32x16(taddr + (uint32_t)(4 * q0), g);
+            if (GATEUP) tmem_ld_32x16(taddr + (uint32_t)(Mpad + 4 * q0), uu);
             ptx::tmem_ld_wait();
             // the C shares in rank order, this CTA's own in its place
             float ga[16], ua[16];
@@ -294,18 +287,17 @@ skinny_cluster_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid
                     const uint32_t slot = r < rank ? r : r - 1u;
                     const float4* sg = stage + ((size_t)(slot * NMAT) * mynq + (q0 - myq0)) * 128 + nl;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (k < nq) {
-                            const float4 a = sg[(size_t)k * 128];
-                            const float4 b = GATEUP ? sg[((size_t)mynq + k) * 128] : make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (r == 0) {
-                                ga[4 * k] = a.x; ga[4 * k + 1] = a.y; ga[4 * k + 2] = a.z; ga[4 * k + 3] = a.w;
-                                ua[4 * k] = b.x; ua[4 * k + 1] = b.y; ua[4 * k + 2] = b.z; ua[4 * k + 3] = b.w;
-                            } else {
-                                ga[4 * k] += a.x; ga[4 * k + 1] += a.y; ga[4 * k + 2] += a.z; ga[4 * k + 3] += a.w;
-                                if (GATEUP) { ua[4 * k] += b.x; ua[4 * k + 1] += b.y; ua[4 * k + 2] += b.z; ua[4 * k + 3] += b.w; }
-                            }
+                    for (int k = 0; k < 4; ++k) {
+                        const float4 a = sg[(size_t)k * 128];
+                        const float4 b = GATEUP ? sg[((size_t)mynq + k) * 128] : make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (r == 0) {
+                            ga[4 * k] = a.x; ga[4 * k + 1] = a.y; ga[4 * k + 2] = a.z; ga[4 * k + 3] = a.w;
+                            ua[4 * k] = b.x; ua[4 * k + 1] = b.y; ua[4 * k + 2] = b.z; ua[4 * k + 3] = b.w;
+                        } else {
+                            ga[4 * k] += a.x; ga[4 * k + 1] += a.y; ga[4 * k + 2] += a.z; ga[4 * k + 3] += a.w;
+                            if (GATEUP) { ua[4 * k] += b.x; ua[4 * k + 1] += b.y; ua[4 * k + 2] += b.z; ua[4 * k + 3] += b.w; }
                         }
+                    }
                 } else {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
@@ -323,7 +315,7 @@ skinny_cluster_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid
                 for (int i = 0; i < 16; ++i) v[i] = ga[i];
             } else if (gelu) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] = (i < 4 * nq) ? gelu_f32(ga[i]) * ua[i] : 0.f;
+                for (int i = 0; i < 16; ++i) v[i] = gelu_f32(ga[i]) * ua[i];
             } else {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) v[i] = __fdividef(glu ? 1.0f : ga[i], 1.0f + __expf(-(beta * ga[i]))) * ua[i];
@@ -332,9 +324,47 @@ skinny_cluster_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const int m = 4 * q0 + i;
-                    if (i < 4 * nq && m < M) {
+                    if (m < M) {
                         if (!GATEUP && out_fp32) reinterpret_cast<float*>(out)[(size_t)m * N + n] = v[i];
                         else out[(size_t)m * N + n] = __float2bfloat16_rn(v[i]);
+                    }
+                }
+            }
+            more = q0 + 4 < myq1;
+            q0 = q0 + 8 <= myq1 ? q0 + 4 : myq1 - 4;
+        }
+        for (int quad = myq0; mynq < 4 && quad < myq1; ++quad) {      // fewer than four quads: one at a time
+            uint32_t g[4], uu[4];
+            tmem_ld_32x4(taddr + (uint32_t)(4 * quad), g);
+            if (GATEUP) tmem_ld_32x4(taddr + (uint32_t)(Mpad + 4 * quad), uu);
+            ptx::tmem_ld_wait();
+            const float4 own_g = make_float4(__uint_as_float(g[0]), __uint_as_float(g[1]), __uint_as_float(g[2]), __uint_as_float(g[3]));
+            const float4 own_u = GATEUP ? make_float4(__uint_as_float(uu[0]), __uint_as_float(uu[1]), __uint_as_float(uu[2]), __uint_as_float(uu[3]))
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+            float4 ga = make_float4(0.f, 0.f, 0.f, 0.f), ua = ga;
+            for (uint32_t r = 0; r < csize; ++r) {                    // fixed rank order, this CTA's own share in its place
+                float4 pg = own_g, pu = own_u;
+                if (r != rank) {
+                    const uint32_t slot = r < rank ? r : r - 1u;
+                    const size_t at = ((size_t)(slot * NMAT) * mynq + (quad - myq0)) * 128 + nl;
+                    pg = stage[at];
+                    if (GATEUP) pu = stage[at + (size_t)mynq * 128];
+                }
+                if (r == 0) { ga = pg; ua = pu; }
+                else {
+                    ga.x += pg.x; ga.y += pg.y; ga.z += pg.z; ga.w += pg.w;
+                    if (GATEUP) { ua.x += pu.x; ua.y += pu.y; ua.z += pu.z; ua.w += pu.w; }
+                }
+            }
+            const float gv[4] = {ga.x, ga.y, ga.z, ga.w}, uv[4] = {ua.x, ua.y, ua.z, ua.w};
+            if (n < N) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int m = 4 * quad + i;
+                    if (m < M) {
+                        const float v = GATEUP ? gate_act_f32(gv[i], act) * uv[i] : gv[i];
+                        if (!GATEUP && out_fp32) reinterpret_cast<float*>(out)[(size_t)m * N + n] = v;
+                        else out[(size_t)m * N + n] = __float2bfloat16_rn(v);
                     }
                 }
             }

@@ -174,8 +174,8 @@ def test_small_m_fused_plan(lib):
     assert plan(1, 2048, 5632)[2] >= plan(16, 2048, 5632)[2] >= 4      # fewer tokens: smaller exchange area, more ring stages
     # at most 16 tokens; 8B and 70B layers do not apply (the partial-Y tiles of a CTA would not fit TMEM / too many slices)
     assert plan(17, 2048, 5632)[0] == 0 and plan(8, 4096, 14336)[0] == 0 and plan(8, 8192, 28672)[0] == 0
-    # applies but is not the default: more than 72 MB of weights, or more than six down tiles per CTA
-    assert plan(8, 1536, 8960)[0] == 2 and plan(8, 1536, 8960)[4] == 0
+    # applies but is not the default: more than 90 MB of weights, or more than six down tiles per CTA
+    assert plan(8, 1536, 8960)[0] == 2 and plan(8, 1536, 8960)[4] == 1 and plan(8, 2048, 8192)[:2] == (2, 64) and plan(8, 2048, 8192)[4] == 0
     assert plan(8, 4096, 5632)[0] == 3 and plan(8, 4096, 5632)[4] == 0
     assert plan(8, 1024, 4096) [:2] == (4, 32) and plan(8, 1024, 4096)[4] == 1
     capacity = {1: 148, 2: 74, 3: 45, 4: 33, 5: 26, 6: 22, 7: 15, 8: 15}
