@@ -341,8 +341,13 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
             const int64_t ctas = (int64_t)tiles * C;
             // 128-column tiles read 256 contiguous bytes per weight row, 64-column tiles 128: the narrow rows use DRAM
             // so much worse (8B down projection, 128 CTAs either way: 34.8 against 26.9 us) that the wide tiles are
-            // taken from 60 % of the SMs on, the narrow ones only if they alone reach 80 %
-            if (ctas > best_ctas && (forced > 0 || ctas * 10 >= (int64_t)sms * (boxes == 2 ? 6 : 8))) {
+            // taken from a quarter of the SMs on, the narrow ones only if they alone reach 80 %.  (The cluster form beats
+            // stream-K, whose partial sums go through global memory, long before it fills the GPU: one SM pulls about 85 GB/s
+            // through a full-size ring, so 77 of them keep up with HBM, and on small layers the hand-over counts for more
+            // than the stream.  us per step, cluster form / stream-K for that GEMM: 4096 x 11008, 86 gate/up tiles with one
+            // CTA each 45.6 / 47.3 at M = 8, 46.4 / 54.7 at 24, 49.2 / 78.5 at 64; 4096 x 9600, 75 tiles 40.0 / 43.1,
+            // 41.5 / 49.8, 44.5 / 69.7; 1024 x 4096 down projection, 8 tiles x 8 CTAs 14.2 / 15.7, 14.7 / 19.9, 17.5 / 62.1.)
+            if (ctas > best_ctas && (forced > 0 || ctas * 100 >= (int64_t)sms * (boxes == 2 ? 25 : 80))) {
                 best_ctas = ctas;
                 p.cluster = C;
                 p.c_boxes = boxes;
