@@ -16,7 +16,11 @@ pytestmark = pytest.mark.gpu
 # (M, d_model, d_ff): clusters of 3 / 4 / 2 CTAs; a d_ff that ends inside a slice; a d_model that ends inside a k-block and
 # inside a down tile; one token; the largest token count the form takes
 SHAPES = [(7, 2048, 5632), (1, 2048, 5632), (16, 2048, 5632), (8, 1024, 4096), (5, 1536, 8960), (3, 2048, 5640),
-          (9, 2056, 5632), (4, 3072, 8192)]
+          (9, 2056, 5632), (4, 3072, 8192),
+          # drawn at random (multiples of 8) and kept for the cluster sizes they give: 8, 1, 6, 5, 4, 1 with the largest token
+          # count, 6 with one token, 3 with twelve partial-Y tiles per CTA, 8 again with every dimension ragged
+          (14, 1648, 1464), (6, 288, 11896), (7, 1104, 2296), (5, 2976, 2976), (9, 1768, 4192), (16, 272, 11792),
+          (1, 2808, 2032), (12, 2512, 4320), (9, 2864, 1600)]
 
 
 def _kernels_of(call):
