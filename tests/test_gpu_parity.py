@@ -83,10 +83,16 @@ def test_tensor_schedule_per_gemm_kernel_choice(shape, rmsnorm):
     check_case(I.custom_inputs(M, dm, dff, 700 + M, rmsnorm=rmsnorm, eps=1e-5), TENSOR, f"tensor{shape}")
 
 
-def test_small_m_path_is_stable_over_many_back_to_back_calls():
+@pytest.mark.parametrize("form", ["fused", "cluster", "stream-k"])
+def test_small_m_path_is_stable_over_many_back_to_back_calls(form, monkeypatch):
     # Decode-shaped calls issued back to back, alternating two inputs.  Every call must reproduce its own
     # first result bit for bit: this would expose a phase-2 read of an H tile that is not final yet, stale
-    # split-K partials, or arrival counters that were not left clean for the next call.
+    # split-K partials (or partial Y of the previous call in the one-kernel form), or arrival counters that were
+    # not left clean for the next call.  Each of the three forms of the schedule on the same layer.
+    monkeypatch.setenv("GMLP_SKINNY_FUSED", "1" if form == "fused" else "0")
+    if form == "stream-k":
+        monkeypatch.setenv("GMLP_SKINNY_CLUSTER1", "0")
+        monkeypatch.setenv("GMLP_SKINNY_CLUSTER2", "0")
     dev = torch.device("cuda")
     a = I.custom_inputs(8, 2048, 5632, 11)
     b = I.custom_inputs(8, 2048, 5632, 12)
@@ -108,11 +114,16 @@ def test_small_m_path_is_stable_over_many_back_to_back_calls():
 
 @pytest.mark.parametrize("rmsnorm", [False, True])
 @pytest.mark.parametrize("shape", [(1, 2048, 5632), (7, 2048, 5632), (16, 2048, 5632), (24, 2048, 5632), (129, 2048, 5632),
-                                   (250, 2048, 5632), (5, 2040, 5624), (8, 4096, 14336), (3, 8192, 8192), (13, 1024, 9000)])
-def test_skinny_schedule_cluster_form(shape, rmsnorm):
+                                   (250, 2048, 5632), (5, 2040, 5624), (8, 4096, 14336), (3, 8192, 8192), (13, 1024, 9000),
+                                   # from a random draw: the largest token count; clusters of 8 and 4 with a rounded-down
+                                   # share of sixteen-token rounds; 6 and 6; one CTA per tile with a cluster of 8 behind it
+                                   (256, 2088, 11464), (65, 3552, 1072), (127, 2312, 2576), (150, 864, 9960), (255, 904, 9640)])
+def test_skinny_schedule_cluster_form(shape, rmsnorm, monkeypatch):
     """Layers with fewer column tiles than SMs: a cluster of CTAs per tile splits K and reduce-scatters the partial sums in
     distributed shared memory (128-column tiles x 3 CTAs and 64-column tiles x 4 CTAs on the 2048 x 5632 layer; more than
-    128 tokens run in this form only).  Ragged widths put the tile and k-block tails in play."""
+    128 tokens run in this form only).  Ragged widths put the tile and k-block tails in play.  (The one-kernel form, which
+    would take the first shapes by default and has its own tests, is switched off here.)"""
+    monkeypatch.setenv("GMLP_SKINNY_FUSED", "0")
     M, dm, dff = shape
     inp = I.custom_inputs(M, dm, dff, seed=M + dm, rmsnorm=rmsnorm, eps=1e-6)
     check_case(inp, SKINNY, f"skinny-cluster {shape} norm={rmsnorm}")
