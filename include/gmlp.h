@@ -359,7 +359,10 @@ int gmlp_workspace_forget(const void* workspace, uint64_t bytes);
  * gmlp_workspace_bytes use it from then on (size workspaces after tuning).  When a single-CTA kernel is part of
  * the winner, a second stage measures its tile forms the same way (gate/up: 64- or 128-column tiles; down: K split
  * over a cluster of 2, 3 or 4 CTAs, or 128- or 256-column tiles without a split) and keeps a form that beats the
- * library's own rule by more than 1 %.  Synchronises the stream.
+ * library's own rule by more than 1 %.  When SKINNY wins, the second stage measures ITS forms instead: the one-kernel
+ * form against the two-kernel forms where gmlp_small_m_fused_plan applies, and, up to 32 tokens, half-size against
+ * full-size weight rings (a half-size ring lets the next kernel on the stream become resident early, a full-size one
+ * keeps more of the weight stream in flight), again keeping what beats the rule by more than 1 %.  Synchronises the stream.
  * best_variant (GMLP_VARIANT_SKINNY or _TENSOR) / best_us (microseconds per call) may be NULL.
  * gmlp_autotune_query returns 1 and the kept choice if the shape was tuned on the current device (gate_up_pair /
  * down_pair: 1 = CTA pairs, 0 = single CTAs, -1 = not applicable), else 0.  gmlp_autotune_clear forgets every
@@ -374,6 +377,8 @@ void gmlp_autotune_clear(void);
  * The tuned choices as a file (the scaled-down image of the paper's per-shape kernel cache, Section 6.5: a
  * search result is kept and reused, not recomputed).  One text line per tuned shape, tab-separated:
  *     gmlp-tune-v1  <library version>  <device name>  M  d_model  d_ff  variant  gate_up_pair  down_pair  gate_up_form  down_form
+ * (gate_up_form / down_form, TENSOR: tile form of the single-CTA kernels, 0 = by rule; SKINNY: gate_up_form = one-kernel
+ * form 0 by rule / 1 on / 2 off, down_form = weight rings 0 by rule / 1 half-size / 2 full-size.)
  * Lines that start with '#' and empty lines are ignored.
  * gmlp_autotune_save writes every choice the process holds (all devices) to `path`, through a temporary file that is
  * renamed over it; returns the number of lines written or a negative status.

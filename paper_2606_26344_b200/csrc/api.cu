@@ -234,6 +234,11 @@ int cluster_capacity_estimate(int C, int sms) {
     return C == 1 ? sms : (sms / C) * 85 / 100;
 }
 
+// Forms of the SKINNY schedule for a shape, as gmlp_autotune measured them or as it is forcing them right now
+// (0 = by the built-in rule): *fused 1 = the one-kernel form wherever its plan applies, 2 = two kernels; *ring
+// 1 = half-size weight rings (up to 32 tokens), 2 = full-size rings.  Defined with the tuned choices below.
+void skinny_forms(int64_t M, int64_t d_model, int64_t d_ff, int* fused, int* ring);
+
 // ------------------------------------------------------------------ skinny (swap-AB tcgen05) plan
 struct SkinnyPlan {
     int Mpad, NH, num_tiles, KB, stages, grid;
@@ -255,7 +260,11 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
     // 1-17 % faster than 256-column tiles for the down projection on nine layer shapes).
     int small_max = 32;
     if (const char* e = getenv("GMLP_SKINNY_SMALL_MPAD")) small_max = atoi(e);                      // tuning override
-    const bool small = p.Mpad <= small_max;
+    int tuned_fused = 0, tuned_ring = 0;         // what gmlp_autotune found for this layer, if it ran
+    skinny_forms(M, nmat == 2 ? K : N, nmat == 2 ? N : K, &tuned_fused, &tuned_ring);
+    (void)tuned_fused;
+    if (p.Mpad > 32 && tuned_ring == 1) tuned_ring = 0;          // half-size rings exist for up to 32 tokens only
+    const bool small = tuned_ring == 0 ? p.Mpad <= small_max : tuned_ring == 1;
     p.NH = (N >= 256 && 2 * nmat * 2 * p.Mpad <= 512 && !small) ? 2 : 1;
     if (const char* e = getenv(nmat == 2 ? "GMLP_SKINNY_NH1" : "GMLP_SKINNY_NH2")) {      // tuning override
         if (e[0] == '1') p.NH = 1;
@@ -314,6 +323,7 @@ SkinnyPlan make_skinny_plan(int64_t M, int64_t K, int64_t N, int nmat, int sm_co
         // (us per step, half / full: 2048 x 5632 20.4 / 22.3 at M = 8, but 22.7 / 21.2 at M = 17; 2048 x 8192 25.2 / 23.7;
         // 3072 x 8192 30.8 / 29.5; 8B layer 60.0 / 55.7; 5120 x 13824 71.8 / 66.0).
         bool c_small = p.Mpad <= 16 && K * N * 2 <= (int64_t)28 << 20;
+        if (tuned_ring != 0) c_small = tuned_ring == 1;
         if (const char* e = getenv("GMLP_SKINNY_CLUSTER_SMALL")) { const int v = atoi(e); if (v == 0 || v == 1) c_small = v == 1; }   // tuning override
         int forced = -1;
         if (const char* e = getenv(nmat == 2 ? "GMLP_SKINNY_CLUSTER1" : "GMLP_SKINNY_CLUSTER2")) forced = atoi(e);   // tuning override: 0 = stream-K, 1..8 = that cluster size
@@ -476,6 +486,9 @@ bool tuned_values_valid(const TunedShape& t) {
     if (t.M <= 0 || check_shape_values(t.M, t.d_model, t.d_ff) != GMLP_OK) return false;
     if (t.variant != GMLP_VARIANT_SKINNY && t.variant != GMLP_VARIANT_TENSOR) return false;
     if (t.gu_pair < -1 || t.gu_pair > 1 || t.down_pair < -1 || t.down_pair > 1) return false;
+    // (a SKINNY choice keeps its own two forms in the same fields: gu_nb = one-kernel form 0 rule / 1 on / 2 off, down_form =
+    // ring size 0 rule / 1 half / 2 full)
+    if (t.variant == GMLP_VARIANT_SKINNY) return t.gu_nb >= 0 && t.gu_nb <= 2 && t.down_form >= 0 && t.down_form <= 2;
     if (t.gu_nb != 0 && t.gu_nb != 2 && t.gu_nb != 4) return false;
     bool form_ok = false;
     for (int f : kDownForms) form_ok = form_ok || f == t.down_form;
@@ -568,6 +581,24 @@ bool tuned_lookup(int64_t M, int64_t d_model, int64_t d_ff, TunedShape* out) {
 int tuned_variant(int64_t M, int64_t d_model, int64_t d_ff) {
     TunedShape t;
     return tuned_lookup(M, d_model, d_ff, &t) ? t.variant : GMLP_VARIANT_AUTO;
+}
+
+// gmlp_autotune forces the forms of the SKINNY schedule while it measures them (t_skinny_forced: also "by the rule", 0 / 0)
+thread_local bool t_skinny_forced = false;
+thread_local int t_force_skinny_fused = 0, t_force_skinny_ring = 0;
+void skinny_forms(int64_t M, int64_t d_model, int64_t d_ff, int* fused, int* ring) {
+    *fused = 0;
+    *ring = 0;
+    if (t_skinny_forced) {
+        *fused = t_force_skinny_fused;
+        *ring = t_force_skinny_ring;
+        return;
+    }
+    TunedShape t;
+    if (tuned_lookup(M, d_model, d_ff, &t) && t.variant == GMLP_VARIANT_SKINNY) {
+        *fused = t.gu_nb;
+        *ring = t.down_form;
+    }
 }
 
 bool skinny_both_cluster(int64_t M, int64_t d_model, int64_t d_ff);
@@ -1233,9 +1264,12 @@ int launch_skinny_fused(DeviceState* dev, const FusedPlan& p, const bf16* X, con
 
 // Whether the SKINNY schedule runs this layer as one fused kernel: where the plan applies and was measured to pay.
 // Tuning override GMLP_SKINNY_FUSED: 0 never, 1 wherever the plan applies.
-bool skinny_use_fused(const FusedPlan& f) {
+bool skinny_use_fused(const FusedPlan& f, int64_t M, int64_t d_model, int64_t d_ff) {
     if (f.cluster < 1) return false;
     if (const char* e = getenv("GMLP_SKINNY_FUSED")) return atoi(e) != 0;
+    int tuned_fused = 0, tuned_ring = 0;
+    skinny_forms(M, d_model, d_ff, &tuned_fused, &tuned_ring);
+    if (tuned_fused != 0) return tuned_fused == 1;
     return f.preferred;
 }
 
@@ -1247,7 +1281,7 @@ int run_skinny(DeviceState* dev, const Layout& L, uint8_t* ws, const bf16* A, co
     unsigned int* c2 = c1 + L.s1.num_tiles;
     int rc = ensure_counters_zero(dev, c1, L.counters_bytes, st);
     if (rc != GMLP_OK) return rc;
-    if (skinny_use_fused(L.sf)) {
+    if (skinny_use_fused(L.sf, M, d_model, d_ff)) {
         rc = launch_skinny_fused(dev, L.sf, A, Wg, Wu, Wd, scratch, Y, M, d_model, d_ff, st, act);
         if (rc != GMLP_ERR_UNSUPPORTED) return rc;          // clusters that do not fit one wave: the two-kernel forms below
     }
@@ -2036,6 +2070,64 @@ int autotune_impl(const gmlp_args* a, int iters, int32_t* best_variant, float* b
             else if (s2 != 0) rc = GMLP_ERR_TIMEOUT;
         }
         if (rc != GMLP_OK) { (void)0; }
+    }
+    // The same for a SKINNY winner: the one-kernel form against the two-kernel forms where its plan applies, and half-size
+    // against full-size weight rings (up to 32 tokens), each against what the built-in rule takes.
+    if (w.variant == GMLP_VARIANT_SKINNY && rc == GMLP_OK) {
+        struct Form { int fused, ring; };
+        Form forms[4] = {{0, 0}, {0, 0}, {0, 0}, {0, 0}};
+        int n_forms = 1;
+        const FusedPlan fp = make_fused_plan(a->M, a->d_model, a->d_ff, dev->sm_count);
+        if (fp.cluster >= 1) forms[n_forms++] = {fp.preferred ? 2 : 1, 0};
+        if (a->M <= 32) { forms[n_forms++] = {0, 1}; forms[n_forms++] = {0, 2}; }
+        float form_ms[4] = {0, 0, 0, 0};
+        bool form_fits[4] = {true, true, true, true};
+        t_skinny_forced = true;
+        for (int c = 0; c < n_forms; ++c) {
+            t_force_skinny_fused = forms[c].fused;
+            t_force_skinny_ring = forms[c].ring;
+            form_fits[c] = a->workspace == nullptr ||
+                           make_layout(a->M, a->d_model, a->d_ff, a->flags, GMLP_VARIANT_SKINNY, dev->sm_count).total <= a->workspace_bytes;
+        }
+        for (int round = 0; round <= kRounds && rc == GMLP_OK && n_forms > 1; ++round)
+            for (int c = 0; c < n_forms && rc == GMLP_OK; ++c) {
+                if (!form_fits[c]) continue;
+                gmlp_args t = *a;
+                t.variant = GMLP_VARIANT_SKINNY;
+                t.flags &= ~(uint32_t)GMLP_FLAG_CHECKED;
+                t_force_skinny_fused = forms[c].fused;
+                t_force_skinny_ring = forms[c].ring;
+                rc = forward_impl(&t);
+                float ms = 0.0f;
+                if (rc == GMLP_OK && cudaEventRecord(e0, st) != cudaSuccess) rc = GMLP_ERR_LAUNCH;
+                for (int i = 0; i < per_round && rc == GMLP_OK; ++i) rc = forward_impl(&t);
+                if (rc != GMLP_OK) break;
+                if (cudaEventRecord(e1, st) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess ||
+                    cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) { rc = GMLP_ERR_LAUNCH; break; }
+                if (round > 0) form_ms[c] += ms;
+            }
+        t_skinny_forced = false;
+        t_force_skinny_fused = t_force_skinny_ring = 0;
+        if (rc == GMLP_OK) {
+            const int s3 = read_device_status();
+            if (s3 < 0) rc = s3;
+            else if (s3 != 0) rc = GMLP_ERR_TIMEOUT;
+        }
+        if (rc == GMLP_OK && n_forms > 1 && form_fits[0]) {
+            int bf = 0;
+            for (int c = 1; c < n_forms; ++c)
+                if (form_fits[c] && form_ms[c] < form_ms[bf]) bf = c;
+            // the rule's own choice is kept unless another form is measurably (1 %) faster
+            if (form_ms[bf] < 0.99f * form_ms[0]) { best_gu_nb = forms[bf].fused; best_down_form = forms[bf].ring; }
+            if (getenv("GMLP_TUNE_VERBOSE")) {
+                fprintf(stderr, "gmlp_autotune   small-M forms (one-kernel form 0 rule / 1 on / 2 off, rings 0 rule / 1 half / 2 full):");
+                for (int c = 0; c < n_forms; ++c)
+                    if (form_fits[c])
+                        fprintf(stderr, " [%d %d: %.1f us]%s", forms[c].fused, forms[c].ring, form_ms[c] * 1000.0f / (float)timed_calls,
+                                (forms[c].fused == best_gu_nb && forms[c].ring == best_down_form) ? "*" : "");
+                fprintf(stderr, "\n");
+            }
+        }
     }
     (void)cudaEventDestroy(e0);
     (void)cudaEventDestroy(e1);
