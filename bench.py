@@ -61,6 +61,11 @@ NCU_TRAFFIC_BYTES = {
     ("llama3-8b-prefill-M2048-rmsnorm", "gate_up"): 256.8e6 + 52.6e6,
     ("llama3-70b-prefill-M4096-outliers", "gate_up"): 3966.1e6 + 233.4e6,     # captured at full size (row tiles in groups of eight)
     ("llama3-8b-batch-M64", "gate_up"): 235.5e6 + 3.1e6,
+    # the small-M schedule's one-kernel form: the weights, read once (the partial Y stay in L2 for the kernel that adds them)
+    ("ragged-M7-plain", "fused"): 69.31e6 + 0.47e6,
+    ("ragged-M7-norm", "fused"): 69.31e6 + 0.47e6,
+    ("ragged-M1-plain", "fused"): 69.28e6 + 0.42e6,
+    ("ragged-M1-norm", "fused"): 69.28e6 + 0.42e6,
 }
 
 
