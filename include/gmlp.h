@@ -34,6 +34,16 @@
  * anything else writes to that memory between two calls (the buffer was freed and handed out again by an
  * allocator, reused as scratch, ...), tell the library with gmlp_workspace_forget() before the next call.
  *
+ * Stream order: X, the outputs and the workspace are used in stream order, like any kernel's operands.  The WEIGHTS
+ * (Wg, Wu, Wd) may be read EARLIER: the kernels of a call are chained by programmatic dependent launch, and the
+ * small-M kernels fetch their first weight tiles before they wait for the work that precedes the call on the stream
+ * (that is where their speed comes from: a call's start overlaps its predecessor's tail).  Weights that are complete
+ * when the call is made - the normal case - need nothing.  If a kernel enqueued shortly before the call on the SAME
+ * stream produces them (dequantisation on the fly, an optimiser step), pass GMLP_FLAG_WEIGHTS_IN_STREAM_ORDER: the
+ * call's first kernel is then launched in plain stream order, nothing of the call starts before that work is
+ * complete, and the call loses the overlap with its predecessor (a few microseconds).  gmlp_forward_static has no
+ * flags: its weights must be complete before it is called.
+ *
  * Errors: every entry point returns a gmlp_status code; nothing throws, aborts or prints.
  * Calls are asynchronous on the given stream: device-side problems (a bounded wait that
  * ran out) surface after the stream is synchronised, through gmlp_device_status(), or at
@@ -90,7 +100,10 @@ enum {
      * accumulator without the final rounding (rounding it to bf16 gives the default output bit for bit).
      * gmlp_forward_ex / gmlp_forward_host with the tensor-core schedules only (SIMT / STREAM:
      * GMLP_ERR_UNSUPPORTED); gmlp_gate_up rejects it (GMLP_ERR_FLAGS). */
-    GMLP_FLAG_Y_FP32 = 1u << 8
+    GMLP_FLAG_Y_FP32 = 1u << 8,
+    /* The weights (or the gain) may still be written by work enqueued earlier on the same stream: see "Stream order"
+     * above.  gmlp_forward_ex, gmlp_forward_host and gmlp_gate_up. */
+    GMLP_FLAG_WEIGHTS_IN_STREAM_ORDER = 1u << 10
 };
 
 /* Kernel schedule.  AUTO picks by shape; the others force one schedule (tests, benchmarks). */

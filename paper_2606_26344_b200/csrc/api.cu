@@ -34,7 +34,7 @@ constexpr int kVersion = 100;
 constexpr int kMaxDevices = 64;
 constexpr int64_t kMaxDim = (int64_t)1 << 30;      // per-dimension limit (TMA coordinates are int32)
 constexpr uint32_t kKnownFlags = GMLP_FLAG_RMSNORM | GMLP_FLAG_CHECKED | GMLP_FLAG_ACT_SWISH | GMLP_FLAG_ACT_GLU |
-                                 GMLP_FLAG_ACT_GELU | GMLP_FLAG_WEIGHTS_OUT_IN | GMLP_FLAG_Y_FP32;
+                                 GMLP_FLAG_ACT_GELU | GMLP_FLAG_WEIGHTS_OUT_IN | GMLP_FLAG_Y_FP32 | GMLP_FLAG_WEIGHTS_IN_STREAM_ORDER;
 constexpr gmlp::GateAct kSilu = {1.0f, 0};
 // weights of the call in flight are stored [out, in] (set by the entry points around their launches)
 thread_local bool t_w_out_in = false;
@@ -50,6 +50,21 @@ struct WeightLayoutScope {                       // sets the switch for one call
     explicit WeightLayoutScope(bool out_in) : prev(t_w_out_in) { t_w_out_in = out_in; }
     ~WeightLayoutScope() { t_w_out_in = prev; }
 };
+// GMLP_FLAG_WEIGHTS_IN_STREAM_ORDER: the FIRST kernel of the call in flight is launched without programmatic stream
+// serialization, so it starts only when everything enqueued before the call is complete; the call's later kernels
+// cannot start before all CTAs of the first one are running, so nothing of the call - in particular none of the weight
+// tiles that the small-M kernels fetch ahead of their griddepcontrol.wait - is read earlier than stream order allows.
+thread_local bool t_first_launch_ordered = false;
+struct StreamOrderScope {
+    bool prev;
+    explicit StreamOrderScope(bool ordered) : prev(t_first_launch_ordered) { t_first_launch_ordered = ordered; }
+    ~StreamOrderScope() { t_first_launch_ordered = prev; }
+};
+inline int pdl_allowed() {                       // value of programmaticStreamSerializationAllowed for the next launch
+    if (!t_first_launch_ordered) return 1;
+    t_first_launch_ordered = false;
+    return 0;
+}
 // tensor map of a weight matrix with `n` output columns and `k` input rows, 64 x 64 boxes either way
 #define GMLP_ENCODE_W(map, ptr, n, k) \
     (t_w_out_in ? encode_2d(map, ptr, (uint64_t)(k), (uint64_t)(n), 64, 64) : encode_2d(map, ptr, (uint64_t)(n), (uint64_t)(k), 64, 64))
@@ -819,7 +834,7 @@ int launch_rmsnorm(const bf16* X, const bf16* gain, bf16* Xn, int64_t M, int64_t
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const int dm = (int)d_model;
@@ -944,7 +959,7 @@ int launch_umma_pair(DeviceState* dev, const bf16* A, const bf16* W0, const bf16
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
@@ -1000,7 +1015,7 @@ int launch_umma_splitk(DeviceState* dev, int S, const CUtensorMap& tmA, const CU
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
@@ -1068,7 +1083,7 @@ int launch_umma(DeviceState* dev, const bf16* A, const bf16* W0, const bf16* W1,
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const int Mi = (int)M, Ki = (int)K, Ni = (int)N;
@@ -1114,7 +1129,7 @@ int launch_skinny_cluster(DeviceState* dev, const SkinnyPlan& p, const CUtensorM
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     int& capacity = dev->cluster_capacity[GATEUP ? 0 : 1][p.cluster];
@@ -1180,7 +1195,7 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const int Mi = (int)M, Ni = (int)N;
@@ -1223,7 +1238,7 @@ int launch_skinny_fused(DeviceState* dev, const FusedPlan& p, const bf16* X, con
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     int& capacity = dev->fused_capacity[p.cluster];
@@ -1331,6 +1346,7 @@ int forward_impl(const gmlp_args* a) {
     if ((w_out_in || y_fp32) && (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM)) return GMLP_ERR_UNSUPPORTED;
     const WeightLayoutScope layout_scope(w_out_in);
     const OutputTypeScope output_scope(y_fp32);
+    const StreamOrderScope order_scope((a->flags & GMLP_FLAG_WEIGHTS_IN_STREAM_ORDER) != 0);
     const Layout L = make_layout(a->M, a->d_model, a->d_ff, a->flags, variant, dev->sm_count);
 
     uint8_t* ws = static_cast<uint8_t*>(a->workspace);
@@ -1508,6 +1524,7 @@ int gate_up_impl(const gmlp_args* a) {
     if (variant == GMLP_VARIANT_SIMT || variant == GMLP_VARIANT_STREAM) return GMLP_ERR_UNSUPPORTED;
     if (a->flags & GMLP_FLAG_Y_FP32) return GMLP_ERR_FLAGS;          // H is the bf16 operand of the next GEMM
     const WeightLayoutScope layout_scope((a->flags & GMLP_FLAG_WEIGHTS_OUT_IN) != 0);
+    const StreamOrderScope order_scope((a->flags & GMLP_FLAG_WEIGHTS_IN_STREAM_ORDER) != 0);
     DeviceState* dev = current_device(&rc);
     if (dev == nullptr) return rc;
     if (variant == GMLP_VARIANT_SKINNY && !skinny_can_run(a->M, a->d_model, a->d_ff, dev->sm_count)) return GMLP_ERR_UNSUPPORTED;
@@ -1641,7 +1658,7 @@ int rmsnorm_matmul_impl(const gmlp_rmsmm_args* a) {
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
         attr[1].id = cudaLaunchAttributeClusterDimension;
         attr[1].val.clusterDim.x = 2;
         attr[1].val.clusterDim.y = 1;
@@ -1737,7 +1754,7 @@ int matmul_add_rmsnorm_impl(const gmlp_mmaddnorm_args* a) {
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
         attr[1].id = cudaLaunchAttributeClusterDimension;
         attr[1].val.clusterDim.x = 2;
         attr[1].val.clusterDim.y = 1;
@@ -1847,7 +1864,7 @@ int qkv_proj_impl(const gmlp_qkv_args* a) {
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
         attr[1].id = cudaLaunchAttributeClusterDimension;
         attr[1].val.clusterDim.x = 2;
         attr[1].val.clusterDim.y = 1;
@@ -1910,7 +1927,7 @@ int gqa_attention_impl(const gmlp_gqa_args* a) {
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const int Mi = (int)a->M, Si = (int)a->S, Hq = (int)a->n_q_heads, group = (int)(a->n_q_heads / a->n_kv_heads);
@@ -2215,7 +2232,7 @@ int gmlp_sum_partials(const void* const* partials, int32_t n_partials, void* Y, 
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (cudaLaunchKernelEx(&cfg, gmlp::sum_partials_bf16_kernel, list, static_cast<bf16*>(Y), nvec4) != cudaSuccess)

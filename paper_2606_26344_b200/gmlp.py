@@ -25,6 +25,7 @@ FLAG_ACT_GLU = 1 << 6
 FLAG_WEIGHTS_OUT_IN = 1 << 7
 FLAG_Y_FP32 = 1 << 8
 FLAG_ACT_GELU = 1 << 9
+FLAG_WEIGHTS_IN_STREAM_ORDER = 1 << 10
 ACT_FLAGS = {"silu": 0, "swish": FLAG_ACT_SWISH, "glu": FLAG_ACT_GLU, "gelu": FLAG_ACT_GELU}
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_STREAM, VARIANT_UMMA, VARIANT_SKINNY, VARIANT_PAIR, VARIANT_TENSOR = 0, 1, 2, 3, 4, 5, 6
 
@@ -249,7 +250,8 @@ def _check_bf16_cuda(t: torch.Tensor, name: str) -> None:
 
 def make_args(X, Wg, Wu, Wd, Y, gamma=None, eps: float = 1e-5, rmsnorm: bool = False, variant: int = VARIANT_AUTO,
               workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
-              checked: bool = False, act: str = "silu", beta: float = 1.0, weights_out_in: bool = False) -> GmlpArgs:
+              checked: bool = False, act: str = "silu", beta: float = 1.0, weights_out_in: bool = False,
+              weights_in_stream_order: bool = False) -> GmlpArgs:
     for t, n in ((X, "X"), (Wg, "Wg"), (Wu, "Wu"), (Wd, "Wd")):
         _check_bf16_cuda(t, n)
     y_fp32 = Y.dtype == torch.float32              # a float32 Y asks for the unrounded down projection
@@ -261,7 +263,8 @@ def make_args(X, Wg, Wu, Wd, Y, gamma=None, eps: float = 1e-5, rmsnorm: bool = F
     if Wg.shape != w_up or Wu.shape != w_up or Wd.shape != w_down or Y.shape != X.shape:
         raise ValueError("shape mismatch")
     flags = (FLAG_RMSNORM if rmsnorm else 0) | (FLAG_CHECKED if checked else 0) | ACT_FLAGS[act] | \
-        (FLAG_WEIGHTS_OUT_IN if weights_out_in else 0) | (FLAG_Y_FP32 if y_fp32 else 0)
+        (FLAG_WEIGHTS_OUT_IN if weights_out_in else 0) | (FLAG_Y_FP32 if y_fp32 else 0) | \
+        (FLAG_WEIGHTS_IN_STREAM_ORDER if weights_in_stream_order else 0)
     if gamma is not None:
         _check_bf16_cuda(gamma, "gamma")
     st = stream if stream is not None else torch.cuda.current_stream(X.device)
@@ -300,16 +303,19 @@ def forward_ex(args: GmlpArgs) -> None:
 
 def forward(X, Wg, Wu, Wd, Y=None, gamma=None, eps: float = 1e-5, rmsnorm: bool = False,
             variant: int = VARIANT_AUTO, workspace=None, stream=None, checked: bool = False,
-            act: str = "silu", beta: float = 1.0, weights_out_in: bool = False) -> torch.Tensor:
+            act: str = "silu", beta: float = 1.0, weights_out_in: bool = False,
+            weights_in_stream_order: bool = False) -> torch.Tensor:
     """Y = (act(Xn Wg) * (Xn Wu)) Wd on the GPU; asynchronous on ``stream`` (default: torch's current stream).
 
     ``act``: "silu" (the paper's operator), "swish" (g * sigmoid(beta * g)) or "glu" (sigmoid(g)).
-    ``weights_out_in``: the weights are stored [out, in] (Wg, Wu [d_ff, d_model], Wd [d_model, d_ff])."""
+    ``weights_out_in``: the weights are stored [out, in] (Wg, Wu [d_ff, d_model], Wd [d_model, d_ff]).
+    ``weights_in_stream_order``: the weights are produced by work enqueued just before on the same stream (the call
+    otherwise may fetch weight tiles while that work is still running)."""
     if Y is None:
         Y = torch.empty_like(X)
     with torch.cuda.device(X.device):
         forward_ex(make_args(X, Wg, Wu, Wd, Y, gamma, eps, rmsnorm, variant, workspace, stream, checked, act, beta,
-                             weights_out_in))
+                             weights_out_in, weights_in_stream_order))
     return Y
 
 

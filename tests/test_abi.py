@@ -60,7 +60,7 @@ def test_argument_validation_happens_before_device_work(lib):
     f = lambda a: lib.gmlp_forward_ex(ctypes.byref(a))
     assert lib.gmlp_forward_ex(None) == gmlp.ERR_NULL
     assert f(_args(struct_bytes=8)) == gmlp.ERR_FLAGS
-    assert f(_args(flags=1 << 10)) == gmlp.ERR_FLAGS
+    assert f(_args(flags=1 << 11)) == gmlp.ERR_FLAGS
     assert f(_args(variant=17)) == gmlp.ERR_FLAGS
     assert f(_args(flags=gmlp.FLAG_ACT_SWISH | gmlp.FLAG_ACT_GLU, act_beta=1.0)) == gmlp.ERR_FLAGS
     assert f(_args(flags=gmlp.FLAG_ACT_GELU | gmlp.FLAG_ACT_GLU, act_beta=1.0)) == gmlp.ERR_FLAGS
