@@ -34,15 +34,17 @@
  * anything else writes to that memory between two calls (the buffer was freed and handed out again by an
  * allocator, reused as scratch, ...), tell the library with gmlp_workspace_forget() before the next call.
  *
- * Stream order: X, the outputs and the workspace are used in stream order, like any kernel's operands.  The WEIGHTS
- * (Wg, Wu, Wd) may be read EARLIER: the kernels of a call are chained by programmatic dependent launch, and the
- * small-M kernels fetch their first weight tiles before they wait for the work that precedes the call on the stream
- * (that is where their speed comes from: a call's start overlaps its predecessor's tail).  Weights that are complete
+ * Stream order: X, the outputs and the workspace are used in stream order, like any kernel's operands.  The WEIGHT
+ * MATRICES (Wg, Wu, Wd here; W, Wq, Wk, Wv of the other operators below) may be read EARLIER: the kernels of a call are
+ * chained by programmatic dependent launch, and the GEMM kernels request their first weight tiles before they wait for
+ * the work that precedes the call on the stream (a call's start overlaps its predecessor's tail; for a few tokens that
+ * is a tenth of the step).  Weights that are complete
  * when the call is made - the normal case - need nothing.  If a kernel enqueued shortly before the call on the SAME
  * stream produces them (dequantisation on the fly, an optimiser step), pass GMLP_FLAG_WEIGHTS_IN_STREAM_ORDER: the
  * call's first kernel is then launched in plain stream order, nothing of the call starts before that work is
- * complete, and the call loses the overlap with its predecessor (a few microseconds).  gmlp_forward_static has no
- * flags: its weights must be complete before it is called.
+ * complete, and the call loses the overlap with its predecessor (a few microseconds).  gmlp_forward_static and the
+ * other operators have no such flag: their weights must be complete before the call is made (or be produced on another
+ * stream and handed over with an event, which orders everything).
  *
  * Errors: every entry point returns a gmlp_status code; nothing throws, aborts or prints.
  * Calls are asynchronous on the given stream: device-side problems (a bounded wait that

@@ -197,40 +197,60 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // (warp-uniform like the MMA issuer: coordinates and addresses by all lanes, the copies by the elected one)
         {
             const bool leader = ptx::elect_one();
-            if (!ROWSCALE) ptx::grid_dependency_wait();           // A (Xn or H) may come from the previous kernel
-            uint32_t s = 0, ph = 0;                                // ring position of the next k-block (stepped, not divided)
-            bool ok = true;
             // the A box holds a_box_rows rows of 128 B (fewer than 128 only when the whole problem has fewer rows:
             // the rest of the 128-row operand tile is never written and feeds accumulator rows nobody stores)
             const uint32_t a_tx_bytes = (uint32_t)a_box_rows * 128u;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % num_m_tiles) * kUmmaBM;
-                int n0 = (tile / num_m_tiles) * BN_OUT;
-                const CUtensorMap* plain_map = &tmB0;
+            auto tile_operands = [&](int tile, int& m0, int& n0, const CUtensorMap*& plain_map) {
+                m0 = (tile % num_m_tiles) * kUmmaBM;
+                n0 = (tile / num_m_tiles) * BN_OUT;
+                plain_map = &tmB0;
                 if (MULTI) {
                     int local;
                     const int seg = multi_segment(multi, tile / num_m_tiles, &local);
                     n0 = local * BN_OUT;
                     plain_map = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &multi.tmB2);
                 }
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!__all_sync(0xFFFFFFFFu, wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1))) { ok = false; break; }
-                    const uint32_t full = full0 + 8 * s;
-                    const uint32_t a_dst = base + s * kStageBytes;
-                    const uint32_t b_dst = a_dst + kUmmaABytes;
-                    if (leader) {
-                        ptx::mbar_arrive_expect_tx(full, a_tx_bytes + NB * kUmmaBoxBBytes);
-                        ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
+            };
+            auto load_weights = [&](int kb, uint32_t stage, int n0, const CUtensorMap* plain_map) {   // arms the barrier for the whole stage
+                const uint32_t full = full0 + 8 * stage;
+                const uint32_t b_dst = base + stage * kStageBytes + kUmmaABytes;
+                if (!leader) return;
+                ptx::mbar_arrive_expect_tx(full, a_tx_bytes + NB * kUmmaBoxBBytes);
 #pragma unroll
-                        for (int i = 0; i < NB; ++i) {
-                            // gate/up: the first NB/2 boxes are gate columns, the rest the same columns of up
-                            const CUtensorMap* map = (GATEUP && i >= NB / 2) ? &tmB1 : plain_map;
-                            const int x = GATEUP ? n0 + (i % (NB / 2)) * 64 : n0 + i * 64;
-                            // [K, N] weights: box of 64 columns x 64 k; [N, K] weights: box of 64 k x 64 rows of N
-                            if (w_kmajor) ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, kb * kUmmaBK, x, full);
-                            else ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
-                        }
-                    }
+                for (int i = 0; i < NB; ++i) {
+                    // gate/up: the first NB/2 boxes are gate columns, the rest the same columns of up
+                    const CUtensorMap* map = (GATEUP && i >= NB / 2) ? &tmB1 : plain_map;
+                    const int x = GATEUP ? n0 + (i % (NB / 2)) * 64 : n0 + i * 64;
+                    // [K, N] weights: box of 64 columns x 64 k; [N, K] weights: box of 64 k x 64 rows of N
+                    if (w_kmajor) ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, kb * kUmmaBK, x, full);
+                    else ptx::tma_load_2d(b_dst + i * kUmmaBoxBBytes, map, x, kb * kUmmaBK, full);
+                }
+            };
+            // The weight tiles of the first ring-full of k-blocks of this CTA's first tile do not depend on the previous
+            // kernel: they are requested ahead of the wait (the caller's contract on when weights are read is in gmlp.h,
+            // "Stream order"); A (Xn or H) may come from the previous kernel
+            int head = 0;
+            if (!ROWSCALE) {
+                if ((int)blockIdx.x < num_tiles) {
+                    int m0, n0;
+                    const CUtensorMap* plain_map;
+                    tile_operands(blockIdx.x, m0, n0, plain_map);
+                    head = num_kb < kStages ? num_kb : kStages;
+                    for (int i = 0; i < head; ++i) load_weights(i, (uint32_t)i, n0, plain_map);
+                }
+                ptx::grid_dependency_wait();
+            }
+            uint32_t s = 0, ph = 0;                                // ring position of the next k-block (stepped, not divided)
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                int m0, n0;
+                const CUtensorMap* plain_map;
+                tile_operands(tile, m0, n0, plain_map);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    const bool ahead = tile == (int)blockIdx.x && kb < head;     // barrier armed, weights on their way
+                    if (!ahead && !__all_sync(0xFFFFFFFFu, wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1))) { ok = false; break; }
+                    if (!ahead) load_weights(kb, s, n0, plain_map);
+                    if (leader) ptx::tma_load_2d(base + s * kStageBytes, &tmA, kb * kUmmaBK, m0, full0 + 8 * s);
                     __syncwarp();
                     if (++s == (uint32_t)kStages) { s = 0; ph ^= 1u; }
                 }

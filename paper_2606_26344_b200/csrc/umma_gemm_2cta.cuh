@@ -191,40 +191,60 @@ umma_pair_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         // (warp-uniform like the MMA issuer: coordinates and addresses by all lanes, the copies by the elected one)
         {
             const bool leader = ptx::elect_one();
-            if (!ROWSCALE) ptx::grid_dependency_wait();
             const uint32_t leader_full0 = ptx::map_to_cta(full0, 0);
-            uint32_t s = 0, ph = 0;                              // ring position of the next k-block
-            bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+            auto tile_operands = [&](int tile, int& m0, int& bx, const CUtensorMap*& bmap) {
                 int mt, nt;
                 tile_coords(tile, mt, nt);
-                const int m0 = mt * 256 + (int)rank * 128;
+                m0 = mt * 256 + (int)rank * 128;
                 int n0 = nt * BN_OUT;
                 // this CTA's half of the B columns: gate/up -> gate (rank 0) or up (rank 1) columns n0..n0+127
-                const CUtensorMap* bmap = (GATEUP && rank == 1) ? &tmB1 : &tmB0;
+                bmap = (GATEUP && rank == 1) ? &tmB1 : &tmB0;
                 if (MULTI) {
                     int local;
                     const int seg = multi_segment(multi, nt, &local);
                     n0 = local * BN_OUT;
                     bmap = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &multi.tmB2);
                 }
-                const int bx = GATEUP ? n0 : n0 + (int)rank * 128;
+                bx = GATEUP ? n0 : n0 + (int)rank * 128;
+            };
+            auto load_weights = [&](int kb, uint32_t stage, int bx, const CUtensorMap* bmap) {   // arms the leader's barrier for this CTA's whole stage
+                const uint32_t full = leader_full0 + 8 * stage;
+                const uint32_t b_dst = base + stage * kPairStageBytes + kPairABytes;
+                if (!leader) return;
+                ptx::mbar_arrive_expect_tx_cluster(full, kPairStageBytes);
+                if (w_kmajor) {                    // [N, K] weights: boxes of 64 k x 64 rows of N
+                    ptx::tma_load_2d_pair(b_dst, bmap, kb * kUmmaBK, bx, full);
+                    ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, kb * kUmmaBK, bx + 64, full);
+                } else {                           // [K, N] weights: boxes of 64 columns x 64 k
+                    ptx::tma_load_2d_pair(b_dst, bmap, bx, kb * kUmmaBK, full);
+                    ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, bx + 64, kb * kUmmaBK, full);
+                }
+            };
+            // The weight tiles of the first ring-full of k-blocks of this pair's first tile do not depend on the previous
+            // kernel: they are requested ahead of the wait (the caller's contract on when weights are read is in gmlp.h,
+            // "Stream order")
+            int head = 0;
+            if (!ROWSCALE) {
+                if (pair < num_tiles) {
+                    int m0, bx;
+                    const CUtensorMap* bmap;
+                    tile_operands(pair, m0, bx, bmap);
+                    head = num_kb < kPairStages ? num_kb : kPairStages;
+                    for (int i = 0; i < head; ++i) load_weights(i, (uint32_t)i, bx, bmap);
+                }
+                ptx::grid_dependency_wait();
+            }
+            uint32_t s = 0, ph = 0;                              // ring position of the next k-block
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+                int m0, bx;
+                const CUtensorMap* bmap;
+                tile_operands(tile, m0, bx, bmap);
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!__all_sync(0xFFFFFFFFu, wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1))) { ok = false; break; }
-                    const uint32_t full = leader_full0 + 8 * s;
-                    const uint32_t a_dst = base + s * kPairStageBytes;
-                    const uint32_t b_dst = a_dst + kPairABytes;
-                    if (leader) {
-                        ptx::mbar_arrive_expect_tx_cluster(full, kPairStageBytes);
-                        ptx::tma_load_2d_pair(a_dst, &tmA, kb * kUmmaBK, m0, full);
-                        if (w_kmajor) {                    // [N, K] weights: boxes of 64 k x 64 rows of N
-                            ptx::tma_load_2d_pair(b_dst, bmap, kb * kUmmaBK, bx, full);
-                            ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, kb * kUmmaBK, bx + 64, full);
-                        } else {                           // [K, N] weights: boxes of 64 columns x 64 k
-                            ptx::tma_load_2d_pair(b_dst, bmap, bx, kb * kUmmaBK, full);
-                            ptx::tma_load_2d_pair(b_dst + kUmmaBoxBBytes, bmap, bx + 64, kb * kUmmaBK, full);
-                        }
-                    }
+                    const bool ahead = tile == pair && kb < head;       // barrier armed, weights on their way
+                    if (!ahead && !__all_sync(0xFFFFFFFFu, wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1))) { ok = false; break; }
+                    if (!ahead) load_weights(kb, s, bx, bmap);
+                    if (leader) ptx::tma_load_2d_pair(base + s * kPairStageBytes, &tmA, kb * kUmmaBK, m0, leader_full0 + 8 * s);
                     __syncwarp();
                     if (++s == (uint32_t)kPairStages) { s = 0; ph ^= 1u; }
                 }

@@ -91,24 +91,30 @@ umma_splitk_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (warp == 0) {
         {
             const bool leader = ptx::elect_one();
+            auto load_weights = [&](int kb, uint32_t stage) {      // arms the stage's barrier for the whole stage
+                const uint32_t full = full0 + 8 * stage;
+                const uint32_t b_dst = base + stage * kSplitStageBytes + kUmmaABytes;
+                if (!leader) return;
+                ptx::mbar_arrive_expect_tx(full, (uint32_t)a_box_rows * 128u + 2 * kUmmaBoxBBytes);
+                if (w_kmajor) {
+                    ptx::tma_load_2d(b_dst, &tmB, kb * kUmmaBK, n0, full);
+                    ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, kb * kUmmaBK, n0 + 64, full);
+                } else {
+                    ptx::tma_load_2d(b_dst, &tmB, n0, kb * kUmmaBK, full);
+                    ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, n0 + 64, kb * kUmmaBK, full);
+                }
+            };
+            // The weight tiles of the first ring-full of k-blocks do not depend on the previous kernel: they are requested
+            // ahead of the wait (the caller's contract on when weights are read is in gmlp.h, "Stream order")
+            const int head = kb1 - kb0 < kSplitStages ? kb1 - kb0 : kSplitStages;
+            for (int i = 0; i < head; ++i) load_weights(kb0 + i, (uint32_t)i);
             ptx::grid_dependency_wait();
             uint32_t s = 0, ph = 0;                                // ring position, stepped
             for (int kb = kb0; kb < kb1; ++kb) {
-                if (!__all_sync(0xFFFFFFFFu, wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1))) break;
-                const uint32_t full = full0 + 8 * s;
-                const uint32_t a_dst = base + s * kSplitStageBytes;
-                const uint32_t b_dst = a_dst + kUmmaABytes;
-                if (leader) {
-                    ptx::mbar_arrive_expect_tx(full, (uint32_t)a_box_rows * 128u + 2 * kUmmaBoxBBytes);
-                    ptx::tma_load_2d(a_dst, &tmA, kb * kUmmaBK, m0, full);
-                    if (w_kmajor) {
-                        ptx::tma_load_2d(b_dst, &tmB, kb * kUmmaBK, n0, full);
-                        ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, kb * kUmmaBK, n0 + 64, full);
-                    } else {
-                        ptx::tma_load_2d(b_dst, &tmB, n0, kb * kUmmaBK, full);
-                        ptx::tma_load_2d(b_dst + kUmmaBoxBBytes, &tmB, n0 + 64, kb * kUmmaBK, full);
-                    }
-                }
+                const bool ahead = kb - kb0 < head;                // this stage's barrier is armed and its weights are on their way
+                if (!ahead && !__all_sync(0xFFFFFFFFu, wait_bounded(empty0 + 8 * s, ph ^ 1u, abort_flag, KERNEL_ID, 1))) break;
+                if (!ahead) load_weights(kb, s);
+                if (leader) ptx::tma_load_2d(base + s * kSplitStageBytes, &tmA, kb * kUmmaBK, m0, full0 + 8 * s);
                 __syncwarp();
                 if (++s == (uint32_t)kSplitStages) { s = 0; ph ^= 1u; }
             }
