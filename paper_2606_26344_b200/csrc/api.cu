@@ -1217,6 +1217,7 @@ int launch_skinny(DeviceState* dev, const SkinnyPlan& p, const bf16* X, const bf
 // GMLP_ERR_UNSUPPORTED when the device cannot hold all clusters at once (the caller then runs the two-kernel forms).
 int launch_skinny_fused(DeviceState* dev, const FusedPlan& p, const bf16* X, const bf16* Wg, const bf16* Wu, const bf16* Wd,
                         float* scratch, bf16* Y, int64_t M, int64_t d_model, int64_t d_ff, cudaStream_t st, gmlp::GateAct act) {
+    if (p.Mpad != 16) return GMLP_ERR_UNSUPPORTED;          // the kernel's epilogue is written for one 16-token accumulator per matrix
     if (!dev->skinny_fused_attr_set) {
         if (cudaFuncSetAttribute(gmlp::skinny_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gmlp::kFusedSmemBudget) != cudaSuccess)
             return GMLP_ERR_LAUNCH;
