@@ -30,7 +30,7 @@ namespace {
 
 using gmlp::bf16;
 
-constexpr int kVersion = 100;
+constexpr int kVersion = 101;            // 101: one-kernel small-M form, tuned small-M forms in the tune file, GMLP_FLAG_WEIGHTS_IN_STREAM_ORDER
 constexpr int kMaxDevices = 64;
 constexpr int64_t kMaxDim = (int64_t)1 << 30;      // per-dimension limit (TMA coordinates are int32)
 constexpr uint32_t kKnownFlags = GMLP_FLAG_RMSNORM | GMLP_FLAG_CHECKED | GMLP_FLAG_ACT_SWISH | GMLP_FLAG_ACT_GLU |
