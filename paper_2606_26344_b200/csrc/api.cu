@@ -60,11 +60,9 @@ struct StreamOrderScope {
     explicit StreamOrderScope(bool ordered) : prev(t_first_launch_ordered) { t_first_launch_ordered = ordered; }
     ~StreamOrderScope() { t_first_launch_ordered = prev; }
 };
-inline int pdl_allowed() {                       // value of programmaticStreamSerializationAllowed for the next launch
-    if (!t_first_launch_ordered) return 1;
-    t_first_launch_ordered = false;
-    return 0;
-}
+// value of programmaticStreamSerializationAllowed for the next launch (GMLP_CHECK_LAUNCH, which follows every launch that
+// went through, ends the "first kernel" state: a launch that is only prepared and then not made does not)
+inline int pdl_allowed() { return t_first_launch_ordered ? 0 : 1; }
 // tensor map of a weight matrix with `n` output columns and `k` input rows, 64 x 64 boxes either way
 #define GMLP_ENCODE_W(map, ptr, n, k) \
     (t_w_out_in ? encode_2d(map, ptr, (uint64_t)(k), (uint64_t)(n), 64, 64) : encode_2d(map, ptr, (uint64_t)(n), (uint64_t)(k), 64, 64))
@@ -825,6 +823,7 @@ void forget_counters(DeviceState* dev) {
     do {                                                      \
         if (cudaPeekAtLastError() != cudaSuccess) return GMLP_ERR_LAUNCH; \
         ++t_launches;                                         \
+        t_first_launch_ordered = false;                       \
     } while (0)
 
 int launch_rmsnorm(const bf16* X, const bf16* gain, bf16* Xn, int64_t M, int64_t d_model, float eps, cudaStream_t st) {
